@@ -1,0 +1,237 @@
+/*
+ * qbp.h -- C ABI of libqbp: the 8-bit training hot path (Quantized
+ * Back-Propagation with Gradients Bifurcation, followed by Range
+ * Batch-Normalization) as hand-written CUDA kernels for sm_100a.
+ *
+ * Paper: "Scalable Methods for 8-bit Training of Neural Networks"
+ * (arXiv 1805.11046).  Each entry point cites the passage that defines the
+ * operation it performs.
+ *
+ * Conventions (all entry points)
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller.  Scalars
+ *     the GPU produces (scale, zero-point, range) stay on the device in a
+ *     qbp_qparams.  The library allocates no device memory and keeps no
+ *     state between calls; scratch comes from the caller's workspace `ws`
+ *     (device memory, 256-byte aligned) of at least qbp_*_workspace_bytes().
+ *   - `stream` is a cudaStream_t passed as void*; work is enqueued on it and
+ *     the call returns without synchronising the host.
+ *   - Layouts: matrices row-major and dense; activations NHWC; filters KRSC.
+ *     Code tensors (int8/uint8) that feed an integer product must start on a
+ *     16-byte boundary and have an innermost extent that is a multiple of 16.
+ *   - Return value: QBP_OK or a negative qbp_status.  Argument and shape
+ *     errors are found on the host before anything is launched; the reason
+ *     is kept per thread and returned by qbp_last_error().
+ *   - Stored codes are signed: stored = unsigned code - 2^(M-1), and the
+ *     stored zero-point is shifted the same way, so that (q - zero_point) is
+ *     the value every product works on.
+ */
+#ifndef QBP_H_
+#define QBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QBP_OK = 0,
+    QBP_ERR_INVALID_ARG = -1,       /* NULL/misaligned pointer, negative size, bad enum */
+    QBP_ERR_UNSUPPORTED_SHAPE = -2, /* shape outside what the kernels implement         */
+    QBP_ERR_OVERFLOW_K = -3,        /* reduction too long for the int32 accumulator     */
+    QBP_ERR_WORKSPACE = -4,         /* ws NULL or smaller than *_workspace_bytes()      */
+    QBP_ERR_CUDA = -5,              /* a CUDA call failed; message holds its text       */
+    QBP_ERR_TIMEOUT = -6            /* a bounded device-side wait gave up               */
+} qbp_status;
+
+/* Quantisation parameters of one tensor (or one channel), device resident.
+ * x ~= scale * (q - zero_point).  vmin/vmax are the clamping values used,
+ * after widening to contain 0 (Appendix B). */
+typedef struct {
+    float   scale;
+    int32_t zero_point;
+    float   vmin;
+    float   vmax;
+} qbp_qparams;
+
+/* Convolution geometry.  Input [N,H,W,C], filter [K,R,S,C], output [N,P,Q,K]
+ * with P = (H + 2*pad - R)/stride + 1 (Q likewise).  The integer products
+ * implement stride 1 with R = S = 2*pad + 1 ("same" convolution, R in {1,3}). */
+typedef struct {
+    int32_t N, H, W, C;
+    int32_t K, R, S;
+    int32_t stride, pad;
+} qbp_conv_desc;
+
+enum { QBP_PER_TENSOR = 0, QBP_PER_CHANNEL = 1 };
+enum { QBP_ROUND_NEAREST = 0, QBP_ROUND_STOCHASTIC = 1 };
+enum { QBP_CONV_FPROP = 0, QBP_CONV_DGRAD = 1 };
+
+/* Text of the last error raised on the calling thread ("" if none). */
+const char *qbp_last_error(void);
+
+/* ------------------------------------------------------------------------
+ * Range quantiser -- Section 4 "Quantization methods" and Appendix B:
+ *   scale = (vmax - vmin) / (2^M - 1), zero-point = round(-vmin / scale),
+ *   output = round(x / scale + zero-point), clamped to the M-bit codes;
+ * clamping values = the tensor's min and max, widened to contain 0.  Nearest
+ * rounding (ties to even) for weights and activations; stochastic rounding
+ * for gradients (Section 4: convergence needed it) -- up with probability
+ * frac, the draw being the top 24 bits of the Philox4x32-10 word of the
+ * element: key = seed, counter = (i/4 low, i/4 high, tensor_id, 0), word i%4,
+ * i = flat index.  All arithmetic is IEEE fp32 in a fixed order, so codes
+ * are reproducible bit for bit.
+ *
+ * x [rows x cols], cols innermost (the channel dimension).  granularity
+ * QBP_PER_CHANNEL keeps one qbp_qparams per column (qp_out has `cols`
+ * entries), else one.  range_in (nullable): take vmin/vmax from these
+ * qbp_qparams (same count as qp_out) instead of scanning x -- the range the
+ * preceding Range BN already knows (Section 4).  row_sums (nullable, [rows],
+ * per-tensor only): sum over the columns of each row's stored codes.
+ * col_sums (nullable, [cols], per-tensor only): sum over rows, int64.
+ * rows*cols == 0 is valid and launches nothing but the parameter kernel.
+ * ---------------------------------------------------------------------- */
+size_t qbp_quantize_workspace_bytes(int64_t rows, int64_t cols, int granularity);
+
+int qbp_quantize_s8(const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
+                    uint64_t seed, uint32_t tensor_id, const qbp_qparams *range_in,
+                    int8_t *q, qbp_qparams *qp_out, int32_t *row_sums, int64_t *col_sums,
+                    void *ws, size_t ws_bytes, void *stream);
+
+/* 16-bit variant.  Any of q (int16 codes), hi (signed high byte) and lo
+ * (unsigned low byte), q = 256*hi + lo, may be NULL, but not all three. */
+int qbp_quantize_s16(const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
+                     uint64_t seed, uint32_t tensor_id, const qbp_qparams *range_in,
+                     int16_t *q, int8_t *hi, uint8_t *lo, qbp_qparams *qp_out,
+                     void *ws, size_t ws_bytes, void *stream);
+
+/* Gradients Bifurcation (Sections 1 and 4, Section 6 "Putting it all
+ * together"): from one read of the fp32 gradient g, write its 8-bit copy
+ * (for the layer gradient) and its 16-bit copy as byte limbs (for the weight
+ * gradient); both per-tensor, both stochastically rounded, from the streams
+ * tensor_id8 and tensor_id16.  row_sums8 (nullable): as in qbp_quantize_s8. */
+int qbp_bifurcate(const float *g, int64_t rows, int64_t cols, uint64_t seed,
+                  uint32_t tensor_id8, uint32_t tensor_id16,
+                  int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8,
+                  int8_t *hi, uint8_t *lo, qbp_qparams *qp16,
+                  void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------
+ * 8-bit products -- Section 1 (the weighted sums y = W x are where the work
+ * is), Eq. (grad_layer) g_{l-1} = g_l W^T; int32 accumulation:
+ *   acc[m,n] = sum_k (A[m,k] - za)(B[k,n] - zb),  C[m,n] = (float)acc * (sa*sb).
+ * A is [M x K] (transA: stored [K x M]), B is [K x N] (transB: stored
+ * [N x K]).  qa/qb give the operands' scale and zero-point (device).  acc_out
+ * and C are each nullable, not both.  K*255*255 must fit int32 (K <= 33025),
+ * else QBP_ERR_OVERFLOW_K.  M, N, K multiples of 16.
+ * ---------------------------------------------------------------------- */
+size_t qbp_gemm_s8_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+int qbp_gemm_s8(int transA, int transB, int64_t M, int64_t N, int64_t K,
+                const int8_t *A, const qbp_qparams *qa,
+                const int8_t *B, const qbp_qparams *qb,
+                int32_t *acc_out, float *C,
+                void *ws, size_t ws_bytes, void *stream);
+
+/* The same products for a convolution, computed as an implicit GEMM over
+ * the filter taps (no im2col buffer).  QBP_CONV_FPROP: x [N,H,W,C] ->
+ * [N,P,Q,K].  QBP_CONV_DGRAD (Eq. grad_layer): g [N,P,Q,K] -> [N,H,W,C].
+ * Padding is real zero, i.e. contributes nothing to (q - zero_point). */
+size_t qbp_conv_s8_workspace_bytes(int mode, const qbp_conv_desc *d);
+
+int qbp_conv_s8_implicit(int mode, const qbp_conv_desc *d,
+                         const int8_t *in, const qbp_qparams *q_in,
+                         const int8_t *w, const qbp_qparams *q_w,
+                         int32_t *acc_out, float *out,
+                         void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Weight gradient -- Eq. (grad_weight) g_W = g_l I_{l-1}^T with the 16-bit
+ * copy of g_l and the 8-bit layer input (Sections 6 and 7):
+ *   d == NULL: acc[k,n]     = sum_m (x[m,k] - zx)(g16[m,n] - zg)     dW [K x N]
+ *   d != NULL: acc[k,r,s,c] = sum over (n,p,q) with the tap in bounds of
+ *              (g16[n,p,q,k] - zg)(x[n,p+r-pad,q+s-pad,c] - zx)      dW [K,R,S,C]
+ * g16 = 256*g_hi + g_lo.  Each limb runs on the int8 tensor cores with an
+ * int32 accumulator over at most 65536 reduction rows at a time (the low
+ * limb's bound is 128*255*rows <= 2^31-1, rows <= 65793); partial results
+ * are combined in int64, exactly.  acc_out (int64) and dW each nullable, not
+ * both; dW = (float)acc * (sx*sg).
+ * ---------------------------------------------------------------------- */
+size_t qbp_wgrad_s16_workspace_bytes(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K);
+
+int qbp_wgrad_s16(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
+                  const int8_t *x, const qbp_qparams *qx,
+                  const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16,
+                  int64_t *acc_out, float *dW,
+                  void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Range Batch-Normalization -- Section 3, Eq. (range):
+ *   xhat = (x - mu) / (C(n) * range(x - mu)),  C(n) = 1/sqrt(2 ln n),
+ *   range = max - min, per channel over the n rows; y = gamma*xhat + beta
+ *   (gamma/beta nullable: 1, 0), optionally followed by ReLU.  A channel of
+ *   zero range yields xhat = 0.  n >= 2.
+ * x, y [n x C], C innermost.  save_mean/min/max [C] are written for the
+ * backward pass.  out_range (nullable): the exact per-tensor min and max of
+ * y, which the next layer's quantiser can take as range_in (Section 4).
+ * ---------------------------------------------------------------------- */
+size_t qbp_rangebn_workspace_bytes(int64_t n, int64_t C);
+
+int qbp_rangebn_fwd(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta,
+                    int relu, float *y, float *save_mean, float *save_min, float *save_max,
+                    qbp_qparams *out_range, void *ws, size_t ws_bytes, void *stream);
+
+/* Backward -- Section 7: the derivative of max (min) is one at every
+ * coordinate attaining it and zero elsewhere; otherwise the chain rule:
+ *   dbeta = sum dy, dgamma = sum dy*xhat, s = 1/(C(n)(max-min)),
+ *   dx = s*(gamma*dy - gamma*dbeta/n - C(n)*gamma*dgamma*([x==max]-[x==min])).
+ * With relu, dy is first zeroed where the forward output was not positive. */
+int qbp_rangebn_bwd(const float *dy, const float *x, int64_t n, int64_t C,
+                    const float *gamma, const float *beta, int relu,
+                    const float *save_mean, const float *save_min, const float *save_max,
+                    float *dx, float *dgamma, float *dbeta,
+                    void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Whole layer -- Sections 4 and 6: forward = quantise x and w to 8 bits
+ * (nearest) -> 8-bit product -> Range BN (+ReLU); backward = Range BN
+ * backward -> bifurcate the gradient (8-bit and 16-bit copies, stochastic)
+ * -> layer gradient from the 8-bit copy and the forward's weight codes, and
+ * weight gradient from the 16-bit copy and the forward's input codes.
+ * Linear: conv.R == 0, x [batch x in_features], w [in_features x
+ * out_features] (y = x w).  Conv: x NHWC, w KRSC.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    qbp_conv_desc conv;          /* conv.R == 0 selects the linear layer   */
+    int64_t batch, in_features, out_features;   /* linear layer only       */
+    int32_t relu;
+    uint64_t seed;               /* Philox key of the stochastic rounding  */
+    uint32_t tensor_id8, tensor_id16;
+} qbp_layer_desc;
+
+/* Caller-owned buffers that carry the forward's results to the backward.
+ * Element counts: x_codes = |x|, w_codes = |w|, z = rows*channels (the fp32
+ * output of the product, input of Range BN), rows = batch or N*P*Q. */
+typedef struct {
+    int8_t *x_codes;  qbp_qparams *qx;
+    int8_t *w_codes;  qbp_qparams *qw;
+    float  *z;
+    float  *save_mean, *save_min, *save_max;
+} qbp_layer_ctx;
+
+size_t qbp_layer_workspace_bytes(const qbp_layer_desc *L);
+
+int qbp_layer_fwd(const qbp_layer_desc *L, const float *x, const float *w,
+                  const float *gamma, const float *beta, float *y, const qbp_layer_ctx *saved,
+                  void *ws, size_t ws_bytes, void *stream);
+
+int qbp_layer_bwd(const qbp_layer_desc *L, const qbp_layer_ctx *saved, const float *dy,
+                  const float *gamma, const float *beta,
+                  float *dx, float *dw, float *dgamma, float *dbeta,
+                  void *ws, size_t ws_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QBP_H_ */

@@ -1,0 +1,246 @@
+"""Thin Python binding over the C ABI of libqbp (include/qbp.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  Tensors are torch CUDA tensors used as device memory (their
+data_ptr() is what crosses the boundary); work is enqueued on torch's current
+stream.  There is no CPU fallback: importing this module without the built
+library raises, and every non-zero status raises QbpError with the library's
+message.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libqbp.so"
+
+QBP_PER_TENSOR, QBP_PER_CHANNEL = 0, 1
+QBP_ROUND_NEAREST, QBP_ROUND_STOCHASTIC = 0, 1
+QBP_CONV_FPROP, QBP_CONV_DGRAD = 0, 1
+QBP_ERR_TIMEOUT = -6
+
+EXPORTS = (
+    "qbp_last_error",
+    "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s16", "qbp_bifurcate",
+    "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8",
+    "qbp_conv_s8_workspace_bytes", "qbp_conv_s8_implicit",
+    "qbp_wgrad_s16_workspace_bytes", "qbp_wgrad_s16",
+    "qbp_rangebn_workspace_bytes", "qbp_rangebn_fwd", "qbp_rangebn_bwd",
+    "qbp_layer_workspace_bytes", "qbp_layer_fwd", "qbp_layer_bwd",
+)
+
+
+class QbpError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"libqbp status {status}: {message}")
+        self.status = status
+
+
+class ConvDesc(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("N", "H", "W", "C", "K", "R", "S", "stride", "pad")]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("conv", ConvDesc), ("batch", C.c_int64), ("in_features", C.c_int64),
+                ("out_features", C.c_int64), ("relu", C.c_int32), ("seed", C.c_uint64),
+                ("tensor_id8", C.c_uint32), ("tensor_id16", C.c_uint32)]
+
+
+class LayerCtx(C.Structure):
+    _fields_ = [("x_codes", C.c_void_p), ("qx", C.c_void_p), ("w_codes", C.c_void_p), ("qw", C.c_void_p),
+                ("z", C.c_void_p), ("save_mean", C.c_void_p), ("save_min", C.c_void_p), ("save_max", C.c_void_p)]
+
+
+def _load() -> C.CDLL:
+    if not _LIB_PATH.exists():
+        raise ImportError(f"{_LIB_PATH} is missing: build it with "
+                          f"`python -m paper_1805_11046_b200.build` (needs nvcc); there is no fallback path")
+    lib = C.CDLL(str(_LIB_PATH))
+    lib.qbp_last_error.restype = C.c_char_p
+    missing = [name for name in EXPORTS if not hasattr(lib, name)]
+    if missing:
+        raise ImportError(f"{_LIB_PATH} lacks {missing}: rebuild it with `python -m paper_1805_11046_b200.build`")
+    for name in EXPORTS:
+        if name.endswith("_workspace_bytes"):
+            getattr(lib, name).restype = C.c_size_t
+    lib.qbp_quantize_workspace_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int]
+    lib.qbp_gemm_s8_workspace_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int64]
+    lib.qbp_conv_s8_workspace_bytes.argtypes = [C.c_int, C.c_void_p]
+    lib.qbp_wgrad_s16_workspace_bytes.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64]
+    lib.qbp_rangebn_workspace_bytes.argtypes = [C.c_int64, C.c_int64]
+    lib.qbp_layer_workspace_bytes.argtypes = [C.c_void_p]
+    return lib
+
+
+lib = _load()
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        raise QbpError(status, lib.qbp_last_error().decode())
+
+
+def _ptr(t) -> C.c_void_p:
+    if t is None:
+        return C.c_void_p(0)
+    if isinstance(t, int):
+        return C.c_void_p(t)
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+_ws_cache: dict = {}
+
+
+def workspace(nbytes: int, device=None) -> torch.Tensor:
+    """A cached device scratch buffer of at least nbytes (grown on demand, 256-byte aligned by torch)."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    t = _ws_cache.get(dev)
+    if t is None or t.numel() < nbytes:
+        t = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=dev)
+        _ws_cache[dev] = t
+    return t
+
+
+def new_qparams(count: int = 1, device="cuda") -> torch.Tensor:
+    """Device storage for `count` qbp_qparams records: int32 [count, 4] = (scale bits, zero_point, vmin bits, vmax bits)."""
+    return torch.zeros((count, 4), dtype=torch.int32, device=device)
+
+
+def read_qparams(qp: torch.Tensor):
+    """Host copy of qbp_qparams records -> (scale, zero_point, vmin, vmax) numpy arrays."""
+    h = qp.detach().cpu()
+    f = h.view(torch.float32)
+    return f[:, 0].numpy().copy(), h[:, 1].numpy().copy(), f[:, 2].numpy().copy(), f[:, 3].numpy().copy()
+
+
+def range_qparams(vmin, vmax, device="cuda") -> torch.Tensor:
+    """qbp_qparams records carrying only clamping values (for range_in)."""
+    lo = torch.as_tensor(vmin, dtype=torch.float32).reshape(-1)
+    hi = torch.as_tensor(vmax, dtype=torch.float32).reshape(-1)
+    qp = torch.zeros((lo.numel(), 4), dtype=torch.float32)
+    qp[:, 2] = lo
+    qp[:, 3] = hi
+    return qp.view(torch.int32).to(device)
+
+
+def status_word(ws: torch.Tensor) -> int:
+    """The int32 at the start of a product's workspace: 0, or QBP_ERR_TIMEOUT if a device-side wait gave up."""
+    return int(ws[:4].view(torch.int32).item())
+
+
+# ------------------------------------------------------------------ quantiser
+def qbp_quantize_s8(x, granularity=QBP_PER_TENSOR, rounding=QBP_ROUND_NEAREST, seed=0, tensor_id=0,
+                    range_in=None, q=None, qp_out=None, row_sums=None, col_sums=None, ws=None):
+    cols = x.shape[-1]; rows = x.numel() // cols if cols else 0
+    if q is None: q = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+    if qp_out is None: qp_out = new_qparams(cols if granularity else 1, x.device)
+    if ws is None: ws = workspace(lib.qbp_quantize_workspace_bytes(rows, cols, granularity), x.device)
+    _check(lib.qbp_quantize_s8(_ptr(x), C.c_int64(rows), C.c_int64(cols), granularity, rounding,
+                               C.c_uint64(seed), C.c_uint32(tensor_id), _ptr(range_in), _ptr(q), _ptr(qp_out),
+                               _ptr(row_sums), _ptr(col_sums), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return q, qp_out
+
+
+def qbp_quantize_s16(x, granularity=QBP_PER_TENSOR, rounding=QBP_ROUND_NEAREST, seed=0, tensor_id=0,
+                     range_in=None, q=None, hi=None, lo=None, qp_out=None, want=("q", "hi", "lo"), ws=None):
+    cols = x.shape[-1]; rows = x.numel() // cols if cols else 0
+    if q is None and "q" in want: q = torch.empty(x.shape, dtype=torch.int16, device=x.device)
+    if hi is None and "hi" in want: hi = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+    if lo is None and "lo" in want: lo = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    if qp_out is None: qp_out = new_qparams(cols if granularity else 1, x.device)
+    if ws is None: ws = workspace(lib.qbp_quantize_workspace_bytes(rows, cols, granularity), x.device)
+    _check(lib.qbp_quantize_s16(_ptr(x), C.c_int64(rows), C.c_int64(cols), granularity, rounding,
+                                C.c_uint64(seed), C.c_uint32(tensor_id), _ptr(range_in), _ptr(q), _ptr(hi), _ptr(lo),
+                                _ptr(qp_out), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return q, hi, lo, qp_out
+
+
+def qbp_bifurcate(g, seed, tensor_id8, tensor_id16, q8=None, hi=None, lo=None, qp8=None, qp16=None,
+                  row_sums8=None, ws=None):
+    cols = g.shape[-1]; rows = g.numel() // cols if cols else 0
+    if q8 is None: q8 = torch.empty(g.shape, dtype=torch.int8, device=g.device)
+    if hi is None: hi = torch.empty(g.shape, dtype=torch.int8, device=g.device)
+    if lo is None: lo = torch.empty(g.shape, dtype=torch.uint8, device=g.device)
+    if qp8 is None: qp8 = new_qparams(1, g.device)
+    if qp16 is None: qp16 = new_qparams(1, g.device)
+    if ws is None: ws = workspace(lib.qbp_quantize_workspace_bytes(rows, cols, 0), g.device)
+    _check(lib.qbp_bifurcate(_ptr(g), C.c_int64(rows), C.c_int64(cols), C.c_uint64(seed), C.c_uint32(tensor_id8),
+                             C.c_uint32(tensor_id16), _ptr(q8), _ptr(qp8), _ptr(row_sums8), _ptr(hi), _ptr(lo),
+                             _ptr(qp16), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return q8, qp8, hi, lo, qp16
+
+
+# ------------------------------------------------------------------- products
+def qbp_gemm_s8(A, qa, B, qb, transA=False, transB=False, want_acc=False, want_out=True, acc_out=None, out=None, ws=None):
+    if transA: K, M = A.shape
+    else:      M, K = A.shape
+    N = B.shape[0] if transB else B.shape[1]
+    if want_acc and acc_out is None: acc_out = torch.empty((M, N), dtype=torch.int32, device=A.device)
+    if want_out and out is None: out = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    if ws is None: ws = workspace(lib.qbp_gemm_s8_workspace_bytes(M, N, K), A.device)
+    _check(lib.qbp_gemm_s8(int(transA), int(transB), C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A), _ptr(qa),
+                           _ptr(B), _ptr(qb), _ptr(acc_out), _ptr(out), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return acc_out, out, ws
+
+
+def conv_desc(N, H, W, C_in, K, R, S, stride=1, pad=0) -> ConvDesc:
+    return ConvDesc(N, H, W, C_in, K, R, S, stride, pad)
+
+
+def qbp_conv_s8_implicit(mode, d: ConvDesc, inp, q_in, w, q_w, want_acc=False, want_out=True, acc_out=None, out=None, ws=None):
+    shape = (d.N, d.H, d.W, d.K) if mode == QBP_CONV_FPROP else (d.N, d.H, d.W, d.C)
+    if want_acc and acc_out is None: acc_out = torch.empty(shape, dtype=torch.int32, device=inp.device)
+    if want_out and out is None: out = torch.empty(shape, dtype=torch.float32, device=inp.device)
+    if ws is None: ws = workspace(lib.qbp_conv_s8_workspace_bytes(mode, C.byref(d)), inp.device)
+    _check(lib.qbp_conv_s8_implicit(mode, C.byref(d), _ptr(inp), _ptr(q_in), _ptr(w), _ptr(q_w), _ptr(acc_out),
+                                    _ptr(out), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return acc_out, out, ws
+
+
+def qbp_wgrad_s16(x, qx, g_hi, g_lo, qg16, d: ConvDesc | None = None, want_acc=False, want_out=True,
+                  acc_out=None, dW=None, ws=None):
+    if d is None:
+        M, K = x.shape; N = g_hi.shape[1]; shape = (K, N)
+        dref = None
+    else:
+        M = d.N * d.H * d.W; K = d.C; N = d.K; shape = (d.K, d.R, d.S, d.C)
+        dref = C.byref(d)
+    if want_acc and acc_out is None: acc_out = torch.empty(shape, dtype=torch.int64, device=x.device)
+    if want_out and dW is None: dW = torch.empty(shape, dtype=torch.float32, device=x.device)
+    if ws is None: ws = workspace(lib.qbp_wgrad_s16_workspace_bytes(dref, M, N, K), x.device)
+    _check(lib.qbp_wgrad_s16(dref, C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(x), _ptr(qx), _ptr(g_hi),
+                             _ptr(g_lo), _ptr(qg16), _ptr(acc_out), _ptr(dW), _ptr(ws), C.c_size_t(ws.numel()),
+                             _stream()))
+    return acc_out, dW, ws
+
+
+# ------------------------------------------------------------------- Range BN
+def qbp_rangebn_fwd(x, gamma=None, beta=None, relu=False, y=None, want_range=False, ws=None):
+    Cc = x.shape[-1]; n = x.numel() // Cc
+    if y is None: y = torch.empty_like(x)
+    mean = torch.empty(Cc, dtype=torch.float32, device=x.device)
+    vmin = torch.empty_like(mean); vmax = torch.empty_like(mean)
+    out_range = new_qparams(1, x.device) if want_range else None
+    if ws is None: ws = workspace(lib.qbp_rangebn_workspace_bytes(n, Cc), x.device)
+    _check(lib.qbp_rangebn_fwd(_ptr(x), C.c_int64(n), C.c_int64(Cc), _ptr(gamma), _ptr(beta), int(relu), _ptr(y),
+                               _ptr(mean), _ptr(vmin), _ptr(vmax), _ptr(out_range), _ptr(ws), C.c_size_t(ws.numel()),
+                               _stream()))
+    return y, mean, vmin, vmax, out_range
+
+
+def qbp_rangebn_bwd(dy, x, mean, vmin, vmax, gamma=None, beta=None, relu=False, dx=None, ws=None):
+    Cc = x.shape[-1]; n = x.numel() // Cc
+    if dx is None: dx = torch.empty_like(x)
+    dgamma = torch.empty(Cc, dtype=torch.float32, device=x.device); dbeta = torch.empty_like(dgamma)
+    if ws is None: ws = workspace(lib.qbp_rangebn_workspace_bytes(n, Cc), x.device)
+    _check(lib.qbp_rangebn_bwd(_ptr(dy), _ptr(x), C.c_int64(n), C.c_int64(Cc), _ptr(gamma), _ptr(beta), int(relu),
+                               _ptr(mean), _ptr(vmin), _ptr(vmax), _ptr(dx), _ptr(dgamma), _ptr(dbeta), _ptr(ws),
+                               C.c_size_t(ws.numel()), _stream()))
+    return dx, dgamma, dbeta

@@ -1,0 +1,89 @@
+// Per-channel scans of a [rows x C] fp32 matrix with the channel innermost
+// (NHWC): the thread/row mapping shared by the per-channel range scan of the
+// quantiser and by both passes of Range BN.
+//
+// Mapping: the matrix is read as vectors of VEC floats (4 when C % 4 == 0 and
+// the base is 16-byte aligned, else 1).  A 256-thread block is TW vector
+// columns wide and 256/TW rows high; blockIdx.y selects the slab of TW vector
+// columns, blockIdx.x the strip of rows, strips advance by gridDim.x.  A
+// thread therefore stays on the same VEC channels for its whole life and a
+// warp always reads 32*VEC consecutive floats.
+#pragma once
+
+#include "qbp_common.cuh"
+
+namespace qbp {
+
+constexpr int kScanThreads = 256;
+constexpr int kScanUnroll = 4;
+constexpr int kScanMaxStrips = 1024;     // bound on gridDim.x, sizes the partial buffers
+
+struct ScanGeom {
+    int vec;        // 4 or 1
+    int cv;         // vector columns = C / vec
+    int tw;         // threads across = min(pow2ceil(cv), 256)
+    int rpb;        // rows per block step = 256 / tw
+    int slabs;      // ceil(cv / tw)
+    int nbx;        // row strips (gridDim.x)
+};
+
+inline int pow2ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+
+// nbx is chosen so that all strips are resident at once (8 blocks of 256
+// threads per SM) and no strip is empty.
+inline ScanGeom scan_geom(int64_t rows, int64_t C, bool aligned)
+{
+    ScanGeom g;
+    g.vec = (aligned && C % 4 == 0) ? 4 : 1;
+    g.cv = (int)(C / g.vec);
+    g.tw = pow2ceil(g.cv) < kScanThreads ? pow2ceil(g.cv) : kScanThreads;
+    g.rpb = kScanThreads / g.tw;
+    g.slabs = (g.cv + g.tw - 1) / g.tw;
+    int64_t steps = (rows + g.rpb - 1) / g.rpb;
+    int64_t want = (int64_t)sm_count() * 8 / g.slabs;
+    if (want < 1) want = 1;
+    if (want > kScanMaxStrips) want = kScanMaxStrips;
+    g.nbx = (int)(steps < want ? (steps > 0 ? steps : 1) : want);
+    return g;
+}
+
+#ifdef __CUDACC__
+
+template <int VEC> struct VecF;
+template <> struct VecF<4> {
+    float v[4];
+    __device__ __forceinline__ void load(const float *p) {
+        float4 t = __ldg(reinterpret_cast<const float4 *>(p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    __device__ __forceinline__ void store(float *p) const {
+        *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+};
+template <> struct VecF<1> {
+    float v[1];
+    __device__ __forceinline__ void load(const float *p) { v[0] = __ldg(p); }
+    __device__ __forceinline__ void store(float *p) const { *p = v[0]; }
+};
+
+// Calls f(row, first_channel, vec_index_in_unroll) for every vector this thread
+// owns; loads are expected to be grouped by the caller via the unroll index.
+struct ScanPos {
+    int tx, ty, col;      // col = first channel of this thread's vector
+    bool active;
+};
+
+template <int VEC>
+__device__ __forceinline__ ScanPos scan_pos(int C, int tw)
+{
+    ScanPos p;
+    p.tx = threadIdx.x % tw;
+    p.ty = threadIdx.x / tw;
+    int cv = blockIdx.y * tw + p.tx;
+    p.col = cv * VEC;
+    p.active = p.col < C;
+    return p;
+}
+
+#endif  // __CUDACC__
+}  // namespace qbp

@@ -1,0 +1,156 @@
+// Whole quantised layer (Sections 4 and 6): the composition of the library's
+// own entry points in the order the method prescribes.
+//   forward : quantise x, w to 8 bits (nearest) -> 8-bit product -> Range BN (+ReLU)
+//   backward: Range BN backward -> gradient bifurcation (8-bit and 16-bit copies,
+//             stochastic rounding) -> layer gradient from the 8-bit copy and the
+//             forward's weight codes; weight gradient from the 16-bit copy and
+//             the forward's input codes.
+// The straight-through estimator through the quantiser is the identity here:
+// the clamping values are the tensor's own min and max, so nothing is clipped.
+// Everything is enqueued on the caller's stream; temporaries live in the
+// caller's workspace.
+#include "qbp_mma.cuh"
+
+#include <algorithm>
+
+namespace qbp {
+
+struct LayerShape {
+    bool conv;
+    int64_t rows;        // batch, or N*H*W
+    int64_t cin, cout;   // reduced / produced channels of the forward product
+    int64_t x_elems, w_elems;
+};
+
+static int layer_shape(const qbp_layer_desc *L, LayerShape &s)
+{
+    if (!L) return fail(QBP_ERR_INVALID_ARG, "layer: descriptor is NULL");
+    s.conv = L->conv.R != 0;
+    if (s.conv) {
+        const qbp_conv_desc &d = L->conv;
+        if (d.N <= 0 || d.H <= 0 || d.W <= 0 || d.C <= 0 || d.K <= 0 || d.R <= 0 || d.S <= 0)
+            return fail(QBP_ERR_INVALID_ARG, "layer: bad convolution geometry");
+        s.rows = (int64_t)d.N * d.H * d.W; s.cin = d.C; s.cout = d.K;
+        s.x_elems = s.rows * d.C; s.w_elems = (int64_t)d.K * d.R * d.S * d.C;
+    } else {
+        if (L->batch <= 0 || L->in_features <= 0 || L->out_features <= 0)
+            return fail(QBP_ERR_INVALID_ARG, "layer: batch, in_features, out_features must be positive");
+        s.rows = L->batch; s.cin = L->in_features; s.cout = L->out_features;
+        s.x_elems = s.rows * s.cin; s.w_elems = s.cin * s.cout;
+    }
+    return QBP_OK;
+}
+
+// Scratch shared by the steps (they run one after another on the stream).
+static size_t step_scratch_bytes(const qbp_layer_desc *L, const LayerShape &s)
+{
+    size_t b = qbp_quantize_workspace_bytes(s.rows, std::max(s.cin, s.cout), QBP_PER_TENSOR);
+    b = std::max(b, qbp_rangebn_workspace_bytes(s.rows, s.cout));
+    if (s.conv) {
+        b = std::max(b, qbp_conv_s8_workspace_bytes(QBP_CONV_FPROP, &L->conv));
+        b = std::max(b, qbp_wgrad_s16_workspace_bytes(&L->conv, 0, 0, 0));
+    } else {
+        b = std::max(b, qbp_gemm_s8_workspace_bytes(s.rows, std::max(s.cin, s.cout), std::max(s.cin, s.cout)));
+        b = std::max(b, qbp_wgrad_s16_workspace_bytes(nullptr, s.rows, s.cout, s.cin));
+    }
+    return align_up(b, 256);
+}
+
+// Backward temporaries: fp32 gradient at the product's output, its three code
+// tensors, two parameter records.
+static size_t bwd_temp_bytes(const LayerShape &s)
+{
+    const size_t g = (size_t)s.rows * s.cout;
+    return align_up(g * sizeof(float), 256) + 3 * align_up(g, 256) + 2 * 256;
+}
+
+}  // namespace qbp
+
+using namespace qbp;
+
+extern "C" __attribute__((visibility("default"))) size_t qbp_layer_workspace_bytes(const qbp_layer_desc *L)
+{
+    LayerShape s;
+    if (layer_shape(L, s)) return 0;
+    return step_scratch_bytes(L, s) + bwd_temp_bytes(s);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_layer_desc *L, const float *x,
+                                                                   const float *w, const float *gamma,
+                                                                   const float *beta, float *y,
+                                                                   const qbp_layer_ctx *saved, void *ws,
+                                                                   size_t ws_bytes, void *stream)
+{
+    LayerShape s;
+    int rc = layer_shape(L, s);
+    if (rc) return rc;
+    if (!x || !w || !y || !saved) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: NULL argument");
+    if (!saved->x_codes || !saved->qx || !saved->w_codes || !saved->qw || !saved->z || !saved->save_mean ||
+        !saved->save_min || !saved->save_max)
+        return fail(QBP_ERR_INVALID_ARG, "layer_fwd: the saved-state record has a NULL buffer");
+    if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
+        return fail(QBP_ERR_WORKSPACE, "layer_fwd: workspace of %zu bytes needed, %zu given",
+                    qbp_layer_workspace_bytes(L), ws_bytes);
+    const size_t scratch = step_scratch_bytes(L, s);
+
+    // weights and activations: nearest rounding, clamping values = min and max (Appendix B)
+    rc = qbp_quantize_s8(x, s.rows, s.cin, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, saved->x_codes, saved->qx,
+                         nullptr, nullptr, ws, scratch, stream);
+    if (rc) return rc;
+    const int64_t w_rows = s.conv ? (int64_t)L->conv.K * L->conv.R * L->conv.S : s.cin;
+    rc = qbp_quantize_s8(w, w_rows, s.w_elems / w_rows, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr,
+                         saved->w_codes, saved->qw, nullptr, nullptr, ws, scratch, stream);
+    if (rc) return rc;
+    if (s.conv)
+        rc = qbp_conv_s8_implicit(QBP_CONV_FPROP, &L->conv, saved->x_codes, saved->qx, saved->w_codes, saved->qw,
+                                  nullptr, saved->z, ws, scratch, stream);
+    else
+        rc = qbp_gemm_s8(0, 0, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr,
+                         saved->z, ws, scratch, stream);
+    if (rc) return rc;
+    return qbp_rangebn_fwd(saved->z, s.rows, s.cout, gamma, beta, L->relu, y, saved->save_mean, saved->save_min,
+                           saved->save_max, nullptr, ws, scratch, stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_layer_desc *L, const qbp_layer_ctx *saved,
+                                                                   const float *dy, const float *gamma,
+                                                                   const float *beta, float *dx, float *dw,
+                                                                   float *dgamma, float *dbeta, void *ws,
+                                                                   size_t ws_bytes, void *stream)
+{
+    LayerShape s;
+    int rc = layer_shape(L, s);
+    if (rc) return rc;
+    if (!saved || !dy || !dx || !dw) return fail(QBP_ERR_INVALID_ARG, "layer_bwd: NULL argument");
+    if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
+        return fail(QBP_ERR_WORKSPACE, "layer_bwd: workspace of %zu bytes needed, %zu given",
+                    qbp_layer_workspace_bytes(L), ws_bytes);
+    const size_t scratch = step_scratch_bytes(L, s);
+    WsCarver c(static_cast<char *>(ws) + scratch, ws_bytes - scratch);
+    const size_t gcount = (size_t)s.rows * s.cout;
+    float *g = c.take<float>(gcount);
+    int8_t *g8 = c.take<int8_t>(gcount);
+    int8_t *ghi = c.take<int8_t>(gcount);
+    uint8_t *glo = c.take<uint8_t>(gcount);
+    qbp_qparams *qp8 = c.take<qbp_qparams>(1);
+    qbp_qparams *qp16 = c.take<qbp_qparams>(1);
+
+    rc = qbp_rangebn_bwd(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
+                         saved->save_max, g, dgamma, dbeta, ws, scratch, stream);
+    if (rc) return rc;
+    // two copies of the gradient: 8 bits for the layer gradient, 16 bits for the weight gradient
+    rc = qbp_bifurcate(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8, nullptr, ghi, glo, qp16, ws,
+                       scratch, stream);
+    if (rc) return rc;
+    if (s.conv) {
+        rc = qbp_conv_s8_implicit(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, ws, scratch,
+                                  stream);
+        if (rc) return rc;
+        return qbp_wgrad_s16(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, ws, scratch, stream);
+    }
+    // dx [batch x in] = g8 [batch x out] . w^T, w stored [in x out]
+    rc = qbp_gemm_s8(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, ws, scratch, stream);
+    if (rc) return rc;
+    return qbp_wgrad_s16(nullptr, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, ws,
+                         scratch, stream);
+}

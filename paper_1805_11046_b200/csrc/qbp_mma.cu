@@ -1,0 +1,604 @@
+// 8-bit integer products on the 5th-generation tensor cores:
+//   y = W x and g_{l-1} = g_l W^T (Section 1; Eq. (grad_layer)) for linear
+//   layers (GEMM) and for convolutions (implicit GEMM over the filter taps).
+//
+// One CTA produces one 128 x BN tile of the output.  Warp 0 drives TMA
+// (cp.async.bulk.tensor into 128B/64B/32B-swizzled shared-memory stages),
+// warp 1 issues tcgen05.mma kind::i8 with the int32 accumulator in tensor
+// memory, warps 2..5 read the accumulator back (tcgen05.ld), apply the
+// zero-point correction, dequantise and store.  Stages are handed over with
+// mbarriers; tcgen05.commit releases a stage when the MMAs that read it are
+// done.  Every wait is bounded; on expiry the CTA raises the status word at
+// the start of the workspace and leaves through the normal exit.
+//
+// The raw MMA sums stored codes; padding taps are zero-filled by TMA and so
+// contribute nothing to the raw sum.  The sum over (q_a - z_a)(q_b - z_b) is
+// recovered in the epilogue from code sums prepared by small helper kernels:
+//   acc = raw + rowterm[m] + colterm[class(m)][n]
+// where, for a convolution, class(m) says which taps of output pixel m fall
+// inside the image (real-zero padding contributes nothing).
+#include "qbp_mma.cuh"
+
+#include <algorithm>
+
+namespace qbp {
+
+// =============================================================== tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return (EncodeTiledFn)p;
+    }();
+    return fn;
+}
+
+static CUtensorMapSwizzle swizzle_for(uint32_t inner_bytes)
+{
+    return inner_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+         : inner_bytes == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
+                              : CU_TENSOR_MAP_SWIZZLE_32B;
+}
+
+int make_map_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    if (box_cols != 32 && box_cols != 64 && box_cols != 128) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "box of %u bytes", box_cols);
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_cols), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled(2d %llu x %llu, box %u x %u) failed: %d",
+                                       (unsigned long long)rows, (unsigned long long)cols, box_rows, box_cols, (int)r);
+    return QBP_OK;
+}
+
+int make_map_nhwc(CUtensorMap *map, const void *base, uint64_t N, uint64_t H, uint64_t W, uint64_t C, uint32_t bn,
+                  uint32_t bh, uint32_t bw, uint32_t box_c)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    if (box_c != 32 && box_c != 64 && box_c != 128) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "box of %u bytes", box_c);
+    cuuint64_t dims[4] = {C, W, H, N};
+    cuuint64_t strides[3] = {C, W * C, H * W * C};
+    cuuint32_t box[4] = {box_c, bw, bh, bn};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_c), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled(nhwc) failed: %d", (int)r);
+    return QBP_OK;
+}
+
+// ========================================================= operand descriptors
+// Shared-memory matrix descriptor (64 bit): start address >> 4 in bits 0..13,
+// leading byte offset >> 4 in 16..29, stride byte offset >> 4 in 32..45, the
+// constant 1 in 46..47, swizzle mode in 61..63 (2 = 128B, 4 = 64B, 6 = 32B).
+static uint32_t swizzle_code(uint32_t row_bytes) { return row_bytes == 128 ? 2u : row_bytes == 64 ? 4u : 6u; }
+
+OperandLayout layout_kmajor(uint32_t rows, uint32_t row_bytes)
+{
+    OperandLayout L;
+    L.tile_bytes = rows * row_bytes;
+    L.desc_lo = 1u << 16;                                    // leading offset: unused for swizzled K-major
+    L.desc_hi = ((8u * row_bytes) >> 4) | (1u << 14) | (swizzle_code(row_bytes) << 29);   // 8-row groups
+    L.kstep = 32u >> 4;                                      // next 32 reduction bytes inside the swizzled row
+    L.major = 0;
+    return L;
+}
+
+OperandLayout layout_mnmajor(uint32_t krows, uint32_t row_bytes, uint32_t chunks, uint32_t chunk_stride)
+{
+    OperandLayout L;
+    L.tile_bytes = chunks > 1 ? chunks * chunk_stride : krows * row_bytes;
+    L.desc_lo = ((chunks > 1 ? chunk_stride : krows * row_bytes) >> 4) << 16;   // between M/N chunks
+    L.desc_hi = ((8u * row_bytes) >> 4) | (1u << 14) | (swizzle_code(row_bytes) << 29);   // between 8-row K groups
+    L.kstep = (32u * row_bytes) >> 4;                        // next 32 reduction rows
+    L.major = 1;
+    return L;
+}
+
+// Instruction descriptor of tcgen05.mma kind::i8: accumulator type in bits 4..5
+// (2 = s32), A/B type in 7..9 / 10..12 (0 = u8, 1 = s8), A/B major in 15 / 16,
+// N >> 3 in 17..22, M >> 4 in 24..28.
+uint32_t make_idesc(bool a_signed, bool b_signed, uint32_t a_major, uint32_t b_major, uint32_t m, uint32_t n)
+{
+    return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | ((b_signed ? 1u : 0u) << 10) | (a_major << 15) | (b_major << 16) |
+           ((n >> 3) << 17) | ((m >> 4) << 24);
+}
+
+// ================================================================== the kernel
+enum { MODE_GEMM = 0, MODE_FPROP = 1, MODE_DGRAD = 2 };
+constexpr int kMaxStages = 10;
+constexpr int kMmaThreads = 192;
+
+struct MmaParams {
+    CUtensorMap mapA, mapB;
+    OperandLayout a, b;
+    uint32_t idesc;
+    int mode;
+    int stages, k_iters, mma_per_iter, bn, tmem_cols;
+    int tiles_n;
+    // output
+    int64_t M, N;                 // rows / columns of the output matrix
+    int32_t *acc_out; float *out;
+    const int32_t *rowterm;       // [M]
+    const int32_t *colterm;       // [classes][N]
+    const qbp_qparams *qa, *qb;
+    int *status;
+    // gemm: element offsets per k iteration handled via kblock
+    int kblock;                   // reduction elements per k iteration
+    // conv geometry (output pixel grid == input pixel grid: stride 1, same padding)
+    int H, W, Nimg, pad, S, cchunks, chunk_bytes, Cred;
+    int bw_log2, bh_log2, tiles_w, tiles_h;
+};
+
+__device__ __forceinline__ void raise_timeout(int *status) { atomicExch(status, (int)QBP_ERR_TIMEOUT); }
+
+__global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_constant__ MmaParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_bar;
+    __shared__ uint32_t tmem_slot;
+
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    uint8_t *smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+    const uint32_t stage_bytes = P.a.tile_bytes + P.b.tile_bytes;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile_n = blockIdx.x % P.tiles_n;
+    const int tile_m = blockIdx.x / P.tiles_n;
+    const int n0 = tile_n * P.bn;
+
+    // tile origin: matrix row for a GEMM, (image, row, column) for a convolution
+    int m0 = tile_m * 128, img0 = 0, h0 = 0, w0 = 0;
+    if (P.mode != MODE_GEMM) {
+        const int tw = tile_m % P.tiles_w;
+        const int th = (tile_m / P.tiles_w) % P.tiles_h;
+        const int tn = tile_m / (P.tiles_w * P.tiles_h);
+        w0 = tw << P.bw_log2;
+        h0 = th << P.bh_log2;
+        img0 = tn * (128 >> (P.bw_log2 + P.bh_log2));
+    }
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&acc_bar, 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&P.mapA);
+        tma_prefetch_desc(&P.mapB);
+    }
+    if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    bool timed_out = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------ TMA producer
+            for (int it = 0; it < P.k_iters; ++it) {
+                const int s = it % P.stages;
+                const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1u)) { timed_out = true; break; }
+                uint8_t *sa = smem + (size_t)s * stage_bytes;
+                uint8_t *sb = sa + P.a.tile_bytes;
+                mbar_expect_tx(&full_bar[s], stage_bytes);
+                if (P.mode == MODE_GEMM) {
+                    const int k0 = it * P.kblock;
+                    if (P.a.major == 0) tma_load_2d(sa, &P.mapA, &full_bar[s], k0, m0);
+                    else                tma_load_2d(sa, &P.mapA, &full_bar[s], m0, k0);
+                    if (P.b.major == 0) tma_load_2d(sb, &P.mapB, &full_bar[s], k0, n0);
+                    else                tma_load_2d(sb, &P.mapB, &full_bar[s], n0, k0);
+                } else {
+                    const int tap = it / P.cchunks, cc = it % P.cchunks;
+                    const int r = tap / P.S, t = tap % P.S;
+                    const int c0 = cc * P.chunk_bytes;
+                    if (P.mode == MODE_FPROP) {
+                        // input pixel of output (p,q) under tap (r,t): (p - pad + r, q - pad + t)
+                        tma_load_4d(sa, &P.mapA, &full_bar[s], c0, w0 - P.pad + t, h0 - P.pad + r, img0);
+                        // filter as [K rows x (R*S*C) columns]: this tap's channel chunk, K-major
+                        tma_load_2d(sb, &P.mapB, &full_bar[s], tap * P.Cred + c0, n0);
+                    } else {
+                        // gradient pixel feeding input (h,w) under tap (r,t): (h + pad - r, w + pad - t)
+                        tma_load_4d(sa, &P.mapA, &full_bar[s], c0, w0 + P.pad - t, h0 + P.pad - r, img0);
+                        // filter rows = output channels (the reduction), columns = this tap's input channels
+                        tma_load_2d(sb, &P.mapB, &full_bar[s], tap * (int)P.N + n0, c0);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // -------------------------------------------------- MMA issuer
+            for (int it = 0; it < P.k_iters; ++it) {
+                const int s = it % P.stages;
+                const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
+                if (!mbar_wait(&full_bar[s], ph)) { timed_out = true; break; }
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+                const uint32_t b_addr = a_addr + P.a.tile_bytes;
+                const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.a.desc_lo;
+                const uint32_t b_lo = ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
+                for (int kk = 0; kk < P.mma_per_iter; ++kk) {
+                    const uint64_t da = ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep);
+                    const uint64_t db = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(b_lo + kk * P.b.kstep);
+                    mma_i8(tmem_base, da, db, P.idesc, (it | kk) != 0 ? 1u : 0u);
+                }
+                mma_commit(&empty_bar[s]);
+            }
+            if (!timed_out) mma_commit(&acc_bar);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------- epilogue
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        if (!mbar_wait(&acc_bar, 0)) timed_out = true;
+        tc_fence_after();
+        if (!timed_out) {
+            int64_t m; bool valid; int cls = 0;
+            if (P.mode == MODE_GEMM) {
+                m = (int64_t)m0 + row;
+                valid = m < P.M;
+            } else {
+                const int dw = row & ((1 << P.bw_log2) - 1);
+                const int dh = (row >> P.bw_log2) & ((1 << P.bh_log2) - 1);
+                const int dn = row >> (P.bw_log2 + P.bh_log2);
+                const int n = img0 + dn, p = h0 + dh, q = w0 + dw;
+                valid = n < P.Nimg && p < P.H && q < P.W;
+                m = ((int64_t)n * P.H + p) * P.W + q;
+                cls = (p == 0 ? 1 : 0) | (p == P.H - 1 ? 2 : 0) | (q == 0 ? 4 : 0) | (q == P.W - 1 ? 8 : 0);
+            }
+            const int rterm = valid ? P.rowterm[m] : 0;
+            const int32_t *cterm = P.colterm + (int64_t)cls * P.N;
+            const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
+            for (int c0 = 0; c0 < P.bn; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, r);
+                tmem_ld_wait();
+                if (!valid) continue;
+                const int64_t ncol = P.N - (n0 + c0);                 // columns left in the matrix
+                if (ncol <= 0) continue;
+                const int lim = ncol < 32 ? (int)ncol : 32;
+                int acc[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[j] = j < lim ? (int)r[j] + rterm + __ldg(cterm + n0 + c0 + j) : 0;
+                if (P.acc_out) {
+                    int32_t *dst = P.acc_out + m * P.N + n0 + c0;
+                    if (lim == 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<int4 *>(dst + j) = make_int4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                    } else {
+                        for (int j = 0; j < lim; ++j) dst[j] = acc[j];
+                    }
+                }
+                if (P.out) {
+                    float *dst = P.out + m * P.N + n0 + c0;
+                    if (lim == 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4 *>(dst + j) =
+                                make_float4(__fmul_rn((float)acc[j], scale), __fmul_rn((float)acc[j + 1], scale),
+                                            __fmul_rn((float)acc[j + 2], scale), __fmul_rn((float)acc[j + 3], scale));
+                    } else {
+                        for (int j = 0; j < lim; ++j) dst[j] = __fmul_rn((float)acc[j], scale);
+                    }
+                }
+            }
+        }
+    }
+
+    if (timed_out) {
+        raise_timeout(P.status);
+        __nanosleep(1000000);          // let copies already in flight land before the CTA retires
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+}
+
+// ================================================= zero-point correction terms
+// GEMM: rowterm[m] = -zb * sum_k A[m,k] + K*za*zb ; colterm[n] = -za * sum_k B[k,n].
+// The code sums arrive as int32 (sums along stored rows) or int64 (along stored columns).
+__global__ void gemm_terms_kernel(const int32_t *ra32, const long long *ra64, const int32_t *cb32, const long long *cb64,
+                                  int64_t M, int64_t N, int64_t K, const qbp_qparams *qa, const qbp_qparams *qb,
+                                  int32_t *rowterm, int32_t *colterm)
+{
+    const int za = qa->zero_point, zb = qb->zero_point;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < M) {
+        const int ra = ra32 ? ra32[i] : (int)ra64[i];
+        rowterm[i] = -zb * ra + (int)K * za * zb;
+    }
+    if (i < N) {
+        const int cb = cb32 ? cb32[i] : (int)cb64[i];
+        colterm[i] = -za * cb;
+    }
+}
+
+// Convolution, per output pixel: the sum of the input's channel sums over the
+// taps that fall inside the image, and how many taps those are.
+//   rowterm[m] = -zw * box[m] + taps_in(m) * Cred * z_in * zw
+__global__ void conv_rowterm_kernel(const int32_t *__restrict__ chan_sum, int Nimg, int H, int W, int pad, int Cred,
+                                    const qbp_qparams *q_in, const qbp_qparams *q_w, int32_t *__restrict__ rowterm)
+{
+    const int64_t m = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= (int64_t)Nimg * H * W) return;
+    const int q = (int)(m % W), p = (int)((m / W) % H);
+    const int64_t img = m / ((int64_t)W * H);
+    int box = 0, taps = 0;
+    for (int dh = -pad; dh <= pad; ++dh) {
+        const int h = p + dh;
+        if (h < 0 || h >= H) continue;
+        for (int dw = -pad; dw <= pad; ++dw) {
+            const int w = q + dw;
+            if (w < 0 || w >= W) continue;
+            box += chan_sum[(img * H + h) * W + w];
+            ++taps;
+        }
+    }
+    rowterm[m] = -q_w->zero_point * box + taps * Cred * q_in->zero_point * q_w->zero_point;
+}
+
+// colterm[cls][n] = -z_in * sum over the taps valid for border class cls of the
+// filter's code sum for that tap and output column n.  cls bits: 1 first row,
+// 2 last row, 4 first column, 8 last column.  wsum32: [n][tap] (forward: sums over
+// the input channels); wsum64: [tap][n] (layer gradient: sums over the output channels).
+__global__ void conv_colterm_kernel(const int32_t *wsum32, const long long *wsum64, int N, int R, int S, int pad,
+                                    int dgrad, const qbp_qparams *q_in, int32_t *colterm)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int cls = blockIdx.y;
+    if (n >= N) return;
+    const bool top = cls & 1, bottom = cls & 2, left = cls & 4, right = cls & 8;
+    long long sum = 0;
+    for (int r = 0; r < R; ++r) {
+        // forward: tap row r reads input row p - pad + r; layer gradient: gradient row h + pad - r
+        const bool low = dgrad ? r > pad : r < pad, high = dgrad ? r < pad : r > pad;
+        if ((low && top) || (high && bottom)) continue;
+        for (int s = 0; s < S; ++s) {
+            const bool lo_c = dgrad ? s > pad : s < pad, hi_c = dgrad ? s < pad : s > pad;
+            if ((lo_c && left) || (hi_c && right)) continue;
+            const int tap = r * S + s;
+            sum += wsum32 ? (long long)wsum32[(int64_t)n * R * S + tap] : wsum64[(int64_t)tap * N + n];
+        }
+    }
+    colterm[cls * N + n] = -q_in->zero_point * (int)sum;
+}
+
+// ================================================================== launchers
+static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
+{
+    const uint32_t stage_bytes = P.a.tile_bytes + P.b.tile_bytes;
+    int stages = (int)((200u * 1024u) / stage_bytes);
+    stages = std::max(2, std::min(stages, kMaxStages));
+    stages = std::min(stages, std::max(2, P.k_iters));
+    P.stages = stages;
+    int cols = 32; while (cols < P.bn) cols <<= 1;
+    P.tmem_cols = cols;
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    static thread_local size_t configured = 0;
+    if (smem > configured) {
+        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        configured = 220 * 1024;
+    }
+    QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
+    qbp_mma_kernel<<<tiles_m * P.tiles_n, kMmaThreads, smem, st>>>(P);
+    QBP_LAUNCH_OK("qbp_mma_kernel");
+    return QBP_OK;
+}
+
+static size_t gemm_ws_bytes(int64_t M, int64_t N)
+{
+    return 256 + align_up(sizeof(int32_t) * M, 256) + align_up(sizeof(int32_t) * N, 256) +
+           align_up(sizeof(int64_t) * M, 256) + align_up(sizeof(int64_t) * N, 256);
+}
+
+static bool conv_supported(const qbp_conv_desc *d)
+{
+    return d->stride == 1 && d->R == d->S && (d->R == 1 || d->R == 3) && d->pad == (d->R - 1) / 2 && d->N > 0 &&
+           d->H > 0 && d->W > 0 && d->C > 0 && d->K > 0 && d->C % 16 == 0 && d->K % 16 == 0;
+}
+
+static size_t conv_ws_bytes(const qbp_conv_desc *d)
+{
+    const int64_t pix = (int64_t)d->N * d->H * d->W;
+    const int64_t nmax = std::max(d->C, d->K);
+    return 256 + align_up(sizeof(int32_t) * pix, 256) * 2 + align_up(sizeof(int32_t) * 16 * nmax, 256) +
+           align_up(sizeof(int64_t) * (int64_t)d->R * d->S * nmax, 256);
+}
+
+// Picks the pixel box (bw x bh x bn = 128, powers of two) that wastes the fewest MMA rows.
+static void pick_pixel_box(int Nimg, int H, int W, int &bwl, int &bhl)
+{
+    long long best = -1;
+    for (int a = 0; a <= 7; ++a)
+        for (int b = 0; a + b <= 7; ++b) {
+            const int bw = 1 << a, bh = 1 << b, bn = 128 >> (a + b);
+            const long long tiles = (long long)((W + bw - 1) / bw) * ((H + bh - 1) / bh) * ((Nimg + bn - 1) / bn);
+            // prefer fewer tiles, then wider rows (longer contiguous runs per TMA row)
+            const long long score = tiles * 64 - a * 8 - b;
+            if (best < 0 || score < best) { best = score; bwl = a; bhl = b; }
+        }
+}
+
+}  // namespace qbp
+
+using namespace qbp;
+
+extern "C" __attribute__((visibility("default"))) size_t qbp_gemm_s8_workspace_bytes(int64_t M, int64_t N, int64_t K)
+{
+    (void)K;
+    return gemm_ws_bytes(M > 0 ? M : 1, N > 0 ? N : 1);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A,
+                           const qbp_qparams *qa, const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C,
+                           void *ws, size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (M <= 0 || N <= 0 || K <= 0) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: M, N, K must be positive");
+    if (M % 16 || N % 16 || K % 16) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "gemm_s8: M, N, K must be multiples of 16");
+    if (K > 33025) return fail(QBP_ERR_OVERFLOW_K, "gemm_s8: K = %lld exceeds 33025 (255*255*K must fit int32)", (long long)K);
+    if (M > INT32_MAX || N > INT32_MAX) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "gemm_s8: extent too large");
+    if (!A || !B || !qa || !qb) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: NULL operand");
+    if (!acc_out && !C) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: acc_out and C are both NULL");
+    if (!aligned16(A) || !aligned16(B) || (C && !aligned16(C)) || (acc_out && !aligned16(acc_out)))
+        return fail(QBP_ERR_INVALID_ARG, "gemm_s8: operands must be 16-byte aligned");
+    if (!ws || ws_bytes < gemm_ws_bytes(M, N))
+        return fail(QBP_ERR_WORKSPACE, "gemm_s8: workspace of %zu bytes needed, %zu given", gemm_ws_bytes(M, N), ws_bytes);
+
+    WsCarver w(ws, ws_bytes);
+    int *status = w.take<int>(1);
+    int32_t *rowterm = w.take<int32_t>(M);
+    int32_t *colterm = w.take<int32_t>(N);
+    int64_t *tmp_m = w.take<int64_t>(M);
+    int64_t *tmp_n = w.take<int64_t>(N);
+
+    // code sums along the reduction
+    int rc;
+    if (!transA) rc = launch_rowsum(A, true, M, K, (int32_t *)tmp_m, st);
+    else         rc = launch_colsum(A, K, M, tmp_m, st);
+    if (rc) return rc;
+    if (transB) rc = launch_rowsum(B, true, N, K, (int32_t *)tmp_n, st);
+    else        rc = launch_colsum(B, K, N, tmp_n, st);
+    if (rc) return rc;
+    const int64_t mx = std::max(M, N);
+    gemm_terms_kernel<<<(int)((mx + 255) / 256), 256, 0, st>>>(
+        transA ? nullptr : (const int32_t *)tmp_m, transA ? (const long long *)tmp_m : nullptr,
+        transB ? (const int32_t *)tmp_n : nullptr, transB ? nullptr : (const long long *)tmp_n, M, N, K, qa, qb,
+        rowterm, colterm);
+    QBP_LAUNCH_OK("gemm_terms_kernel");
+
+    MmaParams P{};
+    P.mode = MODE_GEMM;
+    P.kblock = 128;
+    P.k_iters = (int)((K + 127) / 128);
+    P.mma_per_iter = 4;
+    // A: stored [M x K] -> K-major rows of 128 reduction bytes; stored [K x M] -> MN-major
+    if (!transA) { P.a = layout_kmajor(128, 128); rc = make_map_2d(&P.mapA, A, M, K, 128, 128); }
+    else         { P.a = layout_mnmajor(128, 128, 1, 0); rc = make_map_2d(&P.mapA, A, K, M, 128, 128); }
+    if (rc) return rc;
+    if (transB) {
+        P.bn = (int)std::min<int64_t>(256, N);
+        P.b = layout_kmajor((uint32_t)P.bn, 128);
+        rc = make_map_2d(&P.mapB, B, N, K, (uint32_t)P.bn, 128);
+    } else {
+        // N-contiguous operand: one swizzled row holds min(128, N) output columns
+        const uint32_t rb = N >= 128 ? 128u : N >= 64 ? 64u : 32u;
+        P.bn = (int)rb;
+        P.b = layout_mnmajor(128, rb, 1, 0);
+        rc = make_map_2d(&P.mapB, B, K, N, 128, rb);
+    }
+    if (rc) return rc;
+    P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
+    P.tiles_n = (int)((N + P.bn - 1) / P.bn);
+    P.M = M; P.N = N;
+    P.acc_out = acc_out; P.out = C;
+    P.rowterm = rowterm; P.colterm = colterm; P.qa = qa; P.qb = qb; P.status = status;
+    return launch_mma(P, (int)((M + 127) / 128), st);
+}
+
+extern "C" __attribute__((visibility("default"))) size_t qbp_conv_s8_workspace_bytes(int mode, const qbp_conv_desc *d)
+{
+    (void)mode;
+    if (!d || !conv_supported(d)) return 0;
+    return conv_ws_bytes(d);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in,
+                                    const int8_t *wgt, const qbp_qparams *q_w, int32_t *acc_out, float *out, void *ws,
+                                    size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!d) return fail(QBP_ERR_INVALID_ARG, "conv_s8: descriptor is NULL");
+    if (mode != QBP_CONV_FPROP && mode != QBP_CONV_DGRAD) return fail(QBP_ERR_INVALID_ARG, "conv_s8: bad mode");
+    if (!conv_supported(d))
+        return fail(QBP_ERR_UNSUPPORTED_SHAPE,
+                    "conv_s8: needs stride 1, R = S in {1,3}, pad = (R-1)/2, C and K multiples of 16");
+    if ((int64_t)d->R * d->S * std::max(d->C, d->K) > 33025)
+        return fail(QBP_ERR_OVERFLOW_K, "conv_s8: reduction length exceeds 33025");
+    if (!in || !wgt || !q_in || !q_w) return fail(QBP_ERR_INVALID_ARG, "conv_s8: NULL operand");
+    if (!acc_out && !out) return fail(QBP_ERR_INVALID_ARG, "conv_s8: acc_out and out are both NULL");
+    if (!aligned16(in) || !aligned16(wgt) || (out && !aligned16(out)) || (acc_out && !aligned16(acc_out)))
+        return fail(QBP_ERR_INVALID_ARG, "conv_s8: operands must be 16-byte aligned");
+    if (!ws || ws_bytes < conv_ws_bytes(d))
+        return fail(QBP_ERR_WORKSPACE, "conv_s8: workspace of %zu bytes needed, %zu given", conv_ws_bytes(d), ws_bytes);
+
+    const bool dgrad = mode == QBP_CONV_DGRAD;
+    const int Cred = dgrad ? d->K : d->C;        // channels reduced over
+    const int Nout = dgrad ? d->C : d->K;        // channels produced
+    const int64_t pix = (int64_t)d->N * d->H * d->W;
+    const int taps = d->R * d->S;
+    const int64_t nmax = std::max(d->C, d->K);
+
+    WsCarver w(ws, ws_bytes);
+    int *status = w.take<int>(1);
+    int32_t *rowterm = w.take<int32_t>(pix);
+    int32_t *chan_sum = w.take<int32_t>(pix);
+    int32_t *colterm = w.take<int32_t>(16 * nmax);
+    int64_t *wsum = w.take<int64_t>((int64_t)taps * nmax);
+
+    int rc = launch_rowsum(in, true, pix, Cred, chan_sum, st);
+    if (rc) return rc;
+    conv_rowterm_kernel<<<(int)((pix + 255) / 256), 256, 0, st>>>(chan_sum, d->N, d->H, d->W, d->pad, Cred, q_in, q_w, rowterm);
+    QBP_LAUNCH_OK("conv_rowterm_kernel");
+    if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
+    else        rc = launch_colsum(wgt, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
+    if (rc) return rc;
+    conv_colterm_kernel<<<dim3((Nout + 127) / 128, 16), 128, 0, st>>>(
+        dgrad ? nullptr : (const int32_t *)wsum, dgrad ? (const long long *)wsum : nullptr, Nout, d->R, d->S, d->pad,
+        dgrad ? 1 : 0, q_in, colterm);
+    QBP_LAUNCH_OK("conv_colterm_kernel");
+
+    MmaParams P{};
+    P.mode = dgrad ? MODE_DGRAD : MODE_FPROP;
+    P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.S = d->S; P.Cred = Cred;
+    const uint32_t cb = Cred % 128 == 0 ? 128u : Cred % 64 == 0 ? 64u : 32u;      // reduction bytes per stage row
+    P.chunk_bytes = (int)cb;
+    P.cchunks = (Cred + (int)cb - 1) / (int)cb;      // a ragged last chunk is zero-filled by TMA on the activation side
+    P.k_iters = taps * P.cchunks;
+    P.mma_per_iter = (int)cb / 32;
+    int bwl = 0, bhl = 0;
+    pick_pixel_box(d->N, d->H, d->W, bwl, bhl);
+    P.bw_log2 = bwl; P.bh_log2 = bhl;
+    const int bw = 1 << bwl, bh = 1 << bhl, bn_img = 128 >> (bwl + bhl);
+    P.tiles_w = (d->W + bw - 1) / bw; P.tiles_h = (d->H + bh - 1) / bh;
+    const int tiles_img = (d->N + bn_img - 1) / bn_img;
+    P.a = layout_kmajor(128, cb);
+    rc = make_map_nhwc(&P.mapA, in, d->N, d->H, d->W, Cred, bn_img, bh, bw, cb);
+    if (rc) return rc;
+    if (!dgrad) {
+        P.bn = std::min(256, Nout);
+        P.b = layout_kmajor((uint32_t)P.bn, cb);
+        rc = make_map_2d(&P.mapB, wgt, d->K, (uint64_t)taps * d->C, (uint32_t)P.bn, cb);
+    } else {
+        const uint32_t rb = Nout >= 128 ? 128u : Nout >= 64 ? 64u : 32u;
+        P.bn = (int)rb;
+        P.b = layout_mnmajor(cb, rb, 1, 0);
+        rc = make_map_2d(&P.mapB, wgt, d->K, (uint64_t)taps * d->C, cb, rb);
+    }
+    if (rc) return rc;
+    P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
+    P.tiles_n = (Nout + P.bn - 1) / P.bn;
+    P.M = pix; P.N = Nout;
+    P.acc_out = acc_out; P.out = out;
+    P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
+    return launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st);
+}

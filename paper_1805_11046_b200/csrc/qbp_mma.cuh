@@ -1,0 +1,42 @@
+// Declarations shared by the tensor-core product files: TMA tensor-map
+// construction on the host, the parameter block of the tcgen05 kernels, and
+// the small helper launchers (row/column sums of codes).
+#pragma once
+
+#include <cuda.h>
+
+#include "qbp_common.cuh"
+
+namespace qbp {
+
+// ---- sums of stored codes (qbp_quant.cu) -------------------------------------
+int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int32_t *sums, cudaStream_t st);
+int launch_colsum(const int8_t *q, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st);
+
+// ---- TMA tensor maps ---------------------------------------------------------
+// A dense byte matrix [rows x cols] (cols innermost) read in boxes of
+// box_cols x box_rows; box_cols in {32, 64, 128} selects the matching swizzle.
+int make_map_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols);
+// A dense NHWC byte tensor read in boxes of box_c x bw x bh x bn.
+int make_map_nhwc(CUtensorMap *map, const void *base, uint64_t N, uint64_t H, uint64_t W, uint64_t C, uint32_t bn,
+                  uint32_t bh, uint32_t bw, uint32_t box_c);
+
+// ---- shared-memory operand descriptors ---------------------------------------
+// How one operand tile of a pipeline stage is laid out and walked by the MMAs.
+struct OperandLayout {
+    uint32_t tile_bytes;    // bytes of this operand per stage
+    uint32_t desc_lo;       // descriptor bits 16..31 (leading byte offset), address added at run time
+    uint32_t desc_hi;       // descriptor bits 32..63 (stride byte offset, version, swizzle)
+    uint32_t kstep;         // start-address advance per MMA (K = 32), in 16-byte units
+    uint32_t major;         // 0 = K-major, 1 = MN-major (instruction descriptor bit)
+};
+
+// K-major tile: `rows` rows of `row_bytes` (32/64/128, swizzled alike) reduction bytes.
+OperandLayout layout_kmajor(uint32_t rows, uint32_t row_bytes);
+// MN-major tile: `krows` reduction rows of `row_bytes` (32/64/128) M/N bytes each;
+// `chunks` such tiles side by side (chunk_stride bytes apart) widen M/N beyond row_bytes.
+OperandLayout layout_mnmajor(uint32_t krows, uint32_t row_bytes, uint32_t chunks, uint32_t chunk_stride);
+
+uint32_t make_idesc(bool a_signed, bool b_signed, uint32_t a_major, uint32_t b_major, uint32_t m, uint32_t n);
+
+}  // namespace qbp

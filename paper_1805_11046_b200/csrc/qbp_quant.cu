@@ -1,0 +1,580 @@
+// Range quantiser kernels (Section 4 "Quantization methods", Appendix B):
+// min/max range scan, scale / zero-point, nearest and stochastic rounding to
+// 8 and 16 bits, byte-limb split of the 16-bit codes, and the fused
+// "bifurcation" that writes the 8-bit and 16-bit copies of a gradient from
+// one read.  All of it is HBM-bound streaming work: 16-byte loads, 4 loads in
+// flight per thread, warp-shuffle + shared-memory reductions, grids sized to
+// fill every SM.  Also hosts the library's error-reporting state.
+#include "qbp_colscan.cuh"
+
+#include <cstring>
+
+namespace qbp {
+
+// ------------------------------------------------------------ error state
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...)
+{
+    va_list ap; va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+int fail(int status, const char *fmt, ...)
+{
+    va_list ap; va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return status;
+}
+int sm_count()
+{
+    static thread_local int cached_dev = -1, cached = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) cached = n;
+        else cudaGetLastError();
+        cached_dev = dev;
+    }
+    return cached;
+}
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;
+constexpr int kMaxParts = 4096;          // upper bound on per-tensor scan blocks
+
+// ------------------------------------------------------- per-tensor range
+template <int VEC>
+__global__ void __launch_bounds__(kThreads) range_partial_kernel(const float *__restrict__ x, int64_t n,
+                                                                 float2 *__restrict__ partials)
+{
+    float lo = INFINITY, hi = -INFINITY;
+    const int64_t nv = n / VEC;
+    const int64_t stride = (int64_t)gridDim.x * kThreads * kUnroll;
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * kUnroll; base < nv; base += stride) {
+        VecF<VEC> v[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            int64_t i = base + u * kThreads + threadIdx.x;
+            ok[u] = i < nv;
+            if (ok[u]) v[u].load(x + i * VEC);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (ok[u]) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) { lo = fminf(lo, v[u].v[e]); hi = fmaxf(hi, v[u].v[e]); }
+            }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (int64_t i = nv * VEC; i < n; ++i) { lo = fminf(lo, x[i]); hi = fmaxf(hi, x[i]); }
+    lo = warp_min(lo); hi = warp_max(hi);
+    __shared__ float s_lo[kThreads / 32], s_hi[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        lo = threadIdx.x < kThreads / 32 ? s_lo[threadIdx.x] : INFINITY;
+        hi = threadIdx.x < kThreads / 32 ? s_hi[threadIdx.x] : -INFINITY;
+        lo = warp_min(lo); hi = warp_max(hi);
+        if (threadIdx.x == 0) partials[blockIdx.x] = make_float2(lo, hi);
+    }
+}
+
+// One block: combine the partial ranges, emit the parameters for 8 and/or 16 bits.
+__global__ void __launch_bounds__(kThreads) range_finalize_kernel(const float2 *__restrict__ partials, int nparts,
+                                                                  qbp_qparams *qp8, qbp_qparams *qp16)
+{
+    float lo = INFINITY, hi = -INFINITY;
+    for (int i = threadIdx.x; i < nparts; i += kThreads) {
+        float2 p = partials[i];
+        lo = fminf(lo, p.x); hi = fmaxf(hi, p.y);
+    }
+    lo = warp_min(lo); hi = warp_max(hi);
+    __shared__ float s_lo[kThreads / 32], s_hi[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 0; w < kThreads / 32; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); }
+        if (qp8) *qp8 = make_qparams(lo, hi, 8);
+        if (qp16) *qp16 = make_qparams(lo, hi, 16);
+    }
+}
+
+// Parameters from clamping values the caller already has (one thread each).
+__global__ void qparams_from_range_kernel(const qbp_qparams *__restrict__ in, int count, int bits,
+                                          qbp_qparams *__restrict__ out)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) out[i] = make_qparams(in[i].vmin, in[i].vmax, bits);
+}
+
+// ------------------------------------------------------ per-channel range
+template <int VEC>
+__global__ void __launch_bounds__(kScanThreads) chan_range_partial_kernel(const float *__restrict__ x, int64_t rows,
+                                                                          int C, int tw, float *__restrict__ part_lo,
+                                                                          float *__restrict__ part_hi)
+{
+    const ScanPos p = scan_pos<VEC>(C, tw);
+    const int rpb = kScanThreads / tw;
+    float lo[VEC], hi[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { lo[e] = INFINITY; hi[e] = -INFINITY; }
+    if (p.active) {
+        const int64_t step = (int64_t)gridDim.x * rpb;
+        for (int64_t r0 = (int64_t)blockIdx.x * rpb + p.ty; r0 < rows; r0 += step * kScanUnroll) {
+            VecF<VEC> v[kScanUnroll];
+            bool ok[kScanUnroll];
+#pragma unroll
+            for (int u = 0; u < kScanUnroll; ++u) {
+                int64_t r = r0 + u * step;
+                ok[u] = r < rows;
+                if (ok[u]) v[u].load(x + r * C + p.col);
+            }
+#pragma unroll
+            for (int u = 0; u < kScanUnroll; ++u)
+                if (ok[u]) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) { lo[e] = fminf(lo[e], v[u].v[e]); hi[e] = fmaxf(hi[e], v[u].v[e]); }
+                }
+        }
+    }
+    __shared__ float s_lo[kScanThreads * VEC], s_hi[kScanThreads * VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { s_lo[threadIdx.x * VEC + e] = lo[e]; s_hi[threadIdx.x * VEC + e] = hi[e]; }
+    __syncthreads();
+    if (p.ty == 0 && p.active) {
+        for (int y = 1; y < rpb; ++y)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                lo[e] = fminf(lo[e], s_lo[(y * tw + p.tx) * VEC + e]);
+                hi[e] = fmaxf(hi[e], s_hi[(y * tw + p.tx) * VEC + e]);
+            }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            part_lo[(int64_t)blockIdx.x * C + p.col + e] = lo[e];
+            part_hi[(int64_t)blockIdx.x * C + p.col + e] = hi[e];
+        }
+    }
+}
+
+// One warp per channel over the strip partials.
+__global__ void __launch_bounds__(kThreads) chan_range_finalize_kernel(const float *__restrict__ part_lo,
+                                                                       const float *__restrict__ part_hi, int nparts,
+                                                                       int C, int bits, qbp_qparams *__restrict__ qp)
+{
+    int c = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (c >= C) return;
+    float lo = INFINITY, hi = -INFINITY;
+    for (int i = threadIdx.x & 31; i < nparts; i += 32) {
+        lo = fminf(lo, part_lo[(int64_t)i * C + c]);
+        hi = fmaxf(hi, part_hi[(int64_t)i * C + c]);
+    }
+    lo = warp_min(lo); hi = warp_max(hi);
+    if ((threadIdx.x & 31) == 0) qp[c] = make_qparams(lo, hi, bits);
+}
+
+// ------------------------------------------------------------ quantisation
+struct QuantOut {
+    int8_t *q8;      // 8-bit codes (nullable)
+    int16_t *q16;    // 16-bit codes (nullable)
+    int8_t *hi;      // high byte of the 16-bit code (nullable)
+    uint8_t *lo;     // low byte (nullable)
+};
+
+struct QParamsReg { float inv, zp_u; };
+
+__device__ __forceinline__ QParamsReg load_qp(const qbp_qparams *qp, int bits)
+{
+    QParamsReg r;
+    r.inv = __fdiv_rn(1.0f, qp->scale);
+    r.zp_u = (float)(qp->zero_point + (1 << (bits - 1)));
+    return r;
+}
+
+// Scalar path: unaligned tensors, per-element tails.  One Philox block per element.
+template <bool SR>
+__device__ __forceinline__ void quantize_scalar(const float *x, int64_t i, int cols, bool perch,
+                                                const qbp_qparams *qp8, uint32_t id8, const qbp_qparams *qp16,
+                                                uint32_t id16, uint2 key, const QuantOut &o)
+{
+    const int c = perch ? (int)(i % cols) : 0;
+    const float v = x[i];
+    const uint64_t j = (uint64_t)i >> 2;
+    if (o.q8) {
+        QParamsReg p = load_qp(qp8 + c, 8);
+        uint32_t rnd = 0;
+        if (SR) {
+            uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)(j >> 32), id8, 0u), key);
+            const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+            rnd = w[i & 3];
+        }
+        o.q8[i] = (int8_t)(quantize_code<SR>(v, p.inv, p.zp_u, 255.0f, rnd) - 128);
+    }
+    if (o.q16 || o.hi || o.lo) {
+        QParamsReg p = load_qp(qp16 + c, 16);
+        uint32_t rnd = 0;
+        if (SR) {
+            uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)(j >> 32), id16, 0u), key);
+            const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+            rnd = w[i & 3];
+        }
+        int s = quantize_code<SR>(v, p.inv, p.zp_u, 65535.0f, rnd) - 32768;
+        if (o.q16) o.q16[i] = (int16_t)s;
+        if (o.hi) o.hi[i] = (int8_t)(s >> 8);
+        if (o.lo) o.lo[i] = (uint8_t)(s & 0xFF);
+    }
+}
+
+template <bool SR, int VEC>
+__global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restrict__ x, int64_t n, int cols,
+                                                            int perch, const qbp_qparams *__restrict__ qp8,
+                                                            uint32_t id8, const qbp_qparams *__restrict__ qp16,
+                                                            uint32_t id16, uint2 key, QuantOut o)
+{
+    if (VEC == 1) {
+        const int64_t stride = (int64_t)gridDim.x * kThreads;
+        for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += stride)
+            quantize_scalar<SR>(x, i, cols, perch != 0, qp8, id8, qp16, id16, key, o);
+        return;
+    }
+    const bool want8 = o.q8 != nullptr, want16 = o.q16 || o.hi || o.lo;
+    QParamsReg p8 = {0, 0}, p16 = {0, 0};
+    if (!perch) {
+        if (want8) p8 = load_qp(qp8, 8);
+        if (want16) p16 = load_qp(qp16, 16);
+    }
+    const int64_t nv = n >> 2;
+    const int64_t stride = (int64_t)gridDim.x * kThreads * kUnroll;
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * kUnroll; base < nv; base += stride) {
+        float4 v[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            int64_t j = base + u * kThreads + threadIdx.x;
+            ok[u] = j < nv;
+            if (ok[u]) v[u] = __ldg(reinterpret_cast<const float4 *>(x) + j);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (!ok[u]) continue;
+            const int64_t j = base + u * kThreads + threadIdx.x;
+            const float xs[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            const int c0 = perch ? (int)((j << 2) % cols) : 0;
+            if (want8) {
+                uint32_t r[4] = {0, 0, 0, 0};
+                if (SR) {
+                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id8, 0u), key);
+                    r[0] = b.x; r[1] = b.y; r[2] = b.z; r[3] = b.w;
+                }
+                uint32_t packed = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (perch) p8 = load_qp(qp8 + c0 + e, 8);
+                    int code = quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
+                    packed |= (uint32_t)((code ^ 0x80) & 0xFF) << (8 * e);
+                }
+                reinterpret_cast<uint32_t *>(o.q8)[j] = packed;
+            }
+            if (want16) {
+                uint32_t r[4] = {0, 0, 0, 0};
+                if (SR) {
+                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id16, 0u), key);
+                    r[0] = b.x; r[1] = b.y; r[2] = b.z; r[3] = b.w;
+                }
+                uint32_t s[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (perch) p16 = load_qp(qp16 + c0 + e, 16);
+                    s[e] = (uint32_t)(quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]) ^ 0x8000);
+                }
+                if (o.q16)
+                    reinterpret_cast<uint2 *>(o.q16)[j] = make_uint2(s[0] | (s[1] << 16), s[2] | (s[3] << 16));
+                if (o.hi)
+                    reinterpret_cast<uint32_t *>(o.hi)[j] =
+                        (s[0] >> 8) | ((s[1] >> 8) << 8) | ((s[2] >> 8) << 16) | ((s[3] >> 8) << 24);
+                if (o.lo)
+                    reinterpret_cast<uint32_t *>(o.lo)[j] =
+                        (s[0] & 0xFF) | ((s[1] & 0xFF) << 8) | ((s[2] & 0xFF) << 16) | ((s[3] & 0xFF) << 24);
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (int64_t i = nv << 2; i < n; ++i)
+            quantize_scalar<SR>(x, i, cols, perch != 0, qp8, id8, qp16, id16, key, o);
+}
+
+// Row sums of stored 8-bit codes: a group of G lanes per row (G = smallest power
+// of two covering cols/16, at most 32), 16-byte loads.
+template <bool IS_SIGNED>
+__global__ void __launch_bounds__(kThreads) rowsum_kernel(const uint8_t *__restrict__ q, int64_t rows, int cols,
+                                                          int G, int32_t *__restrict__ sums)
+{
+    const int lane = threadIdx.x & 31;
+    const int gl = lane % G;
+    const int64_t groups_per_block = kThreads / G;
+    const int cv = cols >> 4;
+    for (int64_t r = (int64_t)blockIdx.x * groups_per_block + threadIdx.x / G; r < rows;
+         r += (int64_t)gridDim.x * groups_per_block) {
+        int acc = 0;
+        const uint4 *row = reinterpret_cast<const uint4 *>(q + r * cols);
+        for (int c = gl; c < cv; c += G) {
+            uint4 v = __ldg(row + c);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                acc = IS_SIGNED ? __dp4a((int)w[k], 0x01010101, acc) : (int)__dp4a(w[k], 0x01010101u, (uint32_t)acc);
+        }
+        for (int o = G >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (gl == 0) sums[r] = acc;
+    }
+}
+
+// Column sums (over rows) of stored signed 8-bit codes into int64.  blockIdx.y
+// selects a slab of up to 256 column groups (16 codes each); inside a slab a
+// thread owns one group and every (256 / groups)-th row.  Block partials meet in
+// shared memory, then one atomic per column and block.  The destination must be
+// zeroed beforehand.
+__global__ void __launch_bounds__(kThreads) colsum_kernel(const int8_t *__restrict__ q, int64_t rows, int cols,
+                                                          unsigned long long *__restrict__ sums)
+{
+    const int cv = cols >> 4;
+    const int slab0 = blockIdx.y * kThreads;                 // first column group of this slab
+    const int tw = (cv - slab0) < kThreads ? (cv - slab0) : kThreads;
+    const int rpb = kThreads / tw;
+    const int tx = threadIdx.x % tw, ty = threadIdx.x / tw;
+    __shared__ int s_acc[kThreads * 16];
+    for (int c = threadIdx.x; c < tw * 16; c += kThreads) s_acc[c] = 0;
+    __syncthreads();
+    if (ty < rpb) {
+        int acc[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] = 0;
+        for (int64_t r = (int64_t)blockIdx.x * rpb + ty; r < rows; r += (int64_t)gridDim.x * rpb) {
+            uint4 v = __ldg(reinterpret_cast<const uint4 *>(q + r * cols) + slab0 + tx);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[k * 4 + b] += (int)(int8_t)(w[k] >> (8 * b));
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) atomicAdd(&s_acc[tx * 16 + e], acc[e]);
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < tw * 16; c += kThreads)
+        atomicAdd(&sums[slab0 * 16 + c], (unsigned long long)(long long)s_acc[c]);
+}
+
+// ----------------------------------------------------------------- launchers
+static int grid_for(int64_t work_items_per_thread_group, int64_t n_groups)
+{
+    (void)work_items_per_thread_group;
+    int64_t want = (int64_t)sm_count() * 8;
+    int64_t g = n_groups < want ? n_groups : want;
+    return (int)(g < 1 ? 1 : g);
+}
+
+static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams *qp8, qbp_qparams *qp16,
+                        cudaStream_t st)
+{
+    int nparts = 0;
+    if (n > 0) {
+        const bool vec = aligned16(x);
+        const int64_t per_block = (int64_t)kThreads * kUnroll * (vec ? 4 : 1);
+        nparts = grid_for(1, (n + per_block - 1) / per_block);
+        if (nparts > kMaxParts) nparts = kMaxParts;
+        if (vec) range_partial_kernel<4><<<nparts, kThreads, 0, st>>>(x, n, partials);
+        else     range_partial_kernel<1><<<nparts, kThreads, 0, st>>>(x, n, partials);
+        QBP_LAUNCH_OK("range_partial_kernel");
+    }
+    range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
+    QBP_LAUNCH_OK("range_finalize_kernel");
+    return QBP_OK;
+}
+
+static int launch_chan_range(const float *x, int64_t rows, int64_t cols, int bits, float *part_lo, float *part_hi,
+                             qbp_qparams *qp, cudaStream_t st)
+{
+    ScanGeom g = scan_geom(rows, cols, aligned16(x));
+    int nparts = 0;
+    if (rows > 0) {
+        nparts = g.nbx;
+        dim3 grid(g.nbx, g.slabs);
+        if (g.vec == 4) chan_range_partial_kernel<4><<<grid, kScanThreads, 0, st>>>(x, rows, (int)cols, g.tw, part_lo, part_hi);
+        else            chan_range_partial_kernel<1><<<grid, kScanThreads, 0, st>>>(x, rows, (int)cols, g.tw, part_lo, part_hi);
+        QBP_LAUNCH_OK("chan_range_partial_kernel");
+    }
+    chan_range_finalize_kernel<<<(int)((cols + 7) / 8), kThreads, 0, st>>>(part_lo, part_hi, nparts, (int)cols, bits, qp);
+    QBP_LAUNCH_OK("chan_range_finalize_kernel");
+    return QBP_OK;
+}
+
+static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, int rounding,
+                           const qbp_qparams *qp8, uint32_t id8, const qbp_qparams *qp16, uint32_t id16,
+                           uint64_t seed, const QuantOut &o, cudaStream_t st)
+{
+    if (n == 0) return QBP_OK;
+    const bool vec = aligned16(x) && (!perch || cols % 4 == 0) &&
+                     (!o.q8 || ((uintptr_t)o.q8 & 3) == 0) && (!o.q16 || ((uintptr_t)o.q16 & 7) == 0) &&
+                     (!o.hi || ((uintptr_t)o.hi & 3) == 0) && (!o.lo || ((uintptr_t)o.lo & 3) == 0);
+    const int64_t per_block = (int64_t)kThreads * (vec ? 4 * kUnroll : 1);
+    const int grid = grid_for(1, (n + per_block - 1) / per_block);
+    const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    const int c = (int)cols;
+    if (rounding == QBP_ROUND_STOCHASTIC) {
+        if (vec) quantize_kernel<true, 4><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
+        else     quantize_kernel<true, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
+    } else {
+        if (vec) quantize_kernel<false, 4><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
+        else     quantize_kernel<false, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
+    }
+    QBP_LAUNCH_OK("quantize_kernel");
+    return QBP_OK;
+}
+
+// Row / column sums of stored codes; used by the quantiser's optional outputs
+// and by the integer products' zero-point corrections.
+int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int32_t *sums, cudaStream_t st)
+{
+    if (rows == 0) return QBP_OK;
+    if (cols % 16 || !aligned16(q)) return fail(QBP_ERR_INVALID_ARG, "row sums need 16-byte aligned rows (cols %% 16 == 0)");
+    int G = 1; while (G < 32 && G < cols / 16) G <<= 1;
+    const int64_t groups = kThreads / G;
+    const int grid = grid_for(1, (rows + groups - 1) / groups);
+    if (is_signed) rowsum_kernel<true><<<grid, kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, G, sums);
+    else           rowsum_kernel<false><<<grid, kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, G, sums);
+    QBP_LAUNCH_OK("rowsum_kernel");
+    return QBP_OK;
+}
+
+int launch_colsum(const int8_t *q, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st)
+{
+    if (cols % 16 || !aligned16(q)) return fail(QBP_ERR_INVALID_ARG, "column sums need cols %% 16 == 0");
+    QBP_CUDA_OK(cudaMemsetAsync(sums, 0, sizeof(int64_t) * cols, st));
+    if (rows == 0) return QBP_OK;
+    const int cv = (int)(cols / 16);
+    const int slabs = (cv + kThreads - 1) / kThreads;
+    const int rpb = kThreads / (cv < kThreads ? cv : kThreads);
+    // each thread keeps int32 partials over at most 2^23 rows: 128 * 2^23 < 2^31
+    int64_t min_blocks = (rows >> 23) + 1;
+    int64_t grid = grid_for(1, (rows + rpb - 1) / rpb) / slabs;
+    if (grid < min_blocks) grid = min_blocks;
+    colsum_kernel<<<dim3((unsigned)grid, (unsigned)slabs), kThreads, 0, st>>>(q, rows, (int)cols, (unsigned long long *)sums);
+    QBP_LAUNCH_OK("colsum_kernel");
+    return QBP_OK;
+}
+
+static int check_common(const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
+                        const qbp_qparams *qp_out)
+{
+    if (rows < 0 || cols <= 0) return fail(QBP_ERR_INVALID_ARG, "quantize: rows must be >= 0 and cols > 0");
+    if (granularity != QBP_PER_TENSOR && granularity != QBP_PER_CHANNEL)
+        return fail(QBP_ERR_INVALID_ARG, "quantize: granularity must be QBP_PER_TENSOR or QBP_PER_CHANNEL");
+    if (rounding != QBP_ROUND_NEAREST && rounding != QBP_ROUND_STOCHASTIC)
+        return fail(QBP_ERR_INVALID_ARG, "quantize: rounding must be QBP_ROUND_NEAREST or QBP_ROUND_STOCHASTIC");
+    if (!qp_out) return fail(QBP_ERR_INVALID_ARG, "quantize: qp_out is NULL");
+    if (!x && rows * cols > 0) return fail(QBP_ERR_INVALID_ARG, "quantize: x is NULL");
+    if (((uintptr_t)x & 3) != 0) return fail(QBP_ERR_INVALID_ARG, "quantize: x is not 4-byte aligned");
+    return QBP_OK;
+}
+
+static size_t quant_ws_bytes(int64_t cols, int granularity)
+{
+    if (granularity == QBP_PER_CHANNEL) return 2 * align_up(sizeof(float) * kScanMaxStrips * (size_t)cols, 256) + 256;
+    return align_up(sizeof(float2) * kMaxParts, 256) + 256;
+}
+
+// Shared body of the 8- and 16-bit entry points.
+static int quantize_any(int bits, const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
+                        uint64_t seed, uint32_t tensor_id, const qbp_qparams *range_in, const QuantOut &o,
+                        qbp_qparams *qp_out, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    int rc = check_common(x, rows, cols, granularity, rounding, qp_out);
+    if (rc) return rc;
+    const int perch = granularity == QBP_PER_CHANNEL;
+    if (range_in) {
+        const int count = perch ? (int)cols : 1;
+        qparams_from_range_kernel<<<(count + 255) / 256, 256, 0, st>>>(range_in, count, bits, qp_out);
+        QBP_LAUNCH_OK("qparams_from_range_kernel");
+    } else {
+        if (!ws || ws_bytes < quant_ws_bytes(cols, granularity))
+            return fail(QBP_ERR_WORKSPACE, "quantize: workspace of %zu bytes needed, %zu given",
+                        quant_ws_bytes(cols, granularity), ws_bytes);
+        WsCarver w(ws, ws_bytes);
+        if (perch) {
+            float *plo = w.take<float>((size_t)kScanMaxStrips * cols);
+            float *phi = w.take<float>((size_t)kScanMaxStrips * cols);
+            rc = launch_chan_range(x, rows, cols, bits, plo, phi, qp_out, st);
+        } else {
+            float2 *parts = w.take<float2>(kMaxParts);
+            rc = launch_range(x, rows * cols, parts, bits == 8 ? qp_out : nullptr, bits == 16 ? qp_out : nullptr, st);
+        }
+        if (rc) return rc;
+    }
+    return launch_quantize(x, rows * cols, cols, perch, rounding, qp_out, tensor_id, qp_out, tensor_id, seed, o, st);
+}
+
+}  // namespace qbp
+
+using namespace qbp;
+
+extern "C" __attribute__((visibility("default"))) const char *qbp_last_error(void) { return g_err; }
+
+extern "C" __attribute__((visibility("default"))) size_t qbp_quantize_workspace_bytes(int64_t rows, int64_t cols, int granularity)
+{
+    (void)rows;
+    return quant_ws_bytes(cols > 0 ? cols : 1, granularity);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8(const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
+                               uint64_t seed, uint32_t tensor_id, const qbp_qparams *range_in, int8_t *q,
+                               qbp_qparams *qp_out, int32_t *row_sums, int64_t *col_sums, void *ws, size_t ws_bytes,
+                               void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!q && rows * cols > 0) return fail(QBP_ERR_INVALID_ARG, "quantize_s8: q is NULL");
+    if ((row_sums || col_sums) && granularity != QBP_PER_TENSOR)
+        return fail(QBP_ERR_INVALID_ARG, "quantize_s8: row/column sums are per-tensor only");
+    QuantOut o = {q, nullptr, nullptr, nullptr};
+    int rc = quantize_any(8, x, rows, cols, granularity, rounding, seed, tensor_id, range_in, o, qp_out, ws, ws_bytes, st);
+    if (rc) return rc;
+    if (row_sums) { rc = launch_rowsum(q, true, rows, cols, row_sums, st); if (rc) return rc; }
+    if (col_sums) { rc = launch_colsum(q, rows, cols, col_sums, st); if (rc) return rc; }
+    return QBP_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_quantize_s16(const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
+                                uint64_t seed, uint32_t tensor_id, const qbp_qparams *range_in, int16_t *q,
+                                int8_t *hi, uint8_t *lo, qbp_qparams *qp_out, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!q && !hi && !lo) return fail(QBP_ERR_INVALID_ARG, "quantize_s16: q, hi and lo are all NULL");
+    QuantOut o = {nullptr, q, hi, lo};
+    return quantize_any(16, x, rows, cols, granularity, rounding, seed, tensor_id, range_in, o, qp_out, ws, ws_bytes,
+                        (cudaStream_t)stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_bifurcate(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
+                             uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
+                             uint8_t *lo, qbp_qparams *qp16, void *ws, size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (rows < 0 || cols <= 0) return fail(QBP_ERR_INVALID_ARG, "bifurcate: rows must be >= 0 and cols > 0");
+    if (!qp8 || !qp16) return fail(QBP_ERR_INVALID_ARG, "bifurcate: qp8 / qp16 is NULL");
+    if (rows * cols > 0 && (!g || !q8 || !hi || !lo)) return fail(QBP_ERR_INVALID_ARG, "bifurcate: NULL tensor");
+    if (((uintptr_t)g & 3) != 0) return fail(QBP_ERR_INVALID_ARG, "bifurcate: g is not 4-byte aligned");
+    if (!ws || ws_bytes < quant_ws_bytes(cols, QBP_PER_TENSOR))
+        return fail(QBP_ERR_WORKSPACE, "bifurcate: workspace of %zu bytes needed, %zu given",
+                    quant_ws_bytes(cols, QBP_PER_TENSOR), ws_bytes);
+    WsCarver w(ws, ws_bytes);
+    float2 *parts = w.take<float2>(kMaxParts);
+    int rc = launch_range(g, rows * cols, parts, qp8, qp16, st);
+    if (rc) return rc;
+    QuantOut o = {q8, nullptr, hi, lo};
+    rc = launch_quantize(g, rows * cols, cols, 0, QBP_ROUND_STOCHASTIC, qp8, tensor_id8, qp16, tensor_id16, seed, o, st);
+    if (rc) return rc;
+    if (row_sums8) return launch_rowsum(q8, true, rows, cols, row_sums8, st);
+    return QBP_OK;
+}

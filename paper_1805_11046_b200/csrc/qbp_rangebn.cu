@@ -1,0 +1,419 @@
+// Range Batch-Normalization (Section 3, Eq. (range)) forward and backward
+// (Section 7: derivative of max/min is one where attained).
+//
+// Both directions are two streaming passes over [n x C] fp32 with the channel
+// innermost: a statistics pass (per-channel min, max, sum -- or sum dy,
+// sum dy*xhat) and an apply pass, with a one-warp-per-channel combine between
+// them.  Sums are carried in fp64 per thread (the fp64 pipe is far from being
+// the limit at HBM rate); everything an element's value depends on follows a
+// fixed fp32 operation order so that forward and backward agree on which
+// outputs the ReLU kept.
+#include "qbp_colscan.cuh"
+
+#include <cmath>
+
+namespace qbp {
+
+// xhat and y of one element; the order of operations is part of the contract.
+__device__ __forceinline__ float bn_xhat(float x, float mu, float s) { return __fmul_rn(__fsub_rn(x, mu), s); }
+__device__ __forceinline__ float bn_y(float xh, float g, float b) { return __fadd_rn(__fmul_rn(g, xh), b); }
+__device__ __forceinline__ float bn_scale(float lo, float hi, float Cn)
+{
+    float r = __fsub_rn(hi, lo);
+    return r > 0.0f ? __fdiv_rn(1.0f, __fmul_rn(Cn, r)) : 0.0f;
+}
+
+// ---------------------------------------------------------------- forward
+template <int VEC>
+__global__ void __launch_bounds__(kScanThreads) bn_stats_kernel(const float *__restrict__ x, int64_t rows, int C, int tw,
+                                                                float *__restrict__ part_lo, float *__restrict__ part_hi,
+                                                                double *__restrict__ part_sum)
+{
+    const ScanPos p = scan_pos<VEC>(C, tw);
+    const int rpb = kScanThreads / tw;
+    float lo[VEC], hi[VEC];
+    double sum[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { lo[e] = INFINITY; hi[e] = -INFINITY; sum[e] = 0.0; }
+    if (p.active) {
+        const int64_t step = (int64_t)gridDim.x * rpb;
+        for (int64_t r0 = (int64_t)blockIdx.x * rpb + p.ty; r0 < rows; r0 += step * kScanUnroll) {
+            VecF<VEC> v[kScanUnroll];
+            bool ok[kScanUnroll];
+#pragma unroll
+            for (int u = 0; u < kScanUnroll; ++u) {
+                int64_t r = r0 + u * step;
+                ok[u] = r < rows;
+                if (ok[u]) v[u].load(x + r * C + p.col);
+            }
+#pragma unroll
+            for (int u = 0; u < kScanUnroll; ++u)
+                if (ok[u]) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        lo[e] = fminf(lo[e], v[u].v[e]);
+                        hi[e] = fmaxf(hi[e], v[u].v[e]);
+                        sum[e] += (double)v[u].v[e];
+                    }
+                }
+        }
+    }
+    __shared__ float s_lo[kScanThreads * VEC], s_hi[kScanThreads * VEC];
+    __shared__ double s_sum[kScanThreads * VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        s_lo[threadIdx.x * VEC + e] = lo[e]; s_hi[threadIdx.x * VEC + e] = hi[e]; s_sum[threadIdx.x * VEC + e] = sum[e];
+    }
+    __syncthreads();
+    if (p.ty == 0 && p.active) {
+        for (int y = 1; y < rpb; ++y)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                const int i = (y * tw + p.tx) * VEC + e;
+                lo[e] = fminf(lo[e], s_lo[i]); hi[e] = fmaxf(hi[e], s_hi[i]); sum[e] += s_sum[i];
+            }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const int64_t i = (int64_t)blockIdx.x * C + p.col + e;
+            part_lo[i] = lo[e]; part_hi[i] = hi[e]; part_sum[i] = sum[e];
+        }
+    }
+}
+
+// One warp per channel: mean, min, max.
+__global__ void __launch_bounds__(256) bn_stats_finalize_kernel(const float *__restrict__ part_lo,
+                                                                const float *__restrict__ part_hi,
+                                                                const double *__restrict__ part_sum, int nparts, int C,
+                                                                int64_t n, float *__restrict__ mean,
+                                                                float *__restrict__ vmin, float *__restrict__ vmax)
+{
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c >= C) return;
+    float lo = INFINITY, hi = -INFINITY;
+    double sum = 0.0;
+    for (int i = threadIdx.x & 31; i < nparts; i += 32) {
+        lo = fminf(lo, part_lo[(int64_t)i * C + c]);
+        hi = fmaxf(hi, part_hi[(int64_t)i * C + c]);
+        sum += part_sum[(int64_t)i * C + c];
+    }
+    lo = warp_min(lo); hi = warp_max(hi);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if ((threadIdx.x & 31) == 0) { mean[c] = (float)(sum / (double)n); vmin[c] = lo; vmax[c] = hi; }
+}
+
+template <int VEC, bool RELU>
+__global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__restrict__ x, int64_t rows, int C, int tw,
+                                                                const float *__restrict__ mean,
+                                                                const float *__restrict__ vmin,
+                                                                const float *__restrict__ vmax,
+                                                                const float *__restrict__ gamma,
+                                                                const float *__restrict__ beta, float Cn,
+                                                                float *__restrict__ y)
+{
+    const ScanPos p = scan_pos<VEC>(C, tw);
+    if (!p.active) return;
+    const int rpb = kScanThreads / tw;
+    float mu[VEC], s[VEC], g[VEC], b[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        mu[e] = mean[p.col + e];
+        s[e] = bn_scale(vmin[p.col + e], vmax[p.col + e], Cn);
+        g[e] = gamma ? gamma[p.col + e] : 1.0f;
+        b[e] = beta ? beta[p.col + e] : 0.0f;
+    }
+    const int64_t step = (int64_t)gridDim.x * rpb;
+    for (int64_t r0 = (int64_t)blockIdx.x * rpb + p.ty; r0 < rows; r0 += step * kScanUnroll) {
+        VecF<VEC> v[kScanUnroll];
+        bool ok[kScanUnroll];
+#pragma unroll
+        for (int u = 0; u < kScanUnroll; ++u) {
+            int64_t r = r0 + u * step;
+            ok[u] = r < rows;
+            if (ok[u]) v[u].load(x + r * C + p.col);
+        }
+#pragma unroll
+        for (int u = 0; u < kScanUnroll; ++u)
+            if (ok[u]) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    float yv = bn_y(bn_xhat(v[u].v[e], mu[e], s[e]), g[e], b[e]);
+                    v[u].v[e] = RELU ? fmaxf(yv, 0.0f) : yv;
+                }
+                v[u].store(y + (r0 + u * step) * C + p.col);
+            }
+    }
+}
+
+// Exact range of y over the whole tensor from the per-channel statistics:
+// y is a non-decreasing (gamma >= 0) or non-increasing function of x computed
+// with the same rounded operations, so its extremes sit at x = min and x = max.
+__global__ void __launch_bounds__(256) bn_out_range_kernel(const float *__restrict__ mean, const float *__restrict__ vmin,
+                                                           const float *__restrict__ vmax,
+                                                           const float *__restrict__ gamma,
+                                                           const float *__restrict__ beta, int C, float Cn, int relu,
+                                                           qbp_qparams *__restrict__ out)
+{
+    float lo = INFINITY, hi = -INFINITY;
+    for (int c = threadIdx.x; c < C; c += 256) {
+        float s = bn_scale(vmin[c], vmax[c], Cn);
+        float g = gamma ? gamma[c] : 1.0f, b = beta ? beta[c] : 0.0f;
+        float a = bn_y(bn_xhat(vmin[c], mean[c], s), g, b);
+        float z = bn_y(bn_xhat(vmax[c], mean[c], s), g, b);
+        if (relu) { a = fmaxf(a, 0.0f); z = fmaxf(z, 0.0f); }
+        lo = fminf(lo, fminf(a, z)); hi = fmaxf(hi, fmaxf(a, z));
+    }
+    lo = warp_min(lo); hi = warp_max(hi);
+    __shared__ float s_lo[8], s_hi[8];
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 0; w < 8; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); }
+        out->scale = 0.0f; out->zero_point = 0; out->vmin = lo; out->vmax = hi;
+    }
+}
+
+// --------------------------------------------------------------- backward
+template <int VEC, bool RELU>
+__global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float *__restrict__ dy,
+                                                                    const float *__restrict__ x, int64_t rows, int C,
+                                                                    int tw, const float *__restrict__ mean,
+                                                                    const float *__restrict__ vmin,
+                                                                    const float *__restrict__ vmax,
+                                                                    const float *__restrict__ gamma,
+                                                                    const float *__restrict__ beta, float Cn,
+                                                                    double *__restrict__ part_dy,
+                                                                    double *__restrict__ part_dyx)
+{
+    const ScanPos p = scan_pos<VEC>(C, tw);
+    const int rpb = kScanThreads / tw;
+    double sdy[VEC], sdyx[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { sdy[e] = 0.0; sdyx[e] = 0.0; }
+    if (p.active) {
+        float mu[VEC], s[VEC], g[VEC], b[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            mu[e] = mean[p.col + e];
+            s[e] = bn_scale(vmin[p.col + e], vmax[p.col + e], Cn);
+            g[e] = gamma ? gamma[p.col + e] : 1.0f;
+            b[e] = beta ? beta[p.col + e] : 0.0f;
+        }
+        const int64_t step = (int64_t)gridDim.x * rpb;
+        for (int64_t r0 = (int64_t)blockIdx.x * rpb + p.ty; r0 < rows; r0 += step * kScanUnroll) {
+            VecF<VEC> vx[kScanUnroll], vd[kScanUnroll];
+            bool ok[kScanUnroll];
+#pragma unroll
+            for (int u = 0; u < kScanUnroll; ++u) {
+                int64_t r = r0 + u * step;
+                ok[u] = r < rows;
+                if (ok[u]) { vx[u].load(x + r * C + p.col); vd[u].load(dy + r * C + p.col); }
+            }
+#pragma unroll
+            for (int u = 0; u < kScanUnroll; ++u)
+                if (ok[u]) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        float xh = bn_xhat(vx[u].v[e], mu[e], s[e]);
+                        float d = vd[u].v[e];
+                        if (RELU && !(bn_y(xh, g[e], b[e]) > 0.0f)) d = 0.0f;
+                        sdy[e] += (double)d;
+                        sdyx[e] += (double)d * (double)xh;
+                    }
+                }
+        }
+    }
+    __shared__ double s_a[kScanThreads * VEC], s_b[kScanThreads * VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { s_a[threadIdx.x * VEC + e] = sdy[e]; s_b[threadIdx.x * VEC + e] = sdyx[e]; }
+    __syncthreads();
+    if (p.ty == 0 && p.active) {
+        for (int y = 1; y < rpb; ++y)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                sdy[e] += s_a[(y * tw + p.tx) * VEC + e];
+                sdyx[e] += s_b[(y * tw + p.tx) * VEC + e];
+            }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            part_dy[(int64_t)blockIdx.x * C + p.col + e] = sdy[e];
+            part_dyx[(int64_t)blockIdx.x * C + p.col + e] = sdyx[e];
+        }
+    }
+}
+
+// One warp per channel: dbeta, dgamma, and the two per-channel constants of dx:
+// m1 = gamma*dbeta/n, k2 = C(n)*gamma*dgamma.
+__global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const double *__restrict__ part_dy,
+                                                              const double *__restrict__ part_dyx, int nparts, int C,
+                                                              int64_t n, const float *__restrict__ gamma, double Cn,
+                                                              float *__restrict__ dgamma, float *__restrict__ dbeta,
+                                                              float2 *__restrict__ coef)
+{
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c >= C) return;
+    double a = 0.0, b = 0.0;
+    for (int i = threadIdx.x & 31; i < nparts; i += 32) {
+        a += part_dy[(int64_t)i * C + c];
+        b += part_dyx[(int64_t)i * C + c];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, o);
+        b += __shfl_xor_sync(0xffffffffu, b, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        const double g = gamma ? (double)gamma[c] : 1.0;
+        if (dbeta) dbeta[c] = (float)a;
+        if (dgamma) dgamma[c] = (float)b;
+        coef[c] = make_float2((float)(g * a / (double)n), (float)(Cn * g * b));
+    }
+}
+
+template <int VEC, bool RELU>
+__global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float *__restrict__ dy,
+                                                                    const float *__restrict__ x, int64_t rows, int C,
+                                                                    int tw, const float *__restrict__ mean,
+                                                                    const float *__restrict__ vmin,
+                                                                    const float *__restrict__ vmax,
+                                                                    const float *__restrict__ gamma,
+                                                                    const float *__restrict__ beta, float Cn,
+                                                                    const float2 *__restrict__ coef,
+                                                                    float *__restrict__ dx)
+{
+    const ScanPos p = scan_pos<VEC>(C, tw);
+    if (!p.active) return;
+    const int rpb = kScanThreads / tw;
+    float mu[VEC], s[VEC], g[VEC], b[VEC], lo[VEC], hi[VEC], m1[VEC], k2[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        mu[e] = mean[p.col + e];
+        lo[e] = vmin[p.col + e]; hi[e] = vmax[p.col + e];
+        s[e] = bn_scale(lo[e], hi[e], Cn);
+        g[e] = gamma ? gamma[p.col + e] : 1.0f;
+        b[e] = beta ? beta[p.col + e] : 0.0f;
+        float2 cf = coef[p.col + e];
+        m1[e] = cf.x; k2[e] = cf.y;
+    }
+    const int64_t step = (int64_t)gridDim.x * rpb;
+    for (int64_t r0 = (int64_t)blockIdx.x * rpb + p.ty; r0 < rows; r0 += step * kScanUnroll) {
+        VecF<VEC> vx[kScanUnroll], vd[kScanUnroll];
+        bool ok[kScanUnroll];
+#pragma unroll
+        for (int u = 0; u < kScanUnroll; ++u) {
+            int64_t r = r0 + u * step;
+            ok[u] = r < rows;
+            if (ok[u]) { vx[u].load(x + r * C + p.col); vd[u].load(dy + r * C + p.col); }
+        }
+#pragma unroll
+        for (int u = 0; u < kScanUnroll; ++u)
+            if (ok[u]) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    const float xv = vx[u].v[e];
+                    float d = vd[u].v[e];
+                    if (RELU && !(bn_y(bn_xhat(xv, mu[e], s[e]), g[e], b[e]) > 0.0f)) d = 0.0f;
+                    const float ind = (xv == hi[e] ? 1.0f : 0.0f) - (xv == lo[e] ? 1.0f : 0.0f);
+                    vd[u].v[e] = s[e] * (g[e] * d - m1[e] - k2[e] * ind);
+                }
+                vd[u].store(dx + (r0 + u * step) * C + p.col);
+            }
+    }
+}
+
+static size_t bn_ws_bytes(int64_t C)
+{
+    // forward: lo, hi (float) + sum (double) partials; backward: two double partials + coefficients
+    size_t per = (size_t)kScanMaxStrips * (size_t)C;
+    return 2 * align_up(per * sizeof(double), 256) + 2 * align_up(per * sizeof(float), 256) +
+           align_up((size_t)C * sizeof(float2), 256) + 256;
+}
+
+static int check_bn(const char *who, const void *a, const void *b, int64_t n, int64_t C, const void *ws, size_t ws_bytes)
+{
+    if (n < 2) return fail(QBP_ERR_INVALID_ARG, "%s: n must be at least 2 (C(1) is infinite)", who);
+    if (C <= 0) return fail(QBP_ERR_INVALID_ARG, "%s: C must be positive", who);
+    if (!a || !b) return fail(QBP_ERR_INVALID_ARG, "%s: NULL tensor", who);
+    if (!ws || ws_bytes < bn_ws_bytes(C))
+        return fail(QBP_ERR_WORKSPACE, "%s: workspace of %zu bytes needed, %zu given", who, bn_ws_bytes(C), ws_bytes);
+    return QBP_OK;
+}
+
+}  // namespace qbp
+
+using namespace qbp;
+
+extern "C" __attribute__((visibility("default"))) size_t qbp_rangebn_workspace_bytes(int64_t n, int64_t C)
+{
+    (void)n;
+    return bn_ws_bytes(C > 0 ? C : 1);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu,
+                               float *y, float *save_mean, float *save_min, float *save_max, qbp_qparams *out_range,
+                               void *ws, size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = check_bn("rangebn_fwd", x, y, n, C, ws, ws_bytes);
+    if (rc) return rc;
+    if (!save_mean || !save_min || !save_max) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: NULL statistics buffer");
+    WsCarver w(ws, ws_bytes);
+    double *psum = w.take<double>((size_t)kScanMaxStrips * C);
+    w.take<double>((size_t)kScanMaxStrips * C);
+    float *plo = w.take<float>((size_t)kScanMaxStrips * C);
+    float *phi = w.take<float>((size_t)kScanMaxStrips * C);
+    const bool al = aligned16(x) && aligned16(y);
+    const ScanGeom g = scan_geom(n, C, al);
+    const dim3 grid(g.nbx, g.slabs);
+    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
+    if (g.vec == 4) bn_stats_kernel<4><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
+    else            bn_stats_kernel<1><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
+    QBP_LAUNCH_OK("bn_stats_kernel");
+    bn_stats_finalize_kernel<<<(int)((C + 7) / 8), 256, 0, st>>>(plo, phi, psum, g.nbx, (int)C, n, save_mean, save_min, save_max);
+    QBP_LAUNCH_OK("bn_stats_finalize_kernel");
+#define QBP_BN_APPLY(V, R) bn_apply_kernel<V, R><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, y)
+    if (g.vec == 4) { if (relu) QBP_BN_APPLY(4, true); else QBP_BN_APPLY(4, false); }
+    else            { if (relu) QBP_BN_APPLY(1, true); else QBP_BN_APPLY(1, false); }
+#undef QBP_BN_APPLY
+    QBP_LAUNCH_OK("bn_apply_kernel");
+    if (out_range) {
+        bn_out_range_kernel<<<1, 256, 0, st>>>(save_mean, save_min, save_max, gamma, beta, (int)C, Cn, relu, out_range);
+        QBP_LAUNCH_OK("bn_out_range_kernel");
+    }
+    return QBP_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma,
+                               const float *beta, int relu, const float *save_mean, const float *save_min,
+                               const float *save_max, float *dx, float *dgamma, float *dbeta, void *ws,
+                               size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = check_bn("rangebn_bwd", x, dy, n, C, ws, ws_bytes);
+    if (rc) return rc;
+    if (!dx || !save_mean || !save_min || !save_max) return fail(QBP_ERR_INVALID_ARG, "rangebn_bwd: NULL tensor");
+    WsCarver w(ws, ws_bytes);
+    double *pa = w.take<double>((size_t)kScanMaxStrips * C);
+    double *pb = w.take<double>((size_t)kScanMaxStrips * C);
+    w.take<float>((size_t)kScanMaxStrips * C);
+    w.take<float>((size_t)kScanMaxStrips * C);
+    float2 *coef = w.take<float2>((size_t)C);
+    const bool al = aligned16(x) && aligned16(dy) && aligned16(dx);
+    const ScanGeom g = scan_geom(n, C, al);
+    const dim3 grid(g.nbx, g.slabs);
+    const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n));
+    const float Cn = (float)Cnd;
+#define QBP_BN_BSTATS(V, R) bn_bwd_stats_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, pa, pb)
+    if (g.vec == 4) { if (relu) QBP_BN_BSTATS(4, true); else QBP_BN_BSTATS(4, false); }
+    else            { if (relu) QBP_BN_BSTATS(1, true); else QBP_BN_BSTATS(1, false); }
+#undef QBP_BN_BSTATS
+    QBP_LAUNCH_OK("bn_bwd_stats_kernel");
+    bn_bwd_finalize_kernel<<<(int)((C + 7) / 8), 256, 0, st>>>(pa, pb, g.nbx, (int)C, n, gamma, Cnd, dgamma, dbeta, coef);
+    QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
+#define QBP_BN_BAPPLY(V, R) bn_bwd_apply_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx)
+    if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true); else QBP_BN_BAPPLY(4, false); }
+    else            { if (relu) QBP_BN_BAPPLY(1, true); else QBP_BN_BAPPLY(1, false); }
+#undef QBP_BN_BAPPLY
+    QBP_LAUNCH_OK("bn_bwd_apply_kernel");
+    return QBP_OK;
+}
