@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the 8-bit training hot path: one quantised conv layer + Range BN, forward and backward.
+
+A step is one pass of the whole path over one batch of synthetic input shaped like ResNet-18's conv2_x
+3x3 layer (batch 256, 56x56, 64 -> 64 channels): quantise x and w, int8 implicit-GEMM forward, Range BN
+(+ReLU); Range BN backward, gradient bifurcation (8-bit and 16-bit stochastic copies), int8 layer
+gradient, 16x8-bit weight gradient.  Everything runs in libqbp's CUDA kernels through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  N > 1: one process per GPU under torch.distributed.run; the batches are
+independent, so ranks share nothing on the data path (weak scaling, per-GPU batch statistics).
+--impl reference times the CPU oracle on the host cores instead (bounded sample per step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "QBP layer fwd+bwd int8 TOPS & Range BN GB/s vs B200 roofline; images/s"
+WORKLOAD = "resnet18_conv2x_3x3_layer_fwd_bwd"
+BATCH, HW, CIN, COUT = 256, 56, 64, 64
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
+# (captured at batch 32 and scaled by the elements processed: traffic of these streaming kernels grows in
+# proportion).  None: not captured.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {}
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Reads SM clock and throttle reasons every 25 ms while the GPU works (NVML, read-only)."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.025)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------- the workload
+def conv_workload(batch):
+    from paper_1805_11046_b200 import synth
+    return synth.conv3x3_layer(batch=batch, hw=HW, c_in=CIN, k_out=COUT)
+
+
+# Algorithmic HBM bytes per element of the [N,H,W,64] activation (or int8 ops) of each kernel of a step, in
+# launch order; E = batch*56*56*64 elements.  (name, bytes per element, ops per element)
+OPS_PER_ELEMENT_CONV = 2 * 9 * CIN          # 2*K per output element of fprop / dgrad
+STEP_KERNELS = [
+    ("range_partial_kernel", 4, 0), ("range_finalize_kernel", 0, 0), ("quantize_kernel", 5, 0),        # x
+    ("range_partial_kernel", 0, 0), ("range_finalize_kernel", 0, 0), ("quantize_kernel", 0, 0),        # w (tiny)
+    ("rowsum_kernel", 1, 0), ("conv_rowterm_kernel", 0, 0), ("rowsum_kernel", 0, 0), ("conv_colterm_kernel", 0, 0),
+    ("qbp_mma_kernel", 5, OPS_PER_ELEMENT_CONV),                                                        # fprop
+    ("bn_stats_kernel", 4, 0), ("bn_stats_finalize_kernel", 0, 0), ("bn_apply_kernel", 8, 0),
+    ("bn_bwd_stats_kernel", 8, 0), ("bn_bwd_finalize_kernel", 0, 0), ("bn_bwd_apply_kernel", 12, 0),
+    ("range_partial_kernel", 4, 0), ("range_finalize_kernel", 0, 0), ("quantize_kernel", 7, 0),        # bifurcate
+    ("rowsum_kernel", 1, 0), ("conv_rowterm_kernel", 0, 0), ("colsum_kernel", 0, 0), ("conv_colterm_kernel", 0, 0),
+    ("qbp_mma_kernel", 5, OPS_PER_ELEMENT_CONV),                                                        # dgrad
+    ("class_sums_kernel", 1, 0), ("class_sums_kernel", 1, 0), ("class_sums_kernel", 1, 0),
+    ("qbp_wgrad_kernel", 3, 2 * OPS_PER_ELEMENT_CONV),                                                  # wgrad: two int8 products
+    ("wgrad_finalize_kernel", 0, 0),
+]
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1805_11046_b200 import binding as B
+    from paper_1805_11046_b200 import layer
+    from paper_1805_11046_b200.dist import max_over_ranks, rank_info
+
+    rank, local_rank, world = rank_info()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+
+    cfg = conv_workload(args.batch)
+    host = {k: torch.from_numpy(cfg[k]).pin_memory() for k in ("x", "w", "dy")}
+    x, w, dy = (host[k].to(dev, non_blocking=True) for k in ("x", "w", "dy"))
+    c = cfg["conv"]
+    conv = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    L = layer.QuantizedLayer(conv=conv, relu=True, seed=cfg["seed"], tensor_id8=cfg["id8"], tensor_id16=cfg["id16"], device=dev)
+    E = x.numel()
+
+    def step():
+        L.forward(x, w)
+        L.backward(dy)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    assert L.status() == 0, "a device-side wait timed out"
+
+    # ---- device-resident throughput: exactly K steps between two events on the launching stream
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+    clocks = sampler.stop()
+    ms_step = ms_total / args.steps
+    value = world * args.batch / (ms_step * 1e-3)
+
+    # ---- end to end: inputs start in pinned host memory, the weight gradient is read back, every step
+    out_host = {k: torch.empty(t.shape, dtype=t.dtype).pin_memory() for k, t in
+                (("dw", L.dw), ("dgamma", L.dgamma), ("dbeta", L.dbeta))}
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step():
+        x.copy_(host["x"], non_blocking=True); w.copy_(host["w"], non_blocking=True); dy.copy_(host["dy"], non_blocking=True)
+        step()
+        out_host["dw"].copy_(L.dw, non_blocking=True); out_host["dgamma"].copy_(L.dgamma, non_blocking=True)
+        out_host["dbeta"].copy_(L.dbeta, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / e2e_steps
+    h2d = sum(host[k].numel() * host[k].element_size() for k in host)
+    d2h = sum(t.numel() * t.element_size() for t in out_host.values())
+
+    # ---- per-kernel device times (event pair around every launch), same launch configuration
+    trace_steps = max(3, min(args.steps, 10))
+    B.trace_enable(True)
+    for _ in range(trace_steps):
+        step()
+    recs = B.trace_records()
+    B.trace_enable(False)
+    per_step = len(recs) // trace_steps
+    launches_per_step = per_step
+    kernels = []
+    if per_step == len(STEP_KERNELS):
+        for i, (name, bpe, ope) in enumerate(STEP_KERNELS):
+            times = [recs[s * per_step + i][1] for s in range(trace_steps)]
+            assert all(recs[s * per_step + i][0] == name for s in range(trace_steps)), (i, name)
+            kernels.append({"kernel": name, "ms": sum(times) / len(times), "bytes": bpe * E, "ops": ope * E})
+    traced_ms = sum(k["ms"] for k in kernels) or 1.0
+    peaks, peaks_kind = measured_peaks()
+    hbm_peak = float(peaks["hbm_gbs"])
+    int8_peak_tops = 4500.0                 # nominal dense int8: 2 x nominal dense bf16
+    for k in kernels:
+        k["share"] = k["ms"] / traced_ms
+        k["gbs"] = k["bytes"] / (k["ms"] * 1e-3) / 1e9 if k["ms"] > 0 else 0.0
+        k["tops"] = k["ops"] / (k["ms"] * 1e-3) / 1e12 if k["ms"] > 0 else 0.0
+    roofline = None
+    if kernels:
+        top = max(kernels, key=lambda k: k["ms"])
+        tr = NCU_TRAFFIC_BYTES_PER_ELEMENT.get(top["kernel"])
+        roofline = {"kernel": top["kernel"], "bound": "hbm", "achieved": round(top["gbs"], 1), "peak": hbm_peak,
+                    "unit": "GB/s", "frac": round(top["gbs"] / hbm_peak, 4), "traffic": tr * E if tr else None,
+                    "peak_source": f"{peaks_kind} copy bandwidth", "ms_per_launch": round(top["ms"], 4),
+                    "share_of_step": round(top["share"], 4)}
+    mma_ops = sum(k["ops"] for k in kernels if k["ops"])
+    mma_ms = sum(k["ms"] for k in kernels if k["ops"])
+    bn_bytes = sum(k["bytes"] for k in kernels if k["kernel"].startswith("bn_"))
+    bn_ms = sum(k["ms"] for k in kernels if k["kernel"].startswith("bn_"))
+
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": "images/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "s8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": args.batch, "input": [args.batch, HW, HW, CIN],
+                   "filter": [COUT, 3, 3, CIN], "l2": "inputs (205 MB per activation tensor) larger than the 126 MB L2",
+                   "parallelism": f"dp{world} (independent batches, no data-path collective)"},
+        "clocks": clocks,
+        "e2e": {"value": round(world * args.batch / (e2e_ms * 1e-3), 1), "unit": "images/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4), "steps": e2e_steps},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline,
+        "int8_tops": round(mma_ops / (mma_ms * 1e-3) / 1e12, 1) if mma_ms else None,
+        "int8_tops_frac_of_nominal_4500": round(mma_ops / (mma_ms * 1e-3) / 1e12 / int8_peak_tops, 4) if mma_ms else None,
+        "rangebn_gbs": round(bn_bytes / (bn_ms * 1e-3) / 1e9, 1) if bn_ms else None,
+        "rangebn_frac_of_hbm": round(bn_bytes / (bn_ms * 1e-3) / 1e9 / hbm_peak, 4) if bn_ms else None,
+        "kernels": [{"kernel": k["kernel"], "ms": round(k["ms"], 4), "share": round(k["share"], 4),
+                     "gbs": round(k["gbs"], 1), "tops": round(k["tops"], 1)} for k in kernels if k["ms"] > 0.002],
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(args.cpu_sample_batch)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------- CPU oracle arm
+def oracle_step(cfg):
+    """The whole path once through the oracle, as it stands."""
+    from oracle import qbp_oracle as O
+    c = cfg["conv"]
+    d = O.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    y, saved, _ = O.layer_fwd(cfg["x"], cfg["w"], relu=True, conv=d)
+    g, dgamma, dbeta = O.rangebn_bwd(cfg["dy"], saved.z, saved.mean, saved.vmin, saved.vmax, relu=True)
+    dx, dw, *_ = O.layer_bwd_products(g.astype(np.float32), saved, cfg["seed"], cfg["id8"], cfg["id16"], conv=d)
+    return y, dx, dw
+
+
+def cpu_baseline(sample_batch):
+    from oracle import qbp_oracle as O
+    cfg = conv_workload(sample_batch)
+    O.lib()
+    t0 = time.perf_counter()
+    oracle_step(cfg)
+    dt = time.perf_counter() - t0
+    return {"value": round(sample_batch / dt, 3), "unit": "images/s", "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"one fwd+bwd of the same layer at batch {sample_batch} (of {BATCH}) on the host, {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import qbp_oracle as O
+    cfg = conv_workload(args.cpu_sample_batch)
+    O.lib()
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(cfg)
+    steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(cfg)
+    dt = (time.perf_counter() - t0) / steps
+    value = round(args.cpu_sample_batch / dt, 3)
+    sample = f"each step = one fwd+bwd of the layer at batch {args.cpu_sample_batch} (of {BATCH}); {steps} timed steps"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(dt * 1e3, 2), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "s8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": args.batch, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "images/s", "cores": O.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--batch", type=int, default=BATCH, help="images per GPU (the workload is quoted at 256)")
+    ap.add_argument("--cpu-sample-batch", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

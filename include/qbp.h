@@ -71,6 +71,16 @@ enum { QBP_CONV_FPROP = 0, QBP_CONV_DGRAD = 1 };
 /* Text of the last error raised on the calling thread ("" if none). */
 const char *qbp_last_error(void);
 
+/* Diagnostics (no counterpart in the paper).  While tracing is enabled every
+ * kernel the library launches is bracketed by a CUDA event pair on its stream
+ * (process-wide, one host thread at a time).  After synchronising the
+ * stream(s), qbp_trace_count() records can be read: kernel name and device
+ * time in milliseconds.  qbp_trace_enable(1) discards earlier records; (0)
+ * stops tracing and discards them. */
+int qbp_trace_enable(int on);
+int qbp_trace_count(void);
+int qbp_trace_read(int index, char *name, int name_cap, float *ms);
+
 /* ------------------------------------------------------------------------
  * Range quantiser -- Section 4 "Quantization methods" and Appendix B:
  *   scale = (vmax - vmin) / (2^M - 1), zero-point = round(-vmin / scale),
@@ -210,14 +220,20 @@ typedef struct {
     uint32_t tensor_id8, tensor_id16;
 } qbp_layer_desc;
 
-/* Caller-owned buffers that carry the forward's results to the backward.
- * Element counts: x_codes = |x|, w_codes = |w|, z = rows*channels (the fp32
- * output of the product, input of Range BN), rows = batch or N*P*Q. */
+/* Caller-owned buffers: what the forward leaves for the backward, and the
+ * backward's own intermediates (kept visible so that each stage can be
+ * checked on its own).  Element counts: x_codes = |x|, w_codes = |w|; z, g,
+ * g8, g_hi, g_lo = rows*channels of the product's output (rows = batch or
+ * N*P*Q); z is the fp32 output of the product (the input of Range BN), g the
+ * fp32 gradient arriving at it.  The g* members are used by the backward only. */
 typedef struct {
     int8_t *x_codes;  qbp_qparams *qx;
     int8_t *w_codes;  qbp_qparams *qw;
     float  *z;
     float  *save_mean, *save_min, *save_max;
+    float  *g;
+    int8_t *g8;       qbp_qparams *qg8;
+    int8_t *g_hi;     uint8_t *g_lo;   qbp_qparams *qg16;
 } qbp_layer_ctx;
 
 size_t qbp_layer_workspace_bytes(const qbp_layer_desc *L);

@@ -22,7 +22,7 @@ QBP_CONV_FPROP, QBP_CONV_DGRAD = 0, 1
 QBP_ERR_TIMEOUT = -6
 
 EXPORTS = (
-    "qbp_last_error",
+    "qbp_last_error", "qbp_trace_enable", "qbp_trace_count", "qbp_trace_read",
     "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s16", "qbp_bifurcate",
     "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8",
     "qbp_conv_s8_workspace_bytes", "qbp_conv_s8_implicit",
@@ -50,7 +50,9 @@ class LayerDesc(C.Structure):
 
 class LayerCtx(C.Structure):
     _fields_ = [("x_codes", C.c_void_p), ("qx", C.c_void_p), ("w_codes", C.c_void_p), ("qw", C.c_void_p),
-                ("z", C.c_void_p), ("save_mean", C.c_void_p), ("save_min", C.c_void_p), ("save_max", C.c_void_p)]
+                ("z", C.c_void_p), ("save_mean", C.c_void_p), ("save_min", C.c_void_p), ("save_max", C.c_void_p),
+                ("g", C.c_void_p), ("g8", C.c_void_p), ("qg8", C.c_void_p), ("g_hi", C.c_void_p), ("g_lo", C.c_void_p),
+                ("qg16", C.c_void_p)]
 
 
 def _load() -> C.CDLL:
@@ -244,3 +246,36 @@ def qbp_rangebn_bwd(dy, x, mean, vmin, vmax, gamma=None, beta=None, relu=False, 
                                _ptr(mean), _ptr(vmin), _ptr(vmax), _ptr(dx), _ptr(dgamma), _ptr(dbeta), _ptr(ws),
                                C.c_size_t(ws.numel()), _stream()))
     return dx, dgamma, dbeta
+
+
+# ---------------------------------------------------------------------- layer
+def qbp_layer_workspace_bytes(L: LayerDesc) -> int:
+    return int(lib.qbp_layer_workspace_bytes(C.byref(L)))
+
+
+def qbp_layer_fwd(L: LayerDesc, x, w, gamma, beta, y, ctx: LayerCtx, ws):
+    _check(lib.qbp_layer_fwd(C.byref(L), _ptr(x), _ptr(w), _ptr(gamma), _ptr(beta), _ptr(y), C.byref(ctx), _ptr(ws),
+                             C.c_size_t(ws.numel()), _stream()))
+    return y
+
+
+def qbp_layer_bwd(L: LayerDesc, ctx: LayerCtx, dy, gamma, beta, dx, dw, dgamma, dbeta, ws):
+    _check(lib.qbp_layer_bwd(C.byref(L), C.byref(ctx), _ptr(dy), _ptr(gamma), _ptr(beta), _ptr(dx), _ptr(dw),
+                             _ptr(dgamma), _ptr(dbeta), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return dx, dw, dgamma, dbeta
+
+
+# ---------------------------------------------------------------- diagnostics
+def trace_enable(on: bool) -> None:
+    _check(lib.qbp_trace_enable(int(on)))
+
+
+def trace_records():
+    """[(kernel name, device milliseconds)] of every launch since trace_enable(True); synchronises first."""
+    torch.cuda.synchronize()
+    out = []
+    name = C.create_string_buffer(64); ms = C.c_float()
+    for i in range(lib.qbp_trace_count()):
+        _check(lib.qbp_trace_read(i, name, 64, C.byref(ms)))
+        out.append((name.value.decode(), float(ms.value)))
+    return out

@@ -24,8 +24,15 @@ int fail(int status, const char *fmt, ...);    // sets the message, returns stat
             return ::qbp::fail(QBP_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
     } while (0)
 
+// Optional per-kernel timing (qbp_trace_enable): an event pair around every launch.
+void trace_begin(cudaStream_t st);
+void trace_end(const char *name, cudaStream_t st);
+#define QBP_TRACE_BEGIN(st) ::qbp::trace_begin(st)
+
+// Placed after every kernel launch; expects the stream in a variable named `st`.
 #define QBP_LAUNCH_OK(name)                                                       \
     do {                                                                          \
+        ::qbp::trace_end(name, st);                                               \
         cudaError_t e_ = cudaGetLastError();                                      \
         if (e_ != cudaSuccess)                                                    \
             return ::qbp::fail(QBP_ERR_CUDA, "launch of %s: %s", name, cudaGetErrorString(e_)); \

@@ -56,14 +56,6 @@ static size_t step_scratch_bytes(const qbp_layer_desc *L, const LayerShape &s)
     return align_up(b, 256);
 }
 
-// Backward temporaries: fp32 gradient at the product's output, its three code
-// tensors, two parameter records.
-static size_t bwd_temp_bytes(const LayerShape &s)
-{
-    const size_t g = (size_t)s.rows * s.cout;
-    return align_up(g * sizeof(float), 256) + 3 * align_up(g, 256) + 2 * 256;
-}
-
 }  // namespace qbp
 
 using namespace qbp;
@@ -72,7 +64,7 @@ extern "C" __attribute__((visibility("default"))) size_t qbp_layer_workspace_byt
 {
     LayerShape s;
     if (layer_shape(L, s)) return 0;
-    return step_scratch_bytes(L, s) + bwd_temp_bytes(s);
+    return step_scratch_bytes(L, s);
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_layer_desc *L, const float *x,
@@ -125,15 +117,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
         return fail(QBP_ERR_WORKSPACE, "layer_bwd: workspace of %zu bytes needed, %zu given",
                     qbp_layer_workspace_bytes(L), ws_bytes);
+    if (!saved->g || !saved->g8 || !saved->qg8 || !saved->g_hi || !saved->g_lo || !saved->qg16)
+        return fail(QBP_ERR_INVALID_ARG, "layer_bwd: the saved-state record has a NULL gradient buffer");
     const size_t scratch = step_scratch_bytes(L, s);
-    WsCarver c(static_cast<char *>(ws) + scratch, ws_bytes - scratch);
-    const size_t gcount = (size_t)s.rows * s.cout;
-    float *g = c.take<float>(gcount);
-    int8_t *g8 = c.take<int8_t>(gcount);
-    int8_t *ghi = c.take<int8_t>(gcount);
-    uint8_t *glo = c.take<uint8_t>(gcount);
-    qbp_qparams *qp8 = c.take<qbp_qparams>(1);
-    qbp_qparams *qp16 = c.take<qbp_qparams>(1);
+    float *g = saved->g;
+    int8_t *g8 = saved->g8, *ghi = saved->g_hi;
+    uint8_t *glo = saved->g_lo;
+    qbp_qparams *qp8 = saved->qg8, *qp16 = saved->qg16;
 
     rc = qbp_rangebn_bwd(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
                          saved->save_max, g, dgamma, dbeta, ws, scratch, stream);

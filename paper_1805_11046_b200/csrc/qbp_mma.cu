@@ -399,6 +399,7 @@ static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
         configured = 220 * 1024;
     }
     QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
+    QBP_TRACE_BEGIN(st);
     qbp_mma_kernel<<<tiles_m * P.tiles_n, kMmaThreads, smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_mma_kernel");
     return QBP_OK;
@@ -480,6 +481,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     else        rc = launch_colsum(B, K, N, tmp_n, st);
     if (rc) return rc;
     const int64_t mx = std::max(M, N);
+    QBP_TRACE_BEGIN(st);
     gemm_terms_kernel<<<(int)((mx + 255) / 256), 256, 0, st>>>(
         transA ? nullptr : (const int32_t *)tmp_m, transA ? (const long long *)tmp_m : nullptr,
         transB ? (const int32_t *)tmp_n : nullptr, transB ? nullptr : (const long long *)tmp_n, M, N, K, qa, qb,
@@ -557,11 +559,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
 
     int rc = launch_rowsum(in, true, pix, Cred, chan_sum, st);
     if (rc) return rc;
+    QBP_TRACE_BEGIN(st);
     conv_rowterm_kernel<<<(int)((pix + 255) / 256), 256, 0, st>>>(chan_sum, d->N, d->H, d->W, d->pad, Cred, q_in, q_w, rowterm);
     QBP_LAUNCH_OK("conv_rowterm_kernel");
     if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
     else        rc = launch_colsum(wgt, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
     if (rc) return rc;
+    QBP_TRACE_BEGIN(st);
     conv_colterm_kernel<<<dim3((Nout + 127) / 128, 16), 128, 0, st>>>(
         dgrad ? nullptr : (const int32_t *)wsum, dgrad ? (const long long *)wsum : nullptr, Nout, d->R, d->S, d->pad,
         dgrad ? 1 : 0, q_in, colterm);

@@ -8,6 +8,7 @@
 #include "qbp_colscan.cuh"
 
 #include <cstring>
+#include <vector>
 
 namespace qbp {
 
@@ -39,6 +40,33 @@ int sm_count()
         cached_dev = dev;
     }
     return cached;
+}
+
+// ------------------------------------------------------------ launch tracing
+struct TraceRec { const char *name; cudaEvent_t a, b; };
+static bool g_trace_on = false;
+static std::vector<TraceRec> g_trace;
+static std::vector<cudaEvent_t> g_event_pool;
+
+static cudaEvent_t pool_event()
+{
+    if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+void trace_begin(cudaStream_t st)
+{
+    if (!g_trace_on) return;
+    TraceRec r{nullptr, pool_event(), pool_event()};
+    cudaEventRecord(r.a, st);
+    g_trace.push_back(r);
+}
+void trace_end(const char *name, cudaStream_t st)
+{
+    if (!g_trace_on || g_trace.empty() || g_trace.back().name) return;
+    g_trace.back().name = name;
+    cudaEventRecord(g_trace.back().b, st);
 }
 
 constexpr int kThreads = 256;
@@ -386,10 +414,12 @@ static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams
         const int64_t per_block = (int64_t)kThreads * kUnroll * (vec ? 4 : 1);
         nparts = grid_for(1, (n + per_block - 1) / per_block);
         if (nparts > kMaxParts) nparts = kMaxParts;
+        QBP_TRACE_BEGIN(st);
         if (vec) range_partial_kernel<4><<<nparts, kThreads, 0, st>>>(x, n, partials);
         else     range_partial_kernel<1><<<nparts, kThreads, 0, st>>>(x, n, partials);
         QBP_LAUNCH_OK("range_partial_kernel");
     }
+    QBP_TRACE_BEGIN(st);
     range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
     QBP_LAUNCH_OK("range_finalize_kernel");
     return QBP_OK;
@@ -403,10 +433,12 @@ static int launch_chan_range(const float *x, int64_t rows, int64_t cols, int bit
     if (rows > 0) {
         nparts = g.nbx;
         dim3 grid(g.nbx, g.slabs);
+        QBP_TRACE_BEGIN(st);
         if (g.vec == 4) chan_range_partial_kernel<4><<<grid, kScanThreads, 0, st>>>(x, rows, (int)cols, g.tw, part_lo, part_hi);
         else            chan_range_partial_kernel<1><<<grid, kScanThreads, 0, st>>>(x, rows, (int)cols, g.tw, part_lo, part_hi);
         QBP_LAUNCH_OK("chan_range_partial_kernel");
     }
+    QBP_TRACE_BEGIN(st);
     chan_range_finalize_kernel<<<(int)((cols + 7) / 8), kThreads, 0, st>>>(part_lo, part_hi, nparts, (int)cols, bits, qp);
     QBP_LAUNCH_OK("chan_range_finalize_kernel");
     return QBP_OK;
@@ -424,6 +456,7 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
     const int grid = grid_for(1, (n + per_block - 1) / per_block);
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     const int c = (int)cols;
+    QBP_TRACE_BEGIN(st);
     if (rounding == QBP_ROUND_STOCHASTIC) {
         if (vec) quantize_kernel<true, 4><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
         else     quantize_kernel<true, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
@@ -444,6 +477,7 @@ int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int
     int G = 1; while (G < 32 && G < cols / 16) G <<= 1;
     const int64_t groups = kThreads / G;
     const int grid = grid_for(1, (rows + groups - 1) / groups);
+    QBP_TRACE_BEGIN(st);
     if (is_signed) rowsum_kernel<true><<<grid, kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, G, sums);
     else           rowsum_kernel<false><<<grid, kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, G, sums);
     QBP_LAUNCH_OK("rowsum_kernel");
@@ -462,6 +496,7 @@ int launch_colsum(const int8_t *q, int64_t rows, int64_t cols, int64_t *sums, cu
     int64_t min_blocks = (rows >> 23) + 1;
     int64_t grid = grid_for(1, (rows + rpb - 1) / rpb) / slabs;
     if (grid < min_blocks) grid = min_blocks;
+    QBP_TRACE_BEGIN(st);
     colsum_kernel<<<dim3((unsigned)grid, (unsigned)slabs), kThreads, 0, st>>>(q, rows, (int)cols, (unsigned long long *)sums);
     QBP_LAUNCH_OK("colsum_kernel");
     return QBP_OK;
@@ -497,6 +532,7 @@ static int quantize_any(int bits, const float *x, int64_t rows, int64_t cols, in
     const int perch = granularity == QBP_PER_CHANNEL;
     if (range_in) {
         const int count = perch ? (int)cols : 1;
+        QBP_TRACE_BEGIN(st);
         qparams_from_range_kernel<<<(count + 255) / 256, 256, 0, st>>>(range_in, count, bits, qp_out);
         QBP_LAUNCH_OK("qparams_from_range_kernel");
     } else {
@@ -522,6 +558,27 @@ static int quantize_any(int bits, const float *x, int64_t rows, int64_t cols, in
 using namespace qbp;
 
 extern "C" __attribute__((visibility("default"))) const char *qbp_last_error(void) { return g_err; }
+
+extern "C" __attribute__((visibility("default"))) int qbp_trace_enable(int on)
+{
+    for (TraceRec &r : g_trace) { g_event_pool.push_back(r.a); g_event_pool.push_back(r.b); }
+    g_trace.clear();
+    g_trace_on = on != 0;
+    return QBP_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_trace_count(void) { return (int)g_trace.size(); }
+
+extern "C" __attribute__((visibility("default"))) int qbp_trace_read(int index, char *name, int name_cap, float *ms)
+{
+    if (index < 0 || index >= (int)g_trace.size() || !name || name_cap <= 0 || !ms)
+        return fail(QBP_ERR_INVALID_ARG, "trace_read: bad index or NULL output");
+    const TraceRec &r = g_trace[index];
+    if (!r.name) return fail(QBP_ERR_INVALID_ARG, "trace_read: record %d was never closed", index);
+    snprintf(name, (size_t)name_cap, "%s", r.name);
+    QBP_CUDA_OK(cudaEventElapsedTime(ms, r.a, r.b));
+    return QBP_OK;
+}
 
 extern "C" __attribute__((visibility("default"))) size_t qbp_quantize_workspace_bytes(int64_t rows, int64_t cols, int granularity)
 {

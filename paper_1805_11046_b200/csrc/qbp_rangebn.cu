@@ -366,17 +366,21 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd(const floa
     const ScanGeom g = scan_geom(n, C, al);
     const dim3 grid(g.nbx, g.slabs);
     const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
+    QBP_TRACE_BEGIN(st);
     if (g.vec == 4) bn_stats_kernel<4><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
     else            bn_stats_kernel<1><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
     QBP_LAUNCH_OK("bn_stats_kernel");
+    QBP_TRACE_BEGIN(st);
     bn_stats_finalize_kernel<<<(int)((C + 7) / 8), 256, 0, st>>>(plo, phi, psum, g.nbx, (int)C, n, save_mean, save_min, save_max);
     QBP_LAUNCH_OK("bn_stats_finalize_kernel");
+QBP_TRACE_BEGIN(st);
 #define QBP_BN_APPLY(V, R) bn_apply_kernel<V, R><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, y)
     if (g.vec == 4) { if (relu) QBP_BN_APPLY(4, true); else QBP_BN_APPLY(4, false); }
     else            { if (relu) QBP_BN_APPLY(1, true); else QBP_BN_APPLY(1, false); }
 #undef QBP_BN_APPLY
     QBP_LAUNCH_OK("bn_apply_kernel");
     if (out_range) {
+        QBP_TRACE_BEGIN(st);
         bn_out_range_kernel<<<1, 256, 0, st>>>(save_mean, save_min, save_max, gamma, beta, (int)C, Cn, relu, out_range);
         QBP_LAUNCH_OK("bn_out_range_kernel");
     }
@@ -403,13 +407,16 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const floa
     const dim3 grid(g.nbx, g.slabs);
     const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n));
     const float Cn = (float)Cnd;
+QBP_TRACE_BEGIN(st);
 #define QBP_BN_BSTATS(V, R) bn_bwd_stats_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, pa, pb)
     if (g.vec == 4) { if (relu) QBP_BN_BSTATS(4, true); else QBP_BN_BSTATS(4, false); }
     else            { if (relu) QBP_BN_BSTATS(1, true); else QBP_BN_BSTATS(1, false); }
 #undef QBP_BN_BSTATS
     QBP_LAUNCH_OK("bn_bwd_stats_kernel");
+    QBP_TRACE_BEGIN(st);
     bn_bwd_finalize_kernel<<<(int)((C + 7) / 8), 256, 0, st>>>(pa, pb, g.nbx, (int)C, n, gamma, Cnd, dgamma, dbeta, coef);
     QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
+QBP_TRACE_BEGIN(st);
 #define QBP_BN_BAPPLY(V, R) bn_bwd_apply_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx)
     if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true); else QBP_BN_BAPPLY(4, false); }
     else            { if (relu) QBP_BN_BAPPLY(1, true); else QBP_BN_BAPPLY(1, false); }

@@ -205,11 +205,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
 // ------------------------------------------------------------ code sums
 // Sums of stored codes per channel and per border class of the pixel the code
 // sits at (bit 1: first row, 2: last row, 4: first column, 8: last column);
-// a plain matrix is passed as H = W = 1 and keeps every row in class 0.
+// a plain matrix (plain = 1) keeps every row in class 0.
 // sums[cls][c] (int64, zeroed beforehand).
 template <bool IS_SIGNED>
 __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restrict__ q, int64_t pixels, int H, int W,
-                                                         int C, unsigned long long *__restrict__ sums)
+                                                         int C, int plain, unsigned long long *__restrict__ sums)
 {
     extern __shared__ int s_acc[];                       // [16][C]
     for (int i = threadIdx.x; i < 16 * C; i += 256) s_acc[i] = 0;
@@ -225,8 +225,8 @@ __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restri
             for (int e = 0; e < 16; ++e) interior[e] = 0;
             for (int64_t p = (int64_t)blockIdx.x * rpb + ty; p < pixels; p += (int64_t)gridDim.x * rpb) {
                 const int w = (int)(p % W), h = (int)((p / W) % H);
-                // a plain matrix (H = W = 1) keeps everything in class 0
-                const int cls = (H == 1 && W == 1) ? 0
+                // a plain matrix keeps everything in class 0
+                const int cls = plain ? 0
                               : (h == 0 ? 1 : 0) | (h == H - 1 ? 2 : 0) | (w == 0 ? 4 : 0) | (w == W - 1 ? 8 : 0);
                 uint4 v = __ldg(reinterpret_cast<const uint4 *>(q + p * C) + g);
                 const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
@@ -324,7 +324,7 @@ static size_t wgrad_ws_bytes(const qbp_conv_desc *d, int64_t N, int64_t K)
 }
 
 template <bool IS_SIGNED>
-static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C, int64_t *sums, cudaStream_t st)
+static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C, bool plain, int64_t *sums, cudaStream_t st)
 {
     QBP_CUDA_OK(cudaMemsetAsync(sums, 0, sizeof(int64_t) * 16 * C, st));
     if ((size_t)C * 16 * sizeof(int) > 200 * 1024) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad: more than 3200 channels");
@@ -338,7 +338,8 @@ static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C,
     const int cv = C / 16, tw = cv < 256 ? cv : 256, rpb = 256 / tw;
     int64_t grid = std::min<int64_t>((pixels + rpb - 1) / rpb, (int64_t)sm_count() * 4);
     grid = std::max<int64_t>(grid, pixels / (1 << 22) + 1);
-    class_sums_kernel<IS_SIGNED><<<(unsigned)grid, 256, smem, st>>>((const uint8_t *)q, pixels, H, W, C, (unsigned long long *)sums);
+    QBP_TRACE_BEGIN(st);
+    class_sums_kernel<IS_SIGNED><<<(unsigned)grid, 256, smem, st>>>((const uint8_t *)q, pixels, H, W, C, plain ? 1 : 0, (unsigned long long *)sums);
     QBP_LAUNCH_OK("class_sums_kernel");
     return QBP_OK;
 }
@@ -387,11 +388,11 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
     int64_t *slo = w.take<int64_t>(16 * N);
 
     const int Hc = d ? d->H : 1, Wc = d ? d->W : 1;
-    int rc = launch_class_sums<true>(x, M, Hc, Wc, (int)K, sx, st);
+    int rc = launch_class_sums<true>(x, M, Hc, Wc, (int)K, d == nullptr, sx, st);
     if (rc) return rc;
-    rc = launch_class_sums<true>(g_hi, M, Hc, Wc, (int)N, shi, st);
+    rc = launch_class_sums<true>(g_hi, M, Hc, Wc, (int)N, d == nullptr, shi, st);
     if (rc) return rc;
-    rc = launch_class_sums<false>(g_lo, M, Hc, Wc, (int)N, slo, st);
+    rc = launch_class_sums<false>(g_lo, M, Hc, Wc, (int)N, d == nullptr, slo, st);
     if (rc) return rc;
     QBP_CUDA_OK(cudaMemsetAsync(raw, 0, sizeof(int64_t) * outs, st));
     QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
@@ -454,10 +455,12 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
         QBP_CUDA_OK(cudaFuncSetAttribute(qbp_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         configured = true;
     }
+    QBP_TRACE_BEGIN(st);
     qbp_wgrad_kernel<<<P.slices * out_tiles, kWgThreads, smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_wgrad_kernel");
 
     const int blocks = (int)((outs + 255) / 256);
+    QBP_TRACE_BEGIN(st);
     wgrad_finalize_kernel<<<blocks, 256, 0, st>>>((const long long *)raw, (const long long *)sx, (const long long *)shi,
                                                   (const long long *)slo, P.conv, outs, M, N, K, d ? d->N : 0, Hc, Wc,
                                                   d ? d->pad : 0, d ? d->R : 1, d ? d->S : 1, d ? d->C : (int)K, qx, qg16,

@@ -1,0 +1,61 @@
+"""Device-memory bookkeeping for one quantised layer: owns the buffers that
+qbp_layer_fwd / qbp_layer_bwd need (codes, parameters, saved statistics,
+gradient copies, workspace) as torch tensors and passes their addresses
+through the C ABI.  No arithmetic happens here."""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class QuantizedLayer:
+    """conv: a binding.ConvDesc for a convolution layer (x NHWC, w KRSC), or None for a linear
+    layer y = x w with x [batch, in_features], w [in_features, out_features]."""
+
+    def __init__(self, conv=None, batch=0, in_features=0, out_features=0, relu=False, seed=0,
+                 tensor_id8=1, tensor_id16=2, device="cuda"):
+        self.device = torch.device(device)
+        d = B.LayerDesc()
+        if conv is not None:
+            d.conv = conv
+            self.rows, self.cin, self.cout = conv.N * conv.H * conv.W, conv.C, conv.K
+            self.x_shape = (conv.N, conv.H, conv.W, conv.C)
+            self.w_shape = (conv.K, conv.R, conv.S, conv.C)
+            self.z_shape = (conv.N, conv.H, conv.W, conv.K)
+        else:
+            d.batch, d.in_features, d.out_features = batch, in_features, out_features
+            self.rows, self.cin, self.cout = batch, in_features, out_features
+            self.x_shape, self.w_shape, self.z_shape = (batch, in_features), (in_features, out_features), (batch, out_features)
+        d.relu, d.seed, d.tensor_id8, d.tensor_id16 = int(relu), seed, tensor_id8, tensor_id16
+        self.desc = d
+        dev = self.device
+        e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+        self.x_codes, self.w_codes = e(self.x_shape, torch.int8), e(self.w_shape, torch.int8)
+        self.qx, self.qw, self.qg8, self.qg16 = (B.new_qparams(1, dev) for _ in range(4))
+        self.z, self.g = e(self.z_shape, torch.float32), e(self.z_shape, torch.float32)
+        self.save_mean, self.save_min, self.save_max = (e((self.cout,), torch.float32) for _ in range(3))
+        self.g8, self.ghi, self.glo = e(self.z_shape, torch.int8), e(self.z_shape, torch.int8), e(self.z_shape, torch.uint8)
+        self.y = e(self.z_shape, torch.float32)
+        self.dx, self.dw = e(self.x_shape, torch.float32), e(self.w_shape, torch.float32)
+        self.dgamma, self.dbeta = e((self.cout,), torch.float32), e((self.cout,), torch.float32)
+        self.ws = torch.empty(max(B.qbp_layer_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)
+        c = B.LayerCtx()
+        for name, t in (("x_codes", self.x_codes), ("qx", self.qx), ("w_codes", self.w_codes), ("qw", self.qw),
+                        ("z", self.z), ("save_mean", self.save_mean), ("save_min", self.save_min),
+                        ("save_max", self.save_max), ("g", self.g), ("g8", self.g8), ("qg8", self.qg8),
+                        ("g_hi", self.ghi), ("g_lo", self.glo), ("qg16", self.qg16)):
+            setattr(c, name, t.data_ptr())
+        self.ctx = c
+        self.gamma = self.beta = None
+
+    def forward(self, x, w, gamma=None, beta=None):
+        self.gamma, self.beta = gamma, beta
+        return B.qbp_layer_fwd(self.desc, x, w, gamma, beta, self.y, self.ctx, self.ws)
+
+    def backward(self, dy):
+        return B.qbp_layer_bwd(self.desc, self.ctx, dy, self.gamma, self.beta, self.dx, self.dw, self.dgamma,
+                               self.dbeta, self.ws)
+
+    def status(self) -> int:
+        return B.status_word(self.ws)

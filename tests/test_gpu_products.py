@@ -1,0 +1,128 @@
+"""GPU integer products (tcgen05 int8 GEMM, implicit-GEMM convolution, limb-split weight gradient)
+vs the CPU oracle: int32 / int64 accumulators bit for bit, fp32 outputs identical (same single multiply)."""
+import numpy as np
+import pytest
+
+from oracle import qbp_oracle as O
+from paper_1805_11046_b200 import synth
+from tests.util import random_codes, set_qparams, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import paper_1805_11046_b200.binding as binding
+    return binding
+
+
+def _qp(B, scale, zp):
+    return set_qparams(B.new_qparams(1), scale, zp)
+
+
+# ------------------------------------------------------------------ GEMM
+GEMMS = [(128, 128, 128), (64, 128, 256), (64, 256, 128), (16, 16, 16), (208, 80, 144), (256, 384, 512),
+         (384, 640, 1040), (128, 272, 33024)]
+
+
+@pytest.mark.parametrize("M,N,K", GEMMS)
+@pytest.mark.parametrize("tA,tB", [(False, False), (False, True), (True, False), (True, True)])
+def test_gemm_s8(B, M, N, K, tA, tB):
+    A = random_codes((K, M) if tA else (M, K), 1); Bm = random_codes((N, K) if tB else (K, N), 2)
+    za, zb, sa, sb = 3, -128, 0.5, 0.25
+    if K > 30000:                       # keep the exact sum inside int32: small codes at the longest legal K
+        A = (A // 4).astype(np.int8); Bm = (Bm // 4).astype(np.int8); zb = -5
+    acc, out, ws = B.qbp_gemm_s8(to_dev(A), _qp(B, sa, za), to_dev(Bm), _qp(B, sb, zb), transA=tA, transB=tB, want_acc=True)
+    oacc, oout, bad = O.gemm_s8(A, za, Bm, zb, sa, sb, transA=tA, transB=tB)
+    assert bad == 0 and B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc)
+    assert np.array_equal(to_host(out), oout)
+
+
+def test_gemm_extreme_codes_and_zero_points(B):
+    M, N, K = 128, 128, 33024 // 2
+    A = np.full((M, K), -128, np.int8); Bm = np.full((K, N), 127, np.int8)
+    acc, _, ws = B.qbp_gemm_s8(to_dev(A), _qp(B, 1, 127), to_dev(Bm), _qp(B, 1, -128), want_acc=True, want_out=False)
+    assert B.status_word(ws) == 0
+    assert np.all(to_host(acc) == (-255) * 255 * K)
+
+
+def test_gemm_dense_sweep_shape_sampled_rows(B):
+    """4096^3 from the dense sweep, operands quantised from N(0,1); oracle on 192 sampled rows."""
+    case = synth.dense_gemm(4096, 4096, 4096)
+    qa, qpa = B.qbp_quantize_s8(to_dev(case["a"])); qb, qpb = B.qbp_quantize_s8(to_dev(case["b"]))
+    oa = O.quantize(case["a"], 8); ob = O.quantize(case["b"], 8)
+    assert np.array_equal(to_host(qa), oa.q) and np.array_equal(to_host(qb), ob.q)
+    acc, out, ws = B.qbp_gemm_s8(qa, qpa, qb, qpb, want_acc=True)
+    assert B.status_word(ws) == 0
+    rows = np.unique(np.concatenate([[0, 127, 128, 4095, 3968], np.random.Generator(np.random.PCG64(5)).integers(0, 4096, 187)]))
+    oacc, oout, bad = O.gemm_s8(oa.q[rows], oa.zero_point[0], ob.q, ob.zero_point[0], oa.scale[0], ob.scale[0])
+    assert bad == 0
+    assert np.array_equal(to_host(acc)[rows], oacc) and np.array_equal(to_host(out)[rows], oout)
+
+
+# ----------------------------------------------------------- convolution
+CONVS = [(2, 8, 8, 64, 64, 1), (2, 8, 8, 64, 64, 3), (3, 10, 12, 32, 48, 3), (2, 14, 14, 128, 256, 3),
+         (4, 7, 7, 256, 128, 1), (1, 1, 1, 16, 16, 3), (5, 9, 3, 80, 16, 3), (3, 28, 28, 128, 128, 3),
+         (2, 56, 56, 64, 64, 3), (1, 5, 130, 16, 272, 3)]
+
+
+@pytest.mark.parametrize("N,H,W,C,K,R", CONVS)
+@pytest.mark.parametrize("mode", [0, 1])
+def test_conv_s8(B, N, H, W, C, K, R, mode):
+    pad = (R - 1) // 2
+    d = B.conv_desc(N, H, W, C, K, R, R, 1, pad); od = O.conv_desc(N, H, W, C, K, R, R, 1, pad)
+    inp = random_codes((N, H, W, C if mode == 0 else K), 3); w = random_codes((K, R, R, C), 4)
+    zi, zw = 7, -128
+    acc, out, ws = B.qbp_conv_s8_implicit(mode, d, to_dev(inp), _qp(B, 0.5, zi), to_dev(w), _qp(B, 0.25, zw), want_acc=True)
+    oacc, oout, bad = O.conv_s8(mode, od, inp, zi, w, zw, 0.5, 0.25)
+    assert bad == 0 and B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc)
+    assert np.array_equal(to_host(out), oout)
+
+
+# --------------------------------------------------------- weight gradient
+def _g16(shape, seed):
+    return random_codes(shape, seed, -32768, 32767, np.int16)
+
+
+WGRADS = [(128, 128, 128), (64, 128, 256), (1000, 64, 64), (70000, 32, 48), (4096, 256, 384), (130, 16, 16)]
+
+
+@pytest.mark.parametrize("M,N,K", WGRADS)
+def test_wgrad_plain(B, M, N, K):
+    X = random_codes((M, K), 5); G = _g16((M, N), 6)
+    hi, lo = O.limb_split(G)
+    zx, zg = -128, 32767
+    acc, dW, ws = B.qbp_wgrad_s16(to_dev(X), _qp(B, 0.5, zx), to_dev(hi), to_dev(lo), _qp(B, 0.25, zg), want_acc=True)
+    oacc, oout = O.gemm_s16s8(X, zx, G, zg, 0.5, 0.25)
+    assert B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(dW), oout)
+
+
+def test_wgrad_long_reduction_extreme_codes(B):
+    """131072 rows of extreme codes: each CTA's int32 chunk stays in range, the int64 total is exact."""
+    M, N, K = 131072, 32, 32
+    X = np.full((M, K), -128, np.int8); G = np.full((M, N), 32767, np.int16)
+    G[::2] = -32768
+    hi, lo = O.limb_split(G)
+    acc, _, ws = B.qbp_wgrad_s16(to_dev(X), _qp(B, 1, 127), to_dev(hi), to_dev(lo), _qp(B, 1, 0), want_acc=True, want_out=False)
+    assert B.status_word(ws) == 0
+    assert np.all(to_host(acc) == (-255) * (32767 - 32768) * (M // 2))
+
+
+WCONVS = [(2, 8, 8, 64, 64, 1), (2, 8, 8, 64, 64, 3), (3, 10, 12, 32, 96, 3), (2, 14, 14, 128, 256, 3),
+          (4, 7, 7, 256, 128, 1), (1, 1, 1, 32, 32, 3), (2, 28, 28, 128, 128, 3), (3, 9, 5, 96, 160, 3)]
+
+
+@pytest.mark.parametrize("N,H,W,C,K,R", WCONVS)
+def test_wgrad_conv(B, N, H, W, C, K, R):
+    pad = (R - 1) // 2
+    d = B.conv_desc(N, H, W, C, K, R, R, 1, pad); od = O.conv_desc(N, H, W, C, K, R, R, 1, pad)
+    X = random_codes((N, H, W, C), 7); G = _g16((N, H, W, K), 8)
+    hi, lo = O.limb_split(G)
+    zx, zg = 5, -300
+    acc, dW, ws = B.qbp_wgrad_s16(to_dev(X), _qp(B, 0.5, zx), to_dev(hi), to_dev(lo), _qp(B, 0.25, zg), d=d, want_acc=True)
+    oacc, oout = O.conv_wgrad_s16(od, X, zx, G, zg, 0.5, 0.25)
+    assert B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(dW), oout)
