@@ -29,9 +29,21 @@ struct ScanGeom {
 
 inline int pow2ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
-// nbx is chosen so that all strips are resident at once (8 blocks of 256
-// threads per SM) and no strip is empty.
-inline ScanGeom scan_geom(int64_t rows, int64_t C, bool aligned)
+// Resident blocks per SM of a kernel at `threads` threads and no dynamic shared memory.
+template <typename Kernel>
+inline int blocks_per_sm(Kernel kernel, int threads)
+{
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, 0) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        n = 1;
+    }
+    return n;
+}
+
+// nbx is chosen so that all strips are resident at once (a single wave: `bps`
+// blocks per SM, the occupancy of the kernel that will run) and no strip is empty.
+inline ScanGeom scan_geom(int64_t rows, int64_t C, bool aligned, int bps)
 {
     ScanGeom g;
     g.vec = (aligned && C % 4 == 0) ? 4 : 1;
@@ -40,7 +52,7 @@ inline ScanGeom scan_geom(int64_t rows, int64_t C, bool aligned)
     g.rpb = kScanThreads / g.tw;
     g.slabs = (g.cv + g.tw - 1) / g.tw;
     int64_t steps = (rows + g.rpb - 1) / g.rpb;
-    int64_t want = (int64_t)sm_count() * 8 / g.slabs;
+    int64_t want = (int64_t)sm_count() * bps / g.slabs;
     if (want < 1) want = 1;
     if (want > kScanMaxStrips) want = kScanMaxStrips;
     g.nbx = (int)(steps < want ? (steps > 0 ? steps : 1) : want);

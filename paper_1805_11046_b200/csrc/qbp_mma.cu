@@ -121,8 +121,9 @@ uint32_t make_idesc(bool a_signed, bool b_signed, uint32_t a_major, uint32_t b_m
 
 // ================================================================== the kernel
 enum { MODE_GEMM = 0, MODE_FPROP = 1, MODE_DGRAD = 2 };
-constexpr int kMaxStages = 10;
+constexpr int kMaxStages = 16;
 constexpr int kMmaThreads = 192;
+constexpr int kGroupM = 16;          // GEMM raster: tiles walk down kGroupM rows before moving one column right
 
 struct MmaParams {
     CUtensorMap mapA, mapB;
@@ -130,52 +131,77 @@ struct MmaParams {
     uint32_t idesc;
     int mode;
     int stages, k_iters, mma_per_iter, bn, tmem_cols;
-    int tiles_n;
+    int ips;                      // k iterations (operand tiles) per pipeline stage
+    int b_resident;               // conv: all filter tiles of the CTA's N tile stay in shared memory
+    uint32_t b_res_bytes;         // bytes reserved for them at the start of shared memory
+    int tiles_m, tiles_n, tiles_total;
     // output
     int64_t M, N;                 // rows / columns of the output matrix
     int32_t *acc_out; float *out;
-    const int32_t *rowterm;       // [M]
+    const int32_t *rowterm;       // GEMM: [M]
+    const int32_t *chan_sum;      // conv: per input pixel, the sum of its codes over the reduced channels
     const int32_t *colterm;       // [classes][N]
     const qbp_qparams *qa, *qb;
     int *status;
-    // gemm: element offsets per k iteration handled via kblock
-    int kblock;                   // reduction elements per k iteration
+    int kblock;                   // GEMM: reduction elements per k iteration
     // conv geometry (output pixel grid == input pixel grid: stride 1, same padding)
     int H, W, Nimg, pad, S, cchunks, chunk_bytes, Cred;
     int bw_log2, bh_log2, tiles_w, tiles_h;
 };
 
-__device__ __forceinline__ void raise_timeout(int *status) { atomicExch(status, (int)QBP_ERR_TIMEOUT); }
+struct TileOrigin { int m0, n0, img0, h0, w0; };
 
-__global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_constant__ MmaParams P)
+__device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
 {
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_bar;
-    __shared__ uint32_t tmem_slot;
-
-    const uint32_t raw_addr = smem_u32(smem_raw);
-    uint8_t *smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
-    const uint32_t stage_bytes = P.a.tile_bytes + P.b.tile_bytes;
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile_n = blockIdx.x % P.tiles_n;
-    const int tile_m = blockIdx.x / P.tiles_n;
-    const int n0 = tile_n * P.bn;
-
-    // tile origin: matrix row for a GEMM, (image, row, column) for a convolution
-    int m0 = tile_m * 128, img0 = 0, h0 = 0, w0 = 0;
+    TileOrigin o;
+    int tile_m, tile_n;
+    if (P.mode == MODE_GEMM) {
+        // groups of kGroupM tile rows; inside a group the row index moves fastest, so that the CTAs
+        // running at one time share few A row-blocks and few B column-blocks (L2 reuse)
+        const int per_group = kGroupM * P.tiles_n;
+        const int g = tile / per_group, r = tile % per_group;
+        const int rows_here = min(kGroupM, P.tiles_m - g * kGroupM);
+        tile_m = g * kGroupM + r % rows_here;
+        tile_n = r / rows_here;
+    } else {
+        tile_n = tile % P.tiles_n;
+        tile_m = tile / P.tiles_n;
+    }
+    o.n0 = tile_n * P.bn;
+    o.m0 = tile_m * 128; o.img0 = 0; o.h0 = 0; o.w0 = 0;
     if (P.mode != MODE_GEMM) {
         const int tw = tile_m % P.tiles_w;
         const int th = (tile_m / P.tiles_w) % P.tiles_h;
         const int tn = tile_m / (P.tiles_w * P.tiles_h);
-        w0 = tw << P.bw_log2;
-        h0 = th << P.bh_log2;
-        img0 = tn * (128 >> (P.bw_log2 + P.bh_log2));
+        o.w0 = tw << P.bw_log2;
+        o.h0 = th << P.bh_log2;
+        o.img0 = tn * (128 >> (P.bw_log2 + P.bh_log2));
     }
+    return o;
+}
+
+__device__ __forceinline__ void raise_timeout(int *status) { atomicExch(status, (int)QBP_ERR_TIMEOUT); }
+
+// Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The producer runs ahead of
+// the MMA warp across tile boundaries through the shared-memory ring; the accumulator is double
+// buffered in tensor memory so that the epilogue of tile i overlaps the MMAs of tile i + 1.
+__global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_constant__ MmaParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], b_full;
+    __shared__ uint32_t tmem_slot;
+
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    uint8_t *smem_b = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);     // resident filter tiles (if any)
+    uint8_t *smem = smem_b + P.b_res_bytes;                                  // the stage ring
+    const uint32_t a_stage = P.a.tile_bytes * (uint32_t)P.ips;
+    const uint32_t stage_bytes = a_stage + (P.b_resident ? 0u : P.b.tile_bytes * (uint32_t)P.ips);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        mbar_init(&acc_bar, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        mbar_init(&b_full, 1);
         mbar_fence_init();
         tma_prefetch_desc(&P.mapA);
         tma_prefetch_desc(&P.mapB);
@@ -190,96 +216,170 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
     if (warp == 0) {
         if (lane == 0) {
             // ------------------------------------------------ TMA producer
-            for (int it = 0; it < P.k_iters; ++it) {
-                const int s = it % P.stages;
-                const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
-                if (!mbar_wait(&empty_bar[s], ph ^ 1u)) { timed_out = true; break; }
-                uint8_t *sa = smem + (size_t)s * stage_bytes;
-                uint8_t *sb = sa + P.a.tile_bytes;
-                mbar_expect_tx(&full_bar[s], stage_bytes);
-                if (P.mode == MODE_GEMM) {
-                    const int k0 = it * P.kblock;
-                    if (P.a.major == 0) tma_load_2d(sa, &P.mapA, &full_bar[s], k0, m0);
-                    else                tma_load_2d(sa, &P.mapA, &full_bar[s], m0, k0);
-                    if (P.b.major == 0) tma_load_2d(sb, &P.mapB, &full_bar[s], k0, n0);
-                    else                tma_load_2d(sb, &P.mapB, &full_bar[s], n0, k0);
-                } else {
-                    const int tap = it / P.cchunks, cc = it % P.cchunks;
-                    const int r = tap / P.S, t = tap % P.S;
-                    const int c0 = cc * P.chunk_bytes;
-                    if (P.mode == MODE_FPROP) {
-                        // input pixel of output (p,q) under tap (r,t): (p - pad + r, q - pad + t)
-                        tma_load_4d(sa, &P.mapA, &full_bar[s], c0, w0 - P.pad + t, h0 - P.pad + r, img0);
-                        // filter as [K rows x (R*S*C) columns]: this tap's channel chunk, K-major
-                        tma_load_2d(sb, &P.mapB, &full_bar[s], tap * P.Cred + c0, n0);
-                    } else {
-                        // gradient pixel feeding input (h,w) under tap (r,t): (h + pad - r, w + pad - t)
-                        tma_load_4d(sa, &P.mapA, &full_bar[s], c0, w0 + P.pad - t, h0 + P.pad - r, img0);
-                        // filter rows = output channels (the reduction), columns = this tap's input channels
-                        tma_load_2d(sb, &P.mapB, &full_bar[s], tap * (int)P.N + n0, c0);
+            if (P.b_resident) {
+                // the filter is the same for every tile of this CTA: fetch it once
+                const int n0 = 0;
+                mbar_expect_tx(&b_full, P.b.tile_bytes * (uint32_t)P.k_iters);
+                int it = 0;
+                for (int tap = 0; tap < P.k_iters / P.cchunks; ++tap)
+                    for (int cc = 0; cc < P.cchunks; ++cc, ++it) {
+                        uint8_t *dst = smem_b + (size_t)it * P.b.tile_bytes;
+                        const int c0 = cc * P.chunk_bytes;
+                        if (P.mode == MODE_FPROP) tma_load_2d(dst, &P.mapB, &b_full, tap * P.Cred + c0, n0);
+                        else                      tma_load_2d(dst, &P.mapB, &b_full, tap * (int)P.N + n0, c0);
                     }
+            }
+            uint32_t gs = 0;                                    // ring position, continues across tiles
+            for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
+                const TileOrigin o = tile_origin(P, tile);
+                if (P.mode == MODE_GEMM) {
+                    for (int it = 0; it < P.k_iters; ++it, ++gs) {
+                        const uint32_t s = gs % (uint32_t)P.stages;
+                        if (!mbar_wait(&empty_bar[s], ((gs / (uint32_t)P.stages) & 1u) ^ 1u)) { timed_out = true; break; }
+                        uint8_t *sa = smem + (size_t)s * stage_bytes;
+                        uint8_t *sb = sa + a_stage;
+                        mbar_expect_tx(&full_bar[s], stage_bytes);
+                        const int k0 = it * P.kblock;
+                        if (P.a.major == 0) tma_load_2d(sa, &P.mapA, &full_bar[s], k0, o.m0);
+                        else                tma_load_2d(sa, &P.mapA, &full_bar[s], o.m0, k0);
+                        if (P.b.major == 0) tma_load_2d(sb, &P.mapB, &full_bar[s], k0, o.n0);
+                        else                tma_load_2d(sb, &P.mapB, &full_bar[s], o.n0, k0);
+                    }
+                    continue;
                 }
+                // convolution: one activation tile per (tap, channel chunk), `ips` of them per stage
+                int j = 0, tap = 0;
+                uint32_t s = 0;
+                uint8_t *sa = nullptr;
+                const int R = P.k_iters / (P.cchunks * P.S);
+                for (int r = 0; r < R && !timed_out; ++r)
+                    for (int t = 0; t < P.S && !timed_out; ++t, ++tap)
+                        for (int cc = 0; cc < P.cchunks; ++cc) {
+                            if (j == 0) {
+                                s = gs % (uint32_t)P.stages;
+                                if (!mbar_wait(&empty_bar[s], ((gs / (uint32_t)P.stages) & 1u) ^ 1u)) { timed_out = true; break; }
+                                sa = smem + (size_t)s * stage_bytes;
+                                mbar_expect_tx(&full_bar[s], stage_bytes);
+                            }
+                            const int c0 = cc * P.chunk_bytes;
+                            uint8_t *da = sa + (size_t)j * P.a.tile_bytes;
+                            uint8_t *db = sa + a_stage + (size_t)j * P.b.tile_bytes;
+                            if (P.mode == MODE_FPROP) {
+                                // input pixel of output (p,q) under tap (r,t): (p - pad + r, q - pad + t)
+                                tma_load_4d(da, &P.mapA, &full_bar[s], c0, o.w0 - P.pad + t, o.h0 - P.pad + r, o.img0);
+                                // filter as [K rows x (R*S*C) columns]: this tap's channel chunk, K-major
+                                if (!P.b_resident) tma_load_2d(db, &P.mapB, &full_bar[s], tap * P.Cred + c0, o.n0);
+                            } else {
+                                // gradient pixel feeding input (h,w) under tap (r,t): (h + pad - r, w + pad - t)
+                                tma_load_4d(da, &P.mapA, &full_bar[s], c0, o.w0 + P.pad - t, o.h0 + P.pad - r, o.img0);
+                                // filter rows = output channels (the reduction), columns = this tap's input channels
+                                if (!P.b_resident) tma_load_2d(db, &P.mapB, &full_bar[s], tap * (int)P.N + o.n0, c0);
+                            }
+                            if (++j == P.ips) { j = 0; ++gs; }
+                        }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
             // -------------------------------------------------- MMA issuer
-            for (int it = 0; it < P.k_iters; ++it) {
-                const int s = it % P.stages;
-                const uint32_t ph = (uint32_t)(it / P.stages) & 1u;
-                if (!mbar_wait(&full_bar[s], ph)) { timed_out = true; break; }
+            if (P.b_resident && !mbar_wait(&b_full, 0)) timed_out = true;
+            const uint32_t bres_addr = smem_u32(smem_b);
+            const int groups = P.k_iters / P.ips;
+            uint32_t gs = 0, lt = 0;
+            for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x, ++lt) {
+                const uint32_t buf = lt & 1u;
+                if (!mbar_wait(&acc_empty[buf], ((lt >> 1) & 1u) ^ 1u)) { timed_out = true; break; }
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint32_t b_addr = a_addr + P.a.tile_bytes;
-                const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.a.desc_lo;
-                const uint32_t b_lo = ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
-                for (int kk = 0; kk < P.mma_per_iter; ++kk) {
-                    const uint64_t da = ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep);
-                    const uint64_t db = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(b_lo + kk * P.b.kstep);
-                    mma_i8(tmem_base, da, db, P.idesc, (it | kk) != 0 ? 1u : 0u);
+                const uint32_t d_tmem = tmem_base + buf * (uint32_t)P.bn;
+                int it = 0;
+                for (int g = 0; g < groups; ++g, ++gs) {
+                    const uint32_t s = gs % (uint32_t)P.stages;
+                    if (!mbar_wait(&full_bar[s], (gs / (uint32_t)P.stages) & 1u)) { timed_out = true; break; }
+                    tc_fence_after();
+                    const uint32_t stage_addr = smem_u32(smem + (size_t)s * stage_bytes);
+                    for (int j = 0; j < P.ips; ++j, ++it) {
+                        const uint32_t a_addr = stage_addr + (uint32_t)j * P.a.tile_bytes;
+                        const uint32_t b_addr = P.b_resident ? bres_addr + (uint32_t)it * P.b.tile_bytes
+                                                             : stage_addr + a_stage + (uint32_t)j * P.b.tile_bytes;
+                        const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.a.desc_lo;
+                        const uint32_t b_lo = ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
+                        for (int kk = 0; kk < P.mma_per_iter; ++kk) {
+                            const uint64_t da = ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep);
+                            const uint64_t db = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(b_lo + kk * P.b.kstep);
+                            mma_i8(d_tmem, da, db, P.idesc, (it | kk) != 0 ? 1u : 0u);
+                        }
+                    }
+                    mma_commit(&empty_bar[s]);
                 }
-                mma_commit(&empty_bar[s]);
+                if (!timed_out) mma_commit(&acc_full[buf]);
             }
-            if (!timed_out) mma_commit(&acc_bar);
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------- epilogue
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
-        if (!mbar_wait(&acc_bar, 0)) timed_out = true;
-        tc_fence_after();
-        if (!timed_out) {
-            int64_t m; bool valid; int cls = 0;
+        const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
+        const int za = P.qa->zero_point, zb = P.qb->zero_point;
+        uint32_t lt = 0;
+        for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x, ++lt) {
+            const TileOrigin o = tile_origin(P, tile);
+            const uint32_t buf = lt & 1u;
+            // this row's output position and zero-point row term (independent of the accumulator)
+            int64_t m; bool valid; int cls = 0, rterm = 0;
             if (P.mode == MODE_GEMM) {
-                m = (int64_t)m0 + row;
+                m = (int64_t)o.m0 + row;
                 valid = m < P.M;
+                if (valid) rterm = __ldg(P.rowterm + m);
             } else {
                 const int dw = row & ((1 << P.bw_log2) - 1);
                 const int dh = (row >> P.bw_log2) & ((1 << P.bh_log2) - 1);
                 const int dn = row >> (P.bw_log2 + P.bh_log2);
-                const int n = img0 + dn, p = h0 + dh, q = w0 + dw;
+                const int n = o.img0 + dn, p = o.h0 + dh, q = o.w0 + dw;
                 valid = n < P.Nimg && p < P.H && q < P.W;
                 m = ((int64_t)n * P.H + p) * P.W + q;
                 cls = (p == 0 ? 1 : 0) | (p == P.H - 1 ? 2 : 0) | (q == 0 ? 4 : 0) | (q == P.W - 1 ? 8 : 0);
+                if (valid) {
+                    // sum of the input's channel sums over the taps inside the image, and their count
+                    // (pad is 0 or 1: nine predicated loads, issued together)
+                    int box = 0, taps = 0;
+                    const int32_t *cs = P.chan_sum + ((int64_t)n * P.H + p) * P.W + q;
+#pragma unroll
+                    for (int eh = -1; eh <= 1; ++eh)
+#pragma unroll
+                        for (int ew = -1; ew <= 1; ++ew) {
+                            const bool in = eh >= -P.pad && eh <= P.pad && ew >= -P.pad && ew <= P.pad &&
+                                            p + eh >= 0 && p + eh < P.H && q + ew >= 0 && q + ew < P.W;
+                            box += in ? __ldg(cs + eh * P.W + ew) : 0;
+                            taps += in ? 1 : 0;
+                        }
+                    rterm = -zb * box + taps * P.Cred * za * zb;
+                }
             }
-            const int rterm = valid ? P.rowterm[m] : 0;
             const int32_t *cterm = P.colterm + (int64_t)cls * P.N;
-            const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
+            if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1u)) { timed_out = true; break; }
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * (uint32_t)P.bn;
             for (int c0 = 0; c0 < P.bn; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, r);
+                tmem_ld_32x32(t_addr + (uint32_t)c0, r);
                 tmem_ld_wait();
+                if (c0 + 32 >= P.bn) {
+                    // the accumulator has been read out: hand the buffer back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                }
                 if (!valid) continue;
-                const int64_t ncol = P.N - (n0 + c0);                 // columns left in the matrix
+                const int64_t ncol = P.N - (o.n0 + c0);                 // columns left in the matrix
                 if (ncol <= 0) continue;
                 const int lim = ncol < 32 ? (int)ncol : 32;
                 int acc[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j] = j < lim ? (int)r[j] + rterm + __ldg(cterm + n0 + c0 + j) : 0;
+                for (int j = 0; j < 32; ++j) acc[j] = j < lim ? (int)r[j] + rterm + __ldg(cterm + o.n0 + c0 + j) : 0;
                 if (P.acc_out) {
-                    int32_t *dst = P.acc_out + m * P.N + n0 + c0;
+                    int32_t *dst = P.acc_out + m * P.N + o.n0 + c0;
                     if (lim == 32) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
@@ -289,7 +389,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                     }
                 }
                 if (P.out) {
-                    float *dst = P.out + m * P.N + n0 + c0;
+                    float *dst = P.out + m * P.N + o.n0 + c0;
                     if (lim == 32) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
@@ -332,30 +432,6 @@ __global__ void gemm_terms_kernel(const int32_t *ra32, const long long *ra64, co
     }
 }
 
-// Convolution, per output pixel: the sum of the input's channel sums over the
-// taps that fall inside the image, and how many taps those are.
-//   rowterm[m] = -zw * box[m] + taps_in(m) * Cred * z_in * zw
-__global__ void conv_rowterm_kernel(const int32_t *__restrict__ chan_sum, int Nimg, int H, int W, int pad, int Cred,
-                                    const qbp_qparams *q_in, const qbp_qparams *q_w, int32_t *__restrict__ rowterm)
-{
-    const int64_t m = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (m >= (int64_t)Nimg * H * W) return;
-    const int q = (int)(m % W), p = (int)((m / W) % H);
-    const int64_t img = m / ((int64_t)W * H);
-    int box = 0, taps = 0;
-    for (int dh = -pad; dh <= pad; ++dh) {
-        const int h = p + dh;
-        if (h < 0 || h >= H) continue;
-        for (int dw = -pad; dw <= pad; ++dw) {
-            const int w = q + dw;
-            if (w < 0 || w >= W) continue;
-            box += chan_sum[(img * H + h) * W + w];
-            ++taps;
-        }
-    }
-    rowterm[m] = -q_w->zero_point * box + taps * Cred * q_in->zero_point * q_w->zero_point;
-}
-
 // colterm[cls][n] = -z_in * sum over the taps valid for border class cls of the
 // filter's code sum for that tap and output column n.  cls bits: 1 first row,
 // 2 last row, 4 first column, 8 last column.  wsum32: [n][tap] (forward: sums over
@@ -385,22 +461,36 @@ __global__ void conv_colterm_kernel(const int32_t *wsum32, const long long *wsum
 // ================================================================== launchers
 static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
 {
-    const uint32_t stage_bytes = P.a.tile_bytes + P.b.tile_bytes;
-    int stages = (int)((200u * 1024u) / stage_bytes);
+    const uint32_t budget = 200u * 1024u;
+    P.ips = 1; P.b_resident = 0; P.b_res_bytes = 0;
+    if (P.mode != MODE_GEMM) {
+        // keep the whole filter in shared memory when it fits beside at least three activation stages
+        const uint32_t b_all = P.b.tile_bytes * (uint32_t)P.k_iters;
+        if (P.tiles_n == 1 && b_all + 3 * P.a.tile_bytes <= budget) { P.b_resident = 1; P.b_res_bytes = (uint32_t)align_up(b_all, 1024); }
+        // several small activation tiles share one stage (fewer barrier round trips)
+        const uint32_t per_iter = P.a.tile_bytes + (P.b_resident ? 0u : P.b.tile_bytes);
+        for (int c = 1; c <= P.k_iters; ++c)
+            if (P.k_iters % c == 0 && (uint32_t)c * per_iter <= 32u * 1024u) P.ips = c;
+    }
+    const uint32_t stage_bytes = (uint32_t)P.ips * (P.a.tile_bytes + (P.b_resident ? 0u : P.b.tile_bytes));
+    int stages = (int)((budget - P.b_res_bytes) / stage_bytes);
     stages = std::max(2, std::min(stages, kMaxStages));
-    stages = std::min(stages, std::max(2, P.k_iters));
     P.stages = stages;
-    int cols = 32; while (cols < P.bn) cols <<= 1;
+    int cols = 32; while (cols < 2 * P.bn) cols <<= 1;       // two accumulator buffers
     P.tmem_cols = cols;
-    const size_t smem = (size_t)stages * stage_bytes + 1024;
-    static thread_local size_t configured = 0;
-    if (smem > configured) {
+    P.tiles_m = tiles_m;
+    P.tiles_total = tiles_m * P.tiles_n;
+    const size_t smem = (size_t)P.b_res_bytes + (size_t)stages * stage_bytes + 1024;
+    static thread_local bool configured = false;
+    if (!configured) {
         QBP_CUDA_OK(cudaFuncSetAttribute(qbp_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        configured = 220 * 1024;
+        configured = true;
     }
     QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
+    // one CTA per SM (its shared-memory ring fills the SM), each walking its share of the tiles
+    const int grid = std::min(P.tiles_total, sm_count());
     QBP_TRACE_BEGIN(st);
-    qbp_mma_kernel<<<tiles_m * P.tiles_n, kMmaThreads, smem, st>>>(P);
+    qbp_mma_kernel<<<grid, kMmaThreads, smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_mma_kernel");
     return QBP_OK;
 }
@@ -552,16 +642,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
 
     WsCarver w(ws, ws_bytes);
     int *status = w.take<int>(1);
-    int32_t *rowterm = w.take<int32_t>(pix);
+    w.take<int32_t>(pix);
     int32_t *chan_sum = w.take<int32_t>(pix);
     int32_t *colterm = w.take<int32_t>(16 * nmax);
     int64_t *wsum = w.take<int64_t>((int64_t)taps * nmax);
 
     int rc = launch_rowsum(in, true, pix, Cred, chan_sum, st);
     if (rc) return rc;
-    QBP_TRACE_BEGIN(st);
-    conv_rowterm_kernel<<<(int)((pix + 255) / 256), 256, 0, st>>>(chan_sum, d->N, d->H, d->W, d->pad, Cred, q_in, q_w, rowterm);
-    QBP_LAUNCH_OK("conv_rowterm_kernel");
     if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
     else        rc = launch_colsum(wgt, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
     if (rc) return rc;
@@ -603,6 +690,6 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
     P.tiles_n = (Nout + P.bn - 1) / P.bn;
     P.M = pix; P.N = Nout;
     P.acc_out = acc_out; P.out = out;
-    P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
+    P.rowterm = nullptr; P.chan_sum = chan_sum; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
     return launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st);
 }

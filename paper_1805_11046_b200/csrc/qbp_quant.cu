@@ -397,10 +397,10 @@ __global__ void __launch_bounds__(kThreads) colsum_kernel(const int8_t *__restri
 }
 
 // ----------------------------------------------------------------- launchers
-static int grid_for(int64_t work_items_per_thread_group, int64_t n_groups)
+// One wave: `bps` resident blocks per SM (the kernel's occupancy), never more blocks than work groups.
+static int grid_for(int bps, int64_t n_groups)
 {
-    (void)work_items_per_thread_group;
-    int64_t want = (int64_t)sm_count() * 8;
+    int64_t want = (int64_t)sm_count() * bps;
     int64_t g = n_groups < want ? n_groups : want;
     return (int)(g < 1 ? 1 : g);
 }
@@ -412,7 +412,8 @@ static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams
     if (n > 0) {
         const bool vec = aligned16(x);
         const int64_t per_block = (int64_t)kThreads * kUnroll * (vec ? 4 : 1);
-        nparts = grid_for(1, (n + per_block - 1) / per_block);
+        nparts = grid_for(vec ? blocks_per_sm(range_partial_kernel<4>, kThreads) : blocks_per_sm(range_partial_kernel<1>, kThreads),
+                          (n + per_block - 1) / per_block);
         if (nparts > kMaxParts) nparts = kMaxParts;
         QBP_TRACE_BEGIN(st);
         if (vec) range_partial_kernel<4><<<nparts, kThreads, 0, st>>>(x, n, partials);
@@ -428,7 +429,9 @@ static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams
 static int launch_chan_range(const float *x, int64_t rows, int64_t cols, int bits, float *part_lo, float *part_hi,
                              qbp_qparams *qp, cudaStream_t st)
 {
-    ScanGeom g = scan_geom(rows, cols, aligned16(x));
+    const bool v4 = aligned16(x) && cols % 4 == 0;
+    ScanGeom g = scan_geom(rows, cols, aligned16(x), v4 ? blocks_per_sm(chan_range_partial_kernel<4>, kScanThreads)
+                                                        : blocks_per_sm(chan_range_partial_kernel<1>, kScanThreads));
     int nparts = 0;
     if (rows > 0) {
         nparts = g.nbx;
@@ -453,7 +456,10 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
                      (!o.q8 || ((uintptr_t)o.q8 & 3) == 0) && (!o.q16 || ((uintptr_t)o.q16 & 7) == 0) &&
                      (!o.hi || ((uintptr_t)o.hi & 3) == 0) && (!o.lo || ((uintptr_t)o.lo & 3) == 0);
     const int64_t per_block = (int64_t)kThreads * (vec ? 4 * kUnroll : 1);
-    const int grid = grid_for(1, (n + per_block - 1) / per_block);
+    const bool sr = rounding == QBP_ROUND_STOCHASTIC;
+    const int bps = vec ? (sr ? blocks_per_sm(quantize_kernel<true, 4>, kThreads) : blocks_per_sm(quantize_kernel<false, 4>, kThreads))
+                        : (sr ? blocks_per_sm(quantize_kernel<true, 1>, kThreads) : blocks_per_sm(quantize_kernel<false, 1>, kThreads));
+    const int grid = grid_for(bps, (n + per_block - 1) / per_block);
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     const int c = (int)cols;
     QBP_TRACE_BEGIN(st);
@@ -494,7 +500,7 @@ int launch_colsum(const int8_t *q, int64_t rows, int64_t cols, int64_t *sums, cu
     const int rpb = kThreads / (cv < kThreads ? cv : kThreads);
     // each thread keeps int32 partials over at most 2^23 rows: 128 * 2^23 < 2^31
     int64_t min_blocks = (rows >> 23) + 1;
-    int64_t grid = grid_for(1, (rows + rpb - 1) / rpb) / slabs;
+    int64_t grid = grid_for(blocks_per_sm(colsum_kernel, kThreads), (rows + rpb - 1) / rpb) / slabs;
     if (grid < min_blocks) grid = min_blocks;
     QBP_TRACE_BEGIN(st);
     colsum_kernel<<<dim3((unsigned)grid, (unsigned)slabs), kThreads, 0, st>>>(q, rows, (int)cols, (unsigned long long *)sums);

@@ -80,18 +80,17 @@ __global__ void __launch_bounds__(kScanThreads) bn_stats_kernel(const float *__r
     }
 }
 
-// One warp per channel: mean, min, max.
-__global__ void __launch_bounds__(256) bn_stats_finalize_kernel(const float *__restrict__ part_lo,
+// One block of 128 threads per channel: mean, min, max.
+__global__ void __launch_bounds__(128) bn_stats_finalize_kernel(const float *__restrict__ part_lo,
                                                                 const float *__restrict__ part_hi,
                                                                 const double *__restrict__ part_sum, int nparts, int C,
                                                                 int64_t n, float *__restrict__ mean,
                                                                 float *__restrict__ vmin, float *__restrict__ vmax)
 {
-    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (c >= C) return;
+    const int c = blockIdx.x;
     float lo = INFINITY, hi = -INFINITY;
     double sum = 0.0;
-    for (int i = threadIdx.x & 31; i < nparts; i += 32) {
+    for (int i = threadIdx.x; i < nparts; i += 128) {
         lo = fminf(lo, part_lo[(int64_t)i * C + c]);
         hi = fmaxf(hi, part_hi[(int64_t)i * C + c]);
         sum += part_sum[(int64_t)i * C + c];
@@ -99,7 +98,14 @@ __global__ void __launch_bounds__(256) bn_stats_finalize_kernel(const float *__r
     lo = warp_min(lo); hi = warp_max(hi);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if ((threadIdx.x & 31) == 0) { mean[c] = (float)(sum / (double)n); vmin[c] = lo; vmax[c] = hi; }
+    __shared__ float s_lo[4], s_hi[4];
+    __shared__ double s_sum[4];
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; s_sum[threadIdx.x >> 5] = sum; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 4; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); sum += s_sum[w]; }
+        mean[c] = (float)(sum / (double)n); vmin[c] = lo; vmax[c] = hi;
+    }
 }
 
 template <int VEC, bool RELU>
@@ -242,18 +248,17 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
     }
 }
 
-// One warp per channel: dbeta, dgamma, and the two per-channel constants of dx:
-// m1 = gamma*dbeta/n, k2 = C(n)*gamma*dgamma.
-__global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const double *__restrict__ part_dy,
+// One block of 128 threads per channel: dbeta, dgamma, and the two per-channel
+// constants of dx: m1 = gamma*dbeta/n, k2 = C(n)*gamma*dgamma.
+__global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__restrict__ part_dy,
                                                               const double *__restrict__ part_dyx, int nparts, int C,
                                                               int64_t n, const float *__restrict__ gamma, double Cn,
                                                               float *__restrict__ dgamma, float *__restrict__ dbeta,
                                                               float2 *__restrict__ coef)
 {
-    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (c >= C) return;
+    const int c = blockIdx.x;
     double a = 0.0, b = 0.0;
-    for (int i = threadIdx.x & 31; i < nparts; i += 32) {
+    for (int i = threadIdx.x; i < nparts; i += 128) {
         a += part_dy[(int64_t)i * C + c];
         b += part_dyx[(int64_t)i * C + c];
     }
@@ -262,7 +267,11 @@ __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const double *__re
         a += __shfl_xor_sync(0xffffffffu, a, o);
         b += __shfl_xor_sync(0xffffffffu, b, o);
     }
-    if ((threadIdx.x & 31) == 0) {
+    __shared__ double s_a[4], s_b[4];
+    if ((threadIdx.x & 31) == 0) { s_a[threadIdx.x >> 5] = a; s_b[threadIdx.x >> 5] = b; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 4; ++w) { a += s_a[w]; b += s_b[w]; }
         const double g = gamma ? (double)gamma[c] : 1.0;
         if (dbeta) dbeta[c] = (float)a;
         if (dgamma) dgamma[c] = (float)b;
@@ -363,18 +372,24 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd(const floa
     float *plo = w.take<float>((size_t)kScanMaxStrips * C);
     float *phi = w.take<float>((size_t)kScanMaxStrips * C);
     const bool al = aligned16(x) && aligned16(y);
-    const ScanGeom g = scan_geom(n, C, al);
+    const bool v4 = al && C % 4 == 0;
+    const ScanGeom g = scan_geom(n, C, al, v4 ? blocks_per_sm(bn_stats_kernel<4>, kScanThreads)
+                                              : blocks_per_sm(bn_stats_kernel<1>, kScanThreads));
     const dim3 grid(g.nbx, g.slabs);
+    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_apply_kernel<4, true>, kScanThreads)
+                                                       : blocks_per_sm(bn_apply_kernel<4, false>, kScanThreads))
+                                               : blocks_per_sm(bn_apply_kernel<1, true>, kScanThreads));
+    const dim3 grid_apply(ga.nbx, ga.slabs);
     const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
     QBP_TRACE_BEGIN(st);
     if (g.vec == 4) bn_stats_kernel<4><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
     else            bn_stats_kernel<1><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
     QBP_LAUNCH_OK("bn_stats_kernel");
     QBP_TRACE_BEGIN(st);
-    bn_stats_finalize_kernel<<<(int)((C + 7) / 8), 256, 0, st>>>(plo, phi, psum, g.nbx, (int)C, n, save_mean, save_min, save_max);
+    bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(plo, phi, psum, g.nbx, (int)C, n, save_mean, save_min, save_max);
     QBP_LAUNCH_OK("bn_stats_finalize_kernel");
 QBP_TRACE_BEGIN(st);
-#define QBP_BN_APPLY(V, R) bn_apply_kernel<V, R><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, y)
+#define QBP_BN_APPLY(V, R) bn_apply_kernel<V, R><<<grid_apply, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, y)
     if (g.vec == 4) { if (relu) QBP_BN_APPLY(4, true); else QBP_BN_APPLY(4, false); }
     else            { if (relu) QBP_BN_APPLY(1, true); else QBP_BN_APPLY(1, false); }
 #undef QBP_BN_APPLY
@@ -403,8 +418,15 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const floa
     w.take<float>((size_t)kScanMaxStrips * C);
     float2 *coef = w.take<float2>((size_t)C);
     const bool al = aligned16(x) && aligned16(dy) && aligned16(dx);
-    const ScanGeom g = scan_geom(n, C, al);
+    const bool v4 = al && C % 4 == 0;
+    const ScanGeom g = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_stats_kernel<4, true>, kScanThreads)
+                                                      : blocks_per_sm(bn_bwd_stats_kernel<4, false>, kScanThreads))
+                                              : blocks_per_sm(bn_bwd_stats_kernel<1, true>, kScanThreads));
     const dim3 grid(g.nbx, g.slabs);
+    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_apply_kernel<4, true>, kScanThreads)
+                                                       : blocks_per_sm(bn_bwd_apply_kernel<4, false>, kScanThreads))
+                                               : blocks_per_sm(bn_bwd_apply_kernel<1, true>, kScanThreads));
+    const dim3 grid_apply(ga.nbx, ga.slabs);
     const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n));
     const float Cn = (float)Cnd;
 QBP_TRACE_BEGIN(st);
@@ -414,10 +436,10 @@ QBP_TRACE_BEGIN(st);
 #undef QBP_BN_BSTATS
     QBP_LAUNCH_OK("bn_bwd_stats_kernel");
     QBP_TRACE_BEGIN(st);
-    bn_bwd_finalize_kernel<<<(int)((C + 7) / 8), 256, 0, st>>>(pa, pb, g.nbx, (int)C, n, gamma, Cnd, dgamma, dbeta, coef);
+    bn_bwd_finalize_kernel<<<(int)C, 128, 0, st>>>(pa, pb, g.nbx, (int)C, n, gamma, Cnd, dgamma, dbeta, coef);
     QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
 QBP_TRACE_BEGIN(st);
-#define QBP_BN_BAPPLY(V, R) bn_bwd_apply_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx)
+#define QBP_BN_BAPPLY(V, R) bn_bwd_apply_kernel<V, R><<<grid_apply, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx)
     if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true); else QBP_BN_BAPPLY(4, false); }
     else            { if (relu) QBP_BN_BAPPLY(1, true); else QBP_BN_BAPPLY(1, false); }
 #undef QBP_BN_BAPPLY

@@ -26,7 +26,7 @@ namespace qbp {
 
 constexpr int kWgThreads = 192;
 constexpr int kWgMaxStages = 8;
-constexpr int kMaxChunks = 4;
+constexpr int kWgMaxTiles = 4;       // A tiles (128 accumulator rows each) per CTA: 4 x 2 limbs x 64 columns fill tensor memory
 
 struct WgradParams {
     CUtensorMap mapX, mapHi, mapLo;
@@ -35,11 +35,14 @@ struct WgradParams {
     uint32_t a_chunk_bytes;          // bytes of one A chunk (kr rows x rb_a)
     int conv;                        // 0: x [M x K], g [M x N]; 1: NHWC tensors
     int stages, bn, tmem_cols;
+    int kr;                          // reduction rows per pipeline stage (64 or 128)
     int a_chunks, rb_a;              // chunks per A tile, bytes (= channels / columns) per chunk row
-    int groups;                      // conv: tap groups; plain: 1
-    int tiles_a;                     // plain: K tiles of 128; conv: input-channel tiles of rb_a
+    int ma;                          // A tiles per CTA (they share the g tiles of a stage)
+    int a_tiles;                     // A tiles in all: plain K/128; conv tap groups x channel tiles
+    int a_groups;                    // ceil(a_tiles / ma)
+    int tiles_c;                     // conv: channel tiles per tap group
     int tiles_b;                     // output-channel (N) tiles of bn
-    int slices, iters_total;         // reduction steps (128 rows each) split into `slices` ranges
+    int slices, iters_total;         // reduction steps (kr rows each) split into `slices` ranges
     // conv geometry
     int H, W, Nimg, pad, R, S, C, taps;
     int bw_log2, bh_log2, tiles_w, tiles_h;
@@ -57,24 +60,27 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     uint8_t *smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
-    const uint32_t a_bytes = P.a_chunk_bytes * (uint32_t)P.a_chunks;
+    const uint32_t a_tile_bytes = P.a_chunk_bytes * (uint32_t)P.a_chunks;
+    const uint32_t a_bytes = a_tile_bytes * (uint32_t)P.ma;
     const uint32_t stage_bytes = a_bytes + 2u * P.b.tile_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int bid = blockIdx.x;
     const int tb = bid % P.tiles_b; bid /= P.tiles_b;
-    const int ta = bid % P.tiles_a; bid /= P.tiles_a;
-    const int group = bid % P.groups;
-    const int slice = bid / P.groups;
+    const int ag = bid % P.a_groups;
+    const int slice = bid / P.a_groups;
     const int n0 = tb * P.bn;
     const int it_begin = (int)((int64_t)P.iters_total * slice / P.slices);
     const int it_end = (int)((int64_t)P.iters_total * (slice + 1) / P.slices);
     const int k_iters = it_end - it_begin;
+    const int n_tiles = min(P.ma, P.a_tiles - ag * P.ma);        // A tiles this CTA owns
+    const int kk_per_iter = P.kr / 32;
 
-    // which chunks of the A tile exist for this CTA
-    int n_chunks = P.a_chunks;
-    if (P.conv) n_chunks = min(P.a_chunks, P.taps - group * P.a_chunks);
-    else        n_chunks = min(P.a_chunks, (int)((P.K - (int64_t)ta * 128 + P.rb_a - 1) / P.rb_a));
+    // chunks present in A tile `at`: conv -- taps left in the tap group; plain -- column chunks left in K
+    auto chunks_of = [&](int at) {
+        if (P.conv) return min(P.a_chunks, P.taps - (at / P.tiles_c) * P.a_chunks);
+        return min(P.a_chunks, (int)((P.K - (int64_t)at * 128 + P.rb_a - 1) / P.rb_a));
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -91,7 +97,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
 
     if (warp == 0) {
         if (lane == 0) {
-            const uint32_t tx_bytes = (uint32_t)n_chunks * P.a_chunk_bytes + 2u * P.b.tile_bytes;
+            uint32_t tx_bytes = 2u * P.b.tile_bytes;
+            for (int j = 0; j < n_tiles; ++j) tx_bytes += (uint32_t)chunks_of(ag * P.ma + j) * P.a_chunk_bytes;
             for (int i = 0; i < k_iters; ++i) {
                 const int s = i % P.stages;
                 const uint32_t ph = (uint32_t)(i / P.stages) & 1u;
@@ -102,25 +109,33 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
                 mbar_expect_tx(&full_bar[s], tx_bytes);
                 const int it = it_begin + i;
                 if (!P.conv) {
-                    const int row0 = it * 128;
-                    for (int j = 0; j < n_chunks; ++j)
-                        tma_load_2d(sa + (size_t)j * P.a_chunk_bytes, &P.mapX, &full_bar[s], ta * 128 + j * P.rb_a, row0);
+                    const int row0 = it * P.kr;
                     tma_load_2d(shi, &P.mapHi, &full_bar[s], n0, row0);
                     tma_load_2d(slo, &P.mapLo, &full_bar[s], n0, row0);
+                    for (int j = 0; j < n_tiles; ++j) {
+                        const int at = ag * P.ma + j, nc = chunks_of(at);
+                        for (int c = 0; c < nc; ++c)
+                            tma_load_2d(sa + (size_t)j * a_tile_bytes + (size_t)c * P.a_chunk_bytes, &P.mapX, &full_bar[s],
+                                        at * 128 + c * P.rb_a, row0);
+                    }
                 } else {
                     const int tw = it % P.tiles_w;
                     const int th = (it / P.tiles_w) % P.tiles_h;
                     const int tn = it / (P.tiles_w * P.tiles_h);
                     const int w0 = tw << P.bw_log2, h0 = th << P.bh_log2;
-                    const int img0 = tn * (128 >> (P.bw_log2 + P.bh_log2));
-                    for (int j = 0; j < n_chunks; ++j) {
-                        const int tap = group * P.a_chunks + j;
-                        const int r = tap / P.S, t = tap % P.S;
-                        tma_load_4d(sa + (size_t)j * P.a_chunk_bytes, &P.mapX, &full_bar[s], ta * P.rb_a,
-                                    w0 - P.pad + t, h0 - P.pad + r, img0);
-                    }
+                    const int img0 = tn * (P.kr >> (P.bw_log2 + P.bh_log2));
                     tma_load_4d(shi, &P.mapHi, &full_bar[s], n0, w0, h0, img0);
                     tma_load_4d(slo, &P.mapLo, &full_bar[s], n0, w0, h0, img0);
+                    for (int j = 0; j < n_tiles; ++j) {
+                        const int at = ag * P.ma + j, nc = chunks_of(at);
+                        const int group = at / P.tiles_c, tc = at % P.tiles_c;
+                        for (int c = 0; c < nc; ++c) {
+                            const int tap = group * P.a_chunks + c;
+                            const int r = tap / P.S, t = tap % P.S;
+                            tma_load_4d(sa + (size_t)j * a_tile_bytes + (size_t)c * P.a_chunk_bytes, &P.mapX, &full_bar[s],
+                                        tc * P.rb_a, w0 - P.pad + t, h0 - P.pad + r, img0);
+                        }
+                    }
                 }
             }
         }
@@ -135,17 +150,19 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
                 const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
                 const uint32_t hi_addr = a_addr + a_bytes;
                 const uint32_t lo_addr = hi_addr + P.b.tile_bytes;
-                const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.a.desc_lo;
                 const uint32_t bh_lo = ((hi_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
                 const uint32_t bl_lo = ((lo_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t da = ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep);
-                    const uint64_t dh = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(bh_lo + kk * P.b.kstep);
-                    const uint64_t dl = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(bl_lo + kk * P.b.kstep);
-                    const uint32_t accum = (i | kk) != 0 ? 1u : 0u;
-                    mma_i8(tmem_base, da, dh, P.idesc_hi, accum);
-                    mma_i8(tmem_base + (uint32_t)P.bn, da, dl, P.idesc_lo, accum);
+                for (int j = 0; j < n_tiles; ++j) {
+                    const uint32_t a_lo = (((a_addr + (uint32_t)j * a_tile_bytes) >> 4) & 0x3FFFu) | P.a.desc_lo;
+                    const uint32_t d_hi = tmem_base + (uint32_t)(j * 2 * P.bn);
+                    for (int kk = 0; kk < kk_per_iter; ++kk) {
+                        const uint64_t da = ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep);
+                        const uint64_t dh = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(bh_lo + kk * P.b.kstep);
+                        const uint64_t dl = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(bl_lo + kk * P.b.kstep);
+                        const uint32_t accum = (i | kk) != 0 ? 1u : 0u;
+                        mma_i8(d_hi, da, dh, P.idesc_hi, accum);
+                        mma_i8(d_hi + (uint32_t)P.bn, da, dl, P.idesc_lo, accum);
+                    }
                 }
                 mma_commit(&empty_bar[s]);
             }
@@ -160,33 +177,37 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
             tc_fence_after();
         }
         if (!timed_out && k_iters > 0) {
-            // row of the accumulator -> (chunk, channel); column -> output channel of g
-            const int chunk = row / P.rb_a, cin = row % P.rb_a;
-            bool valid = chunk < n_chunks;
-            int64_t base, col_stride;
-            if (!P.conv) {
-                const int64_t k = (int64_t)ta * 128 + row;
-                valid = valid && k < P.K;
-                base = k * P.N; col_stride = 1;
-            } else {
-                const int tap = group * P.a_chunks + chunk;
-                const int c = ta * P.rb_a + cin;
-                valid = valid && c < P.C;
-                base = (int64_t)tap * P.C + c;                          // [k][tap][c]: + k * taps * C
-                col_stride = (int64_t)P.taps * P.C;
-            }
-            for (int c0 = 0; c0 < P.bn; c0 += 32) {
-                uint32_t rh[32], rl[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, rh);
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(P.bn + c0), rl);
-                tmem_ld_wait();
-                if (!valid) continue;
+            for (int j = 0; j < n_tiles; ++j) {
+                // row of the accumulator -> (chunk, channel); column -> output channel of g
+                const int at = ag * P.ma + j;
+                const int chunk = row / P.rb_a, cin = row % P.rb_a;
+                bool valid = chunk < chunks_of(at);
+                int64_t base, col_stride;
+                if (!P.conv) {
+                    const int64_t k = (int64_t)at * 128 + row;
+                    valid = valid && k < P.K;
+                    base = k * P.N; col_stride = 1;
+                } else {
+                    const int tap = (at / P.tiles_c) * P.a_chunks + chunk;
+                    const int c = (at % P.tiles_c) * P.rb_a + cin;
+                    valid = valid && c < P.C;
+                    base = (int64_t)tap * P.C + c;                          // [k][tap][c]: + k * taps * C
+                    col_stride = (int64_t)P.taps * P.C;
+                }
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(j * 2 * P.bn);
+                for (int c0 = 0; c0 < P.bn; c0 += 32) {
+                    uint32_t rh[32], rl[32];
+                    tmem_ld_32x32(t_addr + (uint32_t)c0, rh);
+                    tmem_ld_32x32(t_addr + (uint32_t)(P.bn + c0), rl);
+                    tmem_ld_wait();
+                    if (!valid) continue;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int64_t n = (int64_t)n0 + c0 + j;
-                    if (n < P.N) {
-                        const long long v = 256ll * (long long)(int)rh[j] + (long long)(int)rl[j];
-                        atomicAdd(P.raw + base + n * col_stride, (unsigned long long)v);
+                    for (int e = 0; e < 32; ++e) {
+                        const int64_t n = (int64_t)n0 + c0 + e;
+                        if (n < P.N) {
+                            const long long v = 256ll * (long long)(int)rh[e] + (long long)(int)rl[e];
+                            atomicAdd(P.raw + base + n * col_stride, (unsigned long long)v);
+                        }
                     }
                 }
             }
@@ -297,12 +318,14 @@ __global__ void wgrad_finalize_kernel(const long long *__restrict__ raw, const l
     if (dW) dW[e] = __fmul_rn((float)acc, __fmul_rn(qx->scale, qg->scale));
 }
 
-static void pick_pixel_box_w(int Nimg, int H, int W, int &bwl, int &bhl)
+// Pixel box of `rows` = bw x bh x bn positions (powers of two) that needs the fewest steps.
+static void pick_pixel_box_w(int rows, int Nimg, int H, int W, int &bwl, int &bhl)
 {
     long long best = -1;
-    for (int a = 0; a <= 7; ++a)
-        for (int b = 0; a + b <= 7; ++b) {
-            const int bw = 1 << a, bh = 1 << b, bn = 128 >> (a + b);
+    int lg = 0; while ((1 << lg) < rows) ++lg;
+    for (int a = 0; a <= lg; ++a)
+        for (int b = 0; a + b <= lg; ++b) {
+            const int bw = 1 << a, bh = 1 << b, bn = rows >> (a + b);
             const long long tiles = (long long)((W + bw - 1) / bw) * ((H + bh - 1) / bh) * ((Nimg + bn - 1) / bn);
             const long long score = tiles * 64 - a * 8 - b;
             if (best < 0 || score < best) { best = score; bwl = a; bhl = b; }
@@ -401,52 +424,62 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
     P.conv = d ? 1 : 0;
     P.M = M; P.N = N; P.K = K;
     P.raw = (unsigned long long *)raw; P.status = status;
-    const uint32_t kr = 128;                                       // reduction rows per stage
     // g side: one swizzled row holds bn output channels
     const uint32_t rb_b = N >= 128 ? 128u : N >= 64 ? 64u : 32u;
     P.bn = (int)rb_b;
-    P.b = layout_mnmajor(kr, rb_b, 1, 0);
     P.tiles_b = (int)((N + P.bn - 1) / P.bn);
     // x side: 128 MMA rows = a_chunks chunks of rb_a columns / channels
     const uint32_t rb_a = K >= 128 ? 128u : K >= 64 ? 64u : 32u;
     P.rb_a = (int)rb_a;
     P.a_chunks = 128 / (int)rb_a;
+    if (!d) {
+        P.a_tiles = (int)((K + 127) / 128);
+        P.tiles_c = 1;
+    } else {
+        P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.R = d->R; P.S = d->S; P.C = d->C;
+        P.taps = d->R * d->S;
+        P.tiles_c = (d->C + (int)rb_a - 1) / (int)rb_a;
+        P.a_tiles = ((P.taps + P.a_chunks - 1) / P.a_chunks) * P.tiles_c;
+    }
+    // A tiles per CTA: as many as tensor memory holds (two accumulators of bn columns each)
+    P.ma = std::max(1, std::min({kWgMaxTiles, 512 / (2 * P.bn), P.a_tiles}));
+    P.a_groups = (P.a_tiles + P.ma - 1) / P.ma;
+    int cols = 32; while (cols < P.ma * 2 * P.bn) cols <<= 1;
+    P.tmem_cols = cols;
+    // reduction rows per stage: 128, or 64 when that is what it takes to keep four stages in flight
+    uint32_t kr = 128;
+    if ((200u * 1024u) / (kr * (rb_a * P.a_chunks * P.ma + 2 * rb_b)) < 4) kr = 64;
+    P.kr = (int)kr;
     P.a_chunk_bytes = kr * rb_a;
     P.a = layout_mnmajor(kr, rb_a, (uint32_t)P.a_chunks, P.a_chunk_bytes);
+    P.b = layout_mnmajor(kr, rb_b, 1, 0);
     P.idesc_hi = make_idesc(true, true, 1, 1, 128, (uint32_t)P.bn);
     P.idesc_lo = make_idesc(true, false, 1, 1, 128, (uint32_t)P.bn);
-    int cols = 32; while (cols < 2 * P.bn) cols <<= 1;
-    P.tmem_cols = cols;
 
     if (!d) {
-        P.groups = 1;
-        P.tiles_a = (int)((K + 127) / 128);
-        P.iters_total = (int)((M + 127) / 128);
+        P.iters_total = (int)((M + kr - 1) / kr);
         if ((rc = make_map_2d(&P.mapX, x, M, K, kr, rb_a))) return rc;
         if ((rc = make_map_2d(&P.mapHi, g_hi, M, N, kr, rb_b))) return rc;
         if ((rc = make_map_2d(&P.mapLo, g_lo, M, N, kr, rb_b))) return rc;
     } else {
-        P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.R = d->R; P.S = d->S; P.C = d->C;
-        P.taps = d->R * d->S;
-        P.groups = (P.taps + P.a_chunks - 1) / P.a_chunks;
-        P.tiles_a = (d->C + (int)rb_a - 1) / (int)rb_a;
         int bwl = 0, bhl = 0;
-        pick_pixel_box_w(d->N, d->H, d->W, bwl, bhl);
+        pick_pixel_box_w((int)kr, d->N, d->H, d->W, bwl, bhl);
         P.bw_log2 = bwl; P.bh_log2 = bhl;
-        const int bw = 1 << bwl, bh = 1 << bhl, bn_img = 128 >> (bwl + bhl);
+        const int bw = 1 << bwl, bh = 1 << bhl, bn_img = (int)kr >> (bwl + bhl);
         P.tiles_w = (d->W + bw - 1) / bw; P.tiles_h = (d->H + bh - 1) / bh;
         P.iters_total = P.tiles_w * P.tiles_h * ((d->N + bn_img - 1) / bn_img);
         if ((rc = make_map_nhwc(&P.mapX, x, d->N, d->H, d->W, d->C, bn_img, bh, bw, rb_a))) return rc;
         if ((rc = make_map_nhwc(&P.mapHi, g_hi, d->N, d->H, d->W, d->K, bn_img, bh, bw, rb_b))) return rc;
         if ((rc = make_map_nhwc(&P.mapLo, g_lo, d->N, d->H, d->W, d->K, bn_img, bh, bw, rb_b))) return rc;
     }
-    // split the reduction: at most 512 steps (65536 rows) per CTA, and enough CTAs to fill the machine
-    const int out_tiles = P.groups * P.tiles_a * P.tiles_b;
-    int slices = (P.iters_total + 511) / 512;
-    slices = std::max(slices, std::min(P.iters_total, std::max(1, 2 * sm_count() / out_tiles)));
+    // split the reduction: at most 65536 rows per CTA, and enough CTAs to fill the machine twice
+    const int out_items = P.a_groups * P.tiles_b;
+    const int max_iters = 65536 / (int)kr;
+    int slices = (P.iters_total + max_iters - 1) / max_iters;
+    slices = std::max(slices, std::min(P.iters_total, std::max(1, 2 * sm_count() / out_items)));
     P.slices = std::max(1, slices);
 
-    const uint32_t stage_bytes = P.a_chunk_bytes * P.a_chunks + 2 * P.b.tile_bytes;
+    const uint32_t stage_bytes = P.a_chunk_bytes * P.a_chunks * P.ma + 2 * P.b.tile_bytes;
     int stages = std::max(2, std::min<int>(kWgMaxStages, (200 * 1024) / stage_bytes));
     P.stages = stages;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
@@ -456,7 +489,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
         configured = true;
     }
     QBP_TRACE_BEGIN(st);
-    qbp_wgrad_kernel<<<P.slices * out_tiles, kWgThreads, smem, st>>>(P);
+    qbp_wgrad_kernel<<<P.slices * out_items, kWgThreads, smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_wgrad_kernel");
 
     const int blocks = (int)((outs + 255) / 256);
