@@ -34,9 +34,8 @@ BATCH, HW, CIN, COUT = 256, 56, 64, 64
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
-# (captured at batch 32 and scaled by the elements processed: traffic of these streaming kernels grows in
-# proportion).  None: not captured.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {}
+# (captured at the full batch of 256).  None: not captured.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 174.70e6 / 51380224}
 
 
 def measured_peaks():
@@ -312,7 +311,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--batch", type=int, default=BATCH, help="images per GPU (the workload is quoted at 256)")
