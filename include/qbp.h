@@ -109,6 +109,36 @@ int qbp_quantize_s8(const float *x, int64_t rows, int64_t cols, int granularity,
                     int8_t *q, qbp_qparams *qp_out, int32_t *row_sums, int64_t *col_sums,
                     void *ws, size_t ws_bytes, void *stream);
 
+/* qbp_quantize_s8 for callers that cannot provide a workspace (the paper has
+ * no counterpart; this is a packaging variant of the same kernels).  Some
+ * hosts of this library may not allocate device memory at the point where
+ * they quantise: code running under a fixed memory plan or inside a region
+ * where cudaMalloc is forbidden (it synchronises the device and can fail late),
+ * or a plugin that is handed its tensors and nothing else.  For them the range
+ * scan's scratch lives inside the library: a file-scope device array of
+ * 2 * 4 * 1024 * QBP_STATIC_MAX_CHANNELS + 256 bytes (2 MiB + 256) that every
+ * GPU which loads the library holds until the process exits.  The call itself
+ * allocates nothing (no cudaMalloc / cudaFree, no allocating library call).
+ *
+ * Same arguments and results as qbp_quantize_s8 without range_in, row_sums,
+ * col_sums and ws.  Limits: per-channel granularity needs cols <=
+ * QBP_STATIC_MAX_CHANNELS, otherwise QBP_ERR_UNSUPPORTED_SHAPE and nothing is
+ * launched; per-tensor granularity has no size limit.  Argument errors are
+ * reported before anything touches the device.
+ *
+ * The first call on each device resolves the array's device address (once per
+ * device, with that device current); make that first call outside any stream
+ * capture.  All calls on a device share the one array: it keeps the previous
+ * call's partial ranges, which is harmless (each call overwrites every entry
+ * it later reads, nothing has to start at zero), but two calls whose kernels
+ * overlap on the GPU (different streams, or different host threads) race on
+ * it -- serialise them on one stream, or use qbp_quantize_s8 with separate
+ * workspaces. */
+#define QBP_STATIC_MAX_CHANNELS 256
+int qbp_quantize_s8_static(const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
+                           uint64_t seed, uint32_t tensor_id, int8_t *q, qbp_qparams *qp_out,
+                           void *stream);
+
 /* 16-bit variant.  Any of q (int16 codes), hi (signed high byte) and lo
  * (unsigned low byte), q = 256*hi + lo, may be NULL, but not all three. */
 int qbp_quantize_s16(const float *x, int64_t rows, int64_t cols, int granularity, int rounding,

@@ -23,7 +23,7 @@ QBP_ERR_TIMEOUT = -6
 
 EXPORTS = (
     "qbp_last_error", "qbp_trace_enable", "qbp_trace_count", "qbp_trace_read",
-    "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s16", "qbp_bifurcate",
+    "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s8_static", "qbp_quantize_s16", "qbp_bifurcate",
     "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8",
     "qbp_conv_s8_workspace_bytes", "qbp_conv_s8_implicit",
     "qbp_wgrad_s16_workspace_bytes", "qbp_wgrad_s16",
@@ -147,6 +147,20 @@ def qbp_quantize_s8(x, granularity=QBP_PER_TENSOR, rounding=QBP_ROUND_NEAREST, s
     _check(lib.qbp_quantize_s8(_ptr(x), C.c_int64(rows), C.c_int64(cols), granularity, rounding,
                                C.c_uint64(seed), C.c_uint32(tensor_id), _ptr(range_in), _ptr(q), _ptr(qp_out),
                                _ptr(row_sums), _ptr(col_sums), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return q, qp_out
+
+
+QBP_STATIC_MAX_CHANNELS = 256
+
+
+def qbp_quantize_s8_static(x, q, qp_out, granularity=QBP_PER_TENSOR, rounding=QBP_ROUND_NEAREST, seed=0, tensor_id=0):
+    """qbp_quantize_s8 on the library's built-in scratch: no workspace argument and no allocation inside the
+    call, for callers that may not allocate device memory (see include/qbp.h).  The outputs q (int8, shape of
+    x) and qp_out (new_qparams(cols or 1)) are the caller's.  Per-channel granularity is limited to
+    QBP_STATIC_MAX_CHANNELS columns; calls that overlap on the GPU share, and race on, the one scratch array."""
+    cols = x.shape[-1]; rows = x.numel() // cols if cols else 0
+    _check(lib.qbp_quantize_s8_static(_ptr(x), C.c_int64(rows), C.c_int64(cols), granularity, rounding,
+                                      C.c_uint64(seed), C.c_uint32(tensor_id), _ptr(q), _ptr(qp_out), _stream()))
     return q, qp_out
 
 

@@ -8,6 +8,7 @@
 #include "qbp_colscan.cuh"
 
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 namespace qbp {
@@ -559,6 +560,35 @@ static int quantize_any(int bits, const float *x, int64_t rows, int64_t cols, in
     return launch_quantize(x, rows * cols, cols, perch, rounding, qp_out, tensor_id, qp_out, tensor_id, seed, o, st);
 }
 
+// ------------------------------------------------- built-in scratch (no allocation)
+// Scratch of qbp_quantize_s8_static: lives in the library's device image, so every GPU that loads the
+// library holds these bytes until the process exits.  Sized for the per-channel range scan of
+// QBP_STATIC_MAX_CHANNELS channels (two float partial tables of kScanMaxStrips rows), which also covers the
+// per-tensor scan.  Host code must not pass this name to a kernel: it is resolved per device below.
+constexpr size_t kStaticScratchBytes = 2 * sizeof(float) * (size_t)kScanMaxStrips * QBP_STATIC_MAX_CHANNELS + 256;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mu;
+static void *g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+static int static_scratch_address(void **out)
+{
+    int dev = -1;
+    QBP_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(QBP_ERR_CUDA, "quantize_s8_static: device ordinal %d not supported", dev);
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void *p = nullptr;
+        QBP_CUDA_OK(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p) return fail(QBP_ERR_CUDA, "quantize_s8_static: the built-in scratch has no device address");
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return QBP_OK;
+}
+
 }  // namespace qbp
 
 using namespace qbp;
@@ -640,4 +670,28 @@ extern "C" __attribute__((visibility("default"))) int qbp_bifurcate(const float 
     if (rc) return rc;
     if (row_sums8) return launch_rowsum(q8, true, rows, cols, row_sums8, st);
     return QBP_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8_static(const float *x, int64_t rows, int64_t cols, int granularity,
+                                      int rounding, uint64_t seed, uint32_t tensor_id, int8_t *q,
+                                      qbp_qparams *qp_out, void *stream)
+{
+    if (!q && rows * cols > 0) return fail(QBP_ERR_INVALID_ARG, "quantize_s8_static: q is NULL");
+    int rc = check_common(x, rows, cols, granularity, rounding, qp_out);
+    if (rc) return rc;
+    if (granularity == QBP_PER_CHANNEL && cols > QBP_STATIC_MAX_CHANNELS)
+        return fail(QBP_ERR_UNSUPPORTED_SHAPE,
+                    "quantize_s8_static: %lld channels exceed the built-in scratch (at most %d per-channel ranges); "
+                    "use qbp_quantize_s8 with a caller workspace",
+                    (long long)cols, QBP_STATIC_MAX_CHANNELS);
+    if (quant_ws_bytes(cols, granularity) > kStaticScratchBytes)
+        return fail(QBP_ERR_UNSUPPORTED_SHAPE, "quantize_s8_static: the scan needs %zu scratch bytes, %zu are built in",
+                    quant_ws_bytes(cols, granularity), kStaticScratchBytes);
+    void *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+    // every partial the finalising kernel reads was written by this call's scan: nothing has to start at zero
+    QuantOut o = {q, nullptr, nullptr, nullptr};
+    return quantize_any(8, x, rows, cols, granularity, rounding, seed, tensor_id, nullptr, o, qp_out, scratch,
+                        kStaticScratchBytes, (cudaStream_t)stream);
 }
