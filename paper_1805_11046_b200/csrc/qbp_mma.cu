@@ -82,6 +82,38 @@ int make_map_nhwc(CUtensorMap *map, const void *base, uint64_t N, uint64_t H, ui
     return QBP_OK;
 }
 
+// fp32 output matrix [rows x cols] stored in boxes of 32 rows x 32 columns (128-byte swizzled slabs).
+int make_map_out_2d(CUtensorMap *map, float *base, uint64_t rows, uint64_t cols)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * sizeof(float)};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled(fp32 output %llu x %llu) failed: %d",
+                                       (unsigned long long)rows, (unsigned long long)cols, (int)r);
+    return QBP_OK;
+}
+
+// fp32 NHWC output stored in boxes of 32 channels x (sw x sh x sn = 32 pixels).
+int make_map_out_nhwc(CUtensorMap *map, float *base, uint64_t N, uint64_t H, uint64_t W, uint64_t C, uint32_t sn,
+                      uint32_t sh, uint32_t sw)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    cuuint64_t dims[4] = {C, W, H, N};
+    cuuint64_t strides[3] = {C * sizeof(float), W * C * sizeof(float), H * W * C * sizeof(float)};
+    cuuint32_t box[4] = {32, sw, sh, sn};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(QBP_ERR_CUDA, "cuTensorMapEncodeTiled(fp32 nhwc output) failed: %d", (int)r);
+    return QBP_OK;
+}
+
 // ========================================================= operand descriptors
 // Shared-memory matrix descriptor (64 bit): start address >> 4 in bits 0..13,
 // leading byte offset >> 4 in 16..29, stride byte offset >> 4 in 32..45, the
@@ -122,31 +154,64 @@ uint32_t make_idesc(bool a_signed, bool b_signed, uint32_t a_major, uint32_t b_m
 // ================================================================== the kernel
 enum { MODE_GEMM = 0, MODE_FPROP = 1, MODE_DGRAD = 2 };
 constexpr int kMaxStages = 16;
-constexpr int kMmaThreads = 192;
-constexpr int kGroupM = 16;          // GEMM raster: tiles walk down kGroupM rows before moving one column right
+constexpr int kMaxStageMmas = 256;                    // 32 operand tiles x 2 sub-tiles x 4 k steps
+constexpr int kMaxAccBufs = 8;                        // accumulator buffers in tensor memory (512 columns in all)
+constexpr int kEpiWarps = 8;                          // two per tensor-memory lane quadrant
+constexpr int kMmaThreads = 64 + 32 * kEpiWarps;      // TMA warp, MMA warp, epilogue warps
+constexpr int kGroupM = 8;           // GEMM raster: tiles walk down kGroupM tile rows before moving one column right
+constexpr uint32_t kStageSlab = 32 * 128;             // epilogue staging per warp: 32 rows x 32 fp32
+constexpr uint32_t kSmemBudget = 226u * 1024u;        // dynamic shared memory of the kernel
+
+// Division of a non-negative int (< 2^31) by a positive constant known at launch: multiply-high and
+// shift (Granlund & Montgomery, "Division by invariant integers using multiplication").  The producer
+// and MMA-issue threads run one dependent instruction at a time, so 32-bit divisions (some 25 dependent
+// instructions each) per tile and per stage would dominate short tiles.
+struct FastDiv {
+    uint32_t mul, shr, d;
+    __device__ __forceinline__ int div(int n) const { return d == 1 ? n : (int)(__umulhi((uint32_t)n, mul) >> shr); }
+    __device__ __forceinline__ void divmod(int n, int &q, int &r) const { q = div(n); r = n - q * (int)d; }
+};
+static FastDiv make_fastdiv(int d)
+{
+    FastDiv f; f.d = (uint32_t)d; f.mul = 0; f.shr = 0;
+    if (d > 1) {
+        int lg = 0; while ((1ll << lg) < d) ++lg;
+        const int p = 31 + lg;
+        f.mul = (uint32_t)(((1ull << p) + (uint64_t)d - 1) / (uint64_t)d);
+        f.shr = (uint32_t)(p - 32);
+    }
+    return f;
+}
 
 struct MmaParams {
-    CUtensorMap mapA, mapB;
+    CUtensorMap mapA, mapB, mapC;
     OperandLayout a, b;
     uint32_t idesc;
     int mode;
     int stages, k_iters, mma_per_iter, bn, tmem_cols;
-    int ips;                      // k iterations (operand tiles) per pipeline stage
+    int msub;                     // 128-row accumulator sub-tiles per CTA tile (1 or 2)
+    int nbuf;                     // accumulator buffers in tensor memory: as many as fit (even when msub == 1)
+    int a_loads, b_loads;         // TMA loads per operand tile (M/N-major operands wider than one swizzled row)
+    uint32_t a_load_bytes, b_load_bytes;
+    int ips;                      // k iterations (operand tiles) per pipeline stage (at most 32: one lane each)
+    int iter_entries;             // entries of the k-iteration table in shared memory (conv), a multiple of 64
     int b_resident;               // conv: all filter tiles of the CTA's N tile stay in shared memory
     uint32_t b_res_bytes;         // bytes reserved for them at the start of shared memory
+    int ncls;                     // rows of the column-term table (1, or 16 border classes)
+    int cterm_all;                // the whole table [ncls][N] is kept in shared memory (else one tile's columns)
     int tiles_m, tiles_n, tiles_total;
     // output
     int64_t M, N;                 // rows / columns of the output matrix
     int32_t *acc_out; float *out;
-    const int32_t *rowterm;       // GEMM: [M]
-    const int32_t *chan_sum;      // conv: per input pixel, the sum of its codes over the reduced channels
-    const int32_t *colterm;       // [classes][N]
+    const int32_t *rowterm;       // [M]
+    const int32_t *colterm;       // [ncls][N]
     const qbp_qparams *qa, *qb;
     int *status;
     int kblock;                   // GEMM: reduction elements per k iteration
     // conv geometry (output pixel grid == input pixel grid: stride 1, same padding)
     int H, W, Nimg, pad, S, cchunks, chunk_bytes, Cred;
     int bw_log2, bh_log2, tiles_w, tiles_h;
+    FastDiv d_tiles_n, d_tiles_w, d_tiles_h, d_group;
 };
 
 struct TileOrigin { int m0, n0, img0, h0, w0; };
@@ -158,21 +223,20 @@ __device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
     if (P.mode == MODE_GEMM) {
         // groups of kGroupM tile rows; inside a group the row index moves fastest, so that the CTAs
         // running at one time share few A row-blocks and few B column-blocks (L2 reuse)
-        const int per_group = kGroupM * P.tiles_n;
-        const int g = tile / per_group, r = tile % per_group;
+        int g, r;
+        P.d_group.divmod(tile, g, r);                    // by kGroupM * tiles_n
         const int rows_here = min(kGroupM, P.tiles_m - g * kGroupM);
-        tile_m = g * kGroupM + r % rows_here;
-        tile_n = r / rows_here;
+        if (rows_here == kGroupM) { tile_n = r / kGroupM; tile_m = g * kGroupM + r % kGroupM; }
+        else                      { tile_n = r / rows_here; tile_m = g * kGroupM + r % rows_here; }   // the last, ragged group
     } else {
-        tile_n = tile % P.tiles_n;
-        tile_m = tile / P.tiles_n;
+        P.d_tiles_n.divmod(tile, tile_m, tile_n);
     }
     o.n0 = tile_n * P.bn;
-    o.m0 = tile_m * 128; o.img0 = 0; o.h0 = 0; o.w0 = 0;
+    o.m0 = tile_m * 128 * P.msub; o.img0 = 0; o.h0 = 0; o.w0 = 0;
     if (P.mode != MODE_GEMM) {
-        const int tw = tile_m % P.tiles_w;
-        const int th = (tile_m / P.tiles_w) % P.tiles_h;
-        const int tn = tile_m / (P.tiles_w * P.tiles_h);
+        int t1, tw, tn, th;
+        P.d_tiles_w.divmod(tile_m, t1, tw);
+        P.d_tiles_h.divmod(t1, tn, th);
         o.w0 = tw << P.bw_log2;
         o.h0 = th << P.bh_log2;
         o.img0 = tn * (128 >> (P.bw_log2 + P.bh_log2));
@@ -180,103 +244,155 @@ __device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
     return o;
 }
 
+// The MMAs of one pipeline stage, from the per-kernel table in shared memory: entry i = (offset of the A
+// descriptor from the stage's first A tile, offset of the B descriptor, accumulator column offset, unused),
+// offsets in 16-byte units (the 14-bit address field cannot carry: shared memory ends below 256 KB).  The
+// single issuing thread is bound by its own instruction latency on narrow tiles, hence one 16-byte load and
+// two adds per MMA instead of index arithmetic.
+__device__ __forceinline__ void issue_stage(const uint4 *__restrict__ tab, int n_mma, uint32_t a_lo, uint32_t a_hi,
+                                            uint32_t b_lo, uint32_t b_hi, uint32_t d_tmem, uint32_t idesc, bool first_stage)
+{
+#pragma unroll 4
+    for (int i = 0; i < n_mma; ++i) {
+        const uint4 e = tab[i];
+        const uint64_t da = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + e.x);
+        const uint64_t db = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + e.y);
+        mma_i8(d_tmem + e.z, da, db, idesc, (first_stage && i < (int)e.w) ? 0u : 1u);
+    }
+}
+
 __device__ __forceinline__ void raise_timeout(int *status) { atomicExch(status, (int)QBP_ERR_TIMEOUT); }
 
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The producer runs ahead of
-// the MMA warp across tile boundaries through the shared-memory ring; the accumulator is double
-// buffered in tensor memory so that the epilogue of tile i overlaps the MMAs of tile i + 1.
+// the MMA warp across tile boundaries through the shared-memory ring.  A CTA tile is msub accumulator
+// sub-tiles of 128 rows x bn columns that share the B operand of every stage (256 x 256 halves the
+// operand bytes fetched per multiply-add against 128 x 256).  When two sets of accumulators fit in
+// tensor memory they are used in turn, so that the epilogues of earlier tiles overlap the MMAs of later ones.
+// Epilogue: tcgen05.ld -> zero-point terms -> fp32 -> swizzled staging slab -> TMA store per warp.
 __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_constant__ MmaParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], b_full;
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[kMaxAccBufs], acc_empty[kMaxAccBufs], b_full;
     __shared__ uint32_t tmem_slot;
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     uint8_t *smem_b = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);     // resident filter tiles (if any)
     uint8_t *smem = smem_b + P.b_res_bytes;                                  // the stage ring
-    const uint32_t a_stage = P.a.tile_bytes * (uint32_t)P.ips;
+    const uint32_t a_iter = P.a.tile_bytes * (uint32_t)P.msub;               // A bytes of one k iteration
+    const uint32_t a_stage = a_iter * (uint32_t)P.ips;
     const uint32_t stage_bytes = a_stage + (P.b_resident ? 0u : P.b.tile_bytes * (uint32_t)P.ips);
+    uint8_t *staging = smem + (((size_t)P.stages * stage_bytes + 1023) & ~(size_t)1023);   // kEpiWarps slabs, 1024-byte aligned
+    int4 *s_iter = reinterpret_cast<int4 *>(staging + kEpiWarps * kStageSlab);          // conv: one entry per k iteration
+    uint4 *s_mma = reinterpret_cast<uint4 *>(s_iter + P.iter_entries);                   // the MMAs of one stage (kMaxStageMmas)
+    int32_t *s_cterm = reinterpret_cast<int32_t *>(s_mma + kMaxStageMmas);               // column terms
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        // an accumulator buffer is read by both epilogue groups (msub == 2) or by one of them
+        for (int b = 0; b < P.nbuf; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], P.msub == 2 ? kEpiWarps : kEpiWarps / 2); }
         mbar_init(&b_full, 1);
         mbar_fence_init();
         tma_prefetch_desc(&P.mapA);
         tma_prefetch_desc(&P.mapB);
+        if (P.out) tma_prefetch_desc(&P.mapC);
     }
     if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
+    for (int i = threadIdx.x; i < P.ips * P.msub * P.mma_per_iter; i += kMmaThreads) {
+        // MMA i of a stage: k iteration j, sub-tile sub, k step kk (innermost)
+        const int kk = i % P.mma_per_iter, sub = (i / P.mma_per_iter) % P.msub, j = i / (P.mma_per_iter * P.msub);
+        // the first MMAs of a tile (j == 0, kk == 0 of every sub-tile) overwrite the accumulator: i < w
+        s_mma[i] = make_uint4(((uint32_t)j * a_iter + (uint32_t)sub * P.a.tile_bytes) / 16u + (uint32_t)kk * P.a.kstep,
+                              ((uint32_t)j * P.b.tile_bytes) / 16u + (uint32_t)kk * P.b.kstep, (uint32_t)(sub * P.bn),
+                              (j == 0 && kk == 0) ? 0xFFFFu : 0u);
+    }
+    if (P.mode != MODE_GEMM)
+        for (int it = threadIdx.x; it < P.k_iters; it += kMmaThreads) {
+            // k iteration -> (channel offset, tap column, tap row, filter coordinate of the tap's channel chunk)
+            const int tap = it / P.cchunks, cc = it % P.cchunks;
+            const int c0 = cc * P.chunk_bytes;
+            s_iter[it] = make_int4(c0, tap % P.S, tap / P.S, P.mode == MODE_FPROP ? tap * P.Cred + c0 : tap * (int)P.N);
+        }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    const uint32_t buf_cols = (uint32_t)(P.msub * P.bn);
     bool timed_out = false;
 
     if (warp == 0) {
-        if (lane == 0) {
-            // ------------------------------------------------ TMA producer
-            if (P.b_resident) {
-                // the filter is the same for every tile of this CTA: fetch it once
-                const int n0 = 0;
-                mbar_expect_tx(&b_full, P.b.tile_bytes * (uint32_t)P.k_iters);
-                int it = 0;
-                for (int tap = 0; tap < P.k_iters / P.cchunks; ++tap)
-                    for (int cc = 0; cc < P.cchunks; ++cc, ++it) {
-                        uint8_t *dst = smem_b + (size_t)it * P.b.tile_bytes;
-                        const int c0 = cc * P.chunk_bytes;
-                        if (P.mode == MODE_FPROP) tma_load_2d(dst, &P.mapB, &b_full, tap * P.Cred + c0, n0);
-                        else                      tma_load_2d(dst, &P.mapB, &b_full, tap * (int)P.N + n0, c0);
-                    }
+        // ---------------------------------------------------- TMA producer
+        // Lane 0 owns the barriers.  Convolution: the `ips` activation tiles of a stage are issued by
+        // `ips` lanes at once, each from its own entry of the k-iteration table.
+        if (P.b_resident && lane == 0) {
+            // the filter is the same for every tile of this CTA: fetch it once
+            mbar_expect_tx(&b_full, P.b.tile_bytes * (uint32_t)P.k_iters);
+            for (int it = 0; it < P.k_iters; ++it) {
+                const int4 e = s_iter[it];
+                uint8_t *dst = smem_b + (size_t)it * P.b.tile_bytes;
+                if (P.mode == MODE_FPROP) tma_load_2d(dst, &P.mapB, &b_full, e.w, 0);
+                else
+                    for (int l = 0; l < P.b_loads; ++l)
+                        tma_load_2d(dst + (size_t)l * P.b_load_bytes, &P.mapB, &b_full, e.w + l * 128, e.x);
             }
-            uint32_t gs = 0;                                    // ring position, continues across tiles
-            for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
-                const TileOrigin o = tile_origin(P, tile);
-                if (P.mode == MODE_GEMM) {
-                    for (int it = 0; it < P.k_iters; ++it, ++gs) {
-                        const uint32_t s = gs % (uint32_t)P.stages;
-                        if (!mbar_wait(&empty_bar[s], ((gs / (uint32_t)P.stages) & 1u) ^ 1u)) { timed_out = true; break; }
+        }
+        uint32_t s = 0, ph = 1;                             // ring position and the parity to wait for, across tiles
+        const int groups = P.k_iters / P.ips;
+        for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
+            const TileOrigin o = tile_origin(P, tile);
+            if (P.mode == MODE_GEMM) {
+                if (lane == 0) {
+                    for (int it = 0; it < P.k_iters; ++it) {
+                        if (!mbar_wait(&empty_bar[s], ph)) { timed_out = true; break; }
                         uint8_t *sa = smem + (size_t)s * stage_bytes;
                         uint8_t *sb = sa + a_stage;
                         mbar_expect_tx(&full_bar[s], stage_bytes);
                         const int k0 = it * P.kblock;
+                        // K-major operands: one box of all rows; M/N-major: one box per 128-byte column chunk
                         if (P.a.major == 0) tma_load_2d(sa, &P.mapA, &full_bar[s], k0, o.m0);
-                        else                tma_load_2d(sa, &P.mapA, &full_bar[s], o.m0, k0);
+                        else
+                            for (int l = 0; l < P.a_loads; ++l)
+                                tma_load_2d(sa + (size_t)l * P.a_load_bytes, &P.mapA, &full_bar[s], o.m0 + l * 128, k0);
                         if (P.b.major == 0) tma_load_2d(sb, &P.mapB, &full_bar[s], k0, o.n0);
-                        else                tma_load_2d(sb, &P.mapB, &full_bar[s], o.n0, k0);
+                        else
+                            for (int l = 0; l < P.b_loads; ++l)
+                                tma_load_2d(sb + (size_t)l * P.b_load_bytes, &P.mapB, &full_bar[s], o.n0 + l * 128, k0);
+                        if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
                     }
-                    continue;
                 }
-                // convolution: one activation tile per (tap, channel chunk), `ips` of them per stage
-                int j = 0, tap = 0;
-                uint32_t s = 0;
-                uint8_t *sa = nullptr;
-                const int R = P.k_iters / (P.cchunks * P.S);
-                for (int r = 0; r < R && !timed_out; ++r)
-                    for (int t = 0; t < P.S && !timed_out; ++t, ++tap)
-                        for (int cc = 0; cc < P.cchunks; ++cc) {
-                            if (j == 0) {
-                                s = gs % (uint32_t)P.stages;
-                                if (!mbar_wait(&empty_bar[s], ((gs / (uint32_t)P.stages) & 1u) ^ 1u)) { timed_out = true; break; }
-                                sa = smem + (size_t)s * stage_bytes;
-                                mbar_expect_tx(&full_bar[s], stage_bytes);
-                            }
-                            const int c0 = cc * P.chunk_bytes;
-                            uint8_t *da = sa + (size_t)j * P.a.tile_bytes;
-                            uint8_t *db = sa + a_stage + (size_t)j * P.b.tile_bytes;
-                            if (P.mode == MODE_FPROP) {
-                                // input pixel of output (p,q) under tap (r,t): (p - pad + r, q - pad + t)
-                                tma_load_4d(da, &P.mapA, &full_bar[s], c0, o.w0 - P.pad + t, o.h0 - P.pad + r, o.img0);
-                                // filter as [K rows x (R*S*C) columns]: this tap's channel chunk, K-major
-                                if (!P.b_resident) tma_load_2d(db, &P.mapB, &full_bar[s], tap * P.Cred + c0, o.n0);
-                            } else {
-                                // gradient pixel feeding input (h,w) under tap (r,t): (h + pad - r, w + pad - t)
-                                tma_load_4d(da, &P.mapA, &full_bar[s], c0, o.w0 + P.pad - t, o.h0 + P.pad - r, o.img0);
-                                // filter rows = output channels (the reduction), columns = this tap's input channels
-                                if (!P.b_resident) tma_load_2d(db, &P.mapB, &full_bar[s], tap * (int)P.N + o.n0, c0);
-                            }
-                            if (++j == P.ips) { j = 0; ++gs; }
-                        }
+                timed_out = __shfl_sync(0xffffffffu, timed_out ? 1 : 0, 0) != 0;
+                continue;
+            }
+            // convolution: one activation tile per (tap, channel chunk), `ips` of them per stage
+            for (int g = 0; g < groups; ++g) {
+                int ok = 1;
+                if (lane == 0) {
+                    ok = mbar_wait(&empty_bar[s], ph) ? 1 : 0;
+                    if (ok) mbar_expect_tx(&full_bar[s], stage_bytes);
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { timed_out = true; break; }
+                if (lane < P.ips) {
+                    const int4 e = s_iter[g * P.ips + lane];   // (channel offset, tap column, tap row, filter coordinate)
+                    uint8_t *sa = smem + (size_t)s * stage_bytes;
+                    uint8_t *da = sa + (size_t)lane * P.a.tile_bytes;
+                    uint8_t *db = sa + a_stage + (size_t)lane * P.b.tile_bytes;
+                    if (P.mode == MODE_FPROP) {
+                        // input pixel of output (p,q) under tap (r,t): (p - pad + r, q - pad + t)
+                        tma_load_4d(da, &P.mapA, &full_bar[s], e.x, o.w0 - P.pad + e.y, o.h0 - P.pad + e.z, o.img0);
+                        // filter as [K rows x (R*S*C) columns]: this tap's channel chunk, K-major
+                        if (!P.b_resident) tma_load_2d(db, &P.mapB, &full_bar[s], e.w, o.n0);
+                    } else {
+                        // gradient pixel feeding input (h,w) under tap (r,t): (h + pad - r, w + pad - t)
+                        tma_load_4d(da, &P.mapA, &full_bar[s], e.x, o.w0 + P.pad - e.y, o.h0 + P.pad - e.z, o.img0);
+                        // filter rows = output channels (the reduction), columns = this tap's input channels
+                        if (!P.b_resident)
+                            for (int l = 0; l < P.b_loads; ++l)
+                                tma_load_2d(db + (size_t)l * P.b_load_bytes, &P.mapB, &full_bar[s], e.w + o.n0 + l * 128, e.x);
+                    }
+                }
+                __syncwarp();
+                if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
             }
         }
         __syncwarp();
@@ -285,123 +401,164 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
             // -------------------------------------------------- MMA issuer
             if (P.b_resident && !mbar_wait(&b_full, 0)) timed_out = true;
             const uint32_t bres_addr = smem_u32(smem_b);
+            const uint32_t ring_addr = smem_u32(smem);
             const int groups = P.k_iters / P.ips;
-            uint32_t gs = 0, lt = 0;
-            for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x, ++lt) {
-                const uint32_t buf = lt & 1u;
-                if (!mbar_wait(&acc_empty[buf], ((lt >> 1) & 1u) ^ 1u)) { timed_out = true; break; }
+            const int n_mma = P.ips * P.msub * P.mma_per_iter;
+            uint32_t s = 0, ph = 0;                          // ring position and parity, across tiles
+            uint32_t buf = 0, bph = 1;                       // accumulator buffer and the parity of its "empty" barrier
+            for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
+                if (!mbar_wait(&acc_empty[buf], bph)) { timed_out = true; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * (uint32_t)P.bn;
-                int it = 0;
-                for (int g = 0; g < groups; ++g, ++gs) {
-                    const uint32_t s = gs % (uint32_t)P.stages;
-                    if (!mbar_wait(&full_bar[s], (gs / (uint32_t)P.stages) & 1u)) { timed_out = true; break; }
+                const uint32_t d_tmem = tmem_base + buf * buf_cols;
+                for (int g = 0; g < groups; ++g) {
+                    if (!mbar_wait(&full_bar[s], ph)) { timed_out = true; break; }
                     tc_fence_after();
-                    const uint32_t stage_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                    for (int j = 0; j < P.ips; ++j, ++it) {
-                        const uint32_t a_addr = stage_addr + (uint32_t)j * P.a.tile_bytes;
-                        const uint32_t b_addr = P.b_resident ? bres_addr + (uint32_t)it * P.b.tile_bytes
-                                                             : stage_addr + a_stage + (uint32_t)j * P.b.tile_bytes;
-                        const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.a.desc_lo;
-                        const uint32_t b_lo = ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
-                        for (int kk = 0; kk < P.mma_per_iter; ++kk) {
-                            const uint64_t da = ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep);
-                            const uint64_t db = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(b_lo + kk * P.b.kstep);
-                            mma_i8(d_tmem, da, db, P.idesc, (it | kk) != 0 ? 1u : 0u);
-                        }
-                    }
+                    const uint32_t stage_addr = ring_addr + s * stage_bytes;
+                    const uint32_t b_addr = P.b_resident ? bres_addr + (uint32_t)(g * P.ips) * P.b.tile_bytes : stage_addr + a_stage;
+                    issue_stage(s_mma, n_mma, ((stage_addr >> 4) & 0x3FFFu) | P.a.desc_lo, P.a.desc_hi,
+                                ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo, P.b.desc_hi, d_tmem, P.idesc, g == 0);
                     mma_commit(&empty_bar[s]);
+                    if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
                 }
                 if (!timed_out) mma_commit(&acc_full[buf]);
+                if (++buf == (uint32_t)P.nbuf) { buf = 0; bph ^= 1u; }
             }
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------- epilogue
-        const int quad = warp & 3;
+        // msub == 2: both groups of four warps work on every tile, one 128-row sub-tile each.
+        // msub == 1: the groups take alternate tiles (and accumulator buffers), so that the latency of one
+        //            tile's read-out and store is hidden behind the other group's tile.
+        const int ew = warp - 2;                         // 0 .. kEpiWarps-1
+        const int quad = warp & 3;                       // the tensor-memory lanes this warp may read
+        const int group = ew >> 2;
         const int row = quad * 32 + lane;
+        uint8_t *slab = staging + (size_t)ew * kStageSlab;
         const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
-        const int za = P.qa->zero_point, zb = P.qb->zero_point;
-        uint32_t lt = 0;
-        for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x, ++lt) {
-            const TileOrigin o = tile_origin(P, tile);
-            const uint32_t buf = lt & 1u;
-            // this row's output position and zero-point row term (independent of the accumulator)
-            int64_t m; bool valid; int cls = 0, rterm = 0;
+        const int sub = P.msub == 2 ? group : 0;
+        const int lt_step = P.msub == 2 ? 1 : 2;
+        const int bar_id = P.msub == 2 ? 1 : 1 + group, bar_cnt = P.msub == 2 ? 32 * kEpiWarps : 128;
+        const int gt = P.msub == 2 ? threadIdx.x - 64 : (threadIdx.x - 64) & 127;     // thread index within the barrier group
+        int32_t *region = s_cterm + (P.cterm_all || P.msub == 2 ? 0 : group * P.ncls * P.bn);
+        if (P.cterm_all) {
+            // the whole column-term table fits: fill it once
+            for (int i = threadIdx.x - 64; i < P.ncls * (int)P.N; i += 32 * kEpiWarps) s_cterm[i] = __ldg(P.colterm + i);
+            named_barrier(1, 32 * kEpiWarps);
+        }
+
+        // where this thread's accumulator row of a tile goes
+        struct RowInfo { int64_t m; bool valid, slab_in; int cls, sx, sy, sz; };
+        auto row_info = [&](const TileOrigin &o) {
+            RowInfo ri; ri.cls = 0; ri.sx = ri.sy = ri.sz = 0;
             if (P.mode == MODE_GEMM) {
-                m = (int64_t)o.m0 + row;
-                valid = m < P.M;
-                if (valid) rterm = __ldg(P.rowterm + m);
+                ri.m = (int64_t)o.m0 + sub * 128 + row;
+                ri.valid = ri.m < P.M;
+                ri.slab_in = (int64_t)o.m0 + sub * 128 + quad * 32 < P.M;
             } else {
                 const int dw = row & ((1 << P.bw_log2) - 1);
                 const int dh = (row >> P.bw_log2) & ((1 << P.bh_log2) - 1);
                 const int dn = row >> (P.bw_log2 + P.bh_log2);
                 const int n = o.img0 + dn, p = o.h0 + dh, q = o.w0 + dw;
-                valid = n < P.Nimg && p < P.H && q < P.W;
-                m = ((int64_t)n * P.H + p) * P.W + q;
-                cls = (p == 0 ? 1 : 0) | (p == P.H - 1 ? 2 : 0) | (q == 0 ? 4 : 0) | (q == P.W - 1 ? 8 : 0);
-                if (valid) {
-                    // sum of the input's channel sums over the taps inside the image, and their count
-                    // (pad is 0 or 1: nine predicated loads, issued together)
-                    int box = 0, taps = 0;
-                    const int32_t *cs = P.chan_sum + ((int64_t)n * P.H + p) * P.W + q;
-#pragma unroll
-                    for (int eh = -1; eh <= 1; ++eh)
-#pragma unroll
-                        for (int ew = -1; ew <= 1; ++ew) {
-                            const bool in = eh >= -P.pad && eh <= P.pad && ew >= -P.pad && ew <= P.pad &&
-                                            p + eh >= 0 && p + eh < P.H && q + ew >= 0 && q + ew < P.W;
-                            box += in ? __ldg(cs + eh * P.W + ew) : 0;
-                            taps += in ? 1 : 0;
-                        }
-                    rterm = -zb * box + taps * P.Cred * za * zb;
-                }
+                ri.valid = n < P.Nimg && p < P.H && q < P.W;
+                ri.m = ((int64_t)n * P.H + p) * P.W + q;
+                ri.cls = (p == 0 ? 1 : 0) | (p == P.H - 1 ? 2 : 0) | (q == 0 ? 4 : 0) | (q == P.W - 1 ? 8 : 0);
+                const int r0 = quad * 32;            // this warp's 32 rows are a sub-box of the pixel box
+                ri.sx = o.w0 + (r0 & ((1 << P.bw_log2) - 1));
+                ri.sy = o.h0 + ((r0 >> P.bw_log2) & ((1 << P.bh_log2) - 1));
+                ri.sz = o.img0 + (r0 >> (P.bw_log2 + P.bh_log2));
+                ri.slab_in = ri.sx < P.W && ri.sy < P.H && ri.sz < P.Nimg;
             }
-            const int32_t *cterm = P.colterm + (int64_t)cls * P.N;
-            if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1u)) { timed_out = true; break; }
-            tc_fence_after();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * (uint32_t)P.bn;
-            for (int c0 = 0; c0 < P.bn; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32(t_addr + (uint32_t)c0, r);
-                tmem_ld_wait();
-                if (c0 + 32 >= P.bn) {
-                    // the accumulator has been read out: hand the buffer back to the MMA warp
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            return ri;
+        };
+
+        const int tile_step = (int)gridDim.x * lt_step;
+        int tile = blockIdx.x + (P.msub == 2 ? 0 : group * (int)gridDim.x);
+        // this group's accumulator buffer and the parity of its "full" barrier; msub == 1: buffers of the group's own parity
+        uint32_t buf = P.msub == 2 ? 0u : (uint32_t)group, fph = 0;
+        TileOrigin o = tile_origin(P, tile < P.tiles_total ? tile : 0);
+        RowInfo ri = row_info(o);
+        int rterm = (tile < P.tiles_total && ri.valid) ? __ldg(P.rowterm + ri.m) : 0;
+        for (; tile < P.tiles_total; tile += tile_step) {
+            // the next tile's row term is fetched now, so that its latency hides behind this tile
+            const int tile_next = tile + tile_step;
+            const TileOrigin o_next = tile_origin(P, tile_next < P.tiles_total ? tile_next : 0);
+            const RowInfo ri_next = row_info(o_next);
+            const int rterm_next = (tile_next < P.tiles_total && ri_next.valid) ? __ldg(P.rowterm + ri_next.m) : 0;
+            if (!P.cterm_all) {
+                // column terms of this tile into shared memory (the previous tile's readers are done first)
+                named_barrier(bar_id, bar_cnt);
+                for (int i = gt; i < P.ncls * P.bn; i += bar_cnt) {
+                    const int cls = i / P.bn, n = o.n0 + i % P.bn;
+                    region[i] = n < P.N ? __ldg(P.colterm + (int64_t)cls * P.N + n) : 0;
                 }
-                if (!valid) continue;
-                const int64_t ncol = P.N - (o.n0 + c0);                 // columns left in the matrix
-                if (ncol <= 0) continue;
-                const int lim = ncol < 32 ? (int)ncol : 32;
-                int acc[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j] = j < lim ? (int)r[j] + rterm + __ldg(cterm + o.n0 + c0 + j) : 0;
-                if (P.acc_out) {
-                    int32_t *dst = P.acc_out + m * P.N + o.n0 + c0;
-                    if (lim == 32) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<int4 *>(dst + j) = make_int4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
-                    } else {
-                        for (int j = 0; j < lim; ++j) dst[j] = acc[j];
+                named_barrier(bar_id, bar_cnt);
+            }
+            const int32_t *cterm = P.cterm_all ? s_cterm + ri.cls * (int)P.N + o.n0 : region + ri.cls * P.bn;
+            const int64_t ncol = P.N - o.n0;                                // columns left in the matrix
+            const int nchunks = (int)((ncol < P.bn ? ncol : P.bn) + 31) / 32;
+            if (!timed_out && !mbar_wait_warp(&acc_full[buf], fph)) timed_out = true;
+            if (!timed_out) {
+                tc_fence_after();
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * buf_cols + (uint32_t)(sub * P.bn);
+                for (int c = 0; c < nchunks; ++c) {
+                    const int c0 = c * 32;
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_addr + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                    if (c == nchunks - 1) {
+                        // the accumulator has been read out: hand the buffer back to the MMA warp
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&acc_empty[buf]);
                     }
-                }
-                if (P.out) {
-                    float *dst = P.out + m * P.N + o.n0 + c0;
-                    if (lim == 32) {
+                    const int lim = (int)(ncol - c0 < 32 ? ncol - c0 : 32);
+                    int acc[32];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const int4 ct = *reinterpret_cast<const int4 *>(cterm + c0 + j);
+                        acc[j] = (int)r[j] + rterm + ct.x; acc[j + 1] = (int)r[j + 1] + rterm + ct.y;
+                        acc[j + 2] = (int)r[j + 2] + rterm + ct.z; acc[j + 3] = (int)r[j + 3] + rterm + ct.w;
+                    }
+                    if (P.acc_out && ri.valid) {
+                        int32_t *dst = P.acc_out + ri.m * P.N + o.n0 + c0;
+                        if (lim == 32) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<int4 *>(dst + j) = make_int4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < lim) dst[j] = acc[j];
+                        }
+                    }
+                    if (P.out) {
+                        // the previous store of this warp must have read the slab before it is overwritten
+                        if (lane == 0) tma_store_wait_read();
+                        __syncwarp();
+                        // 128-byte swizzle: the 16-byte group g of row `lane` sits at group g ^ (lane & 7)
+                        uint8_t *rowp = slab + lane * 128;
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4 *>(dst + j) =
+                            *reinterpret_cast<float4 *>(rowp + (((j >> 2) ^ (lane & 7)) << 4)) =
                                 make_float4(__fmul_rn((float)acc[j], scale), __fmul_rn((float)acc[j + 1], scale),
                                             __fmul_rn((float)acc[j + 2], scale), __fmul_rn((float)acc[j + 3], scale));
-                    } else {
-                        for (int j = 0; j < lim; ++j) dst[j] = __fmul_rn((float)acc[j], scale);
+                        fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0 && ri.slab_in) {
+                            if (P.mode == MODE_GEMM) tma_store_2d(&P.mapC, slab, o.n0 + c0, o.m0 + sub * 128 + quad * 32);
+                            else                     tma_store_4d(&P.mapC, slab, o.n0 + c0, ri.sx, ri.sy, ri.sz);
+                            tma_store_commit();
+                        }
                     }
                 }
             }
+            o = o_next; ri = ri_next; rterm = rterm_next;
+            buf += (uint32_t)lt_step;
+            if (buf >= (uint32_t)P.nbuf) { buf -= (uint32_t)P.nbuf; fph ^= 1u; }
         }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
     }
 
     if (timed_out) {
@@ -458,32 +615,69 @@ __global__ void conv_colterm_kernel(const int32_t *wsum32, const long long *wsum
     colterm[cls * N + n] = -q_in->zero_point * (int)sum;
 }
 
+// rowterm[pixel] = -z_w * (sum of the input's channel sums over the taps inside the image)
+//                   + (taps inside) * Cred * z_in * z_w          (pad is 0 or 1)
+__global__ void __launch_bounds__(256) conv_rowterm_kernel(const int32_t *__restrict__ chan_sum, int64_t pixels, int H,
+                                                           int W, int pad, int Cred, const qbp_qparams *q_in,
+                                                           const qbp_qparams *q_w, int32_t *__restrict__ rowterm)
+{
+    const int64_t m = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (m >= pixels) return;
+    const int za = q_in->zero_point, zb = q_w->zero_point;
+    const int q = (int)(m % W), p = (int)((m / W) % H);
+    int box = 0, taps = 0;
+    for (int eh = -pad; eh <= pad; ++eh)
+        for (int ew = -pad; ew <= pad; ++ew)
+            if (p + eh >= 0 && p + eh < H && q + ew >= 0 && q + ew < W) {
+                box += chan_sum[m + (int64_t)eh * W + ew];
+                ++taps;
+            }
+    rowterm[m] = -zb * box + taps * Cred * za * zb;
+}
+
 // ================================================================== launchers
 static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
 {
-    const uint32_t budget = 200u * 1024u;
+    // shared memory that is not the stage ring: alignment slack, epilogue staging slabs, column terms
+    // column terms: the whole table when it is small, else one tile's columns per epilogue group
+    P.cterm_all = (size_t)P.ncls * P.N * sizeof(int32_t) <= 32u * 1024u ? 1 : 0;
+    const size_t cterm_bytes = P.cterm_all ? ((size_t)P.ncls * P.N + 64) * sizeof(int32_t)
+                                           : (size_t)(P.msub == 1 ? 2 : 1) * P.ncls * P.bn * sizeof(int32_t);
+    P.iter_entries = P.mode == MODE_GEMM ? 0 : (int)align_up((size_t)P.k_iters, 64);
+    const uint32_t fixed = 2048u + kEpiWarps * kStageSlab + (uint32_t)P.iter_entries * 16u + kMaxStageMmas * 16u +
+                           (uint32_t)align_up(cterm_bytes, 1024);
+    const uint32_t budget = kSmemBudget - fixed;
     P.ips = 1; P.b_resident = 0; P.b_res_bytes = 0;
     if (P.mode != MODE_GEMM) {
         // keep the whole filter in shared memory when it fits beside at least three activation stages
         const uint32_t b_all = P.b.tile_bytes * (uint32_t)P.k_iters;
         if (P.tiles_n == 1 && b_all + 3 * P.a.tile_bytes <= budget) { P.b_resident = 1; P.b_res_bytes = (uint32_t)align_up(b_all, 1024); }
-        // several small activation tiles share one stage (fewer barrier round trips)
+        // several operand tiles share one stage: every tcgen05.commit that releases a stage drains the MMA
+        // pipeline (some hundred cycles), which short MMAs cannot afford often; two stages must still fit
         const uint32_t per_iter = P.a.tile_bytes + (P.b_resident ? 0u : P.b.tile_bytes);
         for (int c = 1; c <= P.k_iters; ++c)
-            if (P.k_iters % c == 0 && (uint32_t)c * per_iter <= 32u * 1024u) P.ips = c;
+            if (P.k_iters % c == 0 && c <= 32 && 2u * (uint32_t)c * per_iter <= budget - P.b_res_bytes) P.ips = c;
     }
-    const uint32_t stage_bytes = (uint32_t)P.ips * (P.a.tile_bytes + (P.b_resident ? 0u : P.b.tile_bytes));
+    const uint32_t stage_bytes = (uint32_t)P.ips * (P.a.tile_bytes * (uint32_t)P.msub + (P.b_resident ? 0u : P.b.tile_bytes));
     int stages = (int)((budget - P.b_res_bytes) / stage_bytes);
-    stages = std::max(2, std::min(stages, kMaxStages));
+    if (stages < 2) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "tensor-core tile does not fit shared memory");
+    stages = std::min(stages, kMaxStages);
     P.stages = stages;
-    int cols = 32; while (cols < 2 * P.bn) cols <<= 1;       // two accumulator buffers
+    // several small accumulators let the MMAs run ahead of the epilogue (msub == 1: groups alternate, so an even count)
+    P.nbuf = std::min(kMaxAccBufs, 512 / (P.msub * P.bn));
+    if (P.msub == 1) P.nbuf &= ~1;
+    int cols = 32; while (cols < P.nbuf * P.msub * P.bn) cols <<= 1;
     P.tmem_cols = cols;
     P.tiles_m = tiles_m;
     P.tiles_total = tiles_m * P.tiles_n;
-    const size_t smem = (size_t)P.b_res_bytes + (size_t)stages * stage_bytes + 1024;
+    P.d_tiles_n = make_fastdiv(P.tiles_n);
+    P.d_group = make_fastdiv(kGroupM * P.tiles_n);
+    P.d_tiles_w = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_w);
+    P.d_tiles_h = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_h);
+    const size_t smem = (size_t)fixed + P.b_res_bytes + (size_t)stages * stage_bytes;
     static thread_local bool configured = false;
     if (!configured) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
         configured = true;
     }
     QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
@@ -583,28 +777,39 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     P.kblock = 128;
     P.k_iters = (int)((K + 127) / 128);
     P.mma_per_iter = 4;
-    // A: stored [M x K] -> K-major rows of 128 reduction bytes; stored [K x M] -> MN-major
-    if (!transA) { P.a = layout_kmajor(128, 128); rc = make_map_2d(&P.mapA, A, M, K, 128, 128); }
-    else         { P.a = layout_mnmajor(128, 128, 1, 0); rc = make_map_2d(&P.mapA, A, K, M, 128, 128); }
+    P.msub = M > 128 ? 2 : 1;            // 256-row CTA tiles halve the operand traffic per multiply-add
+    P.ncls = 1;
+    // A: stored [M x K] -> K-major rows of 128 reduction bytes; stored [K x M] -> M-major, one box per sub-tile
+    if (!transA) {
+        P.a = layout_kmajor(128, 128);
+        rc = make_map_2d(&P.mapA, A, M, K, 128u * P.msub, 128);
+    } else {
+        P.a = layout_mnmajor(128, 128, 1, 0);
+        P.a_loads = P.msub; P.a_load_bytes = P.a.tile_bytes;
+        rc = make_map_2d(&P.mapA, A, K, M, 128, 128);
+    }
     if (rc) return rc;
     if (transB) {
         P.bn = (int)std::min<int64_t>(256, N);
         P.b = layout_kmajor((uint32_t)P.bn, 128);
         rc = make_map_2d(&P.mapB, B, N, K, (uint32_t)P.bn, 128);
     } else {
-        // N-contiguous operand: one swizzled row holds min(128, N) output columns
+        // N-contiguous operand: one swizzled row holds min(128, N) output columns; two such chunks make 256
         const uint32_t rb = N >= 128 ? 128u : N >= 64 ? 64u : 32u;
-        P.bn = (int)rb;
-        P.b = layout_mnmajor(128, rb, 1, 0);
+        const uint32_t chunks = (rb == 128 && N >= 256) ? 2u : 1u;
+        P.bn = (int)(rb * chunks);
+        P.b = layout_mnmajor(128, rb, chunks, 128 * rb);
+        P.b_loads = (int)chunks; P.b_load_bytes = 128 * rb;
         rc = make_map_2d(&P.mapB, B, K, N, 128, rb);
     }
     if (rc) return rc;
+    if (C && (rc = make_map_out_2d(&P.mapC, C, M, N))) return rc;
     P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
     P.tiles_n = (int)((N + P.bn - 1) / P.bn);
     P.M = M; P.N = N;
     P.acc_out = acc_out; P.out = C;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = qa; P.qb = qb; P.status = status;
-    return launch_mma(P, (int)((M + 127) / 128), st);
+    return launch_mma(P, (int)((M + 128 * P.msub - 1) / (128 * P.msub)), st);
 }
 
 extern "C" __attribute__((visibility("default"))) size_t qbp_conv_s8_workspace_bytes(int mode, const qbp_conv_desc *d)
@@ -642,7 +847,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
 
     WsCarver w(ws, ws_bytes);
     int *status = w.take<int>(1);
-    w.take<int32_t>(pix);
+    int32_t *rowterm = w.take<int32_t>(pix);
     int32_t *chan_sum = w.take<int32_t>(pix);
     int32_t *colterm = w.take<int32_t>(16 * nmax);
     int64_t *wsum = w.take<int64_t>((int64_t)taps * nmax);
@@ -657,9 +862,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
         dgrad ? nullptr : (const int32_t *)wsum, dgrad ? (const long long *)wsum : nullptr, Nout, d->R, d->S, d->pad,
         dgrad ? 1 : 0, q_in, colterm);
     QBP_LAUNCH_OK("conv_colterm_kernel");
+    QBP_TRACE_BEGIN(st);
+    conv_rowterm_kernel<<<(unsigned)((pix + 255) / 256), 256, 0, st>>>(chan_sum, pix, d->H, d->W, d->pad, Cred, q_in, q_w, rowterm);
+    QBP_LAUNCH_OK("conv_rowterm_kernel");
 
     MmaParams P{};
     P.mode = dgrad ? MODE_DGRAD : MODE_FPROP;
+    P.msub = 1; P.ncls = 16;
     P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.S = d->S; P.Cred = Cred;
     const uint32_t cb = Cred % 128 == 0 ? 128u : Cred % 64 == 0 ? 64u : 32u;      // reduction bytes per stage row
     P.chunk_bytes = (int)cb;
@@ -681,15 +890,22 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
         rc = make_map_2d(&P.mapB, wgt, d->K, (uint64_t)taps * d->C, (uint32_t)P.bn, cb);
     } else {
         const uint32_t rb = Nout >= 128 ? 128u : Nout >= 64 ? 64u : 32u;
-        P.bn = (int)rb;
-        P.b = layout_mnmajor(cb, rb, 1, 0);
+        const uint32_t chunks = (rb == 128 && Nout >= 256) ? 2u : 1u;
+        P.bn = (int)(rb * chunks);
+        P.b = layout_mnmajor(cb, rb, chunks, cb * rb);
+        P.b_loads = (int)chunks; P.b_load_bytes = cb * rb;
         rc = make_map_2d(&P.mapB, wgt, d->K, (uint64_t)taps * d->C, cb, rb);
     }
     if (rc) return rc;
+    if (out) {
+        // a warp's 32 accumulator rows are a sub-box of the 128-pixel box (all extents are powers of two)
+        const uint32_t sw = (uint32_t)std::min(bw, 32), sh = (uint32_t)std::min(bh, 32 / (int)sw), sn = 32 / (sw * sh);
+        if ((rc = make_map_out_nhwc(&P.mapC, out, d->N, d->H, d->W, Nout, sn, sh, sw))) return rc;
+    }
     P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
     P.tiles_n = (Nout + P.bn - 1) / P.bn;
     P.M = pix; P.N = Nout;
     P.acc_out = acc_out; P.out = out;
-    P.rowterm = nullptr; P.chan_sum = chan_sum; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
+    P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
     return launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st);
 }

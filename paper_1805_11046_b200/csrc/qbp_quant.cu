@@ -483,7 +483,8 @@ int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int
     if (cols % 16 || !aligned16(q)) return fail(QBP_ERR_INVALID_ARG, "row sums need 16-byte aligned rows (cols %% 16 == 0)");
     int G = 1; while (G < 32 && G < cols / 16) G <<= 1;
     const int64_t groups = kThreads / G;
-    const int grid = grid_for(1, (rows + groups - 1) / groups);
+    const int grid = grid_for(is_signed ? blocks_per_sm(rowsum_kernel<true>, kThreads) : blocks_per_sm(rowsum_kernel<false>, kThreads),
+                              (rows + groups - 1) / groups);
     QBP_TRACE_BEGIN(st);
     if (is_signed) rowsum_kernel<true><<<grid, kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, G, sums);
     else           rowsum_kernel<false><<<grid, kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, G, sums);
