@@ -162,27 +162,6 @@ constexpr int kGroupM = 8;           // GEMM raster: tiles walk down kGroupM til
 constexpr uint32_t kStageSlab = 32 * 128;             // epilogue staging per warp: 32 rows x 32 fp32
 constexpr uint32_t kSmemBudget = 226u * 1024u;        // dynamic shared memory of the kernel
 
-// Division of a non-negative int (< 2^31) by a positive constant known at launch: multiply-high and
-// shift (Granlund & Montgomery, "Division by invariant integers using multiplication").  The producer
-// and MMA-issue threads run one dependent instruction at a time, so 32-bit divisions (some 25 dependent
-// instructions each) per tile and per stage would dominate short tiles.
-struct FastDiv {
-    uint32_t mul, shr, d;
-    __device__ __forceinline__ int div(int n) const { return d == 1 ? n : (int)(__umulhi((uint32_t)n, mul) >> shr); }
-    __device__ __forceinline__ void divmod(int n, int &q, int &r) const { q = div(n); r = n - q * (int)d; }
-};
-static FastDiv make_fastdiv(int d)
-{
-    FastDiv f; f.d = (uint32_t)d; f.mul = 0; f.shr = 0;
-    if (d > 1) {
-        int lg = 0; while ((1ll << lg) < d) ++lg;
-        const int p = 31 + lg;
-        f.mul = (uint32_t)(((1ull << p) + (uint64_t)d - 1) / (uint64_t)d);
-        f.shr = (uint32_t)(p - 32);
-    }
-    return f;
-}
-
 struct MmaParams {
     CUtensorMap mapA, mapB, mapC;
     OperandLayout a, b;
@@ -252,12 +231,14 @@ __device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
 __device__ __forceinline__ void issue_stage(const uint4 *__restrict__ tab, int n_mma, uint32_t a_lo, uint32_t a_hi,
                                             uint32_t b_lo, uint32_t b_hi, uint32_t d_tmem, uint32_t idesc, bool first_stage)
 {
-#pragma unroll 4
+    uint4 e = tab[0];
+#pragma unroll 2
     for (int i = 0; i < n_mma; ++i) {
-        const uint4 e = tab[i];
+        const uint4 nxt = tab[i + 1 < n_mma ? i + 1 : i];       // fetched while this MMA is being issued
         const uint64_t da = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + e.x);
         const uint64_t db = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + e.y);
-        mma_i8(d_tmem + e.z, da, db, idesc, (first_stage && i < (int)e.w) ? 0u : 1u);
+        mma_i8(d_tmem + e.z, da, db, idesc, (first_stage && e.w != 0u) ? 0u : 1u);
+        e = nxt;
     }
 }
 
@@ -759,10 +740,10 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     // code sums along the reduction
     int rc;
     if (!transA) rc = launch_rowsum(A, true, M, K, (int32_t *)tmp_m, st);
-    else         rc = launch_colsum(A, K, M, tmp_m, st);
+    else         rc = launch_colsum(A, true, K, M, tmp_m, st);
     if (rc) return rc;
     if (transB) rc = launch_rowsum(B, true, N, K, (int32_t *)tmp_n, st);
-    else        rc = launch_colsum(B, K, N, tmp_n, st);
+    else        rc = launch_colsum(B, true, K, N, tmp_n, st);
     if (rc) return rc;
     const int64_t mx = std::max(M, N);
     QBP_TRACE_BEGIN(st);
@@ -855,7 +836,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
     int rc = launch_rowsum(in, true, pix, Cred, chan_sum, st);
     if (rc) return rc;
     if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
-    else        rc = launch_colsum(wgt, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
+    else        rc = launch_colsum(wgt, true, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
     if (rc) return rc;
     QBP_TRACE_BEGIN(st);
     conv_colterm_kernel<<<dim3((Nout + 127) / 128, 16), 128, 0, st>>>(

@@ -11,7 +11,7 @@ namespace qbp {
 
 // ---- sums of stored codes (qbp_quant.cu) -------------------------------------
 int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int32_t *sums, cudaStream_t st);
-int launch_colsum(const int8_t *q, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st);
+int launch_colsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st);
 
 // ---- TMA tensor maps ---------------------------------------------------------
 // A dense byte matrix [rows x cols] (cols innermost) read in boxes of
@@ -36,6 +36,30 @@ OperandLayout layout_kmajor(uint32_t rows, uint32_t row_bytes);
 // MN-major tile: `krows` reduction rows of `row_bytes` (32/64/128) M/N bytes each;
 // `chunks` such tiles side by side (chunk_stride bytes apart) widen M/N beyond row_bytes.
 OperandLayout layout_mnmajor(uint32_t krows, uint32_t row_bytes, uint32_t chunks, uint32_t chunk_stride);
+
+// ---- division by launch-time constants ----------------------------------------
+// Division of a non-negative int (< 2^31) by a positive constant known at launch: multiply-high and
+// shift (Granlund & Montgomery, "Division by invariant integers using multiplication").  The producer
+// and MMA-issue threads run one dependent instruction at a time, so 32-bit divisions (some 25 dependent
+// instructions each) per tile and per stage would dominate short tiles.
+struct FastDiv {
+    uint32_t mul, shr, d;
+#ifdef __CUDACC__
+    __device__ __forceinline__ int div(int n) const { return d == 1 ? n : (int)(__umulhi((uint32_t)n, mul) >> shr); }
+    __device__ __forceinline__ void divmod(int n, int &q, int &r) const { q = div(n); r = n - q * (int)d; }
+#endif
+};
+inline FastDiv make_fastdiv(int d)
+{
+    FastDiv f; f.d = (uint32_t)d; f.mul = 0; f.shr = 0;
+    if (d > 1) {
+        int lg = 0; while ((1ll << lg) < d) ++lg;
+        const int p = 31 + lg;
+        f.mul = (uint32_t)(((1ull << p) + (uint64_t)d - 1) / (uint64_t)d);
+        f.shr = (uint32_t)(p - 32);
+    }
+    return f;
+}
 
 uint32_t make_idesc(bool a_signed, bool b_signed, uint32_t a_major, uint32_t b_major, uint32_t m, uint32_t n);
 

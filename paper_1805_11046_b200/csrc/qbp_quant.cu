@@ -361,12 +361,13 @@ __global__ void __launch_bounds__(kThreads) rowsum_kernel(const uint8_t *__restr
     }
 }
 
-// Column sums (over rows) of stored signed 8-bit codes into int64.  blockIdx.y
+// Column sums (over rows) of stored 8-bit codes (signed or unsigned) into int64.  blockIdx.y
 // selects a slab of up to 256 column groups (16 codes each); inside a slab a
 // thread owns one group and every (256 / groups)-th row.  Block partials meet in
 // shared memory, then one atomic per column and block.  The destination must be
 // zeroed beforehand.
-__global__ void __launch_bounds__(kThreads) colsum_kernel(const int8_t *__restrict__ q, int64_t rows, int cols,
+template <bool IS_SIGNED>
+__global__ void __launch_bounds__(kThreads) colsum_kernel(const uint8_t *__restrict__ q, int64_t rows, int cols,
                                                           unsigned long long *__restrict__ sums)
 {
     const int cv = cols >> 4;
@@ -387,7 +388,8 @@ __global__ void __launch_bounds__(kThreads) colsum_kernel(const int8_t *__restri
 #pragma unroll
             for (int k = 0; k < 4; ++k)
 #pragma unroll
-                for (int b = 0; b < 4; ++b) acc[k * 4 + b] += (int)(int8_t)(w[k] >> (8 * b));
+                for (int b = 0; b < 4; ++b)
+                    acc[k * 4 + b] += IS_SIGNED ? (int)(int8_t)(w[k] >> (8 * b)) : (int)((w[k] >> (8 * b)) & 0xFFu);
         }
 #pragma unroll
         for (int e = 0; e < 16; ++e) atomicAdd(&s_acc[tx * 16 + e], acc[e]);
@@ -492,7 +494,7 @@ int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int
     return QBP_OK;
 }
 
-int launch_colsum(const int8_t *q, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st)
+int launch_colsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st)
 {
     if (cols % 16 || !aligned16(q)) return fail(QBP_ERR_INVALID_ARG, "column sums need cols %% 16 == 0");
     QBP_CUDA_OK(cudaMemsetAsync(sums, 0, sizeof(int64_t) * cols, st));
@@ -500,12 +502,13 @@ int launch_colsum(const int8_t *q, int64_t rows, int64_t cols, int64_t *sums, cu
     const int cv = (int)(cols / 16);
     const int slabs = (cv + kThreads - 1) / kThreads;
     const int rpb = kThreads / (cv < kThreads ? cv : kThreads);
-    // each thread keeps int32 partials over at most 2^23 rows: 128 * 2^23 < 2^31
-    int64_t min_blocks = (rows >> 23) + 1;
-    int64_t grid = grid_for(blocks_per_sm(colsum_kernel, kThreads), (rows + rpb - 1) / rpb) / slabs;
+    // each thread keeps int32 partials over at most 2^22 rows: 255 * 2^22 < 2^31
+    int64_t min_blocks = (rows >> 22) + 1;
+    int64_t grid = grid_for(blocks_per_sm(colsum_kernel<true>, kThreads), (rows + rpb - 1) / rpb) / slabs;
     if (grid < min_blocks) grid = min_blocks;
     QBP_TRACE_BEGIN(st);
-    colsum_kernel<<<dim3((unsigned)grid, (unsigned)slabs), kThreads, 0, st>>>(q, rows, (int)cols, (unsigned long long *)sums);
+    if (is_signed) colsum_kernel<true><<<dim3((unsigned)grid, (unsigned)slabs), kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, (unsigned long long *)sums);
+    else           colsum_kernel<false><<<dim3((unsigned)grid, (unsigned)slabs), kThreads, 0, st>>>((const uint8_t *)q, rows, (int)cols, (unsigned long long *)sums);
     QBP_LAUNCH_OK("colsum_kernel");
     return QBP_OK;
 }
@@ -636,7 +639,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8(const floa
     int rc = quantize_any(8, x, rows, cols, granularity, rounding, seed, tensor_id, range_in, o, qp_out, ws, ws_bytes, st);
     if (rc) return rc;
     if (row_sums) { rc = launch_rowsum(q, true, rows, cols, row_sums, st); if (rc) return rc; }
-    if (col_sums) { rc = launch_colsum(q, rows, cols, col_sums, st); if (rc) return rc; }
+    if (col_sums) { rc = launch_colsum(q, true, rows, cols, col_sums, st); if (rc) return rc; }
     return QBP_OK;
 }
 

@@ -9,15 +9,27 @@
 // (batch x spatial positions for a convolution): both operands are therefore
 // "M/N-major" in shared memory -- the TMA box is [reduction rows x channels].
 // A CTA reduces at most 65536 rows (128*255*65536 < 2^31 bounds the low limb,
-// 128*128*65536 the high one), combines its two accumulators exactly in int64
-// and adds them to the int64 result with red.global.add.u64; integer addition
-// is order-free, so the split over CTAs does not change the result.
+// 128*128*65536 the high one) and combines its two accumulators exactly in
+// int64.  Integer addition is order-free, so the split of the reduction over
+// CTAs does not change the result.
+//
+// Work split: an item is (group of up to `ma` accumulator tiles of 128 output
+// rows, tile of bn output columns); the reduction of an item is cut into
+// slices in proportion to the item's cost per reduction step, so that one
+// wave of CTAs finishes together.  A CTA that owns a whole reduction applies
+// the zero-points and the scale itself; otherwise the CTAs write int64
+// partials and a second kernel adds them up.
 //
 // Convolution: the MMA's 128 rows hold `chunks` filter taps x the input
 // channels of one tap (2 taps x 64 channels, or 1 tap x 128 channels); each
 // tap is its own TMA load of the input, shifted by the tap offset, padding
 // zero-filled.  Zero-points are applied afterwards from per-border-class code
 // sums (a tap near the border sees fewer positions).
+//
+// The TMA-issuing and MMA-issuing threads are bound by their own instruction
+// latency, so both run from small tables built once per CTA (one entry per
+// load / per MMA of a stage), and stages are released in groups: a
+// tcgen05.commit drains the MMA pipeline, which short MMAs cannot afford often.
 #include "qbp_mma.cuh"
 
 #include <algorithm>
@@ -27,6 +39,9 @@ namespace qbp {
 constexpr int kWgThreads = 192;
 constexpr int kWgMaxStages = 8;
 constexpr int kWgMaxTiles = 4;       // A tiles (128 accumulator rows each) per CTA: 4 x 2 limbs x 64 columns fill tensor memory
+constexpr int kWgMaxLoads = 32;      // TMA loads per stage: one lane each
+constexpr int kWgMaxMmas = 128;      // MMAs per stage: 4 tiles x 4 k steps x 2 limbs, with room
+constexpr uint32_t kWgSmem = 220u * 1024u;
 
 struct WgradParams {
     CUtensorMap mapX, mapHi, mapLo;
@@ -34,29 +49,57 @@ struct WgradParams {
     uint32_t idesc_hi, idesc_lo;
     uint32_t a_chunk_bytes;          // bytes of one A chunk (kr rows x rb_a)
     int conv;                        // 0: x [M x K], g [M x N]; 1: NHWC tensors
-    int stages, bn, tmem_cols;
-    int kr;                          // reduction rows per pipeline stage (64 or 128)
+    int stages, cg, bn, tmem_cols;   // cg: stages released by one commit
+    int kr;                          // reduction rows per pipeline stage
     int a_chunks, rb_a;              // chunks per A tile, bytes (= channels / columns) per chunk row
     int ma;                          // A tiles per CTA (they share the g tiles of a stage)
     int a_tiles;                     // A tiles in all: plain K/128; conv tap groups x channel tiles
     int a_groups;                    // ceil(a_tiles / ma)
     int tiles_c;                     // conv: channel tiles per tap group
     int tiles_b;                     // output-channel (N) tiles of bn
-    int slices, iters_total;         // reduction steps (kr rows each) split into `slices` ranges
+    int iters_total;                 // reduction steps of kr rows each
+    int s_full, s_last;              // slices of an item of a full A group / of the last (possibly smaller) group
+    int ctas_full;                   // CTAs working on full groups: (a_groups - 1) * tiles_b * s_full
+    int direct;                      // every item is one slice: the CTA finishes its outputs itself (plain only)
     // conv geometry
     int H, W, Nimg, pad, R, S, C, taps;
     int bw_log2, bh_log2, tiles_w, tiles_h;
+    FastDiv d_tiles_w, d_tiles_h;
     // plain geometry
     int64_t M, N, K;
-    unsigned long long *raw;         // int64 accumulator, zeroed before launch
+    long long *part;                 // int64 partials, one block of part_stride values per CTA
+    int64_t part_stride;             // ma * 128 * bn
+    // direct epilogue (plain): acc = raw + rowterm[k] + colterm[n]
+    const long long *rowterm, *colterm;
+    const qbp_qparams *qx, *qg;
+    long long *acc_out; float *dW;
     int *status;
 };
+
+// Which item and slice a CTA works on.
+struct WgItem { int ag, tb, slice, slices; };
+
+__device__ __forceinline__ WgItem wg_item(const WgradParams &P, int bid)
+{
+    WgItem w;
+    int item;
+    if (bid < P.ctas_full) { item = bid / P.s_full; w.slice = bid % P.s_full; w.slices = P.s_full; }
+    else {
+        const int r = bid - P.ctas_full;
+        item = P.ctas_full / P.s_full + r / P.s_last; w.slice = r % P.s_last; w.slices = P.s_last;
+    }
+    w.ag = item / P.tiles_b; w.tb = item % P.tiles_b;
+    return w;
+}
 
 __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_constant__ WgradParams P)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kWgMaxStages], empty_bar[kWgMaxStages], acc_bar;
     __shared__ uint32_t tmem_slot;
+    __shared__ int4 s_load[kWgMaxLoads];      // (destination offset in the stage, 0 x / 1 hi / 2 lo, channel offset, tap dw | dh << 16)
+    __shared__ uint4 s_mma[kWgMaxMmas];       // (A descriptor offset, B descriptor offset, accumulator column, limb | first k step << 1)
+    __shared__ int s_counts[2];               // loads, MMAs per stage
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     uint8_t *smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
@@ -65,13 +108,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     const uint32_t stage_bytes = a_bytes + 2u * P.b.tile_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int bid = blockIdx.x;
-    const int tb = bid % P.tiles_b; bid /= P.tiles_b;
-    const int ag = bid % P.a_groups;
-    const int slice = bid / P.a_groups;
-    const int n0 = tb * P.bn;
-    const int it_begin = (int)((int64_t)P.iters_total * slice / P.slices);
-    const int it_end = (int)((int64_t)P.iters_total * (slice + 1) / P.slices);
+    const WgItem wi = wg_item(P, blockIdx.x);
+    const int ag = wi.ag;
+    const int n0 = wi.tb * P.bn;
+    const int it_begin = (int)((int64_t)P.iters_total * wi.slice / wi.slices);
+    const int it_end = (int)((int64_t)P.iters_total * (wi.slice + 1) / wi.slices);
     const int k_iters = it_end - it_begin;
     const int n_tiles = min(P.ma, P.a_tiles - ag * P.ma);        // A tiles this CTA owns
     const int kk_per_iter = P.kr / 32;
@@ -87,6 +128,34 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         mbar_init(&acc_bar, 1);
         mbar_fence_init();
         tma_prefetch_desc(&P.mapX); tma_prefetch_desc(&P.mapHi); tma_prefetch_desc(&P.mapLo);
+        // the loads of one stage
+        int nl = 0;
+        s_load[nl++] = make_int4((int)a_bytes, 1, n0, 0);
+        s_load[nl++] = make_int4((int)(a_bytes + P.b.tile_bytes), 2, n0, 0);
+        for (int j = 0; j < n_tiles; ++j) {
+            const int at = ag * P.ma + j, nc = chunks_of(at);
+            for (int c = 0; c < nc; ++c) {
+                const int dst = (int)((uint32_t)j * a_tile_bytes + (uint32_t)c * P.a_chunk_bytes);
+                if (!P.conv) s_load[nl++] = make_int4(dst, 0, at * 128 + c * P.rb_a, 0);
+                else {
+                    const int tap = (at / P.tiles_c) * P.a_chunks + c;
+                    const int dh = tap / P.S - P.pad, dw = tap % P.S - P.pad;
+                    s_load[nl++] = make_int4(dst, 0, (at % P.tiles_c) * P.rb_a, (dw & 0xFFFF) | (dh << 16));
+                }
+            }
+        }
+        s_counts[0] = nl;
+    }
+    if (threadIdx.x == 32) {
+        // the MMAs of one stage: k step outermost, so that consecutive MMAs write different accumulators
+        int nm = 0;
+        for (int kk = 0; kk < kk_per_iter; ++kk)
+            for (int j = 0; j < n_tiles; ++j)
+                for (int limb = 0; limb < 2; ++limb)
+                    s_mma[nm++] = make_uint4(((uint32_t)j * a_tile_bytes) / 16u + (uint32_t)kk * P.a.kstep,
+                                             ((uint32_t)limb * P.b.tile_bytes) / 16u + (uint32_t)kk * P.b.kstep,
+                                             (uint32_t)((j * 2 + limb) * P.bn), (uint32_t)limb | (kk == 0 ? 2u : 0u));
+        s_counts[1] = nm;
     }
     if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
     tc_fence_before();
@@ -96,104 +165,83 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     bool timed_out = false;
 
     if (warp == 0) {
-        if (lane == 0) {
-            uint32_t tx_bytes = 2u * P.b.tile_bytes;
-            for (int j = 0; j < n_tiles; ++j) tx_bytes += (uint32_t)chunks_of(ag * P.ma + j) * P.a_chunk_bytes;
-            for (int i = 0; i < k_iters; ++i) {
-                const int s = i % P.stages;
-                const uint32_t ph = (uint32_t)(i / P.stages) & 1u;
-                if (!mbar_wait(&empty_bar[s], ph ^ 1u)) { timed_out = true; break; }
-                uint8_t *sa = smem + (size_t)s * stage_bytes;
-                uint8_t *shi = sa + a_bytes;
-                uint8_t *slo = shi + P.b.tile_bytes;
-                mbar_expect_tx(&full_bar[s], tx_bytes);
+        // ---------------------------------------------------- TMA producer (lane 0 owns the barriers)
+        const int n_loads = s_counts[0];
+        uint32_t tx_bytes = 2u * P.b.tile_bytes;
+        for (int j = 0; j < n_tiles; ++j) tx_bytes += (uint32_t)chunks_of(ag * P.ma + j) * P.a_chunk_bytes;
+        const int4 ld = lane < n_loads ? s_load[lane] : make_int4(0, 0, 0, 0);
+        const int dw = (int)(short)(ld.w & 0xFFFF), dh = ld.w >> 16;
+        const void *map = ld.y == 0 ? (const void *)&P.mapX : ld.y == 1 ? (const void *)&P.mapHi : (const void *)&P.mapLo;
+        uint32_t s = 0, gph = 1;                      // stage, parity of the stage group's "empty" barrier
+        for (int i = 0; i < k_iters; ++i) {
+            int ok = 1;
+            if (lane == 0) {
+                if (s % (uint32_t)P.cg == 0) ok = mbar_wait(&empty_bar[s / (uint32_t)P.cg], gph) ? 1 : 0;
+                if (ok) mbar_expect_tx(&full_bar[s], tx_bytes);
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) { timed_out = true; break; }
+            if (lane < n_loads) {
+                uint8_t *dst = smem + (size_t)s * stage_bytes + ld.x;
                 const int it = it_begin + i;
-                if (!P.conv) {
-                    const int row0 = it * P.kr;
-                    tma_load_2d(shi, &P.mapHi, &full_bar[s], n0, row0);
-                    tma_load_2d(slo, &P.mapLo, &full_bar[s], n0, row0);
-                    for (int j = 0; j < n_tiles; ++j) {
-                        const int at = ag * P.ma + j, nc = chunks_of(at);
-                        for (int c = 0; c < nc; ++c)
-                            tma_load_2d(sa + (size_t)j * a_tile_bytes + (size_t)c * P.a_chunk_bytes, &P.mapX, &full_bar[s],
-                                        at * 128 + c * P.rb_a, row0);
-                    }
-                } else {
-                    const int tw = it % P.tiles_w;
-                    const int th = (it / P.tiles_w) % P.tiles_h;
-                    const int tn = it / (P.tiles_w * P.tiles_h);
+                if (!P.conv) tma_load_2d(dst, map, &full_bar[s], ld.z, it * P.kr);
+                else {
+                    int t1, tw, tn, th;
+                    P.d_tiles_w.divmod(it, t1, tw);
+                    P.d_tiles_h.divmod(t1, tn, th);
                     const int w0 = tw << P.bw_log2, h0 = th << P.bh_log2;
                     const int img0 = tn * (P.kr >> (P.bw_log2 + P.bh_log2));
-                    tma_load_4d(shi, &P.mapHi, &full_bar[s], n0, w0, h0, img0);
-                    tma_load_4d(slo, &P.mapLo, &full_bar[s], n0, w0, h0, img0);
-                    for (int j = 0; j < n_tiles; ++j) {
-                        const int at = ag * P.ma + j, nc = chunks_of(at);
-                        const int group = at / P.tiles_c, tc = at % P.tiles_c;
-                        for (int c = 0; c < nc; ++c) {
-                            const int tap = group * P.a_chunks + c;
-                            const int r = tap / P.S, t = tap % P.S;
-                            tma_load_4d(sa + (size_t)j * a_tile_bytes + (size_t)c * P.a_chunk_bytes, &P.mapX, &full_bar[s],
-                                        tc * P.rb_a, w0 - P.pad + t, h0 - P.pad + r, img0);
-                        }
-                    }
+                    tma_load_4d(dst, map, &full_bar[s], ld.z, w0 + dw, h0 + dh, img0);
                 }
             }
+            __syncwarp();
+            if (++s == (uint32_t)P.stages) { s = 0; gph ^= 1u; }
         }
-        __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
+            // -------------------------------------------------- MMA issuer
+            const int n_mma = s_counts[1];
+            const uint32_t ring = smem_u32(smem);
+            const uint32_t a_desc_hi = P.a.desc_hi, b_desc_hi = P.b.desc_hi, idesc_hi = P.idesc_hi, idesc_lo = P.idesc_lo;
+            uint32_t s = 0, ph = 0;
             for (int i = 0; i < k_iters; ++i) {
-                const int s = i % P.stages;
-                const uint32_t ph = (uint32_t)(i / P.stages) & 1u;
                 if (!mbar_wait(&full_bar[s], ph)) { timed_out = true; break; }
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint32_t hi_addr = a_addr + a_bytes;
-                const uint32_t lo_addr = hi_addr + P.b.tile_bytes;
-                const uint32_t bh_lo = ((hi_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
-                const uint32_t bl_lo = ((lo_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
-                for (int j = 0; j < n_tiles; ++j) {
-                    const uint32_t a_lo = (((a_addr + (uint32_t)j * a_tile_bytes) >> 4) & 0x3FFFu) | P.a.desc_lo;
-                    const uint32_t d_hi = tmem_base + (uint32_t)(j * 2 * P.bn);
-                    for (int kk = 0; kk < kk_per_iter; ++kk) {
-                        const uint64_t da = ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep);
-                        const uint64_t dh = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(bh_lo + kk * P.b.kstep);
-                        const uint64_t dl = ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(bl_lo + kk * P.b.kstep);
-                        const uint32_t accum = (i | kk) != 0 ? 1u : 0u;
-                        mma_i8(d_hi, da, dh, P.idesc_hi, accum);
-                        mma_i8(d_hi + (uint32_t)P.bn, da, dl, P.idesc_lo, accum);
-                    }
+                const uint32_t a_addr = ring + s * stage_bytes;
+                const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.a.desc_lo;
+                const uint32_t b_lo = (((a_addr + a_bytes) >> 4) & 0x3FFFu) | P.b.desc_lo;
+                uint4 e = s_mma[0];
+#pragma unroll 2
+                for (int m = 0; m < n_mma; ++m) {
+                    const uint4 nxt = s_mma[m + 1 < n_mma ? m + 1 : m];      // fetched while this MMA is being issued
+                    const uint64_t da = ((uint64_t)a_desc_hi << 32) | (uint64_t)(a_lo + e.x);
+                    const uint64_t db = ((uint64_t)b_desc_hi << 32) | (uint64_t)(b_lo + e.y);
+                    mma_i8(tmem_base + e.z, da, db, (e.w & 1u) ? idesc_lo : idesc_hi, (i == 0 && (e.w & 2u)) ? 0u : 1u);
+                    e = nxt;
                 }
-                mma_commit(&empty_bar[s]);
+                // release the group of stages this one completes (the commit covers every MMA issued so far)
+                if ((s + 1) % (uint32_t)P.cg == 0) mma_commit(&empty_bar[s / (uint32_t)P.cg]);
+                if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
             }
             if (!timed_out) mma_commit(&acc_bar);
         }
         __syncwarp();
     } else {
+        // ------------------------------------------------------- epilogue
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
-        if (k_iters > 0) {
-            if (!mbar_wait(&acc_bar, 0)) timed_out = true;
-            tc_fence_after();
-        }
+        if (k_iters > 0 && !mbar_wait_warp(&acc_bar, 0)) timed_out = true;
+        tc_fence_after();
         if (!timed_out && k_iters > 0) {
+            const float scale = P.direct ? __fmul_rn(P.qx->scale, P.qg->scale) : 0.0f;
+            long long *part = P.part + (int64_t)blockIdx.x * P.part_stride;
             for (int j = 0; j < n_tiles; ++j) {
-                // row of the accumulator -> (chunk, channel); column -> output channel of g
                 const int at = ag * P.ma + j;
-                const int chunk = row / P.rb_a, cin = row % P.rb_a;
-                bool valid = chunk < chunks_of(at);
-                int64_t base, col_stride;
-                if (!P.conv) {
-                    const int64_t k = (int64_t)at * 128 + row;
-                    valid = valid && k < P.K;
-                    base = k * P.N; col_stride = 1;
-                } else {
-                    const int tap = (at / P.tiles_c) * P.a_chunks + chunk;
-                    const int c = (at % P.tiles_c) * P.rb_a + cin;
-                    valid = valid && c < P.C;
-                    base = (int64_t)tap * P.C + c;                          // [k][tap][c]: + k * taps * C
-                    col_stride = (int64_t)P.taps * P.C;
-                }
+                bool valid = row / P.rb_a < chunks_of(at);
+                const int64_t k = (int64_t)at * 128 + row;                  // plain: output row
+                if (!P.conv) valid = valid && k < P.K;
+                else         valid = valid && (at % P.tiles_c) * P.rb_a + row % P.rb_a < P.C;
+                const long long rterm = (P.direct && valid) ? P.rowterm[k] : 0;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(j * 2 * P.bn);
                 for (int c0 = 0; c0 < P.bn; c0 += 32) {
                     uint32_t rh[32], rl[32];
@@ -201,12 +249,32 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
                     tmem_ld_32x32(t_addr + (uint32_t)(P.bn + c0), rl);
                     tmem_ld_wait();
                     if (!valid) continue;
+                    if (P.direct) {
+                        // the whole reduction is here: zero-points, scale, store
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int64_t n = (int64_t)n0 + c0 + e;
-                        if (n < P.N) {
-                            const long long v = 256ll * (long long)(int)rh[e] + (long long)(int)rl[e];
-                            atomicAdd(P.raw + base + n * col_stride, (unsigned long long)v);
+                        for (int e = 0; e < 32; ++e) {
+                            const int64_t n = (int64_t)n0 + c0 + e;
+                            if (n < P.N) {
+                                const long long acc = 256ll * (long long)(int)rh[e] + (long long)(int)rl[e] + rterm + P.colterm[n];
+                                if (P.acc_out) P.acc_out[k * P.N + n] = acc;
+                                if (P.dW) P.dW[k * P.N + n] = __fmul_rn((float)acc, scale);
+                            }
+                        }
+                    } else if (P.conv) {
+                        // partial block [tile][column][row]: a warp's 32 rows are contiguous, and so are the
+                        // channels the second kernel reads together
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            part[((int64_t)j * P.bn + c0 + e) * 128 + row] = 256ll * (long long)(int)rh[e] + (long long)(int)rl[e];
+                    } else {
+                        // partial block [tile][row][column]
+                        long long *dst = part + ((int64_t)j * 128 + row) * P.bn + c0;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            longlong2 v;
+                            v.x = 256ll * (long long)(int)rh[e] + (long long)(int)rl[e];
+                            v.y = 256ll * (long long)(int)rh[e + 1] + (long long)(int)rl[e + 1];
+                            *reinterpret_cast<longlong2 *>(dst + e) = v;
                         }
                     }
                 }
@@ -225,12 +293,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
 
 // ------------------------------------------------------------ code sums
 // Sums of stored codes per channel and per border class of the pixel the code
-// sits at (bit 1: first row, 2: last row, 4: first column, 8: last column);
-// a plain matrix (plain = 1) keeps every row in class 0.
+// sits at (bit 1: first row, 2: last row, 4: first column, 8: last column).
 // sums[cls][c] (int64, zeroed beforehand).
 template <bool IS_SIGNED>
 __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restrict__ q, int64_t pixels, int H, int W,
-                                                         int C, int plain, unsigned long long *__restrict__ sums)
+                                                         int C, unsigned long long *__restrict__ sums)
 {
     extern __shared__ int s_acc[];                       // [16][C]
     for (int i = threadIdx.x; i < 16 * C; i += 256) s_acc[i] = 0;
@@ -246,9 +313,7 @@ __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restri
             for (int e = 0; e < 16; ++e) interior[e] = 0;
             for (int64_t p = (int64_t)blockIdx.x * rpb + ty; p < pixels; p += (int64_t)gridDim.x * rpb) {
                 const int w = (int)(p % W), h = (int)((p / W) % H);
-                // a plain matrix keeps everything in class 0
-                const int cls = plain ? 0
-                              : (h == 0 ? 1 : 0) | (h == H - 1 ? 2 : 0) | (w == 0 ? 4 : 0) | (w == W - 1 ? 8 : 0);
+                const int cls = (h == 0 ? 1 : 0) | (h == H - 1 ? 2 : 0) | (w == 0 ? 4 : 0) | (w == W - 1 ? 8 : 0);
                 uint4 v = __ldg(reinterpret_cast<const uint4 *>(q + p * C) + g);
                 const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
                 if (cls == 0) {
@@ -275,47 +340,69 @@ __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restri
         if (s_acc[i] != 0) atomicAdd(&sums[i], (unsigned long long)(long long)s_acc[i]);
 }
 
-// Applies the zero-points and dequantises:
+// Plain product, direct epilogue: rowterm[k] = -zg * SX[k] + M*zx*zg, colterm[n] = -zx * (256*SHI[n] + SLO[n]).
+__global__ void wgrad_terms_kernel(const long long *__restrict__ sx, const long long *__restrict__ shi,
+                                   const long long *__restrict__ slo, int64_t M, int64_t N, int64_t K,
+                                   const qbp_qparams *qx, const qbp_qparams *qg, long long *__restrict__ rowterm,
+                                   long long *__restrict__ colterm)
+{
+    const long long zx = qx->zero_point, zg = qg->zero_point;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < K) rowterm[i] = -zg * sx[i] + M * zx * zg;
+    if (i < N) colterm[i] = -zx * (256 * shi[i] + slo[i]);
+}
+
+// Adds the CTAs' partials, applies the zero-points and dequantises:
 //   acc = raw - zg * SX - zx * SG + count * zx * zg
 // where SX / SG / count are taken over the positions at which the tap is inside
 // the image.  Output element e: plain [k][n]; conv [k][tap][c].
-__global__ void wgrad_finalize_kernel(const long long *__restrict__ raw, const long long *__restrict__ sx,
-                                      const long long *__restrict__ shi, const long long *__restrict__ slo, int conv,
-                                      int64_t total, int64_t Mrows, int64_t Nn, int64_t Kk, int Nimg, int H, int W,
-                                      int pad, int R, int S, int C, const qbp_qparams *qx, const qbp_qparams *qg,
-                                      long long *__restrict__ acc_out, float *__restrict__ dW)
+__global__ void __launch_bounds__(256) wgrad_finalize_kernel(const WgradParams P, const long long *__restrict__ sx,
+                                                             const long long *__restrict__ shi,
+                                                             const long long *__restrict__ slo, int64_t total)
 {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= total) return;
-    const long long zx = qx->zero_point, zg = qg->zero_point;
+    const long long zx = P.qx->zero_point, zg = P.qg->zero_point;
     long long SX = 0, SG = 0, count = 0;
-    if (!conv) {
-        const int64_t k = e / Nn, n = e % Nn;
-        for (int cls = 0; cls < 16; ++cls) {
-            SX += sx[cls * Kk + k];
-            SG += 256 * shi[cls * Nn + n] + slo[cls * Nn + n];
-        }
-        count = Mrows;
+    int at, row, n;                                     // accumulator tile, row in it, output column of g
+    if (!P.conv) {
+        const int64_t k = e / P.N;
+        n = (int)(e % P.N);
+        at = (int)(k / 128); row = (int)(k % 128);
+        SX = sx[k];
+        SG = 256 * shi[n] + slo[n];
+        count = P.M;
     } else {
-        const int c = (int)(e % C);
-        const int tap = (int)((e / C) % (R * S));
-        const int k = (int)(e / ((int64_t)C * R * S));
-        const int r = tap / S, s = tap % S;
+        const int c = (int)(e % P.C);
+        const int tap = (int)((e / P.C) % P.taps);
+        n = (int)(e / ((int64_t)P.C * P.taps));
+        const int r = tap / P.S, s = tap % P.S, pad = P.pad;
+        at = (tap / P.a_chunks) * P.tiles_c + c / P.rb_a;
+        row = (tap % P.a_chunks) * P.rb_a + c % P.rb_a;
         // positions of g that see this tap: p - pad + r in [0,H)  <=>  not (r<pad and first row), not (r>pad and last row);
         // positions of x that are seen:      h + pad - r in [0,H)  <=>  not (r<pad and last row),  not (r>pad and first row).
         for (int cls = 0; cls < 16; ++cls) {
             const bool top = cls & 1, bottom = cls & 2, left = cls & 4, right = cls & 8;
             const bool g_ok = !((r < pad && top) || (r > pad && bottom) || (s < pad && left) || (s > pad && right));
             const bool x_ok = !((r < pad && bottom) || (r > pad && top) || (s < pad && right) || (s > pad && left));
-            if (g_ok) SG += 256 * shi[cls * Nn + k] + slo[cls * Nn + k];
-            if (x_ok) SX += sx[cls * C + c];
+            if (g_ok) SG += 256 * shi[cls * P.N + n] + slo[cls * P.N + n];
+            if (x_ok) SX += sx[cls * P.C + c];
         }
-        const long long rows_ok = H - (r < pad ? pad - r : r - pad), cols_ok = W - (s < pad ? pad - s : s - pad);
-        count = (long long)Nimg * (rows_ok > 0 ? rows_ok : 0) * (cols_ok > 0 ? cols_ok : 0);
+        const long long rows_ok = P.H - (r < pad ? pad - r : r - pad), cols_ok = P.W - (s < pad ? pad - s : s - pad);
+        count = (long long)P.Nimg * (rows_ok > 0 ? rows_ok : 0) * (cols_ok > 0 ? cols_ok : 0);
     }
-    const long long acc = raw[e] - zg * SX - zx * SG + count * zx * zg;
-    if (acc_out) acc_out[e] = acc;
-    if (dW) dW[e] = __fmul_rn((float)acc, __fmul_rn(qx->scale, qg->scale));
+    // the CTAs of this element's item
+    const int ag = at / P.ma, j = at % P.ma, tb = n / P.bn, col = n % P.bn;
+    const int item = ag * P.tiles_b + tb;
+    const int full_items = P.ctas_full / P.s_full;
+    const int first = item < full_items ? item * P.s_full : P.ctas_full + (item - full_items) * P.s_last;
+    const int slices = item < full_items ? P.s_full : P.s_last;
+    const int64_t off = P.conv ? ((int64_t)j * P.bn + col) * 128 + row : ((int64_t)j * 128 + row) * P.bn + col;
+    long long raw = 0;
+    for (int sl = 0; sl < slices; ++sl) raw += P.part[(int64_t)(first + sl) * P.part_stride + off];
+    const long long acc = raw - zg * SX - zx * SG + count * zx * zg;
+    if (P.acc_out) P.acc_out[e] = acc;
+    if (P.dW) P.dW[e] = __fmul_rn((float)acc, __fmul_rn(P.qx->scale, P.qg->scale));
 }
 
 // Pixel box of `rows` = bw x bh x bn positions (powers of two) that needs the fewest steps.
@@ -338,92 +425,20 @@ static bool wgrad_conv_supported(const qbp_conv_desc *d)
            d->H > 0 && d->W > 0 && d->C > 0 && d->K > 0 && d->C % 32 == 0 && d->K % 32 == 0;
 }
 
-static size_t wgrad_ws_bytes(const qbp_conv_desc *d, int64_t N, int64_t K)
+// Everything of the launch that does not depend on pointers: tiling, split, workspace.
+struct WgradPlan {
+    WgradParams P;
+    int grid;
+    size_t smem;
+    int bw, bh, bn_img;
+};
+
+static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, WgradPlan &pl)
 {
-    const int64_t outs = d ? (int64_t)d->K * d->R * d->S * d->C : K * N;
-    const int64_t cx = d ? d->C : K, cg = d ? d->K : N;
-    return 256 + align_up(sizeof(int64_t) * outs, 256) + align_up(sizeof(int64_t) * 16 * cx, 256) +
-           2 * align_up(sizeof(int64_t) * 16 * cg, 256);
-}
-
-template <bool IS_SIGNED>
-static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C, bool plain, int64_t *sums, cudaStream_t st)
-{
-    QBP_CUDA_OK(cudaMemsetAsync(sums, 0, sizeof(int64_t) * 16 * C, st));
-    if ((size_t)C * 16 * sizeof(int) > 200 * 1024) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad: more than 3200 channels");
-    const size_t smem = (size_t)C * 16 * sizeof(int);
-    static thread_local bool configured[2] = {false, false};
-    if (smem > 48 * 1024 && !configured[IS_SIGNED]) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(class_sums_kernel<IS_SIGNED>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        configured[IS_SIGNED] = true;
-    }
-    // int32 partials: a thread sees at most pixels / grid * 255 per channel
-    const int cv = C / 16, tw = cv < 256 ? cv : 256, rpb = 256 / tw;
-    int64_t grid = std::min<int64_t>((pixels + rpb - 1) / rpb, (int64_t)sm_count() * 4);
-    grid = std::max<int64_t>(grid, pixels / (1 << 22) + 1);
-    QBP_TRACE_BEGIN(st);
-    class_sums_kernel<IS_SIGNED><<<(unsigned)grid, 256, smem, st>>>((const uint8_t *)q, pixels, H, W, C, plain ? 1 : 0, (unsigned long long *)sums);
-    QBP_LAUNCH_OK("class_sums_kernel");
-    return QBP_OK;
-}
-
-}  // namespace qbp
-
-using namespace qbp;
-
-extern "C" __attribute__((visibility("default"))) size_t qbp_wgrad_s16_workspace_bytes(const qbp_conv_desc *d, int64_t M,
-                                                                                      int64_t N, int64_t K)
-{
-    (void)M;
-    if (d && !wgrad_conv_supported(d)) return 0;
-    return wgrad_ws_bytes(d, N > 0 ? N : 1, K > 0 ? K : 1);
-}
-
-extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
-                                                                   const int8_t *x, const qbp_qparams *qx,
-                                                                   const int8_t *g_hi, const uint8_t *g_lo,
-                                                                   const qbp_qparams *qg16, int64_t *acc_out, float *dW,
-                                                                   void *ws, size_t ws_bytes, void *stream)
-{
-    cudaStream_t st = (cudaStream_t)stream;
-    if (!x || !g_hi || !g_lo || !qx || !qg16) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: NULL operand");
-    if (!acc_out && !dW) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: acc_out and dW are both NULL");
-    if (!aligned16(x) || !aligned16(g_hi) || !aligned16(g_lo))
-        return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: operands must be 16-byte aligned");
-    if (d) {
-        if (!wgrad_conv_supported(d))
-            return fail(QBP_ERR_UNSUPPORTED_SHAPE,
-                        "wgrad_s16: needs stride 1, R = S in {1,3}, pad = (R-1)/2, C and K multiples of 32");
-        M = (int64_t)d->N * d->H * d->W; N = d->K; K = d->C;
-    } else {
-        if (M <= 0 || N <= 0 || K <= 0) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: M, N, K must be positive");
-        if (N % 16 || K % 16) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad_s16: N and K must be multiples of 16");
-    }
-    if (!ws || ws_bytes < wgrad_ws_bytes(d, N, K))
-        return fail(QBP_ERR_WORKSPACE, "wgrad_s16: workspace of %zu bytes needed, %zu given", wgrad_ws_bytes(d, N, K), ws_bytes);
-
-    const int64_t outs = d ? (int64_t)d->K * d->R * d->S * d->C : K * N;
-    WsCarver w(ws, ws_bytes);
-    int *status = w.take<int>(1);
-    int64_t *raw = w.take<int64_t>(outs);
-    int64_t *sx = w.take<int64_t>(16 * K);
-    int64_t *shi = w.take<int64_t>(16 * N);
-    int64_t *slo = w.take<int64_t>(16 * N);
-
-    const int Hc = d ? d->H : 1, Wc = d ? d->W : 1;
-    int rc = launch_class_sums<true>(x, M, Hc, Wc, (int)K, d == nullptr, sx, st);
-    if (rc) return rc;
-    rc = launch_class_sums<true>(g_hi, M, Hc, Wc, (int)N, d == nullptr, shi, st);
-    if (rc) return rc;
-    rc = launch_class_sums<false>(g_lo, M, Hc, Wc, (int)N, d == nullptr, slo, st);
-    if (rc) return rc;
-    QBP_CUDA_OK(cudaMemsetAsync(raw, 0, sizeof(int64_t) * outs, st));
-    QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
-
-    WgradParams P{};
+    WgradParams &P = pl.P;
+    P = WgradParams{};
     P.conv = d ? 1 : 0;
     P.M = M; P.N = N; P.K = K;
-    P.raw = (unsigned long long *)raw; P.status = status;
     // g side: one swizzled row holds bn output channels
     const uint32_t rb_b = N >= 128 ? 128u : N >= 64 ? 64u : 32u;
     P.bn = (int)rb_b;
@@ -446,58 +461,189 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
     P.a_groups = (P.a_tiles + P.ma - 1) / P.ma;
     int cols = 32; while (cols < P.ma * 2 * P.bn) cols <<= 1;
     P.tmem_cols = cols;
-    // reduction rows per stage: 128, or 64 when that is what it takes to keep four stages in flight
-    uint32_t kr = 128;
-    if ((200u * 1024u) / (kr * (rb_a * P.a_chunks * P.ma + 2 * rb_b)) < 4) kr = 64;
+    // reduction rows per stage: 64 keeps the ring deep and the release groups fine-grained
+    const uint32_t kr = 64;
     P.kr = (int)kr;
     P.a_chunk_bytes = kr * rb_a;
     P.a = layout_mnmajor(kr, rb_a, (uint32_t)P.a_chunks, P.a_chunk_bytes);
     P.b = layout_mnmajor(kr, rb_b, 1, 0);
     P.idesc_hi = make_idesc(true, true, 1, 1, 128, (uint32_t)P.bn);
     P.idesc_lo = make_idesc(true, false, 1, 1, 128, (uint32_t)P.bn);
-
     if (!d) {
         P.iters_total = (int)((M + kr - 1) / kr);
-        if ((rc = make_map_2d(&P.mapX, x, M, K, kr, rb_a))) return rc;
-        if ((rc = make_map_2d(&P.mapHi, g_hi, M, N, kr, rb_b))) return rc;
-        if ((rc = make_map_2d(&P.mapLo, g_lo, M, N, kr, rb_b))) return rc;
+        pl.bw = pl.bh = pl.bn_img = 0;
     } else {
         int bwl = 0, bhl = 0;
         pick_pixel_box_w((int)kr, d->N, d->H, d->W, bwl, bhl);
         P.bw_log2 = bwl; P.bh_log2 = bhl;
-        const int bw = 1 << bwl, bh = 1 << bhl, bn_img = (int)kr >> (bwl + bhl);
-        P.tiles_w = (d->W + bw - 1) / bw; P.tiles_h = (d->H + bh - 1) / bh;
-        P.iters_total = P.tiles_w * P.tiles_h * ((d->N + bn_img - 1) / bn_img);
-        if ((rc = make_map_nhwc(&P.mapX, x, d->N, d->H, d->W, d->C, bn_img, bh, bw, rb_a))) return rc;
-        if ((rc = make_map_nhwc(&P.mapHi, g_hi, d->N, d->H, d->W, d->K, bn_img, bh, bw, rb_b))) return rc;
-        if ((rc = make_map_nhwc(&P.mapLo, g_lo, d->N, d->H, d->W, d->K, bn_img, bh, bw, rb_b))) return rc;
+        pl.bw = 1 << bwl; pl.bh = 1 << bhl; pl.bn_img = (int)kr >> (bwl + bhl);
+        P.tiles_w = (d->W + pl.bw - 1) / pl.bw; P.tiles_h = (d->H + pl.bh - 1) / pl.bh;
+        P.iters_total = P.tiles_w * P.tiles_h * ((d->N + pl.bn_img - 1) / pl.bn_img);
+        P.d_tiles_w = make_fastdiv(P.tiles_w); P.d_tiles_h = make_fastdiv(P.tiles_h);
     }
-    // split the reduction: at most 65536 rows per CTA, and enough CTAs to fill the machine twice
-    const int out_items = P.a_groups * P.tiles_b;
-    const int max_iters = 65536 / (int)kr;
-    int slices = (P.iters_total + max_iters - 1) / max_iters;
-    slices = std::max(slices, std::min(P.iters_total, std::max(1, 2 * sm_count() / out_items)));
-    P.slices = std::max(1, slices);
-
+    // pipeline: stages of kr rows; one commit releases `cg` stages (at least ~24 MMAs between commits when the ring allows)
     const uint32_t stage_bytes = P.a_chunk_bytes * P.a_chunks * P.ma + 2 * P.b.tile_bytes;
-    int stages = std::max(2, std::min<int>(kWgMaxStages, (200 * 1024) / stage_bytes));
-    P.stages = stages;
-    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    int stages = std::max(2, std::min<int>(kWgMaxStages, (int)((kWgSmem - 1024) / stage_bytes)));
+    const int mmas = P.ma * (int)(kr / 32) * 2;
+    int cg = 1;
+    while (cg * mmas < 24 && stages / (cg + 1) >= 2) ++cg;
+    stages -= stages % cg;
+    P.stages = stages; P.cg = cg;
+    pl.smem = (size_t)stages * stage_bytes + 1024;
+    // split of the reductions: at most 65536 rows per CTA; with few items, enough slices to fill the machine
+    // once, in proportion to an item's cost per reduction step: a fixed part (waits, the share of a commit)
+    // worth about four MMAs, plus its MMAs
+    const int max_iters = 65536 / (int)kr;
+    const int min_slices = (P.iters_total + max_iters - 1) / max_iters;
+    const int n_last = P.a_tiles - (P.a_groups - 1) * P.ma;                 // A tiles of the last group
+    auto cost = [&](int tiles) { return (int64_t)(4 + tiles * (int)(kr / 32) * 2); };
+    const int64_t weight = ((int64_t)(P.a_groups - 1) * cost(P.ma) + cost(n_last)) * P.tiles_b;
+    const int T = sm_count();
+    auto slices_for = [&](int tiles) {
+        int64_t s = (int64_t)T * cost(tiles) / weight;
+        s = std::max<int64_t>(s, min_slices);
+        s = std::max<int64_t>(1, std::min<int64_t>(s, P.iters_total));
+        return (int)s;
+    };
+    P.s_full = slices_for(P.ma);
+    P.s_last = slices_for(n_last);
+    P.ctas_full = (P.a_groups - 1) * P.tiles_b * P.s_full;
+    pl.grid = P.ctas_full + P.tiles_b * P.s_last;
+    P.direct = (!d && P.s_full == 1 && P.s_last == 1) ? 1 : 0;
+    P.part_stride = (int64_t)P.ma * 128 * P.bn;
+}
+
+static size_t wgrad_ws_bytes(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K)
+{
+    WgradPlan pl;
+    plan_wgrad(d, M, N, K, pl);
+    const int64_t cx = d ? d->C : K, cg = d ? d->K : N;
+    const size_t sums = align_up(sizeof(int64_t) * 16 * cx, 256) + 2 * align_up(sizeof(int64_t) * 16 * cg, 256);
+    const size_t terms = align_up(sizeof(int64_t) * cx, 256) + align_up(sizeof(int64_t) * cg, 256);
+    const size_t part = pl.P.direct ? 0 : align_up(sizeof(int64_t) * (size_t)pl.grid * (size_t)pl.P.part_stride, 256);
+    return 256 + sums + terms + part;
+}
+
+template <bool IS_SIGNED>
+static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C, int64_t *sums, cudaStream_t st)
+{
+    QBP_CUDA_OK(cudaMemsetAsync(sums, 0, sizeof(int64_t) * 16 * C, st));
+    if ((size_t)C * 16 * sizeof(int) > 200 * 1024) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad: more than 3200 channels");
+    const size_t smem = (size_t)C * 16 * sizeof(int);
+    static thread_local bool configured[2] = {false, false};
+    if (smem > 48 * 1024 && !configured[IS_SIGNED]) {
+        QBP_CUDA_OK(cudaFuncSetAttribute(class_sums_kernel<IS_SIGNED>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        configured[IS_SIGNED] = true;
+    }
+    // int32 partials: a thread sees at most pixels / grid * 255 per channel
+    const int cv = C / 16, tw = cv < 256 ? cv : 256, rpb = 256 / tw;
+    int64_t grid = std::min<int64_t>((pixels + rpb - 1) / rpb, (int64_t)sm_count() * 4);
+    grid = std::max<int64_t>(grid, pixels / (1 << 22) + 1);
+    QBP_TRACE_BEGIN(st);
+    class_sums_kernel<IS_SIGNED><<<(unsigned)grid, 256, smem, st>>>((const uint8_t *)q, pixels, H, W, C, (unsigned long long *)sums);
+    QBP_LAUNCH_OK("class_sums_kernel");
+    return QBP_OK;
+}
+
+}  // namespace qbp
+
+using namespace qbp;
+
+extern "C" __attribute__((visibility("default"))) size_t qbp_wgrad_s16_workspace_bytes(const qbp_conv_desc *d, int64_t M,
+                                                                                      int64_t N, int64_t K)
+{
+    if (d) {
+        if (!wgrad_conv_supported(d)) return 0;
+        M = (int64_t)d->N * d->H * d->W; N = d->K; K = d->C;
+    }
+    return wgrad_ws_bytes(d, M > 0 ? M : 1, N > 0 ? N : 1, K > 0 ? K : 1);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
+                                                                   const int8_t *x, const qbp_qparams *qx,
+                                                                   const int8_t *g_hi, const uint8_t *g_lo,
+                                                                   const qbp_qparams *qg16, int64_t *acc_out, float *dW,
+                                                                   void *ws, size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!x || !g_hi || !g_lo || !qx || !qg16) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: NULL operand");
+    if (!acc_out && !dW) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: acc_out and dW are both NULL");
+    if (!aligned16(x) || !aligned16(g_hi) || !aligned16(g_lo))
+        return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: operands must be 16-byte aligned");
+    if (d) {
+        if (!wgrad_conv_supported(d))
+            return fail(QBP_ERR_UNSUPPORTED_SHAPE,
+                        "wgrad_s16: needs stride 1, R = S in {1,3}, pad = (R-1)/2, C and K multiples of 32");
+        M = (int64_t)d->N * d->H * d->W; N = d->K; K = d->C;
+    } else {
+        if (M <= 0 || N <= 0 || K <= 0) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: M, N, K must be positive");
+        if (N % 16 || K % 16) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad_s16: N and K must be multiples of 16");
+        if (M > (int64_t)INT32_MAX || N > (int64_t)INT32_MAX || K > (int64_t)INT32_MAX)
+            return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad_s16: extent too large");
+    }
+    if (!ws || ws_bytes < wgrad_ws_bytes(d, M, N, K))
+        return fail(QBP_ERR_WORKSPACE, "wgrad_s16: workspace of %zu bytes needed, %zu given", wgrad_ws_bytes(d, M, N, K), ws_bytes);
+
+    WgradPlan pl;
+    plan_wgrad(d, M, N, K, pl);
+    WgradParams &P = pl.P;
+    const int64_t outs = d ? (int64_t)d->K * d->R * d->S * d->C : K * N;
+    WsCarver w(ws, ws_bytes);
+    int *status = w.take<int>(1);
+    int64_t *sx = w.take<int64_t>(16 * K);
+    int64_t *shi = w.take<int64_t>(16 * N);
+    int64_t *slo = w.take<int64_t>(16 * N);
+    int64_t *rowterm = w.take<int64_t>(K);
+    int64_t *colterm = w.take<int64_t>(N);
+    int64_t *part = P.direct ? nullptr : w.take<int64_t>((size_t)pl.grid * (size_t)P.part_stride);
+
+    // code sums for the zero-point terms: per border class (convolution) or plain column sums
+    int rc;
+    if (d) {
+        if ((rc = launch_class_sums<true>(x, M, d->H, d->W, (int)K, sx, st))) return rc;
+        if ((rc = launch_class_sums<true>(g_hi, M, d->H, d->W, (int)N, shi, st))) return rc;
+        if ((rc = launch_class_sums<false>(g_lo, M, d->H, d->W, (int)N, slo, st))) return rc;
+    } else {
+        if ((rc = launch_colsum(x, true, M, K, sx, st))) return rc;
+        if ((rc = launch_colsum(g_hi, true, M, N, shi, st))) return rc;
+        if ((rc = launch_colsum(g_lo, false, M, N, slo, st))) return rc;
+        if (P.direct) {
+            const int64_t mx = std::max(K, N);
+            QBP_TRACE_BEGIN(st);
+            wgrad_terms_kernel<<<(unsigned)((mx + 255) / 256), 256, 0, st>>>((const long long *)sx, (const long long *)shi,
+                                                                            (const long long *)slo, M, N, K, qx, qg16,
+                                                                            (long long *)rowterm, (long long *)colterm);
+            QBP_LAUNCH_OK("wgrad_terms_kernel");
+        }
+    }
+    QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
+
+    P.part = (long long *)part; P.status = status;
+    P.rowterm = (const long long *)rowterm; P.colterm = (const long long *)colterm;
+    P.qx = qx; P.qg = qg16; P.acc_out = (long long *)acc_out; P.dW = dW;
+    const uint32_t kr = (uint32_t)P.kr, rb_a = (uint32_t)P.rb_a, rb_b = (uint32_t)P.bn;
+    if (!d) {
+        if ((rc = make_map_2d(&P.mapX, x, M, K, kr, rb_a))) return rc;
+        if ((rc = make_map_2d(&P.mapHi, g_hi, M, N, kr, rb_b))) return rc;
+        if ((rc = make_map_2d(&P.mapLo, g_lo, M, N, kr, rb_b))) return rc;
+    } else {
+        if ((rc = make_map_nhwc(&P.mapX, x, d->N, d->H, d->W, d->C, pl.bn_img, pl.bh, pl.bw, rb_a))) return rc;
+        if ((rc = make_map_nhwc(&P.mapHi, g_hi, d->N, d->H, d->W, d->K, pl.bn_img, pl.bh, pl.bw, rb_b))) return rc;
+        if ((rc = make_map_nhwc(&P.mapLo, g_lo, d->N, d->H, d->W, d->K, pl.bn_img, pl.bh, pl.bw, rb_b))) return rc;
+    }
     static thread_local bool configured = false;
     if (!configured) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgSmem));
         configured = true;
     }
     QBP_TRACE_BEGIN(st);
-    qbp_wgrad_kernel<<<P.slices * out_items, kWgThreads, smem, st>>>(P);
+    qbp_wgrad_kernel<<<pl.grid, kWgThreads, pl.smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_wgrad_kernel");
-
-    const int blocks = (int)((outs + 255) / 256);
-    QBP_TRACE_BEGIN(st);
-    wgrad_finalize_kernel<<<blocks, 256, 0, st>>>((const long long *)raw, (const long long *)sx, (const long long *)shi,
-                                                  (const long long *)slo, P.conv, outs, M, N, K, d ? d->N : 0, Hc, Wc,
-                                                  d ? d->pad : 0, d ? d->R : 1, d ? d->S : 1, d ? d->C : (int)K, qx, qg16,
-                                                  (long long *)acc_out, dW);
-    QBP_LAUNCH_OK("wgrad_finalize_kernel");
+    if (!P.direct) {
+        const int blocks = (int)((outs + 255) / 256);
+        QBP_TRACE_BEGIN(st);
+        wgrad_finalize_kernel<<<blocks, 256, 0, st>>>(P, (const long long *)sx, (const long long *)shi, (const long long *)slo, outs);
+        QBP_LAUNCH_OK("wgrad_finalize_kernel");
+    }
     return QBP_OK;
 }
