@@ -97,23 +97,22 @@ def conv_workload(batch):
     return synth.conv3x3_layer(batch=batch, hw=HW, c_in=CIN, k_out=COUT)
 
 
-# Algorithmic HBM bytes per element of the [N,H,W,64] activation (or int8 ops) of each kernel of a step, in
-# launch order; E = batch*56*56*64 elements.  (name, bytes per element, ops per element)
+# Algorithmic HBM bytes per element of the [N,H,W,64] activation (E = batch*56*56*64 elements) and int8 ops per
+# element of each kernel of a step, keyed by (kernel name, occurrence within the step); kernels not listed
+# move O(channels) or O(pixels) bytes only.
 OPS_PER_ELEMENT_CONV = 2 * 9 * CIN          # 2*K per output element of fprop / dgrad
-STEP_KERNELS = [
-    ("range_partial_kernel", 4, 0), ("range_finalize_kernel", 0, 0), ("quantize_kernel", 5, 0),        # x
-    ("range_partial_kernel", 0, 0), ("range_finalize_kernel", 0, 0), ("quantize_kernel", 0, 0),        # w (tiny)
-    ("rowsum_kernel", 1, 0), ("rowsum_kernel", 0, 0), ("conv_colterm_kernel", 0, 0),
-    ("qbp_mma_kernel", 5, OPS_PER_ELEMENT_CONV),                                                        # fprop
-    ("bn_stats_kernel", 4, 0), ("bn_stats_finalize_kernel", 0, 0), ("bn_apply_kernel", 8, 0),
-    ("bn_bwd_stats_kernel", 8, 0), ("bn_bwd_finalize_kernel", 0, 0), ("bn_bwd_apply_kernel", 12, 0),
-    ("range_partial_kernel", 4, 0), ("range_finalize_kernel", 0, 0), ("quantize_kernel", 7, 0),        # bifurcate
-    ("rowsum_kernel", 1, 0), ("colsum_kernel", 0, 0), ("conv_colterm_kernel", 0, 0),
-    ("qbp_mma_kernel", 5, OPS_PER_ELEMENT_CONV),                                                        # dgrad
-    ("class_sums_kernel", 1, 0), ("class_sums_kernel", 1, 0), ("class_sums_kernel", 1, 0),
-    ("qbp_wgrad_kernel", 3, 2 * OPS_PER_ELEMENT_CONV),                                                  # wgrad: two int8 products
-    ("wgrad_finalize_kernel", 0, 0),
-]
+KERNEL_WORK = {
+    ("range_partial_kernel", 0): (4, 0), ("quantize_kernel", 0): (5, 0),            # x (occurrence 1: the filter, tiny)
+    ("rowsum_kernel", 0): (1, 0),                                                   # channel sums of the x codes
+    ("qbp_mma_kernel", 0): (5, OPS_PER_ELEMENT_CONV),                               # fprop: 1 B codes in, 4 B fp32 out
+    ("bn_stats_kernel", 0): (4, 0), ("bn_apply_kernel", 0): (8, 0),
+    ("bn_bwd_stats_kernel", 0): (8, 0), ("bn_bwd_apply_kernel", 0): (12, 0),
+    ("range_partial_kernel", 2): (4, 0), ("quantize_kernel", 2): (7, 0),            # bifurcation: 4 B in, 1 + 2 B out
+    ("rowsum_kernel", 2): (1, 0),                                                   # channel sums of the 8-bit gradient codes
+    ("qbp_mma_kernel", 1): (5, OPS_PER_ELEMENT_CONV),                               # dgrad
+    ("class_sums_kernel", 0): (1, 0), ("class_sums_kernel", 1): (1, 0), ("class_sums_kernel", 2): (1, 0),
+    ("qbp_wgrad_kernel", 0): (3, 2 * OPS_PER_ELEMENT_CONV),                         # two int8 products per 16x8-bit product
+}
 
 
 def run_ours(args):
@@ -206,11 +205,14 @@ def run_ours(args):
     per_step = len(recs) // trace_steps
     launches_per_step = per_step
     kernels = []
-    if per_step == len(STEP_KERNELS):
-        for i, (name, bpe, ope) in enumerate(STEP_KERNELS):
-            times = [recs[s * per_step + i][1] for s in range(trace_steps)]
-            assert all(recs[s * per_step + i][0] == name for s in range(trace_steps)), (i, name)
-            kernels.append({"kernel": name, "ms": sum(times) / len(times), "bytes": bpe * E, "ops": ope * E})
+    seen = {}
+    for i in range(per_step):
+        name = recs[i][0]
+        occ = seen.get(name, 0); seen[name] = occ + 1
+        assert all(recs[st * per_step + i][0] == name for st in range(trace_steps)), (i, name)
+        times = [recs[st * per_step + i][1] for st in range(trace_steps)]
+        bpe, ope = KERNEL_WORK.get((name, occ), (0, 0))
+        kernels.append({"kernel": name, "ms": sum(times) / len(times), "bytes": bpe * E, "ops": ope * E})
     traced_ms = sum(k["ms"] for k in kernels) or 1.0
     peaks, peaks_kind = measured_peaks()
     hbm_peak = float(peaks["hbm_gbs"])

@@ -56,6 +56,14 @@ static size_t step_scratch_bytes(const qbp_layer_desc *L, const LayerShape &s)
     return align_up(b, 256);
 }
 
+// Buffers that live across steps, behind the shared step scratch: the per-row sums of the codes feeding the
+// next product (written by the quantiser that makes the codes) and the range partials of the gradient
+// (written by the Range BN backward pass that makes the gradient).
+static size_t chained_bytes(const LayerShape &s)
+{
+    return align_up(sizeof(int32_t) * (size_t)s.rows, 256) + align_up(sizeof(float2) * rangebn_range_parts_capacity(s.cout), 256);
+}
+
 }  // namespace qbp
 
 using namespace qbp;
@@ -64,7 +72,7 @@ extern "C" __attribute__((visibility("default"))) size_t qbp_layer_workspace_byt
 {
     LayerShape s;
     if (layer_shape(L, s)) return 0;
-    return step_scratch_bytes(L, s);
+    return step_scratch_bytes(L, s) + chained_bytes(s);
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_layer_desc *L, const float *x,
@@ -86,16 +94,18 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_la
     const size_t scratch = step_scratch_bytes(L, s);
 
     // weights and activations: nearest rounding, clamping values = min and max (Appendix B)
+    // (convolution: the quantiser also leaves each pixel's code sum for the zero-point correction of the product)
+    int32_t *row_sums = reinterpret_cast<int32_t *>(static_cast<char *>(ws) + scratch);
     rc = qbp_quantize_s8(x, s.rows, s.cin, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, saved->x_codes, saved->qx,
-                         nullptr, nullptr, ws, scratch, stream);
+                         s.conv ? row_sums : nullptr, nullptr, ws, scratch, stream);
     if (rc) return rc;
     const int64_t w_rows = s.conv ? (int64_t)L->conv.K * L->conv.R * L->conv.S : s.cin;
     rc = qbp_quantize_s8(w, w_rows, s.w_elems / w_rows, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr,
                          saved->w_codes, saved->qw, nullptr, nullptr, ws, scratch, stream);
     if (rc) return rc;
     if (s.conv)
-        rc = qbp_conv_s8_implicit(QBP_CONV_FPROP, &L->conv, saved->x_codes, saved->qx, saved->w_codes, saved->qw,
-                                  nullptr, saved->z, ws, scratch, stream);
+        rc = conv_s8_impl(QBP_CONV_FPROP, &L->conv, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr, saved->z,
+                          row_sums, ws, scratch, (cudaStream_t)stream);
     else
         rc = qbp_gemm_s8(0, 0, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr,
                          saved->z, ws, scratch, stream);
@@ -125,16 +135,20 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     uint8_t *glo = saved->g_lo;
     qbp_qparams *qp8 = saved->qg8, *qp16 = saved->qg16;
 
-    rc = qbp_rangebn_bwd(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
-                         saved->save_max, g, dgamma, dbeta, ws, scratch, stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t *row_sums = reinterpret_cast<int32_t *>(static_cast<char *>(ws) + scratch);
+    float2 *range_parts = reinterpret_cast<float2 *>(static_cast<char *>(ws) + scratch + align_up(sizeof(int32_t) * (size_t)s.rows, 256));
+    // the pass that writes the gradient also leaves its range (Section 4: no extra scan for the quantiser)
+    int nparts = 0;
+    rc = rangebn_bwd_impl(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
+                          saved->save_max, g, dgamma, dbeta, ws, scratch, range_parts, &nparts, st);
     if (rc) return rc;
     // two copies of the gradient: 8 bits for the layer gradient, 16 bits for the weight gradient
-    rc = qbp_bifurcate(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8, nullptr, ghi, glo, qp16, ws,
-                       scratch, stream);
+    rc = bifurcate_with_range_partials(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
+                                       s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st);
     if (rc) return rc;
     if (s.conv) {
-        rc = qbp_conv_s8_implicit(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, ws, scratch,
-                                  stream);
+        rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, ws, scratch, st);
         if (rc) return rc;
         return qbp_wgrad_s16(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, ws, scratch, stream);
     }

@@ -804,7 +804,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
                                     const int8_t *wgt, const qbp_qparams *q_w, int32_t *acc_out, float *out, void *ws,
                                     size_t ws_bytes, void *stream)
 {
-    cudaStream_t st = (cudaStream_t)stream;
+    return conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
+                      const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, void *ws,
+                      size_t ws_bytes, cudaStream_t st)
+{
     if (!d) return fail(QBP_ERR_INVALID_ARG, "conv_s8: descriptor is NULL");
     if (mode != QBP_CONV_FPROP && mode != QBP_CONV_DGRAD) return fail(QBP_ERR_INVALID_ARG, "conv_s8: bad mode");
     if (!conv_supported(d))
@@ -833,8 +839,9 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
     int32_t *colterm = w.take<int32_t>(16 * nmax);
     int64_t *wsum = w.take<int64_t>((int64_t)taps * nmax);
 
-    int rc = launch_rowsum(in, true, pix, Cred, chan_sum, st);
-    if (rc) return rc;
+    int rc = QBP_OK;
+    if (in_chan_sum) chan_sum = const_cast<int32_t *>(in_chan_sum);
+    else if ((rc = launch_rowsum(in, true, pix, Cred, chan_sum, st))) return rc;
     if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
     else        rc = launch_colsum(wgt, true, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
     if (rc) return rc;

@@ -13,6 +13,23 @@ namespace qbp {
 int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int32_t *sums, cudaStream_t st);
 int launch_colsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st);
 
+// ---- pieces the whole-layer composition chains without a pass of their own ------
+// Range BN backward that also leaves per-block (min, max) of dx (qbp_rangebn.cu), and the gradient
+// bifurcation that starts from such partials instead of scanning (qbp_quant.cu).
+int rangebn_bwd_impl(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma, const float *beta,
+                     int relu, const float *save_mean, const float *save_min, const float *save_max, float *dx,
+                     float *dgamma, float *dbeta, void *ws, size_t ws_bytes, float2 *range_parts, int *nparts,
+                     cudaStream_t st);
+size_t rangebn_range_parts_capacity(int64_t C);
+int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
+                                  uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
+                                  uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st);
+// The convolution products with the per-pixel channel sums of the input codes supplied by the caller
+// (nullable: computed here) (qbp_mma.cu).
+int conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
+                 const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, void *ws,
+                 size_t ws_bytes, cudaStream_t st);
+
 // ---- TMA tensor maps ---------------------------------------------------------
 // A dense byte matrix [rows x cols] (cols innermost) read in boxes of
 // box_cols x box_rows; box_cols in {32, 64, 128} selects the matching swizzle.

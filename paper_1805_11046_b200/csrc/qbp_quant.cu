@@ -211,6 +211,9 @@ struct QuantOut {
     int16_t *q16;    // 16-bit codes (nullable)
     int8_t *hi;      // high byte of the 16-bit code (nullable)
     uint8_t *lo;     // low byte (nullable)
+    int32_t *rowsum8;   // sums of the stored 8-bit codes over each row of `cols` (nullable; vector path only)
+    int rs_group;       // lanes that share a row: cols / 4, a power of two <= 32
+    int rs_shift;       // log2(rs_group)
 };
 
 struct QParamsReg { float inv, zp_u; };
@@ -287,6 +290,10 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
             if (ok[u]) v[u] = __ldg(reinterpret_cast<const float4 *>(x) + j);
         }
 #pragma unroll
+        int rs[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) rs[u] = 0;
+#pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             if (!ok[u]) continue;
             const int64_t j = base + u * kThreads + threadIdx.x;
@@ -306,6 +313,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                     packed |= (uint32_t)((code ^ 0x80) & 0xFF) << (8 * e);
                 }
                 reinterpret_cast<uint32_t *>(o.q8)[j] = packed;
+                if (o.rowsum8) rs[u] = __dp4a((int)packed, 0x01010101, 0);
             }
             if (want16) {
                 uint32_t r[4] = {0, 0, 0, 0};
@@ -327,6 +335,18 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                 if (o.lo)
                     reinterpret_cast<uint32_t *>(o.lo)[j] =
                         (s[0] & 0xFF) | ((s[1] & 0xFF) << 8) | ((s[2] & 0xFF) << 16) | ((s[3] & 0xFF) << 24);
+            }
+        }
+        if (o.rowsum8) {
+            // a row is rs_group consecutive lanes (groups are aligned: the lane index is j mod 32)
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                int sum = rs[u];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1)
+                    if (off < o.rs_group) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                const int64_t j = base + u * kThreads + threadIdx.x;
+                if (ok[u] && (threadIdx.x & (o.rs_group - 1)) == 0) o.rowsum8[j >> o.rs_shift] = sum;
             }
         }
     }
@@ -458,6 +478,7 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
     const bool vec = aligned16(x) && (!perch || cols % 4 == 0) &&
                      (!o.q8 || ((uintptr_t)o.q8 & 3) == 0) && (!o.q16 || ((uintptr_t)o.q16 & 7) == 0) &&
                      (!o.hi || ((uintptr_t)o.hi & 3) == 0) && (!o.lo || ((uintptr_t)o.lo & 3) == 0);
+    if (o.rowsum8 && !vec) return fail(QBP_ERR_INVALID_ARG, "quantize: fused row sums need the vector path");
     const int64_t per_block = (int64_t)kThreads * (vec ? 4 * kUnroll : 1);
     const bool sr = rounding == QBP_ROUND_STOCHASTIC;
     const int bps = vec ? (sr ? blocks_per_sm(quantize_kernel<true, 4>, kThreads) : blocks_per_sm(quantize_kernel<false, 4>, kThreads))
@@ -475,6 +496,15 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
     }
     QBP_LAUNCH_OK("quantize_kernel");
     return QBP_OK;
+}
+
+// Whether the quantising kernel itself can emit the row sums of its 8-bit codes: per-tensor, 16-byte aligned
+// tensors whose rows are 4, 8, ..., 128 elements (a row is then a power-of-two group of lanes of one warp).
+static bool can_fuse_rowsums(const float *x, const void *q8, int64_t cols, const QuantOut &o)
+{
+    const int64_t g = cols / 4;
+    return cols % 4 == 0 && g >= 1 && g <= 32 && (g & (g - 1)) == 0 && aligned16(x) && ((uintptr_t)q8 & 3) == 0 &&
+           (!o.q16 || ((uintptr_t)o.q16 & 7) == 0) && (!o.hi || ((uintptr_t)o.hi & 3) == 0) && (!o.lo || ((uintptr_t)o.lo & 3) == 0);
 }
 
 // Row / column sums of stored codes; used by the quantiser's optional outputs
@@ -593,6 +623,31 @@ static int static_scratch_address(void **out)
     return QBP_OK;
 }
 
+// The quantising half of the bifurcation, once qp8 / qp16 are known.
+static int bifurcate_tail(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
+                          uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo,
+                          qbp_qparams *qp16, cudaStream_t st)
+{
+    QuantOut o = {q8, nullptr, hi, lo, nullptr, 0, 0};
+    const bool fused = row_sums8 && rows * cols > 0 && can_fuse_rowsums(g, q8, cols, o);
+    if (fused) { o.rowsum8 = row_sums8; o.rs_group = (int)(cols / 4); o.rs_shift = 31 - __builtin_clz((unsigned)o.rs_group); }
+    int rc = launch_quantize(g, rows * cols, cols, 0, QBP_ROUND_STOCHASTIC, qp8, tensor_id8, qp16, tensor_id16, seed, o, st);
+    if (rc) return rc;
+    if (row_sums8 && !fused) return launch_rowsum(q8, true, rows, cols, row_sums8, st);
+    return QBP_OK;
+}
+
+// Bifurcation of a gradient whose range partials (min, max per block) were left by the kernel that wrote it.
+int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
+                                  uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
+                                  uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st)
+{
+    QBP_TRACE_BEGIN(st);
+    range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
+    QBP_LAUNCH_OK("range_finalize_kernel");
+    return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st);
+}
+
 }  // namespace qbp
 
 using namespace qbp;
@@ -635,10 +690,12 @@ extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8(const floa
     if (!q && rows * cols > 0) return fail(QBP_ERR_INVALID_ARG, "quantize_s8: q is NULL");
     if ((row_sums || col_sums) && granularity != QBP_PER_TENSOR)
         return fail(QBP_ERR_INVALID_ARG, "quantize_s8: row/column sums are per-tensor only");
-    QuantOut o = {q, nullptr, nullptr, nullptr};
+    QuantOut o = {q, nullptr, nullptr, nullptr, nullptr, 0, 0};
+    const bool fused = row_sums && rows * cols > 0 && can_fuse_rowsums(x, q, cols, o);
+    if (fused) { o.rowsum8 = row_sums; o.rs_group = (int)(cols / 4); o.rs_shift = 31 - __builtin_clz((unsigned)o.rs_group); }
     int rc = quantize_any(8, x, rows, cols, granularity, rounding, seed, tensor_id, range_in, o, qp_out, ws, ws_bytes, st);
     if (rc) return rc;
-    if (row_sums) { rc = launch_rowsum(q, true, rows, cols, row_sums, st); if (rc) return rc; }
+    if (row_sums && !fused) { rc = launch_rowsum(q, true, rows, cols, row_sums, st); if (rc) return rc; }
     if (col_sums) { rc = launch_colsum(q, true, rows, cols, col_sums, st); if (rc) return rc; }
     return QBP_OK;
 }
@@ -648,7 +705,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_quantize_s16(const flo
                                 int8_t *hi, uint8_t *lo, qbp_qparams *qp_out, void *ws, size_t ws_bytes, void *stream)
 {
     if (!q && !hi && !lo) return fail(QBP_ERR_INVALID_ARG, "quantize_s16: q, hi and lo are all NULL");
-    QuantOut o = {nullptr, q, hi, lo};
+    QuantOut o = {nullptr, q, hi, lo, nullptr, 0, 0};
     return quantize_any(16, x, rows, cols, granularity, rounding, seed, tensor_id, range_in, o, qp_out, ws, ws_bytes,
                         (cudaStream_t)stream);
 }
@@ -669,11 +726,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_bifurcate(const float 
     float2 *parts = w.take<float2>(kMaxParts);
     int rc = launch_range(g, rows * cols, parts, qp8, qp16, st);
     if (rc) return rc;
-    QuantOut o = {q8, nullptr, hi, lo};
-    rc = launch_quantize(g, rows * cols, cols, 0, QBP_ROUND_STOCHASTIC, qp8, tensor_id8, qp16, tensor_id16, seed, o, st);
-    if (rc) return rc;
-    if (row_sums8) return launch_rowsum(q8, true, rows, cols, row_sums8, st);
-    return QBP_OK;
+    return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st);
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8_static(const float *x, int64_t rows, int64_t cols, int granularity,

@@ -9,6 +9,7 @@
 // fixed fp32 operation order so that forward and backward agree on which
 // outputs the ReLU kept.
 #include "qbp_colscan.cuh"
+#include "qbp_mma.cuh"
 
 #include <cmath>
 
@@ -279,7 +280,9 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
     }
 }
 
-template <int VEC, bool RELU>
+// RANGE: also leave the block's (min, max) of the dx values it wrote in range_parts[block], so that the
+// quantiser that follows needs no scan of its own (Section 4: the range comes for free).
+template <int VEC, bool RELU, bool RANGE>
 __global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float *__restrict__ dy,
                                                                     const float *__restrict__ x, int64_t rows, int C,
                                                                     int tw, const float *__restrict__ mean,
@@ -288,10 +291,12 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float 
                                                                     const float *__restrict__ gamma,
                                                                     const float *__restrict__ beta, float Cn,
                                                                     const float2 *__restrict__ coef,
-                                                                    float *__restrict__ dx)
+                                                                    float *__restrict__ dx,
+                                                                    float2 *__restrict__ range_parts)
 {
     const ScanPos p = scan_pos<VEC>(C, tw);
-    if (!p.active) return;
+    float rlo = INFINITY, rhi = -INFINITY;
+    if (p.active) {
     const int rpb = kScanThreads / tw;
     float mu[VEC], s[VEC], g[VEC], b[VEC], lo[VEC], hi[VEC], m1[VEC], k2[VEC];
 #pragma unroll
@@ -324,9 +329,21 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float 
                     if (RELU && !(bn_y(bn_xhat(xv, mu[e], s[e]), g[e], b[e]) > 0.0f)) d = 0.0f;
                     const float ind = (xv == hi[e] ? 1.0f : 0.0f) - (xv == lo[e] ? 1.0f : 0.0f);
                     vd[u].v[e] = s[e] * (g[e] * d - m1[e] - k2[e] * ind);
+                    if (RANGE) { rlo = fminf(rlo, vd[u].v[e]); rhi = fmaxf(rhi, vd[u].v[e]); }
                 }
                 vd[u].store(dx + (r0 + u * step) * C + p.col);
             }
+    }
+    }
+    if (RANGE) {
+        rlo = warp_min(rlo); rhi = warp_max(rhi);
+        __shared__ float s_lo[kScanThreads / 32], s_hi[kScanThreads / 32];
+        if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = rlo; s_hi[threadIdx.x >> 5] = rhi; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < kScanThreads / 32; ++w) { rlo = fminf(rlo, s_lo[w]); rhi = fmaxf(rhi, s_hi[w]); }
+            range_parts[blockIdx.y * gridDim.x + blockIdx.x] = make_float2(rlo, rhi);
+        }
     }
 }
 
@@ -346,6 +363,12 @@ static int check_bn(const char *who, const void *a, const void *b, int64_t n, in
     if (!ws || ws_bytes < bn_ws_bytes(C))
         return fail(QBP_ERR_WORKSPACE, "%s: workspace of %zu bytes needed, %zu given", who, bn_ws_bytes(C), ws_bytes);
     return QBP_OK;
+}
+
+// Upper bound on the (min, max) partials rangebn_bwd_impl writes: row strips x column slabs of the apply grid.
+size_t rangebn_range_parts_capacity(int64_t C)
+{
+    return (size_t)kScanMaxStrips * (size_t)((C + kScanThreads - 1) / kScanThreads + 1);
 }
 
 }  // namespace qbp
@@ -407,7 +430,17 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const floa
                                const float *save_max, float *dx, float *dgamma, float *dbeta, void *ws,
                                size_t ws_bytes, void *stream)
 {
-    cudaStream_t st = (cudaStream_t)stream;
+    return rangebn_bwd_impl(dy, x, n, C, gamma, beta, relu, save_mean, save_min, save_max, dx, dgamma, dbeta, ws, ws_bytes,
+                            nullptr, nullptr, (cudaStream_t)stream);
+}
+
+// range_parts (nullable, room for rangebn_range_parts_capacity(C) entries) receives one (min, max) of dx per
+// block of the apply pass; *nparts their count.
+int qbp::rangebn_bwd_impl(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma, const float *beta,
+                          int relu, const float *save_mean, const float *save_min, const float *save_max, float *dx,
+                          float *dgamma, float *dbeta, void *ws, size_t ws_bytes, float2 *range_parts, int *nparts,
+                          cudaStream_t st)
+{
     int rc = check_bn("rangebn_bwd", x, dy, n, C, ws, ws_bytes);
     if (rc) return rc;
     if (!dx || !save_mean || !save_min || !save_max) return fail(QBP_ERR_INVALID_ARG, "rangebn_bwd: NULL tensor");
@@ -423,9 +456,9 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const floa
                                                       : blocks_per_sm(bn_bwd_stats_kernel<4, false>, kScanThreads))
                                               : blocks_per_sm(bn_bwd_stats_kernel<1, true>, kScanThreads));
     const dim3 grid(g.nbx, g.slabs);
-    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_apply_kernel<4, true>, kScanThreads)
-                                                       : blocks_per_sm(bn_bwd_apply_kernel<4, false>, kScanThreads))
-                                               : blocks_per_sm(bn_bwd_apply_kernel<1, true>, kScanThreads));
+    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_apply_kernel<4, true, true>, kScanThreads)
+                                                       : blocks_per_sm(bn_bwd_apply_kernel<4, false, true>, kScanThreads))
+                                               : blocks_per_sm(bn_bwd_apply_kernel<1, true, true>, kScanThreads));
     const dim3 grid_apply(ga.nbx, ga.slabs);
     const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n));
     const float Cn = (float)Cnd;
@@ -439,9 +472,15 @@ QBP_TRACE_BEGIN(st);
     bn_bwd_finalize_kernel<<<(int)C, 128, 0, st>>>(pa, pb, g.nbx, (int)C, n, gamma, Cnd, dgamma, dbeta, coef);
     QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
 QBP_TRACE_BEGIN(st);
-#define QBP_BN_BAPPLY(V, R) bn_bwd_apply_kernel<V, R><<<grid_apply, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx)
-    if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true); else QBP_BN_BAPPLY(4, false); }
-    else            { if (relu) QBP_BN_BAPPLY(1, true); else QBP_BN_BAPPLY(1, false); }
+#define QBP_BN_BAPPLY(V, R, G) bn_bwd_apply_kernel<V, R, G><<<grid_apply, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx, range_parts)
+    if (range_parts) {
+        if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true, true); else QBP_BN_BAPPLY(4, false, true); }
+        else            { if (relu) QBP_BN_BAPPLY(1, true, true); else QBP_BN_BAPPLY(1, false, true); }
+        if (nparts) *nparts = (int)(grid_apply.x * grid_apply.y);
+    } else {
+        if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true, false); else QBP_BN_BAPPLY(4, false, false); }
+        else            { if (relu) QBP_BN_BAPPLY(1, true, false); else QBP_BN_BAPPLY(1, false, false); }
+    }
 #undef QBP_BN_BAPPLY
     QBP_LAUNCH_OK("bn_bwd_apply_kernel");
     return QBP_OK;

@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
 // sits at (bit 1: first row, 2: last row, 4: first column, 8: last column).
 // sums[cls][c] (int64, zeroed beforehand).
 template <bool IS_SIGNED>
-__global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restrict__ q, int64_t pixels, int H, int W,
+__global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restrict__ q, int pixels, int H, int W,
                                                          int C, unsigned long long *__restrict__ sums)
 {
     extern __shared__ int s_acc[];                       // [16][C]
@@ -306,29 +306,45 @@ __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restri
     const int tw = cv < 256 ? cv : 256;
     const int rpb = 256 / tw;
     const int tx = threadIdx.x % tw, ty = threadIdx.x / tw;
+    constexpr int U = 8;                                 // loads in flight per thread
     if (ty < rpb) {
+        const int step = (int)gridDim.x * rpb;
         for (int g = tx; g < cv; g += tw) {
             int interior[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) interior[e] = 0;
-            for (int64_t p = (int64_t)blockIdx.x * rpb + ty; p < pixels; p += (int64_t)gridDim.x * rpb) {
-                const int w = (int)(p % W), h = (int)((p / W) % H);
-                const int cls = (h == 0 ? 1 : 0) | (h == H - 1 ? 2 : 0) | (w == 0 ? 4 : 0) | (w == W - 1 ? 8 : 0);
-                uint4 v = __ldg(reinterpret_cast<const uint4 *>(q + p * C) + g);
-                const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
-                if (cls == 0) {
+            for (int p0 = (int)blockIdx.x * rpb + ty; p0 < pixels; p0 += U * step) {
+                uint4 v[U];
+                bool ok[U];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
+                for (int u = 0; u < U; ++u) {
+                    const int p = p0 + u * step;
+                    ok[u] = p < pixels;
+                    if (ok[u]) v[u] = __ldg(reinterpret_cast<const uint4 *>(q + (int64_t)p * C) + g);
+                }
 #pragma unroll
-                        for (int b = 0; b < 4; ++b)
-                            interior[k * 4 + b] += IS_SIGNED ? (int)(int8_t)(wd[k] >> (8 * b)) : (int)((wd[k] >> (8 * b)) & 0xFF);
-                } else {
+                for (int u = 0; u < U; ++u) {
+                    if (!ok[u]) continue;
+                    const unsigned p = (unsigned)(p0 + u * step);
+                    const unsigned w = p % (unsigned)W, h = (p / (unsigned)W) % (unsigned)H;
+                    const int cls = (h == 0 ? 1 : 0) | (h == (unsigned)H - 1 ? 2 : 0) | (w == 0 ? 4 : 0) | (w == (unsigned)W - 1 ? 8 : 0);
+                    const uint32_t wd[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    if (cls == 0) {
+                        // one byte per dot product: the selector picks it, sign- or zero-extended
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
+                        for (int k = 0; k < 4; ++k)
 #pragma unroll
-                        for (int b = 0; b < 4; ++b)
-                            atomicAdd(&s_acc[cls * C + g * 16 + k * 4 + b],
-                                      IS_SIGNED ? (int)(int8_t)(wd[k] >> (8 * b)) : (int)((wd[k] >> (8 * b)) & 0xFF));
+                            for (int b = 0; b < 4; ++b)
+                                interior[k * 4 + b] = IS_SIGNED ? __dp4a((int)wd[k], 1 << (8 * b), interior[k * 4 + b])
+                                                                : (int)__dp4a(wd[k], 1u << (8 * b), (unsigned)interior[k * 4 + b]);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+#pragma unroll
+                            for (int b = 0; b < 4; ++b)
+                                atomicAdd(&s_acc[cls * C + g * 16 + k * 4 + b],
+                                          IS_SIGNED ? (int)(int8_t)(wd[k] >> (8 * b)) : (int)((wd[k] >> (8 * b)) & 0xFF));
+                    }
                 }
             }
 #pragma unroll
@@ -535,12 +551,15 @@ static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C,
         QBP_CUDA_OK(cudaFuncSetAttribute(class_sums_kernel<IS_SIGNED>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         configured[IS_SIGNED] = true;
     }
-    // int32 partials: a thread sees at most pixels / grid * 255 per channel
+    if (pixels >= (1ll << 30)) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad: more than 2^30 positions");
+    // int32 partials: a thread sees at most pixels / grid * 255 per channel.  Few blocks (each ends with up to
+    // 16*C atomics on the same 16*C sums), eight 16-byte loads in flight per thread.
     const int cv = C / 16, tw = cv < 256 ? cv : 256, rpb = 256 / tw;
-    int64_t grid = std::min<int64_t>((pixels + rpb - 1) / rpb, (int64_t)sm_count() * 4);
+    const int bps = std::max(1, std::min(2, (int)((200 * 1024) / std::max<size_t>(smem, 1024))));
+    int64_t grid = std::min<int64_t>((pixels + 8 * rpb - 1) / (8 * rpb), (int64_t)sm_count() * bps);
     grid = std::max<int64_t>(grid, pixels / (1 << 22) + 1);
     QBP_TRACE_BEGIN(st);
-    class_sums_kernel<IS_SIGNED><<<(unsigned)grid, 256, smem, st>>>((const uint8_t *)q, pixels, H, W, C, (unsigned long long *)sums);
+    class_sums_kernel<IS_SIGNED><<<(unsigned)grid, 256, smem, st>>>((const uint8_t *)q, (int)pixels, H, W, C, (unsigned long long *)sums);
     QBP_LAUNCH_OK("class_sums_kernel");
     return QBP_OK;
 }
