@@ -68,6 +68,11 @@ template <> struct VecF<4> {
         float4 t = __ldg(reinterpret_cast<const float4 *>(p));
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     }
+    // read-once data of a reduction pass: evict-first, so that it does not push out what a later pass re-reads
+    __device__ __forceinline__ void load_stream(const float *p) {
+        float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
     __device__ __forceinline__ void store(float *p) const {
         *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
     }
@@ -75,6 +80,7 @@ template <> struct VecF<4> {
 template <> struct VecF<1> {
     float v[1];
     __device__ __forceinline__ void load(const float *p) { v[0] = __ldg(p); }
+    __device__ __forceinline__ void load_stream(const float *p) { v[0] = __ldcs(p); }
     __device__ __forceinline__ void store(float *p) const { *p = v[0]; }
 };
 

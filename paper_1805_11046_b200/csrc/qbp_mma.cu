@@ -280,8 +280,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
     }
     if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
     for (int i = threadIdx.x; i < P.ips * P.msub * P.mma_per_iter; i += kMmaThreads) {
-        // MMA i of a stage: k iteration j, sub-tile sub, k step kk (innermost)
-        const int kk = i % P.mma_per_iter, sub = (i / P.mma_per_iter) % P.msub, j = i / (P.mma_per_iter * P.msub);
+        // MMA i of a stage: k iteration j, k step kk, sub-tile sub (innermost: consecutive MMAs then write
+        // different accumulators and do not wait for one another)
+        const int sub = i % P.msub, kk = (i / P.msub) % P.mma_per_iter, j = i / (P.mma_per_iter * P.msub);
         // the first MMAs of a tile (j == 0, kk == 0 of every sub-tile) overwrite the accumulator: i < w
         s_mma[i] = make_uint4(((uint32_t)j * a_iter + (uint32_t)sub * P.a.tile_bytes) / 16u + (uint32_t)kk * P.a.kstep,
                               ((uint32_t)j * P.b.tile_bytes) / 16u + (uint32_t)kk * P.b.kstep, (uint32_t)(sub * P.bn),

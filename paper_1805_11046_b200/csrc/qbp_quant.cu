@@ -72,6 +72,7 @@ void trace_end(const char *name, cudaStream_t st)
 
 constexpr int kThreads = 256;
 constexpr int kUnroll = 4;
+constexpr int kRangeUnroll = 8;          // loads in flight per thread of the read-only range scan
 constexpr int kMaxParts = 4096;          // upper bound on per-tensor scan blocks
 
 // ------------------------------------------------------- per-tensor range
@@ -81,18 +82,18 @@ __global__ void __launch_bounds__(kThreads) range_partial_kernel(const float *__
 {
     float lo = INFINITY, hi = -INFINITY;
     const int64_t nv = n / VEC;
-    const int64_t stride = (int64_t)gridDim.x * kThreads * kUnroll;
-    for (int64_t base = (int64_t)blockIdx.x * kThreads * kUnroll; base < nv; base += stride) {
-        VecF<VEC> v[kUnroll];
-        bool ok[kUnroll];
+    const int64_t stride = (int64_t)gridDim.x * kThreads * kRangeUnroll;
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * kRangeUnroll; base < nv; base += stride) {
+        VecF<VEC> v[kRangeUnroll];
+        bool ok[kRangeUnroll];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < kRangeUnroll; ++u) {
             int64_t i = base + u * kThreads + threadIdx.x;
             ok[u] = i < nv;
-            if (ok[u]) v[u].load(x + i * VEC);
+            if (ok[u]) v[u].load_stream(x + i * VEC);
         }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
+        for (int u = 0; u < kRangeUnroll; ++u)
             if (ok[u]) {
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) { lo = fminf(lo, v[u].v[e]); hi = fmaxf(hi, v[u].v[e]); }
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(kScanThreads) chan_range_partial_kernel(const 
             for (int u = 0; u < kScanUnroll; ++u) {
                 int64_t r = r0 + u * step;
                 ok[u] = r < rows;
-                if (ok[u]) v[u].load(x + r * C + p.col);
+                if (ok[u]) v[u].load_stream(x + r * C + p.col);
             }
 #pragma unroll
             for (int u = 0; u < kScanUnroll; ++u)
@@ -264,7 +265,7 @@ template <bool SR, int VEC>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restrict__ x, int64_t n, int cols,
                                                             int perch, const qbp_qparams *__restrict__ qp8,
                                                             uint32_t id8, const qbp_qparams *__restrict__ qp16,
-                                                            uint32_t id16, uint2 key, QuantOut o)
+                                                            uint32_t id16, uint2 key, QuantOut o, int smem_cols)
 {
     if (VEC == 1) {
         const int64_t stride = (int64_t)gridDim.x * kThreads;
@@ -274,6 +275,17 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     }
     const bool want8 = o.q8 != nullptr, want16 = o.q16 || o.hi || o.lo;
     QParamsReg p8 = {0, 0}, p16 = {0, 0};
+    // per channel: (1/scale, zero-point) of every channel once per block in shared memory (when the launcher
+    // gave it room), instead of a division per element
+    extern __shared__ float2 s_qp[];                         // [cols] for 8 bits, then [cols] for 16 bits
+    const bool table = perch && smem_cols > 0;
+    if (table) {
+        for (int c = threadIdx.x; c < cols; c += kThreads) {
+            if (want8)  { QParamsReg t = load_qp(qp8 + c, 8);   s_qp[c] = make_float2(t.inv, t.zp_u); }
+            if (want16) { QParamsReg t = load_qp(qp16 + c, 16); s_qp[cols + c] = make_float2(t.inv, t.zp_u); }
+        }
+        __syncthreads();
+    }
     if (!perch) {
         if (want8) p8 = load_qp(qp8, 8);
         if (want16) p16 = load_qp(qp16, 16);
@@ -308,7 +320,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                 uint32_t packed = 0;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (perch) p8 = load_qp(qp8 + c0 + e, 8);
+                    if (table) { const float2 t = s_qp[c0 + e]; p8.inv = t.x; p8.zp_u = t.y; }
+                    else if (perch) p8 = load_qp(qp8 + c0 + e, 8);
                     int code = quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
                     packed |= (uint32_t)((code ^ 0x80) & 0xFF) << (8 * e);
                 }
@@ -324,7 +337,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                 uint32_t s[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (perch) p16 = load_qp(qp16 + c0 + e, 16);
+                    if (table) { const float2 t = s_qp[cols + c0 + e]; p16.inv = t.x; p16.zp_u = t.y; }
+                    else if (perch) p16 = load_qp(qp16 + c0 + e, 16);
                     s[e] = (uint32_t)(quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]) ^ 0x8000);
                 }
                 if (o.q16)
@@ -434,7 +448,7 @@ static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams
     int nparts = 0;
     if (n > 0) {
         const bool vec = aligned16(x);
-        const int64_t per_block = (int64_t)kThreads * kUnroll * (vec ? 4 : 1);
+        const int64_t per_block = (int64_t)kThreads * kRangeUnroll * (vec ? 4 : 1);
         nparts = grid_for(vec ? blocks_per_sm(range_partial_kernel<4>, kThreads) : blocks_per_sm(range_partial_kernel<1>, kThreads),
                           (n + per_block - 1) / per_block);
         if (nparts > kMaxParts) nparts = kMaxParts;
@@ -487,12 +501,15 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     const int c = (int)cols;
     QBP_TRACE_BEGIN(st);
+    // per-channel parameter table: 2 x cols x 8 bytes of dynamic shared memory when that stays within 32 KB
+    const int smem_cols = (perch && vec && cols <= 2048) ? c : 0;
+    const size_t smem = (size_t)smem_cols * 2 * sizeof(float2);
     if (rounding == QBP_ROUND_STOCHASTIC) {
-        if (vec) quantize_kernel<true, 4><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
-        else     quantize_kernel<true, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
+        if (vec) quantize_kernel<true, 4><<<grid, kThreads, smem, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, smem_cols);
+        else     quantize_kernel<true, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, 0);
     } else {
-        if (vec) quantize_kernel<false, 4><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
-        else     quantize_kernel<false, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o);
+        if (vec) quantize_kernel<false, 4><<<grid, kThreads, smem, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, smem_cols);
+        else     quantize_kernel<false, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, 0);
     }
     QBP_LAUNCH_OK("quantize_kernel");
     return QBP_OK;

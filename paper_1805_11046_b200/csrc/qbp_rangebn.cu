@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_stats_kernel(const float *__r
             for (int u = 0; u < kScanUnroll; ++u) {
                 int64_t r = r0 + u * step;
                 ok[u] = r < rows;
-                if (ok[u]) v[u].load(x + r * C + p.col);
+                if (ok[u]) v[u].load_stream(x + r * C + p.col);
             }
 #pragma unroll
             for (int u = 0; u < kScanUnroll; ++u)
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
             for (int u = 0; u < kScanUnroll; ++u) {
                 int64_t r = r0 + u * step;
                 ok[u] = r < rows;
-                if (ok[u]) { vx[u].load(x + r * C + p.col); vd[u].load(dy + r * C + p.col); }
+                if (ok[u]) { vx[u].load_stream(x + r * C + p.col); vd[u].load_stream(dy + r * C + p.col); }
             }
 #pragma unroll
             for (int u = 0; u < kScanUnroll; ++u)
