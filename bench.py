@@ -159,13 +159,34 @@ def run_ours(args):
     barrier()
     assert L.status() == 0, "a device-side wait timed out"
 
+    # The step is ~30 short kernels: capture it once in a CUDA graph (the library only enqueues on the stream it is
+    # given) and replay it, so that the gaps between dependent launches do not depend on the host.
+    run_step, graphed = step, False
+    if not args.no_graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.current_stream().wait_stream(side)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            graph.replay()
+            torch.cuda.synchronize()
+            assert L.status() == 0
+            run_step, graphed = graph.replay, True
+        except Exception as exc:            # capture refused: time the plain launches
+            print(f"bench: CUDA graph capture failed ({exc}); timing plain launches", file=sys.stderr)
+            torch.cuda.synchronize()
+
     # ---- device-resident throughput: exactly K steps between two events on the launching stream
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record()
     for _ in range(args.steps):
-        step()
+        run_step()
     ev1.record()
     barrier()
     ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
@@ -180,7 +201,7 @@ def run_ours(args):
 
     def e2e_step():
         x.copy_(host["x"], non_blocking=True); w.copy_(host["w"], non_blocking=True); dy.copy_(host["dy"], non_blocking=True)
-        step()
+        run_step()
         out_host["dw"].copy_(L.dw, non_blocking=True); out_host["dgamma"].copy_(L.dgamma, non_blocking=True)
         out_host["dbeta"].copy_(L.dbeta, non_blocking=True)
 
@@ -240,7 +261,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "s8", "data": "synthetic",
         "config": {"workload": WORKLOAD, "batch_per_gpu": args.batch, "input": [args.batch, HW, HW, CIN],
                    "filter": [COUT, 3, 3, CIN], "l2": "inputs (205 MB per activation tensor) larger than the 126 MB L2",
-                   "parallelism": f"dp{world} (independent batches, no data-path collective)"},
+                   "parallelism": f"dp{world} (independent batches, no data-path collective)", "cuda_graph": graphed},
         "clocks": clocks,
         "e2e": {"value": round(world * args.batch / (e2e_ms * 1e-3), 1), "unit": "images/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4), "steps": e2e_steps},
@@ -319,6 +340,7 @@ def main():
     ap.add_argument("--batch", type=int, default=BATCH, help="images per GPU (the workload is quoted at 256)")
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a captured CUDA graph of the step")
     ap.add_argument("--only-steps", action="store_true", help="run warmup+steps and exit (for captures under ncu)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -231,14 +231,18 @@ __device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
 __device__ __forceinline__ void issue_stage(const uint4 *__restrict__ tab, int n_mma, uint32_t a_lo, uint32_t a_hi,
                                             uint32_t b_lo, uint32_t b_hi, uint32_t d_tmem, uint32_t idesc, bool first_stage)
 {
-    uint4 e = tab[0];
-#pragma unroll 2
-    for (int i = 0; i < n_mma; ++i) {
-        const uint4 nxt = tab[i + 1 < n_mma ? i + 1 : i];       // fetched while this MMA is being issued
-        const uint64_t da = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + e.x);
-        const uint64_t db = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + e.y);
-        mma_i8(d_tmem + e.z, da, db, idesc, (first_stage && e.w != 0u) ? 0u : 1u);
-        e = nxt;
+    // in batches of eight: all table loads first, then the descriptors, then the MMAs back to back
+    for (int i0 = 0; i0 < n_mma; i0 += 8) {
+        uint4 e[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) e[u] = tab[i0 + u < n_mma ? i0 + u : i0];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (i0 + u >= n_mma) break;
+            const uint64_t da = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + e[u].x);
+            const uint64_t db = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + e[u].y);
+            mma_i8(d_tmem + e[u].z, da, db, idesc, (first_stage && e[u].w != 0u) ? 0u : 1u);
+        }
     }
 }
 
@@ -406,7 +410,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                 if (++buf == (uint32_t)P.nbuf) { buf = 0; bph ^= 1u; }
             }
         }
-        __syncwarp();
+        // (the other lanes go on to the closing __syncthreads: a pending warp-level sync would slow the issuing lane)
     } else {
         // ------------------------------------------------------- epilogue
         // msub == 2: both groups of four warps work on every tile, one 128-row sub-tile each.
@@ -549,7 +553,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+    if (warp == 1) { __syncwarp(); tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols); }
 }
 
 // ================================================= zero-point correction terms
@@ -606,7 +610,9 @@ __global__ void __launch_bounds__(256) conv_rowterm_kernel(const int32_t *__rest
     const int64_t m = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (m >= pixels) return;
     const int za = q_in->zero_point, zb = q_w->zero_point;
-    const int q = (int)(m % W), p = (int)((m / W) % H);
+    // (pixels < 2^31: 32-bit divisions)
+    const unsigned mu = (unsigned)m;
+    const int q = (int)(mu % (unsigned)W), p = (int)((mu / (unsigned)W) % (unsigned)H);
     int box = 0, taps = 0;
     for (int eh = -pad; eh <= pad; ++eh)
         for (int ew = -pad; ew <= pad; ++ew)
@@ -819,6 +825,7 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
                     "conv_s8: needs stride 1, R = S in {1,3}, pad = (R-1)/2, C and K multiples of 16");
     if ((int64_t)d->R * d->S * std::max(d->C, d->K) > 33025)
         return fail(QBP_ERR_OVERFLOW_K, "conv_s8: reduction length exceeds 33025");
+    if ((int64_t)d->N * d->H * d->W >= (1ll << 31)) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: 2^31 or more positions");
     if (!in || !wgt || !q_in || !q_w) return fail(QBP_ERR_INVALID_ARG, "conv_s8: NULL operand");
     if (!acc_out && !out) return fail(QBP_ERR_INVALID_ARG, "conv_s8: acc_out and out are both NULL");
     if (!aligned16(in) || !aligned16(wgt) || (out && !aligned16(out)) || (acc_out && !aligned16(acc_out)))

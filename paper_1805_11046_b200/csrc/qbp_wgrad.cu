@@ -147,11 +147,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         s_counts[0] = nl;
     }
     if (threadIdx.x == 32) {
-        // the MMAs of one stage: k step outermost, so that consecutive MMAs write different accumulators
+        // the MMAs of one stage: the limb outermost (switching between the s8 x s8 and s8 x u8 instruction
+        // descriptors stalls the MMA pipe), then the k step, so that consecutive MMAs write different accumulators
         int nm = 0;
-        for (int kk = 0; kk < kk_per_iter; ++kk)
-            for (int j = 0; j < n_tiles; ++j)
-                for (int limb = 0; limb < 2; ++limb)
+        for (int limb = 0; limb < 2; ++limb)
+            for (int kk = 0; kk < kk_per_iter; ++kk)
+                for (int j = 0; j < n_tiles; ++j)
                     s_mma[nm++] = make_uint4(((uint32_t)j * a_tile_bytes) / 16u + (uint32_t)kk * P.a.kstep,
                                              ((uint32_t)limb * P.b.tile_bytes) / 16u + (uint32_t)kk * P.b.kstep,
                                              (uint32_t)((j * 2 + limb) * P.bn), (uint32_t)limb | (kk == 0 ? 2u : 0u));
@@ -225,7 +226,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
             }
             if (!timed_out) mma_commit(&acc_bar);
         }
-        __syncwarp();
+        // (the other lanes go on to the closing __syncthreads: a pending warp-level sync would slow the issuing lane)
     } else {
         // ------------------------------------------------------- epilogue
         const int quad = warp & 3;
@@ -288,7 +289,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+    if (warp == 1) { __syncwarp(); tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols); }
 }
 
 // ------------------------------------------------------------ code sums
@@ -415,7 +416,16 @@ __global__ void __launch_bounds__(256) wgrad_finalize_kernel(const WgradParams P
     const int slices = item < full_items ? P.s_full : P.s_last;
     const int64_t off = P.conv ? ((int64_t)j * P.bn + col) * 128 + row : ((int64_t)j * 128 + row) * P.bn + col;
     long long raw = 0;
-    for (int sl = 0; sl < slices; ++sl) raw += P.part[(int64_t)(first + sl) * P.part_stride + off];
+    const long long *src = P.part + (int64_t)first * P.part_stride + off;
+    int sl = 0;
+    for (; sl + 8 <= slices; sl += 8) {
+        long long v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (int64_t)(sl + u) * P.part_stride);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) raw += v[u];
+    }
+    for (; sl < slices; ++sl) raw += __ldcs(src + (int64_t)sl * P.part_stride);
     const long long acc = raw - zg * SX - zx * SG + count * zx * zg;
     if (P.acc_out) P.acc_out[e] = acc;
     if (P.dW) P.dW[e] = __fmul_rn((float)acc, __fmul_rn(P.qx->scale, P.qg->scale));
