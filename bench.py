@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
 # (captured at the full batch of 256).  None: not captured.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 174.70e6 / 51380224}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 226.9e6 / 51380224, "quantize_kernel": 326.8e6 / 51380224}
 
 
 def measured_peaks():
@@ -331,6 +331,121 @@ def run_reference(args):
     }), flush=True)
 
 
+# ------------------------------------------------- side workloads (not the headline line)
+def _event_ms(fn, iters, flush=None):
+    """Median CUDA-event time of fn over `iters` runs (after 3 warm-ups); an L2 flush before each when given."""
+    import torch
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record(); torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    return statistics.median(ts)
+
+
+def _kernel_ms(B, fn, reps=5, flush=None):
+    """Per-kernel device times (minimum over reps) of one call, from the library's launch trace; an L2 flush
+    (a write larger than the L2) before each call when given."""
+    for _ in range(2):
+        fn()
+    B.trace_enable(True)
+    for _ in range(reps):
+        if flush is not None:
+            flush.zero_()
+        fn()
+    r = B.trace_records(); B.trace_enable(False)
+    n = len(r) // reps
+    return [(r[i][0], min(r[k * n + i][1] for k in range(reps))) for i in range(n)]
+
+
+def run_gemm(args):
+    """Dense quantised GEMM (fp32 N(0,1) operands -> int8 codes -> tcgen05 product with fused zero-point correction
+    and dequantisation) and the limb-split 16x8-bit weight-gradient GEMM at M = N = K = --mnk; one JSON line each."""
+    import torch
+    from paper_1805_11046_b200 import binding as B, synth
+    torch.cuda.set_device(0)
+    n = args.mnk
+    peaks, kind = measured_peaks()
+    int8_peak = 2.0 * float(peaks["bf16_tflops"])        # own-dtype peak: measured bf16 x the nominal int8 : bf16 ratio
+    case = synth.dense_gemm(n, n, n)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    qa, qpa = B.qbp_quantize_s8(dev(case["a"])); qb, qpb = B.qbp_quantize_s8(dev(case["b"]))
+    out = torch.empty((n, n), dtype=torch.float32, device="cuda")
+    ws = B.workspace(B.lib.qbp_gemm_s8_workspace_bytes(n, n, n))
+    if args.only_steps:
+        for _ in range(args.warmup + args.steps):
+            B.qbp_gemm_s8(qa, qpa, qb, qpb, want_acc=False, out=out, ws=ws)
+        torch.cuda.synchronize(); assert B.status_word(ws) == 0
+        return
+    sampler = ClockSampler(0); sampler.start()
+    fn = lambda: B.qbp_gemm_s8(qa, qpa, qb, qpb, want_acc=False, out=out, ws=ws)
+    call_ms = _event_ms(fn, max(args.steps, 5))
+    ker = _kernel_ms(B, fn)
+    clocks = sampler.stop()
+    mma_ms = [t for k, t in ker if k == "qbp_mma_kernel"][0]
+    tops = 2.0 * n ** 3 / mma_ms / 1e9
+    print(json.dumps({"workload": f"dense_gemm_s8_{n}", "metric": "int8 TOPS", "value": round(tops, 1), "unit": "TOP/s",
+                      "call_ms": round(call_ms, 4), "kernels": [(k, round(t, 4)) for k, t in ker], "dtype": "s8", "clocks": clocks,
+                      "roofline": {"kernel": "qbp_mma_kernel", "bound": "tensor", "achieved": round(tops, 1), "peak": int8_peak,
+                                   "unit": "TOP/s", "frac": round(tops / int8_peak, 4), "traffic": None,
+                                   "peak_source": f"{kind} bf16 burst x 2 (nominal int8 : bf16)",
+                                   "frac_of_nominal_4500": round(tops / 4500.0, 4)}}), flush=True)
+    # limb-split weight-gradient GEMM: dW [K x N] = X [M x K]^T G [M x N], X 8-bit, G 16-bit as two byte limbs
+    del qa, qb, out
+    qx, qpx = B.qbp_quantize_s8(dev(case["x"]))
+    _, hi, lo, qpg = B.qbp_quantize_s16(dev(case["g"]), want=("hi", "lo"))
+    dW = torch.empty((n, n), dtype=torch.float32, device="cuda")
+    ws = B.workspace(B.lib.qbp_wgrad_s16_workspace_bytes(None, n, n, n))
+    fn = lambda: B.qbp_wgrad_s16(qx, qpx, hi, lo, qpg, want_acc=False, dW=dW, ws=ws)
+    call_ms = _event_ms(fn, max(min(args.steps, 20), 5))
+    ker = _kernel_ms(B, fn, reps=3)
+    k_ms = [t for k, t in ker if k == "qbp_wgrad_kernel"][0]
+    useful = 2.0 * n ** 3 / k_ms / 1e9
+    print(json.dumps({"workload": f"dense_wgrad_s16xs8_{n}", "metric": "useful 16x8-bit TOPS (executes twice as many int8 ops)",
+                      "value": round(useful, 1), "unit": "TOP/s", "call_ms": round(call_ms, 4),
+                      "kernels": [(k, round(t, 4)) for k, t in ker], "dtype": "s8",
+                      "roofline": {"kernel": "qbp_wgrad_kernel", "bound": "tensor", "achieved": round(2 * useful, 1),
+                                   "peak": int8_peak, "unit": "TOP/s (executed int8)", "frac": round(2 * useful / int8_peak, 4),
+                                   "traffic": None, "peak_source": f"{kind} bf16 burst x 2"}}), flush=True)
+
+
+def run_rangebn(args):
+    """Range BN forward/backward and 8-bit stochastic quantisation (per tensor, per channel) on the sweep shapes
+    (batch 256 x 56^2x64 ... 7^2x2048); one JSON line per shape with GB/s per kernel against the copy bandwidth."""
+    import torch
+    from paper_1805_11046_b200 import binding as B, synth
+    torch.cuda.set_device(0)
+    peaks, kind = measured_peaks()
+    hbm = float(peaks["hbm_gbs"])
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    bpe = {"bn_stats_kernel": 4, "bn_apply_kernel": 8, "bn_bwd_stats_kernel": 8, "bn_bwd_apply_kernel": 12,
+           "range_partial_kernel": 4, "chan_range_partial_kernel": 4, "quantize_kernel": 5}
+    for hw, ch in synth.RANGEBN_SWEEP:
+        case = synth.rangebn_case(args.batch, hw, ch)
+        x = torch.from_numpy(case["x"]).cuda(); dy = torch.from_numpy(case["dy"]).cuda()
+        y = torch.empty_like(x); dx = torch.empty_like(x); q = torch.empty(x.shape, dtype=torch.int8, device="cuda")
+        E = x.numel()
+        _, mean, vmin, vmax, _ = B.qbp_rangebn_fwd(x, relu=True, y=y)
+
+        def timed(fn):
+            return _kernel_ms(B, fn, reps=3, flush=flush)
+        ker = timed(lambda: B.qbp_rangebn_fwd(x, relu=True, y=y)) + \
+            timed(lambda: B.qbp_rangebn_bwd(dy, x, mean, vmin, vmax, relu=True, dx=dx))
+        qt = timed(lambda: B.qbp_quantize_s8(x, granularity=0, rounding=1, seed=1, tensor_id=2, q=q))
+        qc = timed(lambda: B.qbp_quantize_s8(x, granularity=1, rounding=1, seed=1, tensor_id=2, q=q))
+        row = lambda ks: [{"kernel": k, "us": round(t * 1e3, 1), "gbs": round(bpe[k] * E / t / 1e6, 0) if k in bpe else None,
+                           "frac": round(bpe[k] * E / t / 1e6 / hbm, 3) if k in bpe else None} for k, t in ks]
+        print(json.dumps({"workload": f"rangebn_quant_{args.batch}x{hw}x{hw}x{ch}", "tensor_mb": round(E * 4 / 1e6, 1),
+                          "peak_gbs": hbm, "peak_source": f"{kind} copy bandwidth", "rangebn": row(ker),
+                          "quantize_sr_per_tensor": row(qt), "quantize_sr_per_channel": row(qc)}), flush=True)
+        del x, dy, y, dx, q
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -342,9 +457,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a captured CUDA graph of the step")
     ap.add_argument("--only-steps", action="store_true", help="run warmup+steps and exit (for captures under ncu)")
+    ap.add_argument("--workload", choices=["layer", "gemm", "rangebn"], default="layer",
+                    help="layer: the headline line; gemm / rangebn: side measurements of the dense sweep and the Range BN sweep")
+    ap.add_argument("--mnk", type=int, default=8192, help="--workload gemm: M = N = K")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "gemm":
+        run_gemm(args)
+    elif args.workload == "rangebn":
+        run_rangebn(args)
     else:
         run_ours(args)
 
