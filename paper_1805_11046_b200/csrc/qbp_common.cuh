@@ -104,8 +104,31 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, float zp_
         float u = __fmul_rn((float)(rnd >> 8), 0x1p-24f);
         c = (u < frac) ? __fadd_rn(f, 1.0f) : f;
     }
-    c = fminf(fmaxf(c, 0.0f), Lf);
-    return (int)c;
+    // c is integral: the saturating conversion is the clamp to [0, 2^bits - 1] (Lf selects the width)
+    uint32_t code;
+    if (Lf == 255.0f) asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(code) : "f"(c));
+    else              asm("cvt.rni.sat.u16.f32 %0, %1;" : "=r"(code) : "f"(c));
+    return (int)code;
+}
+
+// Philox4x32-10 with the ten round keys precomputed (they depend on the key only).
+struct PhiloxKeys { uint32_t k0[10], k1[10]; };
+__device__ __forceinline__ PhiloxKeys philox_keys(uint2 k)
+{
+    PhiloxKeys r;
+#pragma unroll
+    for (int i = 0; i < 10; ++i) { r.k0[i] = k.x + (uint32_t)i * 0x9E3779B9u; r.k1[i] = k.y + (uint32_t)i * 0xBB67AE85u; }
+    return r;
+}
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys &k)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const unsigned long long p0 = (unsigned long long)0xD2511F53u * c.x;
+        const unsigned long long p1 = (unsigned long long)0xCD9E8D57u * c.z;
+        c = make_uint4((uint32_t)(p1 >> 32) ^ c.y ^ k.k0[r], (uint32_t)p1, (uint32_t)(p0 >> 32) ^ c.w ^ k.k1[r], (uint32_t)p0);
+    }
+    return c;
 }
 
 __device__ __forceinline__ float warp_min(float v)

@@ -261,16 +261,29 @@ __device__ __forceinline__ void quantize_scalar(const float *x, int64_t i, int c
     }
 }
 
-template <bool SR, int VEC>
+// Four codes (low bytes of c[0..3]) into one word.
+__device__ __forceinline__ uint32_t pack_bytes0(const uint32_t (&c)[4])
+{
+    return __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
+}
+// The second bytes of c[0..3] into one word.
+__device__ __forceinline__ uint32_t pack_bytes1(const uint32_t (&c)[4])
+{
+    return __byte_perm(__byte_perm(c[0], c[1], 0x0051), __byte_perm(c[2], c[3], 0x0051), 0x5410);
+}
+
+// PERCH is a template parameter so that the per-tensor instance (the hot one: it is bound by its instruction
+// count when rounding stochastically) carries none of the per-channel parameter handling.
+template <bool SR, int VEC, bool PERCH>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restrict__ x, int64_t n, int cols,
-                                                            int perch, const qbp_qparams *__restrict__ qp8,
+                                                            const qbp_qparams *__restrict__ qp8,
                                                             uint32_t id8, const qbp_qparams *__restrict__ qp16,
                                                             uint32_t id16, uint2 key, QuantOut o, int smem_cols)
 {
     if (VEC == 1) {
         const int64_t stride = (int64_t)gridDim.x * kThreads;
         for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += stride)
-            quantize_scalar<SR>(x, i, cols, perch != 0, qp8, id8, qp16, id16, key, o);
+            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, key, o);
         return;
     }
     const bool want8 = o.q8 != nullptr, want16 = o.q16 || o.hi || o.lo;
@@ -278,7 +291,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     // per channel: (1/scale, zero-point) of every channel once per block in shared memory (when the launcher
     // gave it room), instead of a division per element
     extern __shared__ float2 s_qp[];                         // [cols] for 8 bits, then [cols] for 16 bits
-    const bool table = perch && smem_cols > 0;
+    const bool table = PERCH && smem_cols > 0;
     if (table) {
         for (int c = threadIdx.x; c < cols; c += kThreads) {
             if (want8)  { QParamsReg t = load_qp(qp8 + c, 8);   s_qp[c] = make_float2(t.inv, t.zp_u); }
@@ -286,10 +299,11 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
         }
         __syncthreads();
     }
-    if (!perch) {
+    if (!PERCH) {
         if (want8) p8 = load_qp(qp8, 8);
         if (want16) p16 = load_qp(qp16, 16);
     }
+    const PhiloxKeys keys = philox_keys(key);
     const int64_t nv = n >> 2;
     const int64_t stride = (int64_t)gridDim.x * kThreads * kUnroll;
     for (int64_t base = (int64_t)blockIdx.x * kThreads * kUnroll; base < nv; base += stride) {
@@ -301,7 +315,6 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
             ok[u] = j < nv;
             if (ok[u]) v[u] = __ldg(reinterpret_cast<const float4 *>(x) + j);
         }
-#pragma unroll
         int rs[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) rs[u] = 0;
@@ -310,45 +323,47 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
             if (!ok[u]) continue;
             const int64_t j = base + u * kThreads + threadIdx.x;
             const float xs[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-            const int c0 = perch ? (int)((j << 2) % cols) : 0;
+            const int c0 = PERCH ? (int)((j << 2) % cols) : 0;
             if (want8) {
                 uint32_t r[4] = {0, 0, 0, 0};
                 if (SR) {
-                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id8, 0u), key);
+                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id8, 0u), keys);
                     r[0] = b.x; r[1] = b.y; r[2] = b.z; r[3] = b.w;
                 }
-                uint32_t packed = 0;
+                uint32_t c[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (table) { const float2 t = s_qp[c0 + e]; p8.inv = t.x; p8.zp_u = t.y; }
-                    else if (perch) p8 = load_qp(qp8 + c0 + e, 8);
-                    int code = quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
-                    packed |= (uint32_t)((code ^ 0x80) & 0xFF) << (8 * e);
+                    if (PERCH) {
+                        if (table) { const float2 t = s_qp[c0 + e]; p8.inv = t.x; p8.zp_u = t.y; }
+                        else p8 = load_qp(qp8 + c0 + e, 8);
+                    }
+                    c[e] = (uint32_t)quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
                 }
+                const uint32_t packed = pack_bytes0(c) ^ 0x80808080u;       // stored = unsigned code - 128
                 reinterpret_cast<uint32_t *>(o.q8)[j] = packed;
                 if (o.rowsum8) rs[u] = __dp4a((int)packed, 0x01010101, 0);
             }
             if (want16) {
                 uint32_t r[4] = {0, 0, 0, 0};
                 if (SR) {
-                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id16, 0u), key);
+                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id16, 0u), keys);
                     r[0] = b.x; r[1] = b.y; r[2] = b.z; r[3] = b.w;
                 }
-                uint32_t s[4];
+                uint32_t c[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (table) { const float2 t = s_qp[cols + c0 + e]; p16.inv = t.x; p16.zp_u = t.y; }
-                    else if (perch) p16 = load_qp(qp16 + c0 + e, 16);
-                    s[e] = (uint32_t)(quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]) ^ 0x8000);
+                    if (PERCH) {
+                        if (table) { const float2 t = s_qp[cols + c0 + e]; p16.inv = t.x; p16.zp_u = t.y; }
+                        else p16 = load_qp(qp16 + c0 + e, 16);
+                    }
+                    c[e] = (uint32_t)quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]);
                 }
+                // stored = unsigned code - 32768: flip the top bit of every code (of every high byte)
                 if (o.q16)
-                    reinterpret_cast<uint2 *>(o.q16)[j] = make_uint2(s[0] | (s[1] << 16), s[2] | (s[3] << 16));
-                if (o.hi)
-                    reinterpret_cast<uint32_t *>(o.hi)[j] =
-                        (s[0] >> 8) | ((s[1] >> 8) << 8) | ((s[2] >> 8) << 16) | ((s[3] >> 8) << 24);
-                if (o.lo)
-                    reinterpret_cast<uint32_t *>(o.lo)[j] =
-                        (s[0] & 0xFF) | ((s[1] & 0xFF) << 8) | ((s[2] & 0xFF) << 16) | ((s[3] & 0xFF) << 24);
+                    reinterpret_cast<uint2 *>(o.q16)[j] = make_uint2(__byte_perm(c[0], c[1], 0x5410) ^ 0x80008000u,
+                                                                     __byte_perm(c[2], c[3], 0x5410) ^ 0x80008000u);
+                if (o.hi) reinterpret_cast<uint32_t *>(o.hi)[j] = pack_bytes1(c) ^ 0x80808080u;
+                if (o.lo) reinterpret_cast<uint32_t *>(o.lo)[j] = pack_bytes0(c);
             }
         }
         if (o.rowsum8) {
@@ -366,7 +381,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     }
     if (blockIdx.x == 0 && threadIdx.x == 0)
         for (int64_t i = nv << 2; i < n; ++i)
-            quantize_scalar<SR>(x, i, cols, perch != 0, qp8, id8, qp16, id16, key, o);
+            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, key, o);
 }
 
 // Row sums of stored 8-bit codes: a group of G lanes per row (G = smallest power
@@ -495,22 +510,27 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
     if (o.rowsum8 && !vec) return fail(QBP_ERR_INVALID_ARG, "quantize: fused row sums need the vector path");
     const int64_t per_block = (int64_t)kThreads * (vec ? 4 * kUnroll : 1);
     const bool sr = rounding == QBP_ROUND_STOCHASTIC;
-    const int bps = vec ? (sr ? blocks_per_sm(quantize_kernel<true, 4>, kThreads) : blocks_per_sm(quantize_kernel<false, 4>, kThreads))
-                        : (sr ? blocks_per_sm(quantize_kernel<true, 1>, kThreads) : blocks_per_sm(quantize_kernel<false, 1>, kThreads));
-    const int grid = grid_for(bps, (n + per_block - 1) / per_block);
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     const int c = (int)cols;
-    QBP_TRACE_BEGIN(st);
     // per-channel parameter table: 2 x cols x 8 bytes of dynamic shared memory when that stays within 32 KB
     const int smem_cols = (perch && vec && cols <= 2048) ? c : 0;
     const size_t smem = (size_t)smem_cols * 2 * sizeof(float2);
-    if (rounding == QBP_ROUND_STOCHASTIC) {
-        if (vec) quantize_kernel<true, 4><<<grid, kThreads, smem, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, smem_cols);
-        else     quantize_kernel<true, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, 0);
+    const int64_t groups = (n + per_block - 1) / per_block;
+#define QBP_QUANT(SR_, VEC_, PC_)                                                                                       \
+    do {                                                                                                                \
+        const int grid = grid_for(blocks_per_sm(quantize_kernel<SR_, VEC_, PC_>, kThreads), groups);                    \
+        QBP_TRACE_BEGIN(st);                                                                                            \
+        quantize_kernel<SR_, VEC_, PC_><<<grid, kThreads, (VEC_) == 4 ? smem : 0, st>>>(x, n, c, qp8, id8, qp16, id16,  \
+                                                                                         key, o, (VEC_) == 4 ? smem_cols : 0); \
+    } while (0)
+    if (sr) {
+        if (vec) { if (perch) QBP_QUANT(true, 4, true); else QBP_QUANT(true, 4, false); }
+        else     { if (perch) QBP_QUANT(true, 1, true); else QBP_QUANT(true, 1, false); }
     } else {
-        if (vec) quantize_kernel<false, 4><<<grid, kThreads, smem, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, smem_cols);
-        else     quantize_kernel<false, 1><<<grid, kThreads, 0, st>>>(x, n, c, perch, qp8, id8, qp16, id16, key, o, 0);
+        if (vec) { if (perch) QBP_QUANT(false, 4, true); else QBP_QUANT(false, 4, false); }
+        else     { if (perch) QBP_QUANT(false, 1, true); else QBP_QUANT(false, 1, false); }
     }
+#undef QBP_QUANT
     QBP_LAUNCH_OK("quantize_kernel");
     return QBP_OK;
 }
