@@ -31,7 +31,7 @@ def _run_layer(B, cfg, relu, conv=None):
     return L, y, dx, dw, dgamma, dbeta
 
 
-def _check_layer(B, cfg, relu, conv_kw=None, sample=None):
+def _check_layer(B, cfg, relu, conv_kw=None, sample=None, want_y=False):
     conv = None if conv_kw is None else B.conv_desc(conv_kw["N"], conv_kw["H"], conv_kw["W"], conv_kw["C"], conv_kw["K"],
                                                     conv_kw["R"], conv_kw["S"], conv_kw["stride"], conv_kw["pad"])
     oconv = None if conv_kw is None else O.conv_desc(conv_kw["N"], conv_kw["H"], conv_kw["W"], conv_kw["C"], conv_kw["K"],
@@ -82,6 +82,8 @@ def _check_layer(B, cfg, relu, conv_kw=None, sample=None):
         widx = sample(w.size, 96)
         _, odw = O.conv_wgrad_s16(oconv, ox.q, ox.zero_point[0], g16.q, g16.zero_point[0], ox.scale[0], g16.scale[0], idx=widx)
         assert np.array_equal(to_host(dw).ravel()[widx], odw)
+    if want_y:
+        return to_host(y)
 
 
 def _sampler(seed):
@@ -128,3 +130,14 @@ def test_bottleneck_stack_stagewise(B):
         layers.append(L)
     torch.cuda.synchronize()
     assert a.shape == (8, 28, 28, 512) and a.min() == 0.0
+
+
+def test_bottleneck_stack_full_batch_stagewise(B):
+    """conv3_x bottleneck at the full batch of 256 (input [256,28,28,256]), every layer in the launch configuration
+    a benchmark of it would use; products checked on sampled outputs, Range BN on three channels."""
+    st = synth.bottleneck_stack(batch=256, hw=28)
+    a = st["x"]
+    for i, (w, c) in enumerate(zip(st["w"], st["convs"])):
+        cfg = dict(x=a, w=w, dy=synth.normal((c["N"], c["H"], c["W"], c["K"]), 60 + i, std=0.1), seed=0, id8=2 * i + 1, id16=2 * i + 2)
+        a = _check_layer(B, cfg, True, c, _sampler(13 + i), want_y=True)
+    assert a.shape == (256, 28, 28, 512) and a.min() == 0.0

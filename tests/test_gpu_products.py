@@ -61,6 +61,39 @@ def test_gemm_dense_sweep_shape_sampled_rows(B):
     assert np.array_equal(to_host(acc)[rows], oacc) and np.array_equal(to_host(out)[rows], oout)
 
 
+def test_gemm_dense_sweep_8192_sampled_rows_and_corner_tiles(B):
+    """8192^3 from the dense sweep in the benchmark's launch configuration (256 x 256 tiles, several tiles per CTA);
+    oracle on 64 random rows plus the rows of the four corner tiles' edges."""
+    n = 8192
+    case = synth.dense_gemm(n, n, n)
+    qa, qpa = B.qbp_quantize_s8(to_dev(case["a"])); qb, qpb = B.qbp_quantize_s8(to_dev(case["b"]))
+    oa = O.quantize(case["a"], 8); ob = O.quantize(case["b"], 8)
+    assert np.array_equal(to_host(qa), oa.q) and np.array_equal(to_host(qb), ob.q)
+    acc, out, ws = B.qbp_gemm_s8(qa, qpa, qb, qpb, want_acc=True)
+    assert B.status_word(ws) == 0
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, n - 256, n - 129, n - 128, n - 1],
+                                     np.random.Generator(np.random.PCG64(6)).integers(0, n, 64)]))
+    oacc, oout, bad = O.gemm_s8(oa.q[rows], oa.zero_point[0], ob.q, ob.zero_point[0], oa.scale[0], ob.scale[0])
+    assert bad == 0
+    assert np.array_equal(to_host(acc[rows]), oacc) and np.array_equal(to_host(out[rows]), oout)
+
+
+def test_wgrad_dense_sweep_shape_sampled_columns(B):
+    """The limb-split 16 x 8-bit product at 4096^3 (dense sweep): operands quantised from N(0,1) (nearest for the
+    8-bit side, stochastic for the 16-bit side); oracle on 96 sampled output columns (all 4096 rows of each)."""
+    n = 4096
+    case = synth.dense_gemm(n, n, n)
+    qx, qpx = B.qbp_quantize_s8(to_dev(case["x"]))
+    q16, hi, lo, qpg = B.qbp_quantize_s16(to_dev(case["g"]), rounding=B.QBP_ROUND_STOCHASTIC, seed=3, tensor_id=7)
+    ox = O.quantize(case["x"], 8); og = O.quantize(case["g"], 16, rounding=1, seed=3, tensor_id=7)
+    assert np.array_equal(to_host(qx), ox.q) and np.array_equal(to_host(q16), og.q)
+    acc, dW, ws = B.qbp_wgrad_s16(qx, qpx, hi, lo, qpg, want_acc=True)
+    assert B.status_word(ws) == 0
+    cols = np.unique(np.concatenate([[0, 127, 128, n - 1], np.random.Generator(np.random.PCG64(7)).integers(0, n, 92)]))
+    oacc, oout = O.gemm_s16s8(ox.q, ox.zero_point[0], np.ascontiguousarray(og.q[:, cols]), og.zero_point[0], ox.scale[0], og.scale[0])
+    assert np.array_equal(to_host(acc)[:, cols], oacc) and np.array_equal(to_host(dW)[:, cols], oout)
+
+
 # ----------------------------------------------------------- convolution
 CONVS = [(2, 8, 8, 64, 64, 1), (2, 8, 8, 64, 64, 3), (3, 10, 12, 32, 48, 3), (2, 14, 14, 128, 256, 3),
          (4, 7, 7, 256, 128, 1), (1, 1, 1, 16, 16, 3), (5, 9, 3, 80, 16, 3), (3, 28, 28, 128, 128, 3),
