@@ -387,11 +387,11 @@ def run_gemm(args):
     call_ms = _event_ms(fn, max(args.steps, 5))
     ker = _kernel_ms(B, fn)
     clocks = sampler.stop()
-    mma_ms = [t for k, t in ker if k == "qbp_mma_kernel"][0]
+    mma_ms = [t for k, t in ker if k in ("qbp_mma_kernel", "qbp_mma2_kernel")][0]
     tops = 2.0 * n ** 3 / mma_ms / 1e9
     print(json.dumps({"workload": f"dense_gemm_s8_{n}", "metric": "int8 TOPS", "value": round(tops, 1), "unit": "TOP/s",
                       "call_ms": round(call_ms, 4), "kernels": [(k, round(t, 4)) for k, t in ker], "dtype": "s8", "clocks": clocks,
-                      "roofline": {"kernel": "qbp_mma_kernel", "bound": "tensor", "achieved": round(tops, 1), "peak": int8_peak,
+                      "roofline": {"kernel": [k for k, t in ker if k.startswith("qbp_mma")][0], "bound": "tensor", "achieved": round(tops, 1), "peak": int8_peak,
                                    "unit": "TOP/s", "frac": round(tops / int8_peak, 4), "traffic": None,
                                    "peak_source": f"{kind} bf16 burst x 2 (nominal int8 : bf16)",
                                    "frac_of_nominal_4500": round(tops / 4500.0, 4)}}), flush=True)

@@ -760,6 +760,10 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
         rowterm, colterm);
     QBP_LAUNCH_OK("gemm_terms_kernel");
 
+    // large products run on CTA pairs (256 x 256 tiles across two SMs)
+    if (gemm2_eligible(M, N, K))
+        return launch_gemm2(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, rowterm, colterm, status, st);
+
     MmaParams P{};
     P.mode = MODE_GEMM;
     P.kblock = 128;

@@ -38,6 +38,15 @@ int make_map_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols
 int make_map_nhwc(CUtensorMap *map, const void *base, uint64_t N, uint64_t H, uint64_t W, uint64_t C, uint32_t bn,
                   uint32_t bh, uint32_t bw, uint32_t box_c);
 
+// fp32 output matrix [rows x cols] stored by TMA in boxes of 32 rows x 32 columns (128-byte swizzled slabs).
+int make_map_out_2d(CUtensorMap *map, float *base, uint64_t rows, uint64_t cols);
+
+// ---- the dense product on CTA pairs (qbp_mma2.cu) -------------------------------
+bool gemm2_eligible(int64_t M, int64_t N, int64_t K);
+int launch_gemm2(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
+                 const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const int32_t *rowterm,
+                 const int32_t *colterm, int *status, cudaStream_t st);
+
 // ---- shared-memory operand descriptors ---------------------------------------
 // How one operand tile of a pipeline stage is laid out and walked by the MMAs.
 struct OperandLayout {

@@ -78,6 +78,28 @@ def test_gemm_dense_sweep_8192_sampled_rows_and_corner_tiles(B):
     assert np.array_equal(to_host(acc[rows]), oacc) and np.array_equal(to_host(out[rows]), oout)
 
 
+# Shapes the CTA-pair kernel takes (at least eight rounds of 256 x 256 tiles over the SM pairs) with ragged edges in
+# every dimension: 512 x 256 pair tiles (M >= 2048) and 256 x 256 pair tiles (short M, wide N).
+PAIR_GEMMS = [(8208, 8464, 208), (1104, 38000, 144), (2048, 19216, 400)]
+
+
+@pytest.mark.parametrize("M,N,K", PAIR_GEMMS)
+@pytest.mark.parametrize("tA,tB", [(False, False), (False, True), (True, False), (True, True)])
+def test_gemm_s8_pair_kernel_ragged_sampled_rows(B, M, N, K, tA, tB):
+    """Oracle on the rows at the tile and pair-half edges, the ragged last rows and 48 random ones; every column."""
+    A = random_codes((K, M) if tA else (M, K), 11); Bm = random_codes((N, K) if tB else (K, N), 12)
+    za, zb, sa, sb = -7, 19, 0.125, 0.5
+    acc, out, ws = B.qbp_gemm_s8(to_dev(A), _qp(B, sa, za), to_dev(Bm), _qp(B, sb, zb), transA=tA, transB=tB, want_acc=True)
+    assert B.status_word(ws) == 0
+    edge = [0, 127, 128, 255, 256, 383, 384, 511, 512, M - 1, M - 2, (M // 512) * 512 - 1, (M // 256) * 256 - 1,
+            min((M // 256) * 256, M - 1), min((M // 128) * 128, M - 1)]
+    rows = np.unique(np.concatenate([edge, np.random.Generator(np.random.PCG64(M)).integers(0, M, 48)]))
+    Arows = np.ascontiguousarray(A[:, rows]) if tA else A[rows]
+    oacc, oout, bad = O.gemm_s8(Arows, za, Bm, zb, sa, sb, transA=tA, transB=tB)
+    assert bad == 0
+    assert np.array_equal(to_host(acc[rows]), oacc) and np.array_equal(to_host(out[rows]), oout)
+
+
 def test_wgrad_dense_sweep_shape_sampled_columns(B):
     """The limb-split 16 x 8-bit product at 4096^3 (dense sweep): operands quantised from N(0,1) (nearest for the
     8-bit side, stochastic for the 16-bit side); oracle on 96 sampled output columns (all 4096 rows of each)."""
