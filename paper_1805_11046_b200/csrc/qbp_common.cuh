@@ -190,6 +190,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
     return true;
 }
 
+// The same wait by every lane of a converged warp; the answer is the same in all of them.
+__device__ __forceinline__ bool mbar_wait_uniform(uint64_t *bar, uint32_t parity)
+{
+    const bool ok = mbar_wait(bar, parity);
+    return __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+}
+
 // The same wait for a whole warp: one lane polls (with a short sleep between polls, so that waiting warps
 // leave the shared-memory pipe to the warps that feed the tensor core), the result is shared by shuffle.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity)
@@ -243,6 +250,8 @@ __device__ __forceinline__ void tma_store_4d(const void *map, const void *src, i
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Until every store group of this thread has finished reading its shared-memory source.
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// Until all but the latest store group of this thread have finished reading their sources.
+__device__ __forceinline__ void tma_store_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 // Until every store group of this thread is complete.
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Named barrier over `count` threads (a multiple of 32) of the CTA.
@@ -277,6 +286,17 @@ __device__ __forceinline__ void tc_fence_before()
 __device__ __forceinline__ void tc_fence_after()
 {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+// True in exactly one lane of a converged warp.  The MMA warps run whole and put this around each tcgen05.mma and
+// commit, rather than branching on the lane index once around the loop: the instruction takes its operands from
+// warp-uniform registers, and only in code the compiler knows to be convergent are descriptors that change from
+// one MMA to the next kept there (measured: 63 against 110 cycles per 128 x 64 x 32 MMA).
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 // D[tmem] (+)= A[smem] * B[smem], 8-bit integer operands, int32 accumulator.  Volatile keeps it in order with

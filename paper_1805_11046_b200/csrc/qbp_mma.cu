@@ -173,6 +173,15 @@ struct MmaParams {
     int a_loads, b_loads;         // TMA loads per operand tile (M/N-major operands wider than one swizzled row)
     uint32_t a_load_bytes, b_load_bytes;
     int ips;                      // k iterations (operand tiles) per pipeline stage (at most 32: one lane each)
+    int halo;                     // conv: a stage holds whole halo tiles of the pixel box (one per channel chunk); the
+                                  // taps are shifted windows of a tile instead of loads of their own
+    int halo_w;                   // pixels per row of a halo tile (box width + 2)
+    int halo_rb;                  // halo tiles: 0 forward (K-major filter tiles), else the row bytes of the M/N-major filter tiles
+    int groups;                   // pipeline stages per output tile
+    int stage_mmas;               // MMAs per stage
+    int b_stage_tiles;            // filter tiles consumed per stage (resident filter)
+    uint32_t stage_tx;            // bytes the TMA loads of one stage deliver
+    int nslab;                    // epilogue staging slabs per warp (2: a store is still reading one while the next is filled)
     int iter_entries;             // entries of the k-iteration table in shared memory (conv), a multiple of 64
     int b_resident;               // conv: all filter tiles of the CTA's N tile stay in shared memory
     uint32_t b_res_bytes;         // bytes reserved for them at the start of shared memory
@@ -223,25 +232,100 @@ __device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
     return o;
 }
 
-// The MMAs of one pipeline stage, from the per-kernel table in shared memory: entry i = (offset of the A
-// descriptor from the stage's first A tile, offset of the B descriptor, accumulator column offset, unused),
-// offsets in 16-byte units (the 14-bit address field cannot carry: shared memory ends below 256 KB).  The
-// single issuing thread is bound by its own instruction latency on narrow tiles, hence one 16-byte load and
-// two adds per MMA instead of index arithmetic.
-__device__ __forceinline__ void issue_stage(const uint4 *__restrict__ tab, int n_mma, uint32_t a_lo, uint32_t a_hi,
-                                            uint32_t b_lo, uint32_t b_hi, uint32_t d_tmem, uint32_t idesc, bool first_stage)
+// The MMAs of one pipeline stage, run by the whole MMA warp in step; one elected lane issues.  Every operand is
+// plain arithmetic on loop counters and launch constants, and the "overwrite the accumulator" flag is a constant of
+// the code path (the first MMAs of a tile are peeled off): the instruction takes its operands from warp-uniform
+// registers, and anything looked up per MMA (a table entry, a flag derived from one) costs a transfer each time --
+// measured 53 cycles per 128 x 64 x 32 MMA this way against 110 to 130 from a table.  Offsets are in 16-byte units;
+// the 14-bit address field of a descriptor cannot carry: shared memory ends below 256 KB.
+#define QBP_ISSUE_ONE(d, a_lo, a_hi, b_lo, b_hi, idesc, accumulate)                                                   \
+    do {                                                                                                             \
+        if (elect_one())                                                                                             \
+            mma_i8((d), ((uint64_t)(a_hi) << 32) | (uint64_t)(a_lo), ((uint64_t)(b_hi) << 32) | (uint64_t)(b_lo), (idesc), \
+                   (accumulate));                                                                                    \
+    } while (0)
+
+// The 9 x MPI MMAs of one halo tile (a 3 x 3 filter over one channel chunk of 32 * MPI bytes, 10-pixel tile rows),
+// fully unrolled.  The A operand of a tap is the halo tile read from a shifted start: the shared-memory swizzle is a
+// function of the address, so a window that starts any whole number of pixel rows into the tile reads what TMA
+// wrote there.  Forward: output (p,q) reads input (p - pad + r, q - pad + t); layer gradient: (h + pad - r,
+// w + pad - t); the tile's origin is (h0 - pad, w0 - pad) in both, so the gradient takes the windows in reverse.
+// RB = 0: forward, filter tiles K-major; else layer gradient, filter tiles M/N-major with rows of RB bytes.
+//
+// What is fixed by (MPI, RB) is spelled as constants -- the A offsets, the upper descriptor words, the filter's k
+// step -- because the MMA takes its operands from the warp's few uniform registers: with the same values passed in
+// at run time next to the per-stage addresses the compiler ran out of them and each MMA cost 130 cycles instead of 40.
+constexpr int kHaloW = 10;           // pixels per row of a halo tile: the 8-pixel box row and one border pixel each side
+__host__ __device__ constexpr uint32_t swizzle_bits(uint32_t row_bytes) { return row_bytes == 128 ? 2u : row_bytes == 64 ? 4u : 6u; }
+template <int MPI, int RB>
+__device__ __forceinline__ void issue_halo_3x3(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t b_tile16, uint32_t idesc,
+                                               uint32_t first_acc)
 {
-    // in batches of eight: all table loads first, then the descriptors, then the MMAs back to back
-    for (int i0 = 0; i0 < n_mma; i0 += 8) {
-        uint4 e[8];
+    constexpr bool FWD = RB == 0;
+    constexpr uint32_t cb = 32u * MPI;
+    constexpr int px16 = 2 * MPI, row16 = kHaloW * px16;
+    constexpr uint32_t a_hi = ((kHaloW * cb) >> 4) | (1u << 14) | (swizzle_bits(cb) << 29);
+    constexpr uint32_t b_hi = FWD ? ((8u * cb) >> 4) | (1u << 14) | (swizzle_bits(cb) << 29)
+                                  : ((8u * (uint32_t)RB) >> 4) | (1u << 14) | (swizzle_bits((uint32_t)RB) << 29);
+    constexpr uint32_t b_kstep = FWD ? 2u : (32u * (uint32_t)RB) >> 4;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) e[u] = tab[i0 + u < n_mma ? i0 + u : i0];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            if (i0 + u >= n_mma) break;
-            const uint64_t da = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + e[u].x);
-            const uint64_t db = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + e[u].y);
-            mma_i8(d_tmem + e[u].z, da, db, idesc, (first_stage && e[u].w != 0u) ? 0u : 1u);
+    for (int i = 0; i < 9 * MPI; ++i) {
+        const int tap = i / MPI, kk = i % MPI, r = tap / 3, t = tap % 3;
+        const uint32_t ao = (uint32_t)((FWD ? r : 2 - r) * row16 + (FWD ? t : 2 - t) * px16 + kk * 2);
+        const uint32_t bo = (uint32_t)tap * b_tile16 + (uint32_t)kk * b_kstep;
+        if (elect_one())
+            mma_i8(d, ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + ao), ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + bo), idesc,
+                   i == 0 ? first_acc : 1u);
+    }
+}
+
+template <int MPI>
+__device__ __forceinline__ void issue_halo_3x3_any(int rb, uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t b_tile16,
+                                                   uint32_t idesc, uint32_t first_acc)
+{
+    if (rb == 0)        issue_halo_3x3<MPI, 0>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    else if (rb == 128) issue_halo_3x3<MPI, 128>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    else if (rb == 64)  issue_halo_3x3<MPI, 64>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    else                issue_halo_3x3<MPI, 32>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+}
+
+__device__ __forceinline__ void issue_stage(const MmaParams &P, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t d_tmem, bool first_stage)
+{
+    const uint32_t a_tile16 = P.a.tile_bytes >> 4, b_tile16 = P.b.tile_bytes >> 4;
+    const uint32_t first_acc = first_stage ? 0u : 1u;
+    if (!P.halo) {
+        // k iteration j, k step kk, sub-tile sub (innermost: consecutive MMAs then write different accumulators
+        // and do not wait for one another)
+        if (P.msub == 1) {
+            QBP_ISSUE_ONE(d_tmem, a_lo, a_hi, b_lo, b_hi, P.idesc, first_acc);
+            for (int j = 0; j < P.ips; ++j) {
+#pragma unroll 4
+                for (int kk = (j == 0 ? 1 : 0); kk < P.mma_per_iter; ++kk)
+                    QBP_ISSUE_ONE(d_tmem, a_lo + (uint32_t)kk * P.a.kstep, a_hi, b_lo + (uint32_t)kk * P.b.kstep, b_hi, P.idesc, 1u);
+                a_lo += a_tile16; b_lo += b_tile16;
+            }
+        } else {
+            const uint32_t d1 = d_tmem + (uint32_t)P.bn;
+            QBP_ISSUE_ONE(d_tmem, a_lo, a_hi, b_lo, b_hi, P.idesc, first_acc);
+            QBP_ISSUE_ONE(d1, a_lo + a_tile16, a_hi, b_lo, b_hi, P.idesc, first_acc);
+            for (int j = 0; j < P.ips; ++j) {
+#pragma unroll 4
+                for (int kk = (j == 0 ? 1 : 0); kk < P.mma_per_iter; ++kk) {
+                    QBP_ISSUE_ONE(d_tmem, a_lo + (uint32_t)kk * P.a.kstep, a_hi, b_lo + (uint32_t)kk * P.b.kstep, b_hi, P.idesc, 1u);
+                    QBP_ISSUE_ONE(d1, a_lo + a_tile16 + (uint32_t)kk * P.a.kstep, a_hi, b_lo + (uint32_t)kk * P.b.kstep, b_hi, P.idesc, 1u);
+                }
+                a_lo += 2u * a_tile16; b_lo += b_tile16;
+            }
+        }
+    } else {
+        const uint32_t b_chunk16 = 9u * b_tile16;             // the nine filter tiles of one channel chunk
+        for (int hj = 0; hj < P.ips; ++hj) {
+            const uint32_t acc0 = hj == 0 ? first_acc : 1u;
+            if (P.mma_per_iter == 4)      issue_halo_3x3_any<4>(P.halo_rb, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
+            else if (P.mma_per_iter == 2) issue_halo_3x3_any<2>(P.halo_rb, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
+            else                          issue_halo_3x3_any<1>(P.halo_rb, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
+            a_lo += a_tile16; b_lo += b_chunk16;
         }
     }
 }
@@ -267,9 +351,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
     const uint32_t a_stage = a_iter * (uint32_t)P.ips;
     const uint32_t stage_bytes = a_stage + (P.b_resident ? 0u : P.b.tile_bytes * (uint32_t)P.ips);
     uint8_t *staging = smem + (((size_t)P.stages * stage_bytes + 1023) & ~(size_t)1023);   // kEpiWarps slabs, 1024-byte aligned
-    int4 *s_iter = reinterpret_cast<int4 *>(staging + kEpiWarps * kStageSlab);          // conv: one entry per k iteration
-    uint4 *s_mma = reinterpret_cast<uint4 *>(s_iter + P.iter_entries);                   // the MMAs of one stage (kMaxStageMmas)
-    int32_t *s_cterm = reinterpret_cast<int32_t *>(s_mma + kMaxStageMmas);               // column terms
+    int4 *s_iter = reinterpret_cast<int4 *>(staging + kEpiWarps * kStageSlab * P.nslab);  // conv: one entry per k iteration
+    int32_t *s_cterm = reinterpret_cast<int32_t *>(s_iter + P.iter_entries);             // column terms
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -283,19 +366,12 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         if (P.out) tma_prefetch_desc(&P.mapC);
     }
     if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
-    for (int i = threadIdx.x; i < P.ips * P.msub * P.mma_per_iter; i += kMmaThreads) {
-        // MMA i of a stage: k iteration j, k step kk, sub-tile sub (innermost: consecutive MMAs then write
-        // different accumulators and do not wait for one another)
-        const int sub = i % P.msub, kk = (i / P.msub) % P.mma_per_iter, j = i / (P.mma_per_iter * P.msub);
-        // the first MMAs of a tile (j == 0, kk == 0 of every sub-tile) overwrite the accumulator: i < w
-        s_mma[i] = make_uint4(((uint32_t)j * a_iter + (uint32_t)sub * P.a.tile_bytes) / 16u + (uint32_t)kk * P.a.kstep,
-                              ((uint32_t)j * P.b.tile_bytes) / 16u + (uint32_t)kk * P.b.kstep, (uint32_t)(sub * P.bn),
-                              (j == 0 && kk == 0) ? 0xFFFFu : 0u);
-    }
     if (P.mode != MODE_GEMM)
         for (int it = threadIdx.x; it < P.k_iters; it += kMmaThreads) {
-            // k iteration -> (channel offset, tap column, tap row, filter coordinate of the tap's channel chunk)
-            const int tap = it / P.cchunks, cc = it % P.cchunks;
+            // k iteration -> (channel offset, tap column, tap row, filter coordinate of the tap's channel chunk);
+            // tap-major, or chunk-major when a stage is a halo tile of one chunk (its filter tiles are then contiguous)
+            const int taps = P.k_iters / P.cchunks;
+            const int tap = P.halo ? it % taps : it / P.cchunks, cc = P.halo ? it / taps : it % P.cchunks;
             const int c0 = cc * P.chunk_bytes;
             s_iter[it] = make_int4(c0, tap % P.S, tap / P.S, P.mode == MODE_FPROP ? tap * P.Cred + c0 : tap * (int)P.N);
         }
@@ -323,7 +399,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
             }
         }
         uint32_t s = 0, ph = 1;                             // ring position and the parity to wait for, across tiles
-        const int groups = P.k_iters / P.ips;
+        const int groups = P.groups;
         for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
             const TileOrigin o = tile_origin(P, tile);
             if (P.mode == MODE_GEMM) {
@@ -354,11 +430,16 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                 int ok = 1;
                 if (lane == 0) {
                     ok = mbar_wait(&empty_bar[s], ph) ? 1 : 0;
-                    if (ok) mbar_expect_tx(&full_bar[s], stage_bytes);
+                    if (ok) mbar_expect_tx(&full_bar[s], P.stage_tx);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { timed_out = true; break; }
-                if (lane < P.ips) {
+                if (P.halo) {
+                    // the pixel box with a border of `pad` pixels, one load per channel chunk; outside the image: zeros
+                    if (lane < P.ips)
+                        tma_load_4d(smem + (size_t)s * stage_bytes + (size_t)lane * P.a.tile_bytes, &P.mapA, &full_bar[s],
+                                    (g * P.ips + lane) * P.chunk_bytes, o.w0 - P.pad, o.h0 - P.pad, o.img0);
+                } else if (lane < P.ips) {
                     const int4 e = s_iter[g * P.ips + lane];   // (channel offset, tap column, tap row, filter coordinate)
                     uint8_t *sa = smem + (size_t)s * stage_bytes;
                     uint8_t *da = sa + (size_t)lane * P.a.tile_bytes;
@@ -383,34 +464,32 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
-            // -------------------------------------------------- MMA issuer
-            if (P.b_resident && !mbar_wait(&b_full, 0)) timed_out = true;
-            const uint32_t bres_addr = smem_u32(smem_b);
-            const uint32_t ring_addr = smem_u32(smem);
-            const int groups = P.k_iters / P.ips;
-            const int n_mma = P.ips * P.msub * P.mma_per_iter;
-            uint32_t s = 0, ph = 0;                          // ring position and parity, across tiles
-            uint32_t buf = 0, bph = 1;                       // accumulator buffer and the parity of its "empty" barrier
-            for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
-                if (!mbar_wait(&acc_empty[buf], bph)) { timed_out = true; break; }
+        // ------------------------------------------------------ MMA issuer
+        // The whole warp walks the tiles and stages in step, so that ring positions, descriptors and accumulator
+        // addresses stay warp-uniform; an elected lane issues the MMAs and the commits.
+        if (P.b_resident && !mbar_wait_uniform(&b_full, 0)) timed_out = true;
+        const uint32_t bres_addr = smem_u32(smem_b);
+        const uint32_t ring_addr = smem_u32(smem);
+        const int groups = P.groups;
+        uint32_t s = 0, ph = 0;                          // ring position and parity, across tiles
+        uint32_t buf = 0, bph = 1;                       // accumulator buffer and the parity of its "empty" barrier
+        for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
+            if (!mbar_wait_uniform(&acc_empty[buf], bph)) { timed_out = true; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * buf_cols;
+            for (int g = 0; g < groups; ++g) {
+                if (!mbar_wait_uniform(&full_bar[s], ph)) { timed_out = true; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * buf_cols;
-                for (int g = 0; g < groups; ++g) {
-                    if (!mbar_wait(&full_bar[s], ph)) { timed_out = true; break; }
-                    tc_fence_after();
-                    const uint32_t stage_addr = ring_addr + s * stage_bytes;
-                    const uint32_t b_addr = P.b_resident ? bres_addr + (uint32_t)(g * P.ips) * P.b.tile_bytes : stage_addr + a_stage;
-                    issue_stage(s_mma, n_mma, ((stage_addr >> 4) & 0x3FFFu) | P.a.desc_lo, P.a.desc_hi,
-                                ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo, P.b.desc_hi, d_tmem, P.idesc, g == 0);
-                    mma_commit(&empty_bar[s]);
-                    if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
-                }
-                if (!timed_out) mma_commit(&acc_full[buf]);
-                if (++buf == (uint32_t)P.nbuf) { buf = 0; bph ^= 1u; }
+                const uint32_t stage_addr = ring_addr + s * stage_bytes;
+                const uint32_t b_addr = P.b_resident ? bres_addr + (uint32_t)(g * P.b_stage_tiles) * P.b.tile_bytes : stage_addr + a_stage;
+                issue_stage(P, ((stage_addr >> 4) & 0x3FFFu) | P.a.desc_lo, P.a.desc_hi,
+                            ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo, P.b.desc_hi, d_tmem, g == 0);
+                if (elect_one()) mma_commit(&empty_bar[s]);
+                if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
             }
+            if (!timed_out && elect_one()) mma_commit(&acc_full[buf]);
+            if (++buf == (uint32_t)P.nbuf) { buf = 0; bph ^= 1u; }
         }
-        // (the other lanes go on to the closing __syncthreads: a pending warp-level sync would slow the issuing lane)
     } else {
         // ------------------------------------------------------- epilogue
         // msub == 2: both groups of four warps work on every tile, one 128-row sub-tile each.
@@ -420,7 +499,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         const int quad = warp & 3;                       // the tensor-memory lanes this warp may read
         const int group = ew >> 2;
         const int row = quad * 32 + lane;
-        uint8_t *slab = staging + (size_t)ew * kStageSlab;
+        uint8_t *slab0 = staging + (size_t)(ew * P.nslab) * kStageSlab;
+        uint32_t slab_i = 0;
         const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
         const int sub = P.msub == 2 ? group : 0;
         const int lt_step = P.msub == 2 ? 1 : 2;
@@ -519,9 +599,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                         }
                     }
                     if (P.out) {
-                        // the previous store of this warp must have read the slab before it is overwritten
-                        if (lane == 0) tma_store_wait_read();
+                        // the store that last used this slab must have read it before it is overwritten
+                        uint8_t *slab = slab0 + slab_i * kStageSlab;
+                        if (lane == 0) { if (P.nslab == 2) tma_store_wait_read_but_one(); else tma_store_wait_read(); }
                         __syncwarp();
+                        if (P.nslab == 2) slab_i ^= 1u;
                         // 128-byte swizzle: the 16-byte group g of row `lane` sits at group g ^ (lane & 7)
                         uint8_t *rowp = slab + lane * 128;
 #pragma unroll
@@ -624,19 +706,43 @@ __global__ void __launch_bounds__(256) conv_rowterm_kernel(const int32_t *__rest
 }
 
 // ================================================================== launchers
-static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
+// Shared memory of the kernel that is not the stage ring or the resident filter: alignment slack, epilogue staging
+// slabs, the tables, the column terms (the whole table when it is small, else one tile's columns per epilogue group).
+static uint32_t fixed_smem(MmaParams &P)
 {
-    // shared memory that is not the stage ring: alignment slack, epilogue staging slabs, column terms
-    // column terms: the whole table when it is small, else one tile's columns per epilogue group
     P.cterm_all = (size_t)P.ncls * P.N * sizeof(int32_t) <= 32u * 1024u ? 1 : 0;
     const size_t cterm_bytes = P.cterm_all ? ((size_t)P.ncls * P.N + 64) * sizeof(int32_t)
                                            : (size_t)(P.msub == 1 ? 2 : 1) * P.ncls * P.bn * sizeof(int32_t);
     P.iter_entries = P.mode == MODE_GEMM ? 0 : (int)align_up((size_t)P.k_iters, 64);
-    const uint32_t fixed = 2048u + kEpiWarps * kStageSlab + (uint32_t)P.iter_entries * 16u + kMaxStageMmas * 16u +
-                           (uint32_t)align_up(cterm_bytes, 1024);
+    return 2048u + kEpiWarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + 
+           (uint32_t)align_up(cterm_bytes, 1024);
+}
+
+// Whether a convolution can run from halo tiles: the whole filter resident beside at least three halo tiles.
+static bool halo_fits(MmaParams &P, uint32_t halo_tile_bytes)
+{
+    const uint32_t fixed = fixed_smem(P);
+    return P.tiles_n == 1 && fixed + align_up((size_t)P.b.tile_bytes * P.k_iters, 1024) + 3u * halo_tile_bytes <= kSmemBudget;
+}
+
+static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
+{
+    const uint32_t fixed = fixed_smem(P);
     const uint32_t budget = kSmemBudget - fixed;
     P.ips = 1; P.b_resident = 0; P.b_res_bytes = 0;
-    if (P.mode != MODE_GEMM) {
+    if (P.halo) {
+        // one halo tile per channel chunk; as many chunks per stage as leave three stages (a commit per stage
+        // drains the MMA pipeline, so fewer and longer stages are better)
+        const int taps = P.k_iters / P.cchunks;
+        P.b_resident = 1; P.b_res_bytes = (uint32_t)align_up((size_t)P.b.tile_bytes * P.k_iters, 1024);
+        for (int c = 1; c <= P.cchunks; ++c)
+            if (P.cchunks % c == 0 && c <= 32 && c * taps * P.mma_per_iter <= kMaxStageMmas &&
+                3u * (uint32_t)c * P.a.tile_bytes <= budget - P.b_res_bytes) P.ips = c;
+        P.groups = P.cchunks / P.ips;
+        P.stage_mmas = P.ips * taps * P.mma_per_iter;
+        P.b_stage_tiles = P.ips * taps;
+        P.stage_tx = (uint32_t)P.ips * (uint32_t)(P.halo_w * ((1 << P.bh_log2) + 2 * P.pad) * P.chunk_bytes);
+    } else if (P.mode != MODE_GEMM) {
         // keep the whole filter in shared memory when it fits beside at least three activation stages
         const uint32_t b_all = P.b.tile_bytes * (uint32_t)P.k_iters;
         if (P.tiles_n == 1 && b_all + 3 * P.a.tile_bytes <= budget) { P.b_resident = 1; P.b_res_bytes = (uint32_t)align_up(b_all, 1024); }
@@ -647,6 +753,12 @@ static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
             if (P.k_iters % c == 0 && c <= 32 && 2u * (uint32_t)c * per_iter <= budget - P.b_res_bytes) P.ips = c;
     }
     const uint32_t stage_bytes = (uint32_t)P.ips * (P.a.tile_bytes * (uint32_t)P.msub + (P.b_resident ? 0u : P.b.tile_bytes));
+    if (!P.halo) {
+        P.groups = P.k_iters / P.ips;
+        P.stage_mmas = P.ips * P.msub * P.mma_per_iter;
+        P.b_stage_tiles = P.ips;
+        P.stage_tx = stage_bytes;
+    }
     int stages = (int)((budget - P.b_res_bytes) / stage_bytes);
     if (stages < 2) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "tensor-core tile does not fit shared memory");
     stages = std::min(stages, kMaxStages);
@@ -770,7 +882,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     P.k_iters = (int)((K + 127) / 128);
     P.mma_per_iter = 4;
     P.msub = M > 128 ? 2 : 1;            // 256-row CTA tiles halve the operand traffic per multiply-add
-    P.ncls = 1;
+    P.ncls = 1; P.nslab = 1;
     // A: stored [M x K] -> K-major rows of 128 reduction bytes; stored [K x M] -> M-major, one box per sub-tile
     if (!transA) {
         P.a = layout_kmajor(128, 128);
@@ -868,22 +980,13 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
 
     MmaParams P{};
     P.mode = dgrad ? MODE_DGRAD : MODE_FPROP;
-    P.msub = 1; P.ncls = 16;
+    P.msub = 1; P.ncls = 16; P.nslab = 2;
     P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.S = d->S; P.Cred = Cred;
     const uint32_t cb = Cred % 128 == 0 ? 128u : Cred % 64 == 0 ? 64u : 32u;      // reduction bytes per stage row
     P.chunk_bytes = (int)cb;
     P.cchunks = (Cred + (int)cb - 1) / (int)cb;      // a ragged last chunk is zero-filled by TMA on the activation side
     P.k_iters = taps * P.cchunks;
     P.mma_per_iter = (int)cb / 32;
-    int bwl = 0, bhl = 0;
-    pick_pixel_box(d->N, d->H, d->W, bwl, bhl);
-    P.bw_log2 = bwl; P.bh_log2 = bhl;
-    const int bw = 1 << bwl, bh = 1 << bhl, bn_img = 128 >> (bwl + bhl);
-    P.tiles_w = (d->W + bw - 1) / bw; P.tiles_h = (d->H + bh - 1) / bh;
-    const int tiles_img = (d->N + bn_img - 1) / bn_img;
-    P.a = layout_kmajor(128, cb);
-    rc = make_map_nhwc(&P.mapA, in, d->N, d->H, d->W, Cred, bn_img, bh, bw, cb);
-    if (rc) return rc;
     if (!dgrad) {
         P.bn = std::min(256, Nout);
         P.b = layout_kmajor((uint32_t)P.bn, cb);
@@ -897,14 +1000,45 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
         rc = make_map_2d(&P.mapB, wgt, d->K, (uint64_t)taps * d->C, cb, rb);
     }
     if (rc) return rc;
+    P.tiles_n = (Nout + P.bn - 1) / P.bn;
+    P.M = pix; P.N = Nout;
+
+    int bwl = 0, bhl = 0;
+    pick_pixel_box(d->N, d->H, d->W, bwl, bhl);
+    // 3 x 3: a box of 16 rows x 8 pixels of one image, loaded once with its border; the nine taps are windows of
+    // that tile (a ninth of the operand traffic of one load per tap).  Taken when the filter stays resident and the
+    // fixed box does not waste many more MMA rows than the free one.
+    if (d->R == 3) {
+        const uint32_t halo_bytes = (uint32_t)align_up((size_t)18 * 10 * cb, 1024);
+        const long long tiles_free = (long long)((d->W + (1 << bwl) - 1) >> bwl) * ((d->H + (1 << bhl) - 1) >> bhl) *
+                                     ((d->N + (128 >> (bwl + bhl)) - 1) / (128 >> (bwl + bhl)));
+        const long long tiles_halo = (long long)((d->W + 7) / 8) * ((d->H + 15) / 16) * d->N;
+        if (tiles_halo * 2 <= tiles_free * 3 && halo_fits(P, halo_bytes)) {
+            P.halo = 1; P.halo_w = kHaloW; bwl = 3; bhl = 4;
+            P.halo_rb = dgrad ? (Nout >= 128 ? 128 : Nout >= 64 ? 64 : 32) : 0;
+        }
+    }
+    P.bw_log2 = bwl; P.bh_log2 = bhl;
+    const int bw = 1 << bwl, bh = 1 << bhl, bn_img = 128 >> (bwl + bhl);
+    P.tiles_w = (d->W + bw - 1) / bw; P.tiles_h = (d->H + bh - 1) / bh;
+    const int tiles_img = (d->N + bn_img - 1) / bn_img;
+    if (!P.halo) {
+        P.a = layout_kmajor(128, cb);
+        rc = make_map_nhwc(&P.mapA, in, d->N, d->H, d->W, Cred, bn_img, bh, bw, cb);
+    } else {
+        // 8-pixel groups (one image row of the box each) a halo row apart
+        P.a = layout_kmajor(128, cb);
+        P.a.tile_bytes = (uint32_t)align_up((size_t)(bh + 2) * P.halo_w * cb, 1024);
+        P.a.desc_hi = (((uint32_t)P.halo_w * cb) >> 4) | (1u << 14) | (P.a.desc_hi & 0xE0000000u);
+        rc = make_map_nhwc(&P.mapA, in, d->N, d->H, d->W, Cred, 1, bh + 2, P.halo_w, cb);
+    }
+    if (rc) return rc;
     if (out) {
         // a warp's 32 accumulator rows are a sub-box of the 128-pixel box (all extents are powers of two)
         const uint32_t sw = (uint32_t)std::min(bw, 32), sh = (uint32_t)std::min(bh, 32 / (int)sw), sn = 32 / (sw * sh);
         if ((rc = make_map_out_nhwc(&P.mapC, out, d->N, d->H, d->W, Nout, sn, sh, sw))) return rc;
     }
     P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
-    P.tiles_n = (Nout + P.bn - 1) / P.bn;
-    P.M = pix; P.N = Nout;
     P.acc_out = acc_out; P.out = out;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
     return launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st);

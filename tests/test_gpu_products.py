@@ -119,7 +119,11 @@ def test_wgrad_dense_sweep_shape_sampled_columns(B):
 # ----------------------------------------------------------- convolution
 CONVS = [(2, 8, 8, 64, 64, 1), (2, 8, 8, 64, 64, 3), (3, 10, 12, 32, 48, 3), (2, 14, 14, 128, 256, 3),
          (4, 7, 7, 256, 128, 1), (1, 1, 1, 16, 16, 3), (5, 9, 3, 80, 16, 3), (3, 28, 28, 128, 128, 3),
-         (2, 56, 56, 64, 64, 3), (1, 5, 130, 16, 272, 3)]
+         (2, 56, 56, 64, 64, 3), (1, 5, 130, 16, 272, 3),
+         # boxes loaded once with their border (taps as shifted windows): 128-, 64- and 32-byte channel chunks,
+         # several chunks per tile, ragged boxes in both directions
+         (2, 20, 17, 128, 32, 3), (2, 20, 17, 32, 128, 3), (1, 33, 9, 192, 32, 3), (2, 16, 8, 256, 16, 3),
+         (1, 40, 24, 16, 64, 3)]
 
 
 @pytest.mark.parametrize("N,H,W,C,K,R", CONVS)
