@@ -37,7 +37,7 @@
 namespace qbp {
 
 constexpr int kWgThreads = 192;
-constexpr int kWgMaxStages = 8;
+constexpr int kWgMaxStages = 16;
 constexpr int kWgMaxTiles = 4;       // A tiles (128 accumulator rows each) per CTA: 4 x 2 limbs x 64 columns fill tensor memory
 constexpr int kWgMaxLoads = 32;      // TMA loads per stage: one lane each
 constexpr int kWgMaxMmas = 128;      // MMAs per stage: 4 tiles x 4 k steps x 2 limbs, with room
@@ -50,6 +50,7 @@ struct WgradParams {
     uint32_t a_chunk_bytes;          // bytes of one A chunk (kr rows x rb_a)
     int conv;                        // 0: x [M x K], g [M x N]; 1: NHWC tensors
     int stages, cg, bn, tmem_cols;   // cg: stages released by one commit
+    int stages_last, cg_last;        // the ring of the CTAs of the last A group (fewer A tiles: smaller and more stages)
     int kr;                          // reduction rows per pipeline stage
     int a_chunks, rb_a;              // chunks per A tile, bytes (= channels / columns) per chunk row
     int ma;                          // A tiles per CTA (they share the g tiles of a stage)
@@ -68,7 +69,7 @@ struct WgradParams {
     // plain geometry
     int64_t M, N, K;
     long long *part;                 // int64 partials, one block of part_stride values per CTA
-    int64_t part_stride;             // ma * 128 * bn
+    int64_t part_stride;             // ma * 128 * bn, padded
     // direct epilogue (plain): acc = raw + rowterm[k] + colterm[n]
     const long long *rowterm, *colterm;
     const qbp_qparams *qx, *qg;
@@ -92,20 +93,95 @@ __device__ __forceinline__ WgItem wg_item(const WgradParams &P, int bid)
     return w;
 }
 
+// ---- MMA issue ------------------------------------------------------------------
+// The MMA takes its operands from the warp's few uniform registers.  What the operand layouts (row bytes RBA of the
+// x chunks, RBB of the gradient tiles = output columns per tile) and the number NT of A tiles fix is therefore
+// spelled as constants and the MMAs of a stage are fully unrolled: descriptors that were looked up per MMA, or
+// built from many run-time values, cost 110 to 150 cycles per MMA against 40 to 50 this way.
+struct WgMmaArgs {
+    uint64_t *full_bar, *empty_bar, *acc_bar;
+    uint32_t ring, stage_bytes, a_bytes, tmem;
+    int k_iters;
+    uint32_t stages, cg;
+    uint32_t a_desc_lo, b_desc_lo, idesc_hi;
+};
+
+__host__ __device__ constexpr uint32_t wg_swizzle_bits(uint32_t row_bytes) { return row_bytes == 128 ? 2u : row_bytes == 64 ? 4u : 6u; }
+
+// The 4 * NT MMAs of a stage of 64 reduction rows: the limb outermost (switching between the s8 x s8 and s8 x u8
+// instruction descriptors stalls the MMA pipe), then the k step, then the A tile, so that consecutive MMAs write
+// different accumulators.  FIRST: the stage starts the reduction (its first k step overwrites the accumulators).
+template <int RBA, int RBB, int NT, bool FIRST>
+__device__ __forceinline__ void wg_issue_stage(uint32_t tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc_hi)
+{
+    constexpr uint32_t a_hi = ((8u * RBA) >> 4) | (1u << 14) | (wg_swizzle_bits(RBA) << 29);
+    constexpr uint32_t b_hi = ((8u * RBB) >> 4) | (1u << 14) | (wg_swizzle_bits(RBB) << 29);
+    constexpr uint32_t a_kstep = 2u * RBA, b_kstep = 2u * RBB;     // 32 reduction rows, in 16-byte units
+    constexpr uint32_t a_tile16 = 64u * 128u / 16u;                // an A tile: 64 rows x 128 bytes
+    constexpr uint32_t b_tile16 = 64u * RBB / 16u;                 // a limb's tile: 64 rows x RBB bytes
+    const uint32_t idesc_lo = idesc_hi ^ (1u << 10);               // the low limb is unsigned
+#pragma unroll
+    for (int i = 0; i < 4 * NT; ++i) {
+        const int limb = i / (2 * NT), kk = (i / NT) % 2, j = i % NT;
+        const uint32_t ao = (uint32_t)j * a_tile16 + (uint32_t)kk * a_kstep;
+        const uint32_t bo = (uint32_t)limb * b_tile16 + (uint32_t)kk * b_kstep;
+        if (elect_one())
+            mma_i8(tmem + (uint32_t)((j * 2 + limb) * RBB), ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + ao),
+                   ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + bo), limb ? idesc_lo : idesc_hi, (FIRST && kk == 0) ? 0u : 1u);
+    }
+}
+
+// The MMA warp's loop over its slice of the reduction.  False when a wait ran out.
+template <int RBA, int RBB, int NT>
+__device__ __forceinline__ bool wg_mma_loop(const WgMmaArgs &A)
+{
+    uint32_t s = 0, ph = 0;
+    uint32_t in_group = 0, group = 0;          // stages issued of the current release group, its index (no divisions here:
+                                               // what this warp does between two stages leaves the MMA pipe idle)
+    uint32_t a_addr = A.ring;
+    for (int i = 0; i < A.k_iters; ++i) {
+        if (!mbar_wait_uniform(&A.full_bar[s], ph)) return false;
+        tc_fence_after();
+        const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | A.a_desc_lo;
+        const uint32_t b_lo = (((a_addr + A.a_bytes) >> 4) & 0x3FFFu) | A.b_desc_lo;
+        if (i == 0) wg_issue_stage<RBA, RBB, NT, true>(A.tmem, a_lo, b_lo, A.idesc_hi);
+        else        wg_issue_stage<RBA, RBB, NT, false>(A.tmem, a_lo, b_lo, A.idesc_hi);
+        // release the group of stages this one completes (the commit covers every MMA issued so far)
+        if (++in_group == A.cg) {
+            if (elect_one()) mma_commit(&A.empty_bar[group]);
+            in_group = 0; ++group;
+        }
+        a_addr += A.stage_bytes;
+        if (++s == A.stages) { s = 0; ph ^= 1u; group = 0; a_addr = A.ring; }
+    }
+    if (elect_one()) mma_commit(A.acc_bar);
+    return true;
+}
+
+template <int RBA, int RBB>
+__device__ __forceinline__ bool wg_mma_dispatch_nt(int nt, const WgMmaArgs &A)
+{
+    // (128 output columns per tile leave room for two A tiles in tensor memory)
+    if (nt == 1) return wg_mma_loop<RBA, RBB, 1>(A);
+    if (nt == 2) return wg_mma_loop<RBA, RBB, 2>(A);
+    if (RBB == 128) return false;
+    if (nt == 3) return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 3)>(A);
+    return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 4)>(A);
+}
+
+// One instance per pair of operand layouts: RBA = row bytes of the x chunks, RBB = row bytes of the gradient tiles.
+template <int RBA, int RBB>
 __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_constant__ WgradParams P)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kWgMaxStages], empty_bar[kWgMaxStages], acc_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ int4 s_load[kWgMaxLoads];      // (destination offset in the stage, 0 x / 1 hi / 2 lo, channel offset, tap dw | dh << 16)
-    __shared__ uint4 s_mma[kWgMaxMmas];       // (A descriptor offset, B descriptor offset, accumulator column, limb | first k step << 1)
-    __shared__ int s_counts[2];               // loads, MMAs per stage
+    __shared__ int s_counts[1];               // loads per stage
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     uint8_t *smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
     const uint32_t a_tile_bytes = P.a_chunk_bytes * (uint32_t)P.a_chunks;
-    const uint32_t a_bytes = a_tile_bytes * (uint32_t)P.ma;
-    const uint32_t stage_bytes = a_bytes + 2u * P.b.tile_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const WgItem wi = wg_item(P, blockIdx.x);
@@ -115,6 +191,10 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     const int it_end = (int)((int64_t)P.iters_total * (wi.slice + 1) / wi.slices);
     const int k_iters = it_end - it_begin;
     const int n_tiles = min(P.ma, P.a_tiles - ag * P.ma);        // A tiles this CTA owns
+    const uint32_t a_bytes = a_tile_bytes * (uint32_t)n_tiles;
+    const uint32_t stage_bytes = a_bytes + 2u * P.b.tile_bytes;
+    const bool last_group = ag == P.a_groups - 1;
+    const int stages = last_group ? P.stages_last : P.stages, cg = last_group ? P.cg_last : P.cg;
     const int kk_per_iter = P.kr / 32;
 
     // chunks present in A tile `at`: conv -- taps left in the tap group; plain -- column chunks left in K
@@ -124,7 +204,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < P.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         mbar_init(&acc_bar, 1);
         mbar_fence_init();
         tma_prefetch_desc(&P.mapX); tma_prefetch_desc(&P.mapHi); tma_prefetch_desc(&P.mapLo);
@@ -146,18 +226,6 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         }
         s_counts[0] = nl;
     }
-    if (threadIdx.x == 32) {
-        // the MMAs of one stage: the limb outermost (switching between the s8 x s8 and s8 x u8 instruction
-        // descriptors stalls the MMA pipe), then the k step, so that consecutive MMAs write different accumulators
-        int nm = 0;
-        for (int limb = 0; limb < 2; ++limb)
-            for (int kk = 0; kk < kk_per_iter; ++kk)
-                for (int j = 0; j < n_tiles; ++j)
-                    s_mma[nm++] = make_uint4(((uint32_t)j * a_tile_bytes) / 16u + (uint32_t)kk * P.a.kstep,
-                                             ((uint32_t)limb * P.b.tile_bytes) / 16u + (uint32_t)kk * P.b.kstep,
-                                             (uint32_t)((j * 2 + limb) * P.bn), (uint32_t)limb | (kk == 0 ? 2u : 0u));
-        s_counts[1] = nm;
-    }
     if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
@@ -174,12 +242,14 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         const int dw = (int)(short)(ld.w & 0xFFFF), dh = ld.w >> 16;
         const void *map = ld.y == 0 ? (const void *)&P.mapX : ld.y == 1 ? (const void *)&P.mapHi : (const void *)&P.mapLo;
         uint32_t s = 0, gph = 1;                      // stage, parity of the stage group's "empty" barrier
+        uint32_t in_group = 0, group = 0;             // position in the release group, the group's index
         for (int i = 0; i < k_iters; ++i) {
             int ok = 1;
             if (lane == 0) {
-                if (s % (uint32_t)P.cg == 0) ok = mbar_wait(&empty_bar[s / (uint32_t)P.cg], gph) ? 1 : 0;
+                if (in_group == 0) ok = mbar_wait(&empty_bar[group], gph) ? 1 : 0;
                 if (ok) mbar_expect_tx(&full_bar[s], tx_bytes);
             }
+            if (++in_group == (uint32_t)cg) { in_group = 0; ++group; }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) { timed_out = true; break; }
             if (lane < n_loads) {
@@ -196,37 +266,16 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
                 }
             }
             __syncwarp();
-            if (++s == (uint32_t)P.stages) { s = 0; gph ^= 1u; }
+            if (++s == (uint32_t)stages) { s = 0; gph ^= 1u; group = 0; }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // -------------------------------------------------- MMA issuer
-            const int n_mma = s_counts[1];
-            const uint32_t ring = smem_u32(smem);
-            const uint32_t a_desc_hi = P.a.desc_hi, b_desc_hi = P.b.desc_hi, idesc_hi = P.idesc_hi, idesc_lo = P.idesc_lo;
-            uint32_t s = 0, ph = 0;
-            for (int i = 0; i < k_iters; ++i) {
-                if (!mbar_wait(&full_bar[s], ph)) { timed_out = true; break; }
-                tc_fence_after();
-                const uint32_t a_addr = ring + s * stage_bytes;
-                const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.a.desc_lo;
-                const uint32_t b_lo = (((a_addr + a_bytes) >> 4) & 0x3FFFu) | P.b.desc_lo;
-                uint4 e = s_mma[0];
-#pragma unroll 2
-                for (int m = 0; m < n_mma; ++m) {
-                    const uint4 nxt = s_mma[m + 1 < n_mma ? m + 1 : m];      // fetched while this MMA is being issued
-                    const uint64_t da = ((uint64_t)a_desc_hi << 32) | (uint64_t)(a_lo + e.x);
-                    const uint64_t db = ((uint64_t)b_desc_hi << 32) | (uint64_t)(b_lo + e.y);
-                    mma_i8(tmem_base + e.z, da, db, (e.w & 1u) ? idesc_lo : idesc_hi, (i == 0 && (e.w & 2u)) ? 0u : 1u);
-                    e = nxt;
-                }
-                // release the group of stages this one completes (the commit covers every MMA issued so far)
-                if ((s + 1) % (uint32_t)P.cg == 0) mma_commit(&empty_bar[s / (uint32_t)P.cg]);
-                if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
-            }
-            if (!timed_out) mma_commit(&acc_bar);
-        }
-        // (the other lanes go on to the closing __syncthreads: a pending warp-level sync would slow the issuing lane)
+        // ------------------------------------------------------ MMA issuer (the whole warp in step, an elected lane issues)
+        WgMmaArgs A;
+        A.full_bar = full_bar; A.empty_bar = empty_bar; A.acc_bar = &acc_bar;
+        A.ring = smem_u32(smem); A.stage_bytes = stage_bytes; A.a_bytes = a_bytes; A.tmem = tmem_base;
+        A.k_iters = k_iters; A.stages = (uint32_t)stages; A.cg = (uint32_t)cg;
+        A.a_desc_lo = P.a.desc_lo; A.b_desc_lo = P.b.desc_lo; A.idesc_hi = P.idesc_hi;
+        timed_out = !wg_mma_dispatch_nt<RBA, RBB>(n_tiles, A);
     } else {
         // ------------------------------------------------------- epilogue
         const int quad = warp & 3;
@@ -482,9 +531,11 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
         P.tiles_c = (d->C + (int)rb_a - 1) / (int)rb_a;
         P.a_tiles = ((P.taps + P.a_chunks - 1) / P.a_chunks) * P.tiles_c;
     }
-    // A tiles per CTA: as many as tensor memory holds (two accumulators of bn columns each)
-    P.ma = std::max(1, std::min({kWgMaxTiles, 512 / (2 * P.bn), P.a_tiles}));
-    P.a_groups = (P.a_tiles + P.ma - 1) / P.ma;
+    // A tiles per CTA: at most what tensor memory holds (two accumulators of bn columns each), spread evenly over
+    // the groups that takes (5 tiles: 3 + 2 rather than 4 + 1 -- a stage of few MMAs is bound by its fixed costs)
+    const int ma_max = std::max(1, std::min({kWgMaxTiles, 512 / (2 * P.bn), P.a_tiles}));
+    P.a_groups = (P.a_tiles + ma_max - 1) / ma_max;
+    P.ma = (P.a_tiles + P.a_groups - 1) / P.a_groups;
     int cols = 32; while (cols < P.ma * 2 * P.bn) cols <<= 1;
     P.tmem_cols = cols;
     // reduction rows per stage: 64 keeps the ring deep and the release groups fine-grained
@@ -507,22 +558,27 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
         P.iters_total = P.tiles_w * P.tiles_h * ((d->N + pl.bn_img - 1) / pl.bn_img);
         P.d_tiles_w = make_fastdiv(P.tiles_w); P.d_tiles_h = make_fastdiv(P.tiles_h);
     }
-    // pipeline: stages of kr rows; one commit releases `cg` stages (at least ~24 MMAs between commits when the ring allows)
-    const uint32_t stage_bytes = P.a_chunk_bytes * P.a_chunks * P.ma + 2 * P.b.tile_bytes;
-    int stages = std::max(2, std::min<int>(kWgMaxStages, (int)((kWgSmem - 1024) / stage_bytes)));
-    const int mmas = P.ma * (int)(kr / 32) * 2;
-    int cg = 1;
-    while (cg * mmas < 24 && stages / (cg + 1) >= 2) ++cg;
-    stages -= stages % cg;
-    P.stages = stages; P.cg = cg;
-    pl.smem = (size_t)stages * stage_bytes + 1024;
+    // pipeline: stages of kr rows; one commit releases `cg` stages (some 24 MMAs between commits while that leaves
+    // three groups in the ring).  The CTAs of the last group (fewer A tiles) get a ring of their own shape.
+    const int n_last = P.a_tiles - (P.a_groups - 1) * P.ma;                 // A tiles of the last group
+    auto ring = [&](int tiles, int &stages, int &cg) {
+        const uint32_t stage_bytes = P.a_chunk_bytes * P.a_chunks * (uint32_t)tiles + 2 * P.b.tile_bytes;
+        stages = std::max(2, std::min<int>(kWgMaxStages, (int)((kWgSmem - 1024) / stage_bytes)));
+        const int mmas = tiles * (int)(kr / 32) * 2;
+        cg = 1;
+        while (cg * mmas < 24 && stages / (cg + 1) >= 3) ++cg;
+        stages -= stages % cg;
+        return (size_t)stages * stage_bytes + 1024;
+    };
+    const size_t smem_full = ring(P.ma, P.stages, P.cg);
+    const size_t smem_last = ring(n_last, P.stages_last, P.cg_last);
+    pl.smem = std::max(smem_full, smem_last);
     // split of the reductions: at most 65536 rows per CTA; with few items, enough slices to fill the machine
     // once, in proportion to an item's cost per reduction step: a fixed part (waits, the share of a commit)
-    // worth about four MMAs, plus its MMAs
+    // worth about eight MMAs, plus its MMAs
     const int max_iters = 65536 / (int)kr;
     const int min_slices = (P.iters_total + max_iters - 1) / max_iters;
-    const int n_last = P.a_tiles - (P.a_groups - 1) * P.ma;                 // A tiles of the last group
-    auto cost = [&](int tiles) { return (int64_t)(4 + tiles * (int)(kr / 32) * 2); };
+    auto cost = [&](int tiles) { return (int64_t)(8 + tiles * (int)(kr / 32) * 2); };
     const int64_t weight = ((int64_t)(P.a_groups - 1) * cost(P.ma) + cost(n_last)) * P.tiles_b;
     const int T = sm_count();
     auto slices_for = [&](int tiles) {
@@ -536,7 +592,8 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
     P.ctas_full = (P.a_groups - 1) * P.tiles_b * P.s_full;
     pl.grid = P.ctas_full + P.tiles_b * P.s_last;
     P.direct = (!d && P.s_full == 1 && P.s_last == 1) ? 1 : 0;
-    P.part_stride = (int64_t)P.ma * 128 * P.bn;
+    // (not a power of two apart: the CTAs write their blocks in step, and equal low address bits pile onto few L2 slices)
+    P.part_stride = (int64_t)P.ma * 128 * P.bn + 272;
 }
 
 static size_t wgrad_ws_bytes(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K)
@@ -660,13 +717,27 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
         if ((rc = make_map_nhwc(&P.mapHi, g_hi, d->N, d->H, d->W, d->K, pl.bn_img, pl.bh, pl.bw, rb_b))) return rc;
         if ((rc = make_map_nhwc(&P.mapLo, g_lo, d->N, d->H, d->W, d->K, pl.bn_img, pl.bh, pl.bw, rb_b))) return rc;
     }
-    static thread_local bool configured = false;
-    if (!configured) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgSmem));
-        configured = true;
+    // the kernel instance for this pair of operand layouts
+    void (*kernel)(const WgradParams) = nullptr;
+    const int layout_id = (rb_a == 128 ? 0 : rb_a == 64 ? 1 : 2) * 3 + (rb_b == 128 ? 0 : rb_b == 64 ? 1 : 2);
+    switch (layout_id) {
+    case 0: kernel = qbp_wgrad_kernel<128, 128>; break;
+    case 1: kernel = qbp_wgrad_kernel<128, 64>; break;
+    case 2: kernel = qbp_wgrad_kernel<128, 32>; break;
+    case 3: kernel = qbp_wgrad_kernel<64, 128>; break;
+    case 4: kernel = qbp_wgrad_kernel<64, 64>; break;
+    case 5: kernel = qbp_wgrad_kernel<64, 32>; break;
+    case 6: kernel = qbp_wgrad_kernel<32, 128>; break;
+    case 7: kernel = qbp_wgrad_kernel<32, 64>; break;
+    default: kernel = qbp_wgrad_kernel<32, 32>; break;
+    }
+    static thread_local bool configured[9] = {};
+    if (!configured[layout_id]) {
+        QBP_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgSmem));
+        configured[layout_id] = true;
     }
     QBP_TRACE_BEGIN(st);
-    qbp_wgrad_kernel<<<pl.grid, kWgThreads, pl.smem, st>>>(P);
+    kernel<<<pl.grid, kWgThreads, pl.smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_wgrad_kernel");
     if (!P.direct) {
         const int blocks = (int)((outs + 255) / 256);
