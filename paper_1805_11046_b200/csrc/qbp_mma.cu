@@ -156,7 +156,7 @@ enum { MODE_GEMM = 0, MODE_FPROP = 1, MODE_DGRAD = 2 };
 constexpr int kMaxStages = 16;
 constexpr int kMaxStageMmas = 256;                    // 32 operand tiles x 2 sub-tiles x 4 k steps
 constexpr int kMaxAccBufs = 8;                        // accumulator buffers in tensor memory (512 columns in all)
-constexpr int kEpiWarps = 8;                          // two per tensor-memory lane quadrant
+constexpr int kEpiWarps = 12;                         // three per tensor-memory lane quadrant
 constexpr int kMmaThreads = 64 + 32 * kEpiWarps;      // TMA warp, MMA warp, epilogue warps
 constexpr int kGroupM = 8;           // GEMM raster: tiles walk down kGroupM tile rows before moving one column right
 constexpr uint32_t kStageSlab = 32 * 128;             // epilogue staging per warp: 32 rows x 32 fp32
@@ -181,6 +181,8 @@ struct MmaParams {
     int stage_mmas;               // MMAs per stage
     int b_stage_tiles;            // filter tiles consumed per stage (resident filter)
     uint32_t stage_tx;            // bytes the TMA loads of one stage deliver
+    int egroups;                  // msub == 1: groups of four epilogue warps that take tiles in turn (at most 3, at most nbuf)
+    int ewarps;                   // epilogue warps at work (the rest of the kEpiWarps idle): 8 when msub == 2, else 4 * egroups
     int nslab;                    // epilogue staging slabs per warp (2: a store is still reading one while the next is filled)
     int iter_entries;             // entries of the k-iteration table in shared memory (conv), a multiple of 64
     int b_resident;               // conv: all filter tiles of the CTA's N tile stay in shared memory
@@ -350,15 +352,15 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
     const uint32_t a_iter = P.a.tile_bytes * (uint32_t)P.msub;               // A bytes of one k iteration
     const uint32_t a_stage = a_iter * (uint32_t)P.ips;
     const uint32_t stage_bytes = a_stage + (P.b_resident ? 0u : P.b.tile_bytes * (uint32_t)P.ips);
-    uint8_t *staging = smem + (((size_t)P.stages * stage_bytes + 1023) & ~(size_t)1023);   // kEpiWarps slabs, 1024-byte aligned
-    int4 *s_iter = reinterpret_cast<int4 *>(staging + kEpiWarps * kStageSlab * P.nslab);  // conv: one entry per k iteration
+    uint8_t *staging = smem + (((size_t)P.stages * stage_bytes + 1023) & ~(size_t)1023);   // slabs of the working epilogue warps, 1024-byte aligned
+    int4 *s_iter = reinterpret_cast<int4 *>(staging + P.ewarps * kStageSlab * P.nslab);   // conv: one entry per k iteration
     int32_t *s_cterm = reinterpret_cast<int32_t *>(s_iter + P.iter_entries);             // column terms
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         // an accumulator buffer is read by both epilogue groups (msub == 2) or by one of them
-        for (int b = 0; b < P.nbuf; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], P.msub == 2 ? kEpiWarps : kEpiWarps / 2); }
+        for (int b = 0; b < P.nbuf; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], P.msub == 2 ? 8 : 4); }
         mbar_init(&b_full, 1);
         mbar_fence_init();
         tma_prefetch_desc(&P.mapA);
@@ -490,12 +492,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
             if (!timed_out && elect_one()) mma_commit(&acc_full[buf]);
             if (++buf == (uint32_t)P.nbuf) { buf = 0; bph ^= 1u; }
         }
-    } else {
+    } else if (warp - 2 < P.ewarps) {
         // ------------------------------------------------------- epilogue
-        // msub == 2: both groups of four warps work on every tile, one 128-row sub-tile each.
-        // msub == 1: the groups take alternate tiles (and accumulator buffers), so that the latency of one
-        //            tile's read-out and store is hidden behind the other group's tile.
-        const int ew = warp - 2;                         // 0 .. kEpiWarps-1
+        // msub == 2: two groups of four warps work on every tile, one 128-row sub-tile each.
+        // msub == 1: the groups take tiles (and accumulator buffers) in turn: a warp's read-out, arithmetic and
+        //            store of a tile is one long dependent chain, so the epilogue's throughput is the number of
+        //            tiles in flight.
+        const int ew = warp - 2;                         // 0 .. P.ewarps-1
         const int quad = warp & 3;                       // the tensor-memory lanes this warp may read
         const int group = ew >> 2;
         const int row = quad * 32 + lane;
@@ -503,14 +506,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         uint32_t slab_i = 0;
         const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
         const int sub = P.msub == 2 ? group : 0;
-        const int lt_step = P.msub == 2 ? 1 : 2;
-        const int bar_id = P.msub == 2 ? 1 : 1 + group, bar_cnt = P.msub == 2 ? 32 * kEpiWarps : 128;
+        const int lt_step = P.msub == 2 ? 1 : P.egroups;
+        const int bar_id = P.msub == 2 ? 1 : 1 + group, bar_cnt = P.msub == 2 ? 256 : 128;
         const int gt = P.msub == 2 ? threadIdx.x - 64 : (threadIdx.x - 64) & 127;     // thread index within the barrier group
         int32_t *region = s_cterm + (P.cterm_all || P.msub == 2 ? 0 : group * P.ncls * P.bn);
         if (P.cterm_all) {
             // the whole column-term table fits: fill it once
-            for (int i = threadIdx.x - 64; i < P.ncls * (int)P.N; i += 32 * kEpiWarps) s_cterm[i] = __ldg(P.colterm + i);
-            named_barrier(1, 32 * kEpiWarps);
+            for (int i = threadIdx.x - 64; i < P.ncls * (int)P.N; i += 32 * P.ewarps) s_cterm[i] = __ldg(P.colterm + i);
+            named_barrier(4, 32 * P.ewarps);
         }
 
         // where this thread's accumulator row of a tile goes
@@ -710,11 +713,16 @@ __global__ void __launch_bounds__(256) conv_rowterm_kernel(const int32_t *__rest
 // slabs, the tables, the column terms (the whole table when it is small, else one tile's columns per epilogue group).
 static uint32_t fixed_smem(MmaParams &P)
 {
+    // several small accumulators let the MMAs run ahead of the epilogue (msub == 1: one per epilogue group in turn)
+    P.nbuf = std::min(kMaxAccBufs, 512 / (P.msub * P.bn));
+    P.egroups = P.msub == 2 ? 2 : std::min(kEpiWarps / 4, P.nbuf);
+    if (P.msub == 1) P.nbuf -= P.nbuf % P.egroups;
+    P.ewarps = 4 * P.egroups;
     P.cterm_all = (size_t)P.ncls * P.N * sizeof(int32_t) <= 32u * 1024u ? 1 : 0;
     const size_t cterm_bytes = P.cterm_all ? ((size_t)P.ncls * P.N + 64) * sizeof(int32_t)
-                                           : (size_t)(P.msub == 1 ? 2 : 1) * P.ncls * P.bn * sizeof(int32_t);
+                                           : (size_t)(P.msub == 1 ? P.egroups : 1) * P.ncls * P.bn * sizeof(int32_t);
     P.iter_entries = P.mode == MODE_GEMM ? 0 : (int)align_up((size_t)P.k_iters, 64);
-    return 2048u + kEpiWarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + 
+    return 2048u + (uint32_t)P.ewarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + 
            (uint32_t)align_up(cterm_bytes, 1024);
 }
 
@@ -763,9 +771,6 @@ static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
     if (stages < 2) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "tensor-core tile does not fit shared memory");
     stages = std::min(stages, kMaxStages);
     P.stages = stages;
-    // several small accumulators let the MMAs run ahead of the epilogue (msub == 1: groups alternate, so an even count)
-    P.nbuf = std::min(kMaxAccBufs, 512 / (P.msub * P.bn));
-    if (P.msub == 1) P.nbuf &= ~1;
     int cols = 32; while (cols < P.nbuf * P.msub * P.bn) cols <<= 1;
     P.tmem_cols = cols;
     P.tiles_m = tiles_m;
@@ -980,7 +985,7 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
 
     MmaParams P{};
     P.mode = dgrad ? MODE_DGRAD : MODE_FPROP;
-    P.msub = 1; P.ncls = 16; P.nslab = 2;
+    P.msub = 1; P.ncls = 16; P.nslab = 1;
     P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.S = d->S; P.Cred = Cred;
     const uint32_t cb = Cred % 128 == 0 ? 128u : Cred % 64 == 0 ? 64u : 32u;      // reduction bytes per stage row
     P.chunk_bytes = (int)cb;
@@ -1013,9 +1018,12 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
         const long long tiles_free = (long long)((d->W + (1 << bwl) - 1) >> bwl) * ((d->H + (1 << bhl) - 1) >> bhl) *
                                      ((d->N + (128 >> (bwl + bhl)) - 1) / (128 >> (bwl + bhl)));
         const long long tiles_halo = (long long)((d->W + 7) / 8) * ((d->H + 15) / 16) * d->N;
+        P.nslab = 2;                  // (two slabs per warp: a store is still reading one while the next is filled)
         if (tiles_halo * 2 <= tiles_free * 3 && halo_fits(P, halo_bytes)) {
             P.halo = 1; P.halo_w = kHaloW; bwl = 3; bhl = 4;
             P.halo_rb = dgrad ? (Nout >= 128 ? 128 : Nout >= 64 ? 64 : 32) : 0;
+        } else {
+            P.nslab = 1;
         }
     }
     P.bw_log2 = bwl; P.bh_log2 = bhl;

@@ -406,6 +406,95 @@ __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restri
         if (s_acc[i] != 0) atomicAdd(&sums[i], (unsigned long long)(long long)s_acc[i]);
 }
 
+// The same sums, one image row per block step: thread (w, g) owns 16 channels of column w, so its border class
+// in the w direction never changes, and the row's class is the same for the whole block.  The sums over all rows
+// stay in 16 registers; the first and last row of an image (a few percent of the rows) are added to their row sets
+// in shared memory as well.  No division per pixel, and atomics only for those rows.
+// gs = 16-channel groups per block (a power of two, W * gs <= 256); blockIdx.y selects the channel slab.
+template <bool IS_SIGNED>
+__global__ void __launch_bounds__(256, 3) row_class_sums_kernel(const uint8_t *__restrict__ q, int Nimg, int H, int W,
+                                                                int C, int gs, unsigned long long *__restrict__ sums)
+{
+    extern __shared__ int s_acc[];                       // [3 row sets: all, first, last][4 column classes][gs * 16]
+    const int cw = gs * 16;
+    for (int i = threadIdx.x; i < 12 * cw; i += 256) s_acc[i] = 0;
+    __syncthreads();
+    const int w = threadIdx.x / gs, gl = threadIdx.x % gs;
+    const int g = blockIdx.y * gs + gl;
+    const bool active = w < W && g < (C >> 4);
+    const int colclass = (w == 0 ? 1 : 0) | (w == W - 1 ? 2 : 0);
+    const int lane = threadIdx.x & 31;
+    const int64_t row_bytes = (int64_t)W * C;
+    const uint8_t *base = q + (int64_t)(active ? w : 0) * C + (int64_t)(active ? g : 0) * 16;
+    constexpr int U = 8;                                 // rows in flight per thread
+
+    int acc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0;
+    const bool interior = active && colclass == 0;
+    {
+        // (every thread walks the rows, the idle ones without loading: the shuffles below need whole warps)
+        const int rows = Nimg * H, step = (int)gridDim.x, hstep = step % H;
+        int h = (int)blockIdx.x % H;
+        for (int r = (int)blockIdx.x; r < rows; r += U * step) {
+            uint4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (active && r + u * step < rows) v[u] = __ldcs(reinterpret_cast<const uint4 *>(base + (int64_t)(r + u * step) * row_bytes));
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (r + u * step >= rows) break;
+                const uint32_t wd[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)          // one byte per dot product: the selector picks it, sign- or zero-extended
+                        acc[k * 4 + b] = IS_SIGNED ? __dp4a((int)wd[k], 1 << (8 * b), acc[k * 4 + b])
+                                                   : (int)__dp4a(wd[k], 1u << (8 * b), (unsigned)acc[k * 4 + b]);
+                if (active && H > 1 && (h == 0 || h == H - 1)) {
+                    // a first or last row (the same for the whole block, and rare): its codes also go to that row set
+                    int *dst = &s_acc[((h == 0 ? 1 : 2) * 4 + colclass) * cw + gl * 16];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+#pragma unroll
+                        for (int b = 0; b < 4; ++b)
+                            atomicAdd(dst + k * 4 + b, IS_SIGNED ? (int)(int8_t)(wd[k] >> (8 * b)) : (int)((wd[k] >> (8 * b)) & 0xFF));
+                }
+                h += hstep; if (h >= H) h -= H;
+            }
+        }
+    }
+    {
+        // all rows, reduced the same way
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            int r = interior ? acc[e] : 0;
+            for (int off = gs; off < 32; off <<= 1) r += __shfl_xor_sync(0xffffffffu, r, off);
+            const int ch = gl * 16 + e;
+            if (lane < gs && r) atomicAdd(&s_acc[0 * cw + ch], r);
+            if (active && colclass != 0 && acc[e]) atomicAdd(&s_acc[colclass * cw + ch], acc[e]);
+        }
+    }
+    __syncthreads();
+    // exclusive classes (bit 1: first row, 2: last row, 4: first column, 8: last column); a single row is both
+    for (int i = threadIdx.x; i < 4 * cw; i += 256) {
+        const int cc = i / cw, c = (int)blockIdx.y * cw + i % cw;
+        if (c >= C) continue;
+        const int colbits = (cc & 1 ? 4 : 0) | (cc & 2 ? 8 : 0);
+        const int all = s_acc[(0 * 4 + cc) * cw + i % cw], top = s_acc[(1 * 4 + cc) * cw + i % cw], bot = s_acc[(2 * 4 + cc) * cw + i % cw];
+        if (H == 1) {
+            if (all) atomicAdd(&sums[(3 | colbits) * C + c], (unsigned long long)(long long)all);
+        } else {
+            const int mid = all - top - bot;
+            if (mid) atomicAdd(&sums[(0 | colbits) * C + c], (unsigned long long)(long long)mid);
+            if (top) atomicAdd(&sums[(1 | colbits) * C + c], (unsigned long long)(long long)top);
+            if (bot) atomicAdd(&sums[(2 | colbits) * C + c], (unsigned long long)(long long)bot);
+        }
+    }
+}
+
 // Plain product, direct epilogue: rowterm[k] = -zg * SX[k] + M*zx*zg, colterm[n] = -zx * (256*SHI[n] + SLO[n]).
 __global__ void wgrad_terms_kernel(const long long *__restrict__ sx, const long long *__restrict__ shi,
                                    const long long *__restrict__ slo, int64_t M, int64_t N, int64_t K,
@@ -619,6 +708,22 @@ static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C,
         configured[IS_SIGNED] = true;
     }
     if (pixels >= (1ll << 30)) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad: more than 2^30 positions");
+    if (W <= 256) {
+        // a block step is one image row: W columns x gs channel groups of 16
+        const int cv = C / 16;
+        int gs = 1; while (gs * 2 <= cv && gs * 2 * W <= 256 && gs < 16) gs *= 2;
+        const int slabs = (cv + gs - 1) / gs;
+        const int64_t rows = pixels / W;
+        const int Nimg = (int)(rows / H);
+        // int32 registers: a thread sees at most rows / grid * 255 per channel
+        int64_t grid_x = std::min<int64_t>(rows, std::max<int64_t>(1, (int64_t)sm_count() * 3 / slabs));
+        grid_x = std::max<int64_t>(grid_x, rows / (1 << 22) + 1);
+        QBP_TRACE_BEGIN(st);
+        row_class_sums_kernel<IS_SIGNED><<<dim3((unsigned)grid_x, (unsigned)slabs), 256, (size_t)12 * gs * 16 * sizeof(int), st>>>(
+            (const uint8_t *)q, Nimg, H, W, C, gs, (unsigned long long *)sums);
+        QBP_LAUNCH_OK("class_sums_kernel");
+        return QBP_OK;
+    }
     // int32 partials: a thread sees at most pixels / grid * 255 per channel.  Few blocks (each ends with up to
     // 16*C atomics on the same 16*C sums), eight 16-byte loads in flight per thread.
     const int cv = C / 16, tw = cv < 256 ? cv : 256, rpb = 256 / tw;
