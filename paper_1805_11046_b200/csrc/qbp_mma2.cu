@@ -102,6 +102,66 @@ __device__ __forceinline__ void mma_commit_pair(uint64_t *bar)
                  : "memory");
 }
 
+// ---- MMA issue ------------------------------------------------------------------
+// The MMA takes its operands from the warp's few uniform registers: the loop is written for a whole converged warp
+// with an elected issuer, its MMAs unrolled with constant offsets, and what the operand layout fixes (the k step:
+// 2 sixteen-byte units inside a K-major row, 256 between the 32-row blocks of an M/N-major tile; the upper descriptor
+// word: 128-byte swizzle, 8-row groups 1024 bytes apart) is spelled as constants.
+struct Pair2MmaArgs {
+    uint64_t *full_bar, *empty_bar, *acc_full, *acc_empty;
+    uint32_t ring, stage_bytes, a_bytes, tmem, a_desc_lo, b_desc_lo, idesc;
+    int k_iters;
+    uint32_t stages, cg, nbuf;
+    int tile0, tiles_total, tile_step;
+};
+
+template <uint32_t AK, uint32_t BK, int MSUB, bool FIRST>
+__device__ __forceinline__ void pair_issue_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc)
+{
+    constexpr uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    constexpr uint32_t a_tile16 = 128u * 128u / 16u;              // a CTA's half of one 256-row sub-tile
+#pragma unroll
+    for (int i = 0; i < 4 * MSUB; ++i) {
+        const int kk = i / MSUB, sub = i % MSUB;
+        if (elect_one())
+            mma_i8_pair(d_tmem + 256u * (uint32_t)sub, ((uint64_t)hi << 32) | (uint64_t)(a_lo + (uint32_t)sub * a_tile16 + (uint32_t)kk * AK),
+                        ((uint64_t)hi << 32) | (uint64_t)(b_lo + (uint32_t)kk * BK), idesc, (FIRST && kk == 0) ? 0u : 1u);
+    }
+}
+
+// False when a wait ran out.
+template <uint32_t AK, uint32_t BK, int MSUB>
+__device__ __forceinline__ bool pair_mma_loop(const Pair2MmaArgs &A)
+{
+    uint32_t s = 0, ph = 0, buf = 0, bph = 1;
+    uint32_t in_group = 0, group = 0;              // stages issued of the current release group, its index
+    uint32_t a_addr = A.ring;
+    for (int tile = A.tile0; tile < A.tiles_total; tile += A.tile_step) {
+        if (!mbar_wait_uniform(&A.acc_empty[buf], bph)) return false;
+        tc_fence_after();
+        const uint32_t d_tmem = A.tmem + buf * 256u;              // MSUB == 2: one set, sub-tile s at column 256 s
+        for (int it = 0; it < A.k_iters; ++it) {
+            if (!mbar_wait_uniform(&A.full_bar[s], ph)) return false;
+            tc_fence_after();
+            const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | A.a_desc_lo;
+            const uint32_t b_lo = (((a_addr + A.a_bytes) >> 4) & 0x3FFFu) | A.b_desc_lo;
+            if (it == 0) pair_issue_stage<AK, BK, MSUB, true>(d_tmem, a_lo, b_lo, A.idesc);
+            else         pair_issue_stage<AK, BK, MSUB, false>(d_tmem, a_lo, b_lo, A.idesc);
+            // release the group of stages this one completes, in both CTAs (the last group of a tile too: the
+            // commit of acc_full below covers the same MMAs, but the producers wait on "empty")
+            if (++in_group == A.cg) {
+                if (elect_one()) mma_commit_pair(&A.empty_bar[group]);
+                in_group = 0; ++group;
+            }
+            a_addr += A.stage_bytes;
+            if (++s == A.stages) { s = 0; ph ^= 1u; group = 0; a_addr = A.ring; }
+        }
+        if (elect_one()) mma_commit_pair(&A.acc_full[buf]);
+        if (++buf == A.nbuf) { buf = 0; bph ^= 1u; }
+    }
+    return true;
+}
+
 struct Tile2 { int m0, n0; };
 __device__ __forceinline__ Tile2 tile2_origin(const Mma2Params &P, int tile)
 {
@@ -152,12 +212,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(k2Threads, 1) qbp_mm
         if (lane == 0) {
             // ---------------------------------------------------- TMA producer (both CTAs)
             const uint32_t cg = (uint32_t)P.cg;
-            uint32_t s = 0, gph = 1;
+            uint32_t s = 0, gph = 1, in_group = 0, group = 0;
             for (int tile = pair; tile < P.tiles_total && !timed_out; tile += P.pairs) {
                 const Tile2 o = tile2_origin(P, tile);
                 const int m_mine = o.m0 + 128 * (int)rank, n_mine = o.n0 + 128 * (int)rank;   // sub-tile s: + 256 s rows
                 for (int it = 0; it < P.k_iters; ++it) {
-                    if (s % cg == 0 && !mbar_wait(&empty_bar[s / cg], gph)) { timed_out = true; break; }
+                    if (in_group == 0 && !mbar_wait(&empty_bar[group], gph)) { timed_out = true; break; }
+                    if (++in_group == cg) { in_group = 0; ++group; }
                     uint8_t *sa = smem + (size_t)s * stage_bytes;
                     uint8_t *sb = sa + a_bytes;
                     const uint32_t bar = map_to_cta(&full_bar[s], 0);
@@ -169,41 +230,29 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(k2Threads, 1) qbp_mm
                     }
                     if (P.b.major == 0) tma_load_2d_pair(sb, &P.mapB, bar, k0, n_mine);
                     else                tma_load_2d_pair(sb, &P.mapB, bar, n_mine, k0);
-                    if (++s == (uint32_t)P.stages) { s = 0; gph ^= 1u; }
+                    if (++s == (uint32_t)P.stages) { s = 0; gph ^= 1u; group = 0; }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
-            // -------------------------------------------------- MMA issuer (leader CTA only)
-            const uint32_t ring = smem_u32(smem);
-            const uint32_t cg = (uint32_t)P.cg;
-            uint32_t s = 0, ph = 0, buf = 0, bph = 1;
-            for (int tile = pair; tile < P.tiles_total && !timed_out; tile += P.pairs) {
-                if (!mbar_wait(&acc_empty[buf], bph)) { timed_out = true; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * 256u;          // msub == 2: one set, sub-tile s at column 256 s
-                for (int it = 0; it < P.k_iters; ++it) {
-                    if (!mbar_wait(&full_bar[s], ph)) { timed_out = true; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = ring + s * stage_bytes, b_addr = a_addr + a_bytes;
-                    const uint32_t b_lo = ((b_addr >> 4) & 0x3FFFu) | P.b.desc_lo;
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        for (int sub = 0; sub < P.msub; ++sub) {
-                            const uint32_t a_lo = (((a_addr + sub * P.a.tile_bytes) >> 4) & 0x3FFFu) | P.a.desc_lo;
-                            mma_i8_pair(d_tmem + 256u * sub, ((uint64_t)P.a.desc_hi << 32) | (uint64_t)(a_lo + kk * P.a.kstep),
-                                        ((uint64_t)P.b.desc_hi << 32) | (uint64_t)(b_lo + kk * P.b.kstep), P.idesc,
-                                        (it | kk) != 0 ? 1u : 0u);
-                        }
-                    // release the group of stages this one completes, in both CTAs (the last group of a tile too:
-                    // the commit of acc_full below covers the same MMAs, but the producers wait on "empty")
-                    if ((s + 1) % cg == 0) mma_commit_pair(&empty_bar[s / cg]);
-                    if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
-                }
-                if (!timed_out) mma_commit_pair(&acc_full[buf]);
-                if (++buf == (uint32_t)P.nbuf) { buf = 0; bph ^= 1u; }
+        if (rank == 0) {
+            // ---------------------------------------------------- MMA issuer (leader CTA only): the whole warp in step,
+            // an elected lane issues; one instance of the loop per pair of operand layouts and tile height
+            Pair2MmaArgs A;
+            A.full_bar = full_bar; A.empty_bar = empty_bar; A.acc_full = acc_full; A.acc_empty = acc_empty;
+            A.ring = smem_u32(smem); A.stage_bytes = stage_bytes; A.a_bytes = a_bytes; A.tmem = tmem_base;
+            A.a_desc_lo = P.a.desc_lo; A.b_desc_lo = P.b.desc_lo; A.idesc = P.idesc;
+            A.k_iters = P.k_iters; A.stages = (uint32_t)P.stages; A.cg = (uint32_t)P.cg; A.nbuf = (uint32_t)P.nbuf;
+            A.tile0 = pair; A.tiles_total = P.tiles_total; A.tile_step = P.pairs;
+            bool ok;
+            if (P.msub == 2) {
+                if (P.a.major == 0) ok = P.b.major == 0 ? pair_mma_loop<2, 2, 2>(A) : pair_mma_loop<2, 256, 2>(A);
+                else                ok = P.b.major == 0 ? pair_mma_loop<256, 2, 2>(A) : pair_mma_loop<256, 256, 2>(A);
+            } else {
+                if (P.a.major == 0) ok = P.b.major == 0 ? pair_mma_loop<2, 2, 1>(A) : pair_mma_loop<2, 256, 1>(A);
+                else                ok = P.b.major == 0 ? pair_mma_loop<256, 2, 1>(A) : pair_mma_loop<256, 256, 1>(A);
             }
+            timed_out = !ok;
         }
     } else {
         // ------------------------------------------------------- epilogue (each CTA drains its own 128 rows)
@@ -303,13 +352,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(k2Threads, 1) qbp_mm
     if (warp == 1) { __syncwarp(); tmem_dealloc_pair(tmem_base, 512); }
 }
 
-// Whether the pair kernel takes this product: at least eight rounds of 256 x 256 tiles over the CTA pairs. Below
-// that the single-CTA kernel's finer tile schedule (and its shorter fill and drain) wins.
+// Whether the pair kernel takes this product: anything with at least one whole pair tile's worth of rows and columns
+// (it is the faster kernel from 1024^3 up; the single-CTA kernel keeps the narrow shapes).
 bool gemm2_eligible(int64_t M, int64_t N, int64_t K)
 {
-    if (M < 256 || N < 256 || K < 128) return false;
-    const int64_t tiles = ((M + 255) / 256) * ((N + 255) / 256);
-    return tiles >= 8 * (int64_t)(sm_count() / 2);
+    return M >= 256 && N >= 256 && K >= 128;
 }
 
 int launch_gemm2(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
