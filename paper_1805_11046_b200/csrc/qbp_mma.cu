@@ -259,8 +259,10 @@ __device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
 // at run time next to the per-stage addresses the compiler ran out of them and each MMA cost 130 cycles instead of 40.
 constexpr int kHaloW = 10;           // pixels per row of a halo tile: the 8-pixel box row and one border pixel each side
 __host__ __device__ constexpr uint32_t swizzle_bits(uint32_t row_bytes) { return row_bytes == 128 ? 2u : row_bytes == 64 ? 4u : 6u; }
-template <int MPI, int RB>
-__device__ __forceinline__ void issue_halo_3x3(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t b_tile16, uint32_t idesc,
+// BN: the output columns of the tile when they are one of the common counts (then the filter tile size and the
+// instruction descriptor are constants too), 0: taken from the launch parameters.
+template <int MPI, int RB, int BN>
+__device__ __forceinline__ void issue_halo_3x3(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t b_tile16_rt, uint32_t idesc_rt,
                                                uint32_t first_acc)
 {
     constexpr bool FWD = RB == 0;
@@ -270,6 +272,10 @@ __device__ __forceinline__ void issue_halo_3x3(uint32_t d, uint32_t a_lo, uint32
     constexpr uint32_t b_hi = FWD ? ((8u * cb) >> 4) | (1u << 14) | (swizzle_bits(cb) << 29)
                                   : ((8u * (uint32_t)RB) >> 4) | (1u << 14) | (swizzle_bits((uint32_t)RB) << 29);
     constexpr uint32_t b_kstep = FWD ? 2u : (32u * (uint32_t)RB) >> 4;
+    // a filter tile is BN x 32 * MPI bytes either way round; s8 x s8 -> s32, M = 128, N = BN, B M/N-major for the gradient
+    const uint32_t b_tile16 = BN ? (uint32_t)(2 * MPI * BN) : b_tile16_rt;
+    const uint32_t idesc = BN ? (2u << 4) | (1u << 7) | (1u << 10) | ((FWD ? 0u : 1u) << 16) | (((uint32_t)BN >> 3) << 17) | ((128u >> 4) << 24)
+                              : idesc_rt;
 #pragma unroll
     for (int i = 0; i < 9 * MPI; ++i) {
         const int tap = i / MPI, kk = i % MPI, r = tap / 3, t = tap % 3;
@@ -282,13 +288,21 @@ __device__ __forceinline__ void issue_halo_3x3(uint32_t d, uint32_t a_lo, uint32
 }
 
 template <int MPI>
-__device__ __forceinline__ void issue_halo_3x3_any(int rb, uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t b_tile16,
+__device__ __forceinline__ void issue_halo_3x3_any(int rb, int bn, uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t b_tile16,
                                                    uint32_t idesc, uint32_t first_acc)
 {
-    if (rb == 0)        issue_halo_3x3<MPI, 0>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
-    else if (rb == 128) issue_halo_3x3<MPI, 128>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
-    else if (rb == 64)  issue_halo_3x3<MPI, 64>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
-    else                issue_halo_3x3<MPI, 32>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    if (rb == 0) {
+        if (bn == 64)       issue_halo_3x3<MPI, 0, 64>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+        else if (bn == 128) issue_halo_3x3<MPI, 0, 128>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+        else                issue_halo_3x3<MPI, 0, 0>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    } else if (rb == 128) {
+        if (bn == 128)      issue_halo_3x3<MPI, 128, 128>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+        else                issue_halo_3x3<MPI, 128, 0>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    } else if (rb == 64) {
+        issue_halo_3x3<MPI, 64, 64>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    } else {
+        issue_halo_3x3<MPI, 32, 32>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
+    }
 }
 
 __device__ __forceinline__ void issue_stage(const MmaParams &P, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
@@ -324,9 +338,9 @@ __device__ __forceinline__ void issue_stage(const MmaParams &P, uint32_t a_lo, u
         const uint32_t b_chunk16 = 9u * b_tile16;             // the nine filter tiles of one channel chunk
         for (int hj = 0; hj < P.ips; ++hj) {
             const uint32_t acc0 = hj == 0 ? first_acc : 1u;
-            if (P.mma_per_iter == 4)      issue_halo_3x3_any<4>(P.halo_rb, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
-            else if (P.mma_per_iter == 2) issue_halo_3x3_any<2>(P.halo_rb, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
-            else                          issue_halo_3x3_any<1>(P.halo_rb, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
+            if (P.mma_per_iter == 4)      issue_halo_3x3_any<4>(P.halo_rb, P.bn, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
+            else if (P.mma_per_iter == 2) issue_halo_3x3_any<2>(P.halo_rb, P.bn, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
+            else                          issue_halo_3x3_any<1>(P.halo_rb, P.bn, d_tmem, a_lo, b_lo, b_tile16, P.idesc, acc0);
             a_lo += a_tile16; b_lo += b_chunk16;
         }
     }
