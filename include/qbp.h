@@ -168,10 +168,26 @@ int qbp_bifurcate(const float *g, int64_t rows, int64_t cols, uint64_t seed,
  * ---------------------------------------------------------------------- */
 size_t qbp_gemm_s8_workspace_bytes(int64_t M, int64_t N, int64_t K);
 
+/* Optional extra work of a product's epilogue.  Section 3's Range BN needs
+ * the mean, minimum and maximum of every output channel of the layer; they
+ * are taken here from the fp32 outputs as they are written, so that the
+ * normalisation that follows needs no statistics pass of its own.
+ * col_sum (double), col_min, col_max: [N] each (device), all three or none;
+ * they receive the sum / minimum / maximum over the M rows of each column
+ * of C (of each output channel over all positions for a convolution).
+ * Needs C (out) non-NULL and N <= QBP_EPILOGUE_MAX_COLUMNS, else
+ * QBP_ERR_UNSUPPORTED_SHAPE.  ep == NULL: none of it. */
+#define QBP_EPILOGUE_MAX_COLUMNS 256
+typedef struct qbp_epilogue {
+    double *col_sum;
+    float *col_min;
+    float *col_max;
+} qbp_epilogue;
+
 int qbp_gemm_s8(int transA, int transB, int64_t M, int64_t N, int64_t K,
                 const int8_t *A, const qbp_qparams *qa,
                 const int8_t *B, const qbp_qparams *qb,
-                int32_t *acc_out, float *C,
+                int32_t *acc_out, float *C, const qbp_epilogue *ep,
                 void *ws, size_t ws_bytes, void *stream);
 
 /* The same products for a convolution, computed as an implicit GEMM over
@@ -183,7 +199,7 @@ size_t qbp_conv_s8_workspace_bytes(int mode, const qbp_conv_desc *d);
 int qbp_conv_s8_implicit(int mode, const qbp_conv_desc *d,
                          const int8_t *in, const qbp_qparams *q_in,
                          const int8_t *w, const qbp_qparams *q_w,
-                         int32_t *acc_out, float *out,
+                         int32_t *acc_out, float *out, const qbp_epilogue *ep,
                          void *ws, size_t ws_bytes, void *stream);
 
 /* ------------------------------------------------------------------------

@@ -194,30 +194,51 @@ def qbp_bifurcate(g, seed, tensor_id8, tensor_id16, q8=None, hi=None, lo=None, q
 
 
 # ------------------------------------------------------------------- products
-def qbp_gemm_s8(A, qa, B, qb, transA=False, transB=False, want_acc=False, want_out=True, acc_out=None, out=None, ws=None):
+class Epilogue(C.Structure):
+    """qbp_epilogue: device pointers [N] that receive the per-column sum / min / max of the fp32 output."""
+    _fields_ = [("col_sum", C.c_void_p), ("col_min", C.c_void_p), ("col_max", C.c_void_p)]
+
+
+def _epilogue(col_stats, n, device):
+    """col_stats: None, True (allocate), or a (sum f64, min f32, max f32) triple of device tensors."""
+    if not col_stats:
+        return None, None
+    if col_stats is True:
+        col_stats = (torch.empty(n, dtype=torch.float64, device=device), torch.empty(n, dtype=torch.float32, device=device),
+                     torch.empty(n, dtype=torch.float32, device=device))
+    ep = Epilogue(col_stats[0].data_ptr(), col_stats[1].data_ptr(), col_stats[2].data_ptr())
+    return ep, col_stats
+
+
+def qbp_gemm_s8(A, qa, B, qb, transA=False, transB=False, want_acc=False, want_out=True, acc_out=None, out=None, ws=None,
+                col_stats=None):
     if transA: K, M = A.shape
     else:      M, K = A.shape
     N = B.shape[0] if transB else B.shape[1]
     if want_acc and acc_out is None: acc_out = torch.empty((M, N), dtype=torch.int32, device=A.device)
     if want_out and out is None: out = torch.empty((M, N), dtype=torch.float32, device=A.device)
     if ws is None: ws = workspace(lib.qbp_gemm_s8_workspace_bytes(M, N, K), A.device)
+    ep, stats = _epilogue(col_stats, N, A.device)
     _check(lib.qbp_gemm_s8(int(transA), int(transB), C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A), _ptr(qa),
-                           _ptr(B), _ptr(qb), _ptr(acc_out), _ptr(out), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
-    return acc_out, out, ws
+                           _ptr(B), _ptr(qb), _ptr(acc_out), _ptr(out), C.byref(ep) if ep else None, _ptr(ws),
+                           C.c_size_t(ws.numel()), _stream()))
+    return (acc_out, out, ws, stats) if col_stats else (acc_out, out, ws)
 
 
 def conv_desc(N, H, W, C_in, K, R, S, stride=1, pad=0) -> ConvDesc:
     return ConvDesc(N, H, W, C_in, K, R, S, stride, pad)
 
 
-def qbp_conv_s8_implicit(mode, d: ConvDesc, inp, q_in, w, q_w, want_acc=False, want_out=True, acc_out=None, out=None, ws=None):
+def qbp_conv_s8_implicit(mode, d: ConvDesc, inp, q_in, w, q_w, want_acc=False, want_out=True, acc_out=None, out=None, ws=None,
+                         col_stats=None):
     shape = (d.N, d.H, d.W, d.K) if mode == QBP_CONV_FPROP else (d.N, d.H, d.W, d.C)
     if want_acc and acc_out is None: acc_out = torch.empty(shape, dtype=torch.int32, device=inp.device)
     if want_out and out is None: out = torch.empty(shape, dtype=torch.float32, device=inp.device)
     if ws is None: ws = workspace(lib.qbp_conv_s8_workspace_bytes(mode, C.byref(d)), inp.device)
+    ep, stats = _epilogue(col_stats, shape[3], inp.device)
     _check(lib.qbp_conv_s8_implicit(mode, C.byref(d), _ptr(inp), _ptr(q_in), _ptr(w), _ptr(q_w), _ptr(acc_out),
-                                    _ptr(out), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
-    return acc_out, out, ws
+                                    _ptr(out), C.byref(ep) if ep else None, _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return (acc_out, out, ws, stats) if col_stats else (acc_out, out, ws)
 
 
 def qbp_wgrad_s16(x, qx, g_hi, g_lo, qg16, d: ConvDesc | None = None, want_acc=False, want_out=True,

@@ -59,9 +59,14 @@ static size_t step_scratch_bytes(const qbp_layer_desc *L, const LayerShape &s)
 // Buffers that live across steps, behind the shared step scratch: the per-row sums of the codes feeding the
 // next product (written by the quantiser that makes the codes) and the range partials of the gradient
 // (written by the Range BN backward pass that makes the gradient).
+static bool epilogue_stats(const LayerShape &s) { return s.conv && s.cout <= QBP_EPILOGUE_MAX_COLUMNS; }
+static size_t colstat_cells(const LayerShape &s) { return epilogue_stats(s) ? (size_t)colstat_rows_max() * (size_t)s.cout : 0; }
 static size_t chained_bytes(const LayerShape &s)
 {
-    return align_up(sizeof(int32_t) * (size_t)s.rows, 256) + align_up(sizeof(float2) * rangebn_range_parts_capacity(s.cout), 256);
+    // ... and the per-channel (sum, min, max) partials of the layer output that the convolution's epilogue leaves
+    // for the Range BN forward
+    return align_up(sizeof(int32_t) * (size_t)s.rows, 256) + align_up(sizeof(float2) * rangebn_range_parts_capacity(s.cout), 256) +
+           2 * align_up(sizeof(float) * colstat_cells(s), 256) + align_up(sizeof(double) * colstat_cells(s), 256);
 }
 
 }  // namespace qbp
@@ -103,13 +108,25 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_la
     rc = qbp_quantize_s8(w, w_rows, s.w_elems / w_rows, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr,
                          saved->w_codes, saved->qw, nullptr, nullptr, ws, scratch, stream);
     if (rc) return rc;
+    ColStatParts parts{nullptr, nullptr, nullptr, 0};
+    if (epilogue_stats(s)) {
+        char *base = static_cast<char *>(ws) + scratch + align_up(sizeof(int32_t) * (size_t)s.rows, 256) +
+                     align_up(sizeof(float2) * rangebn_range_parts_capacity(s.cout), 256);
+        parts.lo = reinterpret_cast<float *>(base);
+        parts.hi = reinterpret_cast<float *>(base + align_up(sizeof(float) * colstat_cells(s), 256));
+        parts.sum = reinterpret_cast<double *>(base + 2 * align_up(sizeof(float) * colstat_cells(s), 256));
+    }
     if (s.conv)
         rc = conv_s8_impl(QBP_CONV_FPROP, &L->conv, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr, saved->z,
-                          row_sums, ws, scratch, (cudaStream_t)stream);
+                          row_sums, parts.sum ? &parts : nullptr, ws, scratch, (cudaStream_t)stream);
     else
         rc = qbp_gemm_s8(0, 0, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr,
-                         saved->z, ws, scratch, stream);
+                         saved->z, nullptr, ws, scratch, stream);
     if (rc) return rc;
+    // the convolution's epilogue has left the statistics of z: no pass over z for them
+    if (parts.sum)
+        return rangebn_fwd_from_parts(saved->z, s.rows, s.cout, gamma, beta, L->relu, y, saved->save_mean, saved->save_min,
+                                      saved->save_max, parts, (cudaStream_t)stream);
     return qbp_rangebn_fwd(saved->z, s.rows, s.cout, gamma, beta, L->relu, y, saved->save_mean, saved->save_min,
                            saved->save_max, nullptr, ws, scratch, stream);
 }
@@ -148,12 +165,12 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st);
     if (rc) return rc;
     if (s.conv) {
-        rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, ws, scratch, st);
+        rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, nullptr, ws, scratch, st);
         if (rc) return rc;
         return qbp_wgrad_s16(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, ws, scratch, stream);
     }
     // dx [batch x in] = g8 [batch x out] . w^T, w stored [in x out]
-    rc = qbp_gemm_s8(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, ws, scratch, stream);
+    rc = qbp_gemm_s8(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, nullptr, ws, scratch, stream);
     if (rc) return rc;
     return qbp_wgrad_s16(nullptr, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, ws,
                          scratch, stream);

@@ -184,6 +184,12 @@ struct MmaParams {
     int egroups;                  // msub == 1: groups of four epilogue warps that take tiles in turn (at most 3, at most nbuf)
     int ewarps;                   // epilogue warps at work (the rest of the kEpiWarps idle): 8 when msub == 2, else 4 * egroups
     int nslab;                    // epilogue staging slabs per warp (2: a store is still reading one while the next is filled)
+    // Per-column statistics of the fp32 output (for the Range BN that follows, Section 3): every working epilogue
+    // warp keeps (sum, min, max) of the columns in shared memory and leaves them as row blockIdx.x * ewarps + warp of
+    // these partial arrays [rows][N] when the kernel ends.  One column tile only (N <= 256); NULL: not wanted.
+    float *st_lo, *st_hi; double *st_sum;
+    int grid;                     // CTAs launched
+    uint32_t cterm_span;          // bytes of the column-term region in shared memory (the statistics follow it)
     int iter_entries;             // entries of the k-iteration table in shared memory (conv), a multiple of 64
     int b_resident;               // conv: all filter tiles of the CTA's N tile stay in shared memory
     uint32_t b_res_bytes;         // bytes reserved for them at the start of shared memory
@@ -205,6 +211,7 @@ struct MmaParams {
 };
 
 struct TileOrigin { int m0, n0, img0, h0, w0; };
+struct ColStat { double sum; float lo, hi; };
 
 __device__ __forceinline__ TileOrigin tile_origin(const MmaParams &P, int tile)
 {
@@ -369,6 +376,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
     uint8_t *staging = smem + (((size_t)P.stages * stage_bytes + 1023) & ~(size_t)1023);   // slabs of the working epilogue warps, 1024-byte aligned
     int4 *s_iter = reinterpret_cast<int4 *>(staging + P.ewarps * kStageSlab * P.nslab);   // conv: one entry per k iteration
     int32_t *s_cterm = reinterpret_cast<int32_t *>(s_iter + P.iter_entries);             // column terms
+    ColStat *s_stat = reinterpret_cast<ColStat *>(reinterpret_cast<uint8_t *>(s_cterm) + P.cterm_span);   // [ewarps][N]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -519,6 +527,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         uint8_t *slab0 = staging + (size_t)(ew * P.nslab) * kStageSlab;
         uint32_t slab_i = 0;
         const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
+        ColStat *my_stat = s_stat + (size_t)ew * P.N;
+        if (P.st_sum) {
+            for (int i = lane; i < (int)P.N; i += 32) { my_stat[i].sum = 0.0; my_stat[i].lo = INFINITY; my_stat[i].hi = -INFINITY; }
+            __syncwarp();
+        }
         const int sub = P.msub == 2 ? group : 0;
         const int lt_step = P.msub == 2 ? 1 : P.egroups;
         const int bar_id = P.msub == 2 ? 1 : 1 + group, bar_cnt = P.msub == 2 ? 256 : 128;
@@ -635,6 +648,22 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                             else                     tma_store_4d(&P.mapC, slab, o.n0 + c0, ri.sx, ri.sy, ri.sz);
                             tma_store_commit();
                         }
+                        if (P.st_sum) {
+                            // lane = column of the slab: its 32 rows (the valid ones) read back from shared memory
+                            // (a row's 32 floats lie in one 128-byte line whatever the swizzle: no bank conflicts)
+                            const unsigned vmask = __ballot_sync(0xffffffffu, ri.valid);
+                            float cs = 0.0f, clo = INFINITY, chi = -INFINITY;
+#pragma unroll 8
+                            for (int r = 0; r < 32; ++r) {
+                                if (!((vmask >> r) & 1u)) continue;
+                                const float v = *reinterpret_cast<const float *>(slab + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2)));
+                                cs += v; clo = fminf(clo, v); chi = fmaxf(chi, v);
+                            }
+                            if (lane < lim && vmask) {
+                                ColStat &a = my_stat[o.n0 + c0 + lane];
+                                a.sum += (double)cs; a.lo = fminf(a.lo, clo); a.hi = fmaxf(a.hi, chi);
+                            }
+                        }
                     }
                 }
             }
@@ -644,6 +673,12 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
+        if (P.st_sum) {
+            const int64_t prow = ((int64_t)blockIdx.x * P.ewarps + ew) * P.N;
+            for (int i = lane; i < (int)P.N; i += 32) {
+                P.st_sum[prow + i] = my_stat[i].sum; P.st_lo[prow + i] = my_stat[i].lo; P.st_hi[prow + i] = my_stat[i].hi;
+            }
+        }
     }
 
     if (timed_out) {
@@ -722,6 +757,58 @@ __global__ void __launch_bounds__(256) conv_rowterm_kernel(const int32_t *__rest
     rowterm[m] = -zb * box + taps * Cred * za * zb;
 }
 
+// Per-column sum / min / max from the epilogue warps' partial rows: one block of 128 threads per column.
+__global__ void __launch_bounds__(128) colstat_finalize_kernel(const float *__restrict__ part_lo, const float *__restrict__ part_hi,
+                                                               const double *__restrict__ part_sum, int rows, int N,
+                                                               double *__restrict__ col_sum, float *__restrict__ col_min,
+                                                               float *__restrict__ col_max)
+{
+    const int c = blockIdx.x;
+    float lo = INFINITY, hi = -INFINITY;
+    double sum = 0.0;
+    for (int i = threadIdx.x; i < rows; i += 128) {
+        lo = fminf(lo, part_lo[(int64_t)i * N + c]); hi = fmaxf(hi, part_hi[(int64_t)i * N + c]); sum += part_sum[(int64_t)i * N + c];
+    }
+    lo = warp_min(lo); hi = warp_max(hi);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    __shared__ float s_lo[4], s_hi[4];
+    __shared__ double s_sum[4];
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; s_sum[threadIdx.x >> 5] = sum; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 4; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); sum += s_sum[w]; }
+        col_sum[c] = sum; col_min[c] = lo; col_max[c] = hi;
+    }
+}
+
+int colstat_rows_max() { return sm_count() * kEpiWarps; }
+
+static size_t colstat_ws_bytes(int64_t N)
+{
+    if (N > QBP_EPILOGUE_MAX_COLUMNS) return 0;
+    const size_t cells = (size_t)colstat_rows_max() * (size_t)N;
+    return align_up(cells * sizeof(float), 256) * 2 + align_up(cells * sizeof(double), 256);
+}
+
+static int check_epilogue(const char *who, const qbp_epilogue *ep, const float *out, int64_t N, bool &wanted)
+{
+    wanted = ep && (ep->col_sum || ep->col_min || ep->col_max);
+    if (!wanted) return QBP_OK;
+    if (!ep->col_sum || !ep->col_min || !ep->col_max) return fail(QBP_ERR_INVALID_ARG, "%s: the epilogue needs col_sum, col_min and col_max together", who);
+    if (!out) return fail(QBP_ERR_INVALID_ARG, "%s: column statistics need the fp32 output", who);
+    if (N > QBP_EPILOGUE_MAX_COLUMNS) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "%s: column statistics for at most %d columns", who, QBP_EPILOGUE_MAX_COLUMNS);
+    return QBP_OK;
+}
+
+static int finish_epilogue(const qbp_epilogue *ep, const ColStatParts &parts, int64_t N, cudaStream_t st)
+{
+    QBP_TRACE_BEGIN(st);
+    colstat_finalize_kernel<<<(int)N, 128, 0, st>>>(parts.lo, parts.hi, parts.sum, parts.rows, (int)N, ep->col_sum, ep->col_min, ep->col_max);
+    QBP_LAUNCH_OK("colstat_finalize_kernel");
+    return QBP_OK;
+}
+
 // ================================================================== launchers
 // Shared memory of the kernel that is not the stage ring or the resident filter: alignment slack, epilogue staging
 // slabs, the tables, the column terms (the whole table when it is small, else one tile's columns per epilogue group).
@@ -736,8 +823,9 @@ static uint32_t fixed_smem(MmaParams &P)
     const size_t cterm_bytes = P.cterm_all ? ((size_t)P.ncls * P.N + 64) * sizeof(int32_t)
                                            : (size_t)(P.msub == 1 ? P.egroups : 1) * P.ncls * P.bn * sizeof(int32_t);
     P.iter_entries = P.mode == MODE_GEMM ? 0 : (int)align_up((size_t)P.k_iters, 64);
-    return 2048u + (uint32_t)P.ewarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + 
-           (uint32_t)align_up(cterm_bytes, 1024);
+    P.cterm_span = (uint32_t)align_up(cterm_bytes, 1024);
+    const uint32_t stat_bytes = P.st_sum ? (uint32_t)align_up((size_t)P.ewarps * P.N * sizeof(ColStat), 1024) : 0u;
+    return 2048u + (uint32_t)P.ewarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + P.cterm_span + stat_bytes;
 }
 
 // Whether a convolution can run from halo tiles: the whole filter resident beside at least three halo tiles.
@@ -802,6 +890,7 @@ static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
     QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
     // one CTA per SM (its shared-memory ring fills the SM), each walking its share of the tiles
     const int grid = std::min(P.tiles_total, sm_count());
+    P.grid = grid;
     QBP_TRACE_BEGIN(st);
     qbp_mma_kernel<<<grid, kMmaThreads, smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_mma_kernel");
@@ -811,7 +900,7 @@ static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
 static size_t gemm_ws_bytes(int64_t M, int64_t N)
 {
     return 256 + align_up(sizeof(int32_t) * M, 256) + align_up(sizeof(int32_t) * N, 256) +
-           align_up(sizeof(int64_t) * M, 256) + align_up(sizeof(int64_t) * N, 256);
+           align_up(sizeof(int64_t) * M, 256) + align_up(sizeof(int64_t) * N, 256) + colstat_ws_bytes(N);
 }
 
 static bool conv_supported(const qbp_conv_desc *d)
@@ -820,12 +909,18 @@ static bool conv_supported(const qbp_conv_desc *d)
            d->H > 0 && d->W > 0 && d->C > 0 && d->K > 0 && d->C % 16 == 0 && d->K % 16 == 0;
 }
 
-static size_t conv_ws_bytes(const qbp_conv_desc *d)
+// What the product itself carves from the workspace, and with the room for the column statistics' partial rows
+// (at its end) that the public entry point may need.
+static size_t conv_core_ws_bytes(const qbp_conv_desc *d)
 {
     const int64_t pix = (int64_t)d->N * d->H * d->W;
     const int64_t nmax = std::max(d->C, d->K);
     return 256 + align_up(sizeof(int32_t) * pix, 256) * 2 + align_up(sizeof(int32_t) * 16 * nmax, 256) +
            align_up(sizeof(int64_t) * (int64_t)d->R * d->S * nmax, 256);
+}
+static size_t conv_ws_bytes(const qbp_conv_desc *d)
+{
+    return conv_core_ws_bytes(d) + std::max(colstat_ws_bytes(d->C), colstat_ws_bytes(d->K));
 }
 
 // Picks the pixel box (bw x bh x bn = 128, powers of two) that wastes the fewest MMA rows.
@@ -854,7 +949,7 @@ extern "C" __attribute__((visibility("default"))) size_t qbp_gemm_s8_workspace_b
 
 extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A,
                            const qbp_qparams *qa, const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C,
-                           void *ws, size_t ws_bytes, void *stream)
+                           const qbp_epilogue *ep, void *ws, size_t ws_bytes, void *stream)
 {
     cudaStream_t st = (cudaStream_t)stream;
     if (M <= 0 || N <= 0 || K <= 0) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: M, N, K must be positive");
@@ -868,12 +963,22 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     if (!ws || ws_bytes < gemm_ws_bytes(M, N))
         return fail(QBP_ERR_WORKSPACE, "gemm_s8: workspace of %zu bytes needed, %zu given", gemm_ws_bytes(M, N), ws_bytes);
 
+    bool stats = false;
+    {
+        const int erc = check_epilogue("gemm_s8", ep, C, N, stats);
+        if (erc) return erc;
+    }
     WsCarver w(ws, ws_bytes);
     int *status = w.take<int>(1);
     int32_t *rowterm = w.take<int32_t>(M);
     int32_t *colterm = w.take<int32_t>(N);
     int64_t *tmp_m = w.take<int64_t>(M);
     int64_t *tmp_n = w.take<int64_t>(N);
+    ColStatParts parts{nullptr, nullptr, nullptr, 0};
+    if (stats) {
+        const size_t cells = (size_t)colstat_rows_max() * (size_t)N;
+        parts.lo = w.take<float>(cells); parts.hi = w.take<float>(cells); parts.sum = w.take<double>(cells);
+    }
 
     // code sums along the reduction
     int rc;
@@ -891,8 +996,9 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
         rowterm, colterm);
     QBP_LAUNCH_OK("gemm_terms_kernel");
 
-    // large products run on CTA pairs (256 x 256 tiles across two SMs)
-    if (gemm2_eligible(M, N, K))
+    // large products run on CTA pairs (256 x 256 tiles across two SMs); the column statistics are the
+    // single-CTA kernel's (at most 256 columns: narrow either way)
+    if (gemm2_eligible(M, N, K) && !stats)
         return launch_gemm2(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, rowterm, colterm, status, st);
 
     MmaParams P{};
@@ -932,7 +1038,10 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     P.M = M; P.N = N;
     P.acc_out = acc_out; P.out = C;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = qa; P.qb = qb; P.status = status;
-    return launch_mma(P, (int)((M + 128 * P.msub - 1) / (128 * P.msub)), st);
+    if (stats) { P.st_lo = parts.lo; P.st_hi = parts.hi; P.st_sum = parts.sum; }
+    if ((rc = launch_mma(P, (int)((M + 128 * P.msub - 1) / (128 * P.msub)), st))) return rc;
+    if (stats) { parts.rows = P.grid * P.ewarps; return finish_epilogue(ep, parts, N, st); }
+    return QBP_OK;
 }
 
 extern "C" __attribute__((visibility("default"))) size_t qbp_conv_s8_workspace_bytes(int mode, const qbp_conv_desc *d)
@@ -943,15 +1052,39 @@ extern "C" __attribute__((visibility("default"))) size_t qbp_conv_s8_workspace_b
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in,
-                                    const int8_t *wgt, const qbp_qparams *q_w, int32_t *acc_out, float *out, void *ws,
-                                    size_t ws_bytes, void *stream)
+                                    const int8_t *wgt, const qbp_qparams *q_w, int32_t *acc_out, float *out,
+                                    const qbp_epilogue *ep, void *ws, size_t ws_bytes, void *stream)
 {
-    return conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+    bool stats = false;
+    if (d && ep) {
+        const int64_t Nout = mode == QBP_CONV_DGRAD ? d->C : d->K;
+        const int erc = check_epilogue("conv_s8", ep, out, Nout, stats);
+        if (erc) return erc;
+        if (stats) {
+            // the partial rows sit at the end of the workspace, behind what the product itself carves
+            if (!conv_supported(d))
+                return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: needs stride 1, R = S in {1,3}, pad = (R-1)/2, C and K multiples of 16");
+            const size_t core = conv_core_ws_bytes(d), need = conv_ws_bytes(d);
+            if (!ws || ws_bytes < need)
+                return fail(QBP_ERR_WORKSPACE, "conv_s8: workspace of %zu bytes needed, %zu given", need, ws_bytes);
+            const size_t cells = (size_t)colstat_rows_max() * (size_t)Nout;
+            char *base = static_cast<char *>(ws) + core;
+            ColStatParts parts;
+            parts.lo = reinterpret_cast<float *>(base);
+            parts.hi = reinterpret_cast<float *>(base + align_up(cells * sizeof(float), 256));
+            parts.sum = reinterpret_cast<double *>(base + 2 * align_up(cells * sizeof(float), 256));
+            parts.rows = 0;
+            const int rc = conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, &parts, ws, core, (cudaStream_t)stream);
+            if (rc) return rc;
+            return finish_epilogue(ep, parts, Nout, (cudaStream_t)stream);
+        }
+    }
+    return conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, nullptr, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
-                      const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, void *ws,
-                      size_t ws_bytes, cudaStream_t st)
+                      const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, ColStatParts *stats,
+                      void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (!d) return fail(QBP_ERR_INVALID_ARG, "conv_s8: descriptor is NULL");
     if (mode != QBP_CONV_FPROP && mode != QBP_CONV_DGRAD) return fail(QBP_ERR_INVALID_ARG, "conv_s8: bad mode");
@@ -965,8 +1098,10 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     if (!acc_out && !out) return fail(QBP_ERR_INVALID_ARG, "conv_s8: acc_out and out are both NULL");
     if (!aligned16(in) || !aligned16(wgt) || (out && !aligned16(out)) || (acc_out && !aligned16(acc_out)))
         return fail(QBP_ERR_INVALID_ARG, "conv_s8: operands must be 16-byte aligned");
-    if (!ws || ws_bytes < conv_ws_bytes(d))
+    if (!ws || ws_bytes < conv_core_ws_bytes(d))
         return fail(QBP_ERR_WORKSPACE, "conv_s8: workspace of %zu bytes needed, %zu given", conv_ws_bytes(d), ws_bytes);
+    if (stats && (!out || (mode == QBP_CONV_DGRAD ? d->C : d->K) > QBP_EPILOGUE_MAX_COLUMNS))
+        return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: column statistics need the fp32 output and at most %d channels", QBP_EPILOGUE_MAX_COLUMNS);
 
     const bool dgrad = mode == QBP_CONV_DGRAD;
     const int Cred = dgrad ? d->K : d->C;        // channels reduced over
@@ -1000,6 +1135,7 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     MmaParams P{};
     P.mode = dgrad ? MODE_DGRAD : MODE_FPROP;
     P.msub = 1; P.ncls = 16; P.nslab = 1;
+    if (stats) { P.st_lo = stats->lo; P.st_hi = stats->hi; P.st_sum = stats->sum; }
     P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.S = d->S; P.Cred = Cred;
     const uint32_t cb = Cred % 128 == 0 ? 128u : Cred % 64 == 0 ? 64u : 32u;      // reduction bytes per stage row
     P.chunk_bytes = (int)cb;
@@ -1063,5 +1199,7 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
     P.acc_out = acc_out; P.out = out;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
-    return launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st);
+    if ((rc = launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st))) return rc;
+    if (stats) stats->rows = P.grid * P.ewarps;
+    return QBP_OK;
 }

@@ -26,9 +26,16 @@ int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, ui
                                   uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st);
 // The convolution products with the per-pixel channel sums of the input codes supplied by the caller
 // (nullable: computed here) (qbp_mma.cu).
+// Per-column (sum, min, max) of a product's fp32 output as partial rows [rows][N], one per working epilogue warp
+// of the tensor-core kernel; `rows` is filled in by the launch.  colstat_rows_max(): the most rows a launch leaves.
+struct ColStatParts { float *lo, *hi; double *sum; int rows; };
+int colstat_rows_max();
 int conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
-                 const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, void *ws,
-                 size_t ws_bytes, cudaStream_t st);
+                 const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, ColStatParts *stats,
+                 void *ws, size_t ws_bytes, cudaStream_t st);
+// Range BN forward from such partials instead of a statistics pass over x (qbp_rangebn.cu).
+int rangebn_fwd_from_parts(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu, float *y,
+                           float *save_mean, float *save_min, float *save_max, const ColStatParts &parts, cudaStream_t st);
 
 // ---- TMA tensor maps ---------------------------------------------------------
 // A dense byte matrix [rows x cols] (cols innermost) read in boxes of

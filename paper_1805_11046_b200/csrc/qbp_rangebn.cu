@@ -425,6 +425,34 @@ QBP_TRACE_BEGIN(st);
     return QBP_OK;
 }
 
+// Forward from per-column partials of x that its producer left (rows of [C]: sum, min, max), without a statistics
+// pass over x: finalize, then the apply pass.
+int qbp::rangebn_fwd_from_parts(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu,
+                                float *y, float *save_mean, float *save_min, float *save_max, const ColStatParts &parts,
+                                cudaStream_t st)
+{
+    if (!x || !y || !save_mean || !save_min || !save_max || !parts.lo || !parts.hi || !parts.sum || parts.rows <= 0)
+        return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: NULL tensor");
+    if (n < 2 || C <= 0) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: needs n >= 2 rows");
+    const bool al = aligned16(x) && aligned16(y);
+    const bool v4 = al && C % 4 == 0;
+    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_apply_kernel<4, true>, kScanThreads)
+                                                       : blocks_per_sm(bn_apply_kernel<4, false>, kScanThreads))
+                                               : blocks_per_sm(bn_apply_kernel<1, true>, kScanThreads));
+    const dim3 grid_apply(ga.nbx, ga.slabs);
+    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
+    QBP_TRACE_BEGIN(st);
+    bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(parts.lo, parts.hi, parts.sum, parts.rows, (int)C, n, save_mean, save_min, save_max);
+    QBP_LAUNCH_OK("bn_stats_finalize_kernel");
+    QBP_TRACE_BEGIN(st);
+#define QBP_BN_APPLY(V, R) bn_apply_kernel<V, R><<<grid_apply, kScanThreads, 0, st>>>(x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, y)
+    if (ga.vec == 4) { if (relu) QBP_BN_APPLY(4, true); else QBP_BN_APPLY(4, false); }
+    else             { if (relu) QBP_BN_APPLY(1, true); else QBP_BN_APPLY(1, false); }
+#undef QBP_BN_APPLY
+    QBP_LAUNCH_OK("bn_apply_kernel");
+    return QBP_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma,
                                const float *beta, int relu, const float *save_mean, const float *save_min,
                                const float *save_max, float *dx, float *dgamma, float *dbeta, void *ws,

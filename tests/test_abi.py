@@ -56,20 +56,20 @@ def test_host_side_refusals(lib):
                                C.c_size_t(1 << 30), null) == -1
     assert "at least 2" in _err(lib)
     # reduction too long for an int32 accumulator of 8-bit codes
-    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(33040), fake, fake, fake, fake, null, fake, fake,
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(33040), fake, fake, fake, fake, null, fake, null, fake,
                            C.c_size_t(1 << 30), null) == -3
     assert "33025" in _err(lib)
     # shapes the tensor-core path does not take
-    assert lib.qbp_gemm_s8(0, 0, i64(100), i64(128), i64(128), fake, fake, fake, fake, null, fake, fake,
+    assert lib.qbp_gemm_s8(0, 0, i64(100), i64(128), i64(128), fake, fake, fake, fake, null, fake, null, fake,
                            C.c_size_t(1 << 30), null) == -2
     # both outputs missing; NULL operand; misaligned operand; too small a workspace
-    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, null, fake,
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, null, null, fake,
                            C.c_size_t(1 << 30), null) == -1
-    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), null, fake, fake, fake, null, fake, fake,
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), null, fake, fake, fake, null, fake, null, fake,
                            C.c_size_t(1 << 30), null) == -1
-    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), C.c_void_p(4100), fake, fake, fake, null, fake, fake,
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), C.c_void_p(4100), fake, fake, fake, null, fake, null, fake,
                            C.c_size_t(1 << 30), null) == -1
-    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, fake, fake,
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, fake, null, fake,
                            C.c_size_t(16), null) == -4
     assert "workspace" in _err(lib)
     # quantiser enums
@@ -85,8 +85,21 @@ def test_convolution_shapes_outside_the_implementation_are_refused(lib):
     for d in (ConvDesc(1, 8, 8, 64, 64, 3, 3, 2, 1),      # stride 2
               ConvDesc(1, 8, 8, 64, 64, 5, 5, 1, 2),      # 5x5
               ConvDesc(1, 8, 8, 24, 64, 3, 3, 1, 1)):     # channels not a multiple of 16
-        assert lib.qbp_conv_s8_implicit(0, C.byref(d), fake, fake, fake, fake, null, fake, fake, C.c_size_t(1 << 30),
+        assert lib.qbp_conv_s8_implicit(0, C.byref(d), fake, fake, fake, fake, null, fake, null, fake, C.c_size_t(1 << 30),
                                         null) == -2
+
+
+def test_epilogue_statistics_need_all_three_buffers_the_output_and_few_columns(lib):
+    from paper_1805_11046_b200.binding import Epilogue
+    fake = C.c_void_p(4096); null = C.c_void_p(0); i64 = C.c_int64
+    part = Epilogue(4096, 0, 4096)
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, fake, C.byref(part), fake,
+                           C.c_size_t(1 << 30), null) == -1
+    full = Epilogue(4096, 4096, 4096)
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, fake, null, C.byref(full), fake,
+                           C.c_size_t(1 << 30), null) == -1              # no fp32 output to take them from
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(512), i64(128), fake, fake, fake, fake, null, fake, C.byref(full), fake,
+                           C.c_size_t(1 << 30), null) == -2              # more than 256 columns
 
 
 def test_workspace_queries_are_pure(lib):

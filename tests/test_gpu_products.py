@@ -100,6 +100,44 @@ def test_gemm_s8_pair_kernel_ragged_sampled_rows(B, M, N, K, tA, tB):
     assert np.array_equal(to_host(acc[rows]), oacc) and np.array_equal(to_host(out[rows]), oout)
 
 
+# ------------------------------------------- column statistics from the epilogue
+def _check_col_stats(out, stats):
+    o = to_host(out).reshape(-1, out.shape[-1]).astype(np.float64)
+    csum, cmin, cmax = (to_host(t) for t in stats)
+    assert np.array_equal(cmin, o.min(axis=0).astype(np.float32)) and np.array_equal(cmax, o.max(axis=0).astype(np.float32))
+    # partial sums of at most 32 fp32 values in fp32, the rest in fp64
+    assert np.allclose(csum, o.sum(axis=0), rtol=0, atol=1e-6 * np.abs(o).sum(axis=0).max())
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (208, 80, 144), (1024, 256, 512), (2000, 64, 64)])
+def test_gemm_epilogue_column_statistics(B, M, N, K):
+    """Section 3: the sum, minimum and maximum of every output column, as the following Range BN needs them, taken
+    from the fp32 outputs in the product's epilogue; the product itself is unchanged."""
+    A = random_codes((M, K), 21); Bm = random_codes((K, N), 22)
+    za, zb, sa, sb = 5, -9, 0.5, 0.125
+    acc, out, ws, stats = B.qbp_gemm_s8(to_dev(A), _qp(B, sa, za), to_dev(Bm), _qp(B, sb, zb), want_acc=True, col_stats=True)
+    oacc, oout, bad = O.gemm_s8(A, za, Bm, zb, sa, sb)
+    assert bad == 0 and B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(out), oout)
+    _check_col_stats(out, stats)
+
+
+@pytest.mark.parametrize("N,H,W,C,K,R", [(2, 56, 56, 64, 64, 3), (3, 10, 12, 32, 48, 3), (4, 7, 7, 256, 128, 1), (2, 20, 17, 128, 32, 3)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_conv_epilogue_channel_statistics(B, N, H, W, C, K, R, mode):
+    """The same for a convolution (ragged pixel boxes: positions outside the image must not count)."""
+    pad = (R - 1) // 2
+    d = B.conv_desc(N, H, W, C, K, R, R, 1, pad); od = O.conv_desc(N, H, W, C, K, R, R, 1, pad)
+    inp = random_codes((N, H, W, C if mode == 0 else K), 23); w = random_codes((K, R, R, C), 24)
+    zi, zw = -3, 11
+    acc, out, ws, stats = B.qbp_conv_s8_implicit(mode, d, to_dev(inp), _qp(B, 0.5, zi), to_dev(w), _qp(B, 0.25, zw),
+                                                 want_acc=True, col_stats=True)
+    oacc, oout, bad = O.conv_s8(mode, od, inp, zi, w, zw, 0.5, 0.25)
+    assert bad == 0 and B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(out), oout)
+    _check_col_stats(out, stats)
+
+
 def test_wgrad_dense_sweep_shape_sampled_columns(B):
     """The limb-split 16 x 8-bit product at 4096^3 (dense sweep): operands quantised from N(0,1) (nearest for the
     8-bit side, stochastic for the 16-bit side); oracle on 96 sampled output columns (all 4096 rows of each)."""
