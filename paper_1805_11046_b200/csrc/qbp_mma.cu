@@ -185,8 +185,8 @@ struct MmaParams {
     int ewarps;                   // epilogue warps at work (the rest of the kEpiWarps idle): 8 when msub == 2, else 4 * egroups
     int nslab;                    // epilogue staging slabs per warp (2: a store is still reading one while the next is filled)
     // Per-column statistics of the fp32 output (for the Range BN that follows, Section 3): every working epilogue
-    // warp keeps (sum, min, max) of the columns in shared memory and leaves them as row blockIdx.x * ewarps + warp of
-    // these partial arrays [rows][N] when the kernel ends.  One column tile only (N <= 256); NULL: not wanted.
+    // warp keeps (sum, min, max) of the columns in shared memory; when the kernel ends the CTA's warps add them up
+    // into row blockIdx.x of these partial arrays [rows][N].  One column tile only (N <= 256); NULL: not wanted.
     float *st_lo, *st_hi; double *st_sum;
     int grid;                     // CTAs launched
     uint32_t cterm_span;          // bytes of the column-term region in shared memory (the statistics follow it)
@@ -653,11 +653,24 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                             // (a row's 32 floats lie in one 128-byte line whatever the swizzle: no bank conflicts)
                             const unsigned vmask = __ballot_sync(0xffffffffu, ri.valid);
                             float cs = 0.0f, clo = INFINITY, chi = -INFINITY;
+                            if (vmask == 0xffffffffu) {
+                                // (rows r and r + 8 swizzle alike: eight base addresses, the rest constant offsets)
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const uint8_t *colp = slab + k * 128 + ((((lane >> 2) ^ k) << 4) | ((lane & 3) << 2));
+#pragma unroll
+                                    for (int r8 = 0; r8 < 4; ++r8) {
+                                        const float v = *reinterpret_cast<const float *>(colp + r8 * 1024);
+                                        cs += v; clo = fminf(clo, v); chi = fmaxf(chi, v);
+                                    }
+                                }
+                            } else {
 #pragma unroll 8
-                            for (int r = 0; r < 32; ++r) {
-                                if (!((vmask >> r) & 1u)) continue;
-                                const float v = *reinterpret_cast<const float *>(slab + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2)));
-                                cs += v; clo = fminf(clo, v); chi = fmaxf(chi, v);
+                                for (int r = 0; r < 32; ++r) {
+                                    if (!((vmask >> r) & 1u)) continue;
+                                    const float v = *reinterpret_cast<const float *>(slab + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2)));
+                                    cs += v; clo = fminf(clo, v); chi = fmaxf(chi, v);
+                                }
                             }
                             if (lane < lim && vmask) {
                                 ColStat &a = my_stat[o.n0 + c0 + lane];
@@ -674,9 +687,16 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
         if (P.st_sum) {
-            const int64_t prow = ((int64_t)blockIdx.x * P.ewarps + ew) * P.N;
-            for (int i = lane; i < (int)P.N; i += 32) {
-                P.st_sum[prow + i] = my_stat[i].sum; P.st_lo[prow + i] = my_stat[i].lo; P.st_hi[prow + i] = my_stat[i].hi;
+            // the CTA's warps together: one partial row per CTA
+            named_barrier(5, 32 * P.ewarps);
+            const int64_t prow = (int64_t)blockIdx.x * P.N;
+            for (int i = ew * 32 + lane; i < (int)P.N; i += 32 * P.ewarps) {
+                double sum = 0.0; float lo = INFINITY, hi = -INFINITY;
+                for (int w = 0; w < P.ewarps; ++w) {
+                    const ColStat &a = s_stat[(size_t)w * P.N + i];
+                    sum += a.sum; lo = fminf(lo, a.lo); hi = fmaxf(hi, a.hi);
+                }
+                P.st_sum[prow + i] = sum; P.st_lo[prow + i] = lo; P.st_hi[prow + i] = hi;
             }
         }
     }
@@ -782,7 +802,7 @@ __global__ void __launch_bounds__(128) colstat_finalize_kernel(const float *__re
     }
 }
 
-int colstat_rows_max() { return sm_count() * kEpiWarps; }
+int colstat_rows_max() { return sm_count(); }
 
 static size_t colstat_ws_bytes(int64_t N)
 {
@@ -1040,7 +1060,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     P.rowterm = rowterm; P.colterm = colterm; P.qa = qa; P.qb = qb; P.status = status;
     if (stats) { P.st_lo = parts.lo; P.st_hi = parts.hi; P.st_sum = parts.sum; }
     if ((rc = launch_mma(P, (int)((M + 128 * P.msub - 1) / (128 * P.msub)), st))) return rc;
-    if (stats) { parts.rows = P.grid * P.ewarps; return finish_epilogue(ep, parts, N, st); }
+    if (stats) { parts.rows = P.grid; return finish_epilogue(ep, parts, N, st); }
     return QBP_OK;
 }
 
@@ -1200,6 +1220,6 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     P.acc_out = acc_out; P.out = out;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
     if ((rc = launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st))) return rc;
-    if (stats) stats->rows = P.grid * P.ewarps;
+    if (stats) stats->rows = P.grid;
     return QBP_OK;
 }

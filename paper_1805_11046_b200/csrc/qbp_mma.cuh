@@ -26,7 +26,7 @@ int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, ui
                                   uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st);
 // The convolution products with the per-pixel channel sums of the input codes supplied by the caller
 // (nullable: computed here) (qbp_mma.cu).
-// Per-column (sum, min, max) of a product's fp32 output as partial rows [rows][N], one per working epilogue warp
+// Per-column (sum, min, max) of a product's fp32 output as partial rows [rows][N], one per CTA
 // of the tensor-core kernel; `rows` is filled in by the launch.  colstat_rows_max(): the most rows a launch leaves.
 struct ColStatParts { float *lo, *hi; double *sum; int rows; };
 int colstat_rows_max();
