@@ -115,7 +115,7 @@ KERNEL_WORK = {
     ("range_partial_kernel", 2): (4, 0), ("quantize_kernel", 2): (7, 0),            # bifurcation: 4 B in, 1 + 2 B out
     ("rowsum_kernel", 2): (1, 0),                                                   # channel sums of the 8-bit gradient codes
     ("qbp_mma_kernel", 1): (5, OPS_PER_ELEMENT_CONV),                               # dgrad
-    ("class_sums_kernel", 0): (1, 0), ("class_sums_kernel", 1): (1, 0), ("class_sums_kernel", 2): (1, 0),
+    ("class_sums_kernel", 0): (3, 0),                                               # x, hi and lo codes in one launch
     ("qbp_wgrad_kernel", 0): (3, 2 * OPS_PER_ELEMENT_CONV),                         # two int8 products per 16x8-bit product
 }
 

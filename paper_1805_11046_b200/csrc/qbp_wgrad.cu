@@ -412,8 +412,8 @@ __global__ void __launch_bounds__(256) class_sums_kernel(const uint8_t *__restri
 // in shared memory as well.  No division per pixel, and atomics only for those rows.
 // gs = 16-channel groups per block (a power of two, W * gs <= 256); blockIdx.y selects the channel slab.
 template <bool IS_SIGNED>
-__global__ void __launch_bounds__(256, 3) row_class_sums_kernel(const uint8_t *__restrict__ q, int Nimg, int H, int W,
-                                                                int C, int gs, unsigned long long *__restrict__ sums)
+__device__ __forceinline__ void row_class_sums_body(const uint8_t *__restrict__ q, int Nimg, int H, int W, int C, int gs,
+                                                    unsigned long long *__restrict__ sums)
 {
     extern __shared__ int s_acc[];                       // [3 row sets: all, first, last][4 column classes][gs * 16]
     const int cw = gs * 16;
@@ -493,6 +493,24 @@ __global__ void __launch_bounds__(256, 3) row_class_sums_kernel(const uint8_t *_
             if (bot) atomicAdd(&sums[(2 | colbits) * C + c], (unsigned long long)(long long)bot);
         }
     }
+}
+
+template <bool IS_SIGNED>
+__global__ void __launch_bounds__(256, 3) row_class_sums_kernel(const uint8_t *__restrict__ q, int Nimg, int H, int W,
+                                                                int C, int gs, unsigned long long *__restrict__ sums)
+{
+    row_class_sums_body<IS_SIGNED>(q, Nimg, H, W, C, gs, sums);
+}
+
+// The three tensors of a weight gradient with as many input as output channels in one launch (blockIdx.z: the
+// layer input, the gradient's signed high bytes, its unsigned low bytes); sums: three tables of 16 * C, one after another.
+__global__ void __launch_bounds__(256, 3) row_class_sums3_kernel(const uint8_t *__restrict__ x, const uint8_t *__restrict__ hi,
+                                                                 const uint8_t *__restrict__ lo, int Nimg, int H, int W, int C,
+                                                                 int gs, unsigned long long *__restrict__ sums)
+{
+    if (blockIdx.z == 0)      row_class_sums_body<true>(x, Nimg, H, W, C, gs, sums);
+    else if (blockIdx.z == 1) row_class_sums_body<true>(hi, Nimg, H, W, C, gs, sums + 16 * C);
+    else                      row_class_sums_body<false>(lo, Nimg, H, W, C, gs, sums + 32 * C);
 }
 
 // Plain product, direct epilogue: rowterm[k] = -zg * SX[k] + M*zx*zg, colterm[n] = -zx * (256*SHI[n] + SLO[n]).
@@ -790,7 +808,22 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
 
     // code sums for the zero-point terms: per border class (convolution) or plain column sums
     int rc;
-    if (d) {
+    if (d && K == N && d->W <= 256 && M < (1ll << 30) && shi == sx + 16 * K && slo == shi + 16 * N) {
+        // as many input as output channels: the three tensors in one launch
+        QBP_CUDA_OK(cudaMemsetAsync(sx, 0, sizeof(int64_t) * 48 * K, st));
+        const int cv = (int)K / 16;
+        int gs = 1; while (gs * 2 <= cv && gs * 2 * d->W <= 256 && gs < 16) gs *= 2;
+        const int slabs = (cv + gs - 1) / gs;
+        const int64_t rows = M / d->W;
+        // one wave of three blocks per SM over the three tensors
+        int64_t grid_x = std::min<int64_t>(rows, std::max<int64_t>(1, (int64_t)sm_count() / slabs));
+        grid_x = std::max<int64_t>(grid_x, rows / (1 << 22) + 1);
+        QBP_TRACE_BEGIN(st);
+        row_class_sums3_kernel<<<dim3((unsigned)grid_x, (unsigned)slabs, 3), 256, (size_t)12 * gs * 16 * sizeof(int), st>>>(
+            (const uint8_t *)x, (const uint8_t *)g_hi, (const uint8_t *)g_lo, (int)(rows / d->H), d->H, d->W, (int)K, gs,
+            (unsigned long long *)sx);
+        QBP_LAUNCH_OK("class_sums_kernel");
+    } else if (d) {
         if ((rc = launch_class_sums<true>(x, M, d->H, d->W, (int)K, sx, st))) return rc;
         if ((rc = launch_class_sums<true>(g_hi, M, d->H, d->W, (int)N, shi, st))) return rc;
         if ((rc = launch_class_sums<false>(g_lo, M, d->H, d->W, (int)N, slo, st))) return rc;
