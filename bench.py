@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
 # (captured at the full batch of 256).  None: not captured.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 228.5e6 / 51380224, "quantize_kernel": 326.7e6 / 51380224}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 225.3e6 / 51380224, "quantize_kernel": 326.4e6 / 51380224}
 # Kernels bound by plain instruction issue rather than by HBM: thread instructions per element, from the same
 # captures (smsp__inst_executed.sum x 32 / elements).  Their roofline is the issue rate of the SMs:
 # SMs x 4 schedulers x 1 warp instruction per clock x 32 threads x the maximum SM clock.
@@ -413,6 +413,8 @@ def run_gemm(args):
                                    "unit": "TOP/s", "frac": round(tops / (int8_peak_sustained if capped else int8_peak), 4), "traffic": None,
                                    "peak_source": f"{kind} bf16 {'sustained (the run was power-capped)' if capped else 'burst'} x 2 (nominal int8 : bf16)",
                                    "frac_of_burst_peak": round(tops / int8_peak, 4),
+                                   # 148 SMs x 16384 int8 ops per clock at the SM clock sampled during the run
+                                   "frac_of_clock_adjusted": round(tops / (SM_COUNT * 16384 * float(clocks.get("sm_mhz") or 1965.0) / 1e6), 4),
                                    "frac_of_nominal_4500": round(tops / 4500.0, 4)}}), flush=True)
     # limb-split weight-gradient GEMM: dW [K x N] = X [M x K]^T G [M x N], X 8-bit, G 16-bit as two byte limbs
     del qa, qb, out
