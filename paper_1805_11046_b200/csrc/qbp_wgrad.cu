@@ -37,6 +37,8 @@
 namespace qbp {
 
 constexpr int kWgThreads = 192;
+constexpr int kWgRows = 128;         // reduction rows per pipeline stage: four k steps of 32 (what the MMA warp does
+                                     // between stages is a fixed cost, so a stage should hold many MMAs)
 constexpr int kWgMaxStages = 16;
 constexpr int kWgMaxTiles = 4;       // A tiles (128 accumulator rows each) per CTA: 4 x 2 limbs x 64 columns fill tensor memory
 constexpr int kWgMaxLoads = 32;      // TMA loads per stage: one lane each
@@ -108,7 +110,7 @@ struct WgMmaArgs {
 
 __host__ __device__ constexpr uint32_t wg_swizzle_bits(uint32_t row_bytes) { return row_bytes == 128 ? 2u : row_bytes == 64 ? 4u : 6u; }
 
-// The 4 * NT MMAs of a stage of 64 reduction rows: the limb outermost (switching between the s8 x s8 and s8 x u8
+// The 2 * KK * NT MMAs of a stage of kWgRows reduction rows: the limb outermost (switching between the s8 x s8 and s8 x u8
 // instruction descriptors stalls the MMA pipe), then the k step, then the A tile, so that consecutive MMAs write
 // different accumulators.  FIRST: the stage starts the reduction (its first k step overwrites the accumulators).
 template <int RBA, int RBB, int NT, bool FIRST>
@@ -117,12 +119,13 @@ __device__ __forceinline__ void wg_issue_stage(uint32_t tmem, uint32_t a_lo, uin
     constexpr uint32_t a_hi = ((8u * RBA) >> 4) | (1u << 14) | (wg_swizzle_bits(RBA) << 29);
     constexpr uint32_t b_hi = ((8u * RBB) >> 4) | (1u << 14) | (wg_swizzle_bits(RBB) << 29);
     constexpr uint32_t a_kstep = 2u * RBA, b_kstep = 2u * RBB;     // 32 reduction rows, in 16-byte units
-    constexpr uint32_t a_tile16 = 64u * 128u / 16u;                // an A tile: 64 rows x 128 bytes
-    constexpr uint32_t b_tile16 = 64u * RBB / 16u;                 // a limb's tile: 64 rows x RBB bytes
+    constexpr int KK = kWgRows / 32;                               // k steps per stage
+    constexpr uint32_t a_tile16 = (uint32_t)kWgRows * 128u / 16u;  // an A tile: kWgRows rows x 128 bytes
+    constexpr uint32_t b_tile16 = (uint32_t)kWgRows * RBB / 16u;   // a limb's tile: kWgRows rows x RBB bytes
     const uint32_t idesc_lo = idesc_hi ^ (1u << 10);               // the low limb is unsigned
 #pragma unroll
-    for (int i = 0; i < 4 * NT; ++i) {
-        const int limb = i / (2 * NT), kk = (i / NT) % 2, j = i % NT;
+    for (int i = 0; i < 2 * KK * NT; ++i) {
+        const int limb = i / (KK * NT), kk = (i / NT) % KK, j = i % NT;
         const uint32_t ao = (uint32_t)j * a_tile16 + (uint32_t)kk * a_kstep;
         const uint32_t bo = (uint32_t)limb * b_tile16 + (uint32_t)kk * b_kstep;
         if (elect_one())
@@ -645,8 +648,8 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
     P.ma = (P.a_tiles + P.a_groups - 1) / P.a_groups;
     int cols = 32; while (cols < P.ma * 2 * P.bn) cols <<= 1;
     P.tmem_cols = cols;
-    // reduction rows per stage: 64 keeps the ring deep and the release groups fine-grained
-    const uint32_t kr = 64;
+    // reduction rows per stage: kWgRows (the ring is shallower than with 64, but a stage holds twice the MMAs)
+    const uint32_t kr = kWgRows;
     P.kr = (int)kr;
     P.a_chunk_bytes = kr * rb_a;
     P.a = layout_mnmajor(kr, rb_a, (uint32_t)P.a_chunks, P.a_chunk_bytes);
