@@ -101,6 +101,29 @@ void qbo_range(const float *x, int64_t rows, int64_t cols, int per_channel,
         }
 }
 
+/* Clamping values of an activation tensor as Appendix B defines them for the
+ * high dynamic range of activations: the tensor is cut into `chunks` equal,
+ * contiguous groups of rows (rows must be a multiple of chunks); vmax is the
+ * average of the groups' maxima and vmin the average of their minima
+ * (accumulated in double, returned in fp32).  Values beyond them saturate at
+ * the end codes in qbo_quantize.  chunks = 1 is qbo_range per tensor. */
+void qbo_range_chunked(const float *x, int64_t rows, int64_t cols, int64_t chunks,
+                       float *vmin, float *vmax)
+{
+    const int64_t per = rows / chunks;
+    double slo = 0.0, shi = 0.0;
+    for (int64_t k = 0; k < chunks; ++k) {
+        float lo = INFINITY, hi = -INFINITY;
+        for (int64_t i = k * per * cols; i < (k + 1) * per * cols; ++i) {
+            if (x[i] < lo) lo = x[i];
+            if (x[i] > hi) hi = x[i];
+        }
+        slo += (double)lo; shi += (double)hi;
+    }
+    vmin[0] = (float)(slo / (double)chunks);
+    vmax[0] = (float)(shi / (double)chunks);
+}
+
 /* Appendix B: scale and zero-point from the clamping values, M bits.
  * Readings: the code grid has L = 2^M - 1 steps so that vmax maps to the top
  * M-bit code; the interval is widened to contain 0 so that real zero is a

@@ -136,6 +136,17 @@ def quantize(x, bits=8, per_channel=False, rounding=0, seed=0, tensor_id=0,
     return Quantized(q, scale, zp, lo, hi, bits)
 
 
+def range_chunked(x, chunks):
+    """Appendix B's clamping values for activations: (mean of the chunk minima, mean of the chunk maxima) over
+    `chunks` equal contiguous groups of rows.  Feed them to quantize(range_in=...)."""
+    x = _f32(x); cols = x.shape[-1]; rows = x.size // cols
+    if chunks < 1 or rows % chunks:
+        raise ValueError("rows must be a multiple of chunks")
+    lo = np.zeros(1, np.float32); hi = np.zeros(1, np.float32)
+    lib().qbo_range_chunked(_p(x), C.c_int64(rows), C.c_int64(cols), C.c_int64(chunks), _p(lo), _p(hi))
+    return float(lo[0]), float(hi[0])
+
+
 def dequantize(qt: Quantized) -> np.ndarray:
     """Per-tensor only."""
     out = np.zeros(qt.q.shape, np.float32)

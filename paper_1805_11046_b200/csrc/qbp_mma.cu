@@ -2,14 +2,15 @@
 //   y = W x and g_{l-1} = g_l W^T (Section 1; Eq. (grad_layer)) for linear
 //   layers (GEMM) and for convolutions (implicit GEMM over the filter taps).
 //
-// One CTA produces one 128 x BN tile of the output.  Warp 0 drives TMA
-// (cp.async.bulk.tensor into 128B/64B/32B-swizzled shared-memory stages),
-// warp 1 issues tcgen05.mma kind::i8 with the int32 accumulator in tensor
-// memory, warps 2..5 read the accumulator back (tcgen05.ld), apply the
-// zero-point correction, dequantise and store.  Stages are handed over with
-// mbarriers; tcgen05.commit releases a stage when the MMAs that read it are
-// done.  Every wait is bounded; on expiry the CTA raises the status word at
-// the start of the workspace and leaves through the normal exit.
+// This file: the persistent single-CTA kernel (convolutions, narrow GEMMs) and the entry points; the dense GEMM of
+// at least one 256 x 256 tile runs on CTA pairs (qbp_mma2.cu).  One CTA per SM walks output tiles of 128 (or 2 x 128)
+// rows x BN columns.  Warp 0 drives TMA (cp.async.bulk.tensor into 128B/64B/32B-swizzled shared-memory stages),
+// warp 1 issues tcgen05.mma kind::i8 with int32 accumulators in tensor memory (the whole warp runs the loop, an
+// elected lane issues: see issue_stage), up to twelve epilogue warps read accumulators back (tcgen05.ld), apply the
+// zero-point correction, dequantise and store through swizzled slabs and TMA.  A 3 x 3 convolution loads the
+// pixel box of a tile once with its border and takes the nine taps as shifted windows of that tile.  Stages are
+// handed over with mbarriers; tcgen05.commit releases a stage when the MMAs that read it are done.  Every wait is
+// bounded; on expiry the CTA raises the status word at the start of the workspace and leaves through the normal exit.
 //
 // The raw MMA sums stored codes; padding taps are zero-filled by TMA and so
 // contribute nothing to the raw sum.  The sum over (q_a - z_a)(q_b - z_b) is
@@ -154,7 +155,7 @@ uint32_t make_idesc(bool a_signed, bool b_signed, uint32_t a_major, uint32_t b_m
 // ================================================================== the kernel
 enum { MODE_GEMM = 0, MODE_FPROP = 1, MODE_DGRAD = 2 };
 constexpr int kMaxStages = 16;
-constexpr int kMaxStageMmas = 256;                    // 32 operand tiles x 2 sub-tiles x 4 k steps
+constexpr int kMaxStageMmas = 256;                    // bound on the MMAs of one pipeline stage (several halo tiles per stage)
 constexpr int kMaxAccBufs = 8;                        // accumulator buffers in tensor memory (512 columns in all)
 constexpr int kEpiWarps = 12;                         // three per tensor-memory lane quadrant
 constexpr int kMmaThreads = 64 + 32 * kEpiWarps;      // TMA warp, MMA warp, epilogue warps

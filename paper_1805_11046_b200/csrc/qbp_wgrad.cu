@@ -26,10 +26,10 @@
 // zero-filled.  Zero-points are applied afterwards from per-border-class code
 // sums (a tap near the border sees fewer positions).
 //
-// The TMA-issuing and MMA-issuing threads are bound by their own instruction
-// latency, so both run from small tables built once per CTA (one entry per
-// load / per MMA of a stage), and stages are released in groups: a
-// tcgen05.commit drains the MMA pipeline, which short MMAs cannot afford often.
+// The TMA-issuing lanes run from a small table built once per CTA (one entry per load of a stage); the MMA warp
+// runs whole with an elected issuer and the stage's MMAs fully unrolled for the operand layouts (see
+// wg_issue_stage); stages are released in groups: a tcgen05.commit drains the MMA pipeline, which short MMAs
+// cannot afford often.
 #include "qbp_mma.cuh"
 
 #include <algorithm>
@@ -42,7 +42,6 @@ constexpr int kWgRows = 128;         // reduction rows per pipeline stage: four 
 constexpr int kWgMaxStages = 16;
 constexpr int kWgMaxTiles = 4;       // A tiles (128 accumulator rows each) per CTA: 4 x 2 limbs x 64 columns fill tensor memory
 constexpr int kWgMaxLoads = 32;      // TMA loads per stage: one lane each
-constexpr int kWgMaxMmas = 128;      // MMAs per stage: 4 tiles x 4 k steps x 2 limbs, with room
 constexpr uint32_t kWgSmem = 220u * 1024u;
 
 struct WgradParams {

@@ -124,6 +124,37 @@ def test_supplied_range_and_per_channel():
         assert pc.scale[c] == one.scale[0] and pc.zero_point[c] == one.zero_point[0]
 
 
+def test_chunk_averaged_clamp_values():
+    """Appendix B (activations): clamping values = the average over K chunks of the chunks' maxima and minima."""
+    # worked by hand: chunk 0 = rows 0-1 (min -3, max 5), chunk 1 = rows 2-3 (min -7, max 9)
+    x = np.array([[1, 5], [-3, 2], [0, 9], [-7, 4]], np.float32)
+    assert O.range_chunked(x, 2) == (-5.0, 7.0)
+    assert O.range_chunked(x, 4) == ((1 - 3 + 0 - 7) / 4, (5 + 2 + 9 + 4) / 4)
+    # one chunk: the tensor's own minimum and maximum
+    r = np.random.Generator(np.random.PCG64(7)).standard_normal((96, 40)).astype(np.float32)
+    assert O.range_chunked(r, 1) == (float(r.min()), float(r.max()))
+    # averages of chunk extremes lie inside the global range, shrink (weakly) as the chunks get finer when the chunks
+    # nest, and do not depend on the order of the elements inside a chunk
+    lo1, hi1 = O.range_chunked(r, 1)
+    prev = (lo1, hi1)
+    for k in (2, 4, 8, 16, 32, 96):
+        lo, hi = O.range_chunked(r, k)
+        assert lo1 <= prev[0] <= lo <= hi <= prev[1] <= hi1
+        prev = (lo, hi)
+    shuffled = r.reshape(4, -1).copy()
+    for row in shuffled:
+        np.random.Generator(np.random.PCG64(1)).shuffle(row)
+    assert O.range_chunked(shuffled.reshape(r.shape), 4) == O.range_chunked(r, 4)
+    # values beyond the clamp saturate at the end codes; inside it the error bound of the quantiser holds
+    lo, hi = O.range_chunked(r, 8)
+    qt = O.quantize(r, 8, range_in=(lo, hi))
+    assert np.all(qt.q[r >= hi] == 127) and np.all(qt.q[r <= lo] == -128)
+    inside = (r > lo) & (r < hi)
+    assert np.max(np.abs(O.dequantize(qt)[inside] - r[inside])) <= float(qt.scale[0]) * (0.5 + 1e-4)
+    with pytest.raises(ValueError):
+        O.range_chunked(r, 7)
+
+
 @pytest.mark.parametrize("bits", [8, 16])
 def test_stochastic_rounding_brackets_and_is_unbiased(bits):
     # many copies of a few values inside a fixed range: the mean code tends to t
