@@ -445,7 +445,7 @@ def run_rangebn(args):
     hbm = float(peaks["hbm_gbs"])
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     bpe = {"bn_stats_kernel": 4, "bn_apply_kernel": 8, "bn_bwd_stats_kernel": 8, "bn_bwd_apply_kernel": 12,
-           "range_partial_kernel": 4, "chan_range_partial_kernel": 4, "quantize_kernel": 5}
+           "range_partial_kernel": 4, "chan_range_partial_kernel": 4, "chunk_range_partial_kernel": 4, "quantize_kernel": 5}
     for hw, ch in synth.RANGEBN_SWEEP:
         case = synth.rangebn_case(args.batch, hw, ch)
         x = torch.from_numpy(case["x"]).cuda(); dy = torch.from_numpy(case["dy"]).cuda()
@@ -459,11 +459,14 @@ def run_rangebn(args):
             timed(lambda: B.qbp_rangebn_bwd(dy, x, mean, vmin, vmax, relu=True, dx=dx))
         qt = timed(lambda: B.qbp_quantize_s8(x, granularity=0, rounding=1, seed=1, tensor_id=2, q=q))
         qc = timed(lambda: B.qbp_quantize_s8(x, granularity=1, rounding=1, seed=1, tensor_id=2, q=q))
+        rng = B.new_qparams(1)
+        rc = timed(lambda: B.qbp_range_chunked(x, args.batch, range_out=rng))        # one chunk per image
         row = lambda ks: [{"kernel": k, "us": round(t * 1e3, 1), "gbs": round(bpe[k] * E / t / 1e6, 0) if k in bpe else None,
                            "frac": round(bpe[k] * E / t / 1e6 / hbm, 3) if k in bpe else None} for k, t in ks]
         print(json.dumps({"workload": f"rangebn_quant_{args.batch}x{hw}x{hw}x{ch}", "tensor_mb": round(E * 4 / 1e6, 1),
                           "peak_gbs": hbm, "peak_source": f"{kind} copy bandwidth", "rangebn": row(ker),
-                          "quantize_sr_per_tensor": row(qt), "quantize_sr_per_channel": row(qc)}), flush=True)
+                          "quantize_sr_per_tensor": row(qt), "quantize_sr_per_channel": row(qc),
+                          "range_chunk_averaged": row(rc)}), flush=True)
         del x, dy, y, dx, q
 
 

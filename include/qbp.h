@@ -109,6 +109,20 @@ int qbp_quantize_s8(const float *x, int64_t rows, int64_t cols, int granularity,
                     int8_t *q, qbp_qparams *qp_out, int32_t *row_sums, int64_t *col_sums,
                     void *ws, size_t ws_bytes, void *stream);
 
+/* Clamping values for activations as Appendix B takes them ("the average of
+ * absolute maximum and minimum values of K chunks", which narrows the
+ * quantisation steps of tensors with a high dynamic range): x [rows x cols] is
+ * cut into `chunks` equal contiguous groups of rows (rows a multiple of
+ * chunks, chunks <= 4096); range_out->vmax receives the average of the groups'
+ * maxima, range_out->vmin the average of their minima (sums in double, in
+ * chunk order; scale and zero_point of the record are left 0).  Pass range_out
+ * as range_in to qbp_quantize_s8: values beyond the clamp saturate at the end
+ * codes.  Device pointers; workspace of qbp_range_chunked_workspace_bytes(). */
+size_t qbp_range_chunked_workspace_bytes(void);
+
+int qbp_range_chunked(const float *x, int64_t rows, int64_t cols, int64_t chunks,
+                      qbp_qparams *range_out, void *ws, size_t ws_bytes, void *stream);
+
 /* qbp_quantize_s8 for callers that cannot provide a workspace (the paper has
  * no counterpart; this is a packaging variant of the same kernels).  Some
  * hosts of this library may not allocate device memory at the point where

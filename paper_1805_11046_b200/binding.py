@@ -24,6 +24,7 @@ QBP_ERR_TIMEOUT = -6
 EXPORTS = (
     "qbp_last_error", "qbp_trace_enable", "qbp_trace_count", "qbp_trace_read",
     "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s8_static", "qbp_quantize_s16", "qbp_bifurcate",
+    "qbp_range_chunked_workspace_bytes", "qbp_range_chunked",
     "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8",
     "qbp_conv_s8_workspace_bytes", "qbp_conv_s8_implicit",
     "qbp_wgrad_s16_workspace_bytes", "qbp_wgrad_s16",
@@ -73,6 +74,7 @@ def _load() -> C.CDLL:
     lib.qbp_wgrad_s16_workspace_bytes.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64]
     lib.qbp_rangebn_workspace_bytes.argtypes = [C.c_int64, C.c_int64]
     lib.qbp_layer_workspace_bytes.argtypes = [C.c_void_p]
+    lib.qbp_range_chunked_workspace_bytes.argtypes = []
     return lib
 
 
@@ -148,6 +150,17 @@ def qbp_quantize_s8(x, granularity=QBP_PER_TENSOR, rounding=QBP_ROUND_NEAREST, s
                                C.c_uint64(seed), C.c_uint32(tensor_id), _ptr(range_in), _ptr(q), _ptr(qp_out),
                                _ptr(row_sums), _ptr(col_sums), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
     return q, qp_out
+
+
+def qbp_range_chunked(x, chunks, range_out=None, ws=None):
+    """Appendix B's clamping values for activations (averages of the chunks' minima / maxima over `chunks` equal
+    groups of rows) as a qparams record to pass to qbp_quantize_s8(range_in=...)."""
+    cols = x.shape[-1]; rows = x.numel() // cols if cols else 0
+    if range_out is None: range_out = new_qparams(1, x.device)
+    if ws is None: ws = workspace(lib.qbp_range_chunked_workspace_bytes(), x.device)
+    _check(lib.qbp_range_chunked(_ptr(x), C.c_int64(rows), C.c_int64(cols), C.c_int64(chunks), _ptr(range_out), _ptr(ws),
+                                 C.c_size_t(ws.numel()), _stream()))
+    return range_out
 
 
 QBP_STATIC_MAX_CHANNELS = 256

@@ -133,6 +133,70 @@ __global__ void __launch_bounds__(kThreads) range_finalize_kernel(const float2 *
     }
 }
 
+// ---------------------------------------------- chunk-averaged clamping values
+// Appendix B, activations: the clamping values are the averages, over K chunks of the tensor, of the chunks'
+// minima and maxima.  blockIdx.y = chunk (equal contiguous runs of n_chunk elements), blockIdx.x = block inside it.
+template <int VEC>
+__global__ void __launch_bounds__(kThreads) chunk_range_partial_kernel(const float *__restrict__ x, int64_t n_chunk,
+                                                                       float2 *__restrict__ partials)
+{
+    x += (int64_t)blockIdx.y * n_chunk;
+    float lo = INFINITY, hi = -INFINITY;
+    const int64_t nv = n_chunk / VEC;              // (VEC = 4 only when n_chunk is a multiple of 4)
+    const int64_t stride = (int64_t)gridDim.x * kThreads * kRangeUnroll;
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * kRangeUnroll; base < nv; base += stride) {
+        VecF<VEC> v[kRangeUnroll];
+        bool ok[kRangeUnroll];
+#pragma unroll
+        for (int u = 0; u < kRangeUnroll; ++u) {
+            int64_t i = base + u * kThreads + threadIdx.x;
+            ok[u] = i < nv;
+            if (ok[u]) v[u].load_stream(x + i * VEC);
+        }
+#pragma unroll
+        for (int u = 0; u < kRangeUnroll; ++u)
+            if (ok[u]) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) { lo = fminf(lo, v[u].v[e]); hi = fmaxf(hi, v[u].v[e]); }
+            }
+    }
+    lo = warp_min(lo); hi = warp_max(hi);
+    __shared__ float s_lo[kThreads / 32], s_hi[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        lo = threadIdx.x < kThreads / 32 ? s_lo[threadIdx.x] : INFINITY;
+        hi = threadIdx.x < kThreads / 32 ? s_hi[threadIdx.x] : -INFINITY;
+        lo = warp_min(lo); hi = warp_max(hi);
+        if (threadIdx.x == 0) partials[(int64_t)blockIdx.y * gridDim.x + blockIdx.x] = make_float2(lo, hi);
+    }
+}
+
+// One block: every chunk's (min, max) from its blocks' partials, then the two averages, added up in chunk order in
+// double by one thread (the order is part of the result: it is the reference's).
+__global__ void __launch_bounds__(kThreads) chunk_range_finalize_kernel(const float2 *__restrict__ partials, int chunks,
+                                                                        int blocks_per_chunk, float2 *__restrict__ per_chunk,
+                                                                        qbp_qparams *__restrict__ out)
+{
+    for (int k = threadIdx.x; k < chunks; k += kThreads) {
+        float lo = INFINITY, hi = -INFINITY;
+        for (int b = 0; b < blocks_per_chunk; ++b) {
+            const float2 p = partials[(int64_t)k * blocks_per_chunk + b];
+            lo = fminf(lo, p.x); hi = fmaxf(hi, p.y);
+        }
+        per_chunk[k] = make_float2(lo, hi);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double slo = 0.0, shi = 0.0;
+        for (int k = 0; k < chunks; ++k) { slo += (double)per_chunk[k].x; shi += (double)per_chunk[k].y; }
+        qbp_qparams r;
+        r.scale = 0.0f; r.zero_point = 0;
+        r.vmin = (float)(slo / (double)chunks); r.vmax = (float)(shi / (double)chunks);
+        *out = r;
+    }
+}
+
 // Parameters from clamping values the caller already has (one thread each).
 __global__ void qparams_from_range_kernel(const qbp_qparams *__restrict__ in, int count, int bits,
                                           qbp_qparams *__restrict__ out)
@@ -709,6 +773,45 @@ extern "C" __attribute__((visibility("default"))) int qbp_trace_read(int index, 
     if (!r.name) return fail(QBP_ERR_INVALID_ARG, "trace_read: record %d was never closed", index);
     snprintf(name, (size_t)name_cap, "%s", r.name);
     QBP_CUDA_OK(cudaEventElapsedTime(ms, r.a, r.b));
+    return QBP_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) size_t qbp_range_chunked_workspace_bytes(void)
+{
+    return 2 * align_up(sizeof(float2) * kMaxParts, 256) + 256;
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_range_chunked(const float *x, int64_t rows, int64_t cols, int64_t chunks,
+                                                                       qbp_qparams *range_out, void *ws, size_t ws_bytes,
+                                                                       void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!x || !range_out) return fail(QBP_ERR_INVALID_ARG, "range_chunked: NULL argument");
+    if (rows <= 0 || cols <= 0) return fail(QBP_ERR_INVALID_ARG, "range_chunked: empty tensor");
+    if (chunks < 1 || chunks > kMaxParts || rows % chunks)
+        return fail(QBP_ERR_INVALID_ARG, "range_chunked: rows (%lld) must be a multiple of chunks (%lld), at most %d chunks",
+                    (long long)rows, (long long)chunks, kMaxParts);
+    if (!ws || ws_bytes < qbp_range_chunked_workspace_bytes())
+        return fail(QBP_ERR_WORKSPACE, "range_chunked: workspace of %zu bytes needed, %zu given",
+                    qbp_range_chunked_workspace_bytes(), ws_bytes);
+    WsCarver w(ws, ws_bytes);
+    float2 *parts = w.take<float2>(kMaxParts);
+    float2 *per_chunk = w.take<float2>(kMaxParts);
+    const int64_t n_chunk = rows / chunks * cols;
+    const bool vec = aligned16(x) && n_chunk % 4 == 0;
+    // about one wave of blocks in all, at least one per chunk
+    const int64_t per_block = (int64_t)kThreads * kRangeUnroll * (vec ? 4 : 1);
+    const int wave = grid_for(vec ? blocks_per_sm(chunk_range_partial_kernel<4>, kThreads) : blocks_per_sm(chunk_range_partial_kernel<1>, kThreads),
+                              (rows * cols + per_block - 1) / per_block);
+    int bpc = (int)std::max<int64_t>(1, std::min<int64_t>((n_chunk + per_block - 1) / per_block, wave / chunks));
+    bpc = (int)std::min<int64_t>(bpc, kMaxParts / chunks);
+    QBP_TRACE_BEGIN(st);
+    if (vec) chunk_range_partial_kernel<4><<<dim3(bpc, (unsigned)chunks), kThreads, 0, st>>>(x, n_chunk, parts);
+    else     chunk_range_partial_kernel<1><<<dim3(bpc, (unsigned)chunks), kThreads, 0, st>>>(x, n_chunk, parts);
+    QBP_LAUNCH_OK("chunk_range_partial_kernel");
+    QBP_TRACE_BEGIN(st);
+    chunk_range_finalize_kernel<<<1, kThreads, 0, st>>>(parts, (int)chunks, bpc, per_chunk, range_out);
+    QBP_LAUNCH_OK("chunk_range_finalize_kernel");
     return QBP_OK;
 }
 

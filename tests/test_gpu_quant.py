@@ -88,6 +88,27 @@ def test_supplied_range_and_empty_tensor(B):
     assert q.numel() == 0 and s[0] == 1.0 and z[0] == -128 and lo[0] == 0 and hi[0] == 0
 
 
+@pytest.mark.parametrize("shape,chunks", [((64, 256), 1), ((64, 256), 8), ((96, 40), 96), ((256, 33), 16), ((12, 5, 7, 24), 4),
+                                          ((4096, 3), 4096), ((1000, 64), 125)])
+def test_chunk_averaged_clamp(B, shape, chunks):
+    """Appendix B's clamping values for activations (averages over K chunks of the chunks' extremes): the two values
+    bit for bit, then the codes of the quantiser that clamps to them."""
+    x = synth.channel_gaussian(shape, 31, 32) if len(shape) == 4 else synth.normal(shape, 33)
+    rng = B.qbp_range_chunked(to_dev(x), chunks)
+    lo, hi = O.range_chunked(x, chunks)
+    _, _, glo, ghi = B.read_qparams(rng)
+    assert glo[0] == np.float32(lo) and ghi[0] == np.float32(hi)
+    q, qp = B.qbp_quantize_s8(to_dev(x), range_in=rng)
+    o = O.quantize(x, 8, range_in=(np.float32(lo), np.float32(hi)))
+    _same_params(B, qp, o)
+    assert np.array_equal(to_host(q), o.q)
+
+
+def test_chunk_averaged_clamp_refuses_rows_that_do_not_divide(B):
+    with pytest.raises(B.QbpError):
+        B.qbp_range_chunked(to_dev(synth.normal((10, 8), 1)), 3)
+
+
 def test_bifurcate_and_code_sums(B):
     import torch
     g = synth.normal((130, 64), 12, std=0.1)
