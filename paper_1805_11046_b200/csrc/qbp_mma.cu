@@ -758,23 +758,34 @@ __global__ void conv_colterm_kernel(const int32_t *wsum32, const long long *wsum
 
 // rowterm[pixel] = -z_w * (sum of the input's channel sums over the taps inside the image)
 //                   + (taps inside) * Cred * z_in * z_w          (pad is 0 or 1)
-__global__ void __launch_bounds__(256) conv_rowterm_kernel(const int32_t *__restrict__ chan_sum, int64_t pixels, int H,
-                                                           int W, int pad, int Cred, const qbp_qparams *q_in,
+// blockIdx.y = image, blockIdx.x * 256 + threadIdx.x = position inside it; the nine taps unrolled under predicates
+// and the one division by a multiply-high (with plain divisions and loops this kernel ran 260 instructions per pixel).
+__global__ void __launch_bounds__(256) conv_rowterm_kernel(const int32_t *__restrict__ chan_sum, int HW, int H, int W,
+                                                           FastDiv dW, int pad, int Cred, const qbp_qparams *q_in,
                                                            const qbp_qparams *q_w, int32_t *__restrict__ rowterm)
 {
-    const int64_t m = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (m >= pixels) return;
+    const int i = (int)blockIdx.x * 256 + (int)threadIdx.x;
+    if (i >= HW) return;
+    int p, q;
+    dW.divmod(i, p, q);
+    const int m = (int)blockIdx.y * HW + i;                  // (fewer than 2^31 positions)
+    const bool up = pad && p > 0, down = pad && p + 1 < H, left = pad && q > 0, right = pad && q + 1 < W;
+    const int32_t *c = chan_sum + m;
+    int box = __ldg(c);
+    if (left) box += __ldg(c - 1);
+    if (right) box += __ldg(c + 1);
+    if (up) {
+        box += __ldg(c - W);
+        if (left) box += __ldg(c - W - 1);
+        if (right) box += __ldg(c - W + 1);
+    }
+    if (down) {
+        box += __ldg(c + W);
+        if (left) box += __ldg(c + W - 1);
+        if (right) box += __ldg(c + W + 1);
+    }
+    const int taps = (1 + (up ? 1 : 0) + (down ? 1 : 0)) * (1 + (left ? 1 : 0) + (right ? 1 : 0));
     const int za = q_in->zero_point, zb = q_w->zero_point;
-    // (pixels < 2^31: 32-bit divisions)
-    const unsigned mu = (unsigned)m;
-    const int q = (int)(mu % (unsigned)W), p = (int)((mu / (unsigned)W) % (unsigned)H);
-    int box = 0, taps = 0;
-    for (int eh = -pad; eh <= pad; ++eh)
-        for (int ew = -pad; ew <= pad; ++ew)
-            if (p + eh >= 0 && p + eh < H && q + ew >= 0 && q + ew < W) {
-                box += chan_sum[m + (int64_t)eh * W + ew];
-                ++taps;
-            }
     rowterm[m] = -zb * box + taps * Cred * za * zb;
 }
 
@@ -1150,7 +1161,8 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
         dgrad ? 1 : 0, q_in, colterm);
     QBP_LAUNCH_OK("conv_colterm_kernel");
     QBP_TRACE_BEGIN(st);
-    conv_rowterm_kernel<<<(unsigned)((pix + 255) / 256), 256, 0, st>>>(chan_sum, pix, d->H, d->W, d->pad, Cred, q_in, q_w, rowterm);
+    conv_rowterm_kernel<<<dim3((unsigned)((d->H * d->W + 255) / 256), (unsigned)d->N), 256, 0, st>>>(
+        chan_sum, d->H * d->W, d->H, d->W, make_fastdiv(d->W), d->pad, Cred, q_in, q_w, rowterm);
     QBP_LAUNCH_OK("conv_rowterm_kernel");
 
     MmaParams P{};
