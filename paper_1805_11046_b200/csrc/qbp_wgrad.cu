@@ -37,6 +37,10 @@
 namespace qbp {
 
 constexpr int kWgThreads = 192;
+#ifndef QBP_WG_FIN_LANES
+#define QBP_WG_FIN_LANES 4
+#endif
+constexpr int kWgFinalizeLanes = QBP_WG_FIN_LANES;   // lanes of the second kernel that share one output element's partials
 constexpr int kWgRows = 128;         // reduction rows per pipeline stage: four k steps of 32 (what the MMA warp does
                                      // between stages is a fixed cost, so a stage should hold many MMAs)
 constexpr int kWgMaxStages = 16;
@@ -535,8 +539,13 @@ __global__ void __launch_bounds__(256) wgrad_finalize_kernel(const WgradParams P
                                                              const long long *__restrict__ shi,
                                                              const long long *__restrict__ slo, int64_t total)
 {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= total) return;
+    // kWgFinalizeLanes lanes per output element share its slices (an element's partials are few hundred bytes each, far apart:
+    // one thread walking them alone is bound by latency)
+    constexpr int kLanes = kWgFinalizeLanes;
+    const int64_t e_raw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / kLanes;
+    const int part_lane = threadIdx.x % kLanes;
+    const bool live = e_raw < total;
+    const int64_t e = live ? e_raw : total - 1;           // (idle lanes of the last warp compute a duplicate and do not store)
     const long long zx = P.qx->zero_point, zg = P.qg->zero_point;
     long long SX = 0, SG = 0, count = 0;
     int at, row, n;                                     // accumulator tile, row in it, output column of g
@@ -575,15 +584,18 @@ __global__ void __launch_bounds__(256) wgrad_finalize_kernel(const WgradParams P
     const int64_t off = P.conv ? ((int64_t)j * P.bn + col) * 128 + row : ((int64_t)j * 128 + row) * P.bn + col;
     long long raw = 0;
     const long long *src = P.part + (int64_t)first * P.part_stride + off;
-    int sl = 0;
-    for (; sl + 8 <= slices; sl += 8) {
+    int sl = part_lane;
+    for (; sl + 7 * kLanes < slices; sl += 8 * kLanes) {
         long long v[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (int64_t)(sl + u) * P.part_stride);
+        for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (int64_t)(sl + u * kLanes) * P.part_stride);
 #pragma unroll
         for (int u = 0; u < 8; ++u) raw += v[u];
     }
-    for (; sl < slices; ++sl) raw += __ldcs(src + (int64_t)sl * P.part_stride);
+    for (; sl < slices; sl += kLanes) raw += __ldcs(src + (int64_t)sl * P.part_stride);
+#pragma unroll
+    for (int o = 1; o < kLanes; o <<= 1) raw += __shfl_xor_sync(0xffffffffu, raw, o);
+    if (!live || part_lane != 0) return;
     const long long acc = raw - zg * SX - zx * SG + count * zx * zg;
     if (P.acc_out) P.acc_out[e] = acc;
     if (P.dW) P.dW[e] = __fmul_rn((float)acc, __fmul_rn(P.qx->scale, P.qg->scale));
@@ -880,7 +892,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
     kernel<<<pl.grid, kWgThreads, pl.smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_wgrad_kernel");
     if (!P.direct) {
-        const int blocks = (int)((outs + 255) / 256);
+        const int blocks = (int)((outs * kWgFinalizeLanes + 255) / 256);
         QBP_TRACE_BEGIN(st);
         wgrad_finalize_kernel<<<blocks, 256, 0, st>>>(P, (const long long *)sx, (const long long *)shi, (const long long *)slo, outs);
         QBP_LAUNCH_OK("wgrad_finalize_kernel");
