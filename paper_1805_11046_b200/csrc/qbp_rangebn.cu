@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
         for (int u = 0; u < kScanUnroll; ++u) {
             int64_t r = r0 + u * step;
             ok[u] = r < rows;
-            if (ok[u]) v[u].load(x + r * C + p.col);
+            if (ok[u]) v[u].load_stream(x + r * C + p.col);
         }
 #pragma unroll
         for (int u = 0; u < kScanUnroll; ++u)
@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
                     float yv = bn_y(bn_xhat(v[u].v[e], mu[e], s[e]), g[e], b[e]);
                     v[u].v[e] = RELU ? fmaxf(yv, 0.0f) : yv;
                 }
-                v[u].store(y + (r0 + u * step) * C + p.col);
+                v[u].store_stream(y + (r0 + u * step) * C + p.col);
             }
     }
 }
@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float 
                     vd[u].v[e] = s[e] * (g[e] * d - m1[e] - k2[e] * ind);
                     if (RANGE) { rlo = fminf(rlo, vd[u].v[e]); rhi = fmaxf(rhi, vd[u].v[e]); }
                 }
-                vd[u].store(dx + (r0 + u * step) * C + p.col);
+                vd[u].store_stream(dx + (r0 + u * step) * C + p.col);
             }
     }
     }
