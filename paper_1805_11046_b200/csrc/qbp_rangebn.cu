@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float 
                     vd[u].v[e] = s[e] * (g[e] * d - m1[e] - k2[e] * ind);
                     if (RANGE) { rlo = fminf(rlo, vd[u].v[e]); rhi = fmaxf(rhi, vd[u].v[e]); }
                 }
-                vd[u].store_stream(dx + (r0 + u * step) * C + p.col);
+                vd[u].store(dx + (r0 + u * step) * C + p.col);
             }
     }
     }
