@@ -377,7 +377,9 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
         for (int u = 0; u < kUnroll; ++u) {
             int64_t j = base + u * kThreads + threadIdx.x;
             ok[u] = j < nv;
-            if (ok[u]) v[u] = __ldg(reinterpret_cast<const float4 *>(x) + j);
+            // nearest rounding follows a range scan of the same (large) tensor and is bound by HBM: evict-first loads;
+            // the stochastic instance is bound by arithmetic and often finds the tail of its input in the L2
+            if (ok[u]) v[u] = SR ? __ldg(reinterpret_cast<const float4 *>(x) + j) : __ldcs(reinterpret_cast<const float4 *>(x) + j);
         }
         int rs[kUnroll];
 #pragma unroll
