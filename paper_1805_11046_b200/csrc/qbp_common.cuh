@@ -111,6 +111,20 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, float zp_
     return (int)code;
 }
 
+// The stochastic 8-bit code of one element in fixed point: the same result as quantize_code<true>(.., 255, rnd) with
+// three instructions fewer.  With t = fma(x, inv, zp) >= 0, f = floor(t), frac = t - f and r24 = rnd >> 8, the code
+// is f + [r24 * 2^-24 < frac] = f + [r24 < ceil(frac * 2^24)] (r24 is an integer); t * 2^24 is exact in fp32 and
+// ceil(t * 2^24) = f * 2^24 + ceil(frac * 2^24), so adding 2^24 - 1 - r24 (= ~rnd >> 8) carries into bit 24 exactly
+// when the code rounds up.  The conversion saturates negative t to 0 (code 0, as the clamp gives) and the minimum
+// with 255 * 2^24 is the clamp at the top (then nothing can carry).  Returns the code in the TOP byte of the word.
+__device__ __forceinline__ uint32_t quantize_sr8_top_byte(float x, float inv_scale, float zp_u, uint32_t rnd)
+{
+    const float t = __fmaf_rn(x, inv_scale, zp_u);
+    uint32_t tc;
+    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmul_rn(t, 16777216.0f)));
+    return min(tc, 0xFF000000u) + ((~rnd) >> 8);
+}
+
 // Philox4x32-10 with the ten round keys precomputed (they depend on the key only).
 struct PhiloxKeys { uint32_t k0[10], k1[10]; };
 __device__ __forceinline__ PhiloxKeys philox_keys(uint2 k)

@@ -330,6 +330,11 @@ __device__ __forceinline__ uint32_t pack_bytes0(const uint32_t (&c)[4])
 {
     return __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
 }
+// The top bytes of c[0..3] into one word.
+__device__ __forceinline__ uint32_t pack_bytes3(const uint32_t (&c)[4])
+{
+    return __byte_perm(__byte_perm(c[0], c[1], 0x0073), __byte_perm(c[2], c[3], 0x0073), 0x5410);
+}
 // The second bytes of c[0..3] into one word.
 __device__ __forceinline__ uint32_t pack_bytes1(const uint32_t (&c)[4])
 {
@@ -403,9 +408,10 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                         if (table) { const float2 t = s_qp[c0 + e]; p8.inv = t.x; p8.zp_u = t.y; }
                         else p8 = load_qp(qp8 + c0 + e, 8);
                     }
-                    c[e] = (uint32_t)quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
+                    c[e] = SR ? quantize_sr8_top_byte(xs[e], p8.inv, p8.zp_u, r[e])
+                              : (uint32_t)quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
                 }
-                const uint32_t packed = pack_bytes0(c) ^ 0x80808080u;       // stored = unsigned code - 128
+                const uint32_t packed = (SR ? pack_bytes3(c) : pack_bytes0(c)) ^ 0x80808080u;       // stored = unsigned code - 128
                 reinterpret_cast<uint32_t *>(o.q8)[j] = packed;
                 if (o.rowsum8) rs[u] = __dp4a((int)packed, 0x01010101, 0);
             }
