@@ -35,11 +35,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
 # (captured at the full batch of 256).  None: not captured.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 230.7e6 / 51380224, "quantize_kernel": None}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 230.7e6 / 51380224, "quantize_kernel": 327.4e6 / 51380224}
 # Kernels bound by plain instruction issue rather than by HBM: thread instructions per element, from the same
 # captures (smsp__inst_executed.sum x 32 / elements).  Their roofline is the issue rate of the SMs:
 # SMs x 4 schedulers x 1 warp instruction per clock x 32 threads x the maximum SM clock.
-ALU_INSTR_PER_ELEMENT = {}      # (the stochastic quantiser changed after its last capture: recount before claiming)
+ALU_INSTR_PER_ELEMENT = {("quantize_kernel", 2): 8.678e7 * 32 / 51380224}
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 
 
