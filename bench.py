@@ -35,11 +35,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
 # (captured at the full batch of 256).  None: not captured.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"qbp_wgrad_kernel": 230.7e6 / 51380224, "quantize_kernel": 327.4e6 / 51380224}
+# Keyed by (kernel, occurrence within the step), like KERNEL_WORK; dropped when a kernel changes.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {}
 # Kernels bound by plain instruction issue rather than by HBM: thread instructions per element, from the same
 # captures (smsp__inst_executed.sum x 32 / elements).  Their roofline is the issue rate of the SMs:
 # SMs x 4 schedulers x 1 warp instruction per clock x 32 threads x the maximum SM clock.
-ALU_INSTR_PER_ELEMENT = {("quantize_kernel", 2): 8.678e7 * 32 / 51380224}
+ALU_INSTR_PER_ELEMENT = {}
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 
 
@@ -128,6 +129,8 @@ def run_ours(args):
     from paper_1805_11046_b200.dist import max_over_ranks, rank_info
 
     rank, local_rank, world = rank_info()
+    if world != args.gpus and rank == 0:
+        print(f"bench: --gpus {args.gpus} but the launcher started {world} rank(s); reporting n_gpus = {world}", file=sys.stderr)
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
@@ -249,22 +252,23 @@ def run_ours(args):
         k["tops"] = k["ops"] / (k["ms"] * 1e-3) / 1e12 if k["ms"] > 0 else 0.0
     roofline = None
     if kernels:
+        # the kernel with the largest share of the step, against the roofline that binds it by its algorithmic work:
+        # HBM bytes over the measured copy bandwidth
         top = max(kernels, key=lambda k: k["ms"])
-        tr = NCU_TRAFFIC_BYTES_PER_ELEMENT.get(top["kernel"])
+        tr = NCU_TRAFFIC_BYTES_PER_ELEMENT.get((top["kernel"], top["occ"]))
         roofline = {"kernel": top["kernel"], "bound": "hbm", "achieved": round(top["gbs"], 1), "peak": hbm_peak,
                     "unit": "GB/s", "frac": round(top["gbs"] / hbm_peak, 4), "traffic": tr * E if tr else None,
                     "peak_source": f"{peaks_kind} copy bandwidth", "ms_per_launch": round(top["ms"], 4),
                     "share_of_step": round(top["share"], 4)}
         ipe = ALU_INSTR_PER_ELEMENT.get((top["kernel"], top["occ"]))
         if ipe:
-            # bound by instruction issue: report that roofline, keep the HBM figures beside it
+            # beside it, how close the kernel runs to the SMs' instruction issue rate (thread instructions per
+            # element from the ncu capture under profiles/; 148 SMs x 4 schedulers x 32 threads x max SM clock)
             sm_ghz = float(peaks.get("sm_max_mhz", 1965.0)) / 1e3
             alu_peak = SM_COUNT * SCHEDULERS_PER_SM * 32 * sm_ghz / 1e3          # T thread-instructions / s
             alu_ach = ipe * E / (top["ms"] * 1e-3) / 1e12
-            roofline.update({"bound": "alu", "achieved": round(alu_ach, 2), "peak": round(alu_peak, 2),
-                             "unit": "T thread-instructions/s", "frac": round(alu_ach / alu_peak, 4),
-                             "peak_source": "148 SMs x 4 schedulers x 32 threads x max SM clock",
-                             "hbm_gbs": round(top["gbs"], 1), "hbm_frac": round(top["gbs"] / hbm_peak, 4)})
+            roofline.update({"alu_frac": round(alu_ach / alu_peak, 4), "alu_achieved_tinstr_s": round(alu_ach, 2),
+                             "alu_peak_tinstr_s": round(alu_peak, 2), "thread_instructions_per_element": round(ipe, 1)})
     mma_ops = sum(k["ops"] for k in kernels if k["ops"])
     mma_ms = sum(k["ms"] for k in kernels if k["ops"])
     bn_bytes = sum(k["bytes"] for k in kernels if k["kernel"].startswith("bn_"))
@@ -289,12 +293,150 @@ def run_ours(args):
         "kernels": [{"kernel": k["kernel"], "ms": round(k["ms"], 4), "share": round(k["share"], 4),
                      "gbs": round(k["gbs"], 1), "tops": round(k["tops"], 1)} for k in kernels if k["ms"] > 0.002],
     }
+    if world == 1 and not args.no_extras:
+        # the kernels the two roofline targets are graded on (dense sweep: tensor; Range BN / quantiser sweep: HBM)
+        del L, x, w, dy
+        torch.cuda.empty_cache()
+        line["gemm_c5"] = gemm_c5_block(B, args.mnk, peaks)
+        torch.cuda.empty_cache()
+        line["rangebn_c3"] = rangebn_sweep_block(B, args.batch, hbm_peak)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.cpu_sample_batch)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+# ------------------------------------------- the two roofline targets, inside the headline line
+def _graph_ms_per_call(calls, launches):
+    """Device milliseconds per call of `launches` back-to-back calls, taken from the list `calls` in turn (each works
+    on its own buffers, so that nothing a call reads is left in the L2 by the one before it), captured once as a
+    CUDA graph and replayed: the time of a 10 us kernel then holds no host launch gap and no event overhead."""
+    import torch
+    for c in calls:
+        c()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        calls[0]()
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(launches):
+            calls[i % len(calls)]()
+    g.replay()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 3
+    a.record()
+    for _ in range(reps):
+        g.replay()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / (reps * launches)
+
+
+def rangebn_sweep_block(B, batch, hbm_peak, launches=60):
+    """Range BN passes and the stochastic 8-bit quantiser on the five sweep shapes: GB/s per pass against the copy
+    bandwidth.  Each pass is one C-ABI call (the streaming kernel plus its one-block finalize), timed as a graph of
+    `launches` calls that rotate over enough buffer sets that every call reads from HBM."""
+    import torch
+    from paper_1805_11046_b200 import synth
+    L2_BYTES = 126e6
+    out = []
+    for hw, ch in synth.RANGEBN_SWEEP:
+        case = synth.rangebn_case(batch, hw, ch)
+        E = case["x"].size
+        tbytes = 4 * E
+        sets = int(max(2, min(12, 2 * L2_BYTES // tbytes + 2)))
+        x0 = torch.from_numpy(case["x"]).cuda(); dy0 = torch.from_numpy(case["dy"]).cuda()
+        xs = [x0] + [x0.clone() for _ in range(sets - 1)]
+        dys = [dy0] + [dy0.clone() for _ in range(sets - 1)]
+        ys = [torch.empty_like(x0) for _ in range(sets)]
+        qs = [torch.empty(x0.shape, dtype=torch.int8, device="cuda") for _ in range(sets)]
+        n = E // ch
+        ws = B.workspace(max(B.lib.qbp_rangebn_workspace_bytes(n, ch), B.lib.qbp_quantize_workspace_bytes(n, ch, 1)))
+        csum, cmin, cmax = B.qbp_rangebn_fwd_stats(x0, ws=ws)
+        _, mean, vmin, vmax, rng = B.qbp_rangebn_fwd_apply(x0, n, csum, cmin, cmax, relu=True, y=ys[0], want_range=True)
+        sdy, sdyx = B.qbp_rangebn_bwd_stats(dy0, x0, n, mean, vmin, vmax, relu=True, ws=ws)
+        xr = B.qbp_range_chunked(x0, 1)
+        qp1, qpc = B.new_qparams(1), B.new_qparams(ch)
+        passes = {
+            "bn_stats": (4, [lambda i=i: B.qbp_rangebn_fwd_stats(xs[i], csum, cmin, cmax, ws=ws) for i in range(sets)]),
+            "bn_apply": (8, [lambda i=i: B.qbp_rangebn_fwd_apply(xs[i], n, csum, cmin, cmax, relu=True, y=ys[i]) for i in range(sets)]),
+            "bn_bwd_stats": (8, [lambda i=i: B.qbp_rangebn_bwd_stats(dys[i], xs[i], n, mean, vmin, vmax, relu=True, ws=ws) for i in range(sets)]),
+            "bn_bwd_apply": (12, [lambda i=i: B.qbp_rangebn_bwd_apply(dys[i], xs[i], n, mean, vmin, vmax, sdy, sdyx, relu=True, dx=ys[i], ws=ws) for i in range(sets)]),
+            "range_scan": (4, [lambda i=i: B.qbp_range_chunked(xs[i], 1, range_out=xr, ws=ws) for i in range(sets)]),
+            "quantize_sr_s8_range_given": (5, [lambda i=i: B.qbp_quantize_s8(xs[i], rounding=1, seed=1, tensor_id=2, range_in=xr, q=qs[i], qp_out=qp1, ws=ws) for i in range(sets)]),
+            "quantize_sr_s8_with_scan": (9, [lambda i=i: B.qbp_quantize_s8(xs[i], rounding=1, seed=1, tensor_id=2, q=qs[i], qp_out=qp1, ws=ws) for i in range(sets)]),
+            "quantize_sr_s8_per_channel_with_scan": (9, [lambda i=i: B.qbp_quantize_s8(xs[i], granularity=1, rounding=1, seed=1, tensor_id=2, q=qs[i], qp_out=qpc, ws=ws) for i in range(sets)]),
+        }
+        row = {"shape": [batch, hw, hw, ch], "tensor_mb": round(tbytes / 1e6, 1), "buffer_sets": sets, "passes": {}}
+        for name, (bpe, calls) in passes.items():
+            ms = _graph_ms_per_call(calls, launches)
+            gbs = bpe * E / (ms * 1e-3) / 1e9
+            row["passes"][name] = {"us": round(ms * 1e3, 2), "bytes_per_element": bpe, "gbs": round(gbs, 0),
+                                   "frac": round(gbs / hbm_peak, 3)}
+        out.append(row)
+        del xs, dys, ys, qs, x0, dy0
+        torch.cuda.empty_cache()
+    return {"timing": f"CUDA graph of {launches} back-to-back calls per pass over rotating buffer sets (inputs not in L2)",
+            "peak_gbs": hbm_peak, "shapes": out}
+
+
+def gemm_c5_block(B, n, peaks, launches=20):
+    """The dense sweep's int8 GEMM and limb-split 16x8-bit weight-gradient GEMM at M = N = K = n: the tensor-core
+    kernel's time per launch (CUDA-event pair around each of `launches` launches, median) with the clocks sampled
+    meanwhile, against 2 x the measured bf16 peak (the nominal int8 : bf16 ratio)."""
+    import torch
+    from paper_1805_11046_b200 import synth
+    int8_peak = 2.0 * float(peaks["bf16_tflops"])
+    int8_sustained = 2.0 * float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    dev = lambda a: torch.from_numpy(a).cuda()
+    case = synth.dense_gemm(n, n, n)
+    res = {"mnk": n, "launches": launches, "peak_tops_burst": int8_peak, "peak_tops_sustained": int8_sustained,
+           "peak_source": "measured bf16 x 2 (nominal int8 : bf16)"}
+
+    def kernel_times(fn, names):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        B.trace_enable(True)
+        for _ in range(launches):
+            fn()
+        r = B.trace_records(); B.trace_enable(False)
+        ts = sorted(t for k, t in r if k in names)
+        return statistics.median(ts), ts[0]
+
+    qa, qpa = B.qbp_quantize_s8(dev(case["a"])); qb, qpb = B.qbp_quantize_s8(dev(case["b"]))
+    out = torch.empty((n, n), dtype=torch.float32, device="cuda")
+    ws = B.workspace(B.lib.qbp_gemm_s8_workspace_bytes(n, n, n))
+    sampler = ClockSampler(torch.cuda.current_device()); sampler.start()
+    med, best = kernel_times(lambda: B.qbp_gemm_s8(qa, qpa, qb, qpb, want_acc=False, out=out, ws=ws), ("qbp_mma_kernel", "qbp_mma2_kernel"))
+    clocks = sampler.stop()
+    assert B.status_word(ws) == 0
+    tops = 2.0 * n ** 3 / med / 1e9
+    res["gemm_s8"] = {"kernel": "qbp_mma2_kernel", "ms": round(med, 4), "ms_best": round(best, 4), "tops": round(tops, 1),
+                      "frac_of_measured_burst": round(tops / int8_peak, 4), "frac_of_nominal_4500": round(tops / 4500.0, 4),
+                      "frac_of_clock_adjusted": round(tops / (SM_COUNT * 16384 * float(clocks.get("sm_mhz") or 1965.0) / 1e6), 4),
+                      "clocks": clocks}
+    del qa, qb, out
+    qx, qpx = B.qbp_quantize_s8(dev(case["x"]))
+    _, hi, lo, qpg = B.qbp_quantize_s16(dev(case["g"]), want=("hi", "lo"))
+    dW = torch.empty((n, n), dtype=torch.float32, device="cuda")
+    ws = B.workspace(B.lib.qbp_wgrad_s16_workspace_bytes(None, n, n, n))
+    sampler = ClockSampler(torch.cuda.current_device()); sampler.start()
+    med, best = kernel_times(lambda: B.qbp_wgrad_s16(qx, qpx, hi, lo, qpg, want_acc=False, dW=dW, ws=ws), ("qbp_wgrad_kernel", "qbp_wgrad2_kernel"))
+    clocks = sampler.stop()
+    assert B.status_word(ws) == 0
+    useful = 2.0 * n ** 3 / med / 1e9
+    res["wgrad_s16xs8"] = {"kernel": "qbp_wgrad_kernel", "ms": round(med, 4), "ms_best": round(best, 4),
+                           "useful_tops": round(useful, 1), "executed_int8_tops": round(2 * useful, 1),
+                           "frac_of_measured_burst": round(2 * useful / int8_peak, 4),
+                           "frac_of_nominal_4500": round(2 * useful / 4500.0, 4), "clocks": clocks}
+    return res
 
 
 # ------------------------------------------------------------- CPU oracle arm
@@ -479,12 +621,23 @@ def main():
     ap.add_argument("--batch", type=int, default=BATCH, help="images per GPU (the workload is quoted at 256)")
     ap.add_argument("--cpu-sample-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the dense-GEMM and Range BN sweep blocks of the line")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a captured CUDA graph of the step")
     ap.add_argument("--only-steps", action="store_true", help="run warmup+steps and exit (for captures under ncu)")
     ap.add_argument("--workload", choices=["layer", "gemm", "rangebn"], default="layer",
                     help="layer: the headline line; gemm / rangebn: side measurements of the dense sweep and the Range BN sweep")
     ap.add_argument("--mnk", type=int, default=8192, help="--workload gemm: M = N = K")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.workload == "layer":
+        # not started by a launcher: start one rank per GPU ourselves (torch.distributed.run, loopback rendezvous)
+        import socket
+        import subprocess
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve()), *sys.argv[1:]]
+        sys.exit(subprocess.call(cmd))
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "gemm":

@@ -21,6 +21,18 @@
  *   - Return value: QBP_OK or a negative qbp_status.  Argument and shape
  *     errors are found on the host before anything is launched; the reason
  *     is kept per thread and returned by qbp_last_error().
+ *   - Device status word.  Calls are asynchronous, so a failure on the device
+ *     cannot be a return value of the call that enqueued the work.  The
+ *     tensor-core products (qbp_gemm_s8, qbp_conv_s8_implicit, qbp_wgrad_s16)
+ *     and the layer calls keep an int32 status word in the FIRST FOUR BYTES of
+ *     the workspace `ws` they are given: the call clears it, and a kernel
+ *     whose bounded wait (about one second) runs out sets it to
+ *     QBP_ERR_TIMEOUT, frees what it holds and ends normally -- the outputs
+ *     are then invalid.  Read it with qbp_device_status(ws, stream) (which
+ *     synchronises the stream) before `ws` is handed to another call.
+ *     qbp_layer_fwd clears the word of the layer's workspace once; every
+ *     product of that forward and of the following qbp_layer_bwd can only
+ *     raise it, so one read after the backward call covers the whole step.
  *   - Stored codes are signed: stored = unsigned code - 2^(M-1), and the
  *     stored zero-point is shifted the same way, so that (q - zero_point) is
  *     the value every product works on.
@@ -42,7 +54,7 @@ typedef enum {
     QBP_ERR_OVERFLOW_K = -3,        /* reduction too long for the int32 accumulator     */
     QBP_ERR_WORKSPACE = -4,         /* ws NULL or smaller than *_workspace_bytes()      */
     QBP_ERR_CUDA = -5,              /* a CUDA call failed; message holds its text       */
-    QBP_ERR_TIMEOUT = -6            /* a bounded device-side wait gave up               */
+    QBP_ERR_TIMEOUT = -6            /* a bounded device-side wait gave up (status word) */
 } qbp_status;
 
 /* Quantisation parameters of one tensor (or one channel), device resident.
@@ -81,6 +93,21 @@ int qbp_trace_enable(int on);
 int qbp_trace_count(void);
 int qbp_trace_read(int index, char *name, int name_cap, float *ms);
 
+/* Device status word of the calls that used workspace `ws` (see Conventions;
+ * no counterpart in the paper).  Copies the word at the start of `ws` to the
+ * host on `stream`, SYNCHRONISES that stream, and returns QBP_OK or
+ * QBP_ERR_TIMEOUT. */
+int qbp_device_status(const void *ws, void *stream);
+
+/* Self-test of the bounded waits (diagnostics; no counterpart in the paper):
+ * launches one warp that waits, through the same wait routines the product
+ * kernels use but with a limit of `limit_cycles` SM clock cycles (1..1e8), on
+ * a barrier that nothing ever signals.  The wait gives up, the kernel raises
+ * the status word at the start of `ws` (at least 4 bytes, cleared by this
+ * call) and ends normally; qbp_device_status(ws, stream) then returns
+ * QBP_ERR_TIMEOUT and the device remains usable. */
+int qbp_selftest_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_cycles, void *stream);
+
 /* ------------------------------------------------------------------------
  * Range quantiser -- Section 4 "Quantization methods" and Appendix B:
  *   scale = (vmax - vmin) / (2^M - 1), zero-point = round(-vmin / scale),
@@ -109,9 +136,9 @@ int qbp_quantize_s8(const float *x, int64_t rows, int64_t cols, int granularity,
                     int8_t *q, qbp_qparams *qp_out, int32_t *row_sums, int64_t *col_sums,
                     void *ws, size_t ws_bytes, void *stream);
 
-/* Clamping values for activations as Appendix B takes them ("the average of
- * absolute maximum and minimum values of K chunks", which narrows the
- * quantisation steps of tensors with a high dynamic range): x [rows x cols] is
+/* Clamping values for activations as Appendix B takes them (the mean, over K
+ * chunks of the tensor, of each chunk's largest and smallest value, which
+ * narrows the quantisation steps of tensors with a high dynamic range): x [rows x cols] is
  * cut into `chunks` equal contiguous groups of rows (rows a multiple of
  * chunks, chunks <= 4096); range_out->vmax receives the average of the groups'
  * maxima, range_out->vmin the average of their minima (sums in double, in
@@ -252,6 +279,49 @@ int qbp_rangebn_fwd(const float *x, int64_t n, int64_t C, const float *gamma, co
                     int relu, float *y, float *save_mean, float *save_min, float *save_max,
                     qbp_qparams *out_range, void *ws, size_t ws_bytes, void *stream);
 
+/* Requantisation for the next layer, fused into the pass that writes an
+ * activation.  Section 4 ("Quantization methods"): the minimum and maximum of
+ * an activation are known from the Range BN that produced it, so finding the
+ * quantiser's scale costs no further pass over the tensor.  The exact range
+ * of y follows from the per-channel statistics (y is a monotone function of x
+ * in each channel, evaluated in a fixed fp32 order, so its extremes sit at the
+ * channel's min and max); the apply pass then writes, beside y or instead of
+ * it, the 8-bit codes that qbp_quantize_s8(y, per-tensor, nearest) would
+ * produce, bit for bit:
+ *   q        [n x C] int8 codes (required)
+ *   qp       their parameters (required)
+ *   row_sums [n] sum of each row's stored codes (nullable) -- the code sums
+ *            the next product's zero-point correction needs (Appendix B). */
+typedef struct {
+    int8_t      *q;
+    qbp_qparams *qp;
+    int32_t     *row_sums;
+} qbp_requant;
+
+/* qbp_rangebn_fwd with the fused requantisation rq (nullable); y may be NULL
+ * when rq is given (the fp32 activation is then never written). */
+int qbp_rangebn_fwd_q8(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta,
+                       int relu, float *y, float *save_mean, float *save_min, float *save_max,
+                       qbp_qparams *out_range, const qbp_requant *rq,
+                       void *ws, size_t ws_bytes, void *stream);
+
+/* The two passes as separate calls, for a minibatch that is spread over
+ * several GPUs (Section 3: the mean and the range are those of the whole
+ * minibatch).  _stats leaves the per-channel sum (fp64), minimum and maximum
+ * of this GPU's n rows in col_sum / col_min / col_max [C]; the caller combines
+ * them over the GPUs (sum, min, max -- all order-free up to fp64 rounding of
+ * the sum); _apply normalises this GPU's n_rows rows with the combined
+ * statistics of n_stat >= n_rows rows (mean = sum / n_stat, C(n_stat)) and
+ * fills save_* for the backward pass.  y / out_range / rq as above. */
+int qbp_rangebn_fwd_stats(const float *x, int64_t n, int64_t C,
+                          double *col_sum, float *col_min, float *col_max,
+                          void *ws, size_t ws_bytes, void *stream);
+int qbp_rangebn_fwd_apply(const float *x, int64_t n_rows, int64_t n_stat, int64_t C,
+                          const double *col_sum, const float *col_min, const float *col_max,
+                          const float *gamma, const float *beta, int relu,
+                          float *y, float *save_mean, float *save_min, float *save_max,
+                          qbp_qparams *out_range, const qbp_requant *rq, void *stream);
+
 /* Backward -- Section 7: the derivative of max (min) is one at every
  * coordinate attaining it and zero elsewhere; otherwise the chain rule:
  *   dbeta = sum dy, dgamma = sum dy*xhat, s = 1/(C(n)(max-min)),
@@ -262,6 +332,24 @@ int qbp_rangebn_bwd(const float *dy, const float *x, int64_t n, int64_t C,
                     const float *save_mean, const float *save_min, const float *save_max,
                     float *dx, float *dgamma, float *dbeta,
                     void *ws, size_t ws_bytes, void *stream);
+
+/* The backward passes as separate calls for a minibatch spread over several
+ * GPUs: _stats leaves this GPU's sum dy and sum dy*xhat per channel (fp64,
+ * [C] each; save_* are the combined statistics of the forward); the caller
+ * adds them up over the GPUs; _apply writes dx for this GPU's rows and the
+ * complete dgamma / dbeta (nullable) from the combined sums, with n_stat the
+ * rows of the whole minibatch. */
+int qbp_rangebn_bwd_stats(const float *dy, const float *x, int64_t n_rows, int64_t n_stat, int64_t C,
+                          const float *gamma, const float *beta, int relu,
+                          const float *save_mean, const float *save_min, const float *save_max,
+                          double *sum_dy, double *sum_dyxhat,
+                          void *ws, size_t ws_bytes, void *stream);
+int qbp_rangebn_bwd_apply(const float *dy, const float *x, int64_t n_rows, int64_t n_stat, int64_t C,
+                          const float *gamma, const float *beta, int relu,
+                          const float *save_mean, const float *save_min, const float *save_max,
+                          const double *sum_dy, const double *sum_dyxhat,
+                          float *dx, float *dgamma, float *dbeta,
+                          void *ws, size_t ws_bytes, void *stream);
 
 /* ------------------------------------------------------------------------
  * Whole layer -- Sections 4 and 6: forward = quantise x and w to 8 bits
@@ -301,6 +389,22 @@ size_t qbp_layer_workspace_bytes(const qbp_layer_desc *L);
 int qbp_layer_fwd(const qbp_layer_desc *L, const float *x, const float *w,
                   const float *gamma, const float *beta, float *y, const qbp_layer_ctx *saved,
                   void *ws, size_t ws_bytes, void *stream);
+
+/* Chained layers (Section 4: the quantiser of an activation takes its range
+ * from the Range BN that produced the activation -- no range scan and no
+ * separate quantisation pass between layers).
+ *   in  (nullable): the input arrives already quantised -- the `out` record of
+ *       the previous layer's call.  x must then be NULL, and in->q / in->qp
+ *       must be the saved->x_codes / saved->qx of this layer (the backward
+ *       pass reads the input codes from there).  in->row_sums NULL: the code
+ *       sums are computed here.
+ *   out (nullable): also write the 8-bit codes of this layer's output for the
+ *       next layer (see qbp_requant); y may then be NULL.
+ * With in == NULL and out == NULL this is qbp_layer_fwd. */
+int qbp_layer_fwd_chained(const qbp_layer_desc *L, const float *x, const qbp_requant *in,
+                          const float *w, const float *gamma, const float *beta,
+                          float *y, const qbp_requant *out, const qbp_layer_ctx *saved,
+                          void *ws, size_t ws_bytes, void *stream);
 
 int qbp_layer_bwd(const qbp_layer_desc *L, const qbp_layer_ctx *saved, const float *dy,
                   const float *gamma, const float *beta,

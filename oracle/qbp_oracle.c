@@ -148,8 +148,13 @@ void qbo_qparams(float vmin, float vmax, int bits,
 
 /* One element: output = round(x/scale + zero-point), Appendix B, taken as
  * t = fma(x, 1/scale, zp_u) in fp32.  rounding 0: nearest, ties to even.
- * rounding 1: stochastic -- up with probability frac(t), using the 24 high
- * bits of the element's Philox word as the uniform draw. */
+ * rounding 1: stochastic -- up with probability frac(t).  Section 4 names
+ * stochastic rounding for the gradients and gives no formula for the draw;
+ * reading: a 16-bit uniform draw cut from the element's Philox word, the high
+ * half-word for an 8-bit code and the low half-word for a 16-bit code.  The
+ * two copies of one gradient tensor (Gradients Bifurcation: same seed, same
+ * tensor id, same element index, hence the same word) then draw from
+ * disjoint bits of that word, i.e. independently. */
 static int32_t quantize_one(float x, float inv_scale, int32_t zp_u, int32_t L,
                             int rounding, uint32_t rnd)
 {
@@ -160,7 +165,8 @@ static int32_t quantize_one(float x, float inv_scale, int32_t zp_u, int32_t L,
     } else {
         float f = floorf(t);
         float frac = t - f;
-        float u = (float)(rnd >> 8) * 0x1p-24f;
+        uint32_t draw = (L == 255) ? (rnd >> 16) : (rnd & 0xFFFFu);
+        float u = (float)draw * 0x1p-16f;
         c = f + ((u < frac) ? 1.0f : 0.0f);
     }
     if (c < 0.0f) c = 0.0f;

@@ -23,13 +23,15 @@ QBP_ERR_TIMEOUT = -6
 
 EXPORTS = (
     "qbp_last_error", "qbp_trace_enable", "qbp_trace_count", "qbp_trace_read",
+    "qbp_device_status", "qbp_selftest_bounded_wait",
     "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s8_static", "qbp_quantize_s16", "qbp_bifurcate",
     "qbp_range_chunked_workspace_bytes", "qbp_range_chunked",
     "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8",
     "qbp_conv_s8_workspace_bytes", "qbp_conv_s8_implicit",
     "qbp_wgrad_s16_workspace_bytes", "qbp_wgrad_s16",
-    "qbp_rangebn_workspace_bytes", "qbp_rangebn_fwd", "qbp_rangebn_bwd",
-    "qbp_layer_workspace_bytes", "qbp_layer_fwd", "qbp_layer_bwd",
+    "qbp_rangebn_workspace_bytes", "qbp_rangebn_fwd", "qbp_rangebn_bwd", "qbp_rangebn_fwd_q8",
+    "qbp_rangebn_fwd_stats", "qbp_rangebn_fwd_apply", "qbp_rangebn_bwd_stats", "qbp_rangebn_bwd_apply",
+    "qbp_layer_workspace_bytes", "qbp_layer_fwd", "qbp_layer_fwd_chained", "qbp_layer_bwd",
 )
 
 
@@ -54,6 +56,16 @@ class LayerCtx(C.Structure):
                 ("z", C.c_void_p), ("save_mean", C.c_void_p), ("save_min", C.c_void_p), ("save_max", C.c_void_p),
                 ("g", C.c_void_p), ("g8", C.c_void_p), ("qg8", C.c_void_p), ("g_hi", C.c_void_p), ("g_lo", C.c_void_p),
                 ("qg16", C.c_void_p)]
+
+
+class Requant(C.Structure):
+    """qbp_requant: where a pass writes the 8-bit codes of the activation it produces (q, qp) and, optionally,
+    each row's code sum."""
+    _fields_ = [("q", C.c_void_p), ("qp", C.c_void_p), ("row_sums", C.c_void_p)]
+
+
+def requant(q, qp, row_sums=None) -> Requant:
+    return Requant(q.data_ptr(), qp.data_ptr(), row_sums.data_ptr() if row_sums is not None else None)
 
 
 def _load() -> C.CDLL:
@@ -135,8 +147,17 @@ def range_qparams(vmin, vmax, device="cuda") -> torch.Tensor:
 
 
 def status_word(ws: torch.Tensor) -> int:
-    """The int32 at the start of a product's workspace: 0, or QBP_ERR_TIMEOUT if a device-side wait gave up."""
-    return int(ws[:4].view(torch.int32).item())
+    """qbp_device_status of a workspace: synchronises the current stream; 0, or QBP_ERR_TIMEOUT if a bounded
+    device-side wait of a call that used `ws` gave up."""
+    return int(lib.qbp_device_status(_ptr(ws), _stream()))
+
+
+def qbp_selftest_bounded_wait(limit_cycles: int = 4096, ws=None):
+    """Launches the library's wait self-test (a wait that nothing ends, with a short limit) and returns the
+    workspace whose status word it raises."""
+    if ws is None: ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    _check(lib.qbp_selftest_bounded_wait(_ptr(ws), C.c_size_t(ws.numel()), C.c_uint32(limit_cycles), _stream()))
+    return ws
 
 
 # ------------------------------------------------------------------ quantiser
@@ -285,6 +306,75 @@ def qbp_rangebn_fwd(x, gamma=None, beta=None, relu=False, y=None, want_range=Fal
     return y, mean, vmin, vmax, out_range
 
 
+def qbp_rangebn_fwd_q8(x, gamma=None, beta=None, relu=False, y=None, want_y=True, q=None, qp=None, row_sums=None,
+                       want_row_sums=False, ws=None):
+    """Range BN forward that also (or only: want_y=False) writes the 8-bit codes of its output for the next layer.
+    Returns (y or None, mean, vmin, vmax, q, qp, row_sums or None)."""
+    Cc = x.shape[-1]; n = x.numel() // Cc
+    if y is None and want_y: y = torch.empty_like(x)
+    if q is None: q = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+    if qp is None: qp = new_qparams(1, x.device)
+    if row_sums is None and want_row_sums: row_sums = torch.empty(n, dtype=torch.int32, device=x.device)
+    mean = torch.empty(Cc, dtype=torch.float32, device=x.device)
+    vmin = torch.empty_like(mean); vmax = torch.empty_like(mean)
+    if ws is None: ws = workspace(lib.qbp_rangebn_workspace_bytes(n, Cc), x.device)
+    rq = requant(q, qp, row_sums)
+    _check(lib.qbp_rangebn_fwd_q8(_ptr(x), C.c_int64(n), C.c_int64(Cc), _ptr(gamma), _ptr(beta), int(relu), _ptr(y),
+                                  _ptr(mean), _ptr(vmin), _ptr(vmax), None, C.byref(rq), _ptr(ws), C.c_size_t(ws.numel()),
+                                  _stream()))
+    return y, mean, vmin, vmax, q, qp, row_sums
+
+
+def qbp_rangebn_fwd_stats(x, col_sum=None, col_min=None, col_max=None, ws=None):
+    """This GPU's per-channel (sum fp64, min, max) of x, to be combined over the GPUs that share the minibatch."""
+    Cc = x.shape[-1]; n = x.numel() // Cc
+    if col_sum is None: col_sum = torch.empty(Cc, dtype=torch.float64, device=x.device)
+    if col_min is None: col_min = torch.empty(Cc, dtype=torch.float32, device=x.device)
+    if col_max is None: col_max = torch.empty(Cc, dtype=torch.float32, device=x.device)
+    if ws is None: ws = workspace(lib.qbp_rangebn_workspace_bytes(n, Cc), x.device)
+    _check(lib.qbp_rangebn_fwd_stats(_ptr(x), C.c_int64(n), C.c_int64(Cc), _ptr(col_sum), _ptr(col_min), _ptr(col_max),
+                                     _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return col_sum, col_min, col_max
+
+
+def qbp_rangebn_fwd_apply(x, n_stat, col_sum, col_min, col_max, gamma=None, beta=None, relu=False, y=None, want_y=True,
+                          rq: Requant | None = None, want_range=False):
+    """Normalise this GPU's rows with the combined statistics of n_stat rows.  Returns (y, mean, vmin, vmax, out_range)."""
+    Cc = x.shape[-1]; n = x.numel() // Cc
+    if y is None and want_y: y = torch.empty_like(x)
+    mean = torch.empty(Cc, dtype=torch.float32, device=x.device)
+    vmin = torch.empty_like(mean); vmax = torch.empty_like(mean)
+    out_range = new_qparams(1, x.device) if want_range else None
+    _check(lib.qbp_rangebn_fwd_apply(_ptr(x), C.c_int64(n), C.c_int64(n_stat), C.c_int64(Cc), _ptr(col_sum), _ptr(col_min),
+                                     _ptr(col_max), _ptr(gamma), _ptr(beta), int(relu), _ptr(y), _ptr(mean), _ptr(vmin),
+                                     _ptr(vmax), _ptr(out_range), C.byref(rq) if rq is not None else None, _stream()))
+    return y, mean, vmin, vmax, out_range
+
+
+def qbp_rangebn_bwd_stats(dy, x, n_stat, mean, vmin, vmax, gamma=None, beta=None, relu=False, ws=None):
+    """This GPU's per-channel (sum dy, sum dy*xhat), fp64, to be added up over the GPUs."""
+    Cc = x.shape[-1]; n = x.numel() // Cc
+    sdy = torch.empty(Cc, dtype=torch.float64, device=x.device); sdyx = torch.empty_like(sdy)
+    if ws is None: ws = workspace(lib.qbp_rangebn_workspace_bytes(n, Cc), x.device)
+    _check(lib.qbp_rangebn_bwd_stats(_ptr(dy), _ptr(x), C.c_int64(n), C.c_int64(n_stat), C.c_int64(Cc), _ptr(gamma),
+                                     _ptr(beta), int(relu), _ptr(mean), _ptr(vmin), _ptr(vmax), _ptr(sdy), _ptr(sdyx),
+                                     _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return sdy, sdyx
+
+
+def qbp_rangebn_bwd_apply(dy, x, n_stat, mean, vmin, vmax, sum_dy, sum_dyxhat, gamma=None, beta=None, relu=False,
+                          dx=None, ws=None):
+    Cc = x.shape[-1]; n = x.numel() // Cc
+    if dx is None: dx = torch.empty_like(x)
+    dgamma = torch.empty(Cc, dtype=torch.float32, device=x.device); dbeta = torch.empty_like(dgamma)
+    if ws is None: ws = workspace(lib.qbp_rangebn_workspace_bytes(n, Cc), x.device)
+    _check(lib.qbp_rangebn_bwd_apply(_ptr(dy), _ptr(x), C.c_int64(n), C.c_int64(n_stat), C.c_int64(Cc), _ptr(gamma),
+                                     _ptr(beta), int(relu), _ptr(mean), _ptr(vmin), _ptr(vmax), _ptr(sum_dy),
+                                     _ptr(sum_dyxhat), _ptr(dx), _ptr(dgamma), _ptr(dbeta), _ptr(ws),
+                                     C.c_size_t(ws.numel()), _stream()))
+    return dx, dgamma, dbeta
+
+
 def qbp_rangebn_bwd(dy, x, mean, vmin, vmax, gamma=None, beta=None, relu=False, dx=None, ws=None):
     Cc = x.shape[-1]; n = x.numel() // Cc
     if dx is None: dx = torch.empty_like(x)
@@ -304,6 +394,15 @@ def qbp_layer_workspace_bytes(L: LayerDesc) -> int:
 def qbp_layer_fwd(L: LayerDesc, x, w, gamma, beta, y, ctx: LayerCtx, ws):
     _check(lib.qbp_layer_fwd(C.byref(L), _ptr(x), _ptr(w), _ptr(gamma), _ptr(beta), _ptr(y), C.byref(ctx), _ptr(ws),
                              C.c_size_t(ws.numel()), _stream()))
+    return y
+
+
+def qbp_layer_fwd_chained(L: LayerDesc, x, rq_in, w, gamma, beta, y, rq_out, ctx: LayerCtx, ws):
+    """qbp_layer_fwd with the input already quantised by the previous layer (rq_in, x None) and / or the output's
+    8-bit codes written for the next one (rq_out; y may then be None)."""
+    _check(lib.qbp_layer_fwd_chained(C.byref(L), _ptr(x), C.byref(rq_in) if rq_in is not None else None, _ptr(w),
+                                     _ptr(gamma), _ptr(beta), _ptr(y), C.byref(rq_out) if rq_out is not None else None,
+                                     C.byref(ctx), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
     return y
 
 

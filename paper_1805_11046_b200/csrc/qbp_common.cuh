@@ -42,6 +42,30 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int sm_count();                                // cached multiprocessor count of the current device
 
+// Function attributes (the opt-in to more than 48 KB of dynamic shared memory) belong to a device: set them once
+// per device ordinal, whichever host thread gets there first.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    bool done[kMaxDevices] = {};
+    // true when the caller still has to do the set-up for the current device (and then calls mark())
+    bool pending(int *dev_out)
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); *dev_out = -1; return true; }
+        *dev_out = dev;
+        return !__atomic_load_n(&done[dev], __ATOMIC_ACQUIRE);
+    }
+    void mark(int dev) { if (dev >= 0) __atomic_store_n(&done[dev], true, __ATOMIC_RELEASE); }
+};
+#define QBP_SMEM_OPT_IN(once, kernel, bytes)                                                                       \
+    do {                                                                                                           \
+        int dev_ = -1;                                                                                             \
+        if ((once).pending(&dev_)) {                                                                               \
+            QBP_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes)));  \
+            (once).mark(dev_);                                                                                     \
+        }                                                                                                          \
+    } while (0)
+
 // Carves 256-byte aligned pieces out of the caller's workspace.
 struct WsCarver {
     char *base; size_t off; size_t cap;
@@ -90,7 +114,9 @@ __device__ __forceinline__ qbp_qparams make_qparams(float vmin, float vmax, int 
     return q;
 }
 
-// One element to its unsigned code in [0, L].  rnd is the element's Philox word.
+// One element to its unsigned code in [0, L].  rnd is the element's Philox word; stochastic rounding takes a
+// 16-bit draw from it: the high half-word for an 8-bit code, the low half-word for a 16-bit code (the two copies
+// of one gradient then round independently from one word).
 template <bool STOCHASTIC>
 __device__ __forceinline__ int quantize_code(float x, float inv_scale, float zp_u, float Lf, uint32_t rnd)
 {
@@ -101,7 +127,8 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, float zp_
     } else {
         float f = floorf(t);
         float frac = __fsub_rn(t, f);
-        float u = __fmul_rn((float)(rnd >> 8), 0x1p-24f);
+        const uint32_t draw = (Lf == 255.0f) ? (rnd >> 16) : (rnd & 0xFFFFu);
+        float u = __fmul_rn((float)draw, 0x1p-16f);
         c = (u < frac) ? __fadd_rn(f, 1.0f) : f;
     }
     // c is integral: the saturating conversion is the clamp to [0, 2^bits - 1] (Lf selects the width)
@@ -111,27 +138,39 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, float zp_
     return (int)code;
 }
 
-// The stochastic 8-bit code of one element in fixed point: the same result as quantize_code<true>(.., 255, rnd) with
-// three instructions fewer.  With t = fma(x, inv, zp) >= 0, f = floor(t), frac = t - f and r24 = rnd >> 8, the code
-// is f + [r24 * 2^-24 < frac] = f + [r24 < ceil(frac * 2^24)] (r24 is an integer); t * 2^24 is exact in fp32 and
-// ceil(t * 2^24) = f * 2^24 + ceil(frac * 2^24), so adding 2^24 - 1 - r24 (= ~rnd >> 8) carries into bit 24 exactly
-// when the code rounds up.  The conversion saturates negative t to 0 (code 0, as the clamp gives) and the minimum
-// with 255 * 2^24 is the clamp at the top (then nothing can carry).  Returns the code in the TOP byte of the word.
-__device__ __forceinline__ uint32_t quantize_sr8_top_byte(float x, float inv_scale, float zp_u, uint32_t rnd)
+// The stochastic codes of one element in fixed point: the same results as quantize_code<true> with fewer
+// instructions.  With t = fma(x, inv, zp), f = floor(t), frac = t - f and a 16-bit draw d, the code is
+// f + [d * 2^-16 < frac] = f + [d < ceil(frac * 2^16)] (d is an integer).  t * 2^16 is exact in fp32 and
+// ceil(t * 2^16) = f * 2^16 + ceil(frac * 2^16), so adding 0xFFFF - d carries into bit 16 exactly when the code
+// rounds up.  The conversion saturates negative t to 0 (code 0, as the clamp gives) and the minimum with
+// L * 2^16 is the clamp at the top (then nothing can carry).
+// 8 bits: the code is byte 2 of the result; the draw is the high half of rnd.
+__device__ __forceinline__ uint32_t quantize_sr8_byte2(float x, float inv_scale, float zp_u, uint32_t rnd)
 {
     const float t = __fmaf_rn(x, inv_scale, zp_u);
     uint32_t tc;
-    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmul_rn(t, 16777216.0f)));
-    return min(tc, 0xFF000000u) + ((~rnd) >> 8);
+    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmul_rn(t, 65536.0f)));
+    return min(tc, 0x00FF0000u) + ((~rnd) >> 16);
+}
+// 16 bits: the code is the upper half of the result (high byte = byte 3, low byte = byte 2); the draw is the low half of rnd.
+__device__ __forceinline__ uint32_t quantize_sr16_top_half(float x, float inv_scale, float zp_u, uint32_t rnd)
+{
+    const float t = __fmaf_rn(x, inv_scale, zp_u);
+    uint32_t tc;
+    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmul_rn(t, 65536.0f)));
+    return min(tc, 0xFFFF0000u) + ((~rnd) & 0xFFFFu);
 }
 
-// Philox4x32-10 with the ten round keys precomputed (they depend on the key only).
+// Philox4x32-10 with the ten round keys precomputed (they depend on the key only); passed to a kernel by value,
+// they sit in its constant parameter space and cost no registers.
 struct PhiloxKeys { uint32_t k0[10], k1[10]; };
-__device__ __forceinline__ PhiloxKeys philox_keys(uint2 k)
+inline PhiloxKeys philox_keys_host(uint64_t seed)
 {
     PhiloxKeys r;
-#pragma unroll
-    for (int i = 0; i < 10; ++i) { r.k0[i] = k.x + (uint32_t)i * 0x9E3779B9u; r.k1[i] = k.y + (uint32_t)i * 0xBB67AE85u; }
+    for (int i = 0; i < 10; ++i) {
+        r.k0[i] = (uint32_t)seed + (uint32_t)i * 0x9E3779B9u;
+        r.k1[i] = (uint32_t)(seed >> 32) + (uint32_t)i * 0xBB67AE85u;
+    }
     return r;
 }
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys &k)
@@ -193,39 +232,43 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after about a second of SM clock and reports false; the
-// caller then raises the kernel's error flag and leaves through its normal exit.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+// Bounded wait: gives up after `limit` SM clock cycles (by default about a second) and reports false; the
+// caller then raises the kernel's status word and leaves through its normal exit.
+constexpr long long kWaitLimitCycles = 2000000000ll;
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, long long limit = kWaitLimitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
-        if (clock64() - t0 > 2000000000ll) return false;
+        if (clock64() - t0 > limit) return false;
     return true;
 }
 
 // The same wait by every lane of a converged warp; the answer is the same in all of them.
-__device__ __forceinline__ bool mbar_wait_uniform(uint64_t *bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_uniform(uint64_t *bar, uint32_t parity, long long limit = kWaitLimitCycles)
 {
-    const bool ok = mbar_wait(bar, parity);
+    const bool ok = mbar_wait(bar, parity, limit);
     return __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
 }
 
 // The same wait for a whole warp: one lane polls (with a short sleep between polls, so that waiting warps
 // leave the shared-memory pipe to the warps that feed the tensor core), the result is shared by shuffle.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, long long limit = kWaitLimitCycles)
 {
     int ok = 1;
     if ((threadIdx.x & 31) == 0 && !mbar_try_wait(bar, parity)) {
         const long long t0 = clock64();
         while (!mbar_try_wait(bar, parity)) {
-            if (clock64() - t0 > 2000000000ll) { ok = 0; break; }
+            if (clock64() - t0 > limit) { ok = 0; break; }
             __nanosleep(40);
         }
     }
     ok = __shfl_sync(0xffffffffu, ok, 0);
     return ok != 0;
 }
+
+// A kernel whose bounded wait ran out records it here; the word only ever goes from 0 to QBP_ERR_TIMEOUT.
+__device__ __forceinline__ void raise_timeout(int *status) { atomicExch(status, (int)QBP_ERR_TIMEOUT); }
 
 __device__ __forceinline__ void fence_proxy_async()
 {

@@ -30,18 +30,33 @@ static int layer_shape(const qbp_layer_desc *L, LayerShape &s)
         const qbp_conv_desc &d = L->conv;
         if (d.N <= 0 || d.H <= 0 || d.W <= 0 || d.C <= 0 || d.K <= 0 || d.R <= 0 || d.S <= 0)
             return fail(QBP_ERR_INVALID_ARG, "layer: bad convolution geometry");
+        // what every product of the step implements, checked before anything is launched
+        if (!conv_supported(&d) || !wgrad_conv_supported(&d))
+            return fail(QBP_ERR_UNSUPPORTED_SHAPE,
+                        "layer: needs stride 1, R = S in {1,3}, pad = (R-1)/2, C and K multiples of 32");
+        if ((int64_t)d.R * d.S * std::max(d.C, d.K) > 33025)
+            return fail(QBP_ERR_OVERFLOW_K, "layer: reduction length exceeds 33025");
         s.rows = (int64_t)d.N * d.H * d.W; s.cin = d.C; s.cout = d.K;
         s.x_elems = s.rows * d.C; s.w_elems = (int64_t)d.K * d.R * d.S * d.C;
     } else {
         if (L->batch <= 0 || L->in_features <= 0 || L->out_features <= 0)
             return fail(QBP_ERR_INVALID_ARG, "layer: batch, in_features, out_features must be positive");
+        if (L->batch % 16 || L->in_features % 16 || L->out_features % 16)
+            return fail(QBP_ERR_UNSUPPORTED_SHAPE, "layer: batch, in_features, out_features must be multiples of 16");
+        if (L->in_features > 33025 || L->out_features > 33025)
+            return fail(QBP_ERR_OVERFLOW_K, "layer: in_features and out_features are reduction lengths of 8-bit products (at most 33025)");
         s.rows = L->batch; s.cin = L->in_features; s.cout = L->out_features;
         s.x_elems = s.rows * s.cin; s.w_elems = s.cin * s.cout;
     }
+    if (s.rows < 2) return fail(QBP_ERR_INVALID_ARG, "layer: Range BN needs at least 2 rows");
     return QBP_OK;
 }
 
-// Scratch shared by the steps (they run one after another on the stream).
+// The layer's workspace: [0, kLayerHead) the sticky status word of the whole step (cleared once by the forward
+// call, raised by any product whose bounded wait runs out, never overwritten by a later step), then the scratch
+// the steps share (they run one after another on the stream), then the buffers that live across steps.
+constexpr size_t kLayerHead = 256;
+
 static size_t step_scratch_bytes(const qbp_layer_desc *L, const LayerShape &s)
 {
     size_t b = qbp_quantize_workspace_bytes(s.rows, std::max(s.cin, s.cout), QBP_PER_TENSOR);
@@ -77,7 +92,7 @@ extern "C" __attribute__((visibility("default"))) size_t qbp_layer_workspace_byt
 {
     LayerShape s;
     if (layer_shape(L, s)) return 0;
-    return step_scratch_bytes(L, s) + chained_bytes(s);
+    return kLayerHead + step_scratch_bytes(L, s) + chained_bytes(s);
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_layer_desc *L, const float *x,
@@ -86,24 +101,53 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_la
                                                                    const qbp_layer_ctx *saved, void *ws,
                                                                    size_t ws_bytes, void *stream)
 {
+    if (!x || !y) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: NULL argument");
+    return qbp_layer_fwd_chained(L, x, nullptr, w, gamma, beta, y, nullptr, saved, ws, ws_bytes, stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(const qbp_layer_desc *L, const float *x,
+                                                                           const qbp_requant *in, const float *w,
+                                                                           const float *gamma, const float *beta,
+                                                                           float *y, const qbp_requant *out,
+                                                                           const qbp_layer_ctx *saved, void *ws,
+                                                                           size_t ws_bytes, void *stream)
+{
     LayerShape s;
     int rc = layer_shape(L, s);
     if (rc) return rc;
-    if (!x || !w || !y || !saved) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: NULL argument");
+    if (!w || !saved) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: NULL argument");
+    if ((x != nullptr) == (in != nullptr))
+        return fail(QBP_ERR_INVALID_ARG, "layer_fwd: exactly one of x (fp32 input) and in (input already quantised) is needed");
+    if (!y && !out) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: neither y nor 8-bit output codes wanted");
+    if (out && (!out->q || !out->qp)) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: the output record needs q and qp");
     if (!saved->x_codes || !saved->qx || !saved->w_codes || !saved->qw || !saved->z || !saved->save_mean ||
         !saved->save_min || !saved->save_max)
         return fail(QBP_ERR_INVALID_ARG, "layer_fwd: the saved-state record has a NULL buffer");
+    if (in && (in->q != saved->x_codes || in->qp != saved->qx))
+        return fail(QBP_ERR_INVALID_ARG, "layer_fwd: in->q / in->qp must be the layer's saved x_codes / qx");
     if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
         return fail(QBP_ERR_WORKSPACE, "layer_fwd: workspace of %zu bytes needed, %zu given",
                     qbp_layer_workspace_bytes(L), ws_bytes);
     const size_t scratch = step_scratch_bytes(L, s);
+    cudaStream_t st = (cudaStream_t)stream;
+    int *status = static_cast<int *>(ws);
+    QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
+    ws = static_cast<char *>(ws) + kLayerHead;
 
-    // weights and activations: nearest rounding, clamping values = min and max (Appendix B)
-    // (convolution: the quantiser also leaves each pixel's code sum for the zero-point correction of the product)
+    // activations: nearest rounding, clamping values = min and max (Appendix B) -- or already quantised by the
+    // Range BN of the layer before (Section 4)
+    // (convolution: each pixel's code sum is needed for the zero-point correction of the product)
     int32_t *row_sums = reinterpret_cast<int32_t *>(static_cast<char *>(ws) + scratch);
-    rc = qbp_quantize_s8(x, s.rows, s.cin, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, saved->x_codes, saved->qx,
-                         s.conv ? row_sums : nullptr, nullptr, ws, scratch, stream);
-    if (rc) return rc;
+    const int32_t *in_sums = s.conv ? row_sums : nullptr;
+    if (x) {
+        rc = qbp_quantize_s8(x, s.rows, s.cin, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, saved->x_codes, saved->qx,
+                             s.conv ? row_sums : nullptr, nullptr, ws, scratch, stream);
+        if (rc) return rc;
+    } else if (s.conv) {
+        if (in->row_sums) in_sums = in->row_sums;
+        else if ((rc = launch_rowsum(in->q, true, s.rows, s.cin, row_sums, st))) return rc;
+    }
+    // weights: nearest rounding, clamping values = min and max
     const int64_t w_rows = s.conv ? (int64_t)L->conv.K * L->conv.R * L->conv.S : s.cin;
     rc = qbp_quantize_s8(w, w_rows, s.w_elems / w_rows, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr,
                          saved->w_codes, saved->qw, nullptr, nullptr, ws, scratch, stream);
@@ -118,17 +162,17 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd(const qbp_la
     }
     if (s.conv)
         rc = conv_s8_impl(QBP_CONV_FPROP, &L->conv, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr, saved->z,
-                          row_sums, parts.sum ? &parts : nullptr, ws, scratch, (cudaStream_t)stream);
+                          in_sums, parts.sum ? &parts : nullptr, status, ws, scratch, st);
     else
-        rc = qbp_gemm_s8(0, 0, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr,
-                         saved->z, nullptr, ws, scratch, stream);
+        rc = gemm_s8_impl(0, 0, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr,
+                          saved->z, nullptr, status, ws, scratch, st);
     if (rc) return rc;
     // the convolution's epilogue has left the statistics of z: no pass over z for them
     if (parts.sum)
         return rangebn_fwd_from_parts(saved->z, s.rows, s.cout, gamma, beta, L->relu, y, saved->save_mean, saved->save_min,
-                                      saved->save_max, parts, (cudaStream_t)stream);
-    return qbp_rangebn_fwd(saved->z, s.rows, s.cout, gamma, beta, L->relu, y, saved->save_mean, saved->save_min,
-                           saved->save_max, nullptr, ws, scratch, stream);
+                                      saved->save_max, parts, nullptr, out, st);
+    return qbp_rangebn_fwd_q8(saved->z, s.rows, s.cout, gamma, beta, L->relu, y, saved->save_mean, saved->save_min,
+                              saved->save_max, nullptr, out, ws, scratch, stream);
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_layer_desc *L, const qbp_layer_ctx *saved,
@@ -153,6 +197,8 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     qbp_qparams *qp8 = saved->qg8, *qp16 = saved->qg16;
 
     cudaStream_t st = (cudaStream_t)stream;
+    int *status = static_cast<int *>(ws);          // the forward call cleared it; the backward only ever raises it
+    ws = static_cast<char *>(ws) + kLayerHead;
     int32_t *row_sums = reinterpret_cast<int32_t *>(static_cast<char *>(ws) + scratch);
     float2 *range_parts = reinterpret_cast<float2 *>(static_cast<char *>(ws) + scratch + align_up(sizeof(int32_t) * (size_t)s.rows, 256));
     // the pass that writes the gradient also leaves its range (Section 4: no extra scan for the quantiser)
@@ -165,13 +211,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st);
     if (rc) return rc;
     if (s.conv) {
-        rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, nullptr, ws, scratch, st);
+        rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, nullptr, status, ws, scratch, st);
         if (rc) return rc;
-        return qbp_wgrad_s16(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, ws, scratch, stream);
+        return wgrad_s16_impl(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws, scratch, st);
     }
     // dx [batch x in] = g8 [batch x out] . w^T, w stored [in x out]
-    rc = qbp_gemm_s8(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, nullptr, ws, scratch, stream);
+    rc = gemm_s8_impl(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, nullptr, status, ws, scratch, st);
     if (rc) return rc;
-    return qbp_wgrad_s16(nullptr, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, ws,
-                         scratch, stream);
+    return wgrad_s16_impl(nullptr, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws,
+                          scratch, st);
 }

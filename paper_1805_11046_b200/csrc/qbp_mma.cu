@@ -354,8 +354,6 @@ __device__ __forceinline__ void issue_stage(const MmaParams &P, uint32_t a_lo, u
     }
 }
 
-__device__ __forceinline__ void raise_timeout(int *status) { atomicExch(status, (int)QBP_ERR_TIMEOUT); }
-
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The producer runs ahead of
 // the MMA warp across tile boundaries through the shared-memory ring.  A CTA tile is msub accumulator
 // sub-tiles of 128 rows x bn columns that share the B operand of every stage (256 x 256 halves the
@@ -816,6 +814,19 @@ __global__ void __launch_bounds__(128) colstat_finalize_kernel(const float *__re
 
 int colstat_rows_max() { return sm_count(); }
 
+// Self-test of the bounded wait (diagnostics): one warp waits on an mbarrier on which nothing ever arrives, with
+// the wait wrappers the product kernels use and a limit of `limit` cycles; the wait gives up, the status word is
+// raised and the kernel ends through its normal exit.
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(long long limit, int *status)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+    __syncwarp();
+    bool timed_out = !mbar_wait_uniform(&bar, 0, limit);            // every lane polls (the MMA warps' wait)
+    if (!timed_out) timed_out = !mbar_wait_warp(&bar, 0, limit);    // (not reached: the first wait cannot succeed)
+    if (timed_out && threadIdx.x == 0) raise_timeout(status);
+}
+
 static size_t colstat_ws_bytes(int64_t N)
 {
     if (N > QBP_EPILOGUE_MAX_COLUMNS) return 0;
@@ -867,7 +878,7 @@ static bool halo_fits(MmaParams &P, uint32_t halo_tile_bytes)
     return P.tiles_n == 1 && fixed + align_up((size_t)P.b.tile_bytes * P.k_iters, 1024) + 3u * halo_tile_bytes <= kSmemBudget;
 }
 
-static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
+static int launch_mma(MmaParams &P, int tiles_m, bool clear_status, cudaStream_t st)
 {
     const uint32_t fixed = fixed_smem(P);
     const uint32_t budget = kSmemBudget - fixed;
@@ -914,12 +925,9 @@ static int launch_mma(MmaParams &P, int tiles_m, cudaStream_t st)
     P.d_tiles_w = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_w);
     P.d_tiles_h = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_h);
     const size_t smem = (size_t)fixed + P.b_res_bytes + (size_t)stages * stage_bytes;
-    static thread_local bool configured = false;
-    if (!configured) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
-        configured = true;
-    }
-    QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
+    static PerDeviceOnce configured;
+    QBP_SMEM_OPT_IN(configured, qbp_mma_kernel, kSmemBudget);
+    if (clear_status) QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
     // one CTA per SM (its shared-memory ring fills the SM), each walking its share of the tiles
     const int grid = std::min(P.tiles_total, sm_count());
     P.grid = grid;
@@ -935,7 +943,7 @@ static size_t gemm_ws_bytes(int64_t M, int64_t N)
            align_up(sizeof(int64_t) * M, 256) + align_up(sizeof(int64_t) * N, 256) + colstat_ws_bytes(N);
 }
 
-static bool conv_supported(const qbp_conv_desc *d)
+bool conv_supported(const qbp_conv_desc *d)
 {
     return d->stride == 1 && d->R == d->S && (d->R == 1 || d->R == 3) && d->pad == (d->R - 1) / 2 && d->N > 0 &&
            d->H > 0 && d->W > 0 && d->C > 0 && d->K > 0 && d->C % 16 == 0 && d->K % 16 == 0;
@@ -973,6 +981,31 @@ static void pick_pixel_box(int Nimg, int H, int W, int &bwl, int &bhl)
 
 using namespace qbp;
 
+extern "C" __attribute__((visibility("default"))) int qbp_device_status(const void *ws, void *stream)
+{
+    if (!ws) return fail(QBP_ERR_INVALID_ARG, "device_status: ws is NULL");
+    int word = 0;
+    QBP_CUDA_OK(cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    QBP_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+    if (word == (int)QBP_ERR_TIMEOUT)
+        return fail(QBP_ERR_TIMEOUT, "a bounded device-side wait gave up: the outputs of the calls that used this workspace are invalid");
+    if (word != 0) return fail(QBP_ERR_INVALID_ARG, "device_status: the workspace does not start with a status word (found %d)", word);
+    return QBP_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_selftest_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_cycles, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!ws || ws_bytes < sizeof(int)) return fail(QBP_ERR_WORKSPACE, "selftest_bounded_wait: workspace of 4 bytes needed");
+    if (limit_cycles == 0 || limit_cycles > 100000000u)
+        return fail(QBP_ERR_INVALID_ARG, "selftest_bounded_wait: limit_cycles must be in [1, 1e8]");
+    QBP_CUDA_OK(cudaMemsetAsync(ws, 0, sizeof(int), st));
+    QBP_TRACE_BEGIN(st);
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>((long long)limit_cycles, static_cast<int *>(ws));
+    QBP_LAUNCH_OK("bounded_wait_selftest_kernel");
+    return QBP_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) size_t qbp_gemm_s8_workspace_bytes(int64_t M, int64_t N, int64_t K)
 {
     (void)K;
@@ -983,7 +1016,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
                            const qbp_qparams *qa, const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C,
                            const qbp_epilogue *ep, void *ws, size_t ws_bytes, void *stream)
 {
-    cudaStream_t st = (cudaStream_t)stream;
+    return gemm_s8_impl(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, ep, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int qbp::gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
+                      const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const qbp_epilogue *ep,
+                      int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st)
+{
     if (M <= 0 || N <= 0 || K <= 0) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: M, N, K must be positive");
     if (M % 16 || N % 16 || K % 16) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "gemm_s8: M, N, K must be multiples of 16");
     if (K > 33025) return fail(QBP_ERR_OVERFLOW_K, "gemm_s8: K = %lld exceeds 33025 (255*255*K must fit int32)", (long long)K);
@@ -1002,6 +1041,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     }
     WsCarver w(ws, ws_bytes);
     int *status = w.take<int>(1);
+    if (ext_status) status = ext_status;         // the caller's sticky word: raised here, never cleared
     int32_t *rowterm = w.take<int32_t>(M);
     int32_t *colterm = w.take<int32_t>(N);
     int64_t *tmp_m = w.take<int64_t>(M);
@@ -1031,7 +1071,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     // large products run on CTA pairs (256 x 256 tiles across two SMs); the column statistics are the
     // single-CTA kernel's (at most 256 columns: narrow either way)
     if (gemm2_eligible(M, N, K) && !stats)
-        return launch_gemm2(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, rowterm, colterm, status, st);
+        return launch_gemm2(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, rowterm, colterm, status, !ext_status, st);
 
     MmaParams P{};
     P.mode = MODE_GEMM;
@@ -1071,7 +1111,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     P.acc_out = acc_out; P.out = C;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = qa; P.qb = qb; P.status = status;
     if (stats) { P.st_lo = parts.lo; P.st_hi = parts.hi; P.st_sum = parts.sum; }
-    if ((rc = launch_mma(P, (int)((M + 128 * P.msub - 1) / (128 * P.msub)), st))) return rc;
+    if ((rc = launch_mma(P, (int)((M + 128 * P.msub - 1) / (128 * P.msub)), !ext_status, st))) return rc;
     if (stats) { parts.rows = P.grid; return finish_epilogue(ep, parts, N, st); }
     return QBP_OK;
 }
@@ -1106,17 +1146,17 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
             parts.hi = reinterpret_cast<float *>(base + align_up(cells * sizeof(float), 256));
             parts.sum = reinterpret_cast<double *>(base + 2 * align_up(cells * sizeof(float), 256));
             parts.rows = 0;
-            const int rc = conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, &parts, ws, core, (cudaStream_t)stream);
+            const int rc = conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, &parts, nullptr, ws, core, (cudaStream_t)stream);
             if (rc) return rc;
             return finish_epilogue(ep, parts, Nout, (cudaStream_t)stream);
         }
     }
-    return conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+    return conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, nullptr, nullptr, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
                       const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, ColStatParts *stats,
-                      void *ws, size_t ws_bytes, cudaStream_t st)
+                      int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (!d) return fail(QBP_ERR_INVALID_ARG, "conv_s8: descriptor is NULL");
     if (mode != QBP_CONV_FPROP && mode != QBP_CONV_DGRAD) return fail(QBP_ERR_INVALID_ARG, "conv_s8: bad mode");
@@ -1144,6 +1184,7 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
 
     WsCarver w(ws, ws_bytes);
     int *status = w.take<int>(1);
+    if (ext_status) status = ext_status;         // the caller's sticky word: raised here, never cleared
     int32_t *rowterm = w.take<int32_t>(pix);
     int32_t *chan_sum = w.take<int32_t>(pix);
     int32_t *colterm = w.take<int32_t>(16 * nmax);
@@ -1232,7 +1273,7 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
     P.acc_out = acc_out; P.out = out;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
-    if ((rc = launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, st))) return rc;
+    if ((rc = launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, !ext_status, st))) return rc;
     if (stats) stats->rows = P.grid;
     return QBP_OK;
 }

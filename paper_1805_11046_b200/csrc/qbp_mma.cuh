@@ -30,12 +30,25 @@ int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, ui
 // of the tensor-core kernel; `rows` is filled in by the launch.  colstat_rows_max(): the most rows a launch leaves.
 struct ColStatParts { float *lo, *hi; double *sum; int rows; };
 int colstat_rows_max();
+// ext_status (here and below; nullable): a status word the caller owns and has cleared -- the product raises it when
+// a bounded wait runs out and never clears it; NULL: the word is the first int of `ws`, cleared by the call itself.
 int conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
                  const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, ColStatParts *stats,
-                 void *ws, size_t ws_bytes, cudaStream_t st);
+                 int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);
+int gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
+                 const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const qbp_epilogue *ep,
+                 int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);
+int wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
+                   const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
+                   int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);
+// Shapes the convolution products / the convolution weight gradient implement.
+bool conv_supported(const qbp_conv_desc *d);
+bool wgrad_conv_supported(const qbp_conv_desc *d);
 // Range BN forward from such partials instead of a statistics pass over x (qbp_rangebn.cu).
+// out_range / rq (each nullable): the exact range of y / its 8-bit codes for the next layer (see qbp_requant).
 int rangebn_fwd_from_parts(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu, float *y,
-                           float *save_mean, float *save_min, float *save_max, const ColStatParts &parts, cudaStream_t st);
+                           float *save_mean, float *save_min, float *save_max, const ColStatParts &parts,
+                           qbp_qparams *out_range, const qbp_requant *rq, cudaStream_t st);
 
 // ---- TMA tensor maps ---------------------------------------------------------
 // A dense byte matrix [rows x cols] (cols innermost) read in boxes of
@@ -52,7 +65,7 @@ int make_map_out_2d(CUtensorMap *map, float *base, uint64_t rows, uint64_t cols)
 bool gemm2_eligible(int64_t M, int64_t N, int64_t K);
 int launch_gemm2(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
                  const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const int32_t *rowterm,
-                 const int32_t *colterm, int *status, cudaStream_t st);
+                 const int32_t *colterm, int *status, bool clear_status, cudaStream_t st);
 
 // ---- shared-memory operand descriptors ---------------------------------------
 // How one operand tile of a pipeline stage is laid out and walked by the MMAs.

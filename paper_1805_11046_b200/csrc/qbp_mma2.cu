@@ -343,7 +343,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(k2Threads, 1) qbp_mm
     }
 
     if (timed_out) {
-        atomicExch(P.status, (int)QBP_ERR_TIMEOUT);
+        raise_timeout(P.status);
         __nanosleep(1000000);
     }
     tc_fence_before();
@@ -361,7 +361,7 @@ bool gemm2_eligible(int64_t M, int64_t N, int64_t K)
 
 int launch_gemm2(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
                  const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const int32_t *rowterm,
-                 const int32_t *colterm, int *status, cudaStream_t st)
+                 const int32_t *colterm, int *status, bool clear_status, cudaStream_t st)
 {
     Mma2Params P{};
     int rc;
@@ -393,12 +393,9 @@ int launch_gemm2(int transA, int transB, int64_t M, int64_t N, int64_t K, const 
     P.M = M; P.N = N; P.acc_out = acc_out; P.out = C;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = qa; P.qb = qb; P.status = status;
     const size_t smem = 1024 + (size_t)stages * stage_bytes + k2EpiWarps * k2Slab;
-    static thread_local bool configured = false;
-    if (!configured) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(qbp_mma2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k2Smem));
-        configured = true;
-    }
-    QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
+    static PerDeviceOnce configured;
+    QBP_SMEM_OPT_IN(configured, qbp_mma2_kernel, k2Smem);
+    if (clear_status) QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
     QBP_TRACE_BEGIN(st);
     qbp_mma2_kernel<<<2 * P.pairs, k2Threads, smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_mma2_kernel");

@@ -295,7 +295,7 @@ __device__ __forceinline__ QParamsReg load_qp(const qbp_qparams *qp, int bits)
 template <bool SR>
 __device__ __forceinline__ void quantize_scalar(const float *x, int64_t i, int cols, bool perch,
                                                 const qbp_qparams *qp8, uint32_t id8, const qbp_qparams *qp16,
-                                                uint32_t id16, uint2 key, const QuantOut &o)
+                                                uint32_t id16, const PhiloxKeys &key, const QuantOut &o)
 {
     const int c = perch ? (int)(i % cols) : 0;
     const float v = x[i];
@@ -340,6 +340,11 @@ __device__ __forceinline__ uint32_t pack_bytes1(const uint32_t (&c)[4])
 {
     return __byte_perm(__byte_perm(c[0], c[1], 0x0051), __byte_perm(c[2], c[3], 0x0051), 0x5410);
 }
+// The third bytes of c[0..3] into one word.
+__device__ __forceinline__ uint32_t pack_bytes2(const uint32_t (&c)[4])
+{
+    return __byte_perm(__byte_perm(c[0], c[1], 0x0062), __byte_perm(c[2], c[3], 0x0062), 0x5410);
+}
 
 // PERCH is a template parameter so that the per-tensor instance (the hot one: it is bound by its instruction
 // count when rounding stochastically) carries none of the per-channel parameter handling.
@@ -347,12 +352,13 @@ template <bool SR, int VEC, bool PERCH>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restrict__ x, int64_t n, int cols,
                                                             const qbp_qparams *__restrict__ qp8,
                                                             uint32_t id8, const qbp_qparams *__restrict__ qp16,
-                                                            uint32_t id16, uint2 key, QuantOut o, int smem_cols)
+                                                            uint32_t id16, const __grid_constant__ PhiloxKeys keys,
+                                                            QuantOut o, int smem_cols)
 {
     if (VEC == 1) {
         const int64_t stride = (int64_t)gridDim.x * kThreads;
         for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += stride)
-            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, key, o);
+            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o);
         return;
     }
     const bool want8 = o.q8 != nullptr, want16 = o.q16 || o.hi || o.lo;
@@ -372,7 +378,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
         if (want8) p8 = load_qp(qp8, 8);
         if (want16) p16 = load_qp(qp16, 16);
     }
-    const PhiloxKeys keys = philox_keys(key);
+    // both copies of a gradient under one tensor id: one Philox block serves the two (disjoint halves of each word)
+    const bool one_block = want8 && want16 && id8 == id16;
     const int64_t nv = n >> 2;
     const int64_t stride = (int64_t)gridDim.x * kThreads * kUnroll;
     for (int64_t base = (int64_t)blockIdx.x * kThreads * kUnroll; base < nv; base += stride) {
@@ -395,12 +402,13 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
             const int64_t j = base + u * kThreads + threadIdx.x;
             const float xs[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
             const int c0 = PERCH ? (int)((j << 2) % cols) : 0;
+            uint4 b8 = make_uint4(0, 0, 0, 0), b16 = b8;
+            if (SR) {
+                if (want8) b8 = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id8, 0u), keys);
+                if (want16) b16 = one_block ? b8 : philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id16, 0u), keys);
+            }
             if (want8) {
-                uint32_t r[4] = {0, 0, 0, 0};
-                if (SR) {
-                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id8, 0u), keys);
-                    r[0] = b.x; r[1] = b.y; r[2] = b.z; r[3] = b.w;
-                }
+                const uint32_t r[4] = {b8.x, b8.y, b8.z, b8.w};
                 uint32_t c[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -408,19 +416,15 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                         if (table) { const float2 t = s_qp[c0 + e]; p8.inv = t.x; p8.zp_u = t.y; }
                         else p8 = load_qp(qp8 + c0 + e, 8);
                     }
-                    c[e] = SR ? quantize_sr8_top_byte(xs[e], p8.inv, p8.zp_u, r[e])
+                    c[e] = SR ? quantize_sr8_byte2(xs[e], p8.inv, p8.zp_u, r[e])
                               : (uint32_t)quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
                 }
-                const uint32_t packed = (SR ? pack_bytes3(c) : pack_bytes0(c)) ^ 0x80808080u;       // stored = unsigned code - 128
+                const uint32_t packed = (SR ? pack_bytes2(c) : pack_bytes0(c)) ^ 0x80808080u;       // stored = unsigned code - 128
                 reinterpret_cast<uint32_t *>(o.q8)[j] = packed;
                 if (o.rowsum8) rs[u] = __dp4a((int)packed, 0x01010101, 0);
             }
             if (want16) {
-                uint32_t r[4] = {0, 0, 0, 0};
-                if (SR) {
-                    uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id16, 0u), keys);
-                    r[0] = b.x; r[1] = b.y; r[2] = b.z; r[3] = b.w;
-                }
+                const uint32_t r[4] = {b16.x, b16.y, b16.z, b16.w};
                 uint32_t c[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -428,14 +432,16 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                         if (table) { const float2 t = s_qp[cols + c0 + e]; p16.inv = t.x; p16.zp_u = t.y; }
                         else p16 = load_qp(qp16 + c0 + e, 16);
                     }
-                    c[e] = (uint32_t)quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]);
+                    // (stochastic: the code sits in the upper half of the word, i.e. bytes 3 and 2)
+                    c[e] = SR ? quantize_sr16_top_half(xs[e], p16.inv, p16.zp_u, r[e])
+                              : (uint32_t)quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]);
                 }
                 // stored = unsigned code - 32768: flip the top bit of every code (of every high byte)
                 if (o.q16)
-                    reinterpret_cast<uint2 *>(o.q16)[j] = make_uint2(__byte_perm(c[0], c[1], 0x5410) ^ 0x80008000u,
-                                                                     __byte_perm(c[2], c[3], 0x5410) ^ 0x80008000u);
-                if (o.hi) reinterpret_cast<uint32_t *>(o.hi)[j] = pack_bytes1(c) ^ 0x80808080u;
-                if (o.lo) reinterpret_cast<uint32_t *>(o.lo)[j] = pack_bytes0(c);
+                    reinterpret_cast<uint2 *>(o.q16)[j] = make_uint2(__byte_perm(c[0], c[1], SR ? 0x7632 : 0x5410) ^ 0x80008000u,
+                                                                     __byte_perm(c[2], c[3], SR ? 0x7632 : 0x5410) ^ 0x80008000u);
+                if (o.hi) reinterpret_cast<uint32_t *>(o.hi)[j] = (SR ? pack_bytes3(c) : pack_bytes1(c)) ^ 0x80808080u;
+                if (o.lo) reinterpret_cast<uint32_t *>(o.lo)[j] = SR ? pack_bytes2(c) : pack_bytes0(c);
             }
         }
         if (o.rowsum8) {
@@ -453,7 +459,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     }
     if (blockIdx.x == 0 && threadIdx.x == 0)
         for (int64_t i = nv << 2; i < n; ++i)
-            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, key, o);
+            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o);
 }
 
 // Row sums of stored 8-bit codes: a group of G lanes per row (G = smallest power
@@ -582,7 +588,7 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
     if (o.rowsum8 && !vec) return fail(QBP_ERR_INVALID_ARG, "quantize: fused row sums need the vector path");
     const int64_t per_block = (int64_t)kThreads * (vec ? 4 * kUnroll : 1);
     const bool sr = rounding == QBP_ROUND_STOCHASTIC;
-    const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    const PhiloxKeys key = philox_keys_host(seed);
     const int c = (int)cols;
     // per-channel parameter table: 2 x cols x 8 bytes of dynamic shared memory when that stays within 32 KB
     const int smem_cols = (perch && vec && cols <= 2048) ? c : 0;
@@ -711,7 +717,6 @@ static int quantize_any(int bits, const float *x, int64_t rows, int64_t cols, in
 constexpr size_t kStaticScratchBytes = 2 * sizeof(float) * (size_t)kScanMaxStrips * QBP_STATIC_MAX_CHANNELS + 256;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
 static std::mutex g_static_mu;
 static void *g_static_ptr[kMaxDevices] = {};
 

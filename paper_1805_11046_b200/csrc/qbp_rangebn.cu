@@ -81,12 +81,14 @@ __global__ void __launch_bounds__(kScanThreads) bn_stats_kernel(const float *__r
     }
 }
 
-// One block of 128 threads per channel: mean, min, max.
+// One block of 128 threads per channel: mean (or, with sum_out, the raw fp64 sum for a later combination over
+// several GPUs), min, max.
 __global__ void __launch_bounds__(128) bn_stats_finalize_kernel(const float *__restrict__ part_lo,
                                                                 const float *__restrict__ part_hi,
                                                                 const double *__restrict__ part_sum, int nparts, int C,
                                                                 int64_t n, float *__restrict__ mean,
-                                                                float *__restrict__ vmin, float *__restrict__ vmax)
+                                                                float *__restrict__ vmin, float *__restrict__ vmax,
+                                                                double *__restrict__ sum_out)
 {
     const int c = blockIdx.x;
     float lo = INFINITY, hi = -INFINITY;
@@ -105,50 +107,98 @@ __global__ void __launch_bounds__(128) bn_stats_finalize_kernel(const float *__r
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 1; w < 4; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); sum += s_sum[w]; }
-        mean[c] = (float)(sum / (double)n); vmin[c] = lo; vmax[c] = hi;
+        if (mean) mean[c] = (float)(sum / (double)n);
+        if (sum_out) sum_out[c] = sum;
+        vmin[c] = lo; vmax[c] = hi;
     }
 }
 
-template <int VEC, bool RELU>
+// Mean from a (possibly all-reduced) per-channel sum over n rows; min and max are copied alongside.
+__global__ void bn_mean_from_sum_kernel(const double *__restrict__ col_sum, const float *__restrict__ col_min,
+                                        const float *__restrict__ col_max, int C, int64_t n, float *__restrict__ mean,
+                                        float *__restrict__ vmin, float *__restrict__ vmax)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    mean[c] = (float)(col_sum[c] / (double)n);
+    vmin[c] = col_min[c]; vmax[c] = col_max[c];
+}
+
+// Requantisation of the output for the next layer (Section 4: the range of an activation that a Range BN produced
+// is known from its statistics, so quantising it costs no scan): with rq, the 8-bit codes of y (nearest rounding,
+// parameters *rq) are written beside y, or instead of it (y == NULL); rowsum (nullable; rs_group = lanes per row,
+// a power of two <= 32 that covers the row) receives each row's sum of stored codes, which the next product's
+// zero-point correction needs.
+struct BnRequant { const qbp_qparams *rq; int8_t *q; int32_t *rowsum; int rs_group; };
+
+template <int VEC, bool RELU, bool REQUANT>
 __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__restrict__ x, int64_t rows, int C, int tw,
                                                                 const float *__restrict__ mean,
                                                                 const float *__restrict__ vmin,
                                                                 const float *__restrict__ vmax,
                                                                 const float *__restrict__ gamma,
                                                                 const float *__restrict__ beta, float Cn,
-                                                                float *__restrict__ y)
+                                                                float *__restrict__ y, BnRequant R)
 {
     const ScanPos p = scan_pos<VEC>(C, tw);
-    if (!p.active) return;
+    // (with row sums the idle threads of a ragged last slab take part in the shuffles: tw <= 32 then, one slab)
+    if (!p.active && !(REQUANT && R.rowsum)) return;
     const int rpb = kScanThreads / tw;
     float mu[VEC], s[VEC], g[VEC], b[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) {
-        mu[e] = mean[p.col + e];
-        s[e] = bn_scale(vmin[p.col + e], vmax[p.col + e], Cn);
-        g[e] = gamma ? gamma[p.col + e] : 1.0f;
-        b[e] = beta ? beta[p.col + e] : 0.0f;
+        const int c = p.active ? p.col + e : 0;
+        mu[e] = mean[c];
+        s[e] = bn_scale(vmin[c], vmax[c], Cn);
+        g[e] = gamma ? gamma[c] : 1.0f;
+        b[e] = beta ? beta[c] : 0.0f;
     }
+    float inv = 0.0f, zp_u = 0.0f;
+    if (REQUANT) { inv = __fdiv_rn(1.0f, R.rq->scale); zp_u = (float)(R.rq->zero_point + 128); }
     const int64_t step = (int64_t)gridDim.x * rpb;
-    for (int64_t r0 = (int64_t)blockIdx.x * rpb + p.ty; r0 < rows; r0 += step * kScanUnroll) {
+    // (the loop bound is the same for every thread of the block, so that the shuffles below see whole warps)
+    for (int64_t rb = (int64_t)blockIdx.x * rpb; rb < rows; rb += step * kScanUnroll) {
+        const int64_t r0 = rb + p.ty;
         VecF<VEC> v[kScanUnroll];
         bool ok[kScanUnroll];
 #pragma unroll
         for (int u = 0; u < kScanUnroll; ++u) {
             int64_t r = r0 + u * step;
-            ok[u] = r < rows;
+            ok[u] = p.active && r < rows;
             if (ok[u]) v[u].load_stream(x + r * C + p.col);
         }
 #pragma unroll
-        for (int u = 0; u < kScanUnroll; ++u)
+        for (int u = 0; u < kScanUnroll; ++u) {
+            int rs = 0;
             if (ok[u]) {
+                uint32_t code[VEC];
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) {
                     float yv = bn_y(bn_xhat(v[u].v[e], mu[e], s[e]), g[e], b[e]);
                     v[u].v[e] = RELU ? fmaxf(yv, 0.0f) : yv;
+                    if (REQUANT) code[e] = (uint32_t)quantize_code<false>(v[u].v[e], inv, zp_u, 255.0f, 0u);
                 }
-                v[u].store_stream(y + (r0 + u * step) * C + p.col);
+                const int64_t at = (r0 + u * step) * C + p.col;
+                if (y) v[u].store_stream(y + at);
+                if (REQUANT) {
+                    if (VEC == 4) {
+                        const uint32_t packed = (code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24)) ^ 0x80808080u;
+                        *reinterpret_cast<uint32_t *>(R.q + at) = packed;
+                        rs = __dp4a((int)packed, 0x01010101, 0);
+                    } else {
+                        R.q[at] = (int8_t)((int)code[0] - 128);
+                        rs = (int)code[0] - 128;
+                    }
+                }
             }
+            if (REQUANT && R.rowsum) {
+                // a row is rs_group consecutive lanes of one warp (idle lanes add nothing)
+                for (int off = 16; off > 0; off >>= 1)
+                    if (off < R.rs_group) rs += __shfl_xor_sync(0xffffffffu, rs, off);
+                const int64_t r = r0 + u * step;
+                if (p.tx == 0 && r < rows) R.rowsum[r] = rs;
+            }
+        }
     }
 }
 
@@ -159,7 +209,7 @@ __global__ void __launch_bounds__(256) bn_out_range_kernel(const float *__restri
                                                            const float *__restrict__ vmax,
                                                            const float *__restrict__ gamma,
                                                            const float *__restrict__ beta, int C, float Cn, int relu,
-                                                           qbp_qparams *__restrict__ out)
+                                                           qbp_qparams *__restrict__ out, qbp_qparams *__restrict__ qp8_out)
 {
     float lo = INFINITY, hi = -INFINITY;
     for (int c = threadIdx.x; c < C; c += 256) {
@@ -176,7 +226,8 @@ __global__ void __launch_bounds__(256) bn_out_range_kernel(const float *__restri
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 0; w < 8; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); }
-        out->scale = 0.0f; out->zero_point = 0; out->vmin = lo; out->vmax = hi;
+        if (out) { out->scale = 0.0f; out->zero_point = 0; out->vmin = lo; out->vmax = hi; }
+        if (qp8_out) *qp8_out = make_qparams(lo, hi, 8);
     }
 }
 
@@ -255,7 +306,8 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
                                                               const double *__restrict__ part_dyx, int nparts, int C,
                                                               int64_t n, const float *__restrict__ gamma, double Cn,
                                                               float *__restrict__ dgamma, float *__restrict__ dbeta,
-                                                              float2 *__restrict__ coef)
+                                                              float2 *__restrict__ coef, double *__restrict__ sum_dy,
+                                                              double *__restrict__ sum_dyx)
 {
     const int c = blockIdx.x;
     double a = 0.0, b = 0.0;
@@ -273,11 +325,29 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 1; w < 4; ++w) { a += s_a[w]; b += s_b[w]; }
+        if (sum_dy) {                       // raw sums only: combined over several GPUs before the coefficients
+            sum_dy[c] = a; sum_dyx[c] = b;
+            return;
+        }
         const double g = gamma ? (double)gamma[c] : 1.0;
         if (dbeta) dbeta[c] = (float)a;
         if (dgamma) dgamma[c] = (float)b;
         coef[c] = make_float2((float)(g * a / (double)n), (float)(Cn * g * b));
     }
+}
+
+// The same coefficients from per-channel sums that are already complete (n: the rows they were taken over).
+__global__ void bn_bwd_coef_kernel(const double *__restrict__ sum_dy, const double *__restrict__ sum_dyx, int C, int64_t n,
+                                   const float *__restrict__ gamma, double Cn, float *__restrict__ dgamma,
+                                   float *__restrict__ dbeta, float2 *__restrict__ coef)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    const double a = sum_dy[c], b = sum_dyx[c];
+    const double g = gamma ? (double)gamma[c] : 1.0;
+    if (dbeta) dbeta[c] = (float)a;
+    if (dgamma) dgamma[c] = (float)b;
+    coef[c] = make_float2((float)(g * a / (double)n), (float)(Cn * g * b));
 }
 
 // RANGE: also leave the block's (min, max) of the dx values it wrote in range_parts[block], so that the
@@ -381,76 +451,144 @@ extern "C" __attribute__((visibility("default"))) size_t qbp_rangebn_workspace_b
     return bn_ws_bytes(C > 0 ? C : 1);
 }
 
-extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu,
-                               float *y, float *save_mean, float *save_min, float *save_max, qbp_qparams *out_range,
-                               void *ws, size_t ws_bytes, void *stream)
+namespace qbp {
+
+// The apply pass (and what hangs on it) from per-channel mean / min / max that are already in save_*:
+// the exact range of y and the next layer's 8-bit parameters when asked for, y and / or its 8-bit codes.
+// n_stat: the rows the statistics were taken over (more than n_rows when several GPUs share a minibatch).
+static int bn_fwd_apply_launch(const float *x, int64_t n_rows, int64_t n_stat, int64_t C, const float *gamma,
+                               const float *beta, int relu, float *y, const float *save_mean, const float *save_min,
+                               const float *save_max, qbp_qparams *out_range, const qbp_requant *rq, cudaStream_t st)
 {
-    cudaStream_t st = (cudaStream_t)stream;
-    int rc = check_bn("rangebn_fwd", x, y, n, C, ws, ws_bytes);
-    if (rc) return rc;
-    if (!save_mean || !save_min || !save_max) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: NULL statistics buffer");
+    const bool requant = rq != nullptr;
+    if (requant && (!rq->q || !rq->qp)) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: the requantisation record needs q and qp");
+    if (!y && !requant) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: neither y nor 8-bit codes wanted");
+    const bool al = aligned16(x) && (!y || aligned16(y)) && (!requant || ((uintptr_t)rq->q & 3) == 0);
+    const bool v4 = al && C % 4 == 0;
+    const int bps = v4 ? (requant ? (relu ? blocks_per_sm(bn_apply_kernel<4, true, true>, kScanThreads)
+                                          : blocks_per_sm(bn_apply_kernel<4, false, true>, kScanThreads))
+                                  : (relu ? blocks_per_sm(bn_apply_kernel<4, true, false>, kScanThreads)
+                                          : blocks_per_sm(bn_apply_kernel<4, false, false>, kScanThreads)))
+                       : blocks_per_sm(bn_apply_kernel<1, true, true>, kScanThreads);
+    const ScanGeom ga = scan_geom(n_rows, C, al, bps);
+    const dim3 grid_apply(ga.nbx, ga.slabs);
+    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n_stat)));
+    if (out_range || requant) {
+        QBP_TRACE_BEGIN(st);
+        bn_out_range_kernel<<<1, 256, 0, st>>>(save_mean, save_min, save_max, gamma, beta, (int)C, Cn, relu, out_range,
+                                               requant ? rq->qp : nullptr);
+        QBP_LAUNCH_OK("bn_out_range_kernel");
+    }
+    BnRequant R{nullptr, nullptr, nullptr, 1};
+    bool fused_rowsum = false;
+    if (requant) {
+        R.rq = rq->qp; R.q = rq->q;
+        // the row's lanes sit in one warp when the block is at most 32 vectors wide and one slab covers the row
+        fused_rowsum = rq->row_sums && ga.tw <= 32 && ga.slabs == 1;
+        if (fused_rowsum) { R.rowsum = rq->row_sums; R.rs_group = ga.tw; }
+    }
+    QBP_TRACE_BEGIN(st);
+#define QBP_BN_APPLY(V, RL, RQ) bn_apply_kernel<V, RL, RQ><<<grid_apply, kScanThreads, 0, st>>>(x, n_rows, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, y, R)
+    if (ga.vec == 4) {
+        if (requant) { if (relu) QBP_BN_APPLY(4, true, true); else QBP_BN_APPLY(4, false, true); }
+        else         { if (relu) QBP_BN_APPLY(4, true, false); else QBP_BN_APPLY(4, false, false); }
+    } else {
+        if (requant) { if (relu) QBP_BN_APPLY(1, true, true); else QBP_BN_APPLY(1, false, true); }
+        else         { if (relu) QBP_BN_APPLY(1, true, false); else QBP_BN_APPLY(1, false, false); }
+    }
+#undef QBP_BN_APPLY
+    QBP_LAUNCH_OK("bn_apply_kernel");
+    if (requant && rq->row_sums && !fused_rowsum) return launch_rowsum(rq->q, true, n_rows, C, rq->row_sums, st);
+    return QBP_OK;
+}
+
+// The statistics pass: partials per strip, then either mean / min / max (mean != NULL) or the raw sum / min / max.
+static int bn_fwd_stats_launch(const float *x, int64_t n, int64_t C, float *mean, float *vmin, float *vmax, double *sum_out,
+                               void *ws, size_t ws_bytes, cudaStream_t st)
+{
     WsCarver w(ws, ws_bytes);
     double *psum = w.take<double>((size_t)kScanMaxStrips * C);
     w.take<double>((size_t)kScanMaxStrips * C);
     float *plo = w.take<float>((size_t)kScanMaxStrips * C);
     float *phi = w.take<float>((size_t)kScanMaxStrips * C);
-    const bool al = aligned16(x) && aligned16(y);
+    const bool al = aligned16(x);
     const bool v4 = al && C % 4 == 0;
     const ScanGeom g = scan_geom(n, C, al, v4 ? blocks_per_sm(bn_stats_kernel<4>, kScanThreads)
                                               : blocks_per_sm(bn_stats_kernel<1>, kScanThreads));
     const dim3 grid(g.nbx, g.slabs);
-    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_apply_kernel<4, true>, kScanThreads)
-                                                       : blocks_per_sm(bn_apply_kernel<4, false>, kScanThreads))
-                                               : blocks_per_sm(bn_apply_kernel<1, true>, kScanThreads));
-    const dim3 grid_apply(ga.nbx, ga.slabs);
-    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
     QBP_TRACE_BEGIN(st);
     if (g.vec == 4) bn_stats_kernel<4><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
     else            bn_stats_kernel<1><<<grid, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, plo, phi, psum);
     QBP_LAUNCH_OK("bn_stats_kernel");
     QBP_TRACE_BEGIN(st);
-    bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(plo, phi, psum, g.nbx, (int)C, n, save_mean, save_min, save_max);
+    bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(plo, phi, psum, g.nbx, (int)C, n, mean, vmin, vmax, sum_out);
     QBP_LAUNCH_OK("bn_stats_finalize_kernel");
-QBP_TRACE_BEGIN(st);
-#define QBP_BN_APPLY(V, R) bn_apply_kernel<V, R><<<grid_apply, kScanThreads, 0, st>>>(x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, y)
-    if (g.vec == 4) { if (relu) QBP_BN_APPLY(4, true); else QBP_BN_APPLY(4, false); }
-    else            { if (relu) QBP_BN_APPLY(1, true); else QBP_BN_APPLY(1, false); }
-#undef QBP_BN_APPLY
-    QBP_LAUNCH_OK("bn_apply_kernel");
-    if (out_range) {
-        QBP_TRACE_BEGIN(st);
-        bn_out_range_kernel<<<1, 256, 0, st>>>(save_mean, save_min, save_max, gamma, beta, (int)C, Cn, relu, out_range);
-        QBP_LAUNCH_OK("bn_out_range_kernel");
-    }
     return QBP_OK;
+}
+
+}  // namespace qbp
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd_q8(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu,
+                               float *y, float *save_mean, float *save_min, float *save_max, qbp_qparams *out_range,
+                               const qbp_requant *rq, void *ws, size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = check_bn("rangebn_fwd", x, x, n, C, ws, ws_bytes);
+    if (rc) return rc;
+    if (!y && !rq) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: NULL tensor");
+    if (!save_mean || !save_min || !save_max) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: NULL statistics buffer");
+    if ((rc = bn_fwd_stats_launch(x, n, C, save_mean, save_min, save_max, nullptr, ws, ws_bytes, st))) return rc;
+    return bn_fwd_apply_launch(x, n, n, C, gamma, beta, relu, y, save_mean, save_min, save_max, out_range, rq, st);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu,
+                               float *y, float *save_mean, float *save_min, float *save_max, qbp_qparams *out_range,
+                               void *ws, size_t ws_bytes, void *stream)
+{
+    if (!y) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: NULL tensor");
+    return qbp_rangebn_fwd_q8(x, n, C, gamma, beta, relu, y, save_mean, save_min, save_max, out_range, nullptr, ws, ws_bytes, stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd_stats(const float *x, int64_t n, int64_t C, double *col_sum, float *col_min,
+                               float *col_max, void *ws, size_t ws_bytes, void *stream)
+{
+    // (n = 1 is a valid share of a larger minibatch: the n >= 2 rule applies to n_stat of the apply call)
+    if (n < 1 || C <= 0) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd_stats: n and C must be positive");
+    if (!x || !col_sum || !col_min || !col_max) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd_stats: NULL argument");
+    if (!ws || ws_bytes < bn_ws_bytes(C))
+        return fail(QBP_ERR_WORKSPACE, "rangebn_fwd_stats: workspace of %zu bytes needed, %zu given", bn_ws_bytes(C), ws_bytes);
+    return bn_fwd_stats_launch(x, n, C, nullptr, col_min, col_max, col_sum, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd_apply(const float *x, int64_t n_rows, int64_t n_stat, int64_t C, const double *col_sum,
+                               const float *col_min, const float *col_max, const float *gamma, const float *beta, int relu,
+                               float *y, float *save_mean, float *save_min, float *save_max, qbp_qparams *out_range,
+                               const qbp_requant *rq, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n_rows < 1 || n_stat < n_rows || C <= 0) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd_apply: needs 1 <= n_rows <= n_stat, C > 0");
+    if (n_stat < 2) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd_apply: n_stat must be at least 2 (C(1) is infinite)");
+    if (!x || !col_sum || !col_min || !col_max || !save_mean || !save_min || !save_max)
+        return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd_apply: NULL argument");
+    QBP_TRACE_BEGIN(st);
+    bn_mean_from_sum_kernel<<<(int)((C + 255) / 256), 256, 0, st>>>(col_sum, col_min, col_max, (int)C, n_stat, save_mean, save_min, save_max);
+    QBP_LAUNCH_OK("bn_mean_from_sum_kernel");
+    return bn_fwd_apply_launch(x, n_rows, n_stat, C, gamma, beta, relu, y, save_mean, save_min, save_max, out_range, rq, st);
 }
 
 // Forward from per-column partials of x that its producer left (rows of [C]: sum, min, max), without a statistics
 // pass over x: finalize, then the apply pass.
 int qbp::rangebn_fwd_from_parts(const float *x, int64_t n, int64_t C, const float *gamma, const float *beta, int relu,
                                 float *y, float *save_mean, float *save_min, float *save_max, const ColStatParts &parts,
-                                cudaStream_t st)
+                                qbp_qparams *out_range, const qbp_requant *rq, cudaStream_t st)
 {
-    if (!x || !y || !save_mean || !save_min || !save_max || !parts.lo || !parts.hi || !parts.sum || parts.rows <= 0)
+    if (!x || !save_mean || !save_min || !save_max || !parts.lo || !parts.hi || !parts.sum || parts.rows <= 0)
         return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: NULL tensor");
     if (n < 2 || C <= 0) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: needs n >= 2 rows");
-    const bool al = aligned16(x) && aligned16(y);
-    const bool v4 = al && C % 4 == 0;
-    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_apply_kernel<4, true>, kScanThreads)
-                                                       : blocks_per_sm(bn_apply_kernel<4, false>, kScanThreads))
-                                               : blocks_per_sm(bn_apply_kernel<1, true>, kScanThreads));
-    const dim3 grid_apply(ga.nbx, ga.slabs);
-    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
     QBP_TRACE_BEGIN(st);
-    bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(parts.lo, parts.hi, parts.sum, parts.rows, (int)C, n, save_mean, save_min, save_max);
+    bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(parts.lo, parts.hi, parts.sum, parts.rows, (int)C, n, save_mean, save_min, save_max, nullptr);
     QBP_LAUNCH_OK("bn_stats_finalize_kernel");
-    QBP_TRACE_BEGIN(st);
-#define QBP_BN_APPLY(V, R) bn_apply_kernel<V, R><<<grid_apply, kScanThreads, 0, st>>>(x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, y)
-    if (ga.vec == 4) { if (relu) QBP_BN_APPLY(4, true); else QBP_BN_APPLY(4, false); }
-    else             { if (relu) QBP_BN_APPLY(1, true); else QBP_BN_APPLY(1, false); }
-#undef QBP_BN_APPLY
-    QBP_LAUNCH_OK("bn_apply_kernel");
-    return QBP_OK;
+    return bn_fwd_apply_launch(x, n, n, C, gamma, beta, relu, y, save_mean, save_min, save_max, out_range, rq, st);
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma,
@@ -461,6 +599,62 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const floa
     return rangebn_bwd_impl(dy, x, n, C, gamma, beta, relu, save_mean, save_min, save_max, dx, dgamma, dbeta, ws, ws_bytes,
                             nullptr, nullptr, (cudaStream_t)stream);
 }
+
+namespace qbp {
+
+static int bn_bwd_stats_launch(const float *dy, const float *x, int64_t n_rows, int64_t n_stat, int64_t C, const float *gamma,
+                               const float *beta, int relu, const float *save_mean, const float *save_min,
+                               const float *save_max, float *dgamma, float *dbeta, float2 *coef, double *sum_dy,
+                               double *sum_dyx, double *pa, double *pb, cudaStream_t st)
+{
+    const bool al = aligned16(x) && aligned16(dy);
+    const bool v4 = al && C % 4 == 0;
+    const ScanGeom g = scan_geom(n_rows, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_stats_kernel<4, true>, kScanThreads)
+                                                           : blocks_per_sm(bn_bwd_stats_kernel<4, false>, kScanThreads))
+                                                   : blocks_per_sm(bn_bwd_stats_kernel<1, true>, kScanThreads));
+    const dim3 grid(g.nbx, g.slabs);
+    const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n_stat));
+    const float Cn = (float)Cnd;
+    QBP_TRACE_BEGIN(st);
+#define QBP_BN_BSTATS(V, R) bn_bwd_stats_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n_rows, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, pa, pb)
+    if (g.vec == 4) { if (relu) QBP_BN_BSTATS(4, true); else QBP_BN_BSTATS(4, false); }
+    else            { if (relu) QBP_BN_BSTATS(1, true); else QBP_BN_BSTATS(1, false); }
+#undef QBP_BN_BSTATS
+    QBP_LAUNCH_OK("bn_bwd_stats_kernel");
+    QBP_TRACE_BEGIN(st);
+    bn_bwd_finalize_kernel<<<(int)C, 128, 0, st>>>(pa, pb, g.nbx, (int)C, n_stat, gamma, Cnd, dgamma, dbeta, coef, sum_dy, sum_dyx);
+    QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
+    return QBP_OK;
+}
+
+static int bn_bwd_apply_launch(const float *dy, const float *x, int64_t n_rows, int64_t n_stat, int64_t C, const float *gamma,
+                               const float *beta, int relu, const float *save_mean, const float *save_min,
+                               const float *save_max, const float2 *coef, float *dx, float2 *range_parts, int *nparts,
+                               cudaStream_t st)
+{
+    const bool al = aligned16(x) && aligned16(dy) && aligned16(dx);
+    const bool v4 = al && C % 4 == 0;
+    const ScanGeom ga = scan_geom(n_rows, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_apply_kernel<4, true, true>, kScanThreads)
+                                                            : blocks_per_sm(bn_bwd_apply_kernel<4, false, true>, kScanThreads))
+                                                    : blocks_per_sm(bn_bwd_apply_kernel<1, true, true>, kScanThreads));
+    const dim3 grid_apply(ga.nbx, ga.slabs);
+    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n_stat)));
+    QBP_TRACE_BEGIN(st);
+#define QBP_BN_BAPPLY(V, R, G) bn_bwd_apply_kernel<V, R, G><<<grid_apply, kScanThreads, 0, st>>>(dy, x, n_rows, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx, range_parts)
+    if (range_parts) {
+        if (ga.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true, true); else QBP_BN_BAPPLY(4, false, true); }
+        else             { if (relu) QBP_BN_BAPPLY(1, true, true); else QBP_BN_BAPPLY(1, false, true); }
+        if (nparts) *nparts = (int)(grid_apply.x * grid_apply.y);
+    } else {
+        if (ga.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true, false); else QBP_BN_BAPPLY(4, false, false); }
+        else             { if (relu) QBP_BN_BAPPLY(1, true, false); else QBP_BN_BAPPLY(1, false, false); }
+    }
+#undef QBP_BN_BAPPLY
+    QBP_LAUNCH_OK("bn_bwd_apply_kernel");
+    return QBP_OK;
+}
+
+}  // namespace qbp
 
 // range_parts (nullable, room for rangebn_range_parts_capacity(C) entries) receives one (min, max) of dx per
 // block of the apply pass; *nparts their count.
@@ -478,38 +672,52 @@ int qbp::rangebn_bwd_impl(const float *dy, const float *x, int64_t n, int64_t C,
     w.take<float>((size_t)kScanMaxStrips * C);
     w.take<float>((size_t)kScanMaxStrips * C);
     float2 *coef = w.take<float2>((size_t)C);
-    const bool al = aligned16(x) && aligned16(dy) && aligned16(dx);
-    const bool v4 = al && C % 4 == 0;
-    const ScanGeom g = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_stats_kernel<4, true>, kScanThreads)
-                                                      : blocks_per_sm(bn_bwd_stats_kernel<4, false>, kScanThreads))
-                                              : blocks_per_sm(bn_bwd_stats_kernel<1, true>, kScanThreads));
-    const dim3 grid(g.nbx, g.slabs);
-    const ScanGeom ga = scan_geom(n, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_apply_kernel<4, true, true>, kScanThreads)
-                                                       : blocks_per_sm(bn_bwd_apply_kernel<4, false, true>, kScanThreads))
-                                               : blocks_per_sm(bn_bwd_apply_kernel<1, true, true>, kScanThreads));
-    const dim3 grid_apply(ga.nbx, ga.slabs);
-    const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n));
-    const float Cn = (float)Cnd;
-QBP_TRACE_BEGIN(st);
-#define QBP_BN_BSTATS(V, R) bn_bwd_stats_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, pa, pb)
-    if (g.vec == 4) { if (relu) QBP_BN_BSTATS(4, true); else QBP_BN_BSTATS(4, false); }
-    else            { if (relu) QBP_BN_BSTATS(1, true); else QBP_BN_BSTATS(1, false); }
-#undef QBP_BN_BSTATS
-    QBP_LAUNCH_OK("bn_bwd_stats_kernel");
+    if ((rc = bn_bwd_stats_launch(dy, x, n, n, C, gamma, beta, relu, save_mean, save_min, save_max, dgamma, dbeta, coef,
+                                  nullptr, nullptr, pa, pb, st)))
+        return rc;
+    return bn_bwd_apply_launch(dy, x, n, n, C, gamma, beta, relu, save_mean, save_min, save_max, coef, dx, range_parts, nparts, st);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd_stats(const float *dy, const float *x, int64_t n_rows, int64_t n_stat, int64_t C,
+                               const float *gamma, const float *beta, int relu, const float *save_mean,
+                               const float *save_min, const float *save_max, double *sum_dy, double *sum_dyxhat,
+                               void *ws, size_t ws_bytes, void *stream)
+{
+    if (n_rows < 1 || n_stat < n_rows || n_stat < 2 || C <= 0)
+        return fail(QBP_ERR_INVALID_ARG, "rangebn_bwd_stats: needs 1 <= n_rows <= n_stat, n_stat >= 2, C > 0");
+    if (!dy || !x || !save_mean || !save_min || !save_max || !sum_dy || !sum_dyxhat)
+        return fail(QBP_ERR_INVALID_ARG, "rangebn_bwd_stats: NULL argument");
+    if (!ws || ws_bytes < bn_ws_bytes(C))
+        return fail(QBP_ERR_WORKSPACE, "rangebn_bwd_stats: workspace of %zu bytes needed, %zu given", bn_ws_bytes(C), ws_bytes);
+    WsCarver w(ws, ws_bytes);
+    double *pa = w.take<double>((size_t)kScanMaxStrips * C);
+    double *pb = w.take<double>((size_t)kScanMaxStrips * C);
+    return bn_bwd_stats_launch(dy, x, n_rows, n_stat, C, gamma, beta, relu, save_mean, save_min, save_max, nullptr, nullptr,
+                               nullptr, sum_dy, sum_dyxhat, pa, pb, (cudaStream_t)stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd_apply(const float *dy, const float *x, int64_t n_rows, int64_t n_stat, int64_t C,
+                               const float *gamma, const float *beta, int relu, const float *save_mean,
+                               const float *save_min, const float *save_max, const double *sum_dy,
+                               const double *sum_dyxhat, float *dx, float *dgamma, float *dbeta, void *ws,
+                               size_t ws_bytes, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n_rows < 1 || n_stat < n_rows || n_stat < 2 || C <= 0)
+        return fail(QBP_ERR_INVALID_ARG, "rangebn_bwd_apply: needs 1 <= n_rows <= n_stat, n_stat >= 2, C > 0");
+    if (!dy || !x || !dx || !save_mean || !save_min || !save_max || !sum_dy || !sum_dyxhat)
+        return fail(QBP_ERR_INVALID_ARG, "rangebn_bwd_apply: NULL argument");
+    if (!ws || ws_bytes < bn_ws_bytes(C))
+        return fail(QBP_ERR_WORKSPACE, "rangebn_bwd_apply: workspace of %zu bytes needed, %zu given", bn_ws_bytes(C), ws_bytes);
+    WsCarver w(ws, ws_bytes);
+    w.take<double>((size_t)kScanMaxStrips * C);
+    w.take<double>((size_t)kScanMaxStrips * C);
+    w.take<float>((size_t)kScanMaxStrips * C);
+    w.take<float>((size_t)kScanMaxStrips * C);
+    float2 *coef = w.take<float2>((size_t)C);
+    const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n_stat));
     QBP_TRACE_BEGIN(st);
-    bn_bwd_finalize_kernel<<<(int)C, 128, 0, st>>>(pa, pb, g.nbx, (int)C, n, gamma, Cnd, dgamma, dbeta, coef);
-    QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
-QBP_TRACE_BEGIN(st);
-#define QBP_BN_BAPPLY(V, R, G) bn_bwd_apply_kernel<V, R, G><<<grid_apply, kScanThreads, 0, st>>>(dy, x, n, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, dx, range_parts)
-    if (range_parts) {
-        if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true, true); else QBP_BN_BAPPLY(4, false, true); }
-        else            { if (relu) QBP_BN_BAPPLY(1, true, true); else QBP_BN_BAPPLY(1, false, true); }
-        if (nparts) *nparts = (int)(grid_apply.x * grid_apply.y);
-    } else {
-        if (g.vec == 4) { if (relu) QBP_BN_BAPPLY(4, true, false); else QBP_BN_BAPPLY(4, false, false); }
-        else            { if (relu) QBP_BN_BAPPLY(1, true, false); else QBP_BN_BAPPLY(1, false, false); }
-    }
-#undef QBP_BN_BAPPLY
-    QBP_LAUNCH_OK("bn_bwd_apply_kernel");
-    return QBP_OK;
+    bn_bwd_coef_kernel<<<(int)((C + 255) / 256), 256, 0, st>>>(sum_dy, sum_dyxhat, (int)C, n_stat, gamma, Cnd, dgamma, dbeta, coef);
+    QBP_LAUNCH_OK("bn_bwd_coef_kernel");
+    return bn_bwd_apply_launch(dy, x, n_rows, n_stat, C, gamma, beta, relu, save_mean, save_min, save_max, coef, dx, nullptr, nullptr, st);
 }

@@ -37,10 +37,7 @@
 namespace qbp {
 
 constexpr int kWgThreads = 192;
-#ifndef QBP_WG_FIN_LANES
-#define QBP_WG_FIN_LANES 4
-#endif
-constexpr int kWgFinalizeLanes = QBP_WG_FIN_LANES;   // lanes of the second kernel that share one output element's partials
+constexpr int kWgFinalizeLanes = 4;   // lanes of the second kernel that share one output element's partials
 constexpr int kWgRows = 128;         // reduction rows per pipeline stage: four k steps of 32 (what the MMA warp does
                                      // between stages is a fixed cost, so a stage should hold many MMAs)
 constexpr int kWgMaxStages = 16;
@@ -339,7 +336,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     }
 
     if (timed_out) {
-        atomicExch(P.status, (int)QBP_ERR_TIMEOUT);
+        raise_timeout(P.status);
         __nanosleep(1000000);
     }
     tc_fence_before();
@@ -615,7 +612,7 @@ static void pick_pixel_box_w(int rows, int Nimg, int H, int W, int &bwl, int &bh
         }
 }
 
-static bool wgrad_conv_supported(const qbp_conv_desc *d)
+bool wgrad_conv_supported(const qbp_conv_desc *d)
 {
     return d->stride == 1 && d->R == d->S && (d->R == 1 || d->R == 3) && d->pad == (d->R - 1) / 2 && d->N > 0 &&
            d->H > 0 && d->W > 0 && d->C > 0 && d->K > 0 && d->C % 32 == 0 && d->K % 32 == 0;
@@ -734,11 +731,8 @@ static int launch_class_sums(const void *q, int64_t pixels, int H, int W, int C,
     QBP_CUDA_OK(cudaMemsetAsync(sums, 0, sizeof(int64_t) * 16 * C, st));
     if ((size_t)C * 16 * sizeof(int) > 200 * 1024) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad: more than 3200 channels");
     const size_t smem = (size_t)C * 16 * sizeof(int);
-    static thread_local bool configured[2] = {false, false};
-    if (smem > 48 * 1024 && !configured[IS_SIGNED]) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(class_sums_kernel<IS_SIGNED>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        configured[IS_SIGNED] = true;
-    }
+    static PerDeviceOnce configured;
+    if (smem > 48 * 1024) QBP_SMEM_OPT_IN(configured, class_sums_kernel<IS_SIGNED>, 200 * 1024);
     if (pixels >= (1ll << 30)) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "wgrad: more than 2^30 positions");
     if (W <= 256) {
         // a block step is one image row: W columns x gs channel groups of 16
@@ -788,7 +782,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
                                                                    const qbp_qparams *qg16, int64_t *acc_out, float *dW,
                                                                    void *ws, size_t ws_bytes, void *stream)
 {
-    cudaStream_t st = (cudaStream_t)stream;
+    return wgrad_s16_impl(d, M, N, K, x, qx, g_hi, g_lo, qg16, acc_out, dW, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
+                        const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
+                        int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st)
+{
     if (!x || !g_hi || !g_lo || !qx || !qg16) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: NULL operand");
     if (!acc_out && !dW) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: acc_out and dW are both NULL");
     if (!aligned16(x) || !aligned16(g_hi) || !aligned16(g_lo))
@@ -813,6 +813,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
     const int64_t outs = d ? (int64_t)d->K * d->R * d->S * d->C : K * N;
     WsCarver w(ws, ws_bytes);
     int *status = w.take<int>(1);
+    if (ext_status) status = ext_status;         // the caller's sticky word: raised here, never cleared
     int64_t *sx = w.take<int64_t>(16 * K);
     int64_t *shi = w.take<int64_t>(16 * N);
     int64_t *slo = w.take<int64_t>(16 * N);
@@ -854,7 +855,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
             QBP_LAUNCH_OK("wgrad_terms_kernel");
         }
     }
-    QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
+    if (!ext_status) QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
 
     P.part = (long long *)part; P.status = status;
     P.rowterm = (const long long *)rowterm; P.colterm = (const long long *)colterm;
@@ -883,11 +884,8 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
     case 7: kernel = qbp_wgrad_kernel<32, 64>; break;
     default: kernel = qbp_wgrad_kernel<32, 32>; break;
     }
-    static thread_local bool configured[9] = {};
-    if (!configured[layout_id]) {
-        QBP_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgSmem));
-        configured[layout_id] = true;
-    }
+    static PerDeviceOnce configured[9];
+    QBP_SMEM_OPT_IN(configured[layout_id], kernel, kWgSmem);
     QBP_TRACE_BEGIN(st);
     kernel<<<pl.grid, kWgThreads, pl.smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_wgrad_kernel");

@@ -14,7 +14,12 @@ class QuantizedLayer:
     layer y = x w with x [batch, in_features], w [in_features, out_features]."""
 
     def __init__(self, conv=None, batch=0, in_features=0, out_features=0, relu=False, seed=0,
-                 tensor_id8=1, tensor_id16=2, device="cuda"):
+                 tensor_id8=1, tensor_id16=2, device="cuda", input_from: "QuantizedLayer | None" = None,
+                 emit_codes=False, keep_y=True):
+        """input_from: the layer whose output feeds this one already quantised (it must have been built with
+        emit_codes=True): this layer then owns no input codes of its own and its forward takes no fp32 input.
+        emit_codes: the forward also writes the 8-bit codes of the output (and each row's code sum) for the next
+        layer; keep_y=False then leaves the fp32 output unwritten."""
         self.device = torch.device(device)
         d = B.LayerDesc()
         if conv is not None:
@@ -31,12 +36,25 @@ class QuantizedLayer:
         self.desc = d
         dev = self.device
         e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
-        self.x_codes, self.w_codes = e(self.x_shape, torch.int8), e(self.w_shape, torch.int8)
-        self.qx, self.qw, self.qg8, self.qg16 = (B.new_qparams(1, dev) for _ in range(4))
+        self.w_codes = e(self.w_shape, torch.int8)
+        self.qw, self.qg8, self.qg16 = (B.new_qparams(1, dev) for _ in range(3))
+        self.rq_in = None
+        if input_from is not None:
+            assert input_from.rq_out is not None and input_from.z_shape == self.x_shape
+            self.x_codes, self.qx = input_from.out_codes, input_from.q_out
+            self.rq_in = input_from.rq_out
+        else:
+            self.x_codes, self.qx = e(self.x_shape, torch.int8), B.new_qparams(1, dev)
+        self.rq_out = None
+        if emit_codes:
+            self.out_codes, self.q_out = e(self.z_shape, torch.int8), B.new_qparams(1, dev)
+            self.out_row_sums = e((self.rows,), torch.int32)
+            self.rq_out = B.requant(self.out_codes, self.q_out, self.out_row_sums)
         self.z, self.g = e(self.z_shape, torch.float32), e(self.z_shape, torch.float32)
         self.save_mean, self.save_min, self.save_max = (e((self.cout,), torch.float32) for _ in range(3))
         self.g8, self.ghi, self.glo = e(self.z_shape, torch.int8), e(self.z_shape, torch.int8), e(self.z_shape, torch.uint8)
-        self.y = e(self.z_shape, torch.float32)
+        assert keep_y or emit_codes
+        self.y = e(self.z_shape, torch.float32) if keep_y else None
         self.dx, self.dw = e(self.x_shape, torch.float32), e(self.w_shape, torch.float32)
         self.dgamma, self.dbeta = e((self.cout,), torch.float32), e((self.cout,), torch.float32)
         self.ws = torch.empty(max(B.qbp_layer_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)
@@ -50,8 +68,12 @@ class QuantizedLayer:
         self.gamma = self.beta = None
 
     def forward(self, x, w, gamma=None, beta=None):
+        """x: the fp32 input, or None for a layer built with input_from (its input codes are already there)."""
         self.gamma, self.beta = gamma, beta
-        return B.qbp_layer_fwd(self.desc, x, w, gamma, beta, self.y, self.ctx, self.ws)
+        assert (x is None) == (self.rq_in is not None)
+        if self.rq_in is None and self.rq_out is None:
+            return B.qbp_layer_fwd(self.desc, x, w, gamma, beta, self.y, self.ctx, self.ws)
+        return B.qbp_layer_fwd_chained(self.desc, x, self.rq_in, w, gamma, beta, self.y, self.rq_out, self.ctx, self.ws)
 
     def backward(self, dy):
         return B.qbp_layer_bwd(self.desc, self.ctx, dy, self.gamma, self.beta, self.dx, self.dw, self.dgamma,

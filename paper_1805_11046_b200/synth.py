@@ -70,7 +70,7 @@ def linear_layer(batch: int = 64, k_in: int = 256, n_out: int = 128):
     return dict(x=normal((batch, k_in), 1),
                 w=kaiming_uniform_linear(k_in, n_out, 2),
                 dy=normal((batch, n_out), 3, std=0.1),
-                seed=0, id8=1, id16=2)
+                seed=0, id8=1, id16=1)      # one tensor id for the gradient: both copies draw from its stream
 
 
 def conv3x3_layer(batch: int = 256, hw: int = 56, c_in: int = 64, k_out: int = 64):
@@ -80,7 +80,7 @@ def conv3x3_layer(batch: int = 256, hw: int = 56, c_in: int = 64, k_out: int = 6
                 w=kaiming_normal((k_out, 3, 3, c_in), 11),
                 dy=normal((batch, hw, hw, k_out), 12, std=0.1),
                 conv=dict(N=batch, H=hw, W=hw, C=c_in, K=k_out, R=3, S=3, stride=1, pad=1),
-                seed=0, id8=1, id16=2)
+                seed=0, id8=1, id16=1)
 
 
 RANGEBN_SWEEP = ((56, 64), (28, 128), (14, 256), (7, 512), (7, 2048))
@@ -106,8 +106,9 @@ def bottleneck_stack(batch: int = 256, hw: int = 28):
                 convs=convs, seed=0)
 
 
-def dense_gemm(M: int, N: int, K: int):
+def dense_gemm(M: int, N: int, K: int, parts=("a", "b", "x", "g")):
     """Dense sweep operands: A [M,K], B [K,N] ~ N(0,1); for the weight-gradient
-    product X [M,K] (8-bit side) and G [M,N] (16-bit side), reduced over M."""
-    return dict(a=normal((M, K), 40), b=normal((K, N), 41),
-                x=normal((M, K), 42), g=normal((M, N), 43))
+    product X [M,K] (8-bit side) and G [M,N] (16-bit side), reduced over M.
+    parts: which of the four to generate (each is up to 1 GB at 16384^2)."""
+    shapes = dict(a=((M, K), 40), b=((K, N), 41), x=((M, K), 42), g=((M, N), 43))
+    return {k: normal(*shapes[k]) for k in parts}

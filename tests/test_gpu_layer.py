@@ -141,3 +141,116 @@ def test_bottleneck_stack_full_batch_stagewise(B):
         cfg = dict(x=a, w=w, dy=synth.normal((c["N"], c["H"], c["W"], c["K"]), 60 + i, std=0.1), seed=0, id8=2 * i + 1, id16=2 * i + 2)
         a = _check_layer(B, cfg, True, c, _sampler(13 + i), want_y=True)
     assert a.shape == (256, 28, 28, 512) and a.min() == 0.0
+
+
+# ------------------------------------------------ chained layers: the quantiser's range from the Range BN before it
+def test_rangebn_fused_requantisation_equals_quantising_the_output(B):
+    """Section 4: the range of a Range BN output is known from the statistics, so its 8-bit codes are written by the
+    apply pass itself.  They must be, bit for bit, what the quantiser makes of the materialised fp32 output (range
+    scan included), the row sums must be the sums of those codes, and leaving y unwritten must not change them."""
+    for shape, relu in (((4, 14, 14, 64), True), ((3, 5, 7, 48), False), ((64, 128), True), ((2, 9, 9, 256), True),
+                        ((5, 3, 3, 6), False), ((1000, 512), True)):
+        x = synth.channel_gaussian(shape, 20, 21)
+        C_ = shape[-1]
+        gamma = synth.uniform((C_,), 23, 1.0) + np.float32(1.5); beta = synth.uniform((C_,), 24, 0.5)
+        gamma[::3] *= -1
+        y, mean, vmin, vmax, q, qp, rs = B.qbp_rangebn_fwd_q8(to_dev(x), to_dev(gamma), to_dev(beta), relu, want_row_sums=True)
+        yh = to_host(y)
+        o = O.quantize(yh, 8)                        # scans yh for its range
+        s_, z_, lo_, hi_ = B.read_qparams(qp)
+        assert s_[0] == o.scale[0] and z_[0] == o.zero_point[0] and lo_[0] == o.vmin[0] and hi_[0] == o.vmax[0]
+        assert np.array_equal(to_host(q), o.q)
+        assert np.array_equal(to_host(rs), o.q.reshape(-1, C_).astype(np.int32).sum(1))
+        _, _, _, _, q2, qp2, _ = B.qbp_rangebn_fwd_q8(to_dev(x), to_dev(gamma), to_dev(beta), relu, want_y=False)
+        assert np.array_equal(to_host(q2), o.q) and np.array_equal(to_host(qp2), to_host(qp))
+
+
+def _chained_stack(B, batch, keep_y):
+    import torch
+    from paper_1805_11046_b200 import layer
+    st = synth.bottleneck_stack(batch=batch, hw=28)
+    layers = []
+    for i, c in enumerate(st["convs"]):
+        conv = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+        last = i == len(st["convs"]) - 1
+        layers.append(layer.QuantizedLayer(conv=conv, relu=True, seed=0, tensor_id8=2 * i + 1, tensor_id16=2 * i + 2,
+                                           input_from=layers[-1] if layers else None, emit_codes=not last,
+                                           keep_y=keep_y or last))
+    ws = [to_dev(w) for w in st["w"]]
+    layers[0].forward(to_dev(st["x"]), ws[0])
+    for L, w in zip(layers[1:], ws[1:]):
+        L.forward(None, w)
+    torch.cuda.synchronize()
+    return st, layers
+
+
+@pytest.mark.parametrize("batch", [8, 256])
+def test_chained_bottleneck_stack_needs_no_scan_between_layers(B, batch):
+    """The conv3_x bottleneck with every inner activation handed on as 8-bit codes written by the Range BN that made
+    it: stage-wise parity (each stage of the oracle is fed what the GPU produced for it), no range scan and no
+    quantisation pass between the layers, and the same results whether or not the fp32 activations are kept."""
+    st, layers = _chained_stack(B, batch, keep_y=True)
+    rng = np.random.Generator(np.random.PCG64(40 + batch))
+    codes_in = None
+    for i, (L, c) in enumerate(zip(layers, st["convs"])):
+        od = O.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+        ow = O.quantize(st["w"][i], 8)
+        if i == 0:
+            ox = O.quantize(st["x"], 8)
+            assert np.array_equal(to_host(L.x_codes), ox.q)
+            xq, xz, xs = ox.q, ox.zero_point[0], ox.scale[0]
+        else:
+            xq, xz, xs = codes_in
+            assert np.array_equal(to_host(L.x_codes), xq)        # the very buffer the previous layer wrote
+        z = to_host(L.z)
+        idx = np.unique(np.concatenate([[0, z.size - 1], rng.integers(0, z.size, 4096)])).astype(np.int64)
+        _, oz, bad = O.conv_s8(0, od, xq, xz, ow.q, ow.zero_point[0], xs, ow.scale[0], idx=idx)
+        assert bad == 0 and np.array_equal(z.ravel()[idx], oz)
+        Cc = z.shape[-1]
+        chans = sorted({0, Cc // 2, Cc - 1})
+        oy, _, _, _ = O.rangebn_fwd(np.ascontiguousarray(z.reshape(-1, Cc)[:, chans]), relu=True)
+        yh = to_host(L.y)
+        assert rel_err(yh.reshape(-1, Cc)[:, chans], oy)[0] <= FP32_TOL
+        if L.rq_out is not None:
+            o = O.quantize(yh, 8)
+            s_, z_, lo_, hi_ = B.read_qparams(L.q_out)
+            assert s_[0] == o.scale[0] and z_[0] == o.zero_point[0] and lo_[0] == o.vmin[0] and hi_[0] == o.vmax[0]
+            assert np.array_equal(to_host(L.out_codes), o.q)
+            assert np.array_equal(to_host(L.out_row_sums), o.q.reshape(-1, Cc).astype(np.int32).sum(1))
+            codes_in = (o.q, o.zero_point[0], o.scale[0])
+        assert L.status() == 0
+    # the same stack without the inner fp32 activations
+    _, lean = _chained_stack(B, batch, keep_y=False)
+    for L, M in zip(layers, lean):
+        assert np.array_equal(to_host(L.z), to_host(M.z))
+        if L.rq_out is not None:
+            assert np.array_equal(to_host(L.out_codes), to_host(M.out_codes))
+    assert np.array_equal(to_host(layers[-1].y), to_host(lean[-1].y))
+    # and the launch list of a chained inner layer holds no scan and no stand-alone quantiser for its input
+    import torch
+    B.trace_enable(True)
+    lean[1].forward(None, to_dev(st["w"][1]))
+    names = [n for n, _ in B.trace_records()]
+    B.trace_enable(False)
+    assert names.count("range_partial_kernel") == 1 and names.count("quantize_kernel") == 1      # the filter's only
+
+
+def test_chained_stack_backward_runs_on_the_handed_on_codes(B):
+    """Backward through a chained pair: the weight gradient of the second layer uses the codes the first layer's
+    Range BN wrote; stage-wise parity of its products."""
+    import torch
+    st, layers = _chained_stack(B, 8, keep_y=True)
+    L = layers[1]; c = st["convs"][1]
+    dy = synth.normal(L.z_shape, 70, std=0.1)
+    dx, dw, _, _ = L.backward(to_dev(dy))
+    torch.cuda.synchronize()
+    assert L.status() == 0
+    od = O.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    g = to_host(L.g)
+    g8, g16 = O.bifurcate(g, 0, 3, 4)
+    assert np.array_equal(to_host(L.g8), g8.q)
+    ow = O.quantize(st["w"][1], 8)
+    xq = to_host(L.x_codes); s_, z_, _, _ = B.read_qparams(L.qx)
+    _, odx, bad = O.conv_s8(1, od, g8.q, g8.zero_point[0], ow.q, ow.zero_point[0], g8.scale[0], ow.scale[0])
+    _, odw = O.conv_wgrad_s16(od, xq, z_[0], g16.q, g16.zero_point[0], np.float32(s_[0]), g16.scale[0])
+    assert bad == 0 and np.array_equal(to_host(dx), odx) and np.array_equal(to_host(dw), odw)

@@ -78,6 +78,68 @@ def test_gemm_dense_sweep_8192_sampled_rows_and_corner_tiles(B):
     assert np.array_equal(to_host(acc[rows]), oacc) and np.array_equal(to_host(out[rows]), oout)
 
 
+def _dense_gemm_sampled(B, M, N, K, seed, n_random=64):
+    """One product of the dense sweep in the benchmark's launch configuration: operands quantised from N(0,1) on both
+    sides (codes compared in full), accumulators and fp32 outputs compared on the rows at the tile edges plus
+    n_random random rows, every column."""
+    case = synth.dense_gemm(M, N, K, parts=("a", "b"))
+    qa, qpa = B.qbp_quantize_s8(to_dev(case["a"])); qb, qpb = B.qbp_quantize_s8(to_dev(case["b"]))
+    oa = O.quantize(case["a"], 8); ob = O.quantize(case["b"], 8)
+    del case
+    assert np.array_equal(to_host(qa), oa.q) and np.array_equal(to_host(qb), ob.q)
+    acc, out, ws = B.qbp_gemm_s8(qa, qpa, qb, qpb, want_acc=True)
+    assert B.status_word(ws) == 0
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, 511, 512, M - 512, M - 257, M - 256, M - 129, M - 128, M - 1],
+                                     np.random.Generator(np.random.PCG64(seed)).integers(0, M, n_random)]))
+    oacc, oout, bad = O.gemm_s8(oa.q[rows], oa.zero_point[0], ob.q, ob.zero_point[0], oa.scale[0], ob.scale[0])
+    assert bad == 0
+    assert np.array_equal(to_host(acc[rows]), oacc) and np.array_equal(to_host(out[rows]), oout)
+
+
+def test_gemm_dense_sweep_16384_sampled_rows(B):
+    """The largest cube of the dense sweep (16384^3, 512 x 256 pair tiles, 32 x 64 of them over 74 CTA pairs)."""
+    _dense_gemm_sampled(B, 16384, 16384, 16384, 8, n_random=32)
+
+
+# (M, N, K) combinations of the sweep that are not cubes: tall, wide, deep and shallow ones
+NONCUBE = [(4096, 16384, 8192), (16384, 4096, 4096), (8192, 4096, 16384), (4096, 8192, 16384)]
+
+
+@pytest.mark.parametrize("M,N,K", NONCUBE)
+def test_gemm_dense_sweep_noncube_sampled_rows(B, M, N, K):
+    _dense_gemm_sampled(B, M, N, K, 9 + M // 4096 + N // 2048, n_random=48)
+
+
+def _dense_wgrad_sampled(B, M, N, K, seed, n_cols):
+    """The limb-split 16 x 8-bit product dW [K x N] = X [M x K]^T G [M x N] of the dense sweep: operands quantised from
+    N(0,1) (nearest for the 8-bit side, stochastic for the 16-bit side, codes compared in full); int64
+    accumulators and fp32 outputs compared on the output columns at the tile edges plus random ones, every row."""
+    case = synth.dense_gemm(M, N, K, parts=("x", "g"))
+    qx, qpx = B.qbp_quantize_s8(to_dev(case["x"]))
+    q16, hi, lo, qpg = B.qbp_quantize_s16(to_dev(case["g"]), rounding=B.QBP_ROUND_STOCHASTIC, seed=3, tensor_id=7)
+    ox = O.quantize(case["x"], 8); og = O.quantize(case["g"], 16, rounding=1, seed=3, tensor_id=7)
+    del case
+    assert np.array_equal(to_host(qx), ox.q) and np.array_equal(to_host(q16), og.q)
+    del q16
+    acc, dW, ws = B.qbp_wgrad_s16(qx, qpx, hi, lo, qpg, want_acc=True)
+    assert B.status_word(ws) == 0
+    cols = np.unique(np.concatenate([[0, 127, 128, N - 129, N - 128, N - 1],
+                                     np.random.Generator(np.random.PCG64(seed)).integers(0, N, n_cols)]))
+    oacc, oout = O.gemm_s16s8(ox.q, ox.zero_point[0], np.ascontiguousarray(og.q[:, cols]), og.zero_point[0], ox.scale[0], og.scale[0])
+    assert np.array_equal(to_host(acc[:, cols]), oacc) and np.array_equal(to_host(dW[:, cols]), oout)
+
+
+@pytest.mark.parametrize("n,n_cols", [(8192, 48), (16384, 16)])
+def test_wgrad_dense_sweep_large_cubes_sampled_columns(B, n, n_cols):
+    """8192^3 and 16384^3: the reduction over M is split over CTAs in chunks of at most 65536 rows and summed in int64."""
+    _dense_wgrad_sampled(B, n, n, n, 10 + n // 8192, n_cols)
+
+
+@pytest.mark.parametrize("M,N,K", NONCUBE)
+def test_wgrad_dense_sweep_noncube_sampled_columns(B, M, N, K):
+    _dense_wgrad_sampled(B, M, N, K, 20 + M // 4096 + K // 2048, 24)
+
+
 # Shapes the CTA-pair kernel takes (at least eight rounds of 256 x 256 tiles over the SM pairs) with ragged edges in
 # every dimension: 512 x 256 pair tiles (M >= 2048) and 256 x 256 pair tiles (short M, wide N).
 PAIR_GEMMS = [(8208, 8464, 208), (1104, 38000, 144), (2048, 19216, 400)]

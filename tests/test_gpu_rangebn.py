@@ -1,4 +1,4 @@
-"""GPU Range BN forward / backward vs the CPU oracle (fp64), within 1e-5 relative per channel."""
+"""GPU Range BN forward / backward vs the CPU oracle (fp64): max|a - b| / max|b| <= 1e-5 per channel."""
 import numpy as np
 import pytest
 
@@ -15,21 +15,28 @@ def B():
     return binding
 
 
-def _per_channel_rel(got, want, floor=None):
-    """max|got - want| / max(max|want|, floor) per channel, worst channel.  `floor` is the channel's natural
-    magnitude, for channels whose reference is all (or nearly all) zero: a ReLU that cuts almost everything,
-    or n = 2 where dx cancels exactly."""
+CANCEL = 1.0 / 32.0
+
+
+def _per_channel_rel(got, want, terms=None):
+    """Worst channel of max|got - want| / max|want| (the tolerance definition used for every fp32 output).
+
+    `terms` (per channel) is the magnitude of the terms the output is a sum of.  A fp32 sum carries an absolute
+    error of a few 2^-24 of its largest term, so a channel whose whole reference lies below 1/32 of that magnitude
+    (a ReLU that cut everything but values next to zero; n = 2, where dx cancels to zero identically) cannot
+    meet a bound relative to the result in any fp32 evaluation: such a channel, and only such a channel, is measured
+    against terms / 32 instead.  A channel whose reference is identically zero must agree to within 1e-5 of terms."""
     C = want.shape[-1]
     g = np.asarray(got, np.float64).reshape(-1, C); w = np.asarray(want, np.float64).reshape(-1, C)
     den = np.abs(w).max(0)
-    if floor is not None:
-        den = np.maximum(den, np.asarray(floor, np.float64))
+    if terms is not None:
+        den = np.maximum(den, CANCEL * np.asarray(terms, np.float64))
     den[den == 0] = 1.0
     return float((np.abs(g - w).max(0) / den).max())
 
 
 def _scales(x, dy, vmin, vmax, gamma, beta):
-    """Natural magnitudes per channel: |gamma| * max|xhat| + |beta| for y, s * |gamma| * max|dy| for dx."""
+    """Magnitude of the terms per channel: |gamma| * max|xhat| + |beta| for y, s * |gamma| * max|dy| for dx."""
     C = x.shape[-1]; n = x.size // C
     g = np.ones(C) if gamma is None else np.abs(gamma.astype(np.float64))
     b = np.zeros(C) if beta is None else np.abs(beta.astype(np.float64))
@@ -55,10 +62,9 @@ def _run(B, x, dy, gamma, beta, relu):
     dx, dg, db = B.qbp_rangebn_bwd(to_dev(dy), xd, mean, vmin, vmax, gd, bd, relu)
     odx, odg, odb = O.rangebn_bwd(dy, x, to_host(mean), to_host(vmin), to_host(vmax), gamma, beta, relu)
     assert _per_channel_rel(to_host(dx), odx, dx_scale) <= FP32_TOL
-    n = x.size // x.shape[-1]
-    sum_scale = np.abs(dy).max() * np.sqrt(n)               # sums of n terms of that size
-    assert np.abs(to_host(dg) - odg).max() <= FP32_TOL * max(np.abs(odg).max(), sum_scale)
-    assert np.abs(to_host(db) - odb).max() <= FP32_TOL * max(np.abs(odb).max(), sum_scale)
+    # the two channel-sum vectors: per tensor, max|a - b| / max|b|
+    assert np.abs(to_host(dg) - odg).max() <= FP32_TOL * np.abs(odg).max()
+    assert np.abs(to_host(db) - odb).max() <= FP32_TOL * np.abs(odb).max()
 
 
 CASES = [(2, 1, 1, 4), (64, 1, 1, 128), (4, 7, 7, 64), (3, 5, 5, 6), (2, 3, 3, 2048), (5, 4, 4, 96), (1001, 1, 1, 1)]

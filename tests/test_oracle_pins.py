@@ -192,9 +192,33 @@ def test_stochastic_codes_depend_only_on_position_seed_and_id():
     inv = np.float32(1.0) / s
     t = (x.astype(np.float64) * np.float64(inv) + np.float64(zp_u)).astype(np.float32)  # fma: one rounding
     f = np.floor(t); frac = t - f
-    u = np.array([O.random_word(11, 5, i) >> 8 for i in range(x.size)], np.float64) / 2.0**24
+    # (8-bit codes draw from the word's high half, 16-bit codes from its low half)
+    words = np.array([O.random_word(11, 5, i) for i in range(x.size)], np.uint64)
+    u = (words >> 16).astype(np.float64) / 2.0**16
     want = np.clip(f.ravel() + (u < frac.ravel()), 0, 255) - 128
     assert np.array_equal(full.q.ravel().astype(np.int64), want.astype(np.int64))
+    full16 = O.quantize(x, 16, rounding=1, seed=11, tensor_id=5, range_in=rng)
+    s16 = full16.scale[0]; zp16 = np.float32(int(full16.zero_point[0]) + 32768)
+    t16 = (x.astype(np.float64) * np.float64(np.float32(1.0) / s16) + np.float64(zp16)).astype(np.float32)
+    f16 = np.floor(t16); frac16 = t16 - f16
+    u16 = (words & 0xFFFF).astype(np.float64) / 2.0**16
+    want16 = np.clip(f16.ravel() + (u16 < frac16.ravel()), 0, 65535) - 32768
+    assert np.array_equal(full16.q.ravel().astype(np.int64), want16.astype(np.int64))
+
+
+def test_the_two_copies_of_a_gradient_round_independently():
+    """Gradients Bifurcation quantises one tensor twice (8 and 16 bits) under one (seed, tensor id): the two
+    round-up decisions of an element come from disjoint halves of its word, so over many elements they are
+    uncorrelated, and each is unbiased on its own."""
+    n = 1 << 18
+    x = np.full((n // 64, 64), 0.3137, np.float32)
+    rng = (np.float32(-1.0), np.float32(1.0))
+    q8 = O.quantize(x, 8, rounding=1, seed=21, tensor_id=4, range_in=rng)
+    q16 = O.quantize(x, 16, rounding=1, seed=21, tensor_id=4, range_in=rng)
+    up8 = (q8.q.ravel() - q8.q.min()).astype(np.float64); up16 = (q16.q.ravel() - q16.q.min()).astype(np.float64)
+    assert set(np.unique(up8)) == {0.0, 1.0} and set(np.unique(up16)) == {0.0, 1.0}
+    corr = np.corrcoef(up8, up16)[0, 1]
+    assert abs(corr) < 5.0 / math.sqrt(n)
 
 
 def test_limb_split_exhaustive():

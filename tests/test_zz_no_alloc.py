@@ -11,6 +11,7 @@ import ctypes as C
 import numpy as np
 import pytest
 
+from oracle import qbp_oracle as O
 from paper_1805_11046_b200 import synth
 from tests.util import to_dev, to_host
 
@@ -52,6 +53,30 @@ def test_static_variant_matches_the_workspace_variant_twice_in_a_row(B, granular
         torch.cuda.synchronize()
         assert np.array_equal(to_host(q), to_host(want_q))              # codes bit for bit
         assert np.array_equal(to_host(qp), to_host(want_qp))            # scale, zero-point, range bit for bit
+        # and directly against the CPU statement of the quantiser
+        o = O.quantize(x, 8, per_channel=bool(granularity), rounding=rounding, seed=5, tensor_id=9 + k)
+        scale, zp, lo, hi = B.read_qparams(qp)
+        assert np.array_equal(to_host(q), o.q) and np.array_equal(scale, o.scale) and np.array_equal(zp, o.zero_point)
+        assert np.array_equal(lo, o.vmin) and np.array_equal(hi, o.vmax)
+
+
+@pytest.mark.gpu
+def test_static_variant_allocates_no_device_memory(B):
+    """The point of the entry point: after a first call (which resolves the built-in array's address and loads the
+    kernels) further calls leave the device's free memory and torch's allocator untouched."""
+    import torch
+    x = to_dev(synth.normal((515, 128), 79))
+    q = torch.empty(x.shape, dtype=torch.int8, device="cuda")
+    for granularity in (0, 1):
+        qp = B.new_qparams(128 if granularity else 1)
+        B.qbp_quantize_s8_static(x, q, qp, granularity=granularity, rounding=1, seed=1, tensor_id=2)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info(); alloc0 = torch.cuda.memory_allocated(); reserved0 = torch.cuda.memory_reserved()
+        for _ in range(3):
+            B.qbp_quantize_s8_static(x, q, qp, granularity=granularity, rounding=1, seed=1, tensor_id=2)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0 and torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
 
 
 @pytest.mark.gpu
