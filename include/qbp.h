@@ -115,10 +115,11 @@ int qbp_selftest_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_cycles, 
  * clamping values = the tensor's min and max, widened to contain 0.  Nearest
  * rounding (ties to even) for weights and activations; stochastic rounding
  * for gradients (Section 4: convergence needed it) -- up with probability
- * frac, the draw being the top 24 bits of the Philox4x32-10 word of the
- * element: key = seed, counter = (i/4 low, i/4 high, tensor_id, 0), word i%4,
- * i = flat index.  All arithmetic is IEEE fp32 in a fixed order, so codes
- * are reproducible bit for bit.
+ * frac, the draw being 16 bits of the Philox4x32-10 word of the element (the
+ * high half-word for 8-bit codes, the low half-word for 16-bit codes): key =
+ * seed, counter = (i/4 low, i/4 high, tensor_id, 0), word i%4, i = flat
+ * index.  All arithmetic is IEEE fp32 in a fixed order, so codes are
+ * reproducible bit for bit.
  *
  * x [rows x cols], cols innermost (the channel dimension).  granularity
  * QBP_PER_CHANNEL keeps one qbp_qparams per column (qp_out has `cols`
@@ -191,12 +192,38 @@ int qbp_quantize_s16(const float *x, int64_t rows, int64_t cols, int granularity
  * together"): from one read of the fp32 gradient g, write its 8-bit copy
  * (for the layer gradient) and its 16-bit copy as byte limbs (for the weight
  * gradient); both per-tensor, both stochastically rounded, from the streams
- * tensor_id8 and tensor_id16.  row_sums8 (nullable): as in qbp_quantize_s8. */
+ * tensor_id8 and tensor_id16 (equal ids: both copies draw from one word per
+ * element, the 8-bit copy from its high half, the 16-bit copy from its low
+ * half -- independent draws at half the generator work).  row_sums8
+ * (nullable): as in qbp_quantize_s8. */
 int qbp_bifurcate(const float *g, int64_t rows, int64_t cols, uint64_t seed,
                   uint32_t tensor_id8, uint32_t tensor_id16,
                   int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8,
                   int8_t *hi, uint8_t *lo, qbp_qparams *qp16,
                   void *ws, size_t ws_bytes, void *stream);
+
+/* qbp_bifurcate for one shard of a gradient whose minibatch is spread over
+ * several GPUs (Gradients Bifurcation, Sections 1, 4 and 6; data-parallel
+ * form).  g is this GPU's [rows x cols] part of the whole gradient tensor:
+ * index_base (a multiple of 4) is the flat index of g[0] in the whole tensor,
+ * so that every element keeps the Philox word it has in the undivided tensor,
+ * and range_in carries the clamping values of the WHOLE tensor (the min and
+ * max, combined over the GPUs by the caller), so that all shards share one
+ * scale.  The codes are then, bit for bit, the rows of the codes that the
+ * undivided call would produce.  No workspace: nothing is scanned. */
+int qbp_bifurcate_shard(const float *g, int64_t rows, int64_t cols, uint64_t seed,
+                        uint32_t tensor_id8, uint32_t tensor_id16, uint64_t index_base,
+                        const qbp_qparams *range_in,
+                        int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8,
+                        int8_t *hi, uint8_t *lo, qbp_qparams *qp16, void *stream);
+
+/* Dequantisation of integer accumulators that were combined outside the
+ * product: out[i] = (float)acc[i] * (qa->scale * qb->scale), as the products
+ * themselves do it.  For Eq. (grad_weight) under data parallelism: each GPU
+ * takes its int64 accumulators from qbp_wgrad_s16 (acc_out), the caller adds
+ * them up over the GPUs (exact, order-free), then dequantises here. */
+int qbp_dequant_s64(const int64_t *acc, int64_t count, const qbp_qparams *qa, const qbp_qparams *qb,
+                    float *out, void *stream);
 
 /* ------------------------------------------------------------------------
  * 8-bit products -- Section 1 (the weighted sums y = W x are where the work
@@ -410,6 +437,20 @@ int qbp_layer_bwd(const qbp_layer_desc *L, const qbp_layer_ctx *saved, const flo
                   const float *gamma, const float *beta,
                   float *dx, float *dw, float *dgamma, float *dbeta,
                   void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Weight update -- Section 6 "Putting it all together": the updates are the
+ * one operation kept in float32 (they accumulate small changes and run once
+ * per minibatch).  The paper names stochastic gradient descent and no further
+ * detail; this is the usual step with optional momentum and weight decay:
+ *   g = dw + weight_decay * w;  v = momentum * v + g (momentum_buf non-NULL);
+ *   w = w - lr * v   (or w - lr * g without a buffer),
+ * each operation rounded to fp32 on its own, in this order.  w (master
+ * weights, or gamma / beta of a Range BN) and momentum_buf are updated in
+ * place; `count` elements.
+ * ---------------------------------------------------------------------- */
+int qbp_sgd_update(float *w, const float *dw, float *momentum_buf, int64_t count,
+                   float lr, float momentum, float weight_decay, void *stream);
 
 #ifdef __cplusplus
 }

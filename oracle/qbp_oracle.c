@@ -179,11 +179,31 @@ static int32_t quantize_one(float x, float inv_scale, int32_t zp_u, int32_t L,
  * preceding Range BN: [vmin, vmax] per tensor, or vmin[cols] then vmax[cols].
  * Outputs: signed stored codes (q8 for bits=8, q16 for bits=16), and per
  * tensor (or per channel) scale, stored zero-point, vmin, vmax as used. */
+void qbo_quantize_at(const float *x, int64_t rows, int64_t cols, int bits,
+                     int per_channel, int rounding, uint64_t seed, uint32_t tensor_id,
+                     uint64_t index_base, const float *range_in,
+                     int8_t *q8, int16_t *q16,
+                     float *scale, int32_t *zero_point, float *vmin, float *vmax);
+
 void qbo_quantize(const float *x, int64_t rows, int64_t cols, int bits,
                   int per_channel, int rounding, uint64_t seed, uint32_t tensor_id,
                   const float *range_in,
                   int8_t *q8, int16_t *q16,
                   float *scale, int32_t *zero_point, float *vmin, float *vmax)
+{
+    qbo_quantize_at(x, rows, cols, bits, per_channel, rounding, seed, tensor_id, 0, range_in,
+                    q8, q16, scale, zero_point, vmin, vmax);
+}
+
+/* The same for a block of rows cut out of a larger tensor: index_base is the
+ * flat index of x[0] in that tensor, so that element i draws the random word
+ * of position index_base + i (the data-parallel case: each GPU holds some of
+ * the rows of one gradient tensor). */
+void qbo_quantize_at(const float *x, int64_t rows, int64_t cols, int bits,
+                     int per_channel, int rounding, uint64_t seed, uint32_t tensor_id,
+                     uint64_t index_base, const float *range_in,
+                     int8_t *q8, int16_t *q16,
+                     float *scale, int32_t *zero_point, float *vmin, float *vmax)
 {
     const int64_t nq = per_channel ? cols : 1;
     const int32_t L = (1 << bits) - 1;
@@ -207,7 +227,7 @@ void qbo_quantize(const float *x, int64_t rows, int64_t cols, int bits,
             int64_t p = per_channel ? c : 0;
             float inv = 1.0f / scale[p];
             int32_t zp_u = zero_point[p] + half;
-            uint32_t rnd = rounding ? qbo_random_word(seed, tensor_id, (uint64_t)i) : 0u;
+            uint32_t rnd = rounding ? qbo_random_word(seed, tensor_id, index_base + (uint64_t)i) : 0u;
             int32_t code = quantize_one(x[i], inv, zp_u, L, rounding, rnd) - half;
             if (bits == 8) q8[i] = (int8_t)code; else q16[i] = (int16_t)code;
         }
@@ -520,5 +540,27 @@ void qbo_rangebn_bwd(const float *dy, const float *x, int64_t n, int64_t C,
             dx[i * C + c] = s * (g * d - m1 - Cn * m2 * ind);
         }
         dgamma[c] = sdyx; dbeta[c] = sdy;
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* fp32 weight update (Section 6: the updates are kept in float32)           */
+/* ------------------------------------------------------------------------ */
+
+/* g = dw + wd*w;  v = mu*v + g (when a momentum buffer is kept);  w = w - lr*v.
+ * The paper fixes the precision (float32), so this is float arithmetic, every
+ * operation rounded on its own in this order (no contraction). */
+void qbo_sgd_update(float *w, const float *dw, float *vbuf, int64_t n, float lr, float mu, float wd)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        float t = wd * w[i];
+        float g = dw[i] + t;
+        if (vbuf) {
+            float m = mu * vbuf[i];
+            g = m + g;
+            vbuf[i] = g;
+        }
+        float step = lr * g;
+        w[i] = w[i] - step;
     }
 }

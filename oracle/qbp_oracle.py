@@ -118,8 +118,9 @@ def qparams(vmin: float, vmax: float, bits: int):
 
 
 def quantize(x, bits=8, per_channel=False, rounding=0, seed=0, tensor_id=0,
-             range_in=None) -> Quantized:
-    """rounding 0 = nearest (ties to even), 1 = stochastic.  range_in = (vmin, vmax)."""
+             range_in=None, index_base=0) -> Quantized:
+    """rounding 0 = nearest (ties to even), 1 = stochastic.  range_in = (vmin, vmax).
+    index_base: flat index of x[0] in the larger tensor x is a block of rows of."""
     x = _f32(x); cols = x.shape[-1]; rows = x.size // cols
     nq = cols if per_channel else 1
     q = np.zeros(x.shape, np.int8 if bits == 8 else np.int16)
@@ -129,10 +130,10 @@ def quantize(x, bits=8, per_channel=False, rounding=0, seed=0, tensor_id=0,
     if range_in is not None:
         rng = np.concatenate([np.asarray(range_in[0], np.float32).reshape(nq),
                               np.asarray(range_in[1], np.float32).reshape(nq)])
-    lib().qbo_quantize(_p(x), C.c_int64(rows), C.c_int64(cols), bits, int(per_channel),
-                       int(rounding), C.c_uint64(seed), C.c_uint32(tensor_id), _p(rng),
-                       _p(q) if bits == 8 else None, _p(q) if bits == 16 else None,
-                       _p(scale), _p(zp), _p(lo), _p(hi))
+    lib().qbo_quantize_at(_p(x), C.c_int64(rows), C.c_int64(cols), bits, int(per_channel),
+                          int(rounding), C.c_uint64(seed), C.c_uint32(tensor_id), C.c_uint64(index_base), _p(rng),
+                          _p(q) if bits == 8 else None, _p(q) if bits == 16 else None,
+                          _p(scale), _p(zp), _p(lo), _p(hi))
     return Quantized(q, scale, zp, lo, hi, bits)
 
 
@@ -255,6 +256,15 @@ def rangebn_bwd(dy, x, save_mean, save_min, save_max, gamma=None, beta=None, rel
     lib().qbo_rangebn_bwd(_p(dy), _p(x), C.c_int64(n), C.c_int64(Cc), _p(g), _p(b), int(relu),
                           _p(mu), _p(lo), _p(hi), _p(dx), _p(dg), _p(db))
     return dx, dg, db
+
+
+# ----------------------------------------------------------- weight update
+def sgd_update(w, dw, vbuf=None, lr=0.1, momentum=0.0, weight_decay=0.0):
+    """fp32 step of the master weights (Section 6): returns (new w, new momentum buffer or None); inputs untouched."""
+    w = _f32(w).copy(); dw = _f32(dw)
+    v = None if vbuf is None else _f32(vbuf).copy()
+    lib().qbo_sgd_update(_p(w), _p(dw), _p(v), C.c_int64(w.size), C.c_float(lr), C.c_float(momentum), C.c_float(weight_decay))
+    return w, v
 
 
 # ------------------------------------------------------------------- layer

@@ -25,6 +25,7 @@ EXPORTS = (
     "qbp_last_error", "qbp_trace_enable", "qbp_trace_count", "qbp_trace_read",
     "qbp_device_status", "qbp_selftest_bounded_wait",
     "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s8_static", "qbp_quantize_s16", "qbp_bifurcate",
+    "qbp_bifurcate_shard", "qbp_dequant_s64", "qbp_sgd_update",
     "qbp_range_chunked_workspace_bytes", "qbp_range_chunked",
     "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8",
     "qbp_conv_s8_workspace_bytes", "qbp_conv_s8_implicit",
@@ -115,12 +116,15 @@ _ws_cache: dict = {}
 
 
 def workspace(nbytes: int, device=None) -> torch.Tensor:
-    """A cached device scratch buffer of at least nbytes (grown on demand, 256-byte aligned by torch)."""
+    """A cached device scratch buffer of at least nbytes (grown on demand, 256-byte aligned by torch); one per
+    device and host thread, since calls of different threads may interleave on a stream."""
+    import threading
     dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
-    t = _ws_cache.get(dev)
+    key = (dev, threading.get_ident())
+    t = _ws_cache.get(key)
     if t is None or t.numel() < nbytes:
         t = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=dev)
-        _ws_cache[dev] = t
+        _ws_cache[key] = t
     return t
 
 
@@ -225,6 +229,29 @@ def qbp_bifurcate(g, seed, tensor_id8, tensor_id16, q8=None, hi=None, lo=None, q
                              C.c_uint32(tensor_id16), _ptr(q8), _ptr(qp8), _ptr(row_sums8), _ptr(hi), _ptr(lo),
                              _ptr(qp16), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
     return q8, qp8, hi, lo, qp16
+
+
+def qbp_bifurcate_shard(g, seed, tensor_id8, tensor_id16, index_base, range_in, q8=None, hi=None, lo=None, qp8=None,
+                        qp16=None, row_sums8=None):
+    """qbp_bifurcate for a block of rows of a larger gradient tensor: index_base = flat index of g[0] in it,
+    range_in = the whole tensor's clamping values."""
+    cols = g.shape[-1]; rows = g.numel() // cols if cols else 0
+    if q8 is None: q8 = torch.empty(g.shape, dtype=torch.int8, device=g.device)
+    if hi is None: hi = torch.empty(g.shape, dtype=torch.int8, device=g.device)
+    if lo is None: lo = torch.empty(g.shape, dtype=torch.uint8, device=g.device)
+    if qp8 is None: qp8 = new_qparams(1, g.device)
+    if qp16 is None: qp16 = new_qparams(1, g.device)
+    _check(lib.qbp_bifurcate_shard(_ptr(g), C.c_int64(rows), C.c_int64(cols), C.c_uint64(seed), C.c_uint32(tensor_id8),
+                                   C.c_uint32(tensor_id16), C.c_uint64(index_base), _ptr(range_in), _ptr(q8), _ptr(qp8),
+                                   _ptr(row_sums8), _ptr(hi), _ptr(lo), _ptr(qp16), _stream()))
+    return q8, qp8, hi, lo, qp16
+
+
+def qbp_dequant_s64(acc, qa, qb, out=None):
+    """out = float(acc) * (qa.scale * qb.scale) for int64 accumulators combined outside the product."""
+    if out is None: out = torch.empty(acc.shape, dtype=torch.float32, device=acc.device)
+    _check(lib.qbp_dequant_s64(_ptr(acc), C.c_int64(acc.numel()), _ptr(qa), _ptr(qb), _ptr(out), _stream()))
+    return out
 
 
 # ------------------------------------------------------------------- products
@@ -384,6 +411,13 @@ def qbp_rangebn_bwd(dy, x, mean, vmin, vmax, gamma=None, beta=None, relu=False, 
                                _ptr(mean), _ptr(vmin), _ptr(vmax), _ptr(dx), _ptr(dgamma), _ptr(dbeta), _ptr(ws),
                                C.c_size_t(ws.numel()), _stream()))
     return dx, dgamma, dbeta
+
+
+def qbp_sgd_update(w, dw, momentum_buf=None, lr=0.1, momentum=0.0, weight_decay=0.0):
+    """In-place fp32 update of master weights (Section 6): v = momentum*v + (dw + wd*w); w -= lr*v."""
+    _check(lib.qbp_sgd_update(_ptr(w), _ptr(dw), _ptr(momentum_buf), C.c_int64(w.numel()), C.c_float(lr),
+                              C.c_float(momentum), C.c_float(weight_decay), _stream()))
+    return w
 
 
 # ---------------------------------------------------------------------- layer

@@ -4,10 +4,14 @@
 //
 // Mapping: the matrix is read as vectors of VEC floats (4 when C % 4 == 0 and
 // the base is 16-byte aligned, else 1).  A 256-thread block is TW vector
-// columns wide and 256/TW rows high; blockIdx.y selects the slab of TW vector
-// columns, blockIdx.x the strip of rows, strips advance by gridDim.x.  A
-// thread therefore stays on the same VEC channels for its whole life and a
-// warp always reads 32*VEC consecutive floats.
+// columns wide (at most kScanMaxTw) and 256/TW rows high; blockIdx.y selects
+// the slab of TW vector columns, blockIdx.x the strip of rows, strips advance
+// by gridDim.x.  A thread therefore stays on the same VEC channels for its
+// whole life and a warp always reads 32*VEC consecutive floats.  Every block
+// leaves one partial per channel of its slab, so narrow slabs (many rows per
+// block, few channels) keep the partial arrays small: with 2048 channels, slabs
+// of 256 vectors cost 20 % extra traffic for the partials, slabs of 64 a
+// quarter of that.
 #pragma once
 
 #include "qbp_common.cuh"
@@ -17,11 +21,12 @@ namespace qbp {
 constexpr int kScanThreads = 256;
 constexpr int kScanUnroll = 4;
 constexpr int kScanMaxStrips = 1024;     // bound on gridDim.x, sizes the partial buffers
+constexpr int kScanMaxTw = 64;           // widest block in vector columns (64 float4 = 1 KB of a row)
 
 struct ScanGeom {
     int vec;        // 4 or 1
     int cv;         // vector columns = C / vec
-    int tw;         // threads across = min(pow2ceil(cv), 256)
+    int tw;         // threads across = min(pow2ceil(cv), kScanMaxTw)
     int rpb;        // rows per block step = 256 / tw
     int slabs;      // ceil(cv / tw)
     int nbx;        // row strips (gridDim.x)
@@ -48,7 +53,7 @@ inline ScanGeom scan_geom(int64_t rows, int64_t C, bool aligned, int bps)
     ScanGeom g;
     g.vec = (aligned && C % 4 == 0) ? 4 : 1;
     g.cv = (int)(C / g.vec);
-    g.tw = pow2ceil(g.cv) < kScanThreads ? pow2ceil(g.cv) : kScanThreads;
+    g.tw = pow2ceil(g.cv) < kScanMaxTw ? pow2ceil(g.cv) : kScanMaxTw;
     g.rpb = kScanThreads / g.tw;
     g.slabs = (g.cv + g.tw - 1) / g.tw;
     int64_t steps = (rows + g.rpb - 1) / g.rpb;

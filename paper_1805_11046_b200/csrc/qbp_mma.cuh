@@ -67,6 +67,12 @@ int launch_gemm2(int transA, int transB, int64_t M, int64_t N, int64_t K, const 
                  const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const int32_t *rowterm,
                  const int32_t *colterm, int *status, bool clear_status, cudaStream_t st);
 
+// ---- the dense weight gradient on CTA pairs (qbp_wgrad2.cu) ----------------------
+bool wgrad2_eligible(int64_t M, int64_t N, int64_t K);
+int launch_wgrad2(int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx, const int8_t *g_hi,
+                  const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW, const long long *rowterm,
+                  const long long *colterm, int *status, cudaStream_t st);
+
 // ---- shared-memory operand descriptors ---------------------------------------
 // How one operand tile of a pipeline stage is laid out and walked by the MMAs.
 struct OperandLayout {

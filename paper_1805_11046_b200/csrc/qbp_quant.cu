@@ -7,6 +7,7 @@
 // fill every SM.  Also hosts the library's error-reporting state.
 #include "qbp_colscan.cuh"
 
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -172,19 +173,22 @@ __global__ void __launch_bounds__(kThreads) chunk_range_partial_kernel(const flo
     }
 }
 
-// One block: every chunk's (min, max) from its blocks' partials, then the two averages, added up in chunk order in
-// double by one thread (the order is part of the result: it is the reference's).
+// One block: every chunk's (min, max) from its blocks' partials (a warp per chunk, the lanes stride over the
+// chunk's blocks), then the two averages, added up in chunk order in double by one thread (the order is part of
+// the result: the result depends on it, and the CPU check adds them up the same way).
 __global__ void __launch_bounds__(kThreads) chunk_range_finalize_kernel(const float2 *__restrict__ partials, int chunks,
                                                                         int blocks_per_chunk, float2 *__restrict__ per_chunk,
                                                                         qbp_qparams *__restrict__ out)
 {
-    for (int k = threadIdx.x; k < chunks; k += kThreads) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int k = warp; k < chunks; k += kThreads / 32) {
         float lo = INFINITY, hi = -INFINITY;
-        for (int b = 0; b < blocks_per_chunk; ++b) {
+        for (int b = lane; b < blocks_per_chunk; b += 32) {
             const float2 p = partials[(int64_t)k * blocks_per_chunk + b];
             lo = fminf(lo, p.x); hi = fmaxf(hi, p.y);
         }
-        per_chunk[k] = make_float2(lo, hi);
+        lo = warp_min(lo); hi = warp_max(hi);
+        if (lane == 0) per_chunk[k] = make_float2(lo, hi);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -295,11 +299,11 @@ __device__ __forceinline__ QParamsReg load_qp(const qbp_qparams *qp, int bits)
 template <bool SR>
 __device__ __forceinline__ void quantize_scalar(const float *x, int64_t i, int cols, bool perch,
                                                 const qbp_qparams *qp8, uint32_t id8, const qbp_qparams *qp16,
-                                                uint32_t id16, const PhiloxKeys &key, const QuantOut &o)
+                                                uint32_t id16, const PhiloxKeys &key, const QuantOut &o, uint64_t index_base)
 {
     const int c = perch ? (int)(i % cols) : 0;
     const float v = x[i];
-    const uint64_t j = (uint64_t)i >> 2;
+    const uint64_t j = ((uint64_t)i + index_base) >> 2;          // (index_base is a multiple of 4: word i & 3 is unchanged)
     if (o.q8) {
         QParamsReg p = load_qp(qp8 + c, 8);
         uint32_t rnd = 0;
@@ -353,12 +357,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                                                             const qbp_qparams *__restrict__ qp8,
                                                             uint32_t id8, const qbp_qparams *__restrict__ qp16,
                                                             uint32_t id16, const __grid_constant__ PhiloxKeys keys,
-                                                            QuantOut o, int smem_cols)
+                                                            QuantOut o, int smem_cols, uint64_t index_base)
 {
     if (VEC == 1) {
         const int64_t stride = (int64_t)gridDim.x * kThreads;
         for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += stride)
-            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o);
+            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o, index_base);
         return;
     }
     const bool want8 = o.q8 != nullptr, want16 = o.q16 || o.hi || o.lo;
@@ -404,8 +408,10 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
             const int c0 = PERCH ? (int)((j << 2) % cols) : 0;
             uint4 b8 = make_uint4(0, 0, 0, 0), b16 = b8;
             if (SR) {
-                if (want8) b8 = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id8, 0u), keys);
-                if (want16) b16 = one_block ? b8 : philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id16, 0u), keys);
+                // counter = the block's index in the whole tensor (a shard of a larger tensor starts at index_base)
+                const uint64_t jb = (uint64_t)j + (index_base >> 2);
+                if (want8) b8 = philox4x32_10(make_uint4((uint32_t)jb, (uint32_t)(jb >> 32), id8, 0u), keys);
+                if (want16) b16 = one_block ? b8 : philox4x32_10(make_uint4((uint32_t)jb, (uint32_t)(jb >> 32), id16, 0u), keys);
             }
             if (want8) {
                 const uint32_t r[4] = {b8.x, b8.y, b8.z, b8.w};
@@ -459,7 +465,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     }
     if (blockIdx.x == 0 && threadIdx.x == 0)
         for (int64_t i = nv << 2; i < n; ++i)
-            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o);
+            quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o, index_base);
 }
 
 // Row sums of stored 8-bit codes: a group of G lanes per row (G = smallest power
@@ -579,7 +585,7 @@ static int launch_chan_range(const float *x, int64_t rows, int64_t cols, int bit
 
 static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, int rounding,
                            const qbp_qparams *qp8, uint32_t id8, const qbp_qparams *qp16, uint32_t id16,
-                           uint64_t seed, const QuantOut &o, cudaStream_t st)
+                           uint64_t seed, const QuantOut &o, cudaStream_t st, uint64_t index_base = 0)
 {
     if (n == 0) return QBP_OK;
     const bool vec = aligned16(x) && (!perch || cols % 4 == 0) &&
@@ -599,7 +605,7 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
         const int grid = grid_for(blocks_per_sm(quantize_kernel<SR_, VEC_, PC_>, kThreads), groups);                    \
         QBP_TRACE_BEGIN(st);                                                                                            \
         quantize_kernel<SR_, VEC_, PC_><<<grid, kThreads, (VEC_) == 4 ? smem : 0, st>>>(x, n, c, qp8, id8, qp16, id16,  \
-                                                                                         key, o, (VEC_) == 4 ? smem_cols : 0); \
+                                                                                         key, o, (VEC_) == 4 ? smem_cols : 0, index_base); \
     } while (0)
     if (sr) {
         if (vec) { if (perch) QBP_QUANT(true, 4, true); else QBP_QUANT(true, 4, false); }
@@ -740,12 +746,12 @@ static int static_scratch_address(void **out)
 // The quantising half of the bifurcation, once qp8 / qp16 are known.
 static int bifurcate_tail(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                           uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo,
-                          qbp_qparams *qp16, cudaStream_t st)
+                          qbp_qparams *qp16, cudaStream_t st, uint64_t index_base = 0)
 {
     QuantOut o = {q8, nullptr, hi, lo, nullptr, 0, 0};
     const bool fused = row_sums8 && rows * cols > 0 && can_fuse_rowsums(g, q8, cols, o);
     if (fused) { o.rowsum8 = row_sums8; o.rs_group = (int)(cols / 4); o.rs_shift = 31 - __builtin_clz((unsigned)o.rs_group); }
-    int rc = launch_quantize(g, rows * cols, cols, 0, QBP_ROUND_STOCHASTIC, qp8, tensor_id8, qp16, tensor_id16, seed, o, st);
+    int rc = launch_quantize(g, rows * cols, cols, 0, QBP_ROUND_STOCHASTIC, qp8, tensor_id8, qp16, tensor_id16, seed, o, st, index_base);
     if (rc) return rc;
     if (row_sums8 && !fused) return launch_rowsum(q8, true, rows, cols, row_sums8, st);
     return QBP_OK;
@@ -880,6 +886,81 @@ extern "C" __attribute__((visibility("default"))) int qbp_bifurcate(const float 
     int rc = launch_range(g, rows * cols, parts, qp8, qp16, st);
     if (rc) return rc;
     return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st);
+}
+
+// Both parameter records from clamping values the caller supplies.
+__global__ void qparams_pair_from_range_kernel(const qbp_qparams *__restrict__ in, qbp_qparams *__restrict__ qp8,
+                                               qbp_qparams *__restrict__ qp16)
+{
+    *qp8 = make_qparams(in->vmin, in->vmax, 8);
+    *qp16 = make_qparams(in->vmin, in->vmax, 16);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_bifurcate_shard(const float *g, int64_t rows, int64_t cols, uint64_t seed,
+                                   uint32_t tensor_id8, uint32_t tensor_id16, uint64_t index_base, const qbp_qparams *range_in,
+                                   int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo,
+                                   qbp_qparams *qp16, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (rows < 0 || cols <= 0) return fail(QBP_ERR_INVALID_ARG, "bifurcate_shard: rows must be >= 0 and cols > 0");
+    if (!qp8 || !qp16 || !range_in) return fail(QBP_ERR_INVALID_ARG, "bifurcate_shard: qp8 / qp16 / range_in is NULL");
+    if (rows * cols > 0 && (!g || !q8 || !hi || !lo)) return fail(QBP_ERR_INVALID_ARG, "bifurcate_shard: NULL tensor");
+    if (((uintptr_t)g & 3) != 0) return fail(QBP_ERR_INVALID_ARG, "bifurcate_shard: g is not 4-byte aligned");
+    if (index_base % 4) return fail(QBP_ERR_INVALID_ARG, "bifurcate_shard: index_base must be a multiple of 4");
+    QBP_TRACE_BEGIN(st);
+    qparams_pair_from_range_kernel<<<1, 1, 0, st>>>(range_in, qp8, qp16);
+    QBP_LAUNCH_OK("qparams_pair_from_range_kernel");
+    return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st, index_base);
+}
+
+// out = (float)acc * (sa * sb): the dequantisation of a weight gradient whose int64 accumulators were added up
+// over several GPUs first (integer addition is exact, so the sum does not depend on the order of the GPUs).
+__global__ void dequant_s64_kernel(const long long *__restrict__ acc, int64_t n, const qbp_qparams *qa,
+                                   const qbp_qparams *qb, float *__restrict__ out)
+{
+    const float s = __fmul_rn(qa->scale, qb->scale);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = __fmul_rn((float)acc[i], s);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_dequant_s64(const int64_t *acc, int64_t count, const qbp_qparams *qa,
+                               const qbp_qparams *qb, float *out, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (count < 0 || (count > 0 && (!acc || !out)) || !qa || !qb) return fail(QBP_ERR_INVALID_ARG, "dequant_s64: NULL argument");
+    if (count == 0) return QBP_OK;
+    const int grid = (int)std::min<int64_t>((count + 255) / 256, (int64_t)sm_count() * 8);
+    QBP_TRACE_BEGIN(st);
+    dequant_s64_kernel<<<grid, 256, 0, st>>>((const long long *)acc, count, qa, qb, out);
+    QBP_LAUNCH_OK("dequant_s64_kernel");
+    return QBP_OK;
+}
+
+// fp32 master-weight update (Section 6 "Putting it all together": the updates stay in float32 and run once per
+// minibatch): g = dw + wd * w;  v = mu * v + g (with a momentum buffer);  w = w - lr * v.  Every operation is
+// rounded on its own, in this order.
+__global__ void __launch_bounds__(256) sgd_update_kernel(float *__restrict__ w, const float *__restrict__ dw,
+                                                         float *__restrict__ vbuf, int64_t n, float lr, float mu, float wd)
+{
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256) {
+        const float wi = w[i];
+        float g = __fadd_rn(dw[i], __fmul_rn(wd, wi));
+        if (vbuf) { g = __fadd_rn(__fmul_rn(mu, vbuf[i]), g); vbuf[i] = g; }
+        w[i] = __fsub_rn(wi, __fmul_rn(lr, g));
+    }
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_sgd_update(float *w, const float *dw, float *momentum_buf, int64_t count,
+                              float lr, float momentum, float weight_decay, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (count < 0 || (count > 0 && (!w || !dw))) return fail(QBP_ERR_INVALID_ARG, "sgd_update: NULL tensor");
+    if (count == 0) return QBP_OK;
+    const int grid = (int)std::min<int64_t>((count + 255) / 256, (int64_t)sm_count() * 8);
+    QBP_TRACE_BEGIN(st);
+    sgd_update_kernel<<<grid, 256, 0, st>>>(w, dw, momentum_buf, count, lr, momentum, weight_decay);
+    QBP_LAUNCH_OK("sgd_update_kernel");
+    return QBP_OK;
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8_static(const float *x, int64_t rows, int64_t cols, int granularity,

@@ -438,7 +438,8 @@ static int check_bn(const char *who, const void *a, const void *b, int64_t n, in
 // Upper bound on the (min, max) partials rangebn_bwd_impl writes: row strips x column slabs of the apply grid.
 size_t rangebn_range_parts_capacity(int64_t C)
 {
-    return (size_t)kScanMaxStrips * (size_t)((C + kScanThreads - 1) / kScanThreads + 1);
+    // (vector columns may be single floats: C columns in slabs of kScanMaxTw)
+    return (size_t)kScanMaxStrips * (size_t)((C + kScanMaxTw - 1) / kScanMaxTw + 1);
 }
 
 }  // namespace qbp

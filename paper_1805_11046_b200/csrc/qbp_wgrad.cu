@@ -821,6 +821,8 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
     int64_t *colterm = w.take<int64_t>(N);
     int64_t *part = P.direct ? nullptr : w.take<int64_t>((size_t)pl.grid * (size_t)P.part_stride);
 
+    // large plain products run on CTA pairs (256 x 256 tiles across two SMs, the whole reduction in one pair)
+    const bool pair_kernel = !d && wgrad2_eligible(M, N, K);
     // code sums for the zero-point terms: per border class (convolution) or plain column sums
     int rc;
     if (d && K == N && d->W <= 256 && M < (1ll << 30) && shi == sx + 16 * K && slo == shi + 16 * N) {
@@ -846,7 +848,7 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
         if ((rc = launch_colsum(x, true, M, K, sx, st))) return rc;
         if ((rc = launch_colsum(g_hi, true, M, N, shi, st))) return rc;
         if ((rc = launch_colsum(g_lo, false, M, N, slo, st))) return rc;
-        if (P.direct) {
+        if (P.direct || pair_kernel) {
             const int64_t mx = std::max(K, N);
             QBP_TRACE_BEGIN(st);
             wgrad_terms_kernel<<<(unsigned)((mx + 255) / 256), 256, 0, st>>>((const long long *)sx, (const long long *)shi,
@@ -856,6 +858,9 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
         }
     }
     if (!ext_status) QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
+    if (pair_kernel)
+        return launch_wgrad2(M, N, K, x, qx, g_hi, g_lo, qg16, acc_out, dW, (const long long *)rowterm,
+                             (const long long *)colterm, status, st);
 
     P.part = (long long *)part; P.status = status;
     P.rowterm = (const long long *)rowterm; P.colterm = (const long long *)colterm;

@@ -81,3 +81,59 @@ class QuantizedLayer:
 
     def status(self) -> int:
         return B.status_word(self.ws)
+
+
+class QuantizedStack:
+    """A chain of quantised convolution layers, each followed by Range BN + ReLU, trained as the method prescribes
+    (Sections 4 and 6): every inner activation is handed on as the 8-bit codes its Range BN wrote (no range scan and
+    no quantisation pass between layers), gradients flow back through qbp_layer_bwd, and the fp32 master weights,
+    gamma and beta are updated once per minibatch by qbp_sgd_update.  Buffer bookkeeping and call order only."""
+
+    def __init__(self, convs, weights, seed=0, chained=True, keep_y=False, lr=0.1, momentum=0.9, weight_decay=1e-4,
+                 device="cuda"):
+        """convs: binding.ConvDesc per layer (layer i's output shape = layer i+1's input shape); weights: the fp32
+        master weights (KRSC device tensors, updated in place).  chained=False runs every layer from the fp32
+        activation of the one before (range scan + quantiser per layer) -- the unfused composition, for comparison."""
+        self.chained, self.lr, self.momentum, self.weight_decay = chained, lr, momentum, weight_decay
+        self.w = list(weights)
+        self.layers = []
+        n = len(convs)
+        for i, conv in enumerate(convs):
+            last = i == n - 1
+            prev = self.layers[-1] if (self.layers and chained) else None
+            self.layers.append(QuantizedLayer(conv=conv, relu=True, seed=seed, tensor_id8=i + 1, tensor_id16=i + 1, device=device,
+                                              input_from=prev, emit_codes=chained and not last,
+                                              keep_y=(not chained) or last or keep_y))
+        dev = torch.device(device)
+        self.gamma = [torch.ones(L.cout, dtype=torch.float32, device=dev) for L in self.layers]
+        self.beta = [torch.zeros(L.cout, dtype=torch.float32, device=dev) for L in self.layers]
+        mk = lambda ts: [torch.zeros_like(t) for t in ts] if momentum else [None] * len(ts)
+        self.vw, self.vg, self.vb = mk(self.w), mk(self.gamma), mk(self.beta)
+
+    def forward(self, x):
+        a = x
+        for L, w, g, b in zip(self.layers, self.w, self.gamma, self.beta):
+            y = L.forward(a if L.rq_in is None else None, w, g, b)
+            a = y
+        return self.layers[-1].y
+
+    def backward(self, dy):
+        d = dy
+        for L in reversed(self.layers):
+            d, _, _, _ = L.backward(d)         # dx of a layer is the gradient at the previous layer's output
+        return d
+
+    def update(self):
+        for L, w, g, b, vw, vg, vb in zip(self.layers, self.w, self.gamma, self.beta, self.vw, self.vg, self.vb):
+            B.qbp_sgd_update(w, L.dw, vw, self.lr, self.momentum, self.weight_decay)
+            B.qbp_sgd_update(g, L.dgamma, vg, self.lr, self.momentum, 0.0)
+            B.qbp_sgd_update(b, L.dbeta, vb, self.lr, self.momentum, 0.0)
+
+    def train_step(self, x, dy):
+        self.forward(x)
+        dx = self.backward(dy)
+        self.update()
+        return dx
+
+    def status(self) -> int:
+        return min(L.status() for L in self.layers)

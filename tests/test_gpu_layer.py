@@ -254,3 +254,72 @@ def test_chained_stack_backward_runs_on_the_handed_on_codes(B):
     _, odx, bad = O.conv_s8(1, od, g8.q, g8.zero_point[0], ow.q, ow.zero_point[0], g8.scale[0], ow.scale[0])
     _, odw = O.conv_wgrad_s16(od, xq, z_[0], g16.q, g16.zero_point[0], np.float32(s_[0]), g16.scale[0])
     assert bad == 0 and np.array_equal(to_host(dx), odx) and np.array_equal(to_host(dw), odw)
+
+
+# ------------------------------------------------ fp32 master-weight update and a whole training step of a stack
+@pytest.mark.parametrize("momentum,wd", [(0.0, 0.0), (0.9, 1e-4)])
+def test_sgd_update_matches_the_fp32_statement_bit_for_bit(B, momentum, wd):
+    w = synth.normal((4099,), 81); dw = synth.normal((4099,), 82, std=0.01); v = synth.normal((4099,), 83, std=0.01)
+    wd_ = to_dev(w); vd = to_dev(v) if momentum else None
+    ow, ov = w, (v if momentum else None)
+    for _ in range(3):
+        B.qbp_sgd_update(wd_, to_dev(dw), vd, lr=0.05, momentum=momentum, weight_decay=wd)
+        ow, ov = O.sgd_update(ow, dw, ov, lr=0.05, momentum=momentum, weight_decay=wd)
+    assert np.array_equal(to_host(wd_), ow)
+    if momentum:
+        assert np.array_equal(to_host(vd), ov)
+
+
+def test_training_steps_of_the_chained_bottleneck_stack(B):
+    """Two whole training steps (forward chain on handed-on codes, backward chain, fp32 updates of w, gamma, beta) of
+    the conv3_x bottleneck at a reduced batch.  After each step the updated tensors equal the fp32 statement of the
+    update applied to the gradients the GPU produced, and the next forward quantises exactly those weights."""
+    import torch
+    from paper_1805_11046_b200 import layer
+    st = synth.bottleneck_stack(batch=8, hw=28)
+    convs = [B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"]) for c in st["convs"]]
+    S = layer.QuantizedStack(convs, [to_dev(w) for w in st["w"]], lr=0.05, momentum=0.9, weight_decay=1e-4)
+    x, dy = to_dev(st["x"]), to_dev(st["dy"])
+    ow = [w.copy() for w in st["w"]]; ovw = [np.zeros_like(w) for w in ow]
+    og = [np.ones(L.cout, np.float32) for L in S.layers]; ovg = [np.zeros_like(g) for g in og]
+    ob = [np.zeros(L.cout, np.float32) for L in S.layers]; ovb = [np.zeros_like(b) for b in ob]
+    for step in range(2):
+        S.train_step(x, dy)
+        torch.cuda.synchronize()
+        assert S.status() == 0
+        for i, L in enumerate(S.layers):
+            # the forward of this step quantised the weights as they stood before the update
+            assert np.array_equal(to_host(L.w_codes), O.quantize(ow[i], 8).q)
+            ow[i], ovw[i] = O.sgd_update(ow[i], to_host(L.dw), ovw[i], 0.05, 0.9, 1e-4)
+            og[i], ovg[i] = O.sgd_update(og[i], to_host(L.dgamma), ovg[i], 0.05, 0.9, 0.0)
+            ob[i], ovb[i] = O.sgd_update(ob[i], to_host(L.dbeta), ovb[i], 0.05, 0.9, 0.0)
+            assert np.array_equal(to_host(S.w[i]), ow[i]) and np.array_equal(to_host(S.gamma[i]), og[i])
+            assert np.array_equal(to_host(S.beta[i]), ob[i])
+        if step == 0:
+            # the gradient chain: a layer's dy is the next layer's dx (straight-through estimator through the
+            # quantiser); gamma = 1, beta = 0 in the first step
+            for a, b_ in zip(S.layers[:-1], S.layers[1:]):
+                og_, _, _ = O.rangebn_bwd(to_host(b_.dx), to_host(a.z), to_host(a.save_mean), to_host(a.save_min),
+                                          to_host(a.save_max), relu=True)
+                assert rel_err(to_host(a.g), og_)[0] <= FP32_TOL
+    assert not np.array_equal(ow[0], st["w"][0])
+
+
+def test_chained_and_unchained_stacks_agree(B):
+    """The chained stack (codes handed on by the Range BN) and the unfused composition (every layer scans and
+    quantises the fp32 activation of the one before) compute the same thing: same codes, same outputs, same gradients."""
+    import torch
+    from paper_1805_11046_b200 import layer
+    st = synth.bottleneck_stack(batch=8, hw=28)
+    convs = [B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"]) for c in st["convs"]]
+    x, dy = to_dev(st["x"]), to_dev(st["dy"])
+    A = layer.QuantizedStack(convs, [to_dev(w) for w in st["w"]], chained=True)
+    U = layer.QuantizedStack(convs, [to_dev(w) for w in st["w"]], chained=False)
+    da = A.train_step(x, dy); du = U.train_step(x, dy)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host(da), to_host(du))
+    for La, Lu in zip(A.layers, U.layers):
+        assert np.array_equal(to_host(La.x_codes), to_host(Lu.x_codes)) and np.array_equal(to_host(La.z), to_host(Lu.z))
+        assert np.array_equal(to_host(La.dw), to_host(Lu.dw))
+    for wa, wu in zip(A.w, U.w):
+        assert np.array_equal(to_host(wa), to_host(wu))

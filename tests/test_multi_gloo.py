@@ -1,5 +1,7 @@
-"""The N > 1 path on CPU: two gloo ranks shard independent units with no overlap and agree on the
-max-over-ranks time (the only exchanges the data-parallel use of the path needs)."""
+"""The N > 1 path on CPU, two gloo ranks: (1) independent units are sharded with no overlap and the ranks agree
+on the max-over-ranks time; (2) one minibatch spread over the ranks -- the four exchange steps of the data-parallel
+path (quantiser range, Range BN statistics, Range BN backward sums, int64 weight-gradient accumulators), fed with
+per-shard partials computed on the host, reproduce the CPU oracle's results on the concatenated batch."""
 import os
 import socket
 
@@ -8,7 +10,10 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_1805_11046_b200.dist import max_over_ranks, shard_units, sum_over_ranks
+import numpy as np
+
+from paper_1805_11046_b200.dist import (allreduce_bn_stats, allreduce_range, allreduce_sums, max_over_ranks, shard_units,
+                                        sum_over_ranks)
 
 
 def test_shards_partition_the_units():
@@ -48,3 +53,102 @@ def test_two_gloo_ranks_agree():
         assert p.exitcode == 0
     assert [r[1:3] for r in res] == [(0, 129), (129, 257)]
     assert all(r[3] == 11.0 and r[4] == 257.0 for r in res)
+
+
+# ------------------------------------------------------------------ one minibatch over two ranks
+def _dp_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from oracle import qbp_oracle as O
+        from paper_1805_11046_b200 import synth
+        cfg = synth.conv3x3_layer(batch=4, hw=6, c_in=32, k_out=32)
+        c = cfg["conv"]
+        b, e = shard_units(4, rank, world)
+        x, dy = cfg["x"][b:e], cfg["dy"][b:e]
+        od = O.conv_desc(e - b, c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+        res = {}
+        # exchange 1: the quantiser's range of the whole activation tensor (a qbp_qparams record: scale, zp, vmin, vmax)
+        lo, hi = O.tensor_range(x)
+        rec = torch.zeros((1, 4), dtype=torch.float32); rec[0, 2] = float(lo[0]); rec[0, 3] = float(hi[0])
+        rec = allreduce_range(rec.view(torch.int32)).view(torch.float32)
+        rng = (np.float32(rec[0, 2].item()), np.float32(rec[0, 3].item()))
+        qx = O.quantize(x, 8, range_in=rng); qw = O.quantize(cfg["w"], 8)
+        res["x_codes"] = qx.q; res["x_scale"] = float(qx.scale[0]); res["x_zp"] = int(qx.zero_point[0])
+        _, z, bad = O.conv_s8(0, od, qx.q, qx.zero_point[0], qw.q, qw.zero_point[0], qx.scale[0], qw.scale[0])
+        assert bad == 0
+        res["z"] = z
+        # exchange 2: Range BN statistics per channel
+        z2 = z.reshape(-1, c["K"])
+        s = torch.from_numpy(z2.astype(np.float64).sum(0)); mn = torch.from_numpy(z2.min(0).copy()); mx = torch.from_numpy(z2.max(0).copy())
+        allreduce_bn_stats(s, mn, mx)
+        n_total = 4 * c["H"] * c["W"]
+        res["mean"] = (s.numpy() / n_total).astype(np.float32); res["vmin"] = mn.numpy(); res["vmax"] = mx.numpy()
+        # exchange 3: the backward sums; xhat as Eq. (range) defines it, with the combined statistics
+        Cn = O.rangebn_C(n_total)
+        r = (res["vmax"].astype(np.float64) - res["vmin"]); sc = np.where(r > 0, 1.0 / (Cn * np.where(r > 0, r, 1.0)), 0.0)
+        xhat = (z2.astype(np.float64) - res["mean"]) * sc
+        d2 = dy.reshape(-1, c["K"]).astype(np.float64)
+        sdy = torch.from_numpy(d2.sum(0)); sdyx = torch.from_numpy((d2 * xhat).sum(0))
+        allreduce_sums(sdy, sdyx)
+        res["dbeta"] = sdy.numpy(); res["dgamma"] = sdyx.numpy()
+        # the gradient at the product's output for this shard's rows, from the oracle given the combined statistics
+        # (its own sums are then the whole batch's only if it sees the whole batch: take g from the full-batch
+        # call on rank-local rows is not possible, so g is rebuilt from the closed form with the combined sums)
+        g = (sc * (d2 - sdy.numpy() / n_total - Cn * sdyx.numpy() * ((z2 == res["vmax"]).astype(np.float64) - (z2 == res["vmin"]).astype(np.float64)))).astype(np.float32)
+        res["g"] = g.reshape(dy.shape)
+        # exchange 1 again, for the gradient; codes drawn at the shard's place in the whole tensor
+        lo, hi = O.tensor_range(res["g"])
+        rec = torch.zeros((1, 4), dtype=torch.float32); rec[0, 2] = float(lo[0]); rec[0, 3] = float(hi[0])
+        rec = allreduce_range(rec.view(torch.int32)).view(torch.float32)
+        grng = (np.float32(rec[0, 2].item()), np.float32(rec[0, 3].item()))
+        base = b * c["H"] * c["W"] * c["K"]
+        g8 = O.quantize(res["g"], 8, rounding=1, seed=0, tensor_id=1, range_in=grng, index_base=base)
+        g16 = O.quantize(res["g"], 16, rounding=1, seed=0, tensor_id=1, range_in=grng, index_base=base)
+        res["g8"] = g8.q; res["g16"] = g16.q
+        # exchange 4: the weight gradient's int64 accumulators
+        acc, _ = O.conv_wgrad_s16(od, qx.q, qx.zero_point[0], g16.q, g16.zero_point[0])
+        t = torch.from_numpy(acc.copy()); allreduce_sums(t)
+        res["acc"] = t.numpy()
+        out.put((rank, res))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_share_one_minibatch():
+    from oracle import qbp_oracle as O
+    from paper_1805_11046_b200 import synth
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_dp_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = dict(q.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    cat = lambda k: np.concatenate([res[0][k], res[1][k]])
+    # the oracle on the concatenated batch
+    cfg = synth.conv3x3_layer(batch=4, hw=6, c_in=32, k_out=32)
+    c = cfg["conv"]
+    od = O.conv_desc(4, c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    qx = O.quantize(cfg["x"], 8); qw = O.quantize(cfg["w"], 8)
+    assert np.array_equal(cat("x_codes"), qx.q) and res[0]["x_scale"] == float(qx.scale[0]) and res[1]["x_zp"] == int(qx.zero_point[0])
+    _, z, _ = O.conv_s8(0, od, qx.q, qx.zero_point[0], qw.q, qw.zero_point[0], qx.scale[0], qw.scale[0])
+    assert np.array_equal(cat("z"), z)
+    _, om, olo, ohi = O.rangebn_fwd(z)
+    for r in (0, 1):
+        assert np.array_equal(res[r]["vmin"], olo) and np.array_equal(res[r]["vmax"], ohi)
+        assert np.abs(res[r]["mean"] - om).max() <= 1e-6 * max(1.0, np.abs(om).max())
+    og, odg, odb = O.rangebn_bwd(cfg["dy"], z, res[0]["mean"], olo, ohi)
+    assert np.abs(res[0]["dgamma"] - odg).max() <= 1e-9 * np.abs(odg).max() and np.abs(res[1]["dbeta"] - odb).max() <= 1e-9 * np.abs(odb).max()
+    g = cat("g")
+    assert np.abs(g - og).max() <= 1e-6 * np.abs(og).max()
+    # codes of the shards = rows of the codes of the whole tensor (same range, same random words)
+    g8 = O.quantize(g, 8, rounding=1, seed=0, tensor_id=1); g16 = O.quantize(g, 16, rounding=1, seed=0, tensor_id=1)
+    assert np.array_equal(cat("g8"), g8.q) and np.array_equal(cat("g16"), g16.q)
+    acc, _ = O.conv_wgrad_s16(od, qx.q, qx.zero_point[0], g16.q, g16.zero_point[0])
+    assert np.array_equal(res[0]["acc"], acc) and np.array_equal(res[1]["acc"], acc)

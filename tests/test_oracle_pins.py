@@ -187,6 +187,9 @@ def test_stochastic_codes_depend_only_on_position_seed_and_id():
     # the first 12 rows quantised alone (same flat positions) give the same codes
     head = O.quantize(x[:12], 8, rounding=1, seed=11, tensor_id=5, range_in=rng)
     assert np.array_equal(head.q, full.q[:12])
+    # ... and so do the last 28 when told where they start in the whole tensor
+    tail = O.quantize(x[12:], 8, rounding=1, seed=11, tensor_id=5, range_in=rng, index_base=12 * 50)
+    assert np.array_equal(tail.q, full.q[12:])
     # rebuild every code from the published random word: floor(t) + [u < frac]
     s = full.scale[0]; zp_u = np.float32(int(full.zero_point[0]) + 128)
     inv = np.float32(1.0) / s
@@ -460,3 +463,31 @@ def test_layer_composition_on_the_linear_config():
     # the 16-bit copy is the finer one
     e8 = np.abs(O.dequantize(g8) - dz).max(); e16 = np.abs(O.dequantize(g16) - dz).max()
     assert e16 < e8 / 100
+
+
+# ------------------------------------------------------------------ fp32 weight update
+def test_sgd_update_closed_forms():
+    """Values chosen dyadic so that every fp32 operation is exact and the closed forms hold to the bit."""
+    w0 = np.array([1.0, -2.0, 0.5, 8.0], np.float32); g = np.array([0.25, -0.5, 1.0, 0.0], np.float32)
+    # plain SGD, constant gradient: w_k = w_0 - k lr g
+    w = w0
+    for k in range(1, 6):
+        w, _ = O.sgd_update(w, g, lr=0.5)
+        assert np.array_equal(w, w0 - k * 0.5 * g)
+    # momentum 1/2, constant gradient: v_k = g (2 - 2^(1-k)), w_k = w_0 - lr sum_j v_j
+    w, v = w0, np.zeros(4, np.float32)
+    total = np.zeros(4, np.float64)
+    for k in range(1, 8):
+        w, v = O.sgd_update(w, g, v, lr=0.25, momentum=0.5)
+        assert np.array_equal(v, (g * (2.0 - 2.0 ** (1 - k))).astype(np.float32))
+        total += v
+        assert np.array_equal(w, (w0 - 0.25 * total).astype(np.float32))
+    # weight decay alone: w_k = w_0 (1 - lr wd)^k
+    w = w0
+    for k in range(1, 6):
+        w, _ = O.sgd_update(w, np.zeros(4, np.float32), lr=0.5, weight_decay=0.25)
+        assert np.array_equal(w, (w0 * 0.875 ** k).astype(np.float32))
+    # a dropped or mis-signed term shows: decay and gradient together, one step, by hand
+    w, v = O.sgd_update(np.array([2.0], np.float32), np.array([1.0], np.float32), np.array([4.0], np.float32), lr=0.5, momentum=0.5,
+                        weight_decay=0.25)
+    assert v[0] == 0.5 * 4.0 + (1.0 + 0.25 * 2.0) and w[0] == 2.0 - 0.5 * v[0]
