@@ -184,6 +184,17 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys &k)
     return c;
 }
 
+// Range BN (Section 3, Eq. (range)): xhat and y of one element and the per-channel scale 1 / (C(n) (max - min)).
+// The order of operations is part of the contract: every kernel that normalises (the apply passes, the fused
+// epilogue of a product) must produce the same bits, so that forward, backward and requantisation agree.
+__device__ __forceinline__ float bn_xhat(float x, float mu, float s) { return __fmul_rn(__fsub_rn(x, mu), s); }
+__device__ __forceinline__ float bn_y(float xh, float g, float b) { return __fadd_rn(__fmul_rn(g, xh), b); }
+__device__ __forceinline__ float bn_scale(float lo, float hi, float Cn)
+{
+    float r = __fsub_rn(hi, lo);
+    return r > 0.0f ? __fdiv_rn(1.0f, __fmul_rn(Cn, r)) : 0.0f;
+}
+
 __device__ __forceinline__ float warp_min(float v)
 {
 #pragma unroll

@@ -189,6 +189,13 @@ struct MmaParams {
     // warp keeps (sum, min, max) of the columns in shared memory; when the kernel ends the CTA's warps add them up
     // into row blockIdx.x of these partial arrays [rows][N].  One column tile only (N <= 256); NULL: not wanted.
     float *st_lo, *st_hi; double *st_sum;
+    // Optional tail of the epilogue: per-column normalisation by the Range BN that follows the product (ep_fold:
+    // (mean, scale, gamma, beta) per output column, copied to shared memory), ReLU, and the 8-bit codes of the result
+    // (parameters *ep_rq) written to ep_q [M x N] with each row's code sum in ep_rowsum (one column tile only).  `out`
+    // then receives the transformed value.  Statistics are of the untransformed output and exclude a tail.
+    const float4 *ep_fold; int ep_relu;
+    const qbp_qparams *ep_rq; int8_t *ep_q; int32_t *ep_rowsum;
+    uint32_t stat_span;           // bytes of the statistics region in shared memory (the fold table follows it)
     int grid;                     // CTAs launched
     uint32_t cterm_span;          // bytes of the column-term region in shared memory (the statistics follow it)
     int iter_entries;             // entries of the k-iteration table in shared memory (conv), a multiple of 64
@@ -376,6 +383,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
     int4 *s_iter = reinterpret_cast<int4 *>(staging + P.ewarps * kStageSlab * P.nslab);   // conv: one entry per k iteration
     int32_t *s_cterm = reinterpret_cast<int32_t *>(s_iter + P.iter_entries);             // column terms
     ColStat *s_stat = reinterpret_cast<ColStat *>(reinterpret_cast<uint8_t *>(s_cterm) + P.cterm_span);   // [ewarps][N]
+    float4 *s_fold = reinterpret_cast<float4 *>(reinterpret_cast<uint8_t *>(s_stat) + P.stat_span);       // [N]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -536,11 +544,17 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         const int bar_id = P.msub == 2 ? 1 : 1 + group, bar_cnt = P.msub == 2 ? 256 : 128;
         const int gt = P.msub == 2 ? threadIdx.x - 64 : (threadIdx.x - 64) & 127;     // thread index within the barrier group
         int32_t *region = s_cterm + (P.cterm_all || P.msub == 2 ? 0 : group * P.ncls * P.bn);
-        if (P.cterm_all) {
-            // the whole column-term table fits: fill it once
-            for (int i = threadIdx.x - 64; i < P.ncls * (int)P.N; i += 32 * P.ewarps) s_cterm[i] = __ldg(P.colterm + i);
+        if (P.cterm_all || P.ep_fold) {
+            // the whole column-term table fits: fill it once (and the per-column constants of the normalisation)
+            if (P.cterm_all)
+                for (int i = threadIdx.x - 64; i < P.ncls * (int)P.N; i += 32 * P.ewarps) s_cterm[i] = __ldg(P.colterm + i);
+            if (P.ep_fold)
+                for (int i = threadIdx.x - 64; i < (int)P.N; i += 32 * P.ewarps) s_fold[i] = __ldg(P.ep_fold + i);
             named_barrier(4, 32 * P.ewarps);
         }
+        float rq_inv = 0.0f, rq_zp = 0.0f;
+        if (P.ep_q) { rq_inv = __fdiv_rn(1.0f, P.ep_rq->scale); rq_zp = (float)(P.ep_rq->zero_point + 128); }
+        const bool tail = P.ep_fold || P.ep_relu || P.ep_q;
 
         // where this thread's accumulator row of a tile goes
         struct RowInfo { int64_t m; bool valid, slab_in; int cls, sx, sy, sz; };
@@ -627,7 +641,49 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                                 if (j < lim) dst[j] = acc[j];
                         }
                     }
-                    if (P.out) {
+                    // the fp32 value of the row's 32 outputs: dequantised, then (optionally) normalised and rectified
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __fmul_rn((float)acc[j], scale);
+                    if (tail) {
+                        if (P.ep_fold) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float4 f = s_fold[o.n0 + c0 + (j < lim ? j : 0)];       // (mean, scale, gamma, beta)
+                                v[j] = bn_y(bn_xhat(v[j], f.x, f.y), f.z, f.w);
+                            }
+                        }
+                        if (P.ep_relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+                        }
+                        if (P.ep_q) {
+                            // 8-bit codes of the row's 32 values: two 16-byte stores (the row's bytes are contiguous)
+                            uint32_t w8[8];
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                uint32_t c4[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) c4[e] = (uint32_t)quantize_code<false>(v[j + e], rq_inv, rq_zp, 255.0f, 0u);
+                                w8[j >> 2] = (c4[0] | (c4[1] << 8) | (c4[2] << 16) | (c4[3] << 24)) ^ 0x80808080u;
+                            }
+                            if (ri.valid) {
+                                int8_t *dst = P.ep_q + ri.m * P.N + o.n0 + c0;
+                                if (lim == 32) {
+                                    *reinterpret_cast<uint4 *>(dst) = make_uint4(w8[0], w8[1], w8[2], w8[3]);
+                                    *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(w8[4], w8[5], w8[6], w8[7]);
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) row_code_sum = __dp4a((int)w8[k], 0x01010101, row_code_sum);
+                                } else {
+                                    // (N is a multiple of 16: a ragged chunk holds 16 columns)
+                                    *reinterpret_cast<uint4 *>(dst) = make_uint4(w8[0], w8[1], w8[2], w8[3]);
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) row_code_sum = __dp4a((int)w8[k], 0x01010101, row_code_sum);
+                                }
+                            }
+                        }
+                    }
+                    if (P.out || P.st_sum) {
                         // the store that last used this slab must have read it before it is overwritten
                         uint8_t *slab = slab0 + slab_i * kStageSlab;
                         if (lane == 0) { if (P.nslab == 2) tma_store_wait_read_but_one(); else tma_store_wait_read(); }
@@ -637,12 +693,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                         uint8_t *rowp = slab + lane * 128;
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4 *>(rowp + (((j >> 2) ^ (lane & 7)) << 4)) =
-                                make_float4(__fmul_rn((float)acc[j], scale), __fmul_rn((float)acc[j + 1], scale),
-                                            __fmul_rn((float)acc[j + 2], scale), __fmul_rn((float)acc[j + 3], scale));
+                            *reinterpret_cast<float4 *>(rowp + (((j >> 2) ^ (lane & 7)) << 4)) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                         fence_proxy_async();
                         __syncwarp();
-                        if (lane == 0 && ri.slab_in) {
+                        if (lane == 0 && ri.slab_in && P.out) {
                             if (P.mode == MODE_GEMM) tma_store_2d(&P.mapC, slab, o.n0 + c0, o.m0 + sub * 128 + quad * 32);
                             else                     tma_store_4d(&P.mapC, slab, o.n0 + c0, ri.sx, ri.sy, ri.sz);
                             tma_store_commit();

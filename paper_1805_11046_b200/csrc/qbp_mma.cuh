@@ -30,11 +30,20 @@ int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, ui
 // of the tensor-core kernel; `rows` is filled in by the launch.  colstat_rows_max(): the most rows a launch leaves.
 struct ColStatParts { float *lo, *hi; double *sum; int rows; };
 int colstat_rows_max();
+int rangebn_fold_from_parts(int64_t n, int64_t C, const float *gamma, const float *beta, int relu, float *save_mean,
+                            float *save_min, float *save_max, const ColStatParts &parts, qbp_qparams *qp8_out,
+                            float4 *fold, cudaStream_t st);
+// Optional tail of a product's epilogue: per-column normalisation (fold: (mean, scale, gamma, beta) per output
+// column, as rangebn_fold_from_parts leaves them), ReLU, and 8-bit codes of the result with parameters *rq
+// (q [M x N], row_sums [M] nullable).  keep_terms: the zero-point term kernels ran for the same operands in the
+// call just before on the same workspace and are not run again.
+struct EpilogueTail { const float4 *fold; int relu; const qbp_qparams *rq; int8_t *q; int32_t *row_sums; int keep_terms; };
+
 // ext_status (here and below; nullable): a status word the caller owns and has cleared -- the product raises it when
 // a bounded wait runs out and never clears it; NULL: the word is the first int of `ws`, cleared by the call itself.
 int conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
                  const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, ColStatParts *stats,
-                 int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);
+                 int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const EpilogueTail *tail = nullptr);
 int gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
                  const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const qbp_epilogue *ep,
                  int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);

@@ -15,15 +15,6 @@
 
 namespace qbp {
 
-// xhat and y of one element; the order of operations is part of the contract.
-__device__ __forceinline__ float bn_xhat(float x, float mu, float s) { return __fmul_rn(__fsub_rn(x, mu), s); }
-__device__ __forceinline__ float bn_y(float xh, float g, float b) { return __fadd_rn(__fmul_rn(g, xh), b); }
-__device__ __forceinline__ float bn_scale(float lo, float hi, float Cn)
-{
-    float r = __fsub_rn(hi, lo);
-    return r > 0.0f ? __fdiv_rn(1.0f, __fmul_rn(Cn, r)) : 0.0f;
-}
-
 // ---------------------------------------------------------------- forward
 template <int VEC>
 __global__ void __launch_bounds__(kScanThreads) bn_stats_kernel(const float *__restrict__ x, int64_t rows, int C, int tw,
@@ -209,12 +200,14 @@ __global__ void __launch_bounds__(256) bn_out_range_kernel(const float *__restri
                                                            const float *__restrict__ vmax,
                                                            const float *__restrict__ gamma,
                                                            const float *__restrict__ beta, int C, float Cn, int relu,
-                                                           qbp_qparams *__restrict__ out, qbp_qparams *__restrict__ qp8_out)
+                                                           qbp_qparams *__restrict__ out, qbp_qparams *__restrict__ qp8_out,
+                                                           float4 *__restrict__ fold)
 {
     float lo = INFINITY, hi = -INFINITY;
     for (int c = threadIdx.x; c < C; c += 256) {
         float s = bn_scale(vmin[c], vmax[c], Cn);
         float g = gamma ? gamma[c] : 1.0f, b = beta ? beta[c] : 0.0f;
+        if (fold) fold[c] = make_float4(mean[c], s, g, b);      // what a product's epilogue needs to normalise a column
         float a = bn_y(bn_xhat(vmin[c], mean[c], s), g, b);
         float z = bn_y(bn_xhat(vmax[c], mean[c], s), g, b);
         if (relu) { a = fmaxf(a, 0.0f); z = fmaxf(z, 0.0f); }
@@ -477,7 +470,7 @@ static int bn_fwd_apply_launch(const float *x, int64_t n_rows, int64_t n_stat, i
     if (out_range || requant) {
         QBP_TRACE_BEGIN(st);
         bn_out_range_kernel<<<1, 256, 0, st>>>(save_mean, save_min, save_max, gamma, beta, (int)C, Cn, relu, out_range,
-                                               requant ? rq->qp : nullptr);
+                                               requant ? rq->qp : nullptr, nullptr);
         QBP_LAUNCH_OK("bn_out_range_kernel");
     }
     BnRequant R{nullptr, nullptr, nullptr, 1};
@@ -575,6 +568,26 @@ extern "C" __attribute__((visibility("default"))) int qbp_rangebn_fwd_apply(cons
     bn_mean_from_sum_kernel<<<(int)((C + 255) / 256), 256, 0, st>>>(col_sum, col_min, col_max, (int)C, n_stat, save_mean, save_min, save_max);
     QBP_LAUNCH_OK("bn_mean_from_sum_kernel");
     return bn_fwd_apply_launch(x, n_rows, n_stat, C, gamma, beta, relu, y, save_mean, save_min, save_max, out_range, rq, st);
+}
+
+// The statistics half of the recompute fusion (a convolution run twice: once for the statistics, once to write
+// the normalised output as 8-bit codes): from the partials the first run left, the saved statistics, the 8-bit
+// parameters of the output and, per channel, (mean, scale, gamma, beta) for the second run's epilogue.
+int qbp::rangebn_fold_from_parts(int64_t n, int64_t C, const float *gamma, const float *beta, int relu, float *save_mean,
+                                 float *save_min, float *save_max, const ColStatParts &parts, qbp_qparams *qp8_out,
+                                 float4 *fold, cudaStream_t st)
+{
+    if (!save_mean || !save_min || !save_max || !parts.lo || !parts.hi || !parts.sum || parts.rows <= 0 || !qp8_out || !fold)
+        return fail(QBP_ERR_INVALID_ARG, "rangebn: NULL argument");
+    if (n < 2 || C <= 0) return fail(QBP_ERR_INVALID_ARG, "rangebn: needs n >= 2 rows");
+    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
+    QBP_TRACE_BEGIN(st);
+    bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(parts.lo, parts.hi, parts.sum, parts.rows, (int)C, n, save_mean, save_min, save_max, nullptr);
+    QBP_LAUNCH_OK("bn_stats_finalize_kernel");
+    QBP_TRACE_BEGIN(st);
+    bn_out_range_kernel<<<1, 256, 0, st>>>(save_mean, save_min, save_max, gamma, beta, (int)C, Cn, relu, nullptr, qp8_out, fold);
+    QBP_LAUNCH_OK("bn_out_range_kernel");
+    return QBP_OK;
 }
 
 // Forward from per-column partials of x that its producer left (rows of [C]: sum, min, max), without a statistics

@@ -245,7 +245,9 @@ def _g16(shape, seed):
     return random_codes(shape, seed, -32768, 32767, np.int16)
 
 
-WGRADS = [(128, 128, 128), (64, 128, 256), (1000, 64, 64), (70000, 32, 48), (4096, 256, 384), (130, 16, 16)]
+# (the last four run on CTA pairs: ragged in every dimension, a short and a long reduction)
+WGRADS = [(128, 128, 128), (64, 128, 256), (1000, 64, 64), (70000, 32, 48), (4096, 256, 384), (130, 16, 16),
+          (1000, 272, 400), (520, 528, 256), (2064, 1040, 784), (4096, 2304, 512)]
 
 
 @pytest.mark.parametrize("M,N,K", WGRADS)
@@ -268,6 +270,18 @@ def test_wgrad_long_reduction_extreme_codes(B):
     acc, _, ws = B.qbp_wgrad_s16(to_dev(X), _qp(B, 1, 127), to_dev(hi), to_dev(lo), _qp(B, 1, 0), want_acc=True, want_out=False)
     assert B.status_word(ws) == 0
     assert np.all(to_host(acc) == (-255) * (32767 - 32768) * (M // 2))
+
+
+def test_wgrad_pair_kernel_longest_reduction_extreme_codes(B):
+    """65536 rows, the most one CTA pair accumulates in int32: every low-limb product at 128 * 255, every high-limb
+    product at 128 * 128; the int64 combination must still be exact."""
+    M, N, K = 65536, 256, 256
+    X = np.full((M, K), -128, np.int8); G = np.full((M, N), -32513, np.int16)        # hi = -128, lo = 255
+    hi, lo = O.limb_split(G)
+    assert hi.min() == hi.max() == -128 and lo.min() == lo.max() == 255
+    acc, _, ws = B.qbp_wgrad_s16(to_dev(X), _qp(B, 1, 0), to_dev(hi), to_dev(lo), _qp(B, 1, 0), want_acc=True, want_out=False)
+    assert B.status_word(ws) == 0
+    assert np.all(to_host(acc) == (-128) * (-32513) * M)
 
 
 WCONVS = [(2, 8, 8, 64, 64, 1), (2, 8, 8, 64, 64, 3), (3, 10, 12, 32, 96, 3), (2, 14, 14, 128, 256, 3),
