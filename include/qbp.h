@@ -236,20 +236,39 @@ int qbp_dequant_s64(const int64_t *acc, int64_t count, const qbp_qparams *qa, co
  * ---------------------------------------------------------------------- */
 size_t qbp_gemm_s8_workspace_bytes(int64_t M, int64_t N, int64_t K);
 
-/* Optional extra work of a product's epilogue.  Section 3's Range BN needs
- * the mean, minimum and maximum of every output channel of the layer; they
- * are taken here from the fp32 outputs as they are written, so that the
- * normalisation that follows needs no statistics pass of its own.
- * col_sum (double), col_min, col_max: [N] each (device), all three or none;
- * they receive the sum / minimum / maximum over the M rows of each column
- * of C (of each output channel over all positions for a convolution).
- * Needs C (out) non-NULL and N <= QBP_EPILOGUE_MAX_COLUMNS, else
- * QBP_ERR_UNSUPPORTED_SHAPE.  ep == NULL: none of it. */
+/* Optional extra work of a product's epilogue.
+ *
+ * (1) Statistics.  Section 3's Range BN needs the mean, minimum and maximum
+ * of every output channel of the layer; they are taken here from the fp32
+ * outputs as they are written, so that the normalisation that follows needs
+ * no statistics pass of its own.  col_sum (double), col_min, col_max: [N]
+ * each (device), all three or none; they receive the sum / minimum / maximum
+ * over the M rows of each column of C (of each output channel over all
+ * positions for a convolution).  N <= QBP_EPILOGUE_MAX_COLUMNS, else
+ * QBP_ERR_UNSUPPORTED_SHAPE.
+ *
+ * (2) ReLU and requantisation, for a product whose output feeds the next
+ * layer directly (no Range BN in between; Appendix B's quantiser with
+ * clamping values the caller knows beforehand, e.g. from the previous step):
+ * relu != 0 rectifies the fp32 output (C then holds the rectified values);
+ * with q_out the 8-bit codes of that output under the clamping values of
+ * requant_range (its vmin / vmax; nearest rounding; values beyond the clamp
+ * saturate) are written to q_out [M x N], their parameters to qp_out and,
+ * if row_sums_out is given, each row's sum of stored codes to row_sums_out
+ * [M].  C may then be NULL.  Not together with (1); runs on the single-CTA
+ * kernel.
+ *
+ * ep == NULL: none of it. */
 #define QBP_EPILOGUE_MAX_COLUMNS 256
 typedef struct qbp_epilogue {
     double *col_sum;
     float *col_min;
     float *col_max;
+    int32_t relu;
+    const qbp_qparams *requant_range;
+    int8_t *q_out;
+    qbp_qparams *qp_out;
+    int32_t *row_sums_out;
 } qbp_epilogue;
 
 int qbp_gemm_s8(int transA, int transB, int64_t M, int64_t N, int64_t K,
@@ -427,7 +446,16 @@ int qbp_layer_fwd(const qbp_layer_desc *L, const float *x, const float *w,
  *       sums are computed here.
  *   out (nullable): also write the 8-bit codes of this layer's output for the
  *       next layer (see qbp_requant); y may then be NULL.
- * With in == NULL and out == NULL this is qbp_layer_fwd. */
+ * With in == NULL and out == NULL this is qbp_layer_fwd.
+ *
+ * Recompute instead of store (forward only; Section 7 argues the method's
+ * gain in memory and bandwidth): with saved->z == NULL, y == NULL and out
+ * given, a convolution layer of at most QBP_EPILOGUE_MAX_COLUMNS output
+ * channels never writes the fp32 output of its product.  The convolution is
+ * run twice: the first run leaves only the per-channel statistics of the
+ * Range BN, the second normalises, rectifies and requantises in its epilogue
+ * and writes one byte per output.  The codes and statistics are the same, bit
+ * for bit, as with z kept; qbp_layer_bwd needs z and refuses such a record. */
 int qbp_layer_fwd_chained(const qbp_layer_desc *L, const float *x, const qbp_requant *in,
                           const float *w, const float *gamma, const float *beta,
                           float *y, const qbp_requant *out, const qbp_layer_ctx *saved,

@@ -256,30 +256,41 @@ def qbp_dequant_s64(acc, qa, qb, out=None):
 
 # ------------------------------------------------------------------- products
 class Epilogue(C.Structure):
-    """qbp_epilogue: device pointers [N] that receive the per-column sum / min / max of the fp32 output."""
-    _fields_ = [("col_sum", C.c_void_p), ("col_min", C.c_void_p), ("col_max", C.c_void_p)]
+    """qbp_epilogue: device pointers [N] that receive the per-column sum / min / max of the fp32 output, and / or
+    the ReLU + requantisation of the output (clamping values requant_range -> codes q_out, parameters qp_out, each
+    row's code sum row_sums_out)."""
+    _fields_ = [("col_sum", C.c_void_p), ("col_min", C.c_void_p), ("col_max", C.c_void_p), ("relu", C.c_int32),
+                ("requant_range", C.c_void_p), ("q_out", C.c_void_p), ("qp_out", C.c_void_p), ("row_sums_out", C.c_void_p)]
 
 
-def _epilogue(col_stats, n, device):
-    """col_stats: None, True (allocate), or a (sum f64, min f32, max f32) triple of device tensors."""
-    if not col_stats:
+def _epilogue(col_stats, n, device, relu=False, requant=None):
+    """col_stats: None, True (allocate), or a (sum f64, min f32, max f32) triple of device tensors.
+    requant: None or (range qparams, q int8 [M x N], qp_out, row_sums int32 [M] or None)."""
+    if not col_stats and not relu and requant is None:
         return None, None
-    if col_stats is True:
-        col_stats = (torch.empty(n, dtype=torch.float64, device=device), torch.empty(n, dtype=torch.float32, device=device),
-                     torch.empty(n, dtype=torch.float32, device=device))
-    ep = Epilogue(col_stats[0].data_ptr(), col_stats[1].data_ptr(), col_stats[2].data_ptr())
+    ep = Epilogue()
+    if col_stats:
+        if col_stats is True:
+            col_stats = (torch.empty(n, dtype=torch.float64, device=device), torch.empty(n, dtype=torch.float32, device=device),
+                         torch.empty(n, dtype=torch.float32, device=device))
+        ep.col_sum, ep.col_min, ep.col_max = (t.data_ptr() for t in col_stats)
+    ep.relu = int(bool(relu))
+    if requant is not None:
+        rng, q, qp, rs = requant
+        ep.requant_range, ep.q_out, ep.qp_out = rng.data_ptr(), q.data_ptr(), qp.data_ptr()
+        ep.row_sums_out = rs.data_ptr() if rs is not None else None
     return ep, col_stats
 
 
 def qbp_gemm_s8(A, qa, B, qb, transA=False, transB=False, want_acc=False, want_out=True, acc_out=None, out=None, ws=None,
-                col_stats=None):
+                col_stats=None, relu=False, requant=None):
     if transA: K, M = A.shape
     else:      M, K = A.shape
     N = B.shape[0] if transB else B.shape[1]
     if want_acc and acc_out is None: acc_out = torch.empty((M, N), dtype=torch.int32, device=A.device)
     if want_out and out is None: out = torch.empty((M, N), dtype=torch.float32, device=A.device)
     if ws is None: ws = workspace(lib.qbp_gemm_s8_workspace_bytes(M, N, K), A.device)
-    ep, stats = _epilogue(col_stats, N, A.device)
+    ep, stats = _epilogue(col_stats, N, A.device, relu, requant)
     _check(lib.qbp_gemm_s8(int(transA), int(transB), C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A), _ptr(qa),
                            _ptr(B), _ptr(qb), _ptr(acc_out), _ptr(out), C.byref(ep) if ep else None, _ptr(ws),
                            C.c_size_t(ws.numel()), _stream()))
@@ -291,12 +302,12 @@ def conv_desc(N, H, W, C_in, K, R, S, stride=1, pad=0) -> ConvDesc:
 
 
 def qbp_conv_s8_implicit(mode, d: ConvDesc, inp, q_in, w, q_w, want_acc=False, want_out=True, acc_out=None, out=None, ws=None,
-                         col_stats=None):
+                         col_stats=None, relu=False, requant=None):
     shape = (d.N, d.H, d.W, d.K) if mode == QBP_CONV_FPROP else (d.N, d.H, d.W, d.C)
     if want_acc and acc_out is None: acc_out = torch.empty(shape, dtype=torch.int32, device=inp.device)
     if want_out and out is None: out = torch.empty(shape, dtype=torch.float32, device=inp.device)
     if ws is None: ws = workspace(lib.qbp_conv_s8_workspace_bytes(mode, C.byref(d)), inp.device)
-    ep, stats = _epilogue(col_stats, shape[3], inp.device)
+    ep, stats = _epilogue(col_stats, shape[3], inp.device, relu, requant)
     _check(lib.qbp_conv_s8_implicit(mode, C.byref(d), _ptr(inp), _ptr(q_in), _ptr(w), _ptr(q_w), _ptr(acc_out),
                                     _ptr(out), C.byref(ep) if ep else None, _ptr(ws), C.c_size_t(ws.numel()), _stream()))
     return (acc_out, out, ws, stats) if col_stats else (acc_out, out, ws)

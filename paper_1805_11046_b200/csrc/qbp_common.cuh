@@ -144,20 +144,20 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, float zp_
 // ceil(t * 2^16) = f * 2^16 + ceil(frac * 2^16), so adding 0xFFFF - d carries into bit 16 exactly when the code
 // rounds up.  The conversion saturates negative t to 0 (code 0, as the clamp gives) and the minimum with
 // L * 2^16 is the clamp at the top (then nothing can carry).
+// The caller passes inv_scale and zp_u already multiplied by 2^16: scaling by a power of two commutes with the
+// rounding of the fused multiply-add, so fma(x, inv * 2^16, zp * 2^16) is exactly 2^16 * fma(x, inv, zp).
 // 8 bits: the code is byte 2 of the result; the draw is the high half of rnd.
-__device__ __forceinline__ uint32_t quantize_sr8_byte2(float x, float inv_scale, float zp_u, uint32_t rnd)
+__device__ __forceinline__ uint32_t quantize_sr8_byte2(float x, float inv_scale_2p16, float zp_u_2p16, uint32_t rnd)
 {
-    const float t = __fmaf_rn(x, inv_scale, zp_u);
     uint32_t tc;
-    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmul_rn(t, 65536.0f)));
+    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmaf_rn(x, inv_scale_2p16, zp_u_2p16)));
     return min(tc, 0x00FF0000u) + ((~rnd) >> 16);
 }
 // 16 bits: the code is the upper half of the result (high byte = byte 3, low byte = byte 2); the draw is the low half of rnd.
-__device__ __forceinline__ uint32_t quantize_sr16_top_half(float x, float inv_scale, float zp_u, uint32_t rnd)
+__device__ __forceinline__ uint32_t quantize_sr16_top_half(float x, float inv_scale_2p16, float zp_u_2p16, uint32_t rnd)
 {
-    const float t = __fmaf_rn(x, inv_scale, zp_u);
     uint32_t tc;
-    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmul_rn(t, 65536.0f)));
+    asm("cvt.rpi.sat.u32.f32 %0, %1;" : "=r"(tc) : "f"(__fmaf_rn(x, inv_scale_2p16, zp_u_2p16)));
     return min(tc, 0xFFFF0000u) + ((~rnd) & 0xFFFFu);
 }
 

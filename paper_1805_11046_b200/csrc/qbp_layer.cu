@@ -79,9 +79,27 @@ static size_t colstat_cells(const LayerShape &s) { return epilogue_stats(s) ? (s
 static size_t chained_bytes(const LayerShape &s)
 {
     // ... and the per-channel (sum, min, max) partials of the layer output that the convolution's epilogue leaves
-    // for the Range BN forward
+    // for the Range BN forward, and the per-channel constants of the normalisation for the recompute fusion
     return align_up(sizeof(int32_t) * (size_t)s.rows, 256) + align_up(sizeof(float2) * rangebn_range_parts_capacity(s.cout), 256) +
-           2 * align_up(sizeof(float) * colstat_cells(s), 256) + align_up(sizeof(double) * colstat_cells(s), 256);
+           2 * align_up(sizeof(float) * colstat_cells(s), 256) + align_up(sizeof(double) * colstat_cells(s), 256) +
+           align_up(sizeof(float4) * (size_t)s.cout, 256);
+}
+
+// Recompute instead of store (motivated by Section 7's memory and bandwidth argument): convolution -> Range BN
+// (+ReLU) -> 8-bit codes for the next layer without ever writing the fp32 output of the product.  The
+// convolution runs twice: the first run leaves only the per-channel statistics (its epilogue stores nothing), the
+// second run normalises, rectifies and requantises in its epilogue and writes one byte per output.
+static int conv_rangebn_recompute(const qbp_conv_desc *d, const int8_t *x_codes, const qbp_qparams *qx, const int32_t *in_sums,
+                                  const int8_t *w_codes, const qbp_qparams *qw, const float *gamma, const float *beta, int relu,
+                                  float *save_mean, float *save_min, float *save_max, const qbp_requant *out,
+                                  ColStatParts parts, float4 *fold, int *status, void *ws, size_t scratch, cudaStream_t st)
+{
+    const int64_t rows = (int64_t)d->N * d->H * d->W;
+    int rc = conv_s8_impl(QBP_CONV_FPROP, d, x_codes, qx, w_codes, qw, nullptr, nullptr, in_sums, &parts, status, ws, scratch, st);
+    if (rc) return rc;
+    if ((rc = rangebn_fold_from_parts(rows, d->K, gamma, beta, relu, save_mean, save_min, save_max, parts, out->qp, fold, st))) return rc;
+    const EpilogueTail tail{fold, relu, out->qp, out->q, out->row_sums, 1};
+    return conv_s8_impl(QBP_CONV_FPROP, d, x_codes, qx, w_codes, qw, nullptr, nullptr, in_sums, nullptr, status, ws, scratch, st, &tail);
 }
 
 }  // namespace qbp
@@ -120,9 +138,14 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
         return fail(QBP_ERR_INVALID_ARG, "layer_fwd: exactly one of x (fp32 input) and in (input already quantised) is needed");
     if (!y && !out) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: neither y nor 8-bit output codes wanted");
     if (out && (!out->q || !out->qp)) return fail(QBP_ERR_INVALID_ARG, "layer_fwd: the output record needs q and qp");
-    if (!saved->x_codes || !saved->qx || !saved->w_codes || !saved->qw || !saved->z || !saved->save_mean ||
+    if (!saved->x_codes || !saved->qx || !saved->w_codes || !saved->qw || !saved->save_mean ||
         !saved->save_min || !saved->save_max)
         return fail(QBP_ERR_INVALID_ARG, "layer_fwd: the saved-state record has a NULL buffer");
+    // saved->z == NULL: the fp32 output of the product is not kept (forward only): the convolution is run twice instead
+    const bool recompute = saved->z == nullptr;
+    if (recompute && !(s.conv && epilogue_stats(s) && out && !y))
+        return fail(QBP_ERR_INVALID_ARG, "layer_fwd: without saved->z the layer must be a convolution of at most %d output "
+                    "channels that writes 8-bit codes only (out given, y NULL)", QBP_EPILOGUE_MAX_COLUMNS);
     if (in && (in->q != saved->x_codes || in->qp != saved->qx))
         return fail(QBP_ERR_INVALID_ARG, "layer_fwd: in->q / in->qp must be the layer's saved x_codes / qx");
     if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
@@ -160,6 +183,11 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
         parts.hi = reinterpret_cast<float *>(base + align_up(sizeof(float) * colstat_cells(s), 256));
         parts.sum = reinterpret_cast<double *>(base + 2 * align_up(sizeof(float) * colstat_cells(s), 256));
     }
+    if (recompute) {
+        float4 *fold = reinterpret_cast<float4 *>(reinterpret_cast<char *>(parts.sum) + align_up(sizeof(double) * colstat_cells(s), 256));
+        return conv_rangebn_recompute(&L->conv, saved->x_codes, saved->qx, in_sums, saved->w_codes, saved->qw, gamma, beta, L->relu,
+                                      saved->save_mean, saved->save_min, saved->save_max, out, parts, fold, status, ws, scratch, st);
+    }
     if (s.conv)
         rc = conv_s8_impl(QBP_CONV_FPROP, &L->conv, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr, saved->z,
                           in_sums, parts.sum ? &parts : nullptr, status, ws, scratch, st);
@@ -188,8 +216,8 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
         return fail(QBP_ERR_WORKSPACE, "layer_bwd: workspace of %zu bytes needed, %zu given",
                     qbp_layer_workspace_bytes(L), ws_bytes);
-    if (!saved->g || !saved->g8 || !saved->qg8 || !saved->g_hi || !saved->g_lo || !saved->qg16)
-        return fail(QBP_ERR_INVALID_ARG, "layer_bwd: the saved-state record has a NULL gradient buffer");
+    if (!saved->g || !saved->g8 || !saved->qg8 || !saved->g_hi || !saved->g_lo || !saved->qg16 || !saved->z)
+        return fail(QBP_ERR_INVALID_ARG, "layer_bwd: the saved-state record has a NULL buffer (the backward pass needs z and the gradient buffers)");
     const size_t scratch = step_scratch_bytes(L, s);
     float *g = saved->g;
     int8_t *g8 = saved->g8, *ghi = saved->g_hi;

@@ -367,6 +367,9 @@ __device__ __forceinline__ void issue_stage(const MmaParams &P, uint32_t a_lo, u
 // operand bytes fetched per multiply-add against 128 x 256).  When two sets of accumulators fit in
 // tensor memory they are used in turn, so that the epilogues of earlier tiles overlap the MMAs of later ones.
 // Epilogue: tcgen05.ld -> zero-point terms -> fp32 -> swizzled staging slab -> TMA store per warp.
+// TAIL: the instance with the optional normalise / ReLU / requantise tail of the epilogue (the plain instance, which the
+// bandwidth-bound convolutions of a training step use, carries none of it).
+template <bool TAIL>
 __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_constant__ MmaParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -544,17 +547,16 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         const int bar_id = P.msub == 2 ? 1 : 1 + group, bar_cnt = P.msub == 2 ? 256 : 128;
         const int gt = P.msub == 2 ? threadIdx.x - 64 : (threadIdx.x - 64) & 127;     // thread index within the barrier group
         int32_t *region = s_cterm + (P.cterm_all || P.msub == 2 ? 0 : group * P.ncls * P.bn);
-        if (P.cterm_all || P.ep_fold) {
+        if (P.cterm_all || (TAIL && P.ep_fold)) {
             // the whole column-term table fits: fill it once (and the per-column constants of the normalisation)
             if (P.cterm_all)
                 for (int i = threadIdx.x - 64; i < P.ncls * (int)P.N; i += 32 * P.ewarps) s_cterm[i] = __ldg(P.colterm + i);
-            if (P.ep_fold)
+            if (TAIL && P.ep_fold)
                 for (int i = threadIdx.x - 64; i < (int)P.N; i += 32 * P.ewarps) s_fold[i] = __ldg(P.ep_fold + i);
             named_barrier(4, 32 * P.ewarps);
         }
         float rq_inv = 0.0f, rq_zp = 0.0f;
-        if (P.ep_q) { rq_inv = __fdiv_rn(1.0f, P.ep_rq->scale); rq_zp = (float)(P.ep_rq->zero_point + 128); }
-        const bool tail = P.ep_fold || P.ep_relu || P.ep_q;
+        if (TAIL && P.ep_q) { rq_inv = __fdiv_rn(1.0f, P.ep_rq->scale); rq_zp = (float)(P.ep_rq->zero_point + 128); }
 
         // where this thread's accumulator row of a tile goes
         struct RowInfo { int64_t m; bool valid, slab_in; int cls, sx, sy, sz; };
@@ -610,6 +612,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
             if (!timed_out) {
                 tc_fence_after();
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * buf_cols + (uint32_t)(sub * P.bn);
+                int row_code_sum = 0;                   // of this thread's output row's 8-bit codes (one column tile)
                 for (int c = 0; c < nchunks; ++c) {
                     const int c0 = c * 32;
                     uint32_t r[32];
@@ -642,29 +645,29 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                         }
                     }
                     // the fp32 value of the row's 32 outputs: dequantised, then (optionally) normalised and rectified
-                    float v[32];
+                    float v[TAIL ? 32 : 1];
+                    if (TAIL) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __fmul_rn((float)acc[j], scale);
-                    if (tail) {
+                        for (int j = 0; j < (TAIL ? 32 : 1); ++j) v[j] = __fmul_rn((float)acc[j], scale);
                         if (P.ep_fold) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
+                            for (int j = 0; j < (TAIL ? 32 : 1); ++j) {
                                 const float4 f = s_fold[o.n0 + c0 + (j < lim ? j : 0)];       // (mean, scale, gamma, beta)
                                 v[j] = bn_y(bn_xhat(v[j], f.x, f.y), f.z, f.w);
                             }
                         }
                         if (P.ep_relu) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+                            for (int j = 0; j < (TAIL ? 32 : 1); ++j) v[j] = fmaxf(v[j], 0.0f);
                         }
                         if (P.ep_q) {
                             // 8-bit codes of the row's 32 values: two 16-byte stores (the row's bytes are contiguous)
                             uint32_t w8[8];
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
+                            for (int j = 0; j < (TAIL ? 32 : 1); j += 4) {
                                 uint32_t c4[4];
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) c4[e] = (uint32_t)quantize_code<false>(v[j + e], rq_inv, rq_zp, 255.0f, 0u);
+                                for (int e = 0; e < 4; ++e) c4[e] = (uint32_t)quantize_code<false>(v[TAIL ? j + e : 0], rq_inv, rq_zp, 255.0f, 0u);
                                 w8[j >> 2] = (c4[0] | (c4[1] << 8) | (c4[2] << 16) | (c4[3] << 24)) ^ 0x80808080u;
                             }
                             if (ri.valid) {
@@ -693,7 +696,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                         uint8_t *rowp = slab + lane * 128;
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4 *>(rowp + (((j >> 2) ^ (lane & 7)) << 4)) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            *reinterpret_cast<float4 *>(rowp + (((j >> 2) ^ (lane & 7)) << 4)) =
+                                TAIL ? make_float4(v[TAIL ? j : 0], v[TAIL ? j + 1 : 0], v[TAIL ? j + 2 : 0], v[TAIL ? j + 3 : 0])
+                                     : make_float4(__fmul_rn((float)acc[j], scale), __fmul_rn((float)acc[j + 1], scale),
+                                                   __fmul_rn((float)acc[j + 2], scale), __fmul_rn((float)acc[j + 3], scale));
                         fence_proxy_async();
                         __syncwarp();
                         if (lane == 0 && ri.slab_in && P.out) {
@@ -732,6 +738,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                         }
                     }
                 }
+                if (TAIL && P.ep_rowsum && ri.valid) P.ep_rowsum[ri.m] = row_code_sum;
             }
             o = o_next; ri = ri_next; rterm = rterm_next;
             buf += (uint32_t)lt_step;
@@ -888,13 +895,40 @@ static size_t colstat_ws_bytes(int64_t N)
     return align_up(cells * sizeof(float), 256) * 2 + align_up(cells * sizeof(double), 256);
 }
 
-static int check_epilogue(const char *who, const qbp_epilogue *ep, const float *out, int64_t N, bool &wanted)
+// Parameters of the requantisation in a product's epilogue from the caller's clamping values.
+__global__ void epilogue_qparams_kernel(const qbp_qparams *__restrict__ range, qbp_qparams *__restrict__ qp8)
+{
+    *qp8 = make_qparams(range->vmin, range->vmax, 8);
+}
+
+// What the caller's epilogue record asks for: column statistics (wanted) and / or the ReLU / requantisation tail.
+static int check_epilogue(const char *who, const qbp_epilogue *ep, const float *out, int64_t N, bool &wanted, EpilogueTail &tail,
+                          bool &has_tail)
 {
     wanted = ep && (ep->col_sum || ep->col_min || ep->col_max);
-    if (!wanted) return QBP_OK;
-    if (!ep->col_sum || !ep->col_min || !ep->col_max) return fail(QBP_ERR_INVALID_ARG, "%s: the epilogue needs col_sum, col_min and col_max together", who);
-    if (!out) return fail(QBP_ERR_INVALID_ARG, "%s: column statistics need the fp32 output", who);
-    if (N > QBP_EPILOGUE_MAX_COLUMNS) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "%s: column statistics for at most %d columns", who, QBP_EPILOGUE_MAX_COLUMNS);
+    has_tail = ep && (ep->relu || ep->q_out);
+    tail = EpilogueTail{nullptr, 0, nullptr, nullptr, nullptr, 0};
+    if (wanted) {
+        if (!ep->col_sum || !ep->col_min || !ep->col_max) return fail(QBP_ERR_INVALID_ARG, "%s: the epilogue needs col_sum, col_min and col_max together", who);
+        if (!out) return fail(QBP_ERR_INVALID_ARG, "%s: column statistics need the fp32 output", who);
+        if (N > QBP_EPILOGUE_MAX_COLUMNS) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "%s: column statistics for at most %d columns", who, QBP_EPILOGUE_MAX_COLUMNS);
+        if (has_tail) return fail(QBP_ERR_INVALID_ARG, "%s: column statistics and ReLU / requantisation exclude one another", who);
+    }
+    if (has_tail) {
+        if (ep->q_out && (!ep->requant_range || !ep->qp_out)) return fail(QBP_ERR_INVALID_ARG, "%s: requantisation needs requant_range and qp_out", who);
+        if (!ep->q_out && !out) return fail(QBP_ERR_INVALID_ARG, "%s: ReLU without an output", who);
+        if (ep->q_out && !aligned16(ep->q_out)) return fail(QBP_ERR_INVALID_ARG, "%s: q_out must be 16-byte aligned", who);
+        tail.relu = ep->relu ? 1 : 0; tail.rq = ep->qp_out; tail.q = ep->q_out; tail.row_sums = ep->q_out ? ep->row_sums_out : nullptr;
+    }
+    return QBP_OK;
+}
+
+static int launch_epilogue_qparams(const qbp_epilogue *ep, cudaStream_t st)
+{
+    if (!ep->q_out) return QBP_OK;
+    QBP_TRACE_BEGIN(st);
+    epilogue_qparams_kernel<<<1, 1, 0, st>>>(ep->requant_range, ep->qp_out);
+    QBP_LAUNCH_OK("epilogue_qparams_kernel");
     return QBP_OK;
 }
 
@@ -921,8 +955,10 @@ static uint32_t fixed_smem(MmaParams &P)
                                            : (size_t)(P.msub == 1 ? P.egroups : 1) * P.ncls * P.bn * sizeof(int32_t);
     P.iter_entries = P.mode == MODE_GEMM ? 0 : (int)align_up((size_t)P.k_iters, 64);
     P.cterm_span = (uint32_t)align_up(cterm_bytes, 1024);
-    const uint32_t stat_bytes = P.st_sum ? (uint32_t)align_up((size_t)P.ewarps * P.N * sizeof(ColStat), 1024) : 0u;
-    return 2048u + (uint32_t)P.ewarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + P.cterm_span + stat_bytes;
+    P.stat_span = P.st_sum ? (uint32_t)align_up((size_t)P.ewarps * P.N * sizeof(ColStat), 1024) : 0u;
+    const uint32_t fold_bytes = P.ep_fold ? (uint32_t)align_up((size_t)P.N * sizeof(float4), 1024) : 0u;
+    return 2048u + (uint32_t)P.ewarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + P.cterm_span +
+           P.stat_span + fold_bytes;
 }
 
 // Whether a convolution can run from halo tiles: the whole filter resident beside at least three halo tiles.
@@ -979,14 +1015,17 @@ static int launch_mma(MmaParams &P, int tiles_m, bool clear_status, cudaStream_t
     P.d_tiles_w = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_w);
     P.d_tiles_h = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_h);
     const size_t smem = (size_t)fixed + P.b_res_bytes + (size_t)stages * stage_bytes;
-    static PerDeviceOnce configured;
-    QBP_SMEM_OPT_IN(configured, qbp_mma_kernel, kSmemBudget);
+    const bool tail = P.ep_fold || P.ep_relu || P.ep_q;
+    static PerDeviceOnce configured[2];
+    if (tail) QBP_SMEM_OPT_IN(configured[1], qbp_mma_kernel<true>, kSmemBudget);
+    else      QBP_SMEM_OPT_IN(configured[0], qbp_mma_kernel<false>, kSmemBudget);
     if (clear_status) QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
     // one CTA per SM (its shared-memory ring fills the SM), each walking its share of the tiles
     const int grid = std::min(P.tiles_total, sm_count());
     P.grid = grid;
     QBP_TRACE_BEGIN(st);
-    qbp_mma_kernel<<<grid, kMmaThreads, smem, st>>>(P);
+    if (tail) qbp_mma_kernel<true><<<grid, kMmaThreads, smem, st>>>(P);
+    else      qbp_mma_kernel<false><<<grid, kMmaThreads, smem, st>>>(P);
     QBP_LAUNCH_OK("qbp_mma_kernel");
     return QBP_OK;
 }
@@ -1082,16 +1121,18 @@ int qbp::gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, c
     if (K > 33025) return fail(QBP_ERR_OVERFLOW_K, "gemm_s8: K = %lld exceeds 33025 (255*255*K must fit int32)", (long long)K);
     if (M > INT32_MAX || N > INT32_MAX) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "gemm_s8: extent too large");
     if (!A || !B || !qa || !qb) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: NULL operand");
-    if (!acc_out && !C) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: acc_out and C are both NULL");
+    if (!acc_out && !C && !(ep && ep->q_out)) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: acc_out and C are both NULL");
     if (!aligned16(A) || !aligned16(B) || (C && !aligned16(C)) || (acc_out && !aligned16(acc_out)))
         return fail(QBP_ERR_INVALID_ARG, "gemm_s8: operands must be 16-byte aligned");
     if (!ws || ws_bytes < gemm_ws_bytes(M, N))
         return fail(QBP_ERR_WORKSPACE, "gemm_s8: workspace of %zu bytes needed, %zu given", gemm_ws_bytes(M, N), ws_bytes);
 
-    bool stats = false;
+    bool stats = false, has_tail = false;
+    EpilogueTail tail;
     {
-        const int erc = check_epilogue("gemm_s8", ep, C, N, stats);
+        const int erc = check_epilogue("gemm_s8", ep, C, N, stats, tail, has_tail);
         if (erc) return erc;
+        if (!acc_out && !C && !(has_tail && tail.q)) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: no output wanted");
     }
     WsCarver w(ws, ws_bytes);
     int *status = w.take<int>(1);
@@ -1124,7 +1165,7 @@ int qbp::gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, c
 
     // large products run on CTA pairs (256 x 256 tiles across two SMs); the column statistics are the
     // single-CTA kernel's (at most 256 columns: narrow either way)
-    if (gemm2_eligible(M, N, K) && !stats)
+    if (gemm2_eligible(M, N, K) && !stats && !has_tail)
         return launch_gemm2(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, rowterm, colterm, status, !ext_status, st);
 
     MmaParams P{};
@@ -1165,8 +1206,16 @@ int qbp::gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, c
     P.acc_out = acc_out; P.out = C;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = qa; P.qb = qb; P.status = status;
     if (stats) { P.st_lo = parts.lo; P.st_hi = parts.hi; P.st_sum = parts.sum; }
+    bool fused_row_sums = false;
+    if (has_tail) {
+        if ((rc = launch_epilogue_qparams(ep, st))) return rc;
+        P.ep_relu = tail.relu; P.ep_rq = tail.rq; P.ep_q = tail.q;
+        fused_row_sums = tail.q && tail.row_sums && P.tiles_n == 1;
+        if (fused_row_sums) P.ep_rowsum = tail.row_sums;
+    }
     if ((rc = launch_mma(P, (int)((M + 128 * P.msub - 1) / (128 * P.msub)), !ext_status, st))) return rc;
     if (stats) { parts.rows = P.grid; return finish_epilogue(ep, parts, N, st); }
+    if (has_tail && tail.q && tail.row_sums && !fused_row_sums) return launch_rowsum(tail.q, true, M, N, tail.row_sums, st);
     return QBP_OK;
 }
 
@@ -1181,11 +1230,17 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
                                     const int8_t *wgt, const qbp_qparams *q_w, int32_t *acc_out, float *out,
                                     const qbp_epilogue *ep, void *ws, size_t ws_bytes, void *stream)
 {
-    bool stats = false;
+    bool stats = false, has_tail = false;
+    EpilogueTail tail;
     if (d && ep) {
         const int64_t Nout = mode == QBP_CONV_DGRAD ? d->C : d->K;
-        const int erc = check_epilogue("conv_s8", ep, out, Nout, stats);
+        const int erc = check_epilogue("conv_s8", ep, out, Nout, stats, tail, has_tail);
         if (erc) return erc;
+        if (has_tail) {
+            const int rc = launch_epilogue_qparams(ep, (cudaStream_t)stream);
+            if (rc) return rc;
+            return conv_s8_impl(mode, d, in, q_in, wgt, q_w, acc_out, out, nullptr, nullptr, nullptr, ws, ws_bytes, (cudaStream_t)stream, &tail);
+        }
         if (stats) {
             // the partial rows sit at the end of the workspace, behind what the product itself carves
             if (!conv_supported(d))
@@ -1210,7 +1265,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
 
 int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_qparams *q_in, const int8_t *wgt,
                       const qbp_qparams *q_w, int32_t *acc_out, float *out, const int32_t *in_chan_sum, ColStatParts *stats,
-                      int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st)
+                      int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const EpilogueTail *tail)
 {
     if (!d) return fail(QBP_ERR_INVALID_ARG, "conv_s8: descriptor is NULL");
     if (mode != QBP_CONV_FPROP && mode != QBP_CONV_DGRAD) return fail(QBP_ERR_INVALID_ARG, "conv_s8: bad mode");
@@ -1221,13 +1276,21 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
         return fail(QBP_ERR_OVERFLOW_K, "conv_s8: reduction length exceeds 33025");
     if ((int64_t)d->N * d->H * d->W >= (1ll << 31)) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: 2^31 or more positions");
     if (!in || !wgt || !q_in || !q_w) return fail(QBP_ERR_INVALID_ARG, "conv_s8: NULL operand");
-    if (!acc_out && !out) return fail(QBP_ERR_INVALID_ARG, "conv_s8: acc_out and out are both NULL");
+    const bool want_codes = tail && tail->q;
+    if (!acc_out && !out && !stats && !want_codes) return fail(QBP_ERR_INVALID_ARG, "conv_s8: no output wanted");
     if (!aligned16(in) || !aligned16(wgt) || (out && !aligned16(out)) || (acc_out && !aligned16(acc_out)))
         return fail(QBP_ERR_INVALID_ARG, "conv_s8: operands must be 16-byte aligned");
     if (!ws || ws_bytes < conv_core_ws_bytes(d))
         return fail(QBP_ERR_WORKSPACE, "conv_s8: workspace of %zu bytes needed, %zu given", conv_ws_bytes(d), ws_bytes);
-    if (stats && (!out || (mode == QBP_CONV_DGRAD ? d->C : d->K) > QBP_EPILOGUE_MAX_COLUMNS))
-        return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: column statistics need the fp32 output and at most %d channels", QBP_EPILOGUE_MAX_COLUMNS);
+    if (stats && (mode == QBP_CONV_DGRAD ? d->C : d->K) > QBP_EPILOGUE_MAX_COLUMNS)
+        return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: column statistics for at most %d channels", QBP_EPILOGUE_MAX_COLUMNS);
+    if (tail) {
+        const int n_out = mode == QBP_CONV_DGRAD ? d->C : d->K;
+        if (stats) return fail(QBP_ERR_INVALID_ARG, "conv_s8: column statistics are of the plain output (no epilogue tail)");
+        if (want_codes && (!tail->rq || !aligned16(tail->q))) return fail(QBP_ERR_INVALID_ARG, "conv_s8: 8-bit output needs parameters and a 16-byte aligned buffer");
+        if (tail->fold && n_out > 256)
+            return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: the fused normalisation takes at most 256 output channels");
+    }
 
     const bool dgrad = mode == QBP_CONV_DGRAD;
     const int Cred = dgrad ? d->K : d->C;        // channels reduced over
@@ -1245,25 +1308,28 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     int64_t *wsum = w.take<int64_t>((int64_t)taps * nmax);
 
     int rc = QBP_OK;
-    if (in_chan_sum) chan_sum = const_cast<int32_t *>(in_chan_sum);
-    else if ((rc = launch_rowsum(in, true, pix, Cred, chan_sum, st))) return rc;
-    if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
-    else        rc = launch_colsum(wgt, true, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
-    if (rc) return rc;
-    QBP_TRACE_BEGIN(st);
-    conv_colterm_kernel<<<dim3((Nout + 127) / 128, 16), 128, 0, st>>>(
-        dgrad ? nullptr : (const int32_t *)wsum, dgrad ? (const long long *)wsum : nullptr, Nout, d->R, d->S, d->pad,
-        dgrad ? 1 : 0, q_in, colterm);
-    QBP_LAUNCH_OK("conv_colterm_kernel");
-    QBP_TRACE_BEGIN(st);
-    conv_rowterm_kernel<<<dim3((unsigned)((d->H * d->W + 255) / 256), (unsigned)d->N), 256, 0, st>>>(
-        chan_sum, d->H * d->W, d->H, d->W, make_fastdiv(d->W), d->pad, Cred, q_in, q_w, rowterm);
-    QBP_LAUNCH_OK("conv_rowterm_kernel");
+    if (!(tail && tail->keep_terms)) {
+        if (in_chan_sum) chan_sum = const_cast<int32_t *>(in_chan_sum);
+        else if ((rc = launch_rowsum(in, true, pix, Cred, chan_sum, st))) return rc;
+        if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
+        else        rc = launch_colsum(wgt, true, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
+        if (rc) return rc;
+        QBP_TRACE_BEGIN(st);
+        conv_colterm_kernel<<<dim3((Nout + 127) / 128, 16), 128, 0, st>>>(
+            dgrad ? nullptr : (const int32_t *)wsum, dgrad ? (const long long *)wsum : nullptr, Nout, d->R, d->S, d->pad,
+            dgrad ? 1 : 0, q_in, colterm);
+        QBP_LAUNCH_OK("conv_colterm_kernel");
+        QBP_TRACE_BEGIN(st);
+        conv_rowterm_kernel<<<dim3((unsigned)((d->H * d->W + 255) / 256), (unsigned)d->N), 256, 0, st>>>(
+            chan_sum, d->H * d->W, d->H, d->W, make_fastdiv(d->W), d->pad, Cred, q_in, q_w, rowterm);
+        QBP_LAUNCH_OK("conv_rowterm_kernel");
+    }
 
     MmaParams P{};
     P.mode = dgrad ? MODE_DGRAD : MODE_FPROP;
     P.msub = 1; P.ncls = 16; P.nslab = 1;
     if (stats) { P.st_lo = stats->lo; P.st_hi = stats->hi; P.st_sum = stats->sum; }
+    if (tail) { P.ep_fold = tail->fold; P.ep_relu = tail->relu; P.ep_rq = tail->rq; P.ep_q = tail->q; }
     P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.S = d->S; P.Cred = Cred;
     const uint32_t cb = Cred % 128 == 0 ? 128u : Cred % 64 == 0 ? 64u : 32u;      // reduction bytes per stage row
     P.chunk_bytes = (int)cb;
@@ -1327,7 +1393,11 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     P.idesc = make_idesc(true, true, P.a.major, P.b.major, 128, (uint32_t)P.bn);
     P.acc_out = acc_out; P.out = out;
     P.rowterm = rowterm; P.colterm = colterm; P.qa = q_in; P.qb = q_w; P.status = status;
+    // each row's code sum comes from the epilogue when one column tile holds the whole row, else from a pass over the codes
+    const bool fused_row_sums = want_codes && tail->row_sums && P.tiles_n == 1;
+    if (fused_row_sums) P.ep_rowsum = tail->row_sums;
     if ((rc = launch_mma(P, P.tiles_w * P.tiles_h * tiles_img, !ext_status, st))) return rc;
     if (stats) stats->rows = P.grid;
+    if (want_codes && tail->row_sums && !fused_row_sums) return launch_rowsum(tail->q, true, pix, Nout, tail->row_sums, st);
     return QBP_OK;
 }

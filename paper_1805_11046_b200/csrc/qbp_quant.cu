@@ -381,6 +381,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     if (!PERCH) {
         if (want8) p8 = load_qp(qp8, 8);
         if (want16) p16 = load_qp(qp16, 16);
+        // the stochastic codes are taken in fixed point with 16 fraction bits: fold the factor into the parameters
+        if (SR) { p8.inv *= 65536.0f; p8.zp_u *= 65536.0f; p16.inv *= 65536.0f; p16.zp_u *= 65536.0f; }
     }
     // both copies of a gradient under one tensor id: one Philox block serves the two (disjoint halves of each word)
     const bool one_block = want8 && want16 && id8 == id16;
@@ -421,6 +423,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                     if (PERCH) {
                         if (table) { const float2 t = s_qp[c0 + e]; p8.inv = t.x; p8.zp_u = t.y; }
                         else p8 = load_qp(qp8 + c0 + e, 8);
+                        if (SR) { p8.inv *= 65536.0f; p8.zp_u *= 65536.0f; }
                     }
                     c[e] = SR ? quantize_sr8_byte2(xs[e], p8.inv, p8.zp_u, r[e])
                               : (uint32_t)quantize_code<SR>(xs[e], p8.inv, p8.zp_u, 255.0f, r[e]);
@@ -437,6 +440,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                     if (PERCH) {
                         if (table) { const float2 t = s_qp[cols + c0 + e]; p16.inv = t.x; p16.zp_u = t.y; }
                         else p16 = load_qp(qp16 + c0 + e, 16);
+                        if (SR) { p16.inv *= 65536.0f; p16.zp_u *= 65536.0f; }
                     }
                     // (stochastic: the code sits in the upper half of the word, i.e. bytes 3 and 2)
                     c[e] = SR ? quantize_sr16_top_half(xs[e], p16.inv, p16.zp_u, r[e])
@@ -446,8 +450,15 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                 if (o.q16)
                     reinterpret_cast<uint2 *>(o.q16)[j] = make_uint2(__byte_perm(c[0], c[1], SR ? 0x7632 : 0x5410) ^ 0x80008000u,
                                                                      __byte_perm(c[2], c[3], SR ? 0x7632 : 0x5410) ^ 0x80008000u);
-                if (o.hi) reinterpret_cast<uint32_t *>(o.hi)[j] = (SR ? pack_bytes3(c) : pack_bytes1(c)) ^ 0x80808080u;
-                if (o.lo) reinterpret_cast<uint32_t *>(o.lo)[j] = SR ? pack_bytes2(c) : pack_bytes0(c);
+                if (SR && o.hi && o.lo) {
+                    // (low, low, high, high) bytes of two codes each, then the two words: four permutes for both limbs
+                    const uint32_t t01 = __byte_perm(c[0], c[1], 0x7362), t23 = __byte_perm(c[2], c[3], 0x7362);
+                    reinterpret_cast<uint32_t *>(o.hi)[j] = __byte_perm(t01, t23, 0x7632) ^ 0x80808080u;
+                    reinterpret_cast<uint32_t *>(o.lo)[j] = __byte_perm(t01, t23, 0x5410);
+                } else {
+                    if (o.hi) reinterpret_cast<uint32_t *>(o.hi)[j] = (SR ? pack_bytes3(c) : pack_bytes1(c)) ^ 0x80808080u;
+                    if (o.lo) reinterpret_cast<uint32_t *>(o.lo)[j] = SR ? pack_bytes2(c) : pack_bytes0(c);
+                }
             }
         }
         if (o.rowsum8) {

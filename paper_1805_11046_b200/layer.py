@@ -15,11 +15,12 @@ class QuantizedLayer:
 
     def __init__(self, conv=None, batch=0, in_features=0, out_features=0, relu=False, seed=0,
                  tensor_id8=1, tensor_id16=2, device="cuda", input_from: "QuantizedLayer | None" = None,
-                 emit_codes=False, keep_y=True):
+                 emit_codes=False, keep_y=True, keep_z=True):
         """input_from: the layer whose output feeds this one already quantised (it must have been built with
         emit_codes=True): this layer then owns no input codes of its own and its forward takes no fp32 input.
         emit_codes: the forward also writes the 8-bit codes of the output (and each row's code sum) for the next
-        layer; keep_y=False then leaves the fp32 output unwritten."""
+        layer; keep_y=False then leaves the fp32 output unwritten.  keep_z=False (forward only, with emit_codes and
+        keep_y=False): the fp32 output of the product is not kept either -- the convolution is run twice instead."""
         self.device = torch.device(device)
         d = B.LayerDesc()
         if conv is not None:
@@ -50,9 +51,12 @@ class QuantizedLayer:
             self.out_codes, self.q_out = e(self.z_shape, torch.int8), B.new_qparams(1, dev)
             self.out_row_sums = e((self.rows,), torch.int32)
             self.rq_out = B.requant(self.out_codes, self.q_out, self.out_row_sums)
-        self.z, self.g = e(self.z_shape, torch.float32), e(self.z_shape, torch.float32)
+        assert keep_z or (emit_codes and not keep_y)
+        self.z = e(self.z_shape, torch.float32) if keep_z else None
+        self.g = e(self.z_shape, torch.float32) if keep_z else None
         self.save_mean, self.save_min, self.save_max = (e((self.cout,), torch.float32) for _ in range(3))
-        self.g8, self.ghi, self.glo = e(self.z_shape, torch.int8), e(self.z_shape, torch.int8), e(self.z_shape, torch.uint8)
+        bshape = self.z_shape if keep_z else (0,)          # (no backward pass without z)
+        self.g8, self.ghi, self.glo = e(bshape, torch.int8), e(bshape, torch.int8), e(bshape, torch.uint8)
         assert keep_y or emit_codes
         self.y = e(self.z_shape, torch.float32) if keep_y else None
         self.dx, self.dw = e(self.x_shape, torch.float32), e(self.w_shape, torch.float32)
@@ -63,7 +67,7 @@ class QuantizedLayer:
                         ("z", self.z), ("save_mean", self.save_mean), ("save_min", self.save_min),
                         ("save_max", self.save_max), ("g", self.g), ("g8", self.g8), ("qg8", self.qg8),
                         ("g_hi", self.ghi), ("g_lo", self.glo), ("qg16", self.qg16)):
-            setattr(c, name, t.data_ptr())
+            setattr(c, name, t.data_ptr() if t is not None and t.numel() else None)
         self.ctx = c
         self.gamma = self.beta = None
 

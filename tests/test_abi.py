@@ -40,6 +40,7 @@ def test_struct_layouts_match_the_header():
     assert C.sizeof(binding.ConvDesc) == 36
     assert C.sizeof(binding.LayerDesc) == 36 + 4 + 3 * 8 + 4 + 4 + 8 + 4 + 4
     assert C.sizeof(binding.LayerCtx) == 14 * 8
+    assert C.sizeof(binding.Epilogue) == 8 * 8 and C.sizeof(binding.Requant) == 3 * 8
 
 
 def _err(lib):
@@ -92,14 +93,20 @@ def test_convolution_shapes_outside_the_implementation_are_refused(lib):
 def test_epilogue_statistics_need_all_three_buffers_the_output_and_few_columns(lib):
     from paper_1805_11046_b200.binding import Epilogue
     fake = C.c_void_p(4096); null = C.c_void_p(0); i64 = C.c_int64
-    part = Epilogue(4096, 0, 4096)
+    part = Epilogue(col_sum=4096, col_min=0, col_max=4096)
     assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, fake, C.byref(part), fake,
                            C.c_size_t(1 << 30), null) == -1
-    full = Epilogue(4096, 4096, 4096)
+    full = Epilogue(col_sum=4096, col_min=4096, col_max=4096)
     assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, fake, null, C.byref(full), fake,
                            C.c_size_t(1 << 30), null) == -1              # no fp32 output to take them from
     assert lib.qbp_gemm_s8(0, 0, i64(128), i64(512), i64(128), fake, fake, fake, fake, null, fake, C.byref(full), fake,
                            C.c_size_t(1 << 30), null) == -2              # more than 256 columns
+    both = Epilogue(col_sum=4096, col_min=4096, col_max=4096, relu=1)
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, fake, C.byref(both), fake,
+                           C.c_size_t(1 << 30), null) == -1              # statistics and the ReLU / requantisation tail exclude one another
+    noparams = Epilogue(q_out=4096)
+    assert lib.qbp_gemm_s8(0, 0, i64(128), i64(128), i64(128), fake, fake, fake, fake, null, fake, C.byref(noparams), fake,
+                           C.c_size_t(1 << 30), null) == -1              # requantisation without clamping values
 
 
 def test_workspace_queries_are_pure(lib):

@@ -323,3 +323,37 @@ def test_chained_and_unchained_stacks_agree(B):
         assert np.array_equal(to_host(La.dw), to_host(Lu.dw))
     for wa, wu in zip(A.w, U.w):
         assert np.array_equal(to_host(wa), to_host(wu))
+
+
+# ------------------------------------------------ recompute instead of store: conv -> Range BN -> ReLU -> 8-bit codes
+@pytest.mark.parametrize("batch,hw,cin,cout", [(4, 14, 64, 64), (3, 9, 32, 96), (2, 20, 128, 32), (256, 56, 64, 64)])
+def test_recompute_fusion_writes_the_same_codes_without_storing_the_product(B, batch, hw, cin, cout):
+    """The convolution run twice (statistics only, then normalise + ReLU + requantise in the epilogue) must leave,
+    bit for bit, the codes, parameters, row sums and saved statistics of the path that stores the fp32 product and
+    normalises it in a pass of its own -- and those are checked against the oracle (quantising the fp32 output)."""
+    import torch
+    from paper_1805_11046_b200 import layer
+    cfg = synth.conv3x3_layer(batch=batch, hw=hw, c_in=cin, k_out=cout)
+    c = cfg["conv"]
+    conv = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    gamma = to_dev(synth.uniform((cout,), 23, 1.0) + np.float32(1.5)); beta = to_dev(synth.uniform((cout,), 24, 0.5))
+    x, w = to_dev(cfg["x"]), to_dev(cfg["w"])
+    kept = layer.QuantizedLayer(conv=conv, relu=True, emit_codes=True, keep_y=True)
+    kept.forward(x, w, gamma, beta)
+    lean = layer.QuantizedLayer(conv=conv, relu=True, emit_codes=True, keep_y=False, keep_z=False)
+    lean.forward(x, w, gamma, beta)
+    torch.cuda.synchronize()
+    assert kept.status() == 0 and lean.status() == 0
+    assert np.array_equal(to_host(lean.out_codes), to_host(kept.out_codes))
+    assert np.array_equal(to_host(lean.q_out), to_host(kept.q_out))
+    assert np.array_equal(to_host(lean.out_row_sums), to_host(kept.out_row_sums))
+    for a, b_ in ((lean.save_mean, kept.save_mean), (lean.save_min, kept.save_min), (lean.save_max, kept.save_max)):
+        assert np.array_equal(to_host(a), to_host(b_))
+    # and against the oracle: the codes are those of the fp32 output the storing path wrote
+    o = O.quantize(to_host(kept.y), 8)
+    s_, z_, lo_, hi_ = B.read_qparams(lean.q_out)
+    assert s_[0] == o.scale[0] and z_[0] == o.zero_point[0] and lo_[0] == o.vmin[0] and hi_[0] == o.vmax[0]
+    assert np.array_equal(to_host(lean.out_codes), o.q)
+    # the backward pass needs the stored product and says so
+    with pytest.raises(B.QbpError):
+        lean.backward(to_dev(cfg["dy"]))

@@ -299,3 +299,51 @@ def test_wgrad_conv(B, N, H, W, C, K, R):
     oacc, oout = O.conv_wgrad_s16(od, X, zx, G, zg, 0.5, 0.25)
     assert B.status_word(ws) == 0
     assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(dW), oout)
+
+
+# ------------------------------------------- ReLU and requantisation in the epilogue (no Range BN after the product)
+def _check_requant(B, out_dev, q_dev, qp_dev, rs_dev, oout, relu, rng):
+    want = np.maximum(oout, 0) if relu else oout
+    if out_dev is not None:
+        assert np.array_equal(to_host(out_dev), want)
+    o = O.quantize(want, 8, range_in=rng)                # values beyond the clamp saturate
+    s_, z_, lo_, hi_ = B.read_qparams(qp_dev)
+    assert s_[0] == o.scale[0] and z_[0] == o.zero_point[0] and lo_[0] == o.vmin[0] and hi_[0] == o.vmax[0]
+    assert np.array_equal(to_host(q_dev), o.q)
+    if rs_dev is not None:
+        assert np.array_equal(to_host(rs_dev), o.q.reshape(-1, o.q.shape[-1]).astype(np.int32).sum(1))
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (208, 80, 144), (1024, 256, 512), (2000, 64, 64), (384, 640, 256)])
+@pytest.mark.parametrize("relu,keep_out", [(True, True), (False, False), (True, False)])
+def test_gemm_epilogue_relu_and_requantisation(B, M, N, K, relu, keep_out):
+    import torch
+    A = random_codes((M, K), 31); Bm = random_codes((K, N), 32)
+    za, zb, sa, sb = 5, -9, 0.5, 0.125
+    _, oout, bad = O.gemm_s8(A, za, Bm, zb, sa, sb)
+    assert bad == 0
+    hi = np.float32(0.6 * oout.max()); lo = np.float32(0.0 if relu else 0.5 * oout.min())      # a clamp that cuts the tails
+    q = torch.empty((M, N), dtype=torch.int8, device="cuda"); qp = B.new_qparams(1); rs = torch.empty(M, dtype=torch.int32, device="cuda")
+    res = B.qbp_gemm_s8(to_dev(A), _qp(B, sa, za), to_dev(Bm), _qp(B, sb, zb), want_out=keep_out, relu=relu,
+                        requant=(B.range_qparams(lo, hi), q, qp, rs))
+    assert B.status_word(res[2]) == 0
+    _check_requant(B, res[1] if keep_out else None, q, qp, rs, oout, relu, (lo, hi))
+
+
+@pytest.mark.parametrize("N_,H,W,C_,K_,R", [(2, 56, 56, 64, 64, 3), (3, 10, 12, 32, 48, 3), (4, 7, 7, 256, 128, 1), (1, 5, 130, 16, 272, 3)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_conv_epilogue_relu_and_requantisation(B, N_, H, W, C_, K_, R, mode):
+    import torch
+    pad = (R - 1) // 2
+    d = B.conv_desc(N_, H, W, C_, K_, R, R, 1, pad); od = O.conv_desc(N_, H, W, C_, K_, R, R, 1, pad)
+    inp = random_codes((N_, H, W, C_ if mode == 0 else K_), 33); w = random_codes((K_, R, R, C_), 34)
+    zi, zw = -3, 11
+    _, oout, bad = O.conv_s8(mode, od, inp, zi, w, zw, 0.5, 0.25)
+    assert bad == 0
+    hi = np.float32(0.7 * oout.max()); lo = np.float32(0.0)
+    q = torch.empty(oout.shape, dtype=torch.int8, device="cuda"); qp = B.new_qparams(1)
+    rs = torch.empty(oout.size // oout.shape[-1], dtype=torch.int32, device="cuda")
+    res = B.qbp_conv_s8_implicit(mode, d, to_dev(inp), _qp(B, 0.5, zi), to_dev(w), _qp(B, 0.25, zw), relu=True,
+                                 requant=(B.range_qparams(lo, hi), q, qp, rs))
+    assert B.status_word(res[2]) == 0
+    _check_requant(B, res[1], q, qp, rs, oout, True, (lo, hi))
