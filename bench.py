@@ -300,6 +300,8 @@ def run_ours(args):
         line["gemm_c5"] = gemm_c5_block(B, args.mnk, peaks)
         torch.cuda.empty_cache()
         line["rangebn_c3"] = rangebn_sweep_block(B, args.batch, hbm_peak)
+        torch.cuda.empty_cache()
+        line["stack_c4"] = stack_block(B, args.batch)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.cpu_sample_batch)
     if rank == 0:
@@ -437,6 +439,44 @@ def gemm_c5_block(B, n, peaks, launches=20):
                            "frac_of_measured_burst": round(2 * useful / int8_peak, 4),
                            "frac_of_nominal_4500": round(2 * useful / 4500.0, 4), "clocks": clocks}
     return res
+
+
+def stack_block(B, batch, reps=20):
+    """One training step (forward chain, backward chain, fp32 updates) of the ResNet-50 conv3_x bottleneck stack
+    (1x1 256->128, 3x3 128->128, 1x1 128->512, each + Range BN + ReLU) at batch `batch`: chained (every inner
+    activation handed on as the 8-bit codes its Range BN wrote) against the unfused composition (range scan +
+    quantiser per layer).  Each as a captured CUDA graph, `reps` replays."""
+    import torch
+    from paper_1805_11046_b200 import layer, synth
+    st = synth.bottleneck_stack(batch=batch, hw=28)
+    convs = [B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"]) for c in st["convs"]]
+    x = torch.from_numpy(st["x"]).cuda(); dy = torch.from_numpy(st["dy"]).cuda()
+    out = {"workload": "resnet50_conv3x_bottleneck_train_step", "batch": batch}
+    for name, chained in (("chained", True), ("unfused", False)):
+        S = layer.QuantizedStack(convs, [torch.from_numpy(w).cuda() for w in st["w"]], chained=chained, lr=0.0)
+        for _ in range(3):
+            S.train_step(x, dy)
+        torch.cuda.synchronize()
+        assert S.status() == 0
+        B.trace_enable(True); S.train_step(x, dy); launches = len(B.trace_records()); B.trace_enable(False)
+        side = torch.cuda.Stream(); side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            S.train_step(x, dy)
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            S.train_step(x, dy)
+        g.replay(); torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record(); torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / reps
+        out[name] = {"ms_per_step": round(ms, 4), "images_per_s": round(batch / (ms * 1e-3), 1), "launches": launches}
+        del S, g
+        torch.cuda.empty_cache()
+    return out
 
 
 # ------------------------------------------------------------- CPU oracle arm

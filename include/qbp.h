@@ -336,12 +336,16 @@ int qbp_rangebn_fwd(const float *x, int64_t n, int64_t C, const float *gamma, co
  * produce, bit for bit:
  *   q        [n x C] int8 codes (required)
  *   qp       their parameters (required)
- *   row_sums [n] sum of each row's stored codes (nullable) -- the code sums
- *            the next product's zero-point correction needs (Appendix B). */
+ *   row_sums  [n] sum of each row's stored codes (nullable) -- the code sums
+ *             the next product's zero-point correction needs (Appendix B);
+ *   chan_sums [C] sum of each channel's stored codes over all rows, int64
+ *             (nullable) -- what the next layer's weight gradient needs for
+ *             its zero-point terms (fewer than 2^22 rows). */
 typedef struct {
     int8_t      *q;
     qbp_qparams *qp;
     int32_t     *row_sums;
+    int64_t     *chan_sums;
 } qbp_requant;
 
 /* qbp_rangebn_fwd with the fused requantisation rq (nullable); y may be NULL
@@ -428,6 +432,11 @@ typedef struct {
     float  *g;
     int8_t *g8;       qbp_qparams *qg8;
     int8_t *g_hi;     uint8_t *g_lo;   qbp_qparams *qg16;
+    /* nullable; convolution layers: [C] per-channel sums of the input codes over all positions, written by the
+     * forward (by its quantiser, or handed on as in->chan_sums by the layer before) and read by the backward, whose
+     * weight gradient then builds its zero-point terms from these totals and the border positions instead of a
+     * pass over the three code tensors.  Fewer than 2^22 positions. */
+    int64_t *x_chan_sums;
 } qbp_layer_ctx;
 
 size_t qbp_layer_workspace_bytes(const qbp_layer_desc *L);
@@ -442,8 +451,9 @@ int qbp_layer_fwd(const qbp_layer_desc *L, const float *x, const float *w,
  *   in  (nullable): the input arrives already quantised -- the `out` record of
  *       the previous layer's call.  x must then be NULL, and in->q / in->qp
  *       must be the saved->x_codes / saved->qx of this layer (the backward
- *       pass reads the input codes from there).  in->row_sums NULL: the code
- *       sums are computed here.
+ *       pass reads the input codes from there), and in->chan_sums, if
+ *       saved->x_chan_sums is used, that same buffer.  in->row_sums NULL: the
+ *       code sums are computed here.
  *   out (nullable): also write the 8-bit codes of this layer's output for the
  *       next layer (see qbp_requant); y may then be NULL.
  * With in == NULL and out == NULL this is qbp_layer_fwd.

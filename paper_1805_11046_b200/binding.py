@@ -56,17 +56,18 @@ class LayerCtx(C.Structure):
     _fields_ = [("x_codes", C.c_void_p), ("qx", C.c_void_p), ("w_codes", C.c_void_p), ("qw", C.c_void_p),
                 ("z", C.c_void_p), ("save_mean", C.c_void_p), ("save_min", C.c_void_p), ("save_max", C.c_void_p),
                 ("g", C.c_void_p), ("g8", C.c_void_p), ("qg8", C.c_void_p), ("g_hi", C.c_void_p), ("g_lo", C.c_void_p),
-                ("qg16", C.c_void_p)]
+                ("qg16", C.c_void_p), ("x_chan_sums", C.c_void_p)]
 
 
 class Requant(C.Structure):
     """qbp_requant: where a pass writes the 8-bit codes of the activation it produces (q, qp) and, optionally,
     each row's code sum."""
-    _fields_ = [("q", C.c_void_p), ("qp", C.c_void_p), ("row_sums", C.c_void_p)]
+    _fields_ = [("q", C.c_void_p), ("qp", C.c_void_p), ("row_sums", C.c_void_p), ("chan_sums", C.c_void_p)]
 
 
-def requant(q, qp, row_sums=None) -> Requant:
-    return Requant(q.data_ptr(), qp.data_ptr(), row_sums.data_ptr() if row_sums is not None else None)
+def requant(q, qp, row_sums=None, chan_sums=None) -> Requant:
+    return Requant(q.data_ptr(), qp.data_ptr(), row_sums.data_ptr() if row_sums is not None else None,
+                   chan_sums.data_ptr() if chan_sums is not None else None)
 
 
 def _load() -> C.CDLL:
@@ -345,7 +346,7 @@ def qbp_rangebn_fwd(x, gamma=None, beta=None, relu=False, y=None, want_range=Fal
 
 
 def qbp_rangebn_fwd_q8(x, gamma=None, beta=None, relu=False, y=None, want_y=True, q=None, qp=None, row_sums=None,
-                       want_row_sums=False, ws=None):
+                       want_row_sums=False, ws=None, chan_sums=None):
     """Range BN forward that also (or only: want_y=False) writes the 8-bit codes of its output for the next layer.
     Returns (y or None, mean, vmin, vmax, q, qp, row_sums or None)."""
     Cc = x.shape[-1]; n = x.numel() // Cc
@@ -356,7 +357,7 @@ def qbp_rangebn_fwd_q8(x, gamma=None, beta=None, relu=False, y=None, want_y=True
     mean = torch.empty(Cc, dtype=torch.float32, device=x.device)
     vmin = torch.empty_like(mean); vmax = torch.empty_like(mean)
     if ws is None: ws = workspace(lib.qbp_rangebn_workspace_bytes(n, Cc), x.device)
-    rq = requant(q, qp, row_sums)
+    rq = requant(q, qp, row_sums, chan_sums)
     _check(lib.qbp_rangebn_fwd_q8(_ptr(x), C.c_int64(n), C.c_int64(Cc), _ptr(gamma), _ptr(beta), int(relu), _ptr(y),
                                   _ptr(mean), _ptr(vmin), _ptr(vmax), None, C.byref(rq), _ptr(ws), C.c_size_t(ws.numel()),
                                   _stream()))

@@ -82,7 +82,13 @@ static size_t chained_bytes(const LayerShape &s)
     // for the Range BN forward, and the per-channel constants of the normalisation for the recompute fusion
     return align_up(sizeof(int32_t) * (size_t)s.rows, 256) + align_up(sizeof(float2) * rangebn_range_parts_capacity(s.cout), 256) +
            2 * align_up(sizeof(float) * colstat_cells(s), 256) + align_up(sizeof(double) * colstat_cells(s), 256) +
-           align_up(sizeof(float4) * (size_t)s.cout, 256);
+           align_up(sizeof(float4) * (size_t)s.cout, 256) + align_up(sizeof(int64_t) * (size_t)s.cout, 256);
+}
+// The per-channel totals of the 16-bit gradient codes (last piece of the region above).
+static int64_t *tot_g_buffer(const qbp_layer_desc *L, const LayerShape &s, void *ws_after_head)
+{
+    return reinterpret_cast<int64_t *>(static_cast<char *>(ws_after_head) + step_scratch_bytes(L, s) + chained_bytes(s) -
+                                       align_up(sizeof(int64_t) * (size_t)s.cout, 256));
 }
 
 // Recompute instead of store (motivated by Section 7's memory and bandwidth argument): convolution -> Range BN
@@ -99,7 +105,9 @@ static int conv_rangebn_recompute(const qbp_conv_desc *d, const int8_t *x_codes,
     if (rc) return rc;
     if ((rc = rangebn_fold_from_parts(rows, d->K, gamma, beta, relu, save_mean, save_min, save_max, parts, out->qp, fold, st))) return rc;
     const EpilogueTail tail{fold, relu, out->qp, out->q, out->row_sums, 1};
-    return conv_s8_impl(QBP_CONV_FPROP, d, x_codes, qx, w_codes, qw, nullptr, nullptr, in_sums, nullptr, status, ws, scratch, st, &tail);
+    rc = conv_s8_impl(QBP_CONV_FPROP, d, x_codes, qx, w_codes, qw, nullptr, nullptr, in_sums, nullptr, status, ws, scratch, st, &tail);
+    if (rc || !out->chan_sums) return rc;
+    return launch_colsum(out->q, true, rows, d->K, out->chan_sums, st);
 }
 
 }  // namespace qbp
@@ -148,6 +156,10 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
                     "channels that writes 8-bit codes only (out given, y NULL)", QBP_EPILOGUE_MAX_COLUMNS);
     if (in && (in->q != saved->x_codes || in->qp != saved->qx))
         return fail(QBP_ERR_INVALID_ARG, "layer_fwd: in->q / in->qp must be the layer's saved x_codes / qx");
+    const bool want_totals = s.conv && saved->x_chan_sums != nullptr;
+    if (want_totals && s.rows >= (1ll << 22)) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "layer_fwd: x_chan_sums for fewer than 2^22 positions");
+    if (want_totals && in && in->chan_sums && in->chan_sums != saved->x_chan_sums)
+        return fail(QBP_ERR_INVALID_ARG, "layer_fwd: in->chan_sums must be the layer's saved x_chan_sums");
     if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
         return fail(QBP_ERR_WORKSPACE, "layer_fwd: workspace of %zu bytes needed, %zu given",
                     qbp_layer_workspace_bytes(L), ws_bytes);
@@ -163,12 +175,16 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
     int32_t *row_sums = reinterpret_cast<int32_t *>(static_cast<char *>(ws) + scratch);
     const int32_t *in_sums = s.conv ? row_sums : nullptr;
     if (x) {
-        rc = qbp_quantize_s8(x, s.rows, s.cin, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, saved->x_codes, saved->qx,
-                             s.conv ? row_sums : nullptr, nullptr, ws, scratch, stream);
+        bool left = false;
+        rc = quantize_s8_with_totals(x, s.rows, s.cin, saved->x_codes, saved->qx, s.conv ? row_sums : nullptr,
+                                     want_totals ? saved->x_chan_sums : nullptr, &left, ws, scratch, st);
         if (rc) return rc;
+        // (a shape the quantiser cannot take the totals of: one pass over the codes)
+        if (want_totals && !left && (rc = launch_colsum(saved->x_codes, true, s.rows, s.cin, saved->x_chan_sums, st))) return rc;
     } else if (s.conv) {
         if (in->row_sums) in_sums = in->row_sums;
         else if ((rc = launch_rowsum(in->q, true, s.rows, s.cin, row_sums, st))) return rc;
+        if (want_totals && !in->chan_sums && (rc = launch_colsum(in->q, true, s.rows, s.cin, saved->x_chan_sums, st))) return rc;
     }
     // weights: nearest rounding, clamping values = min and max
     const int64_t w_rows = s.conv ? (int64_t)L->conv.K * L->conv.R * L->conv.S : s.cin;
@@ -235,13 +251,18 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
                           saved->save_max, g, dgamma, dbeta, ws, scratch, range_parts, &nparts, st);
     if (rc) return rc;
     // two copies of the gradient: 8 bits for the layer gradient, 16 bits for the weight gradient
+    // (convolution with the input's per-channel code totals at hand: the bifurcation leaves the gradient's, and the
+    // weight gradient reads only the border positions again for its zero-point terms)
+    const bool totals = s.conv && saved->x_chan_sums && quantizer_totals_supported(s.cout) && s.rows < (1ll << 22);
+    int64_t *tot_g = totals ? tot_g_buffer(L, s, ws) : nullptr;
     rc = bifurcate_with_range_partials(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
-                                       s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st);
+                                       s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st, tot_g);
     if (rc) return rc;
     if (s.conv) {
         rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, nullptr, status, ws, scratch, st);
         if (rc) return rc;
-        return wgrad_s16_impl(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws, scratch, st);
+        return wgrad_s16_impl(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws, scratch, st,
+                              totals ? saved->x_chan_sums : nullptr, tot_g);
     }
     // dx [batch x in] = g8 [batch x out] . w^T, w stored [in x out]
     rc = gemm_s8_impl(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, nullptr, status, ws, scratch, st);

@@ -23,7 +23,12 @@ int rangebn_bwd_impl(const float *dy, const float *x, int64_t n, int64_t C, cons
 size_t rangebn_range_parts_capacity(int64_t C);
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                                   uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
-                                  uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st);
+                                  uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st,
+                                  int64_t *tot16 = nullptr);
+// Whether the quantising kernels can leave per-channel totals for a tensor of `cols` channels.
+bool quantizer_totals_supported(int64_t cols);
+int quantize_s8_with_totals(const float *x, int64_t rows, int64_t cols, int8_t *q, qbp_qparams *qp_out, int32_t *row_sums,
+                            int64_t *tot8, bool *left, void *ws, size_t ws_bytes, cudaStream_t st);
 // The convolution products with the per-pixel channel sums of the input codes supplied by the caller
 // (nullable: computed here) (qbp_mma.cu).
 // Per-column (sum, min, max) of a product's fp32 output as partial rows [rows][N], one per CTA
@@ -47,9 +52,13 @@ int conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_q
 int gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
                  const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const qbp_epilogue *ep,
                  int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);
+// tot_x [C] / tot_g16 [K] (convolution; nullable, both or none): per-channel totals of the stored x codes and of the
+// stored 16-bit gradient codes (256 * hi + lo) over all positions, left by the kernels that wrote the codes.
 int wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
                    const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
-                   int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);
+                   int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int64_t *tot_x = nullptr,
+                   const int64_t *tot_g16 = nullptr);
+// Bifurcation with optional per-channel totals of the 16-bit codes (tot16 [cols], zeroed here) -- see above.
 // Shapes the convolution products / the convolution weight gradient implement.
 bool conv_supported(const qbp_conv_desc *d);
 bool wgrad_conv_supported(const qbp_conv_desc *d);

@@ -283,6 +283,10 @@ struct QuantOut {
     int32_t *rowsum8;   // sums of the stored 8-bit codes over each row of `cols` (nullable; vector path only)
     int rs_group;       // lanes that share a row: cols / 4, a power of two <= 32
     int rs_shift;       // log2(rs_group)
+    // Per-channel totals of the stored codes over all rows, added (64-bit atomics) to chansum8 [cols] / chansum16
+    // [cols] (nullable; vector path, per tensor, cols / 4 a power of two <= 256: a thread then keeps its four
+    // channels for its whole life).  The weight gradient's zero-point terms are built from such totals.
+    unsigned long long *chansum8, *chansum16;
 };
 
 struct QParamsReg { float inv, zp_u; };
@@ -386,6 +390,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     }
     // both copies of a gradient under one tensor id: one Philox block serves the two (disjoint halves of each word)
     const bool one_block = want8 && want16 && id8 == id16;
+    int cs8[4] = {0, 0, 0, 0};                               // this thread's channels: totals of the stored 8-bit codes
+    unsigned cs16[4] = {0, 0, 0, 0};                         // ... and of the unsigned 16-bit codes (fewer than 65536 per thread)
     const int64_t nv = n >> 2;
     const int64_t stride = (int64_t)gridDim.x * kThreads * kUnroll;
     for (int64_t base = (int64_t)blockIdx.x * kThreads * kUnroll; base < nv; base += stride) {
@@ -431,6 +437,10 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                 const uint32_t packed = (SR ? pack_bytes2(c) : pack_bytes0(c)) ^ 0x80808080u;       // stored = unsigned code - 128
                 reinterpret_cast<uint32_t *>(o.q8)[j] = packed;
                 if (o.rowsum8) rs[u] = __dp4a((int)packed, 0x01010101, 0);
+                if (o.chansum8) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) cs8[e] = __dp4a((int)packed, 1 << (8 * e), cs8[e]);
+                }
             }
             if (want16) {
                 const uint32_t r[4] = {b16.x, b16.y, b16.z, b16.w};
@@ -445,6 +455,11 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                     // (stochastic: the code sits in the upper half of the word, i.e. bytes 3 and 2)
                     c[e] = SR ? quantize_sr16_top_half(xs[e], p16.inv, p16.zp_u, r[e])
                               : (uint32_t)quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]);
+                }
+                if (o.chansum16) {
+                    // unsigned codes here (the offset of 32768 per element is taken off when the block adds its totals up)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) cs16[e] += SR ? c[e] >> 16 : c[e];
                 }
                 // stored = unsigned code - 32768: flip the top bit of every code (of every high byte)
                 if (o.q16)
@@ -477,6 +492,28 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     if (blockIdx.x == 0 && threadIdx.x == 0)
         for (int64_t i = nv << 2; i < n; ++i)
             quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o, index_base);
+    if (!PERCH && (o.chansum8 || o.chansum16)) {
+        // (cols / 4 divides the block size and the grid stride: the thread's channels are 4 * (threadIdx.x mod cols / 4) ...)
+        // (a block sees fewer than 65536 rows -- the launcher's rule -- so its totals fit int32)
+        int *s_cs = reinterpret_cast<int *>(s_qp);           // [cols] 8-bit totals, then [cols] 16-bit ones
+        for (int c = threadIdx.x; c < 2 * cols; c += kThreads) s_cs[c] = 0;
+        __syncthreads();
+        const int c0 = 4 * (threadIdx.x & ((cols >> 2) - 1));
+        // how many elements this thread quantised per channel: the 16-bit totals were taken over unsigned codes
+        int64_t mine = 0;
+        for (int64_t base = (int64_t)blockIdx.x * kThreads * kUnroll; base < nv; base += stride)
+            for (int u = 0; u < kUnroll; ++u) mine += (base + u * kThreads + threadIdx.x < nv) ? 1 : 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (o.chansum8 && cs8[e]) atomicAdd(&s_cs[c0 + e], cs8[e]);
+            if (o.chansum16) atomicAdd(&s_cs[cols + c0 + e], (int)((long long)cs16[e] - mine * 32768));
+        }
+        __syncthreads();
+        for (int c = threadIdx.x; c < cols; c += kThreads) {
+            if (o.chansum8 && s_cs[c]) atomicAdd(o.chansum8 + c, (unsigned long long)(long long)s_cs[c]);
+            if (o.chansum16 && s_cs[cols + c]) atomicAdd(o.chansum16 + c, (unsigned long long)(long long)s_cs[cols + c]);
+        }
+    }
 }
 
 // Row sums of stored 8-bit codes: a group of G lanes per row (G = smallest power
@@ -609,7 +646,12 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
     const int c = (int)cols;
     // per-channel parameter table: 2 x cols x 8 bytes of dynamic shared memory when that stays within 32 KB
     const int smem_cols = (perch && vec && cols <= 2048) ? c : 0;
-    const size_t smem = (size_t)smem_cols * 2 * sizeof(float2);
+    const bool totals = o.chansum8 || o.chansum16;
+    // (fewer than 2^22 rows: with a grid of at least one block per SM, or one block per 1024 vectors, a block sees
+    // fewer than 65536 of them, and its int32 totals of 16-bit codes cannot overflow)
+    if (totals && !(vec && !perch && cols % 4 == 0 && cols / 4 <= kThreads && ((cols / 4) & (cols / 4 - 1)) == 0 && n / cols < (1ll << 22)))
+        return fail(QBP_ERR_INVALID_ARG, "quantize: per-channel totals need the vector path and cols / 4 a power of two <= %d", kThreads);
+    const size_t smem = totals ? (size_t)cols * 2 * sizeof(int) : (size_t)smem_cols * 2 * sizeof(float2);
     const int64_t groups = (n + per_block - 1) / per_block;
 #define QBP_QUANT(SR_, VEC_, PC_)                                                                                       \
     do {                                                                                                                \
@@ -757,9 +799,13 @@ static int static_scratch_address(void **out)
 // The quantising half of the bifurcation, once qp8 / qp16 are known.
 static int bifurcate_tail(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                           uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo,
-                          qbp_qparams *qp16, cudaStream_t st, uint64_t index_base = 0)
+                          qbp_qparams *qp16, cudaStream_t st, uint64_t index_base = 0, int64_t *tot16 = nullptr)
 {
-    QuantOut o = {q8, nullptr, hi, lo, nullptr, 0, 0};
+    QuantOut o = {q8, nullptr, hi, lo, nullptr, 0, 0, nullptr, nullptr};
+    if (tot16 && rows * cols > 0) {                       // (the caller asked quantizer_totals_supported(cols) first)
+        QBP_CUDA_OK(cudaMemsetAsync(tot16, 0, sizeof(int64_t) * (size_t)cols, st));
+        o.chansum16 = reinterpret_cast<unsigned long long *>(tot16);
+    }
     const bool fused = row_sums8 && rows * cols > 0 && can_fuse_rowsums(g, q8, cols, o);
     if (fused) { o.rowsum8 = row_sums8; o.rs_group = (int)(cols / 4); o.rs_shift = 31 - __builtin_clz((unsigned)o.rs_group); }
     int rc = launch_quantize(g, rows * cols, cols, 0, QBP_ROUND_STOCHASTIC, qp8, tensor_id8, qp16, tensor_id16, seed, o, st, index_base);
@@ -771,12 +817,38 @@ static int bifurcate_tail(const float *g, int64_t rows, int64_t cols, uint64_t s
 // Bifurcation of a gradient whose range partials (min, max per block) were left by the kernel that wrote it.
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                                   uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
-                                  uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st)
+                                  uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st,
+                                  int64_t *tot16)
 {
     QBP_TRACE_BEGIN(st);
     range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
     QBP_LAUNCH_OK("range_finalize_kernel");
-    return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st);
+    return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st, 0, tot16);
+}
+
+bool quantizer_totals_supported(int64_t cols)
+{
+    return cols % 4 == 0 && cols / 4 <= kThreads && ((cols / 4) & (cols / 4 - 1)) == 0;
+}
+
+// The layer's activation quantiser: qbp_quantize_s8 (per tensor, nearest) that also leaves the per-channel totals
+// of the codes (tot8 [cols], zeroed here) when the tensor's shape allows it; *left says whether it did.
+int quantize_s8_with_totals(const float *x, int64_t rows, int64_t cols, int8_t *q, qbp_qparams *qp_out, int32_t *row_sums,
+                            int64_t *tot8, bool *left, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    *left = false;
+    QuantOut o = {q, nullptr, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
+    const bool fused = row_sums && rows * cols > 0 && can_fuse_rowsums(x, q, cols, o);
+    if (fused) { o.rowsum8 = row_sums; o.rs_group = (int)(cols / 4); o.rs_shift = 31 - __builtin_clz((unsigned)o.rs_group); }
+    if (tot8 && rows * cols > 0 && quantizer_totals_supported(cols) && aligned16(x) && ((uintptr_t)q & 3) == 0) {
+        QBP_CUDA_OK(cudaMemsetAsync(tot8, 0, sizeof(int64_t) * (size_t)cols, st));
+        o.chansum8 = reinterpret_cast<unsigned long long *>(tot8);
+        *left = true;
+    }
+    int rc = quantize_any(8, x, rows, cols, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, o, qp_out, ws, ws_bytes, st);
+    if (rc) return rc;
+    if (row_sums && !fused) return launch_rowsum(q, true, rows, cols, row_sums, st);
+    return QBP_OK;
 }
 
 }  // namespace qbp
@@ -860,7 +932,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8(const floa
     if (!q && rows * cols > 0) return fail(QBP_ERR_INVALID_ARG, "quantize_s8: q is NULL");
     if ((row_sums || col_sums) && granularity != QBP_PER_TENSOR)
         return fail(QBP_ERR_INVALID_ARG, "quantize_s8: row/column sums are per-tensor only");
-    QuantOut o = {q, nullptr, nullptr, nullptr, nullptr, 0, 0};
+    QuantOut o = {q, nullptr, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
     const bool fused = row_sums && rows * cols > 0 && can_fuse_rowsums(x, q, cols, o);
     if (fused) { o.rowsum8 = row_sums; o.rs_group = (int)(cols / 4); o.rs_shift = 31 - __builtin_clz((unsigned)o.rs_group); }
     int rc = quantize_any(8, x, rows, cols, granularity, rounding, seed, tensor_id, range_in, o, qp_out, ws, ws_bytes, st);
@@ -875,7 +947,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_quantize_s16(const flo
                                 int8_t *hi, uint8_t *lo, qbp_qparams *qp_out, void *ws, size_t ws_bytes, void *stream)
 {
     if (!q && !hi && !lo) return fail(QBP_ERR_INVALID_ARG, "quantize_s16: q, hi and lo are all NULL");
-    QuantOut o = {nullptr, q, hi, lo, nullptr, 0, 0};
+    QuantOut o = {nullptr, q, hi, lo, nullptr, 0, 0, nullptr, nullptr};
     return quantize_any(16, x, rows, cols, granularity, rounding, seed, tensor_id, range_in, o, qp_out, ws, ws_bytes,
                         (cudaStream_t)stream);
 }
@@ -993,7 +1065,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_quantize_s8_static(con
     rc = static_scratch_address(&scratch);
     if (rc) return rc;
     // every partial the finalising kernel reads was written by this call's scan: nothing has to start at zero
-    QuantOut o = {q, nullptr, nullptr, nullptr};
+    QuantOut o = {q, nullptr, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
     return quantize_any(8, x, rows, cols, granularity, rounding, seed, tensor_id, nullptr, o, qp_out, scratch,
                         kStaticScratchBytes, (cudaStream_t)stream);
 }

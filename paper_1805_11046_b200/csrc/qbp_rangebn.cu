@@ -120,7 +120,8 @@ __global__ void bn_mean_from_sum_kernel(const double *__restrict__ col_sum, cons
 // parameters *rq) are written beside y, or instead of it (y == NULL); rowsum (nullable; rs_group = lanes per row,
 // a power of two <= 32 that covers the row) receives each row's sum of stored codes, which the next product's
 // zero-point correction needs.
-struct BnRequant { const qbp_qparams *rq; int8_t *q; int32_t *rowsum; int rs_group; };
+// chansum (nullable, [C], added to with 64-bit atomics): per-channel totals of the stored codes over all rows.
+struct BnRequant { const qbp_qparams *rq; int8_t *q; int32_t *rowsum; int rs_group; unsigned long long *chansum; };
 
 template <int VEC, bool RELU, bool REQUANT>
 __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__restrict__ x, int64_t rows, int C, int tw,
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
 {
     const ScanPos p = scan_pos<VEC>(C, tw);
     // (with row sums the idle threads of a ragged last slab take part in the shuffles: tw <= 32 then, one slab)
-    if (!p.active && !(REQUANT && R.rowsum)) return;
+    if (!p.active && !(REQUANT && (R.rowsum || R.chansum))) return;
     const int rpb = kScanThreads / tw;
     float mu[VEC], s[VEC], g[VEC], b[VEC];
 #pragma unroll
@@ -146,6 +147,9 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
     }
     float inv = 0.0f, zp_u = 0.0f;
     if (REQUANT) { inv = __fdiv_rn(1.0f, R.rq->scale); zp_u = (float)(R.rq->zero_point + 128); }
+    int cs[VEC];                                            // totals of the stored codes of this thread's channels
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) cs[e] = 0;
     const int64_t step = (int64_t)gridDim.x * rpb;
     // (the loop bound is the same for every thread of the block, so that the shuffles below see whole warps)
     for (int64_t rb = (int64_t)blockIdx.x * rpb; rb < rows; rb += step * kScanUnroll) {
@@ -176,9 +180,14 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
                         const uint32_t packed = (code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24)) ^ 0x80808080u;
                         *reinterpret_cast<uint32_t *>(R.q + at) = packed;
                         rs = __dp4a((int)packed, 0x01010101, 0);
+                        if (R.chansum) {
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) cs[e] = __dp4a((int)packed, 1 << (8 * (e & 3)), cs[e]);
+                        }
                     } else {
                         R.q[at] = (int8_t)((int)code[0] - 128);
                         rs = (int)code[0] - 128;
+                        cs[0] += rs;
                     }
                 }
             }
@@ -189,6 +198,22 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
                 const int64_t r = r0 + u * step;
                 if (p.tx == 0 && r < rows) R.rowsum[r] = rs;
             }
+        }
+    }
+    if (REQUANT && R.chansum) {
+        // the block's threads meet in shared memory (fewer than 2^22 rows: int32 is enough), then one atomic per channel
+        __shared__ int s_tot[kScanMaxTw * 4];
+        for (int i = threadIdx.x; i < tw * VEC; i += kScanThreads) s_tot[i] = 0;
+        __syncthreads();
+        if (p.active) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+                if (cs[e]) atomicAdd(&s_tot[p.tx * VEC + e], cs[e]);
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < tw * VEC; i += kScanThreads) {
+            const int c = (int)blockIdx.y * tw * VEC + i;
+            if (c < C && s_tot[i]) atomicAdd(R.chansum + c, (unsigned long long)(long long)s_tot[i]);
         }
     }
 }
@@ -473,13 +498,18 @@ static int bn_fwd_apply_launch(const float *x, int64_t n_rows, int64_t n_stat, i
                                                requant ? rq->qp : nullptr, nullptr);
         QBP_LAUNCH_OK("bn_out_range_kernel");
     }
-    BnRequant R{nullptr, nullptr, nullptr, 1};
+    BnRequant R{nullptr, nullptr, nullptr, 1, nullptr};
     bool fused_rowsum = false;
     if (requant) {
         R.rq = rq->qp; R.q = rq->q;
         // the row's lanes sit in one warp when the block is at most 32 vectors wide and one slab covers the row
         fused_rowsum = rq->row_sums && ga.tw <= 32 && ga.slabs == 1;
         if (fused_rowsum) { R.rowsum = rq->row_sums; R.rs_group = ga.tw; }
+        if (rq->chan_sums) {
+            if (n_rows >= (1ll << 22)) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "rangebn_fwd: per-channel code totals for fewer than 2^22 rows");
+            QBP_CUDA_OK(cudaMemsetAsync(rq->chan_sums, 0, sizeof(int64_t) * (size_t)C, st));
+            R.chansum = reinterpret_cast<unsigned long long *>(rq->chan_sums);
+        }
     }
     QBP_TRACE_BEGIN(st);
 #define QBP_BN_APPLY(V, RL, RQ) bn_apply_kernel<V, RL, RQ><<<grid_apply, kScanThreads, 0, st>>>(x, n_rows, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, y, R)

@@ -77,6 +77,10 @@ struct WgradParams {
     const qbp_qparams *qx, *qg;
     long long *acc_out; float *dW;
     int *status;
+    // Convolution: per-channel totals of the stored codes over all positions (x: [C]; the 16-bit gradient codes
+    // 256 * hi + lo: [N]) that the kernels which wrote the codes left.  The class tables then hold the border classes
+    // only, and the interior class is the total minus those.  NULL: the tables hold all sixteen classes.
+    const long long *tot_x, *tot_g;
 };
 
 // Which item and slice a CTA works on.
@@ -516,6 +520,104 @@ __global__ void __launch_bounds__(256, 3) row_class_sums3_kernel(const uint8_t *
     else                      row_class_sums_body<false>(lo, Nimg, H, W, C, gs, sums + 32 * C);
 }
 
+// The border classes only (first / last row, first / last column and the four corners; H, W >= 3) of the three code
+// tensors of a convolution's weight gradient: a few percent of the positions.  blockIdx.z: the layer input, the
+// gradient's signed high bytes, its unsigned low bytes (tables of 16 * Cx / 16 * Cg / 16 * Cg, zeroed beforehand);
+// blockIdx.x strides over groups of four images.  Thread = (16-channel group g, slot k): it walks positions k,
+// k + slots, ... of each of the four edges (corners excluded) and keeps one set of 16 sums per edge in registers;
+// the corners go straight to shared memory.  Few blocks: each ends with one atomic per table entry.
+__device__ __forceinline__ void border_add(bool is_signed, const uint4 &v, int *acc)
+{
+    const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            acc[k * 4 + b] = is_signed ? __dp4a((int)wd[k], 1 << (8 * b), acc[k * 4 + b])
+                                       : (int)__dp4a(wd[k], 1u << (8 * b), (unsigned)acc[k * 4 + b]);
+}
+
+__global__ void __launch_bounds__(256) border_class_sums_kernel(const uint8_t *__restrict__ x, const uint8_t *__restrict__ hi,
+                                                                const uint8_t *__restrict__ lo, int Nimg, int H, int W, int Cx,
+                                                                int Cg, unsigned long long *__restrict__ sums_x,
+                                                                unsigned long long *__restrict__ sums_hi,
+                                                                unsigned long long *__restrict__ sums_lo)
+{
+    extern __shared__ int s_acc[];                       // [16][C]
+    const uint8_t *q = blockIdx.z == 0 ? x : blockIdx.z == 1 ? hi : lo;
+    unsigned long long *sums = blockIdx.z == 0 ? sums_x : blockIdx.z == 1 ? sums_hi : sums_lo;
+    const int C = blockIdx.z == 0 ? Cx : Cg;
+    const bool is_signed = blockIdx.z != 2;
+    for (int i = threadIdx.x; i < 16 * C; i += 256) s_acc[i] = 0;
+    __syncthreads();
+    const int cv = C >> 4;
+    const int slots = 256 / cv;                          // (cv <= 256: C <= 4096)
+    const int g = threadIdx.x % cv, k = threadIdx.x / cv;
+    int top[16], bot[16], lef[16], rig[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) { top[e] = 0; bot[e] = 0; lef[e] = 0; rig[e] = 0; }
+    if (k < slots) {
+        // four images at a time, all their loads first: the positions are few and far apart, so latency is what counts
+        constexpr int U = 4;
+        for (int img0 = blockIdx.x * U; img0 < Nimg; img0 += gridDim.x * U) {
+            const uint4 *base[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) base[u] = reinterpret_cast<const uint4 *>(q + (int64_t)min(img0 + u, Nimg - 1) * H * W * C) + g;
+            for (int w = 1 + k; w < W - 1; w += slots) {
+                uint4 a[U], b[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) { a[u] = __ldg(base[u] + (int64_t)w * cv); b[u] = __ldg(base[u] + ((int64_t)(H - 1) * W + w) * cv); }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (img0 + u < Nimg) { border_add(is_signed, a[u], top); border_add(is_signed, b[u], bot); }
+            }
+            for (int h = 1 + k; h < H - 1; h += slots) {
+                uint4 a[U], b[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) { a[u] = __ldg(base[u] + (int64_t)h * W * cv); b[u] = __ldg(base[u] + ((int64_t)h * W + W - 1) * cv); }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (img0 + u < Nimg) { border_add(is_signed, a[u], lef); border_add(is_signed, b[u], rig); }
+            }
+            if (k < 4) {
+                // the four corners: classes 5, 9 (first row), 6, 10 (last row)
+                const int h = k < 2 ? 0 : H - 1, w = (k & 1) ? W - 1 : 0;
+                int cor[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) cor[e] = 0;
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (img0 + u < Nimg) border_add(is_signed, __ldg(base[u] + ((int64_t)h * W + w) * cv), cor);
+                int *dst = s_acc + ((k < 2 ? 1 : 2) | ((k & 1) ? 8 : 4)) * C + g * 16;
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                    if (cor[e]) atomicAdd(dst + e, cor[e]);
+            }
+        }
+    }
+    // the lanes of a warp that hold the same channel group meet by shuffle (when cv is a power of two below 32: whole
+    // warps are then inside `k < slots`), then one lane per group adds to the block's table
+    const bool shuffle = cv < 32 && (cv & (cv - 1)) == 0;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        int t = top[e], b = bot[e], l = lef[e], r = rig[e];
+        if (shuffle)
+            for (int off = cv; off < 32; off <<= 1) {
+                t += __shfl_xor_sync(0xffffffffu, t, off); b += __shfl_xor_sync(0xffffffffu, b, off);
+                l += __shfl_xor_sync(0xffffffffu, l, off); r += __shfl_xor_sync(0xffffffffu, r, off);
+            }
+        if (k < slots && (!shuffle || (threadIdx.x & 31) < cv)) {
+            if (t) atomicAdd(s_acc + 1 * C + g * 16 + e, t);
+            if (b) atomicAdd(s_acc + 2 * C + g * 16 + e, b);
+            if (l) atomicAdd(s_acc + 4 * C + g * 16 + e, l);
+            if (r) atomicAdd(s_acc + 8 * C + g * 16 + e, r);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 16 * C; i += 256)
+        if (s_acc[i] != 0) atomicAdd(&sums[i], (unsigned long long)(long long)s_acc[i]);
+}
+
 // Plain product, direct epilogue: rowterm[k] = -zg * SX[k] + M*zx*zg, colterm[n] = -zx * (256*SHI[n] + SLO[n]).
 __global__ void wgrad_terms_kernel(const long long *__restrict__ sx, const long long *__restrict__ shi,
                                    const long long *__restrict__ slo, int64_t M, int64_t N, int64_t K,
@@ -562,6 +664,17 @@ __global__ void __launch_bounds__(256) wgrad_finalize_kernel(const WgradParams P
         row = (tap % P.a_chunks) * P.rb_a + c % P.rb_a;
         // positions of g that see this tap: p - pad + r in [0,H)  <=>  not (r<pad and first row), not (r>pad and last row);
         // positions of x that are seen:      h + pad - r in [0,H)  <=>  not (r<pad and last row),  not (r>pad and first row).
+        if (P.tot_x) {
+            // totals over all positions, less the border classes this tap does not see (the interior always counts)
+            SX = P.tot_x[c]; SG = P.tot_g[n];
+            for (int cls = 1; cls < 16; ++cls) {
+                const bool top = cls & 1, bottom = cls & 2, left = cls & 4, right = cls & 8;
+                const bool g_ok = !((r < pad && top) || (r > pad && bottom) || (s < pad && left) || (s > pad && right));
+                const bool x_ok = !((r < pad && bottom) || (r > pad && top) || (s < pad && right) || (s > pad && left));
+                if (!g_ok) SG -= 256 * shi[cls * P.N + n] + slo[cls * P.N + n];
+                if (!x_ok) SX -= sx[cls * P.C + c];
+            }
+        } else
         for (int cls = 0; cls < 16; ++cls) {
             const bool top = cls & 1, bottom = cls & 2, left = cls & 4, right = cls & 8;
             const bool g_ok = !((r < pad && top) || (r > pad && bottom) || (s < pad && left) || (s > pad && right));
@@ -787,7 +900,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
 
 int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
                         const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
-                        int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st)
+                        int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int64_t *tot_x, const int64_t *tot_g16)
 {
     if (!x || !g_hi || !g_lo || !qx || !qg16) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: NULL operand");
     if (!acc_out && !dW) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: acc_out and dW are both NULL");
@@ -825,7 +938,24 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
     const bool pair_kernel = !d && wgrad2_eligible(M, N, K);
     // code sums for the zero-point terms: per border class (convolution) or plain column sums
     int rc;
-    if (d && K == N && d->W <= 256 && M < (1ll << 30) && shi == sx + 16 * K && slo == shi + 16 * N) {
+    // (the border tables stay within int32 per block: a block sees at most Nimg * 2 (W + H) border positions)
+    const bool from_totals = d && tot_x && tot_g16 && d->H >= 3 && d->W >= 3 && std::max(K, N) <= 1536 &&
+                             (int64_t)d->N * 2 * (d->H + d->W) < (1ll << 22);
+    if (from_totals) {
+        // the kernels that wrote the codes left their per-channel totals: only the border positions are read again
+        QBP_CUDA_OK(cudaMemsetAsync(sx, 0, (size_t)((char *)(slo + 16 * N) - (char *)sx), st));
+        if (d->pad > 0) {                // (without padding every tap sees every position: the totals are all there is)
+            static PerDeviceOnce configured;
+            QBP_SMEM_OPT_IN(configured, border_class_sums_kernel, 96 * 1024);
+            const int gx = (int)std::min<int64_t>((d->N + 3) / 4, 48);
+            QBP_TRACE_BEGIN(st);
+            border_class_sums_kernel<<<dim3((unsigned)gx, 1, 3), 256, (size_t)std::max(K, N) * 16 * sizeof(int), st>>>(
+                (const uint8_t *)x, (const uint8_t *)g_hi, g_lo, d->N, d->H, d->W, (int)K, (int)N, (unsigned long long *)sx,
+                (unsigned long long *)shi, (unsigned long long *)slo);
+            QBP_LAUNCH_OK("border_class_sums_kernel");
+        }
+        P.tot_x = (const long long *)tot_x; P.tot_g = (const long long *)tot_g16;
+    } else if (d && K == N && d->W <= 256 && M < (1ll << 30) && shi == sx + 16 * K && slo == shi + 16 * N) {
         // as many input as output channels: the three tensors in one launch
         QBP_CUDA_OK(cudaMemsetAsync(sx, 0, sizeof(int64_t) * 48 * K, st));
         const int cv = (int)K / 16;

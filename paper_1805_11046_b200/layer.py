@@ -44,13 +44,16 @@ class QuantizedLayer:
             assert input_from.rq_out is not None and input_from.z_shape == self.x_shape
             self.x_codes, self.qx = input_from.out_codes, input_from.q_out
             self.rq_in = input_from.rq_out
+            self.x_chan_sums = input_from.out_chan_sums
         else:
             self.x_codes, self.qx = e(self.x_shape, torch.int8), B.new_qparams(1, dev)
+            self.x_chan_sums = e((self.cin,), torch.int64) if conv is not None and self.rows < (1 << 22) else None
         self.rq_out = None
         if emit_codes:
             self.out_codes, self.q_out = e(self.z_shape, torch.int8), B.new_qparams(1, dev)
             self.out_row_sums = e((self.rows,), torch.int32)
-            self.rq_out = B.requant(self.out_codes, self.q_out, self.out_row_sums)
+            self.out_chan_sums = e((self.cout,), torch.int64) if conv is not None and self.rows < (1 << 22) else None
+            self.rq_out = B.requant(self.out_codes, self.q_out, self.out_row_sums, self.out_chan_sums)
         assert keep_z or (emit_codes and not keep_y)
         self.z = e(self.z_shape, torch.float32) if keep_z else None
         self.g = e(self.z_shape, torch.float32) if keep_z else None
@@ -66,7 +69,7 @@ class QuantizedLayer:
         for name, t in (("x_codes", self.x_codes), ("qx", self.qx), ("w_codes", self.w_codes), ("qw", self.qw),
                         ("z", self.z), ("save_mean", self.save_mean), ("save_min", self.save_min),
                         ("save_max", self.save_max), ("g", self.g), ("g8", self.g8), ("qg8", self.qg8),
-                        ("g_hi", self.ghi), ("g_lo", self.glo), ("qg16", self.qg16)):
+                        ("g_hi", self.ghi), ("g_lo", self.glo), ("qg16", self.qg16), ("x_chan_sums", self.x_chan_sums)):
             setattr(c, name, t.data_ptr() if t is not None and t.numel() else None)
         self.ctx = c
         self.gamma = self.beta = None

@@ -39,8 +39,8 @@ def test_struct_layouts_match_the_header():
     from paper_1805_11046_b200 import binding
     assert C.sizeof(binding.ConvDesc) == 36
     assert C.sizeof(binding.LayerDesc) == 36 + 4 + 3 * 8 + 4 + 4 + 8 + 4 + 4
-    assert C.sizeof(binding.LayerCtx) == 14 * 8
-    assert C.sizeof(binding.Epilogue) == 8 * 8 and C.sizeof(binding.Requant) == 3 * 8
+    assert C.sizeof(binding.LayerCtx) == 15 * 8
+    assert C.sizeof(binding.Epilogue) == 8 * 8 and C.sizeof(binding.Requant) == 4 * 8
 
 
 def _err(lib):

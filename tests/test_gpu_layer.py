@@ -154,13 +154,17 @@ def test_rangebn_fused_requantisation_equals_quantising_the_output(B):
         C_ = shape[-1]
         gamma = synth.uniform((C_,), 23, 1.0) + np.float32(1.5); beta = synth.uniform((C_,), 24, 0.5)
         gamma[::3] *= -1
-        y, mean, vmin, vmax, q, qp, rs = B.qbp_rangebn_fwd_q8(to_dev(x), to_dev(gamma), to_dev(beta), relu, want_row_sums=True)
+        import torch
+        cs = torch.empty(C_, dtype=torch.int64, device="cuda")
+        y, mean, vmin, vmax, q, qp, rs = B.qbp_rangebn_fwd_q8(to_dev(x), to_dev(gamma), to_dev(beta), relu, want_row_sums=True,
+                                                              chan_sums=cs)
         yh = to_host(y)
         o = O.quantize(yh, 8)                        # scans yh for its range
         s_, z_, lo_, hi_ = B.read_qparams(qp)
         assert s_[0] == o.scale[0] and z_[0] == o.zero_point[0] and lo_[0] == o.vmin[0] and hi_[0] == o.vmax[0]
         assert np.array_equal(to_host(q), o.q)
         assert np.array_equal(to_host(rs), o.q.reshape(-1, C_).astype(np.int32).sum(1))
+        assert np.array_equal(to_host(cs), o.q.reshape(-1, C_).astype(np.int64).sum(0))
         _, _, _, _, q2, qp2, _ = B.qbp_rangebn_fwd_q8(to_dev(x), to_dev(gamma), to_dev(beta), relu, want_y=False)
         assert np.array_equal(to_host(q2), o.q) and np.array_equal(to_host(qp2), to_host(qp))
 
