@@ -576,8 +576,17 @@ def run_gemm(args):
     out = torch.empty((n, n), dtype=torch.float32, device="cuda")
     ws = B.workspace(B.lib.qbp_gemm_s8_workspace_bytes(n, n, n))
     if args.only_steps:
+        # profiling aid: the GEMM, then the weight-gradient GEMM, warmup + steps calls each; no timing, no JSON line
         for _ in range(args.warmup + args.steps):
             B.qbp_gemm_s8(qa, qpa, qb, qpb, want_acc=False, out=out, ws=ws)
+        torch.cuda.synchronize(); assert B.status_word(ws) == 0
+        del qa, qb, out
+        qx, qpx = B.qbp_quantize_s8(dev(case["x"]))
+        _, hi, lo, qpg = B.qbp_quantize_s16(dev(case["g"]), want=("hi", "lo"))
+        dW = torch.empty((n, n), dtype=torch.float32, device="cuda")
+        ws = B.workspace(B.lib.qbp_wgrad_s16_workspace_bytes(None, n, n, n))
+        for _ in range(args.warmup + args.steps):
+            B.qbp_wgrad_s16(qx, qpx, hi, lo, qpg, want_acc=False, dW=dW, ws=ws)
         torch.cuda.synchronize(); assert B.status_word(ws) == 0
         return
     sampler = ClockSampler(0); sampler.start()

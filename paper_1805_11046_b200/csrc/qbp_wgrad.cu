@@ -947,7 +947,7 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
         if (d->pad > 0) {                // (without padding every tap sees every position: the totals are all there is)
             static PerDeviceOnce configured;
             QBP_SMEM_OPT_IN(configured, border_class_sums_kernel, 96 * 1024);
-            const int gx = (int)std::min<int64_t>((d->N + 3) / 4, 48);
+            const int gx = (int)std::min<int64_t>((d->N + 3) / 4, 128);      // one group of four images per block when possible
             QBP_TRACE_BEGIN(st);
             border_class_sums_kernel<<<dim3((unsigned)gx, 1, 3), 256, (size_t)std::max(K, N) * 16 * sizeof(int), st>>>(
                 (const uint8_t *)x, (const uint8_t *)g_hi, g_lo, d->N, d->H, d->W, (int)K, (int)N, (unsigned long long *)sx,
