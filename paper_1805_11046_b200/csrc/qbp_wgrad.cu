@@ -81,6 +81,12 @@ struct WgradParams {
     // 256 * hi + lo: [N]) that the kernels which wrote the codes left.  The class tables then hold the border classes
     // only, and the interior class is the total minus those.  NULL: the tables hold all sixteen classes.
     const long long *tot_x, *tot_g;
+    // ... and those border classes can be taken by this kernel's epilogue warps while the MMAs run (a few percent of
+    // the positions: the loads hide behind the main loop): cls_x [16][C], cls_hi / cls_lo [16][N] (zeroed beforehand),
+    // the code tensors, and the offset of the CTA's tables in shared memory.  cls_x == NULL: done elsewhere.
+    unsigned long long *cls_x, *cls_hi, *cls_lo;
+    const uint8_t *codes_x, *codes_hi, *codes_lo;
+    uint32_t cls_off;
 };
 
 // Which item and slice a CTA works on.
@@ -174,6 +180,83 @@ __device__ __forceinline__ bool wg_mma_dispatch_nt(int nt, const WgMmaArgs &A)
     if (RBB == 128) return false;
     if (nt == 3) return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 3)>(A);
     return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 4)>(A);
+}
+
+// Sixteen per-channel sums from one 16-byte group of codes (dot products that pick one byte each).
+__device__ __forceinline__ void border_add(bool is_signed, const uint4 &v, int *acc)
+{
+    const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            acc[k * 4 + b] = is_signed ? __dp4a((int)wd[k], 1 << (8 * b), acc[k * 4 + b])
+                                       : (int)__dp4a(wd[k], 1u << (8 * b), (unsigned)acc[k * 4 + b]);
+}
+
+// The border classes (first / last row, first / last column, corners; H, W >= 3) of images [img_begin, img_end) of one
+// code tensor of C channels (C / 16 = 2, 4 or 8 groups), by 128 threads (t = 0..127), into tbl [16][C] (shared
+// memory, zeroed).  Thread = (group, slot): it walks every slots-th position of the four edges, two images at a
+// time, with one set of 16 sums per edge in registers.
+__device__ __forceinline__ void wg_border_sums(bool is_signed, const uint8_t *__restrict__ q, int C, int H, int W, int img_begin,
+                                               int img_end, int *tbl, int t)
+{
+    const int cv = C >> 4, slots = 128 / cv;
+    const int g = t % cv, k = t / cv;
+    int top[16], bot[16], lef[16], rig[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) { top[e] = 0; bot[e] = 0; lef[e] = 0; rig[e] = 0; }
+    constexpr int U = 2;
+    for (int img0 = img_begin; img0 < img_end; img0 += U) {
+        const uint4 *base[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) base[u] = reinterpret_cast<const uint4 *>(q + (int64_t)min(img0 + u, img_end - 1) * H * W * C) + g;
+        for (int w = 1 + k; w < W - 1; w += slots) {
+            uint4 a[U], b[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) { a[u] = __ldg(base[u] + (int64_t)w * cv); b[u] = __ldg(base[u] + ((int64_t)(H - 1) * W + w) * cv); }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (img0 + u < img_end) { border_add(is_signed, a[u], top); border_add(is_signed, b[u], bot); }
+        }
+        for (int h = 1 + k; h < H - 1; h += slots) {
+            uint4 a[U], b[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) { a[u] = __ldg(base[u] + (int64_t)h * W * cv); b[u] = __ldg(base[u] + ((int64_t)h * W + W - 1) * cv); }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (img0 + u < img_end) { border_add(is_signed, a[u], lef); border_add(is_signed, b[u], rig); }
+        }
+        if (k < 4) {
+            // the four corners: classes 5, 9 (first row), 6, 10 (last row)
+            const int h = k < 2 ? 0 : H - 1, w = (k & 1) ? W - 1 : 0;
+            int cor[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) cor[e] = 0;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (img0 + u < img_end) border_add(is_signed, __ldg(base[u] + ((int64_t)h * W + w) * cv), cor);
+            int *dst = tbl + ((k < 2 ? 1 : 2) | ((k & 1) ? 8 : 4)) * C + g * 16;
+#pragma unroll
+            for (int e = 0; e < 16; ++e)
+                if (cor[e]) atomicAdd(dst + e, cor[e]);
+        }
+    }
+    // the lanes of a warp that hold the same group meet by shuffle (cv is 2, 4 or 8), then one lane per group adds
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        int tt = top[e], bb = bot[e], ll = lef[e], rr = rig[e];
+        for (int off = cv; off < 32; off <<= 1) {
+            tt += __shfl_xor_sync(0xffffffffu, tt, off); bb += __shfl_xor_sync(0xffffffffu, bb, off);
+            ll += __shfl_xor_sync(0xffffffffu, ll, off); rr += __shfl_xor_sync(0xffffffffu, rr, off);
+        }
+        if ((t & 31) < cv) {
+            if (tt) atomicAdd(tbl + 1 * C + g * 16 + e, tt);
+            if (bb) atomicAdd(tbl + 2 * C + g * 16 + e, bb);
+            if (ll) atomicAdd(tbl + 4 * C + g * 16 + e, ll);
+            if (rr) atomicAdd(tbl + 8 * C + g * 16 + e, rr);
+        }
+    }
 }
 
 // One instance per pair of operand layouts: RBA = row bytes of the x chunks, RBB = row bytes of the gradient tiles.
@@ -287,6 +370,24 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         // ------------------------------------------------------- epilogue
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
+        if (P.cls_x) {
+            // while the MMAs run: the border classes of this CTA's share of the images (by CTA index, whatever its item)
+            const int t = threadIdx.x - 64;
+            int *tx = reinterpret_cast<int *>(smem + P.cls_off), *th = tx + 16 * P.C, *tl = th + 16 * (int)P.N;
+            for (int i = t; i < 16 * (P.C + 2 * (int)P.N); i += 128) tx[i] = 0;
+            named_barrier(2, 128);
+            const int img_begin = (int)((int64_t)P.Nimg * blockIdx.x / gridDim.x), img_end = (int)((int64_t)P.Nimg * (blockIdx.x + 1) / gridDim.x);
+            wg_border_sums(true, P.codes_x, P.C, P.H, P.W, img_begin, img_end, tx, t);
+            wg_border_sums(true, P.codes_hi, (int)P.N, P.H, P.W, img_begin, img_end, th, t);
+            wg_border_sums(false, P.codes_lo, (int)P.N, P.H, P.W, img_begin, img_end, tl, t);
+            named_barrier(2, 128);
+            for (int i = t; i < 16 * P.C; i += 128)
+                if (tx[i]) atomicAdd(P.cls_x + i, (unsigned long long)(long long)tx[i]);
+            for (int i = t; i < 16 * (int)P.N; i += 128) {
+                if (th[i]) atomicAdd(P.cls_hi + i, (unsigned long long)(long long)th[i]);
+                if (tl[i]) atomicAdd(P.cls_lo + i, (unsigned long long)(long long)tl[i]);
+            }
+        }
         if (k_iters > 0 && !mbar_wait_warp(&acc_bar, 0)) timed_out = true;
         tc_fence_after();
         if (!timed_out && k_iters > 0) {
@@ -526,17 +627,6 @@ __global__ void __launch_bounds__(256, 3) row_class_sums3_kernel(const uint8_t *
 // blockIdx.x strides over groups of four images.  Thread = (16-channel group g, slot k): it walks positions k,
 // k + slots, ... of each of the four edges (corners excluded) and keeps one set of 16 sums per edge in registers;
 // the corners go straight to shared memory.  Few blocks: each ends with one atomic per table entry.
-__device__ __forceinline__ void border_add(bool is_signed, const uint4 &v, int *acc)
-{
-    const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-#pragma unroll
-        for (int b = 0; b < 4; ++b)
-            acc[k * 4 + b] = is_signed ? __dp4a((int)wd[k], 1 << (8 * b), acc[k * 4 + b])
-                                       : (int)__dp4a(wd[k], 1u << (8 * b), (unsigned)acc[k * 4 + b]);
-}
-
 __global__ void __launch_bounds__(256) border_class_sums_kernel(const uint8_t *__restrict__ x, const uint8_t *__restrict__ hi,
                                                                 const uint8_t *__restrict__ lo, int Nimg, int H, int W, int Cx,
                                                                 int Cg, unsigned long long *__restrict__ sums_x,
@@ -739,6 +829,14 @@ struct WgradPlan {
     int bw, bh, bn_img;
 };
 
+// Whether the kernel's epilogue warps can take the border classes themselves: a padded convolution whose x and g
+// tensors have 32, 64 or 128 channels (a pixel is 2, 4 or 8 sixteen-byte groups) and at least 3 x 3 positions.
+static bool wgrad_inline_border(const qbp_conv_desc *d)
+{
+    auto ok = [](int c) { return c == 32 || c == 64 || c == 128; };
+    return d && d->pad > 0 && ok(d->C) && ok(d->K) && d->H >= 3 && d->W >= 3;
+}
+
 static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, WgradPlan &pl)
 {
     WgradParams &P = pl.P;
@@ -792,9 +890,11 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
     // pipeline: stages of kr rows; one commit releases `cg` stages (some 24 MMAs between commits while that leaves
     // three groups in the ring).  The CTAs of the last group (fewer A tiles) get a ring of their own shape.
     const int n_last = P.a_tiles - (P.a_groups - 1) * P.ma;                 // A tiles of the last group
+    // (the border-class tables of the epilogue warps sit behind the ring)
+    const uint32_t cls_bytes = wgrad_inline_border(d) ? (uint32_t)align_up(sizeof(int) * 16 * (size_t)(K + 2 * N), 1024) : 0u;
     auto ring = [&](int tiles, int &stages, int &cg) {
         const uint32_t stage_bytes = P.a_chunk_bytes * P.a_chunks * (uint32_t)tiles + 2 * P.b.tile_bytes;
-        stages = std::max(2, std::min<int>(kWgMaxStages, (int)((kWgSmem - 1024) / stage_bytes)));
+        stages = std::max(2, std::min<int>(kWgMaxStages, (int)((kWgSmem - 1024 - cls_bytes) / stage_bytes)));
         const int mmas = tiles * (int)(kr / 32) * 2;
         cg = 1;
         while (cg * mmas < 24 && stages / (cg + 1) >= 3) ++cg;
@@ -803,7 +903,8 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
     };
     const size_t smem_full = ring(P.ma, P.stages, P.cg);
     const size_t smem_last = ring(n_last, P.stages_last, P.cg_last);
-    pl.smem = std::max(smem_full, smem_last);
+    P.cls_off = (uint32_t)(std::max(smem_full, smem_last) - 1024);           // behind the longer of the two rings
+    pl.smem = std::max(smem_full, smem_last) + cls_bytes;
     // split of the reductions: at most 65536 rows per CTA; with few items, enough slices to fill the machine
     // once, in proportion to an item's cost per reduction step: a fixed part (waits, the share of a commit)
     // worth about eight MMAs, plus its MMAs
@@ -944,7 +1045,11 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
     if (from_totals) {
         // the kernels that wrote the codes left their per-channel totals: only the border positions are read again
         QBP_CUDA_OK(cudaMemsetAsync(sx, 0, (size_t)((char *)(slo + 16 * N) - (char *)sx), st));
-        if (d->pad > 0) {                // (without padding every tap sees every position: the totals are all there is)
+        if (wgrad_inline_border(d)) {
+            // the product kernel's epilogue warps take the border classes while its MMAs run
+            P.cls_x = (unsigned long long *)sx; P.cls_hi = (unsigned long long *)shi; P.cls_lo = (unsigned long long *)slo;
+            P.codes_x = (const uint8_t *)x; P.codes_hi = (const uint8_t *)g_hi; P.codes_lo = g_lo;
+        } else if (d->pad > 0) {         // (without padding every tap sees every position: the totals are all there is)
             static PerDeviceOnce configured;
             QBP_SMEM_OPT_IN(configured, border_class_sums_kernel, 96 * 1024);
             const int gx = (int)std::min<int64_t>((d->N + 3) / 4, 128);      // one group of four images per block when possible
