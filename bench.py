@@ -36,11 +36,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
 # (captured at the full batch of 256).  None: not captured.
 # Keyed by (kernel, occurrence within the step), like KERNEL_WORK; dropped when a kernel changes.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {("quantize_kernel", 2): (205.6e6 + 119.2e6) / 51380224}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {("quantize_kernel", 1): (205.6e6 + 119.2e6) / 51380224}
 # Kernels bound by plain instruction issue rather than by HBM: thread instructions per element, from the same
 # captures (smsp__inst_executed.sum x 32 / elements).  Their roofline is the issue rate of the SMs:
 # SMs x 4 schedulers x 1 warp instruction per clock x 32 threads x the maximum SM clock.
-ALU_INSTR_PER_ELEMENT = {("quantize_kernel", 2): 7.336e7 * 32 / 51380224}
+ALU_INSTR_PER_ELEMENT = {("quantize_kernel", 1): 7.336e7 * 32 / 51380224}
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 
 
@@ -108,15 +108,12 @@ def conv_workload(batch):
 # move O(channels) or O(pixels) bytes only.
 OPS_PER_ELEMENT_CONV = 2 * 9 * CIN          # 2*K per output element of fprop / dgrad
 KERNEL_WORK = {
-    ("range_partial_kernel", 0): (4, 0), ("quantize_kernel", 0): (5, 0),            # x (occurrence 1: the filter, tiny)
-    ("rowsum_kernel", 0): (1, 0),                                                   # channel sums of the x codes
+    ("range_partial_kernel", 0): (4, 0), ("quantize_kernel", 0): (5, 0),            # x: scan, then codes (+ per-pixel sums, per-channel totals)
     ("qbp_mma_kernel", 0): (5, OPS_PER_ELEMENT_CONV),                               # fprop: 1 B codes in, 4 B fp32 out
     ("bn_stats_kernel", 0): (4, 0), ("bn_apply_kernel", 0): (8, 0),
     ("bn_bwd_stats_kernel", 0): (8, 0), ("bn_bwd_apply_kernel", 0): (12, 0),
-    ("range_partial_kernel", 2): (4, 0), ("quantize_kernel", 2): (7, 0),            # bifurcation: 4 B in, 1 + 2 B out
-    ("rowsum_kernel", 2): (1, 0),                                                   # channel sums of the 8-bit gradient codes
+    ("quantize_kernel", 1): (7, 0),                                                 # bifurcation: 4 B in, 1 + 2 B out
     ("qbp_mma_kernel", 1): (5, OPS_PER_ELEMENT_CONV),                               # dgrad
-    ("class_sums_kernel", 0): (3, 0),                                               # x, hi and lo codes in one launch
     ("qbp_wgrad_kernel", 0): (3, 2 * OPS_PER_ELEMENT_CONV),                         # two int8 products per 16x8-bit product
 }
 

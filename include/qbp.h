@@ -277,6 +277,19 @@ int qbp_gemm_s8(int transA, int transB, int64_t M, int64_t N, int64_t K,
                 int32_t *acc_out, float *C, const qbp_epilogue *ep,
                 void *ws, size_t ws_bytes, void *stream);
 
+/* qbp_gemm_s8 with the code sums along the reduction supplied by the caller
+ * (the zero-point correction of Appendix B's scheme needs them; qbp_gemm_s8
+ * computes them in two small kernels per call).  a_sums [M] (nullable): the
+ * sum over k of the stored codes of row m of op(A); b_sums [N] (nullable): the
+ * sum over k of column n of op(B); int32 (K <= 33025 codes always fit).  The
+ * row_sums output of qbp_quantize_s8 / qbp_requant is a_sums of a
+ * non-transposed A (and b_sums of a transposed B). */
+int qbp_gemm_s8_sums(int transA, int transB, int64_t M, int64_t N, int64_t K,
+                     const int8_t *A, const qbp_qparams *qa, const int32_t *a_sums,
+                     const int8_t *B, const qbp_qparams *qb, const int32_t *b_sums,
+                     int32_t *acc_out, float *C, const qbp_epilogue *ep,
+                     void *ws, size_t ws_bytes, void *stream);
+
 /* The same products for a convolution, computed as an implicit GEMM over
  * the filter taps (no im2col buffer).  QBP_CONV_FPROP: x [N,H,W,C] ->
  * [N,P,Q,K].  QBP_CONV_DGRAD (Eq. grad_layer): g [N,P,Q,K] -> [N,H,W,C].

@@ -27,7 +27,7 @@ EXPORTS = (
     "qbp_quantize_workspace_bytes", "qbp_quantize_s8", "qbp_quantize_s8_static", "qbp_quantize_s16", "qbp_bifurcate",
     "qbp_bifurcate_shard", "qbp_dequant_s64", "qbp_sgd_update",
     "qbp_range_chunked_workspace_bytes", "qbp_range_chunked",
-    "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8",
+    "qbp_gemm_s8_workspace_bytes", "qbp_gemm_s8", "qbp_gemm_s8_sums",
     "qbp_conv_s8_workspace_bytes", "qbp_conv_s8_implicit",
     "qbp_wgrad_s16_workspace_bytes", "qbp_wgrad_s16",
     "qbp_rangebn_workspace_bytes", "qbp_rangebn_fwd", "qbp_rangebn_bwd", "qbp_rangebn_fwd_q8",
@@ -284,7 +284,7 @@ def _epilogue(col_stats, n, device, relu=False, requant=None):
 
 
 def qbp_gemm_s8(A, qa, B, qb, transA=False, transB=False, want_acc=False, want_out=True, acc_out=None, out=None, ws=None,
-                col_stats=None, relu=False, requant=None):
+                col_stats=None, relu=False, requant=None, a_sums=None, b_sums=None):
     if transA: K, M = A.shape
     else:      M, K = A.shape
     N = B.shape[0] if transB else B.shape[1]
@@ -292,9 +292,14 @@ def qbp_gemm_s8(A, qa, B, qb, transA=False, transB=False, want_acc=False, want_o
     if want_out and out is None: out = torch.empty((M, N), dtype=torch.float32, device=A.device)
     if ws is None: ws = workspace(lib.qbp_gemm_s8_workspace_bytes(M, N, K), A.device)
     ep, stats = _epilogue(col_stats, N, A.device, relu, requant)
-    _check(lib.qbp_gemm_s8(int(transA), int(transB), C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A), _ptr(qa),
-                           _ptr(B), _ptr(qb), _ptr(acc_out), _ptr(out), C.byref(ep) if ep else None, _ptr(ws),
-                           C.c_size_t(ws.numel()), _stream()))
+    if a_sums is not None or b_sums is not None:
+        _check(lib.qbp_gemm_s8_sums(int(transA), int(transB), C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A), _ptr(qa),
+                                    _ptr(a_sums), _ptr(B), _ptr(qb), _ptr(b_sums), _ptr(acc_out), _ptr(out),
+                                    C.byref(ep) if ep else None, _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    else:
+        _check(lib.qbp_gemm_s8(int(transA), int(transB), C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A), _ptr(qa),
+                               _ptr(B), _ptr(qb), _ptr(acc_out), _ptr(out), C.byref(ep) if ep else None, _ptr(ws),
+                               C.c_size_t(ws.numel()), _stream()))
     return (acc_out, out, ws, stats) if col_stats else (acc_out, out, ws)
 
 

@@ -82,7 +82,15 @@ static size_t chained_bytes(const LayerShape &s)
     // for the Range BN forward, and the per-channel constants of the normalisation for the recompute fusion
     return align_up(sizeof(int32_t) * (size_t)s.rows, 256) + align_up(sizeof(float2) * rangebn_range_parts_capacity(s.cout), 256) +
            2 * align_up(sizeof(float) * colstat_cells(s), 256) + align_up(sizeof(double) * colstat_cells(s), 256) +
-           align_up(sizeof(float4) * (size_t)s.cout, 256) + align_up(sizeof(int64_t) * (size_t)s.cout, 256);
+           align_up(sizeof(float4) * (size_t)s.cout, 256) + align_up(sizeof(int32_t) * 16 * (size_t)std::max(s.cin, s.cout), 256) +
+           align_up(sizeof(int64_t) * (size_t)s.cout, 256);
+}
+// The forward column terms that come with the filter's codes (the piece before the last of the region above).
+static int32_t *colterm_buffer(const qbp_layer_desc *L, const LayerShape &s, void *ws_after_head)
+{
+    return reinterpret_cast<int32_t *>(static_cast<char *>(ws_after_head) + step_scratch_bytes(L, s) + chained_bytes(s) -
+                                       align_up(sizeof(int64_t) * (size_t)s.cout, 256) -
+                                       align_up(sizeof(int32_t) * 16 * (size_t)std::max(s.cin, s.cout), 256));
 }
 // The per-channel totals of the 16-bit gradient codes (last piece of the region above).
 static int64_t *tot_g_buffer(const qbp_layer_desc *L, const LayerShape &s, void *ws_after_head)
@@ -98,13 +106,16 @@ static int64_t *tot_g_buffer(const qbp_layer_desc *L, const LayerShape &s, void 
 static int conv_rangebn_recompute(const qbp_conv_desc *d, const int8_t *x_codes, const qbp_qparams *qx, const int32_t *in_sums,
                                   const int8_t *w_codes, const qbp_qparams *qw, const float *gamma, const float *beta, int relu,
                                   float *save_mean, float *save_min, float *save_max, const qbp_requant *out,
-                                  ColStatParts parts, float4 *fold, int *status, void *ws, size_t scratch, cudaStream_t st)
+                                  ColStatParts parts, float4 *fold, const int32_t *colterm, int *status, void *ws, size_t scratch,
+                                  cudaStream_t st)
 {
     const int64_t rows = (int64_t)d->N * d->H * d->W;
-    int rc = conv_s8_impl(QBP_CONV_FPROP, d, x_codes, qx, w_codes, qw, nullptr, nullptr, in_sums, &parts, status, ws, scratch, st);
+    const EpilogueTail first{nullptr, 0, nullptr, nullptr, nullptr, 0, colterm};
+    int rc = conv_s8_impl(QBP_CONV_FPROP, d, x_codes, qx, w_codes, qw, nullptr, nullptr, in_sums, &parts, status, ws, scratch, st,
+                          colterm ? &first : nullptr);
     if (rc) return rc;
     if ((rc = rangebn_fold_from_parts(rows, d->K, gamma, beta, relu, save_mean, save_min, save_max, parts, out->qp, fold, st))) return rc;
-    const EpilogueTail tail{fold, relu, out->qp, out->q, out->row_sums, 1};
+    const EpilogueTail tail{fold, relu, out->qp, out->q, out->row_sums, 1, colterm};
     rc = conv_s8_impl(QBP_CONV_FPROP, d, x_codes, qx, w_codes, qw, nullptr, nullptr, in_sums, nullptr, status, ws, scratch, st, &tail);
     if (rc || !out->chan_sums) return rc;
     return launch_colsum(out->q, true, rows, d->K, out->chan_sums, st);
@@ -186,11 +197,20 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
         else if ((rc = launch_rowsum(in->q, true, s.rows, s.cin, row_sums, st))) return rc;
         if (want_totals && !in->chan_sums && (rc = launch_colsum(in->q, true, s.rows, s.cin, saved->x_chan_sums, st))) return rc;
     }
-    // weights: nearest rounding, clamping values = min and max
+    // weights: nearest rounding, clamping values = min and max (a small filter: scan, codes, code sums and the forward
+    // product's column terms in one launch)
     const int64_t w_rows = s.conv ? (int64_t)L->conv.K * L->conv.R * L->conv.S : s.cin;
-    rc = qbp_quantize_s8(w, w_rows, s.w_elems / w_rows, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr,
-                         saved->w_codes, saved->qw, nullptr, nullptr, ws, scratch, stream);
-    if (rc) return rc;
+    const int32_t *colterm = nullptr;
+    if (s.conv && filter_prep_supported(&L->conv, w, saved->w_codes)) {
+        int32_t *ct = colterm_buffer(L, s, ws);
+        if ((rc = launch_filter_prep(&L->conv, w, saved->qx, saved->w_codes, saved->qw, ct, st))) return rc;
+        colterm = ct;
+    } else {
+        rc = qbp_quantize_s8(w, w_rows, s.w_elems / w_rows, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr,
+                             saved->w_codes, saved->qw, nullptr, nullptr, ws, scratch, stream);
+        if (rc) return rc;
+    }
+    const EpilogueTail with_colterm{nullptr, 0, nullptr, nullptr, nullptr, 0, colterm};
     ColStatParts parts{nullptr, nullptr, nullptr, 0};
     if (epilogue_stats(s)) {
         char *base = static_cast<char *>(ws) + scratch + align_up(sizeof(int32_t) * (size_t)s.rows, 256) +
@@ -202,11 +222,12 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
     if (recompute) {
         float4 *fold = reinterpret_cast<float4 *>(reinterpret_cast<char *>(parts.sum) + align_up(sizeof(double) * colstat_cells(s), 256));
         return conv_rangebn_recompute(&L->conv, saved->x_codes, saved->qx, in_sums, saved->w_codes, saved->qw, gamma, beta, L->relu,
-                                      saved->save_mean, saved->save_min, saved->save_max, out, parts, fold, status, ws, scratch, st);
+                                      saved->save_mean, saved->save_min, saved->save_max, out, parts, fold, colterm, status, ws,
+                                      scratch, st);
     }
     if (s.conv)
         rc = conv_s8_impl(QBP_CONV_FPROP, &L->conv, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr, saved->z,
-                          in_sums, parts.sum ? &parts : nullptr, status, ws, scratch, st);
+                          in_sums, parts.sum ? &parts : nullptr, status, ws, scratch, st, colterm ? &with_colterm : nullptr);
     else
         rc = gemm_s8_impl(0, 0, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, saved->w_codes, saved->qw, nullptr,
                           saved->z, nullptr, status, ws, scratch, st);
@@ -259,7 +280,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st, tot_g);
     if (rc) return rc;
     if (s.conv) {
-        rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, nullptr, status, ws, scratch, st);
+        // (a small filter: the layer gradient's column terms in one launch, else two kernels inside the product's call)
+        const bool small = (int64_t)L->conv.R * L->conv.S * L->conv.C <= 12288 && s.w_elems <= (1 << 18) && L->conv.C % 4 == 0;
+        int32_t *ct = small ? colterm_buffer(L, s, ws) : nullptr;
+        if (small && (rc = launch_filter_dgrad_colterm(&L->conv, saved->w_codes, qp8, ct, st))) return rc;
+        const EpilogueTail with_colterm{nullptr, 0, nullptr, nullptr, nullptr, 0, ct};
+        rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, nullptr, status, ws, scratch, st,
+                          small ? &with_colterm : nullptr);
         if (rc) return rc;
         return wgrad_s16_impl(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws, scratch, st,
                               totals ? saved->x_chan_sums : nullptr, tot_g);

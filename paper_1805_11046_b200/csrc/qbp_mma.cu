@@ -196,6 +196,8 @@ struct MmaParams {
     const float4 *ep_fold; int ep_relu;
     const qbp_qparams *ep_rq; int8_t *ep_q; int32_t *ep_rowsum;
     uint32_t stat_span;           // bytes of the statistics region in shared memory (the fold table follows it)
+    int direct;                   // the fp32 output goes straight from registers to global memory (32-byte stores: a lane's
+                                  // 32 outputs are 128 contiguous bytes) instead of through a staging slab and a TMA store
     int grid;                     // CTAs launched
     uint32_t cterm_span;          // bytes of the column-term region in shared memory (the statistics follow it)
     int iter_entries;             // entries of the k-iteration table in shared memory (conv), a multiple of 64
@@ -686,7 +688,20 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                             }
                         }
                     }
-                    if (P.out || P.st_sum) {
+                    if (P.out && P.direct && ri.valid) {
+                        float *dst = P.out + ri.m * P.N + o.n0 + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8)
+                            if (j < lim) {
+                                float f[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) f[e] = TAIL ? v[TAIL ? j + e : 0] : __fmul_rn((float)acc[j + e], scale);
+                                asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                             ::"l"(dst + j), "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "f"(f[4]), "f"(f[5]), "f"(f[6]), "f"(f[7])
+                                             : "memory");
+                            }
+                    }
+                    if (P.st_sum || (P.out && !P.direct)) {
                         // the store that last used this slab must have read it before it is overwritten
                         uint8_t *slab = slab0 + slab_i * kStageSlab;
                         if (lane == 0) { if (P.nslab == 2) tma_store_wait_read_but_one(); else tma_store_wait_read(); }
@@ -702,7 +717,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                                                    __fmul_rn((float)acc[j + 2], scale), __fmul_rn((float)acc[j + 3], scale));
                         fence_proxy_async();
                         __syncwarp();
-                        if (lane == 0 && ri.slab_in && P.out) {
+                        if (lane == 0 && ri.slab_in && P.out && !P.direct) {
                             if (P.mode == MODE_GEMM) tma_store_2d(&P.mapC, slab, o.n0 + c0, o.m0 + sub * 128 + quad * 32);
                             else                     tma_store_4d(&P.mapC, slab, o.n0 + c0, ri.sx, ri.sy, ri.sz);
                             tma_store_commit();
@@ -815,6 +830,103 @@ __global__ void conv_colterm_kernel(const int32_t *wsum32, const long long *wsum
     colterm[cls * N + n] = -q_in->zero_point * (int)sum;
 }
 
+// A small filter in one launch (Appendix B's quantiser for the weights, then what the forward convolution's zero-point
+// correction needs of them): min / max scan, scale and zero-point, nearest 8-bit codes, the code sums of every
+// (output channel, tap) over the input channels, and the forward column terms
+//   colterm[cls][k] = -z_in * sum over the taps valid for border class cls of wsum[k][tap].
+// One block of 1024 threads; w [K][taps][C] fp32, C a multiple of 4, 16-byte aligned.  The operation order of the
+// quantiser is the library's (make_qparams, quantize_code), so the codes are those of qbp_quantize_s8.
+__global__ void __launch_bounds__(1024) filter_prep_kernel(const float *__restrict__ w, int K, int taps, int C, int R, int S, int pad,
+                                                            const qbp_qparams *__restrict__ q_in, int8_t *__restrict__ codes,
+                                                            qbp_qparams *__restrict__ qp_out, int32_t *__restrict__ colterm)
+{
+    extern __shared__ int s_wsum[];                      // [K * taps]
+    __shared__ float s_lo[32], s_hi[32];
+    __shared__ float s_inv, s_zp;
+    const int n4 = K * taps * C / 4;
+    const int rows = K * taps;
+    float lo = INFINITY, hi = -INFINITY;
+    for (int i = threadIdx.x; i < n4; i += 1024) {
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(w) + i);
+        lo = fminf(fminf(lo, fminf(v.x, v.y)), fminf(v.z, v.w));
+        hi = fmaxf(fmaxf(hi, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+    }
+    lo = warp_min(lo); hi = warp_max(hi);
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
+    for (int i = threadIdx.x; i < rows; i += 1024) s_wsum[i] = 0;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        lo = warp_min(s_lo[threadIdx.x]); hi = warp_max(s_hi[threadIdx.x]);
+        if (threadIdx.x == 0) {
+            const qbp_qparams qp = make_qparams(lo, hi, 8);
+            *qp_out = qp;
+            s_inv = __fdiv_rn(1.0f, qp.scale); s_zp = (float)(qp.zero_point + 128);
+        }
+    }
+    __syncthreads();
+    const float inv = s_inv, zp_u = s_zp;
+    const int c4 = C / 4;                                 // vectors per (k, tap) row
+    for (int i = threadIdx.x; i < n4; i += 1024) {
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(w) + i);
+        const uint32_t c0 = (uint32_t)quantize_code<false>(v.x, inv, zp_u, 255.0f, 0u), c1 = (uint32_t)quantize_code<false>(v.y, inv, zp_u, 255.0f, 0u);
+        const uint32_t c2 = (uint32_t)quantize_code<false>(v.z, inv, zp_u, 255.0f, 0u), c3 = (uint32_t)quantize_code<false>(v.w, inv, zp_u, 255.0f, 0u);
+        const uint32_t packed = (c0 | (c1 << 8) | (c2 << 16) | (c3 << 24)) ^ 0x80808080u;
+        reinterpret_cast<uint32_t *>(codes)[i] = packed;
+        atomicAdd(&s_wsum[i / c4], __dp4a((int)packed, 0x01010101, 0));
+    }
+    __syncthreads();
+    const int zin = q_in->zero_point;
+    for (int i = threadIdx.x; i < 16 * K; i += 1024) {
+        const int cls = i / K, k = i - cls * K;
+        const bool top = cls & 1, bottom = cls & 2, left = cls & 4, right = cls & 8;
+        int sum = 0;
+        for (int r = 0; r < R; ++r) {
+            if ((r < pad && top) || (r > pad && bottom)) continue;
+            for (int t = 0; t < S; ++t) {
+                if ((t < pad && left) || (t > pad && right)) continue;
+                sum += s_wsum[k * taps + r * S + t];
+            }
+        }
+        colterm[i] = -zin * sum;
+    }
+}
+
+// The layer-gradient product's column terms from a small filter's codes in one launch: the code sums of every
+// (tap, input channel) over the output channels, then
+//   colterm[cls][c] = -z_g * sum over the taps valid for border class cls (gradient orientation) of wsum[tap][c].
+// One block of 1024 threads; codes [K][taps * C], C a multiple of 4.
+__global__ void __launch_bounds__(1024) filter_dgrad_colterm_kernel(const int8_t *__restrict__ codes, int K, int taps, int C, int R,
+                                                                     int S, int pad, const qbp_qparams *__restrict__ q_g,
+                                                                     int32_t *__restrict__ colterm)
+{
+    extern __shared__ int s_wsum[];                      // [taps * C]
+    const int cols4 = taps * C / 4;
+    for (int j = threadIdx.x; j < cols4; j += 1024) {
+        int a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+        for (int k = 0; k < K; ++k) {
+            const int v = (int)__ldg(reinterpret_cast<const uint32_t *>(codes) + (int64_t)k * cols4 + j);
+            a0 = __dp4a(v, 0x00000001, a0); a1 = __dp4a(v, 0x00000100, a1); a2 = __dp4a(v, 0x00010000, a2); a3 = __dp4a(v, 0x01000000, a3);
+        }
+        s_wsum[4 * j] = a0; s_wsum[4 * j + 1] = a1; s_wsum[4 * j + 2] = a2; s_wsum[4 * j + 3] = a3;
+    }
+    __syncthreads();
+    const int zg = q_g->zero_point;
+    for (int i = threadIdx.x; i < 16 * C; i += 1024) {
+        const int cls = i / C, c = i - cls * C;
+        const bool top = cls & 1, bottom = cls & 2, left = cls & 4, right = cls & 8;
+        int sum = 0;
+        for (int r = 0; r < R; ++r) {
+            // gradient row h + pad - r feeds input row h: tap rows below the centre fall off the first row
+            if ((r > pad && top) || (r < pad && bottom)) continue;
+            for (int t = 0; t < S; ++t) {
+                if ((t > pad && left) || (t < pad && right)) continue;
+                sum += s_wsum[(r * S + t) * C + c];
+            }
+        }
+        colterm[i] = -zg * sum;
+    }
+}
+
 // rowterm[pixel] = -z_w * (sum of the input's channel sums over the taps inside the image)
 //                   + (taps inside) * Cred * z_in * z_w          (pad is 0 or 1)
 // blockIdx.y = image, blockIdx.x * 256 + threadIdx.x = position inside it; the nine taps unrolled under predicates
@@ -874,6 +986,32 @@ __global__ void __launch_bounds__(128) colstat_finalize_kernel(const float *__re
 }
 
 int colstat_rows_max() { return sm_count(); }
+
+// Whether filter_prep_kernel takes this filter: small enough for one block and its shared-memory table.
+bool filter_prep_supported(const qbp_conv_desc *d, const float *w, const int8_t *codes)
+{
+    const int64_t elems = (int64_t)d->K * d->R * d->S * d->C;
+    return d->C % 4 == 0 && elems <= (1 << 18) && (int64_t)d->K * d->R * d->S <= 8192 && aligned16(w) && ((uintptr_t)codes & 3) == 0;
+}
+
+int launch_filter_dgrad_colterm(const qbp_conv_desc *d, const int8_t *codes, const qbp_qparams *q_g, int32_t *colterm, cudaStream_t st)
+{
+    const int taps = d->R * d->S;
+    QBP_TRACE_BEGIN(st);
+    filter_dgrad_colterm_kernel<<<1, 1024, sizeof(int) * (size_t)taps * d->C, st>>>(codes, d->K, taps, d->C, d->R, d->S, d->pad, q_g, colterm);
+    QBP_LAUNCH_OK("filter_dgrad_colterm_kernel");
+    return QBP_OK;
+}
+
+int launch_filter_prep(const qbp_conv_desc *d, const float *w, const qbp_qparams *q_in, int8_t *codes, qbp_qparams *qw,
+                       int32_t *colterm, cudaStream_t st)
+{
+    const int taps = d->R * d->S;
+    QBP_TRACE_BEGIN(st);
+    filter_prep_kernel<<<1, 1024, sizeof(int) * (size_t)d->K * taps, st>>>(w, d->K, taps, d->C, d->R, d->S, d->pad, q_in, codes, qw, colterm);
+    QBP_LAUNCH_OK("filter_prep_kernel");
+    return QBP_OK;
+}
 
 // Self-test of the bounded wait (diagnostics): one warp waits on an mbarrier on which nothing ever arrives, with
 // the wait wrappers the product kernels use and a limit of `limit` cycles; the wait gives up, the status word is
@@ -1016,6 +1154,9 @@ static int launch_mma(MmaParams &P, int tiles_m, bool clear_status, cudaStream_t
     P.d_tiles_h = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_h);
     const size_t smem = (size_t)fixed + P.b_res_bytes + (size_t)stages * stage_bytes;
     const bool tail = P.ep_fold || P.ep_relu || P.ep_q;
+    // 32-byte stores need the rows of the output 32-byte aligned (N a multiple of 16 is given)
+    // (not with column statistics: those need the staging slab anyway, and both together were slower: 0.094 against 0.072 ms)
+    P.direct = (P.out && !P.st_sum && ((uintptr_t)P.out & 31) == 0 && P.N % 8 == 0) ? 1 : 0;
     static PerDeviceOnce configured[2];
     if (tail) QBP_SMEM_OPT_IN(configured[1], qbp_mma_kernel<true>, kSmemBudget);
     else      QBP_SMEM_OPT_IN(configured[0], qbp_mma_kernel<false>, kSmemBudget);
@@ -1112,9 +1253,17 @@ extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8(int transA, in
     return gemm_s8_impl(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, ep, nullptr, ws, ws_bytes, (cudaStream_t)stream);
 }
 
+extern "C" __attribute__((visibility("default"))) int qbp_gemm_s8_sums(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A,
+                           const qbp_qparams *qa, const int32_t *a_sums, const int8_t *B, const qbp_qparams *qb,
+                           const int32_t *b_sums, int32_t *acc_out, float *C, const qbp_epilogue *ep, void *ws,
+                           size_t ws_bytes, void *stream)
+{
+    return gemm_s8_impl(transA, transB, M, N, K, A, qa, B, qb, acc_out, C, ep, nullptr, ws, ws_bytes, (cudaStream_t)stream, a_sums, b_sums);
+}
+
 int qbp::gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
                       const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const qbp_epilogue *ep,
-                      int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st)
+                      int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int32_t *a_sums, const int32_t *b_sums)
 {
     if (M <= 0 || N <= 0 || K <= 0) return fail(QBP_ERR_INVALID_ARG, "gemm_s8: M, N, K must be positive");
     if (M % 16 || N % 16 || K % 16) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "gemm_s8: M, N, K must be multiples of 16");
@@ -1148,18 +1297,25 @@ int qbp::gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, c
     }
 
     // code sums along the reduction
-    int rc;
-    if (!transA) rc = launch_rowsum(A, true, M, K, (int32_t *)tmp_m, st);
-    else         rc = launch_colsum(A, true, K, M, tmp_m, st);
-    if (rc) return rc;
-    if (transB) rc = launch_rowsum(B, true, N, K, (int32_t *)tmp_n, st);
-    else        rc = launch_colsum(B, true, K, N, tmp_n, st);
-    if (rc) return rc;
+    int rc = QBP_OK;
+    // (sums along stored rows are int32, along stored columns int64; the caller's are int32 either way)
+    const bool a32 = a_sums || !transA, b32 = b_sums || transB;
+    if (!a_sums) {
+        if (!transA) rc = launch_rowsum(A, true, M, K, (int32_t *)tmp_m, st);
+        else         rc = launch_colsum(A, true, K, M, tmp_m, st);
+        if (rc) return rc;
+    }
+    if (!b_sums) {
+        if (transB) rc = launch_rowsum(B, true, N, K, (int32_t *)tmp_n, st);
+        else        rc = launch_colsum(B, true, K, N, tmp_n, st);
+        if (rc) return rc;
+    }
+    const int32_t *ra32 = a_sums ? a_sums : (const int32_t *)tmp_m, *cb32 = b_sums ? b_sums : (const int32_t *)tmp_n;
     const int64_t mx = std::max(M, N);
     QBP_TRACE_BEGIN(st);
     gemm_terms_kernel<<<(int)((mx + 255) / 256), 256, 0, st>>>(
-        transA ? nullptr : (const int32_t *)tmp_m, transA ? (const long long *)tmp_m : nullptr,
-        transB ? (const int32_t *)tmp_n : nullptr, transB ? nullptr : (const long long *)tmp_n, M, N, K, qa, qb,
+        a32 ? ra32 : nullptr, a32 ? nullptr : (const long long *)tmp_m,
+        b32 ? cb32 : nullptr, b32 ? nullptr : (const long long *)tmp_n, M, N, K, qa, qb,
         rowterm, colterm);
     QBP_LAUNCH_OK("gemm_terms_kernel");
 
@@ -1286,7 +1442,8 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
         return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: column statistics for at most %d channels", QBP_EPILOGUE_MAX_COLUMNS);
     if (tail) {
         const int n_out = mode == QBP_CONV_DGRAD ? d->C : d->K;
-        if (stats) return fail(QBP_ERR_INVALID_ARG, "conv_s8: column statistics are of the plain output (no epilogue tail)");
+        if (stats && (tail->fold || tail->relu || tail->q))
+            return fail(QBP_ERR_INVALID_ARG, "conv_s8: column statistics are of the plain output (no epilogue tail)");
         if (want_codes && (!tail->rq || !aligned16(tail->q))) return fail(QBP_ERR_INVALID_ARG, "conv_s8: 8-bit output needs parameters and a 16-byte aligned buffer");
         if (tail->fold && n_out > 256)
             return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: the fused normalisation takes at most 256 output channels");
@@ -1311,14 +1468,16 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     if (!(tail && tail->keep_terms)) {
         if (in_chan_sum) chan_sum = const_cast<int32_t *>(in_chan_sum);
         else if ((rc = launch_rowsum(in, true, pix, Cred, chan_sum, st))) return rc;
-        if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
-        else        rc = launch_colsum(wgt, true, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
-        if (rc) return rc;
-        QBP_TRACE_BEGIN(st);
-        conv_colterm_kernel<<<dim3((Nout + 127) / 128, 16), 128, 0, st>>>(
-            dgrad ? nullptr : (const int32_t *)wsum, dgrad ? (const long long *)wsum : nullptr, Nout, d->R, d->S, d->pad,
-            dgrad ? 1 : 0, q_in, colterm);
-        QBP_LAUNCH_OK("conv_colterm_kernel");
+        if (!(tail && tail->colterm)) {          // (else: the column terms came with the filter's codes)
+            if (!dgrad) rc = launch_rowsum(wgt, true, (int64_t)d->K * taps, d->C, (int32_t *)wsum, st);   // [k][tap]
+            else        rc = launch_colsum(wgt, true, d->K, (int64_t)taps * d->C, wsum, st);                    // [tap][c]
+            if (rc) return rc;
+            QBP_TRACE_BEGIN(st);
+            conv_colterm_kernel<<<dim3((Nout + 127) / 128, 16), 128, 0, st>>>(
+                dgrad ? nullptr : (const int32_t *)wsum, dgrad ? (const long long *)wsum : nullptr, Nout, d->R, d->S, d->pad,
+                dgrad ? 1 : 0, q_in, colterm);
+            QBP_LAUNCH_OK("conv_colterm_kernel");
+        }
         QBP_TRACE_BEGIN(st);
         conv_rowterm_kernel<<<dim3((unsigned)((d->H * d->W + 255) / 256), (unsigned)d->N), 256, 0, st>>>(
             chan_sum, d->H * d->W, d->H, d->W, make_fastdiv(d->W), d->pad, Cred, q_in, q_w, rowterm);
@@ -1330,6 +1489,7 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
     P.msub = 1; P.ncls = 16; P.nslab = 1;
     if (stats) { P.st_lo = stats->lo; P.st_hi = stats->hi; P.st_sum = stats->sum; }
     if (tail) { P.ep_fold = tail->fold; P.ep_relu = tail->relu; P.ep_rq = tail->rq; P.ep_q = tail->q; }
+    if (tail && tail->colterm) colterm = const_cast<int32_t *>(tail->colterm);
     P.H = d->H; P.W = d->W; P.Nimg = d->N; P.pad = d->pad; P.S = d->S; P.Cred = Cred;
     const uint32_t cb = Cred % 128 == 0 ? 128u : Cred % 64 == 0 ? 64u : 32u;      // reduction bytes per stage row
     P.chunk_bytes = (int)cb;

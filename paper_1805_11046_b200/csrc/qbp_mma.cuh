@@ -42,7 +42,14 @@ int rangebn_fold_from_parts(int64_t n, int64_t C, const float *gamma, const floa
 // column, as rangebn_fold_from_parts leaves them), ReLU, and 8-bit codes of the result with parameters *rq
 // (q [M x N], row_sums [M] nullable).  keep_terms: the zero-point term kernels ran for the same operands in the
 // call just before on the same workspace and are not run again.
-struct EpilogueTail { const float4 *fold; int relu; const qbp_qparams *rq; int8_t *q; int32_t *row_sums; int keep_terms; };
+// colterm (nullable): the column terms [16][N] of this product, already computed (launch_filter_prep).
+struct EpilogueTail { const float4 *fold; int relu; const qbp_qparams *rq; int8_t *q; int32_t *row_sums; int keep_terms; const int32_t *colterm; };
+// A small filter quantised and its forward column terms computed in one launch (qbp_mma.cu).
+bool filter_prep_supported(const qbp_conv_desc *d, const float *w, const int8_t *codes);
+int launch_filter_prep(const qbp_conv_desc *d, const float *w, const qbp_qparams *q_in, int8_t *codes, qbp_qparams *qw,
+                       int32_t *colterm, cudaStream_t st);
+// ... and the layer-gradient product's column terms [16][C] from such a filter's codes, in one launch.
+int launch_filter_dgrad_colterm(const qbp_conv_desc *d, const int8_t *codes, const qbp_qparams *q_g, int32_t *colterm, cudaStream_t st);
 
 // ext_status (here and below; nullable): a status word the caller owns and has cleared -- the product raises it when
 // a bounded wait runs out and never clears it; NULL: the word is the first int of `ws`, cleared by the call itself.
@@ -51,7 +58,8 @@ int conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const qbp_q
                  int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const EpilogueTail *tail = nullptr);
 int gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const int8_t *A, const qbp_qparams *qa,
                  const int8_t *B, const qbp_qparams *qb, int32_t *acc_out, float *C, const qbp_epilogue *ep,
-                 int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st);
+                 int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int32_t *a_sums = nullptr,
+                 const int32_t *b_sums = nullptr);
 // tot_x [C] / tot_g16 [K] (convolution; nullable, both or none): per-channel totals of the stored x codes and of the
 // stored 16-bit gradient codes (256 * hi + lo) over all positions, left by the kernels that wrote the codes.
 int wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,

@@ -236,7 +236,9 @@ def test_chained_bottleneck_stack_needs_no_scan_between_layers(B, batch):
     lean[1].forward(None, to_dev(st["w"][1]))
     names = [n for n, _ in B.trace_records()]
     B.trace_enable(False)
-    assert names.count("range_partial_kernel") == 1 and names.count("quantize_kernel") == 1      # the filter's only
+    # (the small filter is scanned and quantised by one launch of its own; nothing scans or quantises the activation)
+    assert "range_partial_kernel" not in names and "quantize_kernel" not in names and names.count("filter_prep_kernel") == 1
+    assert len(names) <= 7
 
 
 def test_chained_stack_backward_runs_on_the_handed_on_codes(B):

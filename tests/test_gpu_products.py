@@ -347,3 +347,22 @@ def test_conv_epilogue_relu_and_requantisation(B, N_, H, W, C_, K_, R, mode):
                                  requant=(B.range_qparams(lo, hi), q, qp, rs))
     assert B.status_word(res[2]) == 0
     _check_requant(B, res[1], q, qp, rs, oout, True, (lo, hi))
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (208, 80, 144), (1024, 512, 256)])
+@pytest.mark.parametrize("tA,tB", [(False, False), (False, True), (True, False), (True, True)])
+def test_gemm_with_caller_code_sums(B, M, N, K, tA, tB):
+    """The code sums along the reduction handed in (as a chain of calls has them from the quantiser): same product,
+    and no sum kernel in the launch list."""
+    A = random_codes((K, M) if tA else (M, K), 41); Bm = random_codes((N, K) if tB else (K, N), 42)
+    za, zb, sa, sb = 3, -11, 0.5, 0.25
+    a_sums = (A.astype(np.int32).sum(0 if tA else 1)).astype(np.int32); b_sums = (Bm.astype(np.int32).sum(1 if tB else 0)).astype(np.int32)
+    B.trace_enable(True)
+    acc, out, ws = B.qbp_gemm_s8(to_dev(A), _qp(B, sa, za), to_dev(Bm), _qp(B, sb, zb), transA=tA, transB=tB, want_acc=True,
+                                 a_sums=to_dev(a_sums), b_sums=to_dev(b_sums))
+    names = [n for n, _ in B.trace_records()]
+    B.trace_enable(False)
+    assert "rowsum_kernel" not in names and "colsum_kernel" not in names
+    oacc, oout, bad = O.gemm_s8(A, za, Bm, zb, sa, sb, transA=tA, transB=tB)
+    assert bad == 0 and B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(out), oout)
