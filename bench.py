@@ -36,11 +36,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
 # (captured at the full batch of 256).  None: not captured.
 # Keyed by (kernel, occurrence within the step), like KERNEL_WORK; dropped when a kernel changes.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {("quantize_kernel", 1): (205.6e6 + 119.2e6) / 51380224}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {("quantize_kernel", 1): (205.6e6 + 119.7e6) / 51380224}
 # Kernels bound by plain instruction issue rather than by HBM: thread instructions per element, from the same
 # captures (smsp__inst_executed.sum x 32 / elements).  Their roofline is the issue rate of the SMs:
 # SMs x 4 schedulers x 1 warp instruction per clock x 32 threads x the maximum SM clock.
-ALU_INSTR_PER_ELEMENT = {("quantize_kernel", 1): 7.336e7 * 32 / 51380224}
+ALU_INSTR_PER_ELEMENT = {("quantize_kernel", 1): 6.893e7 * 32 / 51380224}
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 
 
@@ -665,8 +665,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--batch", type=int, default=BATCH, help="images per GPU (the workload is quoted at 256)")
-    ap.add_argument("--cpu-sample-batch", type=int, default=BATCH,
-                    help="images of the layer the CPU oracle is timed on (the whole batch takes about 15 s on 16 cores)")
+    ap.add_argument("--cpu-sample-batch", type=int, default=128,
+                    help="images of the layer the CPU oracle is timed on (128 of the 256 take about 15 s on 16 cores)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the dense-GEMM and Range BN sweep blocks of the line")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a captured CUDA graph of the step")

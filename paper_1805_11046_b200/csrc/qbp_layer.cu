@@ -274,14 +274,17 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     // two copies of the gradient: 8 bits for the layer gradient, 16 bits for the weight gradient
     // (convolution with the input's per-channel code totals at hand: the bifurcation leaves the gradient's, and the
     // weight gradient reads only the border positions again for its zero-point terms)
-    const bool totals = s.conv && saved->x_chan_sums && quantizer_totals_supported(s.cout) && s.rows < (1ll << 22);
+    // ... and when the weight-gradient product has a spare chunk of MMA rows, it takes the gradient's totals itself
+    const bool self_totals = s.conv && saved->x_chan_sums && wgrad_self_totals(&L->conv) && s.rows < (1ll << 22);
+    const bool totals = s.conv && saved->x_chan_sums && (self_totals || quantizer_totals_supported(s.cout)) && s.rows < (1ll << 22);
     int64_t *tot_g = totals ? tot_g_buffer(L, s, ws) : nullptr;
     rc = bifurcate_with_range_partials(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
-                                       s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st, tot_g);
+                                       s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st,
+                                       self_totals ? nullptr : tot_g);
     if (rc) return rc;
     if (s.conv) {
         // (a small filter: the layer gradient's column terms in one launch, else two kernels inside the product's call)
-        const bool small = (int64_t)L->conv.R * L->conv.S * L->conv.C <= 12288 && s.w_elems <= (1 << 18) && L->conv.C % 4 == 0;
+        const bool small = (int64_t)L->conv.R * L->conv.S * L->conv.C <= 12288 && s.w_elems <= 49152 && L->conv.C % 4 == 0;
         int32_t *ct = small ? colterm_buffer(L, s, ws) : nullptr;
         if (small && (rc = launch_filter_dgrad_colterm(&L->conv, saved->w_codes, qp8, ct, st))) return rc;
         const EpilogueTail with_colterm{nullptr, 0, nullptr, nullptr, nullptr, 0, ct};
@@ -289,7 +292,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
                           small ? &with_colterm : nullptr);
         if (rc) return rc;
         return wgrad_s16_impl(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws, scratch, st,
-                              totals ? saved->x_chan_sums : nullptr, tot_g);
+                              totals ? saved->x_chan_sums : nullptr, tot_g, !self_totals);
     }
     // dx [batch x in] = g8 [batch x out] . w^T, w stored [in x out]
     rc = gemm_s8_impl(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, nullptr, status, ws, scratch, st);

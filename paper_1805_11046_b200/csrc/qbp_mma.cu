@@ -991,7 +991,8 @@ int colstat_rows_max() { return sm_count(); }
 bool filter_prep_supported(const qbp_conv_desc *d, const float *w, const int8_t *codes)
 {
     const int64_t elems = (int64_t)d->K * d->R * d->S * d->C;
-    return d->C % 4 == 0 && elems <= (1 << 18) && (int64_t)d->K * d->R * d->S <= 8192 && aligned16(w) && ((uintptr_t)codes & 3) == 0;
+    // (one block: beyond some 48 K elements the five launches it replaces are faster)
+    return d->C % 4 == 0 && elems <= 49152 && (int64_t)d->K * d->R * d->S <= 8192 && aligned16(w) && ((uintptr_t)codes & 3) == 0;
 }
 
 int launch_filter_dgrad_colterm(const qbp_conv_desc *d, const int8_t *codes, const qbp_qparams *q_g, int32_t *colterm, cudaStream_t st)

@@ -65,7 +65,9 @@ int gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const 
 int wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
                    const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
                    int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int64_t *tot_x = nullptr,
-                   const int64_t *tot_g16 = nullptr);
+                   const int64_t *tot_g16 = nullptr, bool tot_g_filled = true);
+// tot_g_filled == false: tot_g16 is a buffer [K] that the product fills itself (possible when wgrad_self_totals(d)).
+bool wgrad_self_totals(const qbp_conv_desc *d);
 // Bifurcation with optional per-channel totals of the 16-bit codes (tot16 [cols], zeroed here) -- see above.
 // Shapes the convolution products / the convolution weight gradient implement.
 bool conv_supported(const qbp_conv_desc *d);

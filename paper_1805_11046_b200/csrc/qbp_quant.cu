@@ -356,7 +356,8 @@ __device__ __forceinline__ uint32_t pack_bytes2(const uint32_t (&c)[4])
 
 // PERCH is a template parameter so that the per-tensor instance (the hot one: it is bound by its instruction
 // count when rounding stochastically) carries none of the per-channel parameter handling.
-template <bool SR, int VEC, bool PERCH>
+// TOTALS: the instance that also leaves the per-channel totals (the others carry none of that work).
+template <bool SR, int VEC, bool PERCH, bool TOTALS>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restrict__ x, int64_t n, int cols,
                                                             const qbp_qparams *__restrict__ qp8,
                                                             uint32_t id8, const qbp_qparams *__restrict__ qp16,
@@ -437,7 +438,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                 const uint32_t packed = (SR ? pack_bytes2(c) : pack_bytes0(c)) ^ 0x80808080u;       // stored = unsigned code - 128
                 reinterpret_cast<uint32_t *>(o.q8)[j] = packed;
                 if (o.rowsum8) rs[u] = __dp4a((int)packed, 0x01010101, 0);
-                if (o.chansum8) {
+                if (TOTALS && o.chansum8) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) cs8[e] = __dp4a((int)packed, 1 << (8 * e), cs8[e]);
                 }
@@ -456,7 +457,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                     c[e] = SR ? quantize_sr16_top_half(xs[e], p16.inv, p16.zp_u, r[e])
                               : (uint32_t)quantize_code<SR>(xs[e], p16.inv, p16.zp_u, 65535.0f, r[e]);
                 }
-                if (o.chansum16) {
+                if (TOTALS && o.chansum16) {
                     // unsigned codes here (the offset of 32768 per element is taken off when the block adds its totals up)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) cs16[e] += SR ? c[e] >> 16 : c[e];
@@ -492,7 +493,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     if (blockIdx.x == 0 && threadIdx.x == 0)
         for (int64_t i = nv << 2; i < n; ++i)
             quantize_scalar<SR>(x, i, cols, PERCH, qp8, id8, qp16, id16, keys, o, index_base);
-    if (!PERCH && (o.chansum8 || o.chansum16)) {
+    if (TOTALS && !PERCH && (o.chansum8 || o.chansum16)) {
         // (cols / 4 divides the block size and the grid stride: the thread's channels are 4 * (threadIdx.x mod cols / 4) ...)
         // (a block sees fewer than 65536 rows -- the launcher's rule -- so its totals fit int32)
         int *s_cs = reinterpret_cast<int *>(s_qp);           // [cols] 8-bit totals, then [cols] 16-bit ones
@@ -653,14 +654,17 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
         return fail(QBP_ERR_INVALID_ARG, "quantize: per-channel totals need the vector path and cols / 4 a power of two <= %d", kThreads);
     const size_t smem = totals ? (size_t)cols * 2 * sizeof(int) : (size_t)smem_cols * 2 * sizeof(float2);
     const int64_t groups = (n + per_block - 1) / per_block;
-#define QBP_QUANT(SR_, VEC_, PC_)                                                                                       \
+#define QBP_QUANT2(SR_, VEC_, PC_, TOT_)                                                                                \
     do {                                                                                                                \
-        const int grid = grid_for(blocks_per_sm(quantize_kernel<SR_, VEC_, PC_>, kThreads), groups);                    \
+        const int grid = grid_for(blocks_per_sm(quantize_kernel<SR_, VEC_, PC_, TOT_>, kThreads), groups);              \
         QBP_TRACE_BEGIN(st);                                                                                            \
-        quantize_kernel<SR_, VEC_, PC_><<<grid, kThreads, (VEC_) == 4 ? smem : 0, st>>>(x, n, c, qp8, id8, qp16, id16,  \
+        quantize_kernel<SR_, VEC_, PC_, TOT_><<<grid, kThreads, (VEC_) == 4 ? smem : 0, st>>>(x, n, c, qp8, id8, qp16, id16,  \
                                                                                          key, o, (VEC_) == 4 ? smem_cols : 0, index_base); \
     } while (0)
-    if (sr) {
+#define QBP_QUANT(SR_, VEC_, PC_) QBP_QUANT2(SR_, VEC_, PC_, false)
+    if (totals) {           // (vector path, per tensor: checked above)
+        if (sr) QBP_QUANT2(true, 4, false, true); else QBP_QUANT2(false, 4, false, true);
+    } else if (sr) {
         if (vec) { if (perch) QBP_QUANT(true, 4, true); else QBP_QUANT(true, 4, false); }
         else     { if (perch) QBP_QUANT(true, 1, true); else QBP_QUANT(true, 1, false); }
     } else {
@@ -668,6 +672,7 @@ static int launch_quantize(const float *x, int64_t n, int64_t cols, int perch, i
         else     { if (perch) QBP_QUANT(false, 1, true); else QBP_QUANT(false, 1, false); }
     }
 #undef QBP_QUANT
+#undef QBP_QUANT2
     QBP_LAUNCH_OK("quantize_kernel");
     return QBP_OK;
 }

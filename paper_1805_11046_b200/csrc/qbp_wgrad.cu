@@ -87,6 +87,11 @@ struct WgradParams {
     unsigned long long *cls_x, *cls_hi, *cls_lo;
     const uint8_t *codes_x, *codes_hi, *codes_lo;
     uint32_t cls_off;
+    // The gradient's per-channel totals from the product itself: when the taps do not fill the last A tile, its first
+    // spare chunk is filled with the code 1 once (nothing else writes there), so that the first accumulator row of
+    // that chunk is sum over all positions of 1 * g -- MMA rows that were computed and thrown away before.  The
+    // epilogue adds that row into ones_tot [N] (zeroed beforehand).  NULL: not used.
+    unsigned long long *ones_tot;
 };
 
 // Which item and slice a CTA works on.
@@ -317,6 +322,15 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         s_counts[0] = nl;
     }
     if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
+    if (P.ones_tot && last_group) {
+        // the spare chunk of the last A tile, in every stage: the code 1 in every byte (whatever the swizzle)
+        const int j_last = n_tiles - 1, c_spare = chunks_of(P.a_tiles - 1);
+        for (int st_i = 0; st_i < stages; ++st_i) {
+            uint4 *dst = reinterpret_cast<uint4 *>(smem + (size_t)st_i * stage_bytes + (size_t)j_last * a_tile_bytes + (size_t)c_spare * P.a_chunk_bytes);
+            for (uint32_t i = threadIdx.x; i < P.a_chunk_bytes / 16; i += kWgThreads) dst[i] = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
+        }
+        fence_proxy_async();
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -406,6 +420,13 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
                     tmem_ld_32x32(t_addr + (uint32_t)c0, rh);
                     tmem_ld_32x32(t_addr + (uint32_t)(P.bn + c0), rl);
                     tmem_ld_wait();
+                    if (P.ones_tot && at == P.a_tiles - 1 && row == P.rb_a * chunks_of(at)) {
+                        // the row of ones: this slice's sum of the 16-bit gradient codes, per output channel
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (n0 + c0 + e < P.N)
+                                atomicAdd(P.ones_tot + n0 + c0 + e, (unsigned long long)(256ll * (long long)(int)rh[e] + (long long)(int)rl[e]));
+                    }
                     if (!valid) continue;
                     if (P.direct) {
                         // the whole reduction is here: zero-points, scale, store
@@ -837,6 +858,19 @@ static bool wgrad_inline_border(const qbp_conv_desc *d)
     return d && d->pad > 0 && ok(d->C) && ok(d->K) && d->H >= 3 && d->W >= 3;
 }
 
+}  // namespace qbp
+
+// Whether the product can take the gradient's per-channel totals itself (a spare chunk in its last A tile).
+bool qbp::wgrad_self_totals(const qbp_conv_desc *d)
+{
+    if (!d || !wgrad_conv_supported(d)) return false;
+    const int rb_a = d->C >= 128 ? 128 : d->C >= 64 ? 64 : 32;
+    const int a_chunks = 128 / rb_a;
+    return d->C % rb_a == 0 && (d->R * d->S) % a_chunks != 0;
+}
+
+namespace qbp {
+
 static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, WgradPlan &pl)
 {
     WgradParams &P = pl.P;
@@ -1001,7 +1035,8 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
 
 int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
                         const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
-                        int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int64_t *tot_x, const int64_t *tot_g16)
+                        int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int64_t *tot_x, const int64_t *tot_g16,
+                        bool tot_g_filled)
 {
     if (!x || !g_hi || !g_lo || !qx || !qg16) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: NULL operand");
     if (!acc_out && !dW) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: acc_out and dW are both NULL");
@@ -1041,7 +1076,7 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
     int rc;
     // (the border tables stay within int32 per block: a block sees at most Nimg * 2 (W + H) border positions)
     const bool from_totals = d && tot_x && tot_g16 && d->H >= 3 && d->W >= 3 && std::max(K, N) <= 1536 &&
-                             (int64_t)d->N * 2 * (d->H + d->W) < (1ll << 22);
+                             (int64_t)d->N * 2 * (d->H + d->W) < (1ll << 22) && (tot_g_filled || wgrad_self_totals(d));
     if (from_totals) {
         // the kernels that wrote the codes left their per-channel totals: only the border positions are read again
         QBP_CUDA_OK(cudaMemsetAsync(sx, 0, (size_t)((char *)(slo + 16 * N) - (char *)sx), st));
@@ -1060,6 +1095,11 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
             QBP_LAUNCH_OK("border_class_sums_kernel");
         }
         P.tot_x = (const long long *)tot_x; P.tot_g = (const long long *)tot_g16;
+        if (!tot_g_filled) {
+            // nobody left the gradient's totals: the product takes them itself (a row of ones in its spare chunk)
+            QBP_CUDA_OK(cudaMemsetAsync(const_cast<int64_t *>(tot_g16), 0, sizeof(int64_t) * (size_t)N, st));
+            P.ones_tot = (unsigned long long *)const_cast<int64_t *>(tot_g16);
+        }
     } else if (d && K == N && d->W <= 256 && M < (1ll << 30) && shi == sx + 16 * K && slo == shi + 16 * N) {
         // as many input as output channels: the three tensors in one launch
         QBP_CUDA_OK(cudaMemsetAsync(sx, 0, sizeof(int64_t) * 48 * K, st));
