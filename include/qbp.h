@@ -436,7 +436,11 @@ typedef struct {
  * checked on its own).  Element counts: x_codes = |x|, w_codes = |w|; z, g,
  * g8, g_hi, g_lo = rows*channels of the product's output (rows = batch or
  * N*P*Q); z is the fp32 output of the product (the input of Range BN), g the
- * fp32 gradient arriving at it.  The g* members are used by the backward only. */
+ * fp32 gradient arriving at it.  The g* members are used by the backward only.
+ * g_lo holds the low bytes of the 16-bit codes with their top bit flipped, i.e.
+ * the signed bytes lo - 128 (g16 = 256*g_hi + (lo - 128) + 128): both limbs
+ * then have one operand type and the layer's weight gradient runs them as one
+ * product of twice the columns. */
 typedef struct {
     int8_t *x_codes;  qbp_qparams *qx;
     int8_t *w_codes;  qbp_qparams *qw;

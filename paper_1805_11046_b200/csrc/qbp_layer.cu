@@ -280,7 +280,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     int64_t *tot_g = totals ? tot_g_buffer(L, s, ws) : nullptr;
     rc = bifurcate_with_range_partials(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st,
-                                       self_totals ? nullptr : tot_g);
+                                       self_totals ? nullptr : tot_g, true);
     if (rc) return rc;
     if (s.conv) {
         // (a small filter: the layer gradient's column terms in one launch, else two kernels inside the product's call)
@@ -292,11 +292,11 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
                           small ? &with_colterm : nullptr);
         if (rc) return rc;
         return wgrad_s16_impl(&L->conv, 0, 0, 0, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws, scratch, st,
-                              totals ? saved->x_chan_sums : nullptr, tot_g, !self_totals);
+                              totals ? saved->x_chan_sums : nullptr, tot_g, !self_totals, true);
     }
     // dx [batch x in] = g8 [batch x out] . w^T, w stored [in x out]
     rc = gemm_s8_impl(0, 1, s.rows, s.cin, s.cout, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, nullptr, status, ws, scratch, st);
     if (rc) return rc;
     return wgrad_s16_impl(nullptr, s.rows, s.cout, s.cin, saved->x_codes, saved->qx, ghi, glo, qp16, nullptr, dw, status, ws,
-                          scratch, st);
+                          scratch, st, nullptr, nullptr, true, true);
 }

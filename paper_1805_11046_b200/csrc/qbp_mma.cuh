@@ -24,7 +24,7 @@ size_t rangebn_range_parts_capacity(int64_t C);
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                                   uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
                                   uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st,
-                                  int64_t *tot16 = nullptr);
+                                  int64_t *tot16 = nullptr, bool lo_signed = false);
 // Whether the quantising kernels can leave per-channel totals for a tensor of `cols` channels.
 bool quantizer_totals_supported(int64_t cols);
 int quantize_s8_with_totals(const float *x, int64_t rows, int64_t cols, int8_t *q, qbp_qparams *qp_out, int32_t *row_sums,
@@ -62,10 +62,14 @@ int gemm_s8_impl(int transA, int transB, int64_t M, int64_t N, int64_t K, const 
                  const int32_t *b_sums = nullptr);
 // tot_x [C] / tot_g16 [K] (convolution; nullable, both or none): per-channel totals of the stored x codes and of the
 // stored 16-bit gradient codes (256 * hi + lo) over all positions, left by the kernels that wrote the codes.
+// lo_signed: g_lo holds the low bytes with the top bit flipped, i.e. the signed bytes lo - 128 (lo_signed in
+// bifurcate_with_range_partials): g16 - zg = 256 * hi + (lo - 128) - (zg - 128), so the two limbs have one operand
+// type and run as one product of twice the columns (the x tile is read from shared memory once, not once per limb),
+// with zg - 128 as the zero-point.
 int wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
                    const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
                    int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int64_t *tot_x = nullptr,
-                   const int64_t *tot_g16 = nullptr, bool tot_g_filled = true);
+                   const int64_t *tot_g16 = nullptr, bool tot_g_filled = true, bool lo_signed = false);
 // tot_g_filled == false: tot_g16 is a buffer [K] that the product fills itself (possible when wgrad_self_totals(d)).
 bool wgrad_self_totals(const qbp_conv_desc *d);
 // Bifurcation with optional per-channel totals of the 16-bit codes (tot16 [cols], zeroed here) -- see above.
@@ -99,7 +103,7 @@ int launch_gemm2(int transA, int transB, int64_t M, int64_t N, int64_t K, const 
 bool wgrad2_eligible(int64_t M, int64_t N, int64_t K);
 int launch_wgrad2(int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx, const int8_t *g_hi,
                   const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW, const long long *rowterm,
-                  const long long *colterm, int *status, cudaStream_t st);
+                  const long long *colterm, int *status, cudaStream_t st, bool lo_signed = false);
 
 // ---- shared-memory operand descriptors ---------------------------------------
 // How one operand tile of a pipeline stage is laid out and walked by the MMAs.

@@ -287,6 +287,9 @@ struct QuantOut {
     // [cols] (nullable; vector path, per tensor, cols / 4 a power of two <= 256: a thread then keeps its four
     // channels for its whole life).  The weight gradient's zero-point terms are built from such totals.
     unsigned long long *chansum8, *chansum16;
+    // 0x80808080: the low bytes are stored with their top bit flipped, i.e. as the signed bytes lo - 128 (the weight
+    // gradient then runs both limbs as one s8 x s8 product); 0: plain unsigned low bytes.
+    uint32_t lo_flip;
 };
 
 struct QParamsReg { float inv, zp_u; };
@@ -329,7 +332,7 @@ __device__ __forceinline__ void quantize_scalar(const float *x, int64_t i, int c
         int s = quantize_code<SR>(v, p.inv, p.zp_u, 65535.0f, rnd) - 32768;
         if (o.q16) o.q16[i] = (int16_t)s;
         if (o.hi) o.hi[i] = (int8_t)(s >> 8);
-        if (o.lo) o.lo[i] = (uint8_t)(s & 0xFF);
+        if (o.lo) o.lo[i] = (uint8_t)((s & 0xFF) ^ (o.lo_flip & 0xFF));
     }
 }
 
@@ -470,10 +473,10 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                     // (low, low, high, high) bytes of two codes each, then the two words: four permutes for both limbs
                     const uint32_t t01 = __byte_perm(c[0], c[1], 0x7362), t23 = __byte_perm(c[2], c[3], 0x7362);
                     reinterpret_cast<uint32_t *>(o.hi)[j] = __byte_perm(t01, t23, 0x7632) ^ 0x80808080u;
-                    reinterpret_cast<uint32_t *>(o.lo)[j] = __byte_perm(t01, t23, 0x5410);
+                    reinterpret_cast<uint32_t *>(o.lo)[j] = __byte_perm(t01, t23, 0x5410) ^ o.lo_flip;
                 } else {
                     if (o.hi) reinterpret_cast<uint32_t *>(o.hi)[j] = (SR ? pack_bytes3(c) : pack_bytes1(c)) ^ 0x80808080u;
-                    if (o.lo) reinterpret_cast<uint32_t *>(o.lo)[j] = SR ? pack_bytes2(c) : pack_bytes0(c);
+                    if (o.lo) reinterpret_cast<uint32_t *>(o.lo)[j] = (SR ? pack_bytes2(c) : pack_bytes0(c)) ^ o.lo_flip;
                 }
             }
         }
@@ -804,9 +807,10 @@ static int static_scratch_address(void **out)
 // The quantising half of the bifurcation, once qp8 / qp16 are known.
 static int bifurcate_tail(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                           uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo,
-                          qbp_qparams *qp16, cudaStream_t st, uint64_t index_base = 0, int64_t *tot16 = nullptr)
+                          qbp_qparams *qp16, cudaStream_t st, uint64_t index_base = 0, int64_t *tot16 = nullptr,
+                          bool lo_signed = false)
 {
-    QuantOut o = {q8, nullptr, hi, lo, nullptr, 0, 0, nullptr, nullptr};
+    QuantOut o = {q8, nullptr, hi, lo, nullptr, 0, 0, nullptr, nullptr, lo_signed ? 0x80808080u : 0u};
     if (tot16 && rows * cols > 0) {                       // (the caller asked quantizer_totals_supported(cols) first)
         QBP_CUDA_OK(cudaMemsetAsync(tot16, 0, sizeof(int64_t) * (size_t)cols, st));
         o.chansum16 = reinterpret_cast<unsigned long long *>(tot16);
@@ -823,12 +827,12 @@ static int bifurcate_tail(const float *g, int64_t rows, int64_t cols, uint64_t s
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                                   uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
                                   uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st,
-                                  int64_t *tot16)
+                                  int64_t *tot16, bool lo_signed)
 {
     QBP_TRACE_BEGIN(st);
     range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
     QBP_LAUNCH_OK("range_finalize_kernel");
-    return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st, 0, tot16);
+    return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st, 0, tot16, lo_signed);
 }
 
 bool quantizer_totals_supported(int64_t cols)

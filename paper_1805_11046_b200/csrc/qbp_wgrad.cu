@@ -49,6 +49,20 @@ struct WgradParams {
     CUtensorMap mapX, mapHi, mapLo;
     OperandLayout a, b;
     uint32_t idesc_hi, idesc_lo;
+    // The low bytes stored as lo - 128 (signed): both limbs have one operand type, and a stage's MMAs take the high
+    // and the low tile side by side as one B operand of 2 * bn columns (the x tile is then read from shared memory
+    // once instead of once per limb).  g16 - zg = 256 * hi + (lo - 128) - (zg - 128): everything downstream works on
+    // those limbs with the zero-point zg - 128.
+    int lo_signed;
+    uint32_t b2_desc_lo, idesc_fused;
+    int tot_g_plain;                 // tot_g holds totals of 256 * hi + lo (left by a quantiser), not of the stored limbs
+    // 3 x 3 convolution from halo tiles (with lo_signed): a stage holds the pixel box of x once, with its border of
+    // one position (10 positions per box row), instead of one shifted copy per tap; a tap's operand is that tile read
+    // from a shifted start (see wg_issue_stage_halo).  halo_bh: box rows per image in a stage (8 or 4; 0: not used).
+    int halo_bh;
+    uint32_t halo_bytes;             // the tile's room in a stage (1024-byte multiple)
+    uint32_t halo_box_bytes;         // bytes one load of it brings
+    uint32_t ones_off;               // offset (from the ring's start) of a region of halo_bytes filled with the code 1
     uint32_t a_chunk_bytes;          // bytes of one A chunk (kr rows x rb_a)
     int conv;                        // 0: x [M x K], g [M x N]; 1: NHWC tensors
     int stages, cg, bn, tmem_cols;   // cg: stages released by one commit
@@ -121,14 +135,21 @@ struct WgMmaArgs {
     int k_iters;
     uint32_t stages, cg;
     uint32_t a_desc_lo, b_desc_lo, idesc_hi;
+    // halo tiles: per A tile of the CTA, (start of its first tap in the halo tile) >> 4 | (distance to its second
+    // tap) >> 4 << 16, and what multiplies the stage's address (>> 4) before that is added: 1, or 1 - 65536 for the
+    // tile whose second chunk is the region of ones (its distance is then counted from the ring's start).
+    uint32_t tile_desc[4], tile_mult[4];
 };
+
 
 __host__ __device__ constexpr uint32_t wg_swizzle_bits(uint32_t row_bytes) { return row_bytes == 128 ? 2u : row_bytes == 64 ? 4u : 6u; }
 
 // The 2 * KK * NT MMAs of a stage of kWgRows reduction rows: the limb outermost (switching between the s8 x s8 and s8 x u8
 // instruction descriptors stalls the MMA pipe), then the k step, then the A tile, so that consecutive MMAs write
 // different accumulators.  FIRST: the stage starts the reduction (its first k step overwrites the accumulators).
-template <int RBA, int RBB, int NT, bool FIRST>
+// FUSED: both limbs are signed and one MMA takes them side by side (N = 2 * RBB; b_lo then carries the distance
+// between the two tiles as its leading byte offset and idesc_hi that N): KK * NT MMAs.
+template <int RBA, int RBB, int NT, bool FIRST, bool FUSED>
 __device__ __forceinline__ void wg_issue_stage(uint32_t tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc_hi)
 {
     constexpr uint32_t a_hi = ((8u * RBA) >> 4) | (1u << 14) | (wg_swizzle_bits(RBA) << 29);
@@ -137,6 +158,17 @@ __device__ __forceinline__ void wg_issue_stage(uint32_t tmem, uint32_t a_lo, uin
     constexpr int KK = kWgRows / 32;                               // k steps per stage
     constexpr uint32_t a_tile16 = (uint32_t)kWgRows * 128u / 16u;  // an A tile: kWgRows rows x 128 bytes
     constexpr uint32_t b_tile16 = (uint32_t)kWgRows * RBB / 16u;   // a limb's tile: kWgRows rows x RBB bytes
+    if (FUSED) {
+#pragma unroll
+        for (int i = 0; i < KK * NT; ++i) {
+            const int kk = i / NT, j = i % NT;
+            const uint32_t ao = (uint32_t)j * a_tile16 + (uint32_t)kk * a_kstep;
+            if (elect_one())
+                mma_i8(tmem + (uint32_t)(j * 2 * RBB), ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + ao),
+                       ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + (uint32_t)kk * b_kstep), idesc_hi, (FIRST && kk == 0) ? 0u : 1u);
+        }
+        return;
+    }
     const uint32_t idesc_lo = idesc_hi ^ (1u << 10);               // the low limb is unsigned
 #pragma unroll
     for (int i = 0; i < 2 * KK * NT; ++i) {
@@ -150,7 +182,7 @@ __device__ __forceinline__ void wg_issue_stage(uint32_t tmem, uint32_t a_lo, uin
 }
 
 // The MMA warp's loop over its slice of the reduction.  False when a wait ran out.
-template <int RBA, int RBB, int NT>
+template <int RBA, int RBB, int NT, bool FUSED>
 __device__ __forceinline__ bool wg_mma_loop(const WgMmaArgs &A)
 {
     uint32_t s = 0, ph = 0;
@@ -162,8 +194,8 @@ __device__ __forceinline__ bool wg_mma_loop(const WgMmaArgs &A)
         tc_fence_after();
         const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | A.a_desc_lo;
         const uint32_t b_lo = (((a_addr + A.a_bytes) >> 4) & 0x3FFFu) | A.b_desc_lo;
-        if (i == 0) wg_issue_stage<RBA, RBB, NT, true>(A.tmem, a_lo, b_lo, A.idesc_hi);
-        else        wg_issue_stage<RBA, RBB, NT, false>(A.tmem, a_lo, b_lo, A.idesc_hi);
+        if (i == 0) wg_issue_stage<RBA, RBB, NT, true, FUSED>(A.tmem, a_lo, b_lo, A.idesc_hi);
+        else        wg_issue_stage<RBA, RBB, NT, false, FUSED>(A.tmem, a_lo, b_lo, A.idesc_hi);
         // release the group of stages this one completes (the commit covers every MMA issued so far)
         if (++in_group == A.cg) {
             if (elect_one()) mma_commit(&A.empty_bar[group]);
@@ -176,15 +208,87 @@ __device__ __forceinline__ bool wg_mma_loop(const WgMmaArgs &A)
     return true;
 }
 
-template <int RBA, int RBB>
+template <int RBA, int RBB, bool FUSED>
 __device__ __forceinline__ bool wg_mma_dispatch_nt(int nt, const WgMmaArgs &A)
 {
     // (128 output columns per tile leave room for two A tiles in tensor memory)
-    if (nt == 1) return wg_mma_loop<RBA, RBB, 1>(A);
-    if (nt == 2) return wg_mma_loop<RBA, RBB, 2>(A);
+    if (nt == 1) return wg_mma_loop<RBA, RBB, 1, FUSED>(A);
+    if (nt == 2) return wg_mma_loop<RBA, RBB, 2, FUSED>(A);
     if (RBB == 128) return false;
-    if (nt == 3) return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 3)>(A);
-    return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 4)>(A);
+    if (nt == 3) return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 3), FUSED>(A);
+    return wg_mma_loop<RBA, RBB, (RBB == 128 ? 1 : 4), FUSED>(A);
+}
+
+// ---- the same from halo tiles ---------------------------------------------------
+// The x tile of a stage is the pixel box (8 positions wide, BH rows, 16 / BH images) with a border of one position:
+// rows of kWgHaloW positions.  The operand of tap (r, s) is the tile read from r * kWgHaloW + s positions in: the
+// shared-memory swizzle is a function of the address, so a window that starts any whole number of positions into the
+// tile reads what TMA wrote there.  A k step of 32 positions is four box rows: groups of eight positions a tile row
+// apart (the stride byte offset), starting at the box row's place in the tile.
+constexpr int kWgHaloW = 10;
+template <int RBA, int BH>
+__host__ __device__ constexpr uint32_t wg_halo_kstep16(int kk)
+{
+    return (uint32_t)((((kk * 4) / BH) * (BH + 2) * kWgHaloW + ((kk * 4) % BH) * kWgHaloW) * RBA / 16);
+}
+
+template <int RBA, int RBB, int NT, bool FIRST, int BH>
+__device__ __forceinline__ void wg_issue_stage_halo(uint32_t tmem, const uint32_t (&a_lo)[NT], uint32_t b_lo, uint32_t idesc)
+{
+    constexpr uint32_t a_hi = (((uint32_t)kWgHaloW * RBA) >> 4) | (1u << 14) | (wg_swizzle_bits(RBA) << 29);
+    constexpr uint32_t b_hi = ((8u * RBB) >> 4) | (1u << 14) | (wg_swizzle_bits(RBB) << 29);
+    constexpr uint32_t b_kstep = 2u * RBB;
+    constexpr int KK = kWgRows / 32;
+#pragma unroll
+    for (int i = 0; i < KK * NT; ++i) {
+        const int kk = i / NT, j = i % NT;
+        if (elect_one())
+            mma_i8(tmem + (uint32_t)(j * 2 * RBB), ((uint64_t)a_hi << 32) | (uint64_t)(a_lo[j] + wg_halo_kstep16<RBA, BH>(kk)),
+                   ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + (uint32_t)kk * b_kstep), idesc, (FIRST && kk == 0) ? 0u : 1u);
+    }
+}
+
+template <int RBA, int RBB, int NT, int BH>
+__device__ __forceinline__ bool wg_mma_loop_halo(const WgMmaArgs &A)
+{
+    uint32_t s = 0, ph = 0, in_group = 0, group = 0;
+    uint32_t a_addr = A.ring;
+    for (int i = 0; i < A.k_iters; ++i) {
+        if (!mbar_wait_uniform(&A.full_bar[s], ph)) return false;
+        tc_fence_after();
+        const uint32_t base = (a_addr >> 4) & 0x3FFFu;
+        uint32_t a_lo[NT];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) a_lo[j] = base * A.tile_mult[j] + A.tile_desc[j];
+        const uint32_t b_lo = (((a_addr + A.a_bytes) >> 4) & 0x3FFFu) | A.b_desc_lo;
+        if (i == 0) wg_issue_stage_halo<RBA, RBB, NT, true, BH>(A.tmem, a_lo, b_lo, A.idesc_hi);
+        else        wg_issue_stage_halo<RBA, RBB, NT, false, BH>(A.tmem, a_lo, b_lo, A.idesc_hi);
+        if (++in_group == A.cg) {
+            if (elect_one()) mma_commit(&A.empty_bar[group]);
+            in_group = 0; ++group;
+        }
+        a_addr += A.stage_bytes;
+        if (++s == A.stages) { s = 0; ph ^= 1u; group = 0; a_addr = A.ring; }
+    }
+    if (elect_one()) mma_commit(A.acc_bar);
+    return true;
+}
+
+template <int RBA, int RBB>
+__device__ __forceinline__ bool wg_mma_dispatch_halo(int nt, int bh, const WgMmaArgs &A)
+{
+    if (RBA < 64 || nt < 1 || nt > 4 || (RBB == 128 && nt > 2)) return false;
+    constexpr int R = RBA < 64 ? 64 : RBA;             // (instances for the layouts that can occur only)
+    if (bh == 8) {
+        if (nt == 1) return wg_mma_loop_halo<R, RBB, 1, 8>(A);
+        if (nt == 2) return wg_mma_loop_halo<R, RBB, 2, 8>(A);
+        if (nt == 3) return wg_mma_loop_halo<R, RBB, (RBB == 128 ? 1 : 3), 8>(A);
+        return wg_mma_loop_halo<R, RBB, (RBB == 128 ? 1 : 4), 8>(A);
+    }
+    if (nt == 1) return wg_mma_loop_halo<R, RBB, 1, 4>(A);
+    if (nt == 2) return wg_mma_loop_halo<R, RBB, 2, 4>(A);
+    if (nt == 3) return wg_mma_loop_halo<R, RBB, (RBB == 128 ? 1 : 3), 4>(A);
+    return wg_mma_loop_halo<R, RBB, (RBB == 128 ? 1 : 4), 4>(A);
 }
 
 // Sixteen per-channel sums from one 16-byte group of codes (dot products that pick one byte each).
@@ -286,7 +390,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     const int it_end = (int)((int64_t)P.iters_total * (wi.slice + 1) / wi.slices);
     const int k_iters = it_end - it_begin;
     const int n_tiles = min(P.ma, P.a_tiles - ag * P.ma);        // A tiles this CTA owns
-    const uint32_t a_bytes = a_tile_bytes * (uint32_t)n_tiles;
+    const uint32_t a_bytes = P.halo_bh ? P.halo_bytes : a_tile_bytes * (uint32_t)n_tiles;
     const uint32_t stage_bytes = a_bytes + 2u * P.b.tile_bytes;
     const bool last_group = ag == P.a_groups - 1;
     const int stages = last_group ? P.stages_last : P.stages, cg = last_group ? P.cg_last : P.cg;
@@ -307,7 +411,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         int nl = 0;
         s_load[nl++] = make_int4((int)a_bytes, 1, n0, 0);
         s_load[nl++] = make_int4((int)(a_bytes + P.b.tile_bytes), 2, n0, 0);
-        for (int j = 0; j < n_tiles; ++j) {
+        if (P.halo_bh) s_load[nl++] = make_int4(0, 0, 0, ((-P.pad) & 0xFFFF) | ((-P.pad) << 16));     // the box with its border
+        for (int j = 0; j < (P.halo_bh ? 0 : n_tiles); ++j) {
             const int at = ag * P.ma + j, nc = chunks_of(at);
             for (int c = 0; c < nc; ++c) {
                 const int dst = (int)((uint32_t)j * a_tile_bytes + (uint32_t)c * P.a_chunk_bytes);
@@ -322,7 +427,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         s_counts[0] = nl;
     }
     if (warp == 1) { tmem_alloc(&tmem_slot, (uint32_t)P.tmem_cols); tmem_relinquish(); }
-    if (P.ones_tot && last_group) {
+    if (P.ones_tot && last_group && P.halo_bh) {
+        // halo tiles: the spare chunk of the last A tile is read from a region of its own, filled with the code 1
+        uint4 *dst = reinterpret_cast<uint4 *>(smem + P.ones_off);
+        for (uint32_t i = threadIdx.x; i < P.halo_bytes / 16; i += kWgThreads) dst[i] = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
+        fence_proxy_async();
+    } else if (P.ones_tot && last_group) {
         // the spare chunk of the last A tile, in every stage: the code 1 in every byte (whatever the swizzle)
         const int j_last = n_tiles - 1, c_spare = chunks_of(P.a_tiles - 1);
         for (int st_i = 0; st_i < stages; ++st_i) {
@@ -340,8 +450,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
     if (warp == 0) {
         // ---------------------------------------------------- TMA producer (lane 0 owns the barriers)
         const int n_loads = s_counts[0];
-        uint32_t tx_bytes = 2u * P.b.tile_bytes;
-        for (int j = 0; j < n_tiles; ++j) tx_bytes += (uint32_t)chunks_of(ag * P.ma + j) * P.a_chunk_bytes;
+        uint32_t tx_bytes = 2u * P.b.tile_bytes + (P.halo_bh ? P.halo_box_bytes : 0u);
+        for (int j = 0; j < (P.halo_bh ? 0 : n_tiles); ++j) tx_bytes += (uint32_t)chunks_of(ag * P.ma + j) * P.a_chunk_bytes;
         const int4 ld = lane < n_loads ? s_load[lane] : make_int4(0, 0, 0, 0);
         const int dw = (int)(short)(ld.w & 0xFFFF), dh = ld.w >> 16;
         const void *map = ld.y == 0 ? (const void *)&P.mapX : ld.y == 1 ? (const void *)&P.mapHi : (const void *)&P.mapLo;
@@ -378,8 +488,33 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
         A.full_bar = full_bar; A.empty_bar = empty_bar; A.acc_bar = &acc_bar;
         A.ring = smem_u32(smem); A.stage_bytes = stage_bytes; A.a_bytes = a_bytes; A.tmem = tmem_base;
         A.k_iters = k_iters; A.stages = (uint32_t)stages; A.cg = (uint32_t)cg;
-        A.a_desc_lo = P.a.desc_lo; A.b_desc_lo = P.b.desc_lo; A.idesc_hi = P.idesc_hi;
-        timed_out = !wg_mma_dispatch_nt<RBA, RBB>(n_tiles, A);
+        A.a_desc_lo = P.a.desc_lo;
+        if (P.halo_bh) {
+            // where each A tile's taps start in the halo tile (tap (r, s): r tile rows and s positions in)
+            for (int j = 0; j < 4; ++j) {
+                const int at = min(ag * P.ma + j, P.a_tiles - 1);
+                const int tap0 = at * P.a_chunks, tap1 = tap0 + 1;
+                const uint32_t off0 = (uint32_t)((tap0 / P.S) * kWgHaloW + tap0 % P.S) * (uint32_t)P.rb_a >> 4;
+                uint32_t lbo = 0, mult = 1u;
+                if (P.a_chunks == 2 && tap1 < P.taps)
+                    lbo = ((uint32_t)((tap1 / P.S) * kWgHaloW + tap1 % P.S) * (uint32_t)P.rb_a >> 4) - off0;
+                else if (P.a_chunks == 2 && P.ones_tot) {
+                    // the region of ones, from wherever the stage is: (ones - (stage + off0)) << 16 = (ones - off0) << 16 - (stage << 16)
+                    lbo = ((A.ring + P.ones_off) >> 4) - off0;
+                    mult = 1u - 65536u;
+                }
+                A.tile_desc[j] = off0 + (lbo << 16);
+                A.tile_mult[j] = mult;
+            }
+            A.b_desc_lo = P.b2_desc_lo; A.idesc_hi = P.idesc_fused;
+            timed_out = !wg_mma_dispatch_halo<RBA, RBB>(n_tiles, P.halo_bh, A);
+        } else if (P.lo_signed) {
+            A.b_desc_lo = P.b2_desc_lo; A.idesc_hi = P.idesc_fused;
+            timed_out = !wg_mma_dispatch_nt<RBA, RBB, true>(n_tiles, A);
+        } else {
+            A.b_desc_lo = P.b.desc_lo; A.idesc_hi = P.idesc_hi;
+            timed_out = !wg_mma_dispatch_nt<RBA, RBB, false>(n_tiles, A);
+        }
     } else {
         // ------------------------------------------------------- epilogue
         const int quad = warp & 3;
@@ -393,7 +528,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) qbp_wgrad_kernel(const __grid_c
             const int img_begin = (int)((int64_t)P.Nimg * blockIdx.x / gridDim.x), img_end = (int)((int64_t)P.Nimg * (blockIdx.x + 1) / gridDim.x);
             wg_border_sums(true, P.codes_x, P.C, P.H, P.W, img_begin, img_end, tx, t);
             wg_border_sums(true, P.codes_hi, (int)P.N, P.H, P.W, img_begin, img_end, th, t);
-            wg_border_sums(false, P.codes_lo, (int)P.N, P.H, P.W, img_begin, img_end, tl, t);
+            wg_border_sums(P.lo_signed != 0, P.codes_lo, (int)P.N, P.H, P.W, img_begin, img_end, tl, t);
             named_barrier(2, 128);
             for (int i = t; i < 16 * P.C; i += 128)
                 if (tx[i]) atomicAdd(P.cls_x + i, (unsigned long long)(long long)tx[i]);
@@ -635,10 +770,11 @@ __global__ void __launch_bounds__(256, 3) row_class_sums_kernel(const uint8_t *_
 // layer input, the gradient's signed high bytes, its unsigned low bytes); sums: three tables of 16 * C, one after another.
 __global__ void __launch_bounds__(256, 3) row_class_sums3_kernel(const uint8_t *__restrict__ x, const uint8_t *__restrict__ hi,
                                                                  const uint8_t *__restrict__ lo, int Nimg, int H, int W, int C,
-                                                                 int gs, unsigned long long *__restrict__ sums)
+                                                                 int gs, unsigned long long *__restrict__ sums, int lo_signed)
 {
     if (blockIdx.z == 0)      row_class_sums_body<true>(x, Nimg, H, W, C, gs, sums);
     else if (blockIdx.z == 1) row_class_sums_body<true>(hi, Nimg, H, W, C, gs, sums + 16 * C);
+    else if (lo_signed)       row_class_sums_body<true>(lo, Nimg, H, W, C, gs, sums + 32 * C);
     else                      row_class_sums_body<false>(lo, Nimg, H, W, C, gs, sums + 32 * C);
 }
 
@@ -652,13 +788,13 @@ __global__ void __launch_bounds__(256) border_class_sums_kernel(const uint8_t *_
                                                                 const uint8_t *__restrict__ lo, int Nimg, int H, int W, int Cx,
                                                                 int Cg, unsigned long long *__restrict__ sums_x,
                                                                 unsigned long long *__restrict__ sums_hi,
-                                                                unsigned long long *__restrict__ sums_lo)
+                                                                unsigned long long *__restrict__ sums_lo, int lo_signed)
 {
     extern __shared__ int s_acc[];                       // [16][C]
     const uint8_t *q = blockIdx.z == 0 ? x : blockIdx.z == 1 ? hi : lo;
     unsigned long long *sums = blockIdx.z == 0 ? sums_x : blockIdx.z == 1 ? sums_hi : sums_lo;
     const int C = blockIdx.z == 0 ? Cx : Cg;
-    const bool is_signed = blockIdx.z != 2;
+    const bool is_signed = blockIdx.z != 2 || lo_signed;
     for (int i = threadIdx.x; i < 16 * C; i += 256) s_acc[i] = 0;
     __syncthreads();
     const int cv = C >> 4;
@@ -733,9 +869,9 @@ __global__ void __launch_bounds__(256) border_class_sums_kernel(const uint8_t *_
 __global__ void wgrad_terms_kernel(const long long *__restrict__ sx, const long long *__restrict__ shi,
                                    const long long *__restrict__ slo, int64_t M, int64_t N, int64_t K,
                                    const qbp_qparams *qx, const qbp_qparams *qg, long long *__restrict__ rowterm,
-                                   long long *__restrict__ colterm)
+                                   long long *__restrict__ colterm, int zg_shift)
 {
-    const long long zx = qx->zero_point, zg = qg->zero_point;
+    const long long zx = qx->zero_point, zg = qg->zero_point - zg_shift;      // (signed low bytes: lo - 128 against zg - 128)
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < K) rowterm[i] = -zg * sx[i] + M * zx * zg;
     if (i < N) colterm[i] = -zx * (256 * shi[i] + slo[i]);
@@ -756,7 +892,8 @@ __global__ void __launch_bounds__(256) wgrad_finalize_kernel(const WgradParams P
     const int part_lane = threadIdx.x % kLanes;
     const bool live = e_raw < total;
     const int64_t e = live ? e_raw : total - 1;           // (idle lanes of the last warp compute a duplicate and do not store)
-    const long long zx = P.qx->zero_point, zg = P.qg->zero_point;
+    // (signed low bytes: the limbs hold g16 - 128, against the zero-point zg - 128)
+    const long long zx = P.qx->zero_point, zg = P.qg->zero_point - (P.lo_signed ? 128 : 0);
     long long SX = 0, SG = 0, count = 0;
     int at, row, n;                                     // accumulator tile, row in it, output column of g
     if (!P.conv) {
@@ -778,6 +915,7 @@ __global__ void __launch_bounds__(256) wgrad_finalize_kernel(const WgradParams P
         if (P.tot_x) {
             // totals over all positions, less the border classes this tap does not see (the interior always counts)
             SX = P.tot_x[c]; SG = P.tot_g[n];
+            if (P.lo_signed && P.tot_g_plain) SG -= 128ll * P.Nimg * P.H * P.W;
             for (int cls = 1; cls < 16; ++cls) {
                 const bool top = cls & 1, bottom = cls & 2, left = cls & 4, right = cls & 8;
                 const bool g_ok = !((r < pad && top) || (r > pad && bottom) || (s < pad && left) || (s > pad && right));
@@ -871,7 +1009,7 @@ bool qbp::wgrad_self_totals(const qbp_conv_desc *d)
 
 namespace qbp {
 
-static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, WgradPlan &pl)
+static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, WgradPlan &pl, bool lo_signed = false)
 {
     WgradParams &P = pl.P;
     P = WgradParams{};
@@ -909,12 +1047,32 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
     P.b = layout_mnmajor(kr, rb_b, 1, 0);
     P.idesc_hi = make_idesc(true, true, 1, 1, 128, (uint32_t)P.bn);
     P.idesc_lo = make_idesc(true, false, 1, 1, 128, (uint32_t)P.bn);
+    P.lo_signed = lo_signed ? 1 : 0;
+    P.b2_desc_lo = layout_mnmajor(kr, rb_b, 2, P.b.tile_bytes).desc_lo;      // the low tile follows the high one in a stage
+    P.idesc_fused = make_idesc(true, true, 1, 1, 128, 2u * (uint32_t)P.bn);
     if (!d) {
         P.iters_total = (int)((M + kr - 1) / kr);
         pl.bw = pl.bh = pl.bn_img = 0;
     } else {
         int bwl = 0, bhl = 0;
         pick_pixel_box_w((int)kr, d->N, d->H, d->W, bwl, bhl);
+        if (lo_signed && d->R == 3 && P.tiles_c == 1 && P.a_chunks <= 2) {
+            // halo tiles: boxes 8 positions wide and 8 or 4 rows high, when that costs at most a fifth more steps
+            // than the free choice of box
+            const long long free_tiles = (long long)((d->W + (1 << bwl) - 1) >> bwl) * ((d->H + (1 << bhl) - 1) >> bhl) *
+                                         ((d->N + ((int)kr >> (bwl + bhl)) - 1) / ((int)kr >> (bwl + bhl)));
+            long long best = -1;
+            for (int bh = 8; bh >= 4; bh >>= 1) {
+                const long long t = (long long)((d->W + 7) / 8) * ((d->H + bh - 1) / bh) * ((d->N + 16 / bh - 1) / (16 / bh));
+                if (best < 0 || t < best) { best = t; P.halo_bh = bh; }
+            }
+            if (best * 5 > free_tiles * 6) P.halo_bh = 0;
+            if (P.halo_bh) {
+                bwl = 3; bhl = P.halo_bh == 8 ? 3 : 2;
+                P.halo_box_bytes = (uint32_t)(kWgHaloW * (P.halo_bh + 2) * (16 / P.halo_bh)) * rb_a;
+                P.halo_bytes = (uint32_t)align_up((size_t)P.halo_box_bytes, 1024);
+            }
+        }
         P.bw_log2 = bwl; P.bh_log2 = bhl;
         pl.bw = 1 << bwl; pl.bh = 1 << bhl; pl.bn_img = (int)kr >> (bwl + bhl);
         P.tiles_w = (d->W + pl.bw - 1) / pl.bw; P.tiles_h = (d->H + pl.bh - 1) / pl.bh;
@@ -925,11 +1083,13 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
     // three groups in the ring).  The CTAs of the last group (fewer A tiles) get a ring of their own shape.
     const int n_last = P.a_tiles - (P.a_groups - 1) * P.ma;                 // A tiles of the last group
     // (the border-class tables of the epilogue warps sit behind the ring)
-    const uint32_t cls_bytes = wgrad_inline_border(d) ? (uint32_t)align_up(sizeof(int) * 16 * (size_t)(K + 2 * N), 1024) : 0u;
+    // (... and behind those the region of ones of the halo variant)
+    const uint32_t cls_only = wgrad_inline_border(d) ? (uint32_t)align_up(sizeof(int) * 16 * (size_t)(K + 2 * N), 1024) : 0u;
+    const uint32_t cls_bytes = cls_only + (P.halo_bh ? P.halo_bytes : 0u);
     auto ring = [&](int tiles, int &stages, int &cg) {
-        const uint32_t stage_bytes = P.a_chunk_bytes * P.a_chunks * (uint32_t)tiles + 2 * P.b.tile_bytes;
+        const uint32_t stage_bytes = (P.halo_bh ? P.halo_bytes : P.a_chunk_bytes * P.a_chunks * (uint32_t)tiles) + 2 * P.b.tile_bytes;
         stages = std::max(2, std::min<int>(kWgMaxStages, (int)((kWgSmem - 1024 - cls_bytes) / stage_bytes)));
-        const int mmas = tiles * (int)(kr / 32) * 2;
+        const int mmas = tiles * (int)(kr / 32) * 2;       // (in MMAs of bn columns: a fused one counts twice)
         cg = 1;
         while (cg * mmas < 24 && stages / (cg + 1) >= 3) ++cg;
         stages -= stages % cg;
@@ -938,6 +1098,7 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
     const size_t smem_full = ring(P.ma, P.stages, P.cg);
     const size_t smem_last = ring(n_last, P.stages_last, P.cg_last);
     P.cls_off = (uint32_t)(std::max(smem_full, smem_last) - 1024);           // behind the longer of the two rings
+    P.ones_off = P.cls_off + cls_only;
     pl.smem = std::max(smem_full, smem_last) + cls_bytes;
     // split of the reductions: at most 65536 rows per CTA; with few items, enough slices to fill the machine
     // once, in proportion to an item's cost per reduction step: a fixed part (waits, the share of a commit)
@@ -964,12 +1125,16 @@ static void plan_wgrad(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, 
 
 static size_t wgrad_ws_bytes(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K)
 {
-    WgradPlan pl;
-    plan_wgrad(d, M, N, K, pl);
     const int64_t cx = d ? d->C : K, cg = d ? d->K : N;
     const size_t sums = align_up(sizeof(int64_t) * 16 * cx, 256) + 2 * align_up(sizeof(int64_t) * 16 * cg, 256);
     const size_t terms = align_up(sizeof(int64_t) * cx, 256) + align_up(sizeof(int64_t) * cg, 256);
-    const size_t part = pl.P.direct ? 0 : align_up(sizeof(int64_t) * (size_t)pl.grid * (size_t)pl.P.part_stride, 256);
+    // (the split, and with it the partials, may differ between the two forms of the low limb: room for either)
+    size_t part = 0;
+    for (int lo_signed = 0; lo_signed < 2; ++lo_signed) {
+        WgradPlan pl;
+        plan_wgrad(d, M, N, K, pl, lo_signed != 0);
+        part = std::max(part, pl.P.direct ? (size_t)0 : align_up(sizeof(int64_t) * (size_t)pl.grid * (size_t)pl.P.part_stride, 256));
+    }
     return 256 + sums + terms + part;
 }
 
@@ -1036,7 +1201,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_wgrad_s16(const qbp_co
 int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx,
                         const int8_t *g_hi, const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW,
                         int *ext_status, void *ws, size_t ws_bytes, cudaStream_t st, const int64_t *tot_x, const int64_t *tot_g16,
-                        bool tot_g_filled)
+                        bool tot_g_filled, bool lo_signed)
 {
     if (!x || !g_hi || !g_lo || !qx || !qg16) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: NULL operand");
     if (!acc_out && !dW) return fail(QBP_ERR_INVALID_ARG, "wgrad_s16: acc_out and dW are both NULL");
@@ -1057,7 +1222,7 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
         return fail(QBP_ERR_WORKSPACE, "wgrad_s16: workspace of %zu bytes needed, %zu given", wgrad_ws_bytes(d, M, N, K), ws_bytes);
 
     WgradPlan pl;
-    plan_wgrad(d, M, N, K, pl);
+    plan_wgrad(d, M, N, K, pl, lo_signed);
     WgradParams &P = pl.P;
     const int64_t outs = d ? (int64_t)d->K * d->R * d->S * d->C : K * N;
     WsCarver w(ws, ws_bytes);
@@ -1091,10 +1256,11 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
             QBP_TRACE_BEGIN(st);
             border_class_sums_kernel<<<dim3((unsigned)gx, 1, 3), 256, (size_t)std::max(K, N) * 16 * sizeof(int), st>>>(
                 (const uint8_t *)x, (const uint8_t *)g_hi, g_lo, d->N, d->H, d->W, (int)K, (int)N, (unsigned long long *)sx,
-                (unsigned long long *)shi, (unsigned long long *)slo);
+                (unsigned long long *)shi, (unsigned long long *)slo, lo_signed ? 1 : 0);
             QBP_LAUNCH_OK("border_class_sums_kernel");
         }
         P.tot_x = (const long long *)tot_x; P.tot_g = (const long long *)tot_g16;
+        P.tot_g_plain = tot_g_filled ? 1 : 0;
         if (!tot_g_filled) {
             // nobody left the gradient's totals: the product takes them itself (a row of ones in its spare chunk)
             QBP_CUDA_OK(cudaMemsetAsync(const_cast<int64_t *>(tot_g16), 0, sizeof(int64_t) * (size_t)N, st));
@@ -1113,29 +1279,30 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
         QBP_TRACE_BEGIN(st);
         row_class_sums3_kernel<<<dim3((unsigned)grid_x, (unsigned)slabs, 3), 256, (size_t)12 * gs * 16 * sizeof(int), st>>>(
             (const uint8_t *)x, (const uint8_t *)g_hi, (const uint8_t *)g_lo, (int)(rows / d->H), d->H, d->W, (int)K, gs,
-            (unsigned long long *)sx);
+            (unsigned long long *)sx, lo_signed ? 1 : 0);
         QBP_LAUNCH_OK("class_sums_kernel");
     } else if (d) {
         if ((rc = launch_class_sums<true>(x, M, d->H, d->W, (int)K, sx, st))) return rc;
         if ((rc = launch_class_sums<true>(g_hi, M, d->H, d->W, (int)N, shi, st))) return rc;
-        if ((rc = launch_class_sums<false>(g_lo, M, d->H, d->W, (int)N, slo, st))) return rc;
+        if ((rc = lo_signed ? launch_class_sums<true>(g_lo, M, d->H, d->W, (int)N, slo, st)
+                            : launch_class_sums<false>(g_lo, M, d->H, d->W, (int)N, slo, st))) return rc;
     } else {
         if ((rc = launch_colsum(x, true, M, K, sx, st))) return rc;
         if ((rc = launch_colsum(g_hi, true, M, N, shi, st))) return rc;
-        if ((rc = launch_colsum(g_lo, false, M, N, slo, st))) return rc;
+        if ((rc = launch_colsum(g_lo, lo_signed, M, N, slo, st))) return rc;
         if (P.direct || pair_kernel) {
             const int64_t mx = std::max(K, N);
             QBP_TRACE_BEGIN(st);
             wgrad_terms_kernel<<<(unsigned)((mx + 255) / 256), 256, 0, st>>>((const long long *)sx, (const long long *)shi,
                                                                             (const long long *)slo, M, N, K, qx, qg16,
-                                                                            (long long *)rowterm, (long long *)colterm);
+                                                                            (long long *)rowterm, (long long *)colterm, lo_signed ? 128 : 0);
             QBP_LAUNCH_OK("wgrad_terms_kernel");
         }
     }
     if (!ext_status) QBP_CUDA_OK(cudaMemsetAsync(status, 0, sizeof(int), st));
     if (pair_kernel)
         return launch_wgrad2(M, N, K, x, qx, g_hi, g_lo, qg16, acc_out, dW, (const long long *)rowterm,
-                             (const long long *)colterm, status, st);
+                             (const long long *)colterm, status, st, lo_signed);
 
     P.part = (long long *)part; P.status = status;
     P.rowterm = (const long long *)rowterm; P.colterm = (const long long *)colterm;
@@ -1146,7 +1313,8 @@ int qbp::wgrad_s16_impl(const qbp_conv_desc *d, int64_t M, int64_t N, int64_t K,
         if ((rc = make_map_2d(&P.mapHi, g_hi, M, N, kr, rb_b))) return rc;
         if ((rc = make_map_2d(&P.mapLo, g_lo, M, N, kr, rb_b))) return rc;
     } else {
-        if ((rc = make_map_nhwc(&P.mapX, x, d->N, d->H, d->W, d->C, pl.bn_img, pl.bh, pl.bw, rb_a))) return rc;
+        if ((rc = P.halo_bh ? make_map_nhwc(&P.mapX, x, d->N, d->H, d->W, d->C, pl.bn_img, pl.bh + 2, kWgHaloW, rb_a)
+                            : make_map_nhwc(&P.mapX, x, d->N, d->H, d->W, d->C, pl.bn_img, pl.bh, pl.bw, rb_a))) return rc;
         if ((rc = make_map_nhwc(&P.mapHi, g_hi, d->N, d->H, d->W, d->K, pl.bn_img, pl.bh, pl.bw, rb_b))) return rc;
         if ((rc = make_map_nhwc(&P.mapLo, g_lo, d->N, d->H, d->W, d->K, pl.bn_img, pl.bh, pl.bw, rb_b))) return rc;
     }

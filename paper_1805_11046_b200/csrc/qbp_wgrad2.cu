@@ -35,7 +35,8 @@ constexpr uint32_t kW2Smem = 1024u + kW2Stages * kW2StageBytes + kW2EpiWarps * k
 struct Wgrad2Params {
     CUtensorMap mapX, mapHi, mapLo, mapC;
     uint32_t desc_lo;                // descriptor bits 16..31 of the M/N-major 128 x 128 tiles
-    uint32_t idesc_hi;               // s8 x s8, M = 256, N = 256, both operands M/N-major; the low limb's flips the B sign bit
+    uint32_t idesc_hi;               // s8 x s8, M = 256, N = 256, both operands M/N-major
+    uint32_t lo_flip;                // the low limb's descriptor = idesc_hi ^ lo_flip: the B sign bit for unsigned low bytes, 0 for lo - 128
     int k_iters;                     // reduction steps of 128 rows
     int tiles_m, tiles_n, tiles_total, pairs;
     FastDiv d_group;
@@ -94,10 +95,10 @@ __device__ __forceinline__ void w2_commit(uint64_t *bar)
 // between the two instruction descriptors stalls the MMA pipe.  Offsets in 16-byte units: 256 per k step of an
 // M/N-major 128-byte-row tile, 1024 per 128 x 128 tile.
 template <bool FIRST>
-__device__ __forceinline__ void w2_issue_stage(uint32_t tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc_hi)
+__device__ __forceinline__ void w2_issue_stage(uint32_t tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc_hi, uint32_t lo_flip)
 {
     constexpr uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-    const uint32_t idesc_lo = idesc_hi ^ (1u << 10);
+    const uint32_t idesc_lo = idesc_hi ^ lo_flip;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int limb = i >> 2, kk = i & 3;
@@ -189,8 +190,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kW2Threads, 1) qbp_w
                     tc_fence_after();
                     const uint32_t a_lo = ((a_addr >> 4) & 0x3FFFu) | P.desc_lo;
                     const uint32_t b_lo = (((a_addr + 16384u) >> 4) & 0x3FFFu) | P.desc_lo;
-                    if (it == 0) w2_issue_stage<true>(tmem_base, a_lo, b_lo, P.idesc_hi);
-                    else         w2_issue_stage<false>(tmem_base, a_lo, b_lo, P.idesc_hi);
+                    if (it == 0) w2_issue_stage<true>(tmem_base, a_lo, b_lo, P.idesc_hi, P.lo_flip);
+                    else         w2_issue_stage<false>(tmem_base, a_lo, b_lo, P.idesc_hi, P.lo_flip);
                     if (++in_group == (uint32_t)kW2Cg) {
                         if (elect_one()) w2_commit(&empty_bar[group]);
                         in_group = 0; ++group;
@@ -309,7 +310,7 @@ bool wgrad2_eligible(int64_t M, int64_t N, int64_t K)
 
 int launch_wgrad2(int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qparams *qx, const int8_t *g_hi,
                   const uint8_t *g_lo, const qbp_qparams *qg16, int64_t *acc_out, float *dW, const long long *rowterm,
-                  const long long *colterm, int *status, cudaStream_t st)
+                  const long long *colterm, int *status, cudaStream_t st, bool lo_signed)
 {
     Wgrad2Params P{};
     int rc;
@@ -321,6 +322,7 @@ int launch_wgrad2(int64_t M, int64_t N, int64_t K, const int8_t *x, const qbp_qp
     if (dW && (rc = make_map_out_2d(&P.mapC, dW, K, N))) return rc;
     P.desc_lo = L.desc_lo;
     P.idesc_hi = make_idesc(true, true, 1, 1, 256, 256);
+    P.lo_flip = lo_signed ? 0u : (1u << 10);
     P.k_iters = (int)((M + 127) / 128);
     P.tiles_m = (int)((K + 255) / 256); P.tiles_n = (int)((N + 255) / 256);
     P.tiles_total = P.tiles_m * P.tiles_n;

@@ -69,7 +69,7 @@ def _check_layer(B, cfg, relu, conv_kw=None, sample=None, want_y=False):
     # stage 5: bifurcation of the GPU's fp32 gradient
     g8, g16 = O.bifurcate(g, cfg["seed"], cfg["id8"], cfg["id16"])
     ohi_, olo_ = O.limb_split(g16.q)
-    assert np.array_equal(to_host(L.g8), g8.q) and np.array_equal(to_host(L.ghi), ohi_) and np.array_equal(to_host(L.glo), olo_)
+    assert np.array_equal(to_host(L.g8), g8.q) and np.array_equal(to_host(L.ghi), ohi_) and np.array_equal(to_host(L.glo) ^ np.uint8(0x80), olo_)     # (the layer stores lo - 128)
     # stage 6: the two backward products from those codes
     if oconv is None:
         _, odx, bad = O.gemm_s8(g8.q, g8.zero_point[0], ow.q, ow.zero_point[0], g8.scale[0], ow.scale[0], transB=True)
