@@ -356,6 +356,20 @@ __device__ __forceinline__ void tc_fence_after()
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
+// Three-input minimum / maximum (one instruction on sm_100).
+__device__ __forceinline__ float fmin3(float a, float b, float c)
+{
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // True in exactly one lane of a converged warp.  The MMA warps run whole and put this around each tcgen05.mma and
 // commit, rather than branching on the lane index once around the loop: the instruction takes its operands from
 // warp-uniform registers, and only in code the compiler knows to be convergent are descriptors that change from

@@ -196,8 +196,6 @@ struct MmaParams {
     const float4 *ep_fold; int ep_relu;
     const qbp_qparams *ep_rq; int8_t *ep_q; int32_t *ep_rowsum;
     uint32_t stat_span;           // bytes of the statistics region in shared memory (the fold table follows it)
-    int direct;                   // the fp32 output goes straight from registers to global memory (32-byte stores: a lane's
-                                  // 32 outputs are 128 contiguous bytes) instead of through a staging slab and a TMA store
     int grid;                     // CTAs launched
     uint32_t cterm_span;          // bytes of the column-term region in shared memory (the statistics follow it)
     int iter_entries;             // entries of the k-iteration table in shared memory (conv), a multiple of 64
@@ -320,6 +318,35 @@ __device__ __forceinline__ void issue_halo_3x3_any(int rb, int bn, uint32_t d, u
     } else {
         issue_halo_3x3<MPI, 32, 32>(d, a_lo, b_lo, b_tile16, idesc, first_acc);
     }
+}
+
+// The MMA warp's whole loop for the common 3 x 3 case: one halo tile per CTA tile (one channel chunk), the filter resident,
+// the output columns one of the common counts.  The general loop below builds each stage's operands from launch
+// parameters inside a loop over the stage's halo tiles, which keeps them out of the warp's uniform registers: its
+// MMAs then issue every 70 cycles, against the 48 that a 128 x 64 x 32 product takes (measured); here everything but
+// the two ring addresses is a constant.  False when a wait ran out.
+struct HaloLoopArgs {
+    uint64_t *full_bar, *empty_bar, *acc_full, *acc_empty;
+    uint32_t tmem, ring, b_lo, a_desc_lo, stage_bytes;
+    int stages, nbuf, tiles_total;
+};
+template <int MPI, int RB, int BN>
+__device__ __forceinline__ bool mma_loop_halo1(const HaloLoopArgs &A)
+{
+    uint32_t s = 0, ph = 0, buf = 0, bph = 1;
+    uint32_t stage_addr = A.ring, d = A.tmem;
+    for (int tile = blockIdx.x; tile < A.tiles_total; tile += gridDim.x) {
+        if (!mbar_wait_uniform(&A.acc_empty[buf], bph)) return false;
+        if (!mbar_wait_uniform(&A.full_bar[s], ph)) return false;
+        tc_fence_after();
+        issue_halo_3x3<MPI, RB, BN>(d, ((stage_addr >> 4) & 0x3FFFu) | A.a_desc_lo, A.b_lo, 0u, 0u, 0u);
+        if (elect_one()) mma_commit(&A.empty_bar[s]);
+        if (elect_one()) mma_commit(&A.acc_full[buf]);
+        stage_addr += A.stage_bytes; d += (uint32_t)BN;
+        if (++s == (uint32_t)A.stages) { s = 0; ph ^= 1u; stage_addr = A.ring; }
+        if (++buf == (uint32_t)A.nbuf) { buf = 0; bph ^= 1u; d = A.tmem; }
+    }
+    return true;
 }
 
 __device__ __forceinline__ void issue_stage(const MmaParams &P, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
@@ -509,6 +536,21 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         const int groups = P.groups;
         uint32_t s = 0, ph = 0;                          // ring position and parity, across tiles
         uint32_t buf = 0, bph = 1;                       // accumulator buffer and the parity of its "empty" barrier
+        // the common 3 x 3 case has a loop of its own (one halo tile per CTA tile; see mma_loop_halo1)
+        const int fast = (P.halo && P.ips == 1 && groups == 1 && P.msub == 1 && P.b_resident && !timed_out)
+                             ? (P.halo_rb == 0 ? (P.mma_per_iter == 2 && P.bn == 64 ? 1 : P.mma_per_iter == 4 && P.bn == 128 ? 2 : 0)
+                                               : (P.mma_per_iter == 2 && P.halo_rb == 64 && P.bn == 64 ? 3
+                                                  : P.mma_per_iter == 4 && P.halo_rb == 128 && P.bn == 128 ? 4 : 0))
+                             : 0;
+        if (fast) {
+            HaloLoopArgs A;
+            A.full_bar = full_bar; A.empty_bar = empty_bar; A.acc_full = acc_full; A.acc_empty = acc_empty;
+            A.tmem = tmem_base; A.ring = ring_addr; A.b_lo = ((bres_addr >> 4) & 0x3FFFu) | P.b.desc_lo; A.a_desc_lo = P.a.desc_lo;
+            A.stage_bytes = stage_bytes; A.stages = P.stages; A.nbuf = P.nbuf; A.tiles_total = P.tiles_total;
+            const bool ok = fast == 1 ? mma_loop_halo1<2, 0, 64>(A) : fast == 2 ? mma_loop_halo1<4, 0, 128>(A)
+                          : fast == 3 ? mma_loop_halo1<2, 64, 64>(A) : mma_loop_halo1<4, 128, 128>(A);
+            if (!ok) timed_out = true;
+        } else
         for (int tile = blockIdx.x; tile < P.tiles_total && !timed_out; tile += gridDim.x) {
             if (!mbar_wait_uniform(&acc_empty[buf], bph)) { timed_out = true; break; }
             tc_fence_after();
@@ -688,20 +730,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                             }
                         }
                     }
-                    if (P.out && P.direct && ri.valid) {
-                        float *dst = P.out + ri.m * P.N + o.n0 + c0;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8)
-                            if (j < lim) {
-                                float f[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) f[e] = TAIL ? v[TAIL ? j + e : 0] : __fmul_rn((float)acc[j + e], scale);
-                                asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                                             ::"l"(dst + j), "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "f"(f[4]), "f"(f[5]), "f"(f[6]), "f"(f[7])
-                                             : "memory");
-                            }
-                    }
-                    if (P.st_sum || (P.out && !P.direct)) {
+                    if (P.st_sum || P.out) {
                         // the store that last used this slab must have read it before it is overwritten
                         uint8_t *slab = slab0 + slab_i * kStageSlab;
                         if (lane == 0) { if (P.nslab == 2) tma_store_wait_read_but_one(); else tma_store_wait_read(); }
@@ -717,7 +746,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                                                    __fmul_rn((float)acc[j + 2], scale), __fmul_rn((float)acc[j + 3], scale));
                         fence_proxy_async();
                         __syncwarp();
-                        if (lane == 0 && ri.slab_in && P.out && !P.direct) {
+                        if (lane == 0 && ri.slab_in && P.out) {
                             if (P.mode == MODE_GEMM) tma_store_2d(&P.mapC, slab, o.n0 + c0, o.m0 + sub * 128 + quad * 32);
                             else                     tma_store_4d(&P.mapC, slab, o.n0 + c0, ri.sx, ri.sy, ri.sz);
                             tma_store_commit();
@@ -733,9 +762,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                                 for (int k = 0; k < 8; ++k) {
                                     const uint8_t *colp = slab + k * 128 + ((((lane >> 2) ^ k) << 4) | ((lane & 3) << 2));
 #pragma unroll
-                                    for (int r8 = 0; r8 < 4; ++r8) {
-                                        const float v = *reinterpret_cast<const float *>(colp + r8 * 1024);
-                                        cs += v; clo = fminf(clo, v); chi = fmaxf(chi, v);
+                                    for (int r8 = 0; r8 < 4; r8 += 2) {
+                                        // (two rows per three-input min / max)
+                                        const float v0 = *reinterpret_cast<const float *>(colp + r8 * 1024);
+                                        const float v1 = *reinterpret_cast<const float *>(colp + (r8 + 1) * 1024);
+                                        cs += v0; cs += v1; clo = fmin3(clo, v0, v1); chi = fmax3(chi, v0, v1);
                                     }
                                 }
                             } else {
@@ -1155,9 +1186,6 @@ static int launch_mma(MmaParams &P, int tiles_m, bool clear_status, cudaStream_t
     P.d_tiles_h = make_fastdiv(P.mode == MODE_GEMM ? 1 : P.tiles_h);
     const size_t smem = (size_t)fixed + P.b_res_bytes + (size_t)stages * stage_bytes;
     const bool tail = P.ep_fold || P.ep_relu || P.ep_q;
-    // 32-byte stores need the rows of the output 32-byte aligned (N a multiple of 16 is given)
-    // (not with column statistics: those need the staging slab anyway, and both together were slower: 0.094 against 0.072 ms)
-    P.direct = (P.out && !P.st_sum && ((uintptr_t)P.out & 31) == 0 && P.N % 8 == 0) ? 1 : 0;
     static PerDeviceOnce configured[2];
     if (tail) QBP_SMEM_OPT_IN(configured[1], qbp_mma_kernel<true>, kSmemBudget);
     else      QBP_SMEM_OPT_IN(configured[0], qbp_mma_kernel<false>, kSmemBudget);
