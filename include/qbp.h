@@ -11,8 +11,11 @@
  *   - Every tensor pointer is a DEVICE pointer owned by the caller.  Scalars
  *     the GPU produces (scale, zero-point, range) stay on the device in a
  *     qbp_qparams.  The library allocates no device memory and keeps no
- *     state between calls; scratch comes from the caller's workspace `ws`
+ *     results between calls; scratch comes from the caller's workspace `ws`
  *     (device memory, 256-byte aligned) of at least qbp_*_workspace_bytes().
+ *     (Host-side objects it does keep: the per-device function attributes,
+ *     and, for the layer calls, one stream and two events per host thread
+ *     and device -- see qbp_layer_fwd.)
  *   - `stream` is a cudaStream_t passed as void*; work is enqueued on it and
  *     the call returns without synchronising the host.
  *   - Layouts: matrices row-major and dense; activations NHWC; filters KRSC.
@@ -458,6 +461,13 @@ typedef struct {
 
 size_t qbp_layer_workspace_bytes(const qbp_layer_desc *L);
 
+/* A convolution layer with a small filter runs the filter's one-block kernels
+ * on a stream of the library's own, forked from `stream` once the range of the
+ * activation (forward) or gradient (backward) is enqueued and joined again
+ * before the product, so that they overlap the pass that writes the codes.
+ * That stream and its two events are created at the first such call of a host
+ * thread on a device: make that call before any stream capture.  Under stream
+ * capture the fork and join become part of the captured graph. */
 int qbp_layer_fwd(const qbp_layer_desc *L, const float *x, const float *w,
                   const float *gamma, const float *beta, float *y, const qbp_layer_ctx *saved,
                   void *ws, size_t ws_bytes, void *stream);

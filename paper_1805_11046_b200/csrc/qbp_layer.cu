@@ -57,6 +57,37 @@ static int layer_shape(const qbp_layer_desc *L, LayerShape &s)
 // the steps share (they run one after another on the stream), then the buffers that live across steps.
 constexpr size_t kLayerHead = 256;
 
+// A small filter's kernels (one block each, some ten microseconds of latency) need the quantiser parameters of the
+// activation or gradient they are paired with, but not its codes: they run on a stream of the library's own beside
+// the pass that writes those codes, forked from the caller's stream after the parameters and joined before the
+// product.  One stream and two events per host thread and device, made at first use (a first call should therefore
+// come before any stream capture); when they cannot be made the kernels simply run in line.
+struct SideStream { cudaStream_t s; cudaEvent_t fork, join; bool ok; };
+static SideStream *side_stream()
+{
+    thread_local SideStream cache[kMaxDevices] = {};
+    thread_local bool tried[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    SideStream &c = cache[dev];
+    if (!tried[dev]) {
+        tried[dev] = true;
+        c.ok = cudaStreamCreateWithFlags(&c.s, cudaStreamNonBlocking) == cudaSuccess &&
+               cudaEventCreateWithFlags(&c.fork, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&c.join, cudaEventDisableTiming) == cudaSuccess;
+        if (!c.ok) (void)cudaGetLastError();
+    }
+    return c.ok ? &c : nullptr;
+}
+// Runs what the caller enqueues on `side` between the event `fork` (already recorded on st) and the rest of st.
+static int side_begin(SideStream *sd) { QBP_CUDA_OK(cudaStreamWaitEvent(sd->s, sd->fork, 0)); return QBP_OK; }
+static int side_end(SideStream *sd, cudaStream_t st)
+{
+    QBP_CUDA_OK(cudaEventRecord(sd->join, sd->s));
+    QBP_CUDA_OK(cudaStreamWaitEvent(st, sd->join, 0));
+    return QBP_OK;
+}
+
 static size_t step_scratch_bytes(const qbp_layer_desc *L, const LayerShape &s)
 {
     size_t b = qbp_quantize_workspace_bytes(s.rows, std::max(s.cin, s.cout), QBP_PER_TENSOR);
@@ -185,10 +216,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
     // (convolution: each pixel's code sum is needed for the zero-point correction of the product)
     int32_t *row_sums = reinterpret_cast<int32_t *>(static_cast<char *>(ws) + scratch);
     const int32_t *in_sums = s.conv ? row_sums : nullptr;
+    // (a small filter's launch runs beside the pass that writes the input codes)
+    const bool small_filter = s.conv && filter_prep_supported(&L->conv, w, saved->w_codes);
+    SideStream *sd = (x && small_filter) ? side_stream() : nullptr;
     if (x) {
         bool left = false;
         rc = quantize_s8_with_totals(x, s.rows, s.cin, saved->x_codes, saved->qx, s.conv ? row_sums : nullptr,
-                                     want_totals ? saved->x_chan_sums : nullptr, &left, ws, scratch, st);
+                                     want_totals ? saved->x_chan_sums : nullptr, &left, ws, scratch, st, sd ? sd->fork : nullptr);
         if (rc) return rc;
         // (a shape the quantiser cannot take the totals of: one pass over the codes)
         if (want_totals && !left && (rc = launch_colsum(saved->x_codes, true, s.rows, s.cin, saved->x_chan_sums, st))) return rc;
@@ -201,9 +235,11 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
     // product's column terms in one launch)
     const int64_t w_rows = s.conv ? (int64_t)L->conv.K * L->conv.R * L->conv.S : s.cin;
     const int32_t *colterm = nullptr;
-    if (s.conv && filter_prep_supported(&L->conv, w, saved->w_codes)) {
+    if (small_filter) {
         int32_t *ct = colterm_buffer(L, s, ws);
-        if ((rc = launch_filter_prep(&L->conv, w, saved->qx, saved->w_codes, saved->qw, ct, st))) return rc;
+        if (sd && (rc = side_begin(sd))) return rc;
+        if ((rc = launch_filter_prep(&L->conv, w, saved->qx, saved->w_codes, saved->qw, ct, sd ? sd->s : st))) return rc;
+        if (sd && (rc = side_end(sd, st))) return rc;
         colterm = ct;
     } else {
         rc = qbp_quantize_s8(w, w_rows, s.w_elems / w_rows, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr,
@@ -278,15 +314,21 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     const bool self_totals = s.conv && saved->x_chan_sums && wgrad_self_totals(&L->conv) && s.rows < (1ll << 22);
     const bool totals = s.conv && saved->x_chan_sums && (self_totals || quantizer_totals_supported(s.cout)) && s.rows < (1ll << 22);
     int64_t *tot_g = totals ? tot_g_buffer(L, s, ws) : nullptr;
+    // (a small filter: the layer gradient's column terms in one launch, beside the bifurcation -- they need the
+    // gradient's parameters only; else two kernels inside the product's call)
+    const bool small = s.conv && (int64_t)L->conv.R * L->conv.S * L->conv.C <= 12288 && s.w_elems <= 49152 && L->conv.C % 4 == 0;
+    SideStream *sd = small ? side_stream() : nullptr;
     rc = bifurcate_with_range_partials(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st,
-                                       self_totals ? nullptr : tot_g, true);
+                                       self_totals ? nullptr : tot_g, true, sd ? sd->fork : nullptr);
     if (rc) return rc;
     if (s.conv) {
-        // (a small filter: the layer gradient's column terms in one launch, else two kernels inside the product's call)
-        const bool small = (int64_t)L->conv.R * L->conv.S * L->conv.C <= 12288 && s.w_elems <= 49152 && L->conv.C % 4 == 0;
         int32_t *ct = small ? colterm_buffer(L, s, ws) : nullptr;
-        if (small && (rc = launch_filter_dgrad_colterm(&L->conv, saved->w_codes, qp8, ct, st))) return rc;
+        if (small) {
+            if (sd && (rc = side_begin(sd))) return rc;
+            if ((rc = launch_filter_dgrad_colterm(&L->conv, saved->w_codes, qp8, ct, sd ? sd->s : st))) return rc;
+            if (sd && (rc = side_end(sd, st))) return rc;
+        }
         const EpilogueTail with_colterm{nullptr, 0, nullptr, nullptr, nullptr, 0, ct};
         rc = conv_s8_impl(QBP_CONV_DGRAD, &L->conv, g8, qp8, saved->w_codes, saved->qw, nullptr, dx, row_sums, nullptr, status, ws, scratch, st,
                           small ? &with_colterm : nullptr);

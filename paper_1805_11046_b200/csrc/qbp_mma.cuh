@@ -24,11 +24,13 @@ size_t rangebn_range_parts_capacity(int64_t C);
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                                   uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
                                   uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st,
-                                  int64_t *tot16 = nullptr, bool lo_signed = false);
+                                  int64_t *tot16 = nullptr, bool lo_signed = false, cudaEvent_t after_range = nullptr);
+// after_range (here and in quantize_s8_with_totals; nullable): an event recorded on the stream as soon as the quantiser's
+// parameters are enqueued, before the pass that writes the codes.
 // Whether the quantising kernels can leave per-channel totals for a tensor of `cols` channels.
 bool quantizer_totals_supported(int64_t cols);
 int quantize_s8_with_totals(const float *x, int64_t rows, int64_t cols, int8_t *q, qbp_qparams *qp_out, int32_t *row_sums,
-                            int64_t *tot8, bool *left, void *ws, size_t ws_bytes, cudaStream_t st);
+                            int64_t *tot8, bool *left, void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range = nullptr);
 // The convolution products with the per-pixel channel sums of the input codes supplied by the caller
 // (nullable: computed here) (qbp_mma.cu).
 // Per-column (sum, min, max) of a product's fp32 output as partial rows [rows][N], one per CTA

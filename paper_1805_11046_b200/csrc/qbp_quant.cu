@@ -593,8 +593,10 @@ static int grid_for(int bps, int64_t n_groups)
     return (int)(g < 1 ? 1 : g);
 }
 
+// after_range (nullable): recorded on the stream once the parameters are enqueued -- a caller that has work for
+// another stream which needs only them (and not the codes) starts it from there.
 static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams *qp8, qbp_qparams *qp16,
-                        cudaStream_t st)
+                        cudaStream_t st, cudaEvent_t after_range = nullptr)
 {
     int nparts = 0;
     if (n > 0) {
@@ -611,6 +613,7 @@ static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams
     QBP_TRACE_BEGIN(st);
     range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
     QBP_LAUNCH_OK("range_finalize_kernel");
+    if (after_range) QBP_CUDA_OK(cudaEventRecord(after_range, st));
     return QBP_OK;
 }
 
@@ -748,7 +751,7 @@ static size_t quant_ws_bytes(int64_t cols, int granularity)
 // Shared body of the 8- and 16-bit entry points.
 static int quantize_any(int bits, const float *x, int64_t rows, int64_t cols, int granularity, int rounding,
                         uint64_t seed, uint32_t tensor_id, const qbp_qparams *range_in, const QuantOut &o,
-                        qbp_qparams *qp_out, void *ws, size_t ws_bytes, cudaStream_t st)
+                        qbp_qparams *qp_out, void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range = nullptr)
 {
     int rc = check_common(x, rows, cols, granularity, rounding, qp_out);
     if (rc) return rc;
@@ -769,7 +772,7 @@ static int quantize_any(int bits, const float *x, int64_t rows, int64_t cols, in
             rc = launch_chan_range(x, rows, cols, bits, plo, phi, qp_out, st);
         } else {
             float2 *parts = w.take<float2>(kMaxParts);
-            rc = launch_range(x, rows * cols, parts, bits == 8 ? qp_out : nullptr, bits == 16 ? qp_out : nullptr, st);
+            rc = launch_range(x, rows * cols, parts, bits == 8 ? qp_out : nullptr, bits == 16 ? qp_out : nullptr, st, after_range);
         }
         if (rc) return rc;
     }
@@ -827,11 +830,12 @@ static int bifurcate_tail(const float *g, int64_t rows, int64_t cols, uint64_t s
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                                   uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
                                   uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st,
-                                  int64_t *tot16, bool lo_signed)
+                                  int64_t *tot16, bool lo_signed, cudaEvent_t after_range)
 {
     QBP_TRACE_BEGIN(st);
     range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
     QBP_LAUNCH_OK("range_finalize_kernel");
+    if (after_range) QBP_CUDA_OK(cudaEventRecord(after_range, st));
     return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st, 0, tot16, lo_signed);
 }
 
@@ -843,7 +847,7 @@ bool quantizer_totals_supported(int64_t cols)
 // The layer's activation quantiser: qbp_quantize_s8 (per tensor, nearest) that also leaves the per-channel totals
 // of the codes (tot8 [cols], zeroed here) when the tensor's shape allows it; *left says whether it did.
 int quantize_s8_with_totals(const float *x, int64_t rows, int64_t cols, int8_t *q, qbp_qparams *qp_out, int32_t *row_sums,
-                            int64_t *tot8, bool *left, void *ws, size_t ws_bytes, cudaStream_t st)
+                            int64_t *tot8, bool *left, void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range)
 {
     *left = false;
     QuantOut o = {q, nullptr, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
@@ -854,7 +858,7 @@ int quantize_s8_with_totals(const float *x, int64_t rows, int64_t cols, int8_t *
         o.chansum8 = reinterpret_cast<unsigned long long *>(tot8);
         *left = true;
     }
-    int rc = quantize_any(8, x, rows, cols, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, o, qp_out, ws, ws_bytes, st);
+    int rc = quantize_any(8, x, rows, cols, QBP_PER_TENSOR, QBP_ROUND_NEAREST, 0, 0, nullptr, o, qp_out, ws, ws_bytes, st, after_range);
     if (rc) return rc;
     if (row_sums && !fused) return launch_rowsum(q, true, rows, cols, row_sums, st);
     return QBP_OK;
