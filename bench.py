@@ -113,6 +113,7 @@ KERNEL_WORK = {
     ("bn_stats_kernel", 0): (4, 0), ("bn_apply_kernel", 0): (8, 0),
     ("bn_bwd_stats_kernel", 0): (8, 0), ("bn_bwd_apply_kernel", 0): (12, 0),
     ("quantize_kernel", 1): (7, 0),                                                 # bifurcation: 4 B in, 1 + 2 B out
+    ("bn_bwd_apply_bifurcate_kernel", 0): (11, 0),                                  # dy and z in (8 B), the gradient's 8-bit copy and two limbs out (3 B)
     ("qbp_mma_kernel", 1): (5, OPS_PER_ELEMENT_CONV),                               # dgrad
     ("qbp_wgrad_kernel", 0): (3, 2 * OPS_PER_ELEMENT_CONV),                         # two int8 products per 16x8-bit product
 }
@@ -138,7 +139,8 @@ def run_ours(args):
     x, w, dy = (host[k].to(dev, non_blocking=True) for k in ("x", "w", "dy"))
     c = cfg["conv"]
     conv = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
-    L = layer.QuantizedLayer(conv=conv, relu=True, seed=cfg["seed"], tensor_id8=cfg["id8"], tensor_id16=cfg["id16"], device=dev)
+    L = layer.QuantizedLayer(conv=conv, relu=True, seed=cfg["seed"], tensor_id8=cfg["id8"], tensor_id16=cfg["id16"], device=dev,
+                             keep_g=False)      # (the fp32 gradient at the product is an intermediate: only its two copies are kept)
     E = x.numel()
 
     def step():

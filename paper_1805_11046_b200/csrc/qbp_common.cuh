@@ -189,6 +189,18 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys &k)
 // epilogue of a product) must produce the same bits, so that forward, backward and requantisation agree.
 __device__ __forceinline__ float bn_xhat(float x, float mu, float s) { return __fmul_rn(__fsub_rn(x, mu), s); }
 __device__ __forceinline__ float bn_y(float xh, float g, float b) { return __fadd_rn(__fmul_rn(g, xh), b); }
+// One element of the Range BN backward (the derivative stated with Eq. (rangebn) in Section 3, ties as in the forward):
+// dx = s * (gamma * dy - m1 - k2 * ind), ind = [x == max] - [x == min].  Every operation is rounded on its own and
+// none is contracted, so the value is a monotone function of dy for fixed (s >= 0, gamma, m1, k2, ind): the extremes of
+// dx over a set of positions are this function of the extremes of dy (which is how the gradient's range is known
+// before the gradient is written).
+__device__ __forceinline__ float bn_dx(float d, float ind, float s, float g, float m1, float k2)
+{
+    return __fmul_rn(s, __fsub_rn(__fsub_rn(__fmul_rn(g, d), m1), __fmul_rn(k2, ind)));
+}
+// Floats as integers that compare the same way (and back): for atomic minima and maxima of floats.
+__device__ __forceinline__ int float_order(float f) { const int b = __float_as_int(f); return b ^ ((b >> 31) & 0x7fffffff); }
+__device__ __forceinline__ float order_float(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 __device__ __forceinline__ float bn_scale(float lo, float hi, float Cn)
 {
     float r = __fsub_rn(hi, lo);

@@ -289,7 +289,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     if (!ws || ws_bytes < qbp_layer_workspace_bytes(L))
         return fail(QBP_ERR_WORKSPACE, "layer_bwd: workspace of %zu bytes needed, %zu given",
                     qbp_layer_workspace_bytes(L), ws_bytes);
-    if (!saved->g || !saved->g8 || !saved->qg8 || !saved->g_hi || !saved->g_lo || !saved->qg16 || !saved->z)
+    if (!saved->g8 || !saved->qg8 || !saved->g_hi || !saved->g_lo || !saved->qg16 || !saved->z)
         return fail(QBP_ERR_INVALID_ARG, "layer_bwd: the saved-state record has a NULL buffer (the backward pass needs z and the gradient buffers)");
     const size_t scratch = step_scratch_bytes(L, s);
     float *g = saved->g;
@@ -302,11 +302,6 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     ws = static_cast<char *>(ws) + kLayerHead;
     int32_t *row_sums = reinterpret_cast<int32_t *>(static_cast<char *>(ws) + scratch);
     float2 *range_parts = reinterpret_cast<float2 *>(static_cast<char *>(ws) + scratch + align_up(sizeof(int32_t) * (size_t)s.rows, 256));
-    // the pass that writes the gradient also leaves its range (Section 4: no extra scan for the quantiser)
-    int nparts = 0;
-    rc = rangebn_bwd_impl(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
-                          saved->save_max, g, dgamma, dbeta, ws, scratch, range_parts, &nparts, st);
-    if (rc) return rc;
     // two copies of the gradient: 8 bits for the layer gradient, 16 bits for the weight gradient
     // (convolution with the input's per-channel code totals at hand: the bifurcation leaves the gradient's, and the
     // weight gradient reads only the border positions again for its zero-point terms)
@@ -318,9 +313,26 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     // gradient's parameters only; else two kernels inside the product's call)
     const bool small = s.conv && (int64_t)L->conv.R * L->conv.S * L->conv.C <= 12288 && s.w_elems <= 49152 && L->conv.C % 4 == 0;
     SideStream *sd = small ? side_stream() : nullptr;
-    rc = bifurcate_with_range_partials(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
-                                       s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st,
-                                       self_totals ? nullptr : tot_g, true, sd ? sd->fork : nullptr);
+    // Range BN backward and the two copies of its result.  Where the shape allows, in two passes over (dy, z): the
+    // statistics pass also takes the extremes of dy, from which the exact range of the gradient follows (Section 4:
+    // the range without a scan), and the second pass quantises the gradient as it computes it -- the fp32 gradient is
+    // written only when the caller keeps saved->g.  Else: the pass that writes the gradient leaves its range, and the
+    // bifurcation reads the gradient back.
+    const bool two_pass = rangebn_bwd_bifurcate_supported(dy, saved->z, g, s.rows, s.cout, s.conv) && !(totals && !self_totals);
+    if (two_pass) {
+        rc = rangebn_bwd_bifurcate_impl(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
+                                        saved->save_max, g, dgamma, dbeta, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
+                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, true, ws, scratch, st, sd ? sd->fork : nullptr);
+    } else {
+        if (!g) return fail(QBP_ERR_INVALID_ARG, "layer_bwd: this shape needs saved->g (the fp32 gradient is written and read back)");
+        int nparts = 0;
+        rc = rangebn_bwd_impl(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
+                              saved->save_max, g, dgamma, dbeta, ws, scratch, range_parts, &nparts, st);
+        if (rc) return rc;
+        rc = bifurcate_with_range_partials(g, s.rows, s.cout, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
+                                           s.conv ? row_sums : nullptr, ghi, glo, qp16, range_parts, nparts, st,
+                                           self_totals ? nullptr : tot_g, true, sd ? sd->fork : nullptr);
+    }
     if (rc) return rc;
     if (s.conv) {
         int32_t *ct = small ? colterm_buffer(L, s, ws) : nullptr;

@@ -21,6 +21,15 @@ int rangebn_bwd_impl(const float *dy, const float *x, int64_t n, int64_t C, cons
                      float *dgamma, float *dbeta, void *ws, size_t ws_bytes, float2 *range_parts, int *nparts,
                      cudaStream_t st);
 size_t rangebn_range_parts_capacity(int64_t C);
+// Range BN backward and the bifurcation of the gradient in two passes, the fp32 gradient optional (qbp_rangebn.cu).
+bool rangebn_bwd_bifurcate_supported(const float *dy, const float *x, const float *g_out, int64_t n, int64_t C, bool row_sums);
+int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma, const float *beta,
+                               int relu, const float *save_mean, const float *save_min, const float *save_max, float *g_out,
+                               float *dgamma, float *dbeta, uint64_t seed, uint32_t id8, uint32_t id16, int8_t *q8,
+                               qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo, qbp_qparams *qp16, bool lo_signed,
+                               void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range = nullptr);
+int launch_range_finalize(const float2 *partials, int nparts, qbp_qparams *qp8, qbp_qparams *qp16, cudaStream_t st,
+                          cudaEvent_t after_range = nullptr);
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,
                                   uint32_t tensor_id16, int8_t *q8, qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi,
                                   uint8_t *lo, qbp_qparams *qp16, const float2 *partials, int nparts, cudaStream_t st,

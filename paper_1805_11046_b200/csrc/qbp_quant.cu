@@ -839,6 +839,17 @@ int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, ui
     return bifurcate_tail(g, rows, cols, seed, tensor_id8, tensor_id16, q8, qp8, row_sums8, hi, lo, qp16, st, 0, tot16, lo_signed);
 }
 
+// The parameters of both copies from per-block (or per-channel) (min, max) pairs.
+int launch_range_finalize(const float2 *partials, int nparts, qbp_qparams *qp8, qbp_qparams *qp16, cudaStream_t st,
+                          cudaEvent_t after_range)
+{
+    QBP_TRACE_BEGIN(st);
+    range_finalize_kernel<<<1, kThreads, 0, st>>>(partials, nparts, qp8, qp16);
+    QBP_LAUNCH_OK("range_finalize_kernel");
+    if (after_range) QBP_CUDA_OK(cudaEventRecord(after_range, st));
+    return QBP_OK;
+}
+
 bool quantizer_totals_supported(int64_t cols)
 {
     return cols % 4 == 0 && cols / 4 <= kThreads && ((cols / 4) & (cols / 4 - 1)) == 0;

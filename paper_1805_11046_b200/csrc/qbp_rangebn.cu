@@ -250,7 +250,11 @@ __global__ void __launch_bounds__(256) bn_out_range_kernel(const float *__restri
 }
 
 // --------------------------------------------------------------- backward
-template <int VEC, bool RELU>
+// EXT: also the extremes of the (rectifier-masked) dy of each channel over three sets of positions -- where x is the
+// channel's maximum, where it is its minimum, and everywhere else -- as ext [6][blocks][C] (min, max of the ordinary
+// positions, then of the maxima, then of the minima).  dx is a monotone function of dy on each set (bn_dx), so the
+// finalize kernel knows the exact range of dx from these, before dx is computed.
+template <int VEC, bool RELU, bool EXT>
 __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float *__restrict__ dy,
                                                                     const float *__restrict__ x, int64_t rows, int C,
                                                                     int tw, const float *__restrict__ mean,
@@ -259,19 +263,29 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
                                                                     const float *__restrict__ gamma,
                                                                     const float *__restrict__ beta, float Cn,
                                                                     double *__restrict__ part_dy,
-                                                                    double *__restrict__ part_dyx)
+                                                                    double *__restrict__ part_dyx,
+                                                                    float *__restrict__ ext)
 {
     const ScanPos p = scan_pos<VEC>(C, tw);
     const int rpb = kScanThreads / tw;
     double sdy[VEC], sdyx[VEC];
+    // (the extremes of the ordinary positions in registers; those of the few positions at a channel's maximum or
+    // minimum in shared memory, as integers that order like the floats)
+    float elo[VEC], ehi[VEC];
+    __shared__ int s_tie[EXT ? 4 * kScanThreads * VEC / 4 : 1];      // [min at max, max at max, min at min, max at min][tw * VEC]
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) { sdy[e] = 0.0; sdyx[e] = 0.0; }
+    for (int e = 0; e < VEC; ++e) { sdy[e] = 0.0; sdyx[e] = 0.0; elo[e] = INFINITY; ehi[e] = -INFINITY; }
+    if (EXT) {
+        for (int i = threadIdx.x; i < 4 * tw * VEC; i += kScanThreads) s_tie[i] = ((i / (tw * VEC)) & 1) ? float_order(-INFINITY) : float_order(INFINITY);
+        __syncthreads();
+    }
     if (p.active) {
-        float mu[VEC], s[VEC], g[VEC], b[VEC];
+        float mu[VEC], s[VEC], g[VEC], b[VEC], lo[VEC], hi[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) {
             mu[e] = mean[p.col + e];
-            s[e] = bn_scale(vmin[p.col + e], vmax[p.col + e], Cn);
+            lo[e] = vmin[p.col + e]; hi[e] = vmax[p.col + e];
+            s[e] = bn_scale(lo[e], hi[e], Cn);
             g[e] = gamma ? gamma[p.col + e] : 1.0f;
             b[e] = beta ? beta[p.col + e] : 0.0f;
         }
@@ -295,11 +309,20 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
                         if (RELU && !(bn_y(xh, g[e], b[e]) > 0.0f)) d = 0.0f;
                         sdy[e] += (double)d;
                         sdyx[e] += (double)d * (double)xh;
+                        if (EXT) {
+                            const bool ih = vx[u].v[e] == hi[e], il = vx[u].v[e] == lo[e];
+                            if (ih == il) { elo[e] = fminf(elo[e], d); ehi[e] = fmaxf(ehi[e], d); }
+                            else {
+                                int *t = s_tie + (ih ? 0 : 2) * tw * VEC + p.tx * VEC + e;
+                                atomicMin(t, float_order(d)); atomicMax(t + tw * VEC, float_order(d));
+                            }
+                        }
                     }
                 }
         }
     }
-    __shared__ double s_a[kScanThreads * VEC], s_b[kScanThreads * VEC];
+    __shared__ double s_ab[2 * kScanThreads * VEC];
+    double *s_a = s_ab, *s_b = s_ab + kScanThreads * VEC;
 #pragma unroll
     for (int e = 0; e < VEC; ++e) { s_a[threadIdx.x * VEC + e] = sdy[e]; s_b[threadIdx.x * VEC + e] = sdyx[e]; }
     __syncthreads();
@@ -316,6 +339,32 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
             part_dyx[(int64_t)blockIdx.x * C + p.col + e] = sdyx[e];
         }
     }
+    if (EXT) {
+        // the block's rows meet in shared memory (the arrays of the sums, read by now, hold two tables each)
+        float *s_f = reinterpret_cast<float *>(s_ab);          // room for four tables of kScanThreads * VEC floats
+        static_assert(sizeof(double) == 2 * sizeof(float), "two float tables per double table");
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            s_f[threadIdx.x * VEC + e] = elo[e];
+            s_f[(kScanThreads + threadIdx.x) * VEC + e] = ehi[e];
+        }
+        __syncthreads();
+        if (p.ty == 0 && p.active) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                float lo0 = elo[e], hi0 = ehi[e];
+                for (int y = 1; y < rpb; ++y) {
+                    lo0 = fminf(lo0, s_f[(y * tw + p.tx) * VEC + e]);
+                    hi0 = fmaxf(hi0, s_f[(kScanThreads + y * tw + p.tx) * VEC + e]);
+                }
+                const int64_t at = (int64_t)blockIdx.x * C + p.col + e, tbl = (int64_t)gridDim.x * C;
+                ext[at] = lo0; ext[tbl + at] = hi0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) ext[(2 + k) * tbl + at] = order_float(s_tie[k * tw * VEC + p.tx * VEC + e]);
+            }
+        }
+    }
 }
 
 // One block of 128 threads per channel: dbeta, dgamma, and the two per-channel
@@ -325,13 +374,37 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
                                                               int64_t n, const float *__restrict__ gamma, double Cn,
                                                               float *__restrict__ dgamma, float *__restrict__ dbeta,
                                                               float2 *__restrict__ coef, double *__restrict__ sum_dy,
-                                                              double *__restrict__ sum_dyx)
+                                                              double *__restrict__ sum_dyx,
+                                                              const float *__restrict__ ext = nullptr,
+                                                              const float *__restrict__ vmin = nullptr,
+                                                              const float *__restrict__ vmax = nullptr, float Cn_f = 0.0f,
+                                                              float2 *__restrict__ chan_range = nullptr)
 {
     const int c = blockIdx.x;
     double a = 0.0, b = 0.0;
     for (int i = threadIdx.x; i < nparts; i += 128) {
-        a += part_dy[(int64_t)i * C + c];
-        b += part_dyx[(int64_t)i * C + c];
+        const double pa_ = part_dy[(int64_t)i * C + c], pb_ = part_dyx[(int64_t)i * C + c];
+        a += pa_; b += pb_;
+    }
+    // ext (see bn_bwd_stats_kernel): the extremes of dy over the three sets of positions, then (below) the exact range
+    // of this channel's dx, left in chan_range[c] for the quantiser of the gradient
+    float ev[6];
+    __shared__ float s_e[6][4];
+    if (ext) {
+#pragma unroll
+        for (int k = 0; k < 6; ++k) ev[k] = (k & 1) ? -INFINITY : INFINITY;
+        for (int i = threadIdx.x; i < nparts; i += 128) {
+            float o[6];
+#pragma unroll
+            for (int k = 0; k < 6; ++k) o[k] = ext[((int64_t)k * nparts + i) * C + c];
+#pragma unroll
+            for (int k = 0; k < 6; ++k) ev[k] = (k & 1) ? fmaxf(ev[k], o[k]) : fminf(ev[k], o[k]);
+        }
+#pragma unroll
+        for (int k = 0; k < 6; ++k) {
+            ev[k] = (k & 1) ? warp_max(ev[k]) : warp_min(ev[k]);
+            if ((threadIdx.x & 31) == 0) s_e[k][threadIdx.x >> 5] = ev[k];
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -350,7 +423,111 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
         const double g = gamma ? (double)gamma[c] : 1.0;
         if (dbeta) dbeta[c] = (float)a;
         if (dgamma) dgamma[c] = (float)b;
-        coef[c] = make_float2((float)(g * a / (double)n), (float)(Cn * g * b));
+        const float m1 = (float)(g * a / (double)n), k2 = (float)(Cn * g * b);
+        coef[c] = make_float2(m1, k2);
+        if (ext) {
+            const float s = bn_scale(vmin[c], vmax[c], Cn_f), gf = gamma ? gamma[c] : 1.0f;
+            float rlo = INFINITY, rhi = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {
+                float lo = ev[2 * k], hi = ev[2 * k + 1];
+                for (int w = 1; w < 4; ++w) { lo = fminf(lo, s_e[2 * k][w]); hi = fmaxf(hi, s_e[2 * k + 1][w]); }
+                if (lo <= hi) {              // (a set with no position keeps +inf, -inf)
+                    const float ind = k == 0 ? 0.0f : k == 1 ? 1.0f : -1.0f;
+                    const float v0 = bn_dx(lo, ind, s, gf, m1, k2), v1 = bn_dx(hi, ind, s, gf, m1, k2);
+                    rlo = fminf(rlo, fminf(v0, v1)); rhi = fmaxf(rhi, fmaxf(v0, v1));
+                }
+            }
+            chan_range[c] = make_float2(rlo, rhi);
+        }
+    }
+}
+
+// The Range BN backward apply pass and the bifurcation of the gradient it computes (Sections 3 and 6) in one pass:
+// dx goes from registers into its 8-bit copy (stochastic rounding), the two limbs of its 16-bit copy and each row's
+// 8-bit code sum; the fp32 dx itself is written only when the caller keeps it (g_out).  The parameters of both copies
+// are known beforehand (bn_bwd_finalize_kernel + the range finalize).  Element i of the [rows x C] tensor draws from
+// Philox block i / 4 as in quantize_kernel: a thread's four channels are one block.  Whole rows lie inside a warp
+// (tw = C / 4 lanes, a power of two <= 32) when rowsum8 is given.
+constexpr int kBabUnroll = 2;     // rows in flight per thread (two loads each): the pass is bound by arithmetic, so more resident warps
+template <bool RELU, bool STORE_G>
+__global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel(
+    const float *__restrict__ dy, const float *__restrict__ x, int64_t rows, int C, int tw, const float *__restrict__ mean,
+    const float *__restrict__ vmin, const float *__restrict__ vmax, const float *__restrict__ gamma,
+    const float *__restrict__ beta, float Cn, const float2 *__restrict__ coef, float *__restrict__ g_out,
+    const qbp_qparams *__restrict__ qp8, const qbp_qparams *__restrict__ qp16, uint32_t id8, uint32_t id16,
+    const __grid_constant__ PhiloxKeys keys, uint32_t *__restrict__ q8, uint32_t *__restrict__ q_hi, uint32_t *__restrict__ q_lo,
+    uint32_t lo_flip, int32_t *__restrict__ rowsum8)
+{
+    const ScanPos p = scan_pos<4>(C, tw);
+    const int rpb = kScanThreads / tw;
+    float mu[4], s[4], g[4], b[4], lo[4], hi[4], m1[4], k2[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int c = p.active ? p.col + e : 0;
+        mu[e] = mean[c];
+        lo[e] = vmin[c]; hi[e] = vmax[c];
+        s[e] = bn_scale(lo[e], hi[e], Cn);
+        g[e] = gamma ? gamma[c] : 1.0f;
+        b[e] = beta ? beta[c] : 0.0f;
+        const float2 cf = coef[c];
+        m1[e] = cf.x; k2[e] = cf.y;
+    }
+    // both codes in fixed point with 16 fraction bits (quantize_sr8_byte2 / quantize_sr16_top_half)
+    const float inv8 = __fdiv_rn(1.0f, qp8->scale) * 65536.0f, zp8 = (float)(qp8->zero_point + 128) * 65536.0f;
+    const float inv16 = __fdiv_rn(1.0f, qp16->scale) * 65536.0f, zp16 = (float)(qp16->zero_point + 32768) * 65536.0f;
+    const bool one_block = id8 == id16;
+    const int64_t step = (int64_t)gridDim.x * rpb;
+    // (the loop bound is the block's: every lane takes part in the row-sum shuffles)
+    for (int64_t base = (int64_t)blockIdx.x * rpb; base < rows; base += step * kBabUnroll) {
+        const int64_t r0 = base + p.ty;
+        VecF<4> vx[kBabUnroll], vd[kBabUnroll];
+        bool ok[kBabUnroll];
+#pragma unroll
+        for (int u = 0; u < kBabUnroll; ++u) {
+            const int64_t r = r0 + u * step;
+            ok[u] = p.active && r < rows;
+            if (ok[u]) { vx[u].load_stream(x + r * C + p.col); vd[u].load_stream(dy + r * C + p.col); }
+        }
+#pragma unroll
+        for (int u = 0; u < kBabUnroll; ++u) {
+            const int64_t r = r0 + u * step;
+            int rs = 0;
+            if (ok[u]) {
+                float v[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float xv = vx[u].v[e];
+                    float d = vd[u].v[e];
+                    if (RELU && !(bn_y(bn_xhat(xv, mu[e], s[e]), g[e], b[e]) > 0.0f)) d = 0.0f;
+                    const float ind = (xv == hi[e] ? 1.0f : 0.0f) - (xv == lo[e] ? 1.0f : 0.0f);
+                    v[e] = bn_dx(d, ind, s[e], g[e], m1[e], k2[e]);
+                }
+                const int64_t j = (r * C + p.col) >> 2;                 // the thread's Philox block = its float4's index
+                if (STORE_G) __stcs(reinterpret_cast<float4 *>(g_out) + j, make_float4(v[0], v[1], v[2], v[3]));
+                const uint4 r8 = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id8, 0u), keys);
+                const uint4 r16 = one_block ? r8 : philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), id16, 0u), keys);
+                const uint32_t w8[4] = {r8.x, r8.y, r8.z, r8.w}, w16[4] = {r16.x, r16.y, r16.z, r16.w};
+                uint32_t c8[4], c16[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    c8[e] = quantize_sr8_byte2(v[e], inv8, zp8, w8[e]);
+                    c16[e] = quantize_sr16_top_half(v[e], inv16, zp16, w16[e]);
+                }
+                // the 8-bit codes are byte 2 of each word; the 16-bit codes bytes 3 (high) and 2 (low)
+                const uint32_t packed = __byte_perm(__byte_perm(c8[0], c8[1], 0x0062), __byte_perm(c8[2], c8[3], 0x0062), 0x5410) ^ 0x80808080u;
+                q8[j] = packed;
+                const uint32_t t01 = __byte_perm(c16[0], c16[1], 0x7362), t23 = __byte_perm(c16[2], c16[3], 0x7362);
+                q_hi[j] = __byte_perm(t01, t23, 0x7632) ^ 0x80808080u;
+                q_lo[j] = __byte_perm(t01, t23, 0x5410) ^ lo_flip;
+                rs = __dp4a((int)packed, 0x01010101, 0);
+            }
+            if (rowsum8) {
+                for (int off = 16; off > 0; off >>= 1)
+                    if (off < tw) rs += __shfl_xor_sync(0xffffffffu, rs, off);
+                if (ok[u] && p.tx == 0) rowsum8[r] = rs;
+            }
+        }
     }
 }
 
@@ -416,7 +593,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float 
                     float d = vd[u].v[e];
                     if (RELU && !(bn_y(bn_xhat(xv, mu[e], s[e]), g[e], b[e]) > 0.0f)) d = 0.0f;
                     const float ind = (xv == hi[e] ? 1.0f : 0.0f) - (xv == lo[e] ? 1.0f : 0.0f);
-                    vd[u].v[e] = s[e] * (g[e] * d - m1[e] - k2[e] * ind);
+                    vd[u].v[e] = bn_dx(d, ind, s[e], g[e], m1[e], k2[e]);
                     if (RANGE) { rlo = fminf(rlo, vd[u].v[e]); rhi = fmaxf(rhi, vd[u].v[e]); }
                 }
                 vd[u].store(dx + (r0 + u * step) * C + p.col);
@@ -438,9 +615,11 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_apply_kernel(const float 
 static size_t bn_ws_bytes(int64_t C)
 {
     // forward: lo, hi (float) + sum (double) partials; backward: two double partials + coefficients
+    // (... and, for the backward pass that also bifurcates, six float tables of dy extremes and the channels' ranges)
     size_t per = (size_t)kScanMaxStrips * (size_t)C;
     return 2 * align_up(per * sizeof(double), 256) + 2 * align_up(per * sizeof(float), 256) +
-           align_up((size_t)C * sizeof(float2), 256) + 256;
+           align_up((size_t)C * sizeof(float2), 256) + 256 + align_up(6 * per * sizeof(float), 256) +
+           align_up((size_t)C * sizeof(float2), 256);
 }
 
 static int check_bn(const char *who, const void *a, const void *b, int64_t n, int64_t C, const void *ws, size_t ws_bytes)
@@ -649,24 +828,30 @@ namespace qbp {
 static int bn_bwd_stats_launch(const float *dy, const float *x, int64_t n_rows, int64_t n_stat, int64_t C, const float *gamma,
                                const float *beta, int relu, const float *save_mean, const float *save_min,
                                const float *save_max, float *dgamma, float *dbeta, float2 *coef, double *sum_dy,
-                               double *sum_dyx, double *pa, double *pb, cudaStream_t st)
+                               double *sum_dyx, double *pa, double *pb, cudaStream_t st, float *ext = nullptr,
+                               float2 *chan_range = nullptr)
 {
     const bool al = aligned16(x) && aligned16(dy);
     const bool v4 = al && C % 4 == 0;
-    const ScanGeom g = scan_geom(n_rows, C, al, v4 ? (relu ? blocks_per_sm(bn_bwd_stats_kernel<4, true>, kScanThreads)
-                                                           : blocks_per_sm(bn_bwd_stats_kernel<4, false>, kScanThreads))
-                                                   : blocks_per_sm(bn_bwd_stats_kernel<1, true>, kScanThreads));
+    const ScanGeom g = scan_geom(n_rows, C, al, v4 ? (ext ? blocks_per_sm(bn_bwd_stats_kernel<4, true, true>, kScanThreads)
+                                                          : relu ? blocks_per_sm(bn_bwd_stats_kernel<4, true, false>, kScanThreads)
+                                                                 : blocks_per_sm(bn_bwd_stats_kernel<4, false, false>, kScanThreads))
+                                                   : blocks_per_sm(bn_bwd_stats_kernel<1, true, false>, kScanThreads));
     const dim3 grid(g.nbx, g.slabs);
     const double Cnd = 1.0 / std::sqrt(2.0 * std::log((double)n_stat));
     const float Cn = (float)Cnd;
     QBP_TRACE_BEGIN(st);
-#define QBP_BN_BSTATS(V, R) bn_bwd_stats_kernel<V, R><<<grid, kScanThreads, 0, st>>>(dy, x, n_rows, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, pa, pb)
-    if (g.vec == 4) { if (relu) QBP_BN_BSTATS(4, true); else QBP_BN_BSTATS(4, false); }
-    else            { if (relu) QBP_BN_BSTATS(1, true); else QBP_BN_BSTATS(1, false); }
+#define QBP_BN_BSTATS(V, R, E) bn_bwd_stats_kernel<V, R, E><<<grid, kScanThreads, 0, st>>>(dy, x, n_rows, (int)C, g.tw, save_mean, save_min, save_max, gamma, beta, Cn, pa, pb, ext)
+    if (ext) {
+        if (g.vec != 4) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "rangebn_bwd: the pass with dy extremes needs aligned tensors and C a multiple of 4");
+        if (relu) QBP_BN_BSTATS(4, true, true); else QBP_BN_BSTATS(4, false, true);
+    } else if (g.vec == 4) { if (relu) QBP_BN_BSTATS(4, true, false); else QBP_BN_BSTATS(4, false, false); }
+    else                   { if (relu) QBP_BN_BSTATS(1, true, false); else QBP_BN_BSTATS(1, false, false); }
 #undef QBP_BN_BSTATS
     QBP_LAUNCH_OK("bn_bwd_stats_kernel");
     QBP_TRACE_BEGIN(st);
-    bn_bwd_finalize_kernel<<<(int)C, 128, 0, st>>>(pa, pb, g.nbx, (int)C, n_stat, gamma, Cnd, dgamma, dbeta, coef, sum_dy, sum_dyx);
+    bn_bwd_finalize_kernel<<<(int)C, 128, 0, st>>>(pa, pb, g.nbx, (int)C, n_stat, gamma, Cnd, dgamma, dbeta, coef, sum_dy, sum_dyx,
+                                                   ext, save_min, save_max, Cn, chan_range);
     QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
     return QBP_OK;
 }
@@ -695,6 +880,62 @@ static int bn_bwd_apply_launch(const float *dy, const float *x, int64_t n_rows, 
     }
 #undef QBP_BN_BAPPLY
     QBP_LAUNCH_OK("bn_bwd_apply_kernel");
+    return QBP_OK;
+}
+
+// Whether rangebn_bwd_bifurcate_impl takes a tensor of C channels (row_sums: each row's 8-bit code sum is wanted).
+bool rangebn_bwd_bifurcate_supported(const float *dy, const float *x, const float *g_out, int64_t n, int64_t C, bool row_sums)
+{
+    if (!aligned16(x) || !aligned16(dy) || (g_out && !aligned16(g_out)) || C % 4 || n < 2 || n * C >= (1ll << 40)) return false;
+    (void)row_sums;      // (rows wider than a warp's lanes: the sums are taken from the codes afterwards)
+    return true;
+}
+
+// Range BN backward and the bifurcation of its result in two passes over (dy, x): statistics with the extremes of dy
+// (from which the exact range of the gradient follows), then the pass that computes the gradient and writes its 8-bit
+// copy, the limbs of its 16-bit copy and the rows' code sums -- and the fp32 gradient only when g_out is given.
+int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma, const float *beta,
+                               int relu, const float *save_mean, const float *save_min, const float *save_max, float *g_out,
+                               float *dgamma, float *dbeta, uint64_t seed, uint32_t id8, uint32_t id16, int8_t *q8,
+                               qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo, qbp_qparams *qp16, bool lo_signed,
+                               void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range)
+{
+    int rc = check_bn("rangebn_bwd", dy, x, n, C, ws, ws_bytes);
+    if (rc) return rc;
+    if (!rangebn_bwd_bifurcate_supported(dy, x, g_out, n, C, row_sums8 != nullptr) || ((uintptr_t)q8 & 3) || ((uintptr_t)hi & 3) || ((uintptr_t)lo & 3))
+        return fail(QBP_ERR_UNSUPPORTED_SHAPE, "rangebn_bwd (bifurcating): shape or alignment not taken");
+    WsCarver w(ws, ws_bytes);
+    double *pa = w.take<double>((size_t)kScanMaxStrips * C);
+    double *pb = w.take<double>((size_t)kScanMaxStrips * C);
+    w.take<float>((size_t)kScanMaxStrips * C);
+    w.take<float>((size_t)kScanMaxStrips * C);
+    float2 *coef = w.take<float2>((size_t)C);
+    w.take<char>(256);
+    float *ext = w.take<float>(6 * (size_t)kScanMaxStrips * C);
+    float2 *chan_range = w.take<float2>((size_t)C);
+    if ((rc = bn_bwd_stats_launch(dy, x, n, n, C, gamma, beta, relu, save_mean, save_min, save_max, dgamma, dbeta, coef, nullptr,
+                                  nullptr, pa, pb, st, ext, chan_range)))
+        return rc;
+    if ((rc = launch_range_finalize(chan_range, (int)C, qp8, qp16, st, after_range))) return rc;
+    const ScanGeom ga = scan_geom(n, C, true, g_out ? (relu ? blocks_per_sm(bn_bwd_apply_bifurcate_kernel<true, true>, kScanThreads)
+                                                            : blocks_per_sm(bn_bwd_apply_bifurcate_kernel<false, true>, kScanThreads))
+                                                    : (relu ? blocks_per_sm(bn_bwd_apply_bifurcate_kernel<true, false>, kScanThreads)
+                                                            : blocks_per_sm(bn_bwd_apply_bifurcate_kernel<false, false>, kScanThreads)));
+    const dim3 grid(ga.nbx, ga.slabs);
+    const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
+    const PhiloxKeys keys = philox_keys_host(seed);
+    const uint32_t flip = lo_signed ? 0x80808080u : 0u;
+    // each row's code sum by shuffles when a row's lanes lie inside one warp, else from the codes afterwards
+    const int64_t cv = C / 4;
+    const bool rows_in_warp = cv <= 32 && (cv & (cv - 1)) == 0;
+    int32_t *row_sums_arg = (row_sums8 && rows_in_warp) ? row_sums8 : nullptr;
+    QBP_TRACE_BEGIN(st);
+#define QBP_BN_BAB(R, G) bn_bwd_apply_bifurcate_kernel<R, G><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg)
+    if (g_out) { if (relu) QBP_BN_BAB(true, true); else QBP_BN_BAB(false, true); }
+    else       { if (relu) QBP_BN_BAB(true, false); else QBP_BN_BAB(false, false); }
+#undef QBP_BN_BAB
+    QBP_LAUNCH_OK("bn_bwd_apply_bifurcate_kernel");
+    if (row_sums8 && !rows_in_warp) return launch_rowsum(q8, true, n, C, row_sums8, st);
     return QBP_OK;
 }
 

@@ -15,12 +15,14 @@ class QuantizedLayer:
 
     def __init__(self, conv=None, batch=0, in_features=0, out_features=0, relu=False, seed=0,
                  tensor_id8=1, tensor_id16=2, device="cuda", input_from: "QuantizedLayer | None" = None,
-                 emit_codes=False, keep_y=True, keep_z=True):
+                 emit_codes=False, keep_y=True, keep_z=True, keep_g=True):
         """input_from: the layer whose output feeds this one already quantised (it must have been built with
         emit_codes=True): this layer then owns no input codes of its own and its forward takes no fp32 input.
         emit_codes: the forward also writes the 8-bit codes of the output (and each row's code sum) for the next
         layer; keep_y=False then leaves the fp32 output unwritten.  keep_z=False (forward only, with emit_codes and
-        keep_y=False): the fp32 output of the product is not kept either -- the convolution is run twice instead."""
+        keep_y=False): the fp32 output of the product is not kept either -- the convolution is run twice instead.
+        keep_g=False: the backward pass does not write the fp32 gradient arriving at the product (only its 8-bit and
+        16-bit copies); for shapes the library quantises as it computes the gradient (it says so otherwise)."""
         self.device = torch.device(device)
         d = B.LayerDesc()
         if conv is not None:
@@ -56,7 +58,7 @@ class QuantizedLayer:
             self.rq_out = B.requant(self.out_codes, self.q_out, self.out_row_sums, self.out_chan_sums)
         assert keep_z or (emit_codes and not keep_y)
         self.z = e(self.z_shape, torch.float32) if keep_z else None
-        self.g = e(self.z_shape, torch.float32) if keep_z else None
+        self.g = e(self.z_shape, torch.float32) if (keep_z and keep_g) else None
         self.save_mean, self.save_min, self.save_max = (e((self.cout,), torch.float32) for _ in range(3))
         bshape = self.z_shape if keep_z else (0,)          # (no backward pass without z)
         self.g8, self.ghi, self.glo = e(bshape, torch.int8), e(bshape, torch.int8), e(bshape, torch.uint8)

@@ -113,6 +113,37 @@ def test_conv2_x_layer_full_size(B):
     _check_layer(B, cfg, True, cfg["conv"], _sampler(2))
 
 
+@pytest.mark.parametrize("kind", ["linear", "conv_small", "conv_wide", "conv2_x"])
+def test_backward_without_the_fp32_gradient_buffer(B, kind):
+    """keep_g=False: the gradient arriving at the product is quantised as the Range BN backward computes it and never
+    written as fp32.  Everything the backward leaves must equal, bit for bit, what the layer that keeps the buffer
+    leaves (that layer is the one the stage-wise tests check against the oracle)."""
+    import torch
+    from paper_1805_11046_b200 import layer
+    if kind == "linear":
+        cfg, conv = synth.linear_layer(), None
+    else:
+        cfg = {"conv_small": lambda: synth.conv3x3_layer(batch=4, hw=14), "conv_wide": lambda: synth.conv3x3_layer(batch=2, hw=9, c_in=32, k_out=160),
+               "conv2_x": lambda: synth.conv3x3_layer()}[kind]()
+        c = cfg["conv"]
+        conv = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    x, w, dy = to_dev(cfg["x"]), to_dev(cfg["w"]), to_dev(cfg["dy"])
+    outs = []
+    for keep_g in (True, False):
+        L = layer.QuantizedLayer(conv=conv, batch=cfg["x"].shape[0], in_features=cfg["x"].shape[-1],
+                                 out_features=cfg["w"].shape[-1] if conv is None else None, relu=True, seed=cfg["seed"],
+                                 tensor_id8=cfg["id8"], tensor_id16=cfg["id16"], keep_g=keep_g)
+        L.forward(x, w)
+        dx, dw, dgamma, dbeta = L.backward(dy)
+        torch.cuda.synchronize()
+        assert L.status() == 0 and (L.g is None) == (not keep_g)
+        outs.append([to_host(t) for t in (L.g8, L.ghi, L.glo, dx, dw, dgamma, dbeta)] + [B.read_qparams(L.qg8), B.read_qparams(L.qg16)])
+    for a_, b_ in zip(outs[0][:7], outs[1][:7]):
+        assert np.array_equal(a_, b_)
+    for qa, qb in zip(outs[0][7:], outs[1][7:]):
+        assert all(np.array_equal(u, v) for u, v in zip(qa, qb))
+
+
 def test_bottleneck_stack_stagewise(B):
     """conv3_x bottleneck (1x1, 3x3, 1x1, each + Range BN + ReLU) at a reduced batch; every layer checked
     stage-wise on the activations the GPU handed to it."""
