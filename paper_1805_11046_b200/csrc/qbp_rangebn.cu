@@ -299,6 +299,11 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
                 ok[u] = r < rows;
                 if (ok[u]) { vx[u].load_stream(x + r * C + p.col); vd[u].load_stream(dy + r * C + p.col); }
             }
+            // (the few rows of one step are added in fp32, the steps in fp64: a quarter of the conversions and fp64
+            // additions, and an error of a few ulp of four terms)
+            float fs[VEC], fp[VEC];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) { fs[e] = 0.0f; fp[e] = 0.0f; }
 #pragma unroll
             for (int u = 0; u < kScanUnroll; ++u)
                 if (ok[u]) {
@@ -307,8 +312,8 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
                         float xh = bn_xhat(vx[u].v[e], mu[e], s[e]);
                         float d = vd[u].v[e];
                         if (RELU && !(bn_y(xh, g[e], b[e]) > 0.0f)) d = 0.0f;
-                        sdy[e] += (double)d;
-                        sdyx[e] += (double)d * (double)xh;
+                        fs[e] += d;
+                        fp[e] = fmaf(d, xh, fp[e]);
                         if (EXT) {
                             const bool ih = vx[u].v[e] == hi[e], il = vx[u].v[e] == lo[e];
                             if (ih == il) { elo[e] = fminf(elo[e], d); ehi[e] = fmaxf(ehi[e], d); }
@@ -319,6 +324,8 @@ __global__ void __launch_bounds__(kScanThreads) bn_bwd_stats_kernel(const float 
                         }
                     }
                 }
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) { sdy[e] += (double)fs[e]; sdyx[e] += (double)fp[e]; }
         }
     }
     __shared__ double s_ab[2 * kScanThreads * VEC];
