@@ -440,6 +440,12 @@ typedef struct {
  * g8, g_hi, g_lo = rows*channels of the product's output (rows = batch or
  * N*P*Q); z is the fp32 output of the product (the input of Range BN), g the
  * fp32 gradient arriving at it.  The g* members are used by the backward only.
+ * g may be NULL: the backward pass then quantises the gradient as it computes
+ * it and never writes it as fp32 (the exact range of the gradient follows from
+ * per-channel extremes of dy that the statistics pass of the Range BN backward
+ * takes: Section 4 takes a tensor's range from the operator that makes it).
+ * That needs dy and z 16-byte aligned and the channel count a multiple of 4;
+ * qbp_layer_bwd says so otherwise.
  * g_lo holds the low bytes of the 16-bit codes with their top bit flipped, i.e.
  * the signed bytes lo - 128 (g16 = 256*g_hi + (lo - 128) + 128): both limbs
  * then have one operand type and the layer's weight gradient runs them as one
