@@ -318,11 +318,12 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_bwd(const qbp_la
     // the range without a scan), and the second pass quantises the gradient as it computes it -- the fp32 gradient is
     // written only when the caller keeps saved->g.  Else: the pass that writes the gradient leaves its range, and the
     // bifurcation reads the gradient back.
-    const bool two_pass = rangebn_bwd_bifurcate_supported(dy, saved->z, g, s.rows, s.cout, s.conv) && !(totals && !self_totals);
+    const bool two_pass = rangebn_bwd_bifurcate_supported(dy, saved->z, g, s.rows, s.cout, s.conv);
     if (two_pass) {
         rc = rangebn_bwd_bifurcate_impl(dy, saved->z, s.rows, s.cout, gamma, beta, L->relu, saved->save_mean, saved->save_min,
                                         saved->save_max, g, dgamma, dbeta, L->seed, L->tensor_id8, L->tensor_id16, g8, qp8,
-                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, true, ws, scratch, st, sd ? sd->fork : nullptr);
+                                        s.conv ? row_sums : nullptr, ghi, glo, qp16, true, ws, scratch, st, sd ? sd->fork : nullptr,
+                                        self_totals ? nullptr : tot_g);
     } else {
         if (!g) return fail(QBP_ERR_INVALID_ARG, "layer_bwd: this shape needs saved->g (the fp32 gradient is written and read back)");
         int nparts = 0;

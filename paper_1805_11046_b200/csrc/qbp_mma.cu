@@ -746,9 +746,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                                                    __fmul_rn((float)acc[j + 2], scale), __fmul_rn((float)acc[j + 3], scale));
                         fence_proxy_async();
                         __syncwarp();
-                        if (lane == 0 && ri.slab_in && P.out) {
-                            if (P.mode == MODE_GEMM) tma_store_2d(&P.mapC, slab, o.n0 + c0, o.m0 + sub * 128 + quad * 32);
-                            else                     tma_store_4d(&P.mapC, slab, o.n0 + c0, ri.sx, ri.sy, ri.sz);
+                        if (lane == 0 && P.out) {
+                            if (ri.slab_in) {
+                                if (P.mode == MODE_GEMM) tma_store_2d(&P.mapC, slab, o.n0 + c0, o.m0 + sub * 128 + quad * 32);
+                                else                     tma_store_4d(&P.mapC, slab, o.n0 + c0, ri.sx, ri.sy, ri.sz);
+                            }
+                            // a group per chunk, stored or not (a slab outside the matrix): "all but the latest group
+                            // have been read" must mean "the other slab's store", or the wait before the next fill lets a
+                            // store that is still reading this slab pass
                             tma_store_commit();
                         }
                         if (P.st_sum) {

@@ -27,7 +27,8 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
                                int relu, const float *save_mean, const float *save_min, const float *save_max, float *g_out,
                                float *dgamma, float *dbeta, uint64_t seed, uint32_t id8, uint32_t id16, int8_t *q8,
                                qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo, qbp_qparams *qp16, bool lo_signed,
-                               void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range = nullptr);
+                               void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range = nullptr,
+                               int64_t *tot16 = nullptr);      // tot16 (nullable) [C]: per-channel totals of the stored 16-bit codes
 int launch_range_finalize(const float2 *partials, int nparts, qbp_qparams *qp8, qbp_qparams *qp16, cudaStream_t st,
                           cudaEvent_t after_range = nullptr);
 int bifurcate_with_range_partials(const float *g, int64_t rows, int64_t cols, uint64_t seed, uint32_t tensor_id8,

@@ -456,17 +456,22 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
 // are known beforehand (bn_bwd_finalize_kernel + the range finalize).  Element i of the [rows x C] tensor draws from
 // Philox block i / 4 as in quantize_kernel: a thread's four channels are one block.  Whole rows lie inside a warp
 // (tw = C / 4 lanes, a power of two <= 32) when rowsum8 is given.
+// TOTALS: also each channel's total of the stored 16-bit codes (256 * hi + lo with lo unsigned, whatever lo_flip) over
+// all rows, added to chansum16 [C] (zeroed beforehand): a thread keeps its four channels for its whole life, a block
+// adds its threads' totals in shared memory and ends with one 64-bit atomic per channel.
 constexpr int kBabUnroll = 2;     // rows in flight per thread (two loads each): the pass is bound by arithmetic, so more resident warps
-template <bool RELU, bool STORE_G>
+template <bool RELU, bool STORE_G, bool TOTALS>
 __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel(
     const float *__restrict__ dy, const float *__restrict__ x, int64_t rows, int C, int tw, const float *__restrict__ mean,
     const float *__restrict__ vmin, const float *__restrict__ vmax, const float *__restrict__ gamma,
     const float *__restrict__ beta, float Cn, const float2 *__restrict__ coef, float *__restrict__ g_out,
     const qbp_qparams *__restrict__ qp8, const qbp_qparams *__restrict__ qp16, uint32_t id8, uint32_t id16,
     const __grid_constant__ PhiloxKeys keys, uint32_t *__restrict__ q8, uint32_t *__restrict__ q_hi, uint32_t *__restrict__ q_lo,
-    uint32_t lo_flip, int32_t *__restrict__ rowsum8)
+    uint32_t lo_flip, int32_t *__restrict__ rowsum8, unsigned long long *__restrict__ chansum16)
 {
     const ScanPos p = scan_pos<4>(C, tw);
+    uint32_t cs16[4] = {0u, 0u, 0u, 0u};          // unsigned codes of this thread's rows (fewer than 65536 rows)
+    int mine = 0;
     const int rpb = kScanThreads / tw;
     float mu[4], s[4], g[4], b[4], lo[4], hi[4], m1[4], k2[4];
 #pragma unroll
@@ -528,12 +533,31 @@ __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel
                 q_hi[j] = __byte_perm(t01, t23, 0x7632) ^ 0x80808080u;
                 q_lo[j] = __byte_perm(t01, t23, 0x5410) ^ lo_flip;
                 rs = __dp4a((int)packed, 0x01010101, 0);
+                if (TOTALS) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) cs16[e] += c16[e] >> 16;
+                    ++mine;
+                }
             }
             if (rowsum8) {
                 for (int off = 16; off > 0; off >>= 1)
                     if (off < tw) rs += __shfl_xor_sync(0xffffffffu, rs, off);
                 if (ok[u] && p.tx == 0) rowsum8[r] = rs;
             }
+        }
+    }
+    if (TOTALS) {
+        __shared__ int s_tot[kScanMaxTw * 4];
+        for (int i = threadIdx.x; i < tw * 4; i += kScanThreads) s_tot[i] = 0;
+        __syncthreads();
+        if (p.active && mine) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) atomicAdd(&s_tot[p.tx * 4 + e], (int)((long long)cs16[e] - (long long)mine * 32768));
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < tw * 4; i += kScanThreads) {
+            const int c = blockIdx.y * tw * 4 + i;
+            if (c < C && s_tot[i]) atomicAdd(chansum16 + c, (unsigned long long)(long long)s_tot[i]);
         }
     }
 }
@@ -905,7 +929,7 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
                                int relu, const float *save_mean, const float *save_min, const float *save_max, float *g_out,
                                float *dgamma, float *dbeta, uint64_t seed, uint32_t id8, uint32_t id16, int8_t *q8,
                                qbp_qparams *qp8, int32_t *row_sums8, int8_t *hi, uint8_t *lo, qbp_qparams *qp16, bool lo_signed,
-                               void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range)
+                               void *ws, size_t ws_bytes, cudaStream_t st, cudaEvent_t after_range, int64_t *tot16)
 {
     int rc = check_bn("rangebn_bwd", dy, x, n, C, ws, ws_bytes);
     if (rc) return rc;
@@ -924,10 +948,9 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
                                   nullptr, pa, pb, st, ext, chan_range)))
         return rc;
     if ((rc = launch_range_finalize(chan_range, (int)C, qp8, qp16, st, after_range))) return rc;
-    const ScanGeom ga = scan_geom(n, C, true, g_out ? (relu ? blocks_per_sm(bn_bwd_apply_bifurcate_kernel<true, true>, kScanThreads)
-                                                            : blocks_per_sm(bn_bwd_apply_bifurcate_kernel<false, true>, kScanThreads))
-                                                    : (relu ? blocks_per_sm(bn_bwd_apply_bifurcate_kernel<true, false>, kScanThreads)
-                                                            : blocks_per_sm(bn_bwd_apply_bifurcate_kernel<false, false>, kScanThreads)));
+    if (tot16) QBP_CUDA_OK(cudaMemsetAsync(tot16, 0, sizeof(int64_t) * (size_t)C, st));
+    // (three resident blocks per SM by the kernel's launch bounds, whatever the instance)
+    const ScanGeom ga = scan_geom(n, C, true, blocks_per_sm(bn_bwd_apply_bifurcate_kernel<true, true, true>, kScanThreads));
     const dim3 grid(ga.nbx, ga.slabs);
     const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
     const PhiloxKeys keys = philox_keys_host(seed);
@@ -937,9 +960,11 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
     const bool rows_in_warp = cv <= 32 && (cv & (cv - 1)) == 0;
     int32_t *row_sums_arg = (row_sums8 && rows_in_warp) ? row_sums8 : nullptr;
     QBP_TRACE_BEGIN(st);
-#define QBP_BN_BAB(R, G) bn_bwd_apply_bifurcate_kernel<R, G><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg)
-    if (g_out) { if (relu) QBP_BN_BAB(true, true); else QBP_BN_BAB(false, true); }
-    else       { if (relu) QBP_BN_BAB(true, false); else QBP_BN_BAB(false, false); }
+#define QBP_BN_BAB(R, G, T) bn_bwd_apply_bifurcate_kernel<R, G, T><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg, reinterpret_cast<unsigned long long *>(tot16))
+#define QBP_BN_BAB2(R, G) do { if (tot16) QBP_BN_BAB(R, G, true); else QBP_BN_BAB(R, G, false); } while (0)
+    if (g_out) { if (relu) QBP_BN_BAB2(true, true); else QBP_BN_BAB2(false, true); }
+    else       { if (relu) QBP_BN_BAB2(true, false); else QBP_BN_BAB2(false, false); }
+#undef QBP_BN_BAB2
 #undef QBP_BN_BAB
     QBP_LAUNCH_OK("bn_bwd_apply_bifurcate_kernel");
     if (row_sums8 && !rows_in_warp) return launch_rowsum(q8, true, n, C, row_sums8, st);

@@ -366,3 +366,31 @@ def test_gemm_with_caller_code_sums(B, M, N, K, tA, tB):
     oacc, oout, bad = O.gemm_s8(A, za, Bm, zb, sa, sb, transA=tA, transB=tB)
     assert bad == 0 and B.status_word(ws) == 0
     assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(out), oout)
+
+
+@pytest.mark.parametrize("mode", ["fprop", "dgrad"])
+def test_conv_at_full_size_is_reproducible(B, mode):
+    """The 64-channel 3x3 convolution of the benchmark, twenty times on the same codes: every run must write the same
+    bits.  (Integer accumulators and one fp32 scale leave no room for run-to-run differences; a difference means a
+    race -- one was found this way: an output slab refilled while the store of the tile before was still reading it,
+    in tiles whose rows lie partly outside the image.)  Each run starts from an output filled with NaN."""
+    import torch
+    cfg = synth.conv3x3_layer()
+    c = cfg["conv"]
+    d = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    src = to_dev(cfg["x"] if mode == "fprop" else cfg["dy"])
+    q_in, p_in = B.qbp_quantize_s8(src)
+    w = to_dev(cfg["w"])
+    q_w, p_w = B.qbp_quantize_s8(w.reshape(c["K"], -1))
+    out = torch.empty((c["N"], c["H"], c["W"], 64), dtype=torch.float32, device="cuda")
+    ref = None
+    for rep in range(20):
+        out.fill_(float("nan"))
+        B.qbp_conv_s8_implicit(B.QBP_CONV_FPROP if mode == "fprop" else B.QBP_CONV_DGRAD, d, q_in, p_in, q_w.reshape(w.shape), p_w, out=out)
+        torch.cuda.synchronize()
+        bits = out.view(torch.int32)
+        if ref is None:
+            ref = bits.clone()
+            assert not bool(torch.isnan(out).any())
+        else:
+            assert int((bits != ref).sum()) == 0, f"run {rep} differs from run 0"
