@@ -144,6 +144,30 @@ def test_backward_without_the_fp32_gradient_buffer(B, kind):
         assert all(np.array_equal(u, v) for u, v in zip(qa, qb))
 
 
+def test_layer_step_at_full_size_is_reproducible(B):
+    """Eight forward + backward steps of the benchmark's layer on the same tensors: every output and every kept
+    intermediate must come out with the same bits each time (integers, fixed summation orders, counter-based random
+    numbers: nothing in the path depends on timing)."""
+    import torch
+    from paper_1805_11046_b200 import layer
+    cfg = synth.conv3x3_layer()
+    c = cfg["conv"]
+    conv = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    x, w, dy = to_dev(cfg["x"]), to_dev(cfg["w"]), to_dev(cfg["dy"])
+    L = layer.QuantizedLayer(conv=conv, relu=True, seed=cfg["seed"], tensor_id8=cfg["id8"], tensor_id16=cfg["id16"], keep_g=False)
+    ref = None
+    for rep in range(8):
+        L.forward(x, w)
+        dx, dw, dgamma, dbeta = L.backward(dy)
+        torch.cuda.synchronize()
+        outs = [t.contiguous().view(torch.uint8).clone() for t in (L.x_codes, L.z, L.y, L.g8, L.ghi, L.glo, dx, dw, dgamma, dbeta, L.save_mean)]
+        if ref is None:
+            ref = outs
+        else:
+            assert all(int((a_ != b_).sum()) == 0 for a_, b_ in zip(outs, ref)), f"step {rep} differs from step 0"
+    assert L.status() == 0
+
+
 def test_bottleneck_stack_stagewise(B):
     """conv3_x bottleneck (1x1, 3x3, 1x1, each + Range BN + ReLU) at a reduced batch; every layer checked
     stage-wise on the activations the GPU handed to it."""
