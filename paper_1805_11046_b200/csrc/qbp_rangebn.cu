@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
                                                                 const float *__restrict__ vmax,
                                                                 const float *__restrict__ gamma,
                                                                 const float *__restrict__ beta, float Cn,
-                                                                float *__restrict__ y, BnRequant R)
+                                                                float *__restrict__ y, BnRequant R, int reverse)
 {
     const ScanPos p = scan_pos<VEC>(C, tw);
     // (with row sums the idle threads of a ragged last slab take part in the shuffles: tw <= 32 then, one slab)
@@ -160,7 +160,9 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
         for (int u = 0; u < kScanUnroll; ++u) {
             int64_t r = r0 + u * step;
             ok[u] = p.active && r < rows;
-            if (ok[u]) v[u].load_stream(x + r * C + p.col);
+            // (reverse: rows from the last to the first, when the kernel that wrote x ran just before and has left the
+            // tail of x in the L2)
+            if (ok[u]) v[u].load_stream(x + (reverse ? rows - 1 - r : r) * C + p.col);
         }
 #pragma unroll
         for (int u = 0; u < kScanUnroll; ++u) {
@@ -173,7 +175,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
                     v[u].v[e] = RELU ? fmaxf(yv, 0.0f) : yv;
                     if (REQUANT) code[e] = (uint32_t)quantize_code<false>(v[u].v[e], inv, zp_u, 255.0f, 0u);
                 }
-                const int64_t at = (r0 + u * step) * C + p.col;
+                const int64_t at = (reverse ? rows - 1 - (r0 + u * step) : r0 + u * step) * C + p.col;
                 if (y) v[u].store_stream(y + at);
                 if (REQUANT) {
                     if (VEC == 4) {
@@ -196,7 +198,7 @@ __global__ void __launch_bounds__(kScanThreads) bn_apply_kernel(const float *__r
                 for (int off = 16; off > 0; off >>= 1)
                     if (off < R.rs_group) rs += __shfl_xor_sync(0xffffffffu, rs, off);
                 const int64_t r = r0 + u * step;
-                if (p.tx == 0 && r < rows) R.rowsum[r] = rs;
+                if (p.tx == 0 && r < rows) R.rowsum[reverse ? rows - 1 - r : r] = rs;
             }
         }
     }
@@ -687,7 +689,8 @@ namespace qbp {
 // n_stat: the rows the statistics were taken over (more than n_rows when several GPUs share a minibatch).
 static int bn_fwd_apply_launch(const float *x, int64_t n_rows, int64_t n_stat, int64_t C, const float *gamma,
                                const float *beta, int relu, float *y, const float *save_mean, const float *save_min,
-                               const float *save_max, qbp_qparams *out_range, const qbp_requant *rq, cudaStream_t st)
+                               const float *save_max, qbp_qparams *out_range, const qbp_requant *rq, cudaStream_t st,
+                               bool reverse = false)
 {
     const bool requant = rq != nullptr;
     if (requant && (!rq->q || !rq->qp)) return fail(QBP_ERR_INVALID_ARG, "rangebn_fwd: the requantisation record needs q and qp");
@@ -722,7 +725,7 @@ static int bn_fwd_apply_launch(const float *x, int64_t n_rows, int64_t n_stat, i
         }
     }
     QBP_TRACE_BEGIN(st);
-#define QBP_BN_APPLY(V, RL, RQ) bn_apply_kernel<V, RL, RQ><<<grid_apply, kScanThreads, 0, st>>>(x, n_rows, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, y, R)
+#define QBP_BN_APPLY(V, RL, RQ) bn_apply_kernel<V, RL, RQ><<<grid_apply, kScanThreads, 0, st>>>(x, n_rows, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, y, R, reverse ? 1 : 0)
     if (ga.vec == 4) {
         if (requant) { if (relu) QBP_BN_APPLY(4, true, true); else QBP_BN_APPLY(4, false, true); }
         else         { if (relu) QBP_BN_APPLY(4, true, false); else QBP_BN_APPLY(4, false, false); }
@@ -842,7 +845,8 @@ int qbp::rangebn_fwd_from_parts(const float *x, int64_t n, int64_t C, const floa
     QBP_TRACE_BEGIN(st);
     bn_stats_finalize_kernel<<<(int)C, 128, 0, st>>>(parts.lo, parts.hi, parts.sum, parts.rows, (int)C, n, save_mean, save_min, save_max, nullptr);
     QBP_LAUNCH_OK("bn_stats_finalize_kernel");
-    return bn_fwd_apply_launch(x, n, n, C, gamma, beta, relu, y, save_mean, save_min, save_max, out_range, rq, st);
+    // (the product that left the statistics has just written x: its tail is in the L2)
+    return bn_fwd_apply_launch(x, n, n, C, gamma, beta, relu, y, save_mean, save_min, save_max, out_range, rq, st, true);
 }
 
 extern "C" __attribute__((visibility("default"))) int qbp_rangebn_bwd(const float *dy, const float *x, int64_t n, int64_t C, const float *gamma,
