@@ -461,7 +461,12 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
 // TOTALS: also each channel's total of the stored 16-bit codes (256 * hi + lo with lo unsigned, whatever lo_flip) over
 // all rows, added to chansum16 [C] (zeroed beforehand): a thread keeps its four channels for its whole life, a block
 // adds its threads' totals in shared memory and ends with one 64-bit atomic per channel.
-constexpr int kBabUnroll = 2;     // rows in flight per thread (two loads each): the pass is bound by arithmetic, so more resident warps
+// The pass is bound by arithmetic (Philox), and a thread that computes has no load in flight: the operands come through a
+// ring in shared memory, filled by each thread's own asynchronous copies kBabSlots - 1 steps ahead of the step it
+// computes (a thread reads back only what it copied itself: no barrier), so the memory system always has work.
+constexpr int kBabUnroll = 2;     // rows per thread and step (two operands each)
+constexpr int kBabSlots = 3;      // ring depth in steps
+constexpr size_t kBabRingBytes = (size_t)kBabSlots * kBabUnroll * 2 * kScanThreads * sizeof(float4);
 template <bool RELU, bool STORE_G, bool TOTALS>
 __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel(
     const float *__restrict__ dy, const float *__restrict__ x, int64_t rows, int C, int tw, const float *__restrict__ mean,
@@ -493,26 +498,42 @@ __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel
     const bool one_block = id8 == id16;
     const int64_t step = (int64_t)gridDim.x * rpb;
     // (the loop bound is the block's: every lane takes part in the row-sum shuffles)
-    for (int64_t base = (int64_t)blockIdx.x * rpb; base < rows; base += step * kBabUnroll) {
-        const int64_t r0 = base + p.ty;
-        VecF<4> vx[kBabUnroll], vd[kBabUnroll];
-        bool ok[kBabUnroll];
+    extern __shared__ __align__(16) float4 bab_ring[];         // [slot][row of the step][x | dy][thread]
+    float4 *const mine_ring = bab_ring + threadIdx.x;
+    const int64_t stride = step * kBabUnroll;
+    auto fetch = [&](int64_t base, int slot) {
 #pragma unroll
         for (int u = 0; u < kBabUnroll; ++u) {
-            const int64_t r = r0 + u * step;
-            ok[u] = p.active && r < rows;
-            if (ok[u]) { vx[u].load_stream(x + r * C + p.col); vd[u].load_stream(dy + r * C + p.col); }
+            const int64_t r = base + p.ty + u * step;
+            if (p.active && r < rows) {
+                cp_async16(mine_ring + ((slot * kBabUnroll + u) * 2 + 0) * kScanThreads, x + r * C + p.col);
+                cp_async16(mine_ring + ((slot * kBabUnroll + u) * 2 + 1) * kScanThreads, dy + r * C + p.col);
+            }
         }
+        cp_async_commit();                                     // (a group per step, empty past the end: the count below is uniform)
+    };
+#pragma unroll
+    for (int k = 0; k < kBabSlots - 1; ++k) fetch((int64_t)blockIdx.x * rpb + k * stride, k);
+    int slot = 0;
+    for (int64_t base = (int64_t)blockIdx.x * rpb; base < rows; base += stride) {
+        const int64_t r0 = base + p.ty;
+        // the slot this thread emptied in the step before takes the step kBabSlots - 1 ahead; then this step's data is in
+        fetch(base + (kBabSlots - 1) * stride, slot == 0 ? kBabSlots - 1 : slot - 1);
+        cp_async_wait<kBabSlots - 1>();
 #pragma unroll
         for (int u = 0; u < kBabUnroll; ++u) {
             const int64_t r = r0 + u * step;
+            const bool ok_u = p.active && r < rows;
             int rs = 0;
-            if (ok[u]) {
+            if (ok_u) {
+                const float4 fx = mine_ring[((slot * kBabUnroll + u) * 2 + 0) * kScanThreads];
+                const float4 fd = mine_ring[((slot * kBabUnroll + u) * 2 + 1) * kScanThreads];
+                const float ax[4] = {fx.x, fx.y, fx.z, fx.w}, ad[4] = {fd.x, fd.y, fd.z, fd.w};
                 float v[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float xv = vx[u].v[e];
-                    float d = vd[u].v[e];
+                    const float xv = ax[e];
+                    float d = ad[e];
                     if (RELU && !(bn_y(bn_xhat(xv, mu[e], s[e]), g[e], b[e]) > 0.0f)) d = 0.0f;
                     const float ind = (xv == hi[e] ? 1.0f : 0.0f) - (xv == lo[e] ? 1.0f : 0.0f);
                     v[e] = bn_dx(d, ind, s[e], g[e], m1[e], k2[e]);
@@ -544,10 +565,12 @@ __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel
             if (rowsum8) {
                 for (int off = 16; off > 0; off >>= 1)
                     if (off < tw) rs += __shfl_xor_sync(0xffffffffu, rs, off);
-                if (ok[u] && p.tx == 0) rowsum8[r] = rs;
+                if (ok_u && p.tx == 0) rowsum8[r] = rs;
             }
         }
+        slot = slot + 1 == kBabSlots ? 0 : slot + 1;
     }
+    cp_async_wait<0>();
     if (TOTALS) {
         __shared__ int s_tot[kScanMaxTw * 4];
         for (int i = threadIdx.x; i < tw * 4; i += kScanThreads) s_tot[i] = 0;
@@ -964,7 +987,7 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
     const bool rows_in_warp = cv <= 32 && (cv & (cv - 1)) == 0;
     int32_t *row_sums_arg = (row_sums8 && rows_in_warp) ? row_sums8 : nullptr;
     QBP_TRACE_BEGIN(st);
-#define QBP_BN_BAB(R, G, T) bn_bwd_apply_bifurcate_kernel<R, G, T><<<grid, kScanThreads, 0, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg, reinterpret_cast<unsigned long long *>(tot16))
+#define QBP_BN_BAB(R, G, T) do { static PerDeviceOnce once_; QBP_SMEM_OPT_IN(once_, (bn_bwd_apply_bifurcate_kernel<R, G, T>), kBabRingBytes); bn_bwd_apply_bifurcate_kernel<R, G, T><<<grid, kScanThreads, kBabRingBytes, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg, reinterpret_cast<unsigned long long *>(tot16)); } while (0)
 #define QBP_BN_BAB2(R, G) do { if (tot16) QBP_BN_BAB(R, G, true); else QBP_BN_BAB(R, G, false); } while (0)
     if (g_out) { if (relu) QBP_BN_BAB2(true, true); else QBP_BN_BAB2(false, true); }
     else       { if (relu) QBP_BN_BAB2(true, false); else QBP_BN_BAB2(false, false); }
