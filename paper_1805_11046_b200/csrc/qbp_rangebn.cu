@@ -456,8 +456,9 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
 // dx goes from registers into its 8-bit copy (stochastic rounding), the two limbs of its 16-bit copy and each row's
 // 8-bit code sum; the fp32 dx itself is written only when the caller keeps it (g_out).  The parameters of both copies
 // are known beforehand (bn_bwd_finalize_kernel + the range finalize).  Element i of the [rows x C] tensor draws from
-// Philox block i / 4 as in quantize_kernel: a thread's four channels are one block.  Whole rows lie inside a warp
-// (tw = C / 4 lanes, a power of two <= 32) when rowsum8 is given.
+// Philox block i / 4 as in quantize_kernel: a thread's four channels are one block.  rowsum8: a row's lanes
+// of one warp add up by shuffles; when a row spans several warps or blocks (tw > 32 or several slabs) the pieces are added
+// to rowsum8 [rows], zeroed beforehand.
 // TOTALS: also each channel's total of the stored 16-bit codes (256 * hi + lo with lo unsigned, whatever lo_flip) over
 // all rows, added to chansum16 [C] (zeroed beforehand): a thread keeps its four channels for its whole life, a block
 // adds its threads' totals in shared memory and ends with one 64-bit atomic per channel.
@@ -476,6 +477,7 @@ __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel
     const __grid_constant__ PhiloxKeys keys, uint32_t *__restrict__ q8, uint32_t *__restrict__ q_hi, uint32_t *__restrict__ q_lo,
     uint32_t lo_flip, int32_t *__restrict__ rowsum8, unsigned long long *__restrict__ chansum16)
 {
+    const bool rowsum_pieces = tw > 32 || gridDim.y > 1;
     const ScanPos p = scan_pos<4>(C, tw);
     uint32_t cs16[4] = {0u, 0u, 0u, 0u};          // unsigned codes of this thread's rows (fewer than 65536 rows)
     int mine = 0;
@@ -565,7 +567,11 @@ __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel
             if (rowsum8) {
                 for (int off = 16; off > 0; off >>= 1)
                     if (off < tw) rs += __shfl_xor_sync(0xffffffffu, rs, off);
-                if (ok_u && p.tx == 0) rowsum8[r] = rs;
+                // (a row wider than a warp's lanes, or than the block: each piece is added to the zeroed sum)
+                if (ok_u && (p.tx & 31) == 0) {
+                    if (rowsum_pieces) atomicAdd(rowsum8 + r, rs);
+                    else rowsum8[r] = rs;
+                }
             }
         }
         slot = slot + 1 == kBabSlots ? 0 : slot + 1;
@@ -945,7 +951,7 @@ static int bn_bwd_apply_launch(const float *dy, const float *x, int64_t n_rows, 
 bool rangebn_bwd_bifurcate_supported(const float *dy, const float *x, const float *g_out, int64_t n, int64_t C, bool row_sums)
 {
     if (!aligned16(x) || !aligned16(dy) || (g_out && !aligned16(g_out)) || C % 4 || n < 2 || n * C >= (1ll << 40)) return false;
-    (void)row_sums;      // (rows wider than a warp's lanes: the sums are taken from the codes afterwards)
+    (void)row_sums;      // (any row width: rows wider than a warp's lanes are added up from their pieces)
     return true;
 }
 
@@ -982,10 +988,10 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
     const float Cn = (float)(1.0 / std::sqrt(2.0 * std::log((double)n)));
     const PhiloxKeys keys = philox_keys_host(seed);
     const uint32_t flip = lo_signed ? 0x80808080u : 0u;
-    // each row's code sum by shuffles when a row's lanes lie inside one warp, else from the codes afterwards
-    const int64_t cv = C / 4;
-    const bool rows_in_warp = cv <= 32 && (cv & (cv - 1)) == 0;
-    int32_t *row_sums_arg = (row_sums8 && rows_in_warp) ? row_sums8 : nullptr;
+    // each row's code sum by shuffles over the row's lanes of a warp; a row that spans several warps or blocks is
+    // added up from its pieces (integer atomics on the zeroed sums: the result does not depend on the order)
+    int32_t *row_sums_arg = row_sums8;
+    if (row_sums8 && (ga.tw > 32 || ga.slabs > 1)) QBP_CUDA_OK(cudaMemsetAsync(row_sums8, 0, sizeof(int32_t) * (size_t)n, st));
     QBP_TRACE_BEGIN(st);
 #define QBP_BN_BAB(R, G, T) do { static PerDeviceOnce once_; QBP_SMEM_OPT_IN(once_, (bn_bwd_apply_bifurcate_kernel<R, G, T>), kBabRingBytes); bn_bwd_apply_bifurcate_kernel<R, G, T><<<grid, kScanThreads, kBabRingBytes, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg, reinterpret_cast<unsigned long long *>(tot16)); } while (0)
 #define QBP_BN_BAB2(R, G) do { if (tot16) QBP_BN_BAB(R, G, true); else QBP_BN_BAB(R, G, false); } while (0)
@@ -994,7 +1000,6 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
 #undef QBP_BN_BAB2
 #undef QBP_BN_BAB
     QBP_LAUNCH_OK("bn_bwd_apply_bifurcate_kernel");
-    if (row_sums8 && !rows_in_warp) return launch_rowsum(q8, true, n, C, row_sums8, st);
     return QBP_OK;
 }
 
