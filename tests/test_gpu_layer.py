@@ -421,11 +421,12 @@ def test_recompute_fusion_writes_the_same_codes_without_storing_the_product(B, b
 
 
 @pytest.mark.parametrize("batch,hw,cin,cout,R", [(3, 9, 32, 96, 3), (2, 12, 64, 32, 3), (2, 7, 96, 64, 3), (4, 6, 128, 128, 3),
-                                                   (3, 10, 64, 128, 1), (2, 5, 32, 32, 3)])
+                                                   (3, 10, 64, 128, 1), (2, 5, 32, 32, 3), (2, 6, 32, 320, 1)])
 def test_conv_layers_of_other_shapes_stagewise(B, batch, hw, cin, cout, R):
     """Forward and backward of convolution layers whose shapes take the other routes to the weight gradient's
     zero-point sums (with and without a spare chunk for the row of ones, channel counts the epilogue warps do or
-    do not take, 1x1 filters), each stage against the oracle."""
+    do not take, 1x1 filters, output rows wider than one block of the backward pass with a partly filled last slab),
+    each stage against the oracle."""
     pad = (R - 1) // 2
     cfg = dict(x=synth.relu_normal((batch, hw, hw, cin), 90), w=synth.kaiming_normal((cout, R, R, cin), 91),
                dy=synth.normal((batch, hw, hw, cout), 92, std=0.1), seed=5, id8=7, id16=7,
