@@ -247,8 +247,9 @@ size_t qbp_gemm_s8_workspace_bytes(int64_t M, int64_t N, int64_t K);
  * no statistics pass of its own.  col_sum (double), col_min, col_max: [N]
  * each (device), all three or none; they receive the sum / minimum / maximum
  * over the M rows of each column of C (of each output channel over all
- * positions for a convolution).  N <= QBP_EPILOGUE_MAX_COLUMNS, else
- * QBP_ERR_UNSUPPORTED_SHAPE.
+ * positions for a convolution).  qbp_gemm_s8: N <= QBP_EPILOGUE_MAX_COLUMNS,
+ * else QBP_ERR_UNSUPPORTED_SHAPE; qbp_conv_s8_implicit: any number of
+ * channels (at most 256 per SM of the device).
  *
  * (2) ReLU and requantisation, for a product whose output feeds the next
  * layer directly (no Range BN in between; Appendix B's quantiser with

@@ -105,7 +105,9 @@ static size_t step_scratch_bytes(const qbp_layer_desc *L, const LayerShape &s)
 // Buffers that live across steps, behind the shared step scratch: the per-row sums of the codes feeding the
 // next product (written by the quantiser that makes the codes) and the range partials of the gradient
 // (written by the Range BN backward pass that makes the gradient).
-static bool epilogue_stats(const LayerShape &s) { return s.conv && s.cout <= QBP_EPILOGUE_MAX_COLUMNS; }
+// (a convolution's epilogue takes the output's per-channel statistics for any number of channels that leaves a CTA one
+// column tile: 256 channels per tile, one CTA per SM)
+static bool epilogue_stats(const LayerShape &s) { return s.conv && (s.cout + 255) / 256 <= sm_count(); }
 static size_t colstat_cells(const LayerShape &s) { return epilogue_stats(s) ? (size_t)colstat_rows_max() * (size_t)s.cout : 0; }
 static size_t chained_bytes(const LayerShape &s)
 {
@@ -193,7 +195,7 @@ extern "C" __attribute__((visibility("default"))) int qbp_layer_fwd_chained(cons
         return fail(QBP_ERR_INVALID_ARG, "layer_fwd: the saved-state record has a NULL buffer");
     // saved->z == NULL: the fp32 output of the product is not kept (forward only): the convolution is run twice instead
     const bool recompute = saved->z == nullptr;
-    if (recompute && !(s.conv && epilogue_stats(s) && out && !y))
+    if (recompute && !(s.conv && s.cout <= QBP_EPILOGUE_MAX_COLUMNS && out && !y))
         return fail(QBP_ERR_INVALID_ARG, "layer_fwd: without saved->z the layer must be a convolution of at most %d output "
                     "channels that writes 8-bit codes only (out given, y NULL)", QBP_EPILOGUE_MAX_COLUMNS);
     if (in && (in->q != saved->x_codes || in->qp != saved->qx))

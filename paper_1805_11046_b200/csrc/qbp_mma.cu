@@ -187,8 +187,12 @@ struct MmaParams {
     int nslab;                    // epilogue staging slabs per warp (2: a store is still reading one while the next is filled)
     // Per-column statistics of the fp32 output (for the Range BN that follows, Section 3): every working epilogue
     // warp keeps (sum, min, max) of the columns in shared memory; when the kernel ends the CTA's warps add them up
-    // into row blockIdx.x of these partial arrays [rows][N].  One column tile only (N <= 256); NULL: not wanted.
+    // into row blockIdx.x of these partial arrays [rows][N].  NULL: not wanted.  Up to 256 columns every CTA keeps all of
+    // them (stat_cols = N); beyond (convolutions only) the grid is a multiple of the column tiles, so that a CTA meets one
+    // column tile in all its tiles (tile mod tiles_n = blockIdx.x mod tiles_n) and keeps that tile's stat_cols = bn
+    // columns only (stat_local), leaving the neutral element in the rest of its partial row.
     float *st_lo, *st_hi; double *st_sum;
+    int stat_cols, stat_local;
     // Optional tail of the epilogue: per-column normalisation by the Range BN that follows the product (ep_fold:
     // (mean, scale, gamma, beta) per output column, copied to shared memory), ReLU, and the 8-bit codes of the result
     // (parameters *ep_rq) written to ep_q [M x N] with each row's code sum in ep_rowsum (one column tile only).  `out`
@@ -581,9 +585,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
         uint8_t *slab0 = staging + (size_t)(ew * P.nslab) * kStageSlab;
         uint32_t slab_i = 0;
         const float scale = __fmul_rn(P.qa->scale, P.qb->scale);
-        ColStat *my_stat = s_stat + (size_t)ew * P.N;
+        ColStat *my_stat = s_stat + (size_t)ew * P.stat_cols;
+        const int stat_base = P.stat_local ? (int)(blockIdx.x % (unsigned)P.tiles_n) * P.bn : 0;     // first column this CTA keeps
         if (P.st_sum) {
-            for (int i = lane; i < (int)P.N; i += 32) { my_stat[i].sum = 0.0; my_stat[i].lo = INFINITY; my_stat[i].hi = -INFINITY; }
+            for (int i = lane; i < P.stat_cols; i += 32) { my_stat[i].sum = 0.0; my_stat[i].lo = INFINITY; my_stat[i].hi = -INFINITY; }
             __syncwarp();
         }
         const int sub = P.msub == 2 ? group : 0;
@@ -783,7 +788,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
                                 }
                             }
                             if (lane < lim && vmask) {
-                                ColStat &a = my_stat[o.n0 + c0 + lane];
+                                ColStat &a = my_stat[o.n0 - stat_base + c0 + lane];
                                 a.sum += (double)cs; a.lo = fminf(a.lo, clo); a.hi = fmaxf(a.hi, chi);
                             }
                         }
@@ -803,10 +808,12 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qbp_mma_kernel(const __grid_co
             const int64_t prow = (int64_t)blockIdx.x * P.N;
             for (int i = ew * 32 + lane; i < (int)P.N; i += 32 * P.ewarps) {
                 double sum = 0.0; float lo = INFINITY, hi = -INFINITY;
-                for (int w = 0; w < P.ewarps; ++w) {
-                    const ColStat &a = s_stat[(size_t)w * P.N + i];
-                    sum += a.sum; lo = fminf(lo, a.lo); hi = fmaxf(hi, a.hi);
-                }
+                const int li = i - stat_base;
+                if (li >= 0 && li < P.stat_cols)
+                    for (int w = 0; w < P.ewarps; ++w) {
+                        const ColStat &a = s_stat[(size_t)w * P.stat_cols + li];
+                        sum += a.sum; lo = fminf(lo, a.lo); hi = fmaxf(hi, a.hi);
+                    }
                 P.st_sum[prow + i] = sum; P.st_lo[prow + i] = lo; P.st_hi[prow + i] = hi;
             }
         }
@@ -1063,9 +1070,9 @@ __global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(long long lim
     if (timed_out && threadIdx.x == 0) raise_timeout(status);
 }
 
-static size_t colstat_ws_bytes(int64_t N)
+static size_t colstat_ws_bytes(int64_t N, bool conv = false)
 {
-    if (N > QBP_EPILOGUE_MAX_COLUMNS) return 0;
+    if (N > QBP_EPILOGUE_MAX_COLUMNS && !conv) return 0;
     const size_t cells = (size_t)colstat_rows_max() * (size_t)N;
     return align_up(cells * sizeof(float), 256) * 2 + align_up(cells * sizeof(double), 256);
 }
@@ -1078,7 +1085,7 @@ __global__ void epilogue_qparams_kernel(const qbp_qparams *__restrict__ range, q
 
 // What the caller's epilogue record asks for: column statistics (wanted) and / or the ReLU / requantisation tail.
 static int check_epilogue(const char *who, const qbp_epilogue *ep, const float *out, int64_t N, bool &wanted, EpilogueTail &tail,
-                          bool &has_tail)
+                          bool &has_tail, int64_t max_stat_cols = QBP_EPILOGUE_MAX_COLUMNS)
 {
     wanted = ep && (ep->col_sum || ep->col_min || ep->col_max);
     has_tail = ep && (ep->relu || ep->q_out);
@@ -1086,7 +1093,7 @@ static int check_epilogue(const char *who, const qbp_epilogue *ep, const float *
     if (wanted) {
         if (!ep->col_sum || !ep->col_min || !ep->col_max) return fail(QBP_ERR_INVALID_ARG, "%s: the epilogue needs col_sum, col_min and col_max together", who);
         if (!out) return fail(QBP_ERR_INVALID_ARG, "%s: column statistics need the fp32 output", who);
-        if (N > QBP_EPILOGUE_MAX_COLUMNS) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "%s: column statistics for at most %d columns", who, QBP_EPILOGUE_MAX_COLUMNS);
+        if (N > max_stat_cols) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "%s: column statistics for at most %lld columns", who, (long long)max_stat_cols);
         if (has_tail) return fail(QBP_ERR_INVALID_ARG, "%s: column statistics and ReLU / requantisation exclude one another", who);
     }
     if (has_tail) {
@@ -1130,7 +1137,9 @@ static uint32_t fixed_smem(MmaParams &P)
                                            : (size_t)(P.msub == 1 ? P.egroups : 1) * P.ncls * P.bn * sizeof(int32_t);
     P.iter_entries = P.mode == MODE_GEMM ? 0 : (int)align_up((size_t)P.k_iters, 64);
     P.cterm_span = (uint32_t)align_up(cterm_bytes, 1024);
-    P.stat_span = P.st_sum ? (uint32_t)align_up((size_t)P.ewarps * P.N * sizeof(ColStat), 1024) : 0u;
+    P.stat_local = (P.st_sum && P.N > QBP_EPILOGUE_MAX_COLUMNS) ? 1 : 0;
+    P.stat_cols = P.stat_local ? P.bn : (int)P.N;
+    P.stat_span = P.st_sum ? (uint32_t)align_up((size_t)P.ewarps * P.stat_cols * sizeof(ColStat), 1024) : 0u;
     const uint32_t fold_bytes = P.ep_fold ? (uint32_t)align_up((size_t)P.N * sizeof(float4), 1024) : 0u;
     return 2048u + (uint32_t)P.ewarps * kStageSlab * (uint32_t)P.nslab + (uint32_t)P.iter_entries * 16u + P.cterm_span +
            P.stat_span + fold_bytes;
@@ -1196,7 +1205,12 @@ static int launch_mma(MmaParams &P, int tiles_m, bool clear_status, cudaStream_t
     else      QBP_SMEM_OPT_IN(configured[0], qbp_mma_kernel<false>, kSmemBudget);
     if (clear_status) QBP_CUDA_OK(cudaMemsetAsync(P.status, 0, sizeof(int), st));
     // one CTA per SM (its shared-memory ring fills the SM), each walking its share of the tiles
-    const int grid = std::min(P.tiles_total, sm_count());
+    int grid = std::min(P.tiles_total, sm_count());
+    if (P.stat_local) {
+        // (a CTA then meets one column tile only: its tiles are blockIdx.x + k * grid)
+        if (P.mode == MODE_GEMM || P.tiles_n > grid) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "column statistics: too many columns");
+        grid -= grid % P.tiles_n;
+    }
     P.grid = grid;
     QBP_TRACE_BEGIN(st);
     if (tail) qbp_mma_kernel<true><<<grid, kMmaThreads, smem, st>>>(P);
@@ -1228,7 +1242,7 @@ static size_t conv_core_ws_bytes(const qbp_conv_desc *d)
 }
 static size_t conv_ws_bytes(const qbp_conv_desc *d)
 {
-    return conv_core_ws_bytes(d) + std::max(colstat_ws_bytes(d->C), colstat_ws_bytes(d->K));
+    return conv_core_ws_bytes(d) + std::max(colstat_ws_bytes(d->C, true), colstat_ws_bytes(d->K, true));
 }
 
 // Picks the pixel box (bw x bh x bn = 128, powers of two) that wastes the fewest MMA rows.
@@ -1424,7 +1438,8 @@ extern "C" __attribute__((visibility("default"))) int qbp_conv_s8_implicit(int m
     EpilogueTail tail;
     if (d && ep) {
         const int64_t Nout = mode == QBP_CONV_DGRAD ? d->C : d->K;
-        const int erc = check_epilogue("conv_s8", ep, out, Nout, stats, tail, has_tail);
+        // (a convolution takes the statistics of any number of channels: see MmaParams::stat_local)
+        const int erc = check_epilogue("conv_s8", ep, out, Nout, stats, tail, has_tail, INT32_MAX);
         if (erc) return erc;
         if (has_tail) {
             const int rc = launch_epilogue_qparams(ep, (cudaStream_t)stream);
@@ -1472,8 +1487,6 @@ int qbp::conv_s8_impl(int mode, const qbp_conv_desc *d, const int8_t *in, const 
         return fail(QBP_ERR_INVALID_ARG, "conv_s8: operands must be 16-byte aligned");
     if (!ws || ws_bytes < conv_core_ws_bytes(d))
         return fail(QBP_ERR_WORKSPACE, "conv_s8: workspace of %zu bytes needed, %zu given", conv_ws_bytes(d), ws_bytes);
-    if (stats && (mode == QBP_CONV_DGRAD ? d->C : d->K) > QBP_EPILOGUE_MAX_COLUMNS)
-        return fail(QBP_ERR_UNSUPPORTED_SHAPE, "conv_s8: column statistics for at most %d channels", QBP_EPILOGUE_MAX_COLUMNS);
     if (tail) {
         const int n_out = mode == QBP_CONV_DGRAD ? d->C : d->K;
         if (stats && (tail->fold || tail->relu || tail->q))

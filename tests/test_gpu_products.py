@@ -200,6 +200,23 @@ def test_conv_epilogue_channel_statistics(B, N, H, W, C, K, R, mode):
     _check_col_stats(out, stats)
 
 
+@pytest.mark.parametrize("N,H,W,C,K,R,mode", [(8, 14, 14, 128, 512, 1, 0), (2, 9, 9, 64, 768, 1, 0), (2, 10, 10, 640, 64, 3, 1),
+                                              (64, 28, 28, 128, 512, 1, 0), (64, 14, 14, 64, 768, 1, 0)])
+def test_conv_epilogue_channel_statistics_of_wide_outputs(B, N, H, W, C, K, R, mode):
+    """More than 256 output channels: several column tiles, each CTA keeping the statistics of the one it meets (two
+    and three column tiles, a ragged last one, grids smaller than and as large as the device)."""
+    pad = (R - 1) // 2
+    d = B.conv_desc(N, H, W, C, K, R, R, 1, pad); od = O.conv_desc(N, H, W, C, K, R, R, 1, pad)
+    inp = random_codes((N, H, W, C if mode == 0 else K), 25); w = random_codes((K, R, R, C), 26)
+    zi, zw = 7, -2
+    acc, out, ws, stats = B.qbp_conv_s8_implicit(mode, d, to_dev(inp), _qp(B, 0.5, zi), to_dev(w), _qp(B, 0.25, zw),
+                                                 want_acc=True, col_stats=True)
+    oacc, oout, bad = O.conv_s8(mode, od, inp, zi, w, zw, 0.5, 0.25)
+    assert bad == 0 and B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), oacc) and np.array_equal(to_host(out), oout)
+    _check_col_stats(out, stats)
+
+
 def test_wgrad_dense_sweep_shape_sampled_columns(B):
     """The limb-split 16 x 8-bit product at 4096^3 (dense sweep): operands quantised from N(0,1) (nearest for the
     8-bit side, stochastic for the 16-bit side); oracle on 96 sampled output columns (all 4096 rows of each)."""
