@@ -31,6 +31,14 @@
  *   qbo_rangebn_fwd       output range == sqrt(2 ln n), affine invariance,
  *                         C(n) closed form and the paper's worked number
  *   qbo_rangebn_bwd       central finite differences in fp64, sum identities
+ *   qbo_binarize/_pack    sign convention on hand-written values, bit order
+ *   qbo_xnor_gemm         the +-1 dot product written as a plain integer loop
+ *   qbo_stc_tern          exact cases (|g| = max, g = 0), unbiasedness within
+ *                         the binomial bound over many samples, sample index
+ *                         in the Philox counter
+ *   qbo_gated_xnor_gemm   the ternary x binary dot product as a plain loop
+ *   qbo_tbp_update        one sample == one product; the mean over many
+ *                         samples approaches the exact product g^T a
  */
 #include <math.h>
 #include <stdint.h>
@@ -563,4 +571,128 @@ void qbo_sgd_update(float *w, const float *dw, float *vbuf, int64_t n, float lr,
         float step = lr * g;
         w[i] = w[i] - step;
     }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Appendix C: Ternarized Back-Propagation (1-bit weights and activations,   */
+/* ternary gradients, XNOR + popcount products) and Algorithm 1              */
+/* ------------------------------------------------------------------------ */
+
+/* 1-bit weights / activations: b(x) = +1 for x >= 0, else -1 (the
+ * deterministic sign of the binarised networks Appendix C builds on). */
+void qbo_binarize(const float *x, int64_t n, int8_t *b)
+{
+    for (int64_t i = 0; i < n; ++i) b[i] = (x[i] >= 0.0f) ? 1 : -1;
+}
+
+/* [rows x cols] codes of +-1 (or a 0/1 mask when `mask`) to bit rows: element
+ * c of a row is bit c % 32 of word c / 32 (1 = "+1" or "set"); a row takes
+ * ceil(cols / 32) words, the spare bits of the last word are 0. */
+void qbo_pack_bits(const int8_t *b, int64_t rows, int64_t cols, int mask, uint32_t *words)
+{
+    int64_t wpr = (cols + 31) / 32;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t w = 0; w < wpr; ++w) {
+            uint32_t v = 0;
+            for (int64_t c = w * 32; c < cols && c < w * 32 + 32; ++c) {
+                int on = mask ? (b[r * cols + c] != 0) : (b[r * cols + c] > 0);
+                if (on) v |= 1u << (c - w * 32);
+            }
+            words[r * wpr + w] = v;
+        }
+}
+
+static int popcount32(uint32_t v) { int n = 0; while (v) { n += (int)(v & 1u); v >>= 1; } return n; }
+
+/* Forward product of a binarised layer (Appendix C: every MAC replaced by
+ * XNOR and population count): A [M x K bits], B [N x K bits], both as rows
+ * of ceil(K/32) words; C[m][n] = sum_k a*b over +-1 values
+ *   = (#equal bits) - (#different bits) = K - 2 popcount(a xor b). */
+void qbo_xnor_gemm(int64_t M, int64_t N, int64_t K, const uint32_t *A, const uint32_t *B, int32_t *C)
+{
+    int64_t wpr = (K + 31) / 32;
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            int diff = 0;
+            for (int64_t w = 0; w < wpr; ++w) diff += popcount32(A[m * wpr + w] ^ B[n * wpr + w]);
+            C[m * N + n] = (int32_t)(K - 2 * diff);      /* (spare bits are 0 in both: they never differ) */
+        }
+}
+
+/* Random word of element i for sample `sample`: as qbo_random_word, with the
+ * sample index in the last counter word. */
+uint32_t qbo_random_word_sample(uint64_t seed, uint32_t tensor_id, uint64_t i, uint32_t sample)
+{
+    uint64_t j = i >> 2;
+    uint32_t ctr[4] = { (uint32_t)j, (uint32_t)(j >> 32), tensor_id, sample };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    qbo_philox4x32_10(ctr, key, out);
+    return out[i & 3];
+}
+
+/* Stochastic ternarisation StcTern (Appendix C; the paper names it without a
+ * formula -- the reading taken is the one of the ternary-gradient work it
+ * cites): s = max |g| over the tensor, t_i = sign(g_i) with probability
+ * |g_i| / s, else 0, so that E[s t_i] = g_i.  The draw decides an integer, so
+ * it is taken in fp32 in a fixed order: p = |g_i| / s (one fp32 division),
+ * u = (word >> 8) * 2^-24 (exact), t_i != 0 iff u < p.  Returns s. */
+float qbo_stc_tern(const float *g, int64_t n, uint64_t seed, uint32_t tensor_id, uint32_t sample, int8_t *t)
+{
+    float s = 0.0f;
+    for (int64_t i = 0; i < n; ++i) { float a = fabsf(g[i]); if (a > s) s = a; }
+    for (int64_t i = 0; i < n; ++i) {
+        int8_t v = 0;
+        if (s > 0.0f) {
+            float p = fabsf(g[i]) / s;
+            float u = (float)(qbo_random_word_sample(seed, tensor_id, (uint64_t)i, sample) >> 8) * 0x1p-24f;
+            if (u < p) v = (g[i] > 0.0f) ? 1 : -1;
+        }
+        t[i] = v;
+    }
+    return s;
+}
+
+/* Backward product with ternary gradients and binary weights (the "gated
+ * XNOR"): T [M x K] ternary as two bit planes (nz: t != 0, sg: t > 0),
+ * B [N x K bits]; C[m][n] = sum_k t*b = popcount(nz & ~(sg ^ b)) -
+ * popcount(nz & (sg ^ b)): where t is non-zero, equal signs add one and
+ * different signs take one away. */
+void qbo_gated_xnor_gemm(int64_t M, int64_t N, int64_t K, const uint32_t *nz, const uint32_t *sg,
+                         const uint32_t *B, int32_t *C)
+{
+    int64_t wpr = (K + 31) / 32;
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            int acc = 0;
+            for (int64_t w = 0; w < wpr; ++w) {
+                uint32_t z = nz[m * wpr + w], d = sg[m * wpr + w] ^ B[n * wpr + w];
+                acc += popcount32(z & ~d) - popcount32(z & d);
+            }
+            C[m * N + n] = acc;
+        }
+}
+
+/* Algorithm 1 (multiple stochastic ternarisation sampling for the update
+ * phase): g [rows x N] gradients at the layer's output, a [rows x K] binarised
+ * activations (+-1); for every sample: ternarise g, add the product of the
+ * ternary tensor with the activations to the accumulator; return the
+ * accumulator over the number of samples.  gW [K x N], in units of g: the
+ * ternary values stand for s t.  The products are integers: they are
+ * accumulated exactly (int64) and scaled once at the end. */
+void qbo_tbp_update(const float *g, const int8_t *a, int64_t rows, int64_t N, int64_t K, int samples,
+                    uint64_t seed, uint32_t tensor_id, double *gW)
+{
+    int8_t *t = (int8_t *)malloc((size_t)(rows * N));
+    int64_t *acc = (int64_t *)calloc((size_t)(K * N), sizeof(int64_t));
+    float s = 0.0f;
+    for (int k = 0; k < samples; ++k) {
+        s = qbo_stc_tern(g, rows * N, seed, tensor_id, (uint32_t)k, t);
+        for (int64_t r = 0; r < rows; ++r)
+            for (int64_t c = 0; c < K; ++c)
+                for (int64_t n = 0; n < N; ++n)
+                    acc[c * N + n] += (int64_t)a[r * K + c] * (int64_t)t[r * N + n];
+    }
+    for (int64_t i = 0; i < K * N; ++i) gW[i] = (double)s * (double)acc[i] / (double)samples;
+    free(t); free(acc);
 }

@@ -62,6 +62,12 @@ def lib() -> C.CDLL:
         _lib.qbo_rangebn_C.argtypes = [C.c_int64]
         _lib.qbo_gemm_s8.restype = C.c_int64
         _lib.qbo_conv_s8.restype = C.c_int64
+        _lib.qbo_random_word_sample.restype = C.c_uint32
+        _lib.qbo_random_word_sample.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint32]
+        _lib.qbo_stc_tern.restype = C.c_float
+        _lib.qbo_stc_tern.argtypes = [C.c_void_p, C.c_int64, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p]
+        _lib.qbo_tbp_update.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_uint64,
+                                        C.c_uint32, C.c_void_p]
     return _lib
 
 
@@ -315,3 +321,56 @@ def layer_bwd_products(g, saved: LayerSaved, seed, id8, id16, conv: ConvDesc | N
                                     qx.scale[0], g16.scale[0])
     assert bad == 0
     return dx, dw, acc_dx, acc_dw, g8, g16
+
+
+# ------------------------------------------------- Appendix C: low-bit variants
+def random_word_sample(seed: int, tensor_id: int, i: int, sample: int) -> int:
+    return int(lib().qbo_random_word_sample(seed, tensor_id, i, sample))
+
+
+def binarize(x) -> np.ndarray:
+    """+1 for x >= 0, else -1 (int8, the shape of x)."""
+    x = _f32(x); b = np.empty(x.shape, dtype=np.int8)
+    lib().qbo_binarize(_p(x), C.c_int64(x.size), _p(b))
+    return b
+
+
+def pack_bits(codes, mask=False) -> np.ndarray:
+    """[rows x cols] int8 -> [rows x ceil(cols / 32)] uint32 bit rows (bit = code > 0, or code != 0 with mask)."""
+    b = np.ascontiguousarray(codes, dtype=np.int8); rows, cols = b.shape
+    w = np.zeros((rows, (cols + 31) // 32), dtype=np.uint32)
+    lib().qbo_pack_bits(_p(b), C.c_int64(rows), C.c_int64(cols), C.c_int(1 if mask else 0), _p(w))
+    return w
+
+
+def xnor_gemm(A_bits, B_bits, K) -> np.ndarray:
+    """C [M x N] int32 = K - 2 popcount(a xor b) for bit rows A [M x words], B [N x words]."""
+    A = np.ascontiguousarray(A_bits, dtype=np.uint32); Bm = np.ascontiguousarray(B_bits, dtype=np.uint32)
+    out = np.zeros((A.shape[0], Bm.shape[0]), dtype=np.int32)
+    lib().qbo_xnor_gemm(C.c_int64(A.shape[0]), C.c_int64(Bm.shape[0]), C.c_int64(K), _p(A), _p(Bm), _p(out))
+    return out
+
+
+def stc_tern(g, seed=0, tensor_id=0, sample=0):
+    """(t int8 in {-1, 0, 1} of g's shape, s = max |g|): one stochastic ternarisation of g."""
+    g = _f32(g); t = np.empty(g.shape, dtype=np.int8)
+    s = lib().qbo_stc_tern(_p(g), g.size, seed, tensor_id, sample, _p(t))
+    return t, np.float32(s)
+
+
+def gated_xnor_gemm(nz_bits, sign_bits, B_bits, K) -> np.ndarray:
+    """C [M x N] int32 = sum_k t b for ternary rows (non-zero and sign bit planes) against binary rows."""
+    nz = np.ascontiguousarray(nz_bits, dtype=np.uint32); sg = np.ascontiguousarray(sign_bits, dtype=np.uint32)
+    Bm = np.ascontiguousarray(B_bits, dtype=np.uint32)
+    out = np.zeros((nz.shape[0], Bm.shape[0]), dtype=np.int32)
+    lib().qbo_gated_xnor_gemm(C.c_int64(nz.shape[0]), C.c_int64(Bm.shape[0]), C.c_int64(K), _p(nz), _p(sg), _p(Bm), _p(out))
+    return out
+
+
+def tbp_update(g, a_bin, samples, seed=0, tensor_id=0) -> np.ndarray:
+    """Algorithm 1: gW [K x N] float64 from g [rows x N] and the binarised activations a [rows x K]."""
+    g = _f32(g); a = np.ascontiguousarray(a_bin, dtype=np.int8)
+    rows, N = g.shape; K = a.shape[1]
+    out = np.zeros((K, N), dtype=np.float64)
+    lib().qbo_tbp_update(_p(g), _p(a), rows, N, K, samples, seed, tensor_id, _p(out))
+    return out
