@@ -524,6 +524,56 @@ int qbp_layer_bwd(const qbp_layer_desc *L, const qbp_layer_ctx *saved, const flo
 int qbp_sgd_update(float *w, const float *dw, float *momentum_buf, int64_t count,
                    float lr, float momentum, float weight_decay, void *stream);
 
+/* ------------------------------------------------------------------------
+ * Appendix C -- Ternarized Back-Propagation: 1-bit weights and activations,
+ * ternary gradients, every forward MAC an XNOR + popcount.
+ *
+ * Binary and ternary tensors are int8 codes with zero-point 0 here: the
+ * +-1 dot product that XNOR + popcount computes is run by the int8 tensor
+ * cores through qbp_gemm_s8 / qbp_conv_s8_implicit / qbp_wgrad_s16, whose
+ * integer accumulators are that result exactly.
+ *
+ * qbp_binarize_s8: q[i] = +1 for x[i] >= 0 (also -0.0), else -1; n elements;
+ * x 4-byte aligned (device), q (device).  qp_out (nullable, device) receives
+ * scale 1, zero-point 0, the parameters to pass with q to a product.
+ * Allocates nothing.
+ *
+ * qbp_stc_ternarize_s8: the stochastic ternarisation the appendix and its
+ * Algorithm 1 use (not spelled out there; the one of the ternary-gradient
+ * work the paper cites): s = max |g| over the n elements; a sample keeps
+ * element i as sign(g[i]) with probability |g[i]| / s, else 0.  The draw is
+ * taken in fp32: p = |g| / s, u = (word >> 8) * 2^-24 with the element's
+ * Philox4x32-10 word (block i / 4, word i % 4, counter words 2 and 3 =
+ * tensor_id and the sample index, key = seed), kept iff u < p.  q[i] = the
+ * sum of the element's `samples` (1..127) samples, in [-samples, samples];
+ * qp_out: scale = s / samples (1 when s = 0), zero-point 0, vmin / vmax =
+ * -s / s, so that scale * q[i] estimates g[i] without bias.  samples = 1 is
+ * a ternary tensor.  ws of qbp_stc_ternarize_workspace_bytes() bytes.
+ *
+ * qbp_tbp_weight_gradient: Algorithm 1 (multiple stochastic ternarisation
+ * sampling): the weight gradient of a binarised layer as the mean over
+ * `samples` ternarisations of g of the product (ternary g)^T (binary a).
+ * The samples are added per element first (the product is linear in them)
+ * and one 16-bit x 8-bit product is run.  d == NULL: a [rows x K] (+-1
+ * codes, parameters qa from qbp_binarize_s8), g [rows x N] fp32, gW [K x N];
+ * d != NULL: a is the layer's NHWC input, g its NHWC output gradient, gW
+ * [K][R][S][C] (rows, N, K are then taken from d).  t_hi / t_lo (device,
+ * rows * N bytes each, 16-byte aligned) receive the byte limbs of the summed
+ * samples, qp_t their parameters; acc_out (int64, nullable) the integer
+ * accumulators, gW (nullable) = accumulator * qa.scale * qp_t.scale.  Shape
+ * limits and errors as qbp_wgrad_s16.
+ * ---------------------------------------------------------------------- */
+int qbp_binarize_s8(const float *x, int64_t n, int8_t *q, qbp_qparams *qp_out, void *stream);
+size_t qbp_stc_ternarize_workspace_bytes(void);
+int qbp_stc_ternarize_s8(const float *g, int64_t n, int samples, uint64_t seed, uint32_t tensor_id,
+                         int8_t *q, qbp_qparams *qp_out, void *ws, size_t ws_bytes, void *stream);
+size_t qbp_tbp_weight_gradient_workspace_bytes(const qbp_conv_desc *d, int64_t rows, int64_t N, int64_t K);
+int qbp_tbp_weight_gradient(const qbp_conv_desc *d, int64_t rows, int64_t N, int64_t K,
+                            const int8_t *a_codes, const qbp_qparams *qa, const float *g,
+                            int samples, uint64_t seed, uint32_t tensor_id,
+                            int8_t *t_hi, uint8_t *t_lo, qbp_qparams *qp_t,
+                            int64_t *acc_out, float *gW, void *ws, size_t ws_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -33,6 +33,8 @@ EXPORTS = (
     "qbp_rangebn_workspace_bytes", "qbp_rangebn_fwd", "qbp_rangebn_bwd", "qbp_rangebn_fwd_q8",
     "qbp_rangebn_fwd_stats", "qbp_rangebn_fwd_apply", "qbp_rangebn_bwd_stats", "qbp_rangebn_bwd_apply",
     "qbp_layer_workspace_bytes", "qbp_layer_fwd", "qbp_layer_fwd_chained", "qbp_layer_bwd",
+    "qbp_binarize_s8", "qbp_stc_ternarize_workspace_bytes", "qbp_stc_ternarize_s8",
+    "qbp_tbp_weight_gradient_workspace_bytes", "qbp_tbp_weight_gradient",
 )
 
 
@@ -89,6 +91,8 @@ def _load() -> C.CDLL:
     lib.qbp_rangebn_workspace_bytes.argtypes = [C.c_int64, C.c_int64]
     lib.qbp_layer_workspace_bytes.argtypes = [C.c_void_p]
     lib.qbp_range_chunked_workspace_bytes.argtypes = []
+    lib.qbp_stc_ternarize_workspace_bytes.argtypes = []
+    lib.qbp_tbp_weight_gradient_workspace_bytes.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64]
     return lib
 
 
@@ -334,6 +338,41 @@ def qbp_wgrad_s16(x, qx, g_hi, g_lo, qg16, d: ConvDesc | None = None, want_acc=F
                              _ptr(g_lo), _ptr(qg16), _ptr(acc_out), _ptr(dW), _ptr(ws), C.c_size_t(ws.numel()),
                              _stream()))
     return acc_out, dW, ws
+
+
+# ------------------------------------------------- Appendix C: 1-bit operands, ternary gradients
+def qbp_binarize_s8(x, q=None, qp_out=None):
+    if q is None: q = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+    if qp_out is None: qp_out = new_qparams(1, x.device)
+    _check(lib.qbp_binarize_s8(_ptr(x), C.c_int64(x.numel()), _ptr(q), _ptr(qp_out), _stream()))
+    return q, qp_out
+
+
+def qbp_stc_ternarize_s8(g, samples=1, seed=0, tensor_id=0, q=None, qp_out=None, ws=None):
+    if q is None: q = torch.empty(g.shape, dtype=torch.int8, device=g.device)
+    if qp_out is None: qp_out = new_qparams(1, g.device)
+    if ws is None: ws = workspace(lib.qbp_stc_ternarize_workspace_bytes(), g.device)
+    _check(lib.qbp_stc_ternarize_s8(_ptr(g), C.c_int64(g.numel()), int(samples), C.c_uint64(seed), C.c_uint32(tensor_id),
+                                    _ptr(q), _ptr(qp_out), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return q, qp_out
+
+
+def qbp_tbp_weight_gradient(a_codes, qa, g, samples, seed=0, tensor_id=0, d: ConvDesc | None = None, want_acc=False, ws=None):
+    """Algorithm 1: (acc int64 or None, gW fp32, t_hi, t_lo, qp_t)."""
+    if d is None:
+        rows, K = a_codes.shape; N = g.shape[1]; shape = (K, N); dref = None
+    else:
+        rows = d.N * d.H * d.W; K = d.C; N = d.K; shape = (d.K, d.R, d.S, d.C); dref = C.byref(d)
+    dev = g.device
+    t_hi = torch.empty(g.shape, dtype=torch.int8, device=dev); t_lo = torch.empty(g.shape, dtype=torch.uint8, device=dev)
+    qp_t = new_qparams(1, dev)
+    acc = torch.empty(shape, dtype=torch.int64, device=dev) if want_acc else None
+    gW = torch.empty(shape, dtype=torch.float32, device=dev)
+    if ws is None: ws = workspace(lib.qbp_tbp_weight_gradient_workspace_bytes(dref, rows, N, K), dev)
+    _check(lib.qbp_tbp_weight_gradient(dref, C.c_int64(rows), C.c_int64(N), C.c_int64(K), _ptr(a_codes), _ptr(qa), _ptr(g),
+                                       int(samples), C.c_uint64(seed), C.c_uint32(tensor_id), _ptr(t_hi), _ptr(t_lo), _ptr(qp_t),
+                                       _ptr(acc), _ptr(gW), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
+    return acc, gW, t_hi, t_lo, qp_t
 
 
 # ------------------------------------------------------------------- Range BN

@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libqbp.so"
-SOURCES = ["qbp_quant.cu", "qbp_rangebn.cu", "qbp_mma.cu", "qbp_mma2.cu", "qbp_wgrad.cu", "qbp_wgrad2.cu", "qbp_layer.cu"]
+SOURCES = ["qbp_quant.cu", "qbp_rangebn.cu", "qbp_mma.cu", "qbp_mma2.cu", "qbp_wgrad.cu", "qbp_wgrad2.cu", "qbp_layer.cu", "qbp_tbp.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -13,6 +13,10 @@ namespace qbp {
 int launch_rowsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int32_t *sums, cudaStream_t st);
 int launch_colsum(const void *q, bool is_signed, int64_t rows, int64_t cols, int64_t *sums, cudaStream_t st);
 
+// ---- per-tensor range scan (qbp_quant.cu): *qp = 8-bit parameters of [min(lowest, 0), max(highest, 0)] -------------
+size_t range_scan_ws_bytes();
+int range_scan(const float *x, int64_t n, void *ws, size_t ws_bytes, qbp_qparams *qp, cudaStream_t st);
+
 // ---- pieces the whole-layer composition chains without a pass of their own ------
 // Range BN backward that also leaves per-block (min, max) of dx (qbp_rangebn.cu), and the gradient
 // bifurcation that starts from such partials instead of scanning (qbp_quant.cu).

@@ -617,6 +617,15 @@ static int launch_range(const float *x, int64_t n, float2 *partials, qbp_qparams
     return QBP_OK;
 }
 
+// The per-tensor scan for callers in other files: *qp receives the 8-bit parameters of the tensor's range widened to
+// hold 0 (vmin = min(lowest, 0), vmax = max(highest, 0)).
+size_t range_scan_ws_bytes() { return align_up(sizeof(float2) * kMaxParts, 256); }
+int range_scan(const float *x, int64_t n, void *ws, size_t ws_bytes, qbp_qparams *qp, cudaStream_t st)
+{
+    if (!ws || ws_bytes < range_scan_ws_bytes()) return fail(QBP_ERR_WORKSPACE, "range scan: workspace too small");
+    return launch_range(x, n, static_cast<float2 *>(ws), qp, nullptr, st);
+}
+
 static int launch_chan_range(const float *x, int64_t rows, int64_t cols, int bits, float *part_lo, float *part_hi,
                              qbp_qparams *qp, cudaStream_t st)
 {

@@ -1,0 +1,133 @@
+"""Appendix C on the GPU against the CPU oracle: binarisation, stochastic ternarisation (one sample and the sum of
+several), the XNOR-popcount forward product and the gated-XNOR backward product as int8 tensor-core products on +-1
+and ternary bytes, and Algorithm 1.  Codes and integer accumulators bit for bit."""
+import numpy as np
+import pytest
+
+from oracle import qbp_oracle as O
+from paper_1805_11046_b200 import synth
+from tests.util import to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import paper_1805_11046_b200.binding as binding
+    return binding
+
+
+def _tern_sum(g, samples, seed, tid):
+    tot = np.zeros(g.shape, dtype=np.int32)
+    s = np.float32(0)
+    for k in range(samples):
+        t, s = O.stc_tern(g, seed, tid, k)
+        tot += t
+    return tot, s
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 1027, 64 * 256, 1 << 20])
+def test_binarize(B, n):
+    x = synth.normal((n,), 31)
+    x[:: 7] = 0.0
+    if n > 2: x[2] = -0.0
+    q, qp = B.qbp_binarize_s8(to_dev(x))
+    assert np.array_equal(to_host(q), O.binarize(x))
+    s, z, lo, hi = B.read_qparams(qp)
+    assert s[0] == 1.0 and z[0] == 0 and lo[0] == -1.0 and hi[0] == 1.0
+    # a tensor that starts 4 bytes into a 16-byte line takes the element-wise path
+    if n > 8:
+        import torch
+        buf = to_dev(np.concatenate([[np.float32(0)], x]))
+        q2, _ = B.qbp_binarize_s8(buf[1:], q=torch.empty(n, dtype=torch.int8, device="cuda"))
+        assert np.array_equal(to_host(q2), O.binarize(x))
+
+
+@pytest.mark.parametrize("n,samples", [(1, 1), (5, 3), (1027, 1), (4096, 6), (64 * 300 + 2, 2), (1 << 18, 20)])
+def test_stochastic_ternarisation_codes(B, n, samples):
+    g = synth.normal((n,), 32, std=0.3)
+    g[:: 5] = 0.0
+    q, qp = B.qbp_stc_ternarize_s8(to_dev(g), samples=samples, seed=77, tensor_id=9)
+    want, s = _tern_sum(g, samples, 77, 9)
+    assert np.array_equal(to_host(q).astype(np.int32), want)
+    sc, z, lo, hi = B.read_qparams(qp)
+    assert z[0] == 0 and hi[0] == s and lo[0] == -s
+    assert sc[0] == (np.float32(s) / np.float32(samples) if s > 0 else np.float32(1))
+    if n > 8:
+        import torch
+        buf = to_dev(np.concatenate([[np.float32(0)], g]))
+        q2, _ = B.qbp_stc_ternarize_s8(buf[1:], samples=samples, seed=77, tensor_id=9)
+        assert np.array_equal(to_host(q2).astype(np.int32), want)
+
+
+def test_ternarisation_of_zeros_and_of_the_full_size_gradient(B):
+    q, qp = B.qbp_stc_ternarize_s8(to_dev(np.zeros(100, dtype=np.float32)), samples=4)
+    assert not to_host(q).any() and B.read_qparams(qp)[0][0] == 1.0
+    g = synth.normal((256 * 56 * 56 * 64,), 33, std=0.05)           # the benchmark layer's gradient tensor
+    q, qp = B.qbp_stc_ternarize_s8(to_dev(g), samples=1, seed=5, tensor_id=6)
+    want, s = O.stc_tern(g, 5, 6, 0)
+    assert np.array_equal(to_host(q), want) and B.read_qparams(qp)[3][0] == s
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 48, 128), (256, 128, 1024), (16, 16, 16), (512, 272, 2064)])
+def test_forward_product_equals_xnor_popcount(B, M, N, K):
+    """Appendix C: the forward MACs of a binarised layer as XNOR + popcount; here the int8 tensor-core product on the
+    +-1 bytes, whose accumulators must be the popcount results."""
+    a = synth.normal((M, K), 34); w = synth.normal((N, K), 35)
+    qa, pa = B.qbp_binarize_s8(to_dev(a)); qw, pw = B.qbp_binarize_s8(to_dev(w))
+    acc, out, ws = B.qbp_gemm_s8(qa, pa, qw, pw, transB=True, want_acc=True)
+    want = O.xnor_gemm(O.pack_bits(O.binarize(a)), O.pack_bits(O.binarize(w)), K)
+    assert B.status_word(ws) == 0
+    assert np.array_equal(to_host(acc), want) and np.array_equal(to_host(out), want.astype(np.float32))
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 128, 48), (256, 512, 128), (16, 32, 16)])
+def test_backward_product_equals_gated_xnor(B, M, N, K):
+    """The layer gradient of a binarised layer from a ternary gradient: dx [M x K] = t [M x N] . W [N x K]."""
+    g = synth.normal((M, N), 36, std=0.2); w = synth.normal((N, K), 37)
+    t, pt = B.qbp_stc_ternarize_s8(to_dev(g), samples=1, seed=3, tensor_id=4)
+    qw, pw = B.qbp_binarize_s8(to_dev(w))
+    acc, out, ws = B.qbp_gemm_s8(t, pt, qw, pw, want_acc=True)
+    ot, s = O.stc_tern(g, 3, 4, 0)
+    wb = O.binarize(w)
+    want = O.gated_xnor_gemm(O.pack_bits(ot, mask=True), O.pack_bits(ot), O.pack_bits(np.ascontiguousarray(wb.T)), N)
+    assert B.status_word(ws) == 0 and np.array_equal(to_host(acc), want)
+    assert np.array_equal(to_host(out), (want.astype(np.float32) * np.float32(s)))      # in units of g: s * t
+
+
+@pytest.mark.parametrize("rows,K,N,samples", [(256, 64, 48, 1), (256, 64, 48, 6), (1024, 128, 256, 12), (70000, 32, 32, 3)])
+def test_algorithm_1_linear(B, rows, K, N, samples):
+    g = synth.normal((rows, N), 38, std=0.1); a = synth.normal((rows, K), 39)
+    qa, pa = B.qbp_binarize_s8(to_dev(a))
+    acc, gW, t_hi, t_lo, pt = B.qbp_tbp_weight_gradient(qa, pa, to_dev(g), samples, seed=11, tensor_id=12, want_acc=True)
+    tsum, s = _tern_sum(g, samples, 11, 12)
+    ab = O.binarize(a).astype(np.int64)
+    want = ab.T @ tsum.astype(np.int64)                                  # the sum of the samples' products (exact integers)
+    assert np.array_equal(to_host(acc), want)
+    # the limbs hold the summed samples as a 16-bit code
+    assert np.array_equal(to_host(t_hi).astype(np.int32) * 256 + to_host(t_lo).astype(np.int32), tsum)
+    scale = np.float32(s) / np.float32(samples)
+    assert np.array_equal(to_host(gW), want.astype(np.float32) * scale)
+    if rows <= 1024:
+        ref = O.tbp_update(g, O.binarize(a), samples, seed=11, tensor_id=12)
+        assert np.max(np.abs(to_host(gW) - ref)) <= 1e-6 * max(1.0, np.max(np.abs(ref)))
+
+
+@pytest.mark.parametrize("N,H,W,C,K,R,samples", [(2, 8, 8, 32, 32, 3, 3), (4, 14, 14, 64, 64, 3, 2), (2, 7, 7, 64, 128, 1, 4)])
+def test_algorithm_1_convolution(B, N, H, W, C, K, R, samples):
+    """Algorithm 1 for a convolution layer, in the algorithm's order on the oracle's side: one weight-gradient product
+    per sample, added up."""
+    pad = (R - 1) // 2
+    d = B.conv_desc(N, H, W, C, K, R, R, 1, pad); od = O.conv_desc(N, H, W, C, K, R, R, 1, pad)
+    a = synth.normal((N, H, W, C), 40); g = synth.normal((N, H, W, K), 41, std=0.1)
+    qa, pa = B.qbp_binarize_s8(to_dev(a))
+    acc, gW, _, _, pt = B.qbp_tbp_weight_gradient(qa, pa, to_dev(g), samples, seed=21, tensor_id=22, d=d, want_acc=True)
+    ab = O.binarize(a)
+    want = np.zeros((K, R, R, C), dtype=np.int64)
+    s = np.float32(0)
+    for k in range(samples):
+        t, s = O.stc_tern(g, 21, 22, k)
+        oacc, _ = O.conv_wgrad_s16(od, ab, 0, t.astype(np.int16), 0, 1.0, 1.0)
+        want += oacc.reshape(want.shape)
+    assert np.array_equal(to_host(acc), want)
+    assert np.array_equal(to_host(gW), want.astype(np.float32) * (np.float32(s) / np.float32(samples)))
