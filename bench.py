@@ -301,6 +301,8 @@ def run_ours(args):
         line["rangebn_c3"] = rangebn_sweep_block(B, args.batch, hbm_peak)
         torch.cuda.empty_cache()
         line["stack_c4"] = stack_block(B, args.batch)
+        torch.cuda.empty_cache()
+        line["tbp_appendix_c"] = tbp_block(B, args.batch, hbm_peak, peaks)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.cpu_sample_batch)
     if rank == 0:
@@ -475,6 +477,52 @@ def stack_block(B, batch, reps=20):
         out[name] = {"ms_per_step": round(ms, 4), "images_per_s": round(batch / (ms * 1e-3), 1), "launches": launches}
         del S, g
         torch.cuda.empty_cache()
+    return out
+
+
+def tbp_block(B, batch, hbm_peak, peaks, launches=30):
+    """Appendix C (1-bit operands, ternary gradients) at the benchmark layer's size: the binarisation and the stochastic
+    ternarisation (1 sample, and the sum of 6 for Algorithm 1) of the 51.4 M-element activation / gradient tensor as
+    graph-timed calls over rotating buffers (bytes per element: 4 in + 1 out, plus 4 for the ternariser's range scan),
+    the forward product of a binarised 4096^3 layer (XNOR-popcount result on the int8 tensor cores), and Algorithm 1
+    for the conv2_x layer (ternarise 6 samples + one weight-gradient product)."""
+    import torch
+    from paper_1805_11046_b200 import synth
+    cfg = conv_workload(batch)
+    E = cfg["dy"].size
+    g0 = torch.from_numpy(cfg["dy"]).cuda()
+    gs = [g0, g0.clone(), g0.clone()]
+    qs = [torch.empty(g0.shape, dtype=torch.int8, device="cuda") for _ in gs]
+    qp = B.new_qparams(1); ws = B.workspace(B.lib.qbp_stc_ternarize_workspace_bytes())
+    passes = {
+        "binarize": (5, [lambda i=i: B.qbp_binarize_s8(gs[i], q=qs[i], qp_out=qp) for i in range(3)]),
+        "stc_ternarize_1_sample_with_scan": (9, [lambda i=i: B.qbp_stc_ternarize_s8(gs[i], 1, 1, 2, q=qs[i], qp_out=qp, ws=ws) for i in range(3)]),
+        "stc_ternarize_6_samples_with_scan": (9, [lambda i=i: B.qbp_stc_ternarize_s8(gs[i], 6, 1, 2, q=qs[i], qp_out=qp, ws=ws) for i in range(3)]),
+    }
+    out = {"tensor_elements": E, "passes": {}}
+    for name, (bpe, calls) in passes.items():
+        ms = _graph_ms_per_call(calls, launches)
+        gbs = bpe * E / (ms * 1e-3) / 1e9
+        out["passes"][name] = {"us": round(ms * 1e3, 2), "bytes_per_element": bpe, "gbs": round(gbs, 0), "frac": round(gbs / hbm_peak, 3)}
+    # forward product of a binarised layer, 4096^3
+    n = 4096
+    case = synth.dense_gemm(n, n, n)
+    qa, pa = B.qbp_binarize_s8(torch.from_numpy(case["a"]).cuda()); qb, pb = B.qbp_binarize_s8(torch.from_numpy(case["b"]).cuda())
+    o = torch.empty((n, n), dtype=torch.float32, device="cuda"); wsg = B.workspace(B.lib.qbp_gemm_s8_workspace_bytes(n, n, n))
+    ms = _graph_ms_per_call([lambda: B.qbp_gemm_s8(qa, pa, qb, pb, out=o, ws=wsg)], 20)
+    out["xnor_forward_4096"] = {"ms": round(ms, 4), "tera_bit_macs_per_s": round(n ** 3 / (ms * 1e-3) / 1e12, 1),
+                                "int8_tops": round(2 * n ** 3 / (ms * 1e-3) / 1e12, 1),
+                                "frac_of_measured_burst": round(2 * n ** 3 / (ms * 1e-3) / 1e12 / (2 * float(peaks["bf16_tflops"])), 3),
+                                "includes": "the two code-sum kernels and the terms kernel of the call"}
+    del qa, qb, o, wsg, case
+    # Algorithm 1 for the benchmark layer: 6 samples
+    import ctypes
+    c = cfg["conv"]
+    d = B.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["stride"], c["pad"])
+    a_codes, qa = B.qbp_binarize_s8(torch.from_numpy(cfg["x"]).cuda())
+    wsa = B.workspace(B.lib.qbp_tbp_weight_gradient_workspace_bytes(ctypes.byref(d), 0, 0, 0))
+    ms = _graph_ms_per_call([lambda: B.qbp_tbp_weight_gradient(a_codes, qa, g0, 6, seed=1, tensor_id=2, d=d, ws=wsa)], 10)
+    out["algorithm_1_conv2x_6_samples"] = {"ms": round(ms, 4), "images_per_s": round(batch / (ms * 1e-3), 1)}
     return out
 
 
