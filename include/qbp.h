@@ -542,9 +542,9 @@ int qbp_sgd_update(float *w, const float *dw, float *momentum_buf, int64_t count
  * Algorithm 1 use (not spelled out there; the one of the ternary-gradient
  * work the paper cites): s = max |g| over the n elements; a sample keeps
  * element i as sign(g[i]) with probability |g[i]| / s, else 0.  The draw is
- * taken in fp32: p = |g| / s, u = (word >> 8) * 2^-24 with the element's
- * Philox4x32-10 word (block i / 4, word i % 4, counter words 2 and 3 =
- * tensor_id and the sample index, key = seed), kept iff u < p.  q[i] = the
+ * taken in fp32: u = (word >> 8) * 2^-24 with the element's Philox4x32-10
+ * word (block i / 4, word i % 4, counter words 2 and 3 = tensor_id and the
+ * sample index, key = seed), kept iff u * s < |g[i]| (s > 0).  q[i] = the
  * sum of the element's `samples` (1..127) samples, in [-samples, samples];
  * qp_out: scale = s / samples (1 when s = 0), zero-point 0, vmin / vmax =
  * -s / s, so that scale * q[i] estimates g[i] without bias.  samples = 1 is

@@ -635,8 +635,10 @@ uint32_t qbo_random_word_sample(uint64_t seed, uint32_t tensor_id, uint64_t i, u
  * formula -- the reading taken is the one of the ternary-gradient work it
  * cites): s = max |g| over the tensor, t_i = sign(g_i) with probability
  * |g_i| / s, else 0, so that E[s t_i] = g_i.  The draw decides an integer, so
- * it is taken in fp32 in a fixed order: p = |g_i| / s (one fp32 division),
- * u = (word >> 8) * 2^-24 (exact), t_i != 0 iff u < p.  Returns s. */
+ * it is taken in fp32 in a fixed order: u = (word >> 8) * 2^-24 (exact),
+ * t_i != 0 iff u * s < |g_i| (one fp32 product, rounded to nearest: for
+ * |g_i| = s it is always below s, so the largest element is always kept).
+ * Returns s. */
 float qbo_stc_tern(const float *g, int64_t n, uint64_t seed, uint32_t tensor_id, uint32_t sample, int8_t *t)
 {
     float s = 0.0f;
@@ -644,9 +646,9 @@ float qbo_stc_tern(const float *g, int64_t n, uint64_t seed, uint32_t tensor_id,
     for (int64_t i = 0; i < n; ++i) {
         int8_t v = 0;
         if (s > 0.0f) {
-            float p = fabsf(g[i]) / s;
             float u = (float)(qbo_random_word_sample(seed, tensor_id, (uint64_t)i, sample) >> 8) * 0x1p-24f;
-            if (u < p) v = (g[i] > 0.0f) ? 1 : -1;
+            float us = u * s;
+            if (us < fabsf(g[i])) v = (g[i] > 0.0f) ? 1 : -1;
         }
         t[i] = v;
     }

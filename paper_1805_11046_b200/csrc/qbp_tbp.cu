@@ -41,10 +41,13 @@ __global__ void __launch_bounds__(kTbpThreads) binarize_kernel(const float *__re
     }
 }
 
-// One element: how many of its `samples` draws keep it.  p = |g| / s in fp32 (one division), a draw keeps the element
-// when (word >> 8) * 2^-24 < p; the words of sample k are Philox block (j, id, k).
-__device__ __forceinline__ float tern_prob(float g, float s) { return s > 0.0f ? __fdiv_rn(fabsf(g), s) : 0.0f; }
-__device__ __forceinline__ int tern_keep(uint32_t word, float p) { return __fmul_rn((float)(word >> 8), 0x1p-24f) < p ? 1 : 0; }
+// One element: how many of its `samples` draws keep it.  A draw u = (word >> 8) * 2^-24 keeps the element when
+// u * s < |g| (one fp32 product, rounded to nearest; with s = 0 nothing is kept); the words of sample k are Philox
+// block (j, id, k).
+__device__ __forceinline__ int tern_keep(uint32_t word, float s, float a)
+{
+    return __fmul_rn(__fmul_rn((float)(word >> 8), 0x1p-24f), s) < a ? 1 : 0;
+}
 
 // Sum over `samples` stochastic ternarisations of g: code = sign(g) * (number of samples that keep the element), as
 // int8 (q), and / or as the two byte limbs of the same value as a 16-bit code (hi: 0 or -1, lo: the low byte), which
@@ -72,11 +75,11 @@ __global__ void __launch_bounds__(kTbpThreads) stc_ternarize_kernel(const float 
             const float xs[4] = {v.x, v.y, v.z, v.w};
             float p[4]; int cnt[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int e = 0; e < 4; ++e) p[e] = tern_prob(xs[e], s);
+            for (int e = 0; e < 4; ++e) p[e] = fabsf(xs[e]);
             for (int k = 0; k < samples; ++k) {
                 const uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), tensor_id, (uint32_t)k), keys);
-                cnt[0] += tern_keep(b.x, p[0]); cnt[1] += tern_keep(b.y, p[1]);
-                cnt[2] += tern_keep(b.z, p[2]); cnt[3] += tern_keep(b.w, p[3]);
+                cnt[0] += tern_keep(b.x, s, p[0]); cnt[1] += tern_keep(b.y, s, p[1]);
+                cnt[2] += tern_keep(b.z, s, p[2]); cnt[3] += tern_keep(b.w, s, p[3]);
             }
             uint32_t w8 = 0, whi = 0;
 #pragma unroll
@@ -93,13 +96,13 @@ __global__ void __launch_bounds__(kTbpThreads) stc_ternarize_kernel(const float 
     // elements the vector loop leaves (all of them when VEC == 1)
     const int64_t first = VEC == 4 ? (n >> 2) << 2 : 0;
     for (int64_t i = first + (int64_t)blockIdx.x * kTbpThreads + threadIdx.x; i < n; i += stride) {
-        const float p = tern_prob(g[i], s);
+        const float p = fabsf(g[i]);
         const int64_t j = i >> 2;
         int cnt = 0;
         for (int k = 0; k < samples; ++k) {
             const uint4 b = philox4x32_10(make_uint4((uint32_t)j, (uint32_t)((uint64_t)j >> 32), tensor_id, (uint32_t)k), keys);
             const uint32_t w[4] = {b.x, b.y, b.z, b.w};
-            cnt += tern_keep(w[i & 3], p);
+            cnt += tern_keep(w[i & 3], s, p);
         }
         const int c = g[i] > 0.0f ? cnt : -cnt;
         if (q) q[i] = (int8_t)c;
