@@ -708,6 +708,17 @@ def run_rangebn(args):
         del x, dy, y, dx, q
 
 
+def run_tbp(args):
+    """The low-bit variant's kernels (Appendix C) at the benchmark layer's size: one JSON line (see tbp_block)."""
+    import torch
+    from paper_1805_11046_b200 import binding as B
+    torch.cuda.set_device(0)
+    peaks, kind = measured_peaks()
+    out = tbp_block(B, args.batch, float(peaks["hbm_gbs"]), peaks)
+    out.update({"workload": "tbp_appendix_c", "peak_gbs": float(peaks["hbm_gbs"]), "peak_source": f"{kind} copy bandwidth"})
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -721,8 +732,9 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the dense-GEMM and Range BN sweep blocks of the line")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a captured CUDA graph of the step")
     ap.add_argument("--only-steps", action="store_true", help="run warmup+steps and exit (for captures under ncu)")
-    ap.add_argument("--workload", choices=["layer", "gemm", "rangebn"], default="layer",
-                    help="layer: the headline line; gemm / rangebn: side measurements of the dense sweep and the Range BN sweep")
+    ap.add_argument("--workload", choices=["layer", "gemm", "rangebn", "tbp"], default="layer",
+                    help="layer: the headline line; gemm / rangebn / tbp: side measurements of the dense sweep, the Range BN "
+                         "sweep and the low-bit variant's kernels (Appendix C)")
     ap.add_argument("--mnk", type=int, default=8192, help="--workload gemm: M = N = K")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.workload == "layer":
@@ -741,6 +753,8 @@ def main():
         run_gemm(args)
     elif args.workload == "rangebn":
         run_rangebn(args)
+    elif args.workload == "tbp":
+        run_tbp(args)
     else:
         run_ours(args)
 
