@@ -574,6 +574,28 @@ int qbp_tbp_weight_gradient(const qbp_conv_desc *d, int64_t rows, int64_t N, int
                             int8_t *t_hi, uint8_t *t_lo, qbp_qparams *qp_t,
                             int64_t *acc_out, float *gW, void *ws, size_t ws_bytes, void *stream);
 
+/* Bit rows and the literal XNOR + popcount products (Appendix C), for operands
+ * kept at one bit per element (an eighth of the bytes of the code tensors).
+ *
+ * qbp_pack_bits: codes [rows x cols] (int8, device) to bit rows: element c of
+ * a row is bit c % 32 of word c / 32 (1 for a code > 0; with mask != 0 for a
+ * code != 0: the non-zero plane of a ternary tensor, whose sign plane is the
+ * mask == 0 form); ceil(cols / 32) words per row, spare bits 0.
+ *
+ * qbp_xnor_gemm_bits: A_bits [M rows], B_bits [N rows] of K bits each;
+ * C [M x N] (int32) = K - 2 popcount(a xor b), the dot product of the +-1
+ * rows.  qbp_gated_xnor_gemm_bits: the same for a ternary left operand given
+ * as its non-zero and sign planes: C = popcount(nz & ~(sg xor b)) -
+ * popcount(nz & (sg xor b)).  Plain CUDA-core kernels bound by the popcount
+ * unit; the same integers as qbp_gemm_s8 on the byte codes, which is the
+ * faster route when the operands are bytes already.  M <= 4194240.  Allocate
+ * nothing. */
+int qbp_pack_bits(const int8_t *codes, int64_t rows, int64_t cols, int mask, uint32_t *words, void *stream);
+int qbp_xnor_gemm_bits(int64_t M, int64_t N, int64_t K, const uint32_t *A_bits, const uint32_t *B_bits,
+                       int32_t *C, void *stream);
+int qbp_gated_xnor_gemm_bits(int64_t M, int64_t N, int64_t K, const uint32_t *nz_bits,
+                             const uint32_t *sign_bits, const uint32_t *B_bits, int32_t *C, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

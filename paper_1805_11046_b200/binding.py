@@ -35,6 +35,7 @@ EXPORTS = (
     "qbp_layer_workspace_bytes", "qbp_layer_fwd", "qbp_layer_fwd_chained", "qbp_layer_bwd",
     "qbp_binarize_s8", "qbp_stc_ternarize_workspace_bytes", "qbp_stc_ternarize_s8",
     "qbp_tbp_weight_gradient_workspace_bytes", "qbp_tbp_weight_gradient",
+    "qbp_pack_bits", "qbp_xnor_gemm_bits", "qbp_gated_xnor_gemm_bits",
 )
 
 
@@ -373,6 +374,28 @@ def qbp_tbp_weight_gradient(a_codes, qa, g, samples, seed=0, tensor_id=0, d: Con
                                        int(samples), C.c_uint64(seed), C.c_uint32(tensor_id), _ptr(t_hi), _ptr(t_lo), _ptr(qp_t),
                                        _ptr(acc), _ptr(gW), _ptr(ws), C.c_size_t(ws.numel()), _stream()))
     return acc, gW, t_hi, t_lo, qp_t
+
+
+def qbp_pack_bits(codes, mask=False, words=None):
+    rows, cols = codes.shape
+    if words is None: words = torch.empty((rows, (cols + 31) // 32), dtype=torch.int32, device=codes.device)
+    _check(lib.qbp_pack_bits(_ptr(codes), C.c_int64(rows), C.c_int64(cols), int(mask), _ptr(words), _stream()))
+    return words
+
+
+def qbp_xnor_gemm_bits(A_bits, B_bits, K, out=None):
+    M, N = A_bits.shape[0], B_bits.shape[0]
+    if out is None: out = torch.empty((M, N), dtype=torch.int32, device=A_bits.device)
+    _check(lib.qbp_xnor_gemm_bits(C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A_bits), _ptr(B_bits), _ptr(out), _stream()))
+    return out
+
+
+def qbp_gated_xnor_gemm_bits(nz_bits, sign_bits, B_bits, K, out=None):
+    M, N = nz_bits.shape[0], B_bits.shape[0]
+    if out is None: out = torch.empty((M, N), dtype=torch.int32, device=nz_bits.device)
+    _check(lib.qbp_gated_xnor_gemm_bits(C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(nz_bits), _ptr(sign_bits), _ptr(B_bits),
+                                        _ptr(out), _stream()))
+    return out
 
 
 # ------------------------------------------------------------------- Range BN

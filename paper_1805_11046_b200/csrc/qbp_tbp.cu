@@ -135,9 +135,123 @@ static int stc_ternarize_impl(const float *g, int64_t n, int samples, uint64_t s
     return QBP_OK;
 }
 
+// ---------------------------------------------------------------- bit rows and the literal XNOR + popcount products
+// [rows x cols] codes to bit rows: element c of a row is bit c % 32 of word c / 32 (1 for a code > 0, or for a code
+// != 0 with `mask`), ceil(cols / 32) words per row, spare bits 0.  One warp per word (a ballot).
+__global__ void __launch_bounds__(256) pack_bits_kernel(const int8_t *__restrict__ codes, int64_t rows, int64_t cols, int mask,
+                                                        uint32_t *__restrict__ words)
+{
+    const int64_t wpr = (cols + 31) / 32;
+    const int lane = threadIdx.x & 31;
+    for (int64_t word = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); word < rows * wpr; word += (int64_t)gridDim.x * 8) {
+        const int64_t r = word / wpr, c = (word - r * wpr) * 32 + lane;
+        const int v = c < cols ? (int)codes[r * cols + c] : 0;
+        const uint32_t bits = __ballot_sync(0xffffffffu, mask ? v != 0 : v > 0);
+        if (lane == 0) words[word] = bits;
+    }
+}
+
+// C [M x N] from bit rows of K bits (wpr words each): 64 x 64 outputs per block, 4 x 4 per thread, 32 words of every
+// row staged in shared memory per step (rows padded to 33 words: the threads of a warp read 16 different banks).
+//   plain:  C = K - 2 popcount(a xor b)                                   (the +-1 dot product, Appendix C)
+//   GATED:  C = popcount(nz & ~(sg xor b)) - popcount(nz & (sg xor b))    (ternary a as non-zero and sign planes)
+// The popcount unit retires 16 results per clock and SM, which bounds this form at about 0.15 P bit-products/s; the
+// products of the layer path run on the int8 tensor cores instead (qbp_gemm_s8 on +-1 bytes).  This kernel is the
+// form for operands kept as bit rows (an eighth of the bytes).
+template <bool GATED>
+__global__ void __launch_bounds__(256) xnor_gemm_bits_kernel(int M, int N, int K, int wpr, const uint32_t *__restrict__ A,
+                                                             const uint32_t *__restrict__ S, const uint32_t *__restrict__ B,
+                                                             int32_t *__restrict__ C)
+{
+    __shared__ uint32_t sA[64][33], sB[64][33], sS[GATED ? 64 : 1][33];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    int acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0;
+    for (int w0 = 0; w0 < wpr; w0 += 32) {
+        // (thread t: word t % 32 of rows t / 32, t / 32 + 8, ...: 128-byte segments)
+        const int lw = threadIdx.x & 31, w = w0 + lw;
+#pragma unroll
+        for (int r = threadIdx.x >> 5; r < 64; r += 8) {
+            const bool in_a = m0 + r < M && w < wpr, in_b = n0 + r < N && w < wpr;
+            sA[r][lw] = in_a ? A[(int64_t)(m0 + r) * wpr + w] : 0u;
+            if (GATED) sS[r][lw] = in_a ? S[(int64_t)(m0 + r) * wpr + w] : 0u;
+            sB[r][lw] = in_b ? B[(int64_t)(n0 + r) * wpr + w] : 0u;
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int k = 0; k < 32; ++k) {
+            uint32_t a[4], sg[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = sA[ty + 16 * i][k]; sg[i] = GATED ? sS[ty + 16 * i][k] : 0u; b[i] = sB[tx + 16 * i][k]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (GATED) { const uint32_t d = sg[i] ^ b[j]; acc[i][j] += __popc(a[i] & ~d) - __popc(a[i] & d); }
+                    else acc[i][j] += __popc(a[i] ^ b[j]);
+                }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int m = m0 + ty + 16 * i, n = n0 + tx + 16 * j;
+            if (m < M && n < N) C[(int64_t)m * N + n] = GATED ? acc[i][j] : K - 2 * acc[i][j];
+        }
+}
+
+static int xnor_bits_launch(bool gated, int64_t M, int64_t N, int64_t K, const uint32_t *A, const uint32_t *S, const uint32_t *B,
+                            int32_t *C, cudaStream_t st)
+{
+    if (M <= 0 || N <= 0 || K <= 0 || M > INT32_MAX || N > INT32_MAX || K > INT32_MAX)
+        return fail(QBP_ERR_INVALID_ARG, "xnor_gemm_bits: M, N, K must be positive and fit int32");
+    if (!A || !B || !C || (gated && !S)) return fail(QBP_ERR_INVALID_ARG, "xnor_gemm_bits: NULL argument");
+    if ((N + 63) / 64 > 2147483647ll || (M + 63) / 64 > 65535) return fail(QBP_ERR_UNSUPPORTED_SHAPE, "xnor_gemm_bits: at most 4 M rows");
+    const dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64));
+    const int wpr = (int)((K + 31) / 32);
+    QBP_TRACE_BEGIN(st);
+    if (gated) xnor_gemm_bits_kernel<true><<<grid, 256, 0, st>>>((int)M, (int)N, (int)K, wpr, A, S, B, C);
+    else       xnor_gemm_bits_kernel<false><<<grid, 256, 0, st>>>((int)M, (int)N, (int)K, wpr, A, nullptr, B, C);
+    QBP_LAUNCH_OK("xnor_gemm_bits_kernel");
+    return QBP_OK;
+}
+
 }  // namespace qbp
 
 using namespace qbp;
+
+extern "C" __attribute__((visibility("default"))) int qbp_pack_bits(const int8_t *codes, int64_t rows, int64_t cols, int mask, uint32_t *words, void *stream)
+{
+    cudaStream_t st = (cudaStream_t)stream;
+    if (rows < 0 || cols <= 0) return fail(QBP_ERR_INVALID_ARG, "pack_bits: rows must be >= 0 and cols > 0");
+    if (rows == 0) return QBP_OK;
+    if (!codes || !words) return fail(QBP_ERR_INVALID_ARG, "pack_bits: NULL argument");
+    const int64_t total = rows * ((cols + 31) / 32);
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((total + 7) / 8, (int64_t)sm_count() * 16));
+    QBP_TRACE_BEGIN(st);
+    pack_bits_kernel<<<grid, 256, 0, st>>>(codes, rows, cols, mask, words);
+    QBP_LAUNCH_OK("pack_bits_kernel");
+    return QBP_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_xnor_gemm_bits(int64_t M, int64_t N, int64_t K, const uint32_t *A_bits, const uint32_t *B_bits,
+                                                                         int32_t *C, void *stream)
+{
+    return xnor_bits_launch(false, M, N, K, A_bits, nullptr, B_bits, C, (cudaStream_t)stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int qbp_gated_xnor_gemm_bits(int64_t M, int64_t N, int64_t K, const uint32_t *nz_bits,
+                                                                               const uint32_t *sign_bits, const uint32_t *B_bits, int32_t *C,
+                                                                               void *stream)
+{
+    return xnor_bits_launch(true, M, N, K, nz_bits, sign_bits, B_bits, C, (cudaStream_t)stream);
+}
 
 extern "C" __attribute__((visibility("default"))) int qbp_binarize_s8(const float *x, int64_t n, int8_t *q, qbp_qparams *qp_out, void *stream)
 {

@@ -126,6 +126,22 @@ def test_bifurcate_and_code_sums(B):
     assert np.array_equal(to_host(cols), on.q.astype(np.int64).sum(0))
 
 
+@pytest.mark.parametrize("rows,cols", [(130, 128), (77, 256), (300, 512), (33, 2048), (9, 96), (5, 4096)])
+def test_row_sums_of_rows_of_any_width(B, rows, cols):
+    """Row sums taken inside the quantising kernel (power-of-two rows up to 128 elements) or by the pass over the codes
+    (other widths): the same sums, nearest and stochastic."""
+    import torch
+    g = synth.normal((rows, cols), 14, std=0.5)
+    rs = torch.full((rows,), 12345, dtype=torch.int32, device="cuda")
+    q, _ = B.qbp_quantize_s8(to_dev(g), row_sums=rs)
+    on = O.quantize(g, 8)
+    assert np.array_equal(to_host(q), on.q) and np.array_equal(to_host(rs), on.q.astype(np.int32).sum(1))
+    rs.fill_(-7)
+    q8, qp8, hi, lo, qp16 = B.qbp_bifurcate(to_dev(g), 3, 1, 2, row_sums8=rs)
+    o8 = O.quantize(g, 8, rounding=1, seed=3, tensor_id=1)
+    assert np.array_equal(to_host(q8), o8.q) and np.array_equal(to_host(rs), o8.q.astype(np.int32).sum(1))
+
+
 def test_full_size_activation_tensor(B):
     """The 51.4M-element conv2_x activation, nearest and stochastic, every code."""
     x = synth.relu_normal((256, 56, 56, 64), 10)

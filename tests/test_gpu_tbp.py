@@ -6,7 +6,7 @@ import pytest
 
 from oracle import qbp_oracle as O
 from paper_1805_11046_b200 import synth
-from tests.util import to_dev, to_host
+from tests.util import set_qparams, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -131,3 +131,29 @@ def test_algorithm_1_convolution(B, N, H, W, C, K, R, samples):
         want += oacc.reshape(want.shape)
     assert np.array_equal(to_host(acc), want)
     assert np.array_equal(to_host(gW), want.astype(np.float32) * (np.float32(s) / np.float32(samples)))
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 1), (3, 35), (64, 64), (130, 257), (7, 4096)])
+def test_bit_rows(B, rows, cols):
+    t = np.random.Generator(np.random.PCG64(50 + cols)).integers(-1, 2, (rows, cols)).astype(np.int8)
+    assert np.array_equal(to_host(B.qbp_pack_bits(to_dev(t))).view(np.uint32), O.pack_bits(t))
+    assert np.array_equal(to_host(B.qbp_pack_bits(to_dev(t), mask=True)).view(np.uint32), O.pack_bits(t, mask=True))
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (5, 7, 70), (64, 64, 1024), (130, 67, 1057), (256, 300, 4096)])
+def test_popcount_products_on_bit_rows(B, M, N, K):
+    """The literal XNOR + popcount and gated-XNOR products on bit rows (ragged sizes) against the oracle's, and against
+    the tensor-core route on the byte codes where its shape rules allow."""
+    rng = np.random.Generator(np.random.PCG64(60 + K))
+    a = (rng.integers(0, 2, (M, K)) * 2 - 1).astype(np.int8); b = (rng.integers(0, 2, (N, K)) * 2 - 1).astype(np.int8)
+    t = rng.integers(-1, 2, (M, K)).astype(np.int8)
+    ab, bb = B.qbp_pack_bits(to_dev(a)), B.qbp_pack_bits(to_dev(b))
+    got = to_host(B.qbp_xnor_gemm_bits(ab, bb, K))
+    assert np.array_equal(got, O.xnor_gemm(O.pack_bits(a), O.pack_bits(b), K))
+    nz, sg = B.qbp_pack_bits(to_dev(t), mask=True), B.qbp_pack_bits(to_dev(t))
+    gated = to_host(B.qbp_gated_xnor_gemm_bits(nz, sg, bb, K))
+    assert np.array_equal(gated, O.gated_xnor_gemm(O.pack_bits(t, mask=True), O.pack_bits(t), O.pack_bits(b), K))
+    if M % 16 == 0 and N % 16 == 0 and K % 16 == 0:
+        one = set_qparams(B.new_qparams(1), 1.0, 0)
+        acc, _, _ = B.qbp_gemm_s8(to_dev(a), one, to_dev(b), one, transB=True, want_acc=True)
+        assert np.array_equal(to_host(acc), got)
