@@ -514,7 +514,13 @@ def tbp_block(B, batch, hbm_peak, peaks, launches=30):
                                 "int8_tops": round(2 * n ** 3 / (ms * 1e-3) / 1e12, 1),
                                 "frac_of_measured_burst": round(2 * n ** 3 / (ms * 1e-3) / 1e12 / (2 * float(peaks["bf16_tflops"])), 3),
                                 "includes": "the two code-sum kernels and the terms kernel of the call"}
-    del qa, qb, o, wsg, case
+    # the same product from bit rows on the popcount unit of the CUDA cores
+    ab, bb = B.qbp_pack_bits(qa), B.qbp_pack_bits(qb.t().contiguous())
+    oc = torch.empty((n, n), dtype=torch.int32, device="cuda")
+    msb = _graph_ms_per_call([lambda: B.qbp_xnor_gemm_bits(ab, bb, n, out=oc)], 5)
+    out["xnor_forward_4096_popcount_on_bit_rows"] = {"ms": round(msb, 4), "tera_bit_macs_per_s": round(n ** 3 / (msb * 1e-3) / 1e12, 1),
+                                                     "tensor_core_route_speedup": round(msb / ms, 2)}
+    del qa, qb, o, wsg, case, ab, bb, oc
     # Algorithm 1 for the benchmark layer: 6 samples
     import ctypes
     c = cfg["conv"]
