@@ -146,3 +146,40 @@ class QuantizedStack:
 
     def status(self) -> int:
         return min(L.status() for L in self.layers)
+
+
+class TernarizedLayer:
+    """The low-bit form of the quantised layer (Appendix C, Ternarized Back-Propagation): 1-bit weights and activations,
+    a ternary gradient for the layer-gradient product, and Algorithm 1 (the mean over `samples` ternarisations) for the
+    weight gradient; Range BN after the product as in the 8-bit layer.  Call order and buffers only: binarise x and w
+    -> product (the +-1 dot product of XNOR + popcount, on the int8 tensor cores) -> Range BN; backwards Range BN ->
+    ternarise the gradient -> layer-gradient product; ternarise `samples` times -> weight-gradient product."""
+
+    def __init__(self, conv=None, relu=False, seed=0, tensor_id=1, samples=1):
+        self.conv, self.relu, self.seed, self.tensor_id, self.samples = conv, relu, seed, tensor_id, samples
+        self.saved = None
+
+    def forward(self, x, w, gamma=None, beta=None):
+        a, qa = B.qbp_binarize_s8(x)
+        wb, qw = B.qbp_binarize_s8(w)
+        if self.conv is not None:
+            _, z, _ = B.qbp_conv_s8_implicit(B.QBP_CONV_FPROP, self.conv, a, qa, wb, qw)
+        else:
+            _, z, _ = B.qbp_gemm_s8(a, qa, wb, qw)                     # x [batch x in] . w [in x out]
+        y, mean, vmin, vmax, _ = B.qbp_rangebn_fwd(z, gamma, beta, relu=self.relu)
+        self.saved = dict(a=a, qa=qa, wb=wb, qw=qw, z=z, mean=mean, vmin=vmin, vmax=vmax, gamma=gamma, beta=beta)
+        return y
+
+    def backward(self, dy):
+        s = self.saved
+        g, dgamma, dbeta = B.qbp_rangebn_bwd(dy, s["z"], s["mean"], s["vmin"], s["vmax"], s["gamma"], s["beta"], relu=self.relu)
+        # sample 0 of the gradient's stream serves the layer gradient; the weight gradient draws its own samples
+        t, qt = B.qbp_stc_ternarize_s8(g, samples=1, seed=self.seed, tensor_id=self.tensor_id)
+        if self.conv is not None:
+            _, dx, _ = B.qbp_conv_s8_implicit(B.QBP_CONV_DGRAD, self.conv, t, qt, s["wb"], s["qw"])
+        else:
+            _, dx, _ = B.qbp_gemm_s8(t, qt, s["wb"], s["qw"], transB=True)
+        _, dw, _, _, _ = B.qbp_tbp_weight_gradient(s["a"], s["qa"], g, self.samples, seed=self.seed, tensor_id=self.tensor_id + 1,
+                                                   d=self.conv)
+        self.g, self.t, self.qt = g, t, qt
+        return dx, dw, dgamma, dbeta

@@ -157,3 +157,58 @@ def test_popcount_products_on_bit_rows(B, M, N, K):
         one = set_qparams(B.new_qparams(1), 1.0, 0)
         acc, _, _ = B.qbp_gemm_s8(to_dev(a), one, to_dev(b), one, transB=True, want_acc=True)
         assert np.array_equal(to_host(acc), got)
+
+
+@pytest.mark.parametrize("kind,samples", [("conv", 1), ("conv", 4), ("linear", 3)])
+def test_ternarized_layer_stagewise(B, kind, samples):
+    """The low-bit layer (1-bit x and w, Range BN, ternary gradient, Algorithm 1) stage by stage against the oracle."""
+    from paper_1805_11046_b200 import layer
+    from tests.util import FP32_TOL, rel_err
+    relu = True
+    if kind == "conv":
+        N, H, W, C, K, R = 2, 8, 8, 32, 64, 3
+        d = B.conv_desc(N, H, W, C, K, R, R, 1, 1); od = O.conv_desc(N, H, W, C, K, R, R, 1, 1)
+        x = synth.normal((N, H, W, C), 80); w = synth.normal((K, R, R, C), 81); dy = synth.normal((N, H, W, K), 82, std=0.1)
+    else:
+        d = od = None
+        x = synth.normal((64, 128), 80); w = synth.normal((128, 64), 81); dy = synth.normal((64, 64), 82, std=0.1)
+        K = 64
+    gamma = synth.normal((K,), 83) * np.float32(0.5) + np.float32(1); beta = synth.normal((K,), 84) * np.float32(0.1)
+    L = layer.TernarizedLayer(conv=d, relu=relu, seed=9, tensor_id=5, samples=samples)
+    y = L.forward(to_dev(x), to_dev(w), to_dev(gamma), to_dev(beta))
+    dx, dw, dgamma, dbeta = L.backward(to_dev(dy))
+    ab, wb = O.binarize(x), O.binarize(w)
+    assert np.array_equal(to_host(L.saved["a"]), ab) and np.array_equal(to_host(L.saved["wb"]), wb)
+    if od is not None:
+        _, oz, bad = O.conv_s8(0, od, ab, 0, wb, 0, 1.0, 1.0)
+    else:
+        _, oz, bad = O.gemm_s8(ab, 0, wb, 0, 1.0, 1.0)
+    z = to_host(L.saved["z"])
+    assert bad == 0 and np.array_equal(z.ravel(), np.asarray(oz).ravel())
+    z2 = z.reshape(-1, K); dy2 = dy.reshape(-1, K)
+    oy, om, olo, ohi = O.rangebn_fwd(z2, gamma, beta, relu=relu)
+    assert rel_err(to_host(y).reshape(-1, K), oy)[0] <= FP32_TOL
+    mean, vmin, vmax = (to_host(L.saved[k]) for k in ("mean", "vmin", "vmax"))
+    og, odg, odb = O.rangebn_bwd(dy2, z2, mean, vmin, vmax, gamma, beta, relu=relu)
+    g = to_host(L.g)
+    assert rel_err(g.reshape(-1, K), og)[0] <= FP32_TOL
+    assert rel_err(to_host(dgamma), odg)[0] <= FP32_TOL and rel_err(to_host(dbeta), odb)[0] <= FP32_TOL
+    ot, s = O.stc_tern(g, 9, 5, 0)
+    assert np.array_equal(to_host(L.t), ot)
+    if od is not None:
+        _, odx, bad = O.conv_s8(1, od, ot, 0, wb, 0, float(s), 1.0)
+        assert bad == 0 and np.array_equal(to_host(dx).ravel(), np.asarray(odx).ravel())
+        want = np.zeros(w.shape, dtype=np.int64)
+        for k in range(samples):
+            tk, s2 = O.stc_tern(g, 9, 6, k)
+            oacc, _ = O.conv_wgrad_s16(od, ab, 0, tk.astype(np.int16), 0, 1.0, 1.0)
+            want += np.asarray(oacc).reshape(want.shape)
+    else:
+        _, odx, bad = O.gemm_s8(ot, 0, wb, 0, float(s), 1.0, transB=True)
+        assert bad == 0 and np.array_equal(to_host(dx), odx)
+        tot = np.zeros(g.shape, dtype=np.int64)
+        for k in range(samples):
+            tk, s2 = O.stc_tern(g, 9, 6, k)
+            tot += tk
+        want = ab.astype(np.int64).T @ tot
+    assert np.array_equal(to_host(dw), want.astype(np.float32) * (np.float32(s2) / np.float32(samples)))
