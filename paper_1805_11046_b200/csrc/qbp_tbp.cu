@@ -295,6 +295,13 @@ extern "C" __attribute__((visibility("default"))) int qbp_tbp_weight_gradient(co
     if (d) { rows = (int64_t)d->N * d->H * d->W; N = d->K; K = d->C; }
     if (rows <= 0 || N <= 0 || K <= 0) return fail(QBP_ERR_INVALID_ARG, "tbp_weight_gradient: sizes must be positive");
     if (!a_codes || !qa || !g || !t_hi || !t_lo || !qp_t) return fail(QBP_ERR_INVALID_ARG, "tbp_weight_gradient: NULL argument");
+    // (everything the product would refuse is refused here, before the ternariser is launched)
+    if (d ? !wgrad_conv_supported(d) : (N % 16 != 0 || K % 16 != 0))
+        return fail(QBP_ERR_UNSUPPORTED_SHAPE, "tbp_weight_gradient: shape outside what qbp_wgrad_s16 takes");
+    if (!aligned16(a_codes) || !aligned16(t_hi) || !aligned16(t_lo) || ((uintptr_t)g & 3) != 0)
+        return fail(QBP_ERR_INVALID_ARG, "tbp_weight_gradient: a_codes, t_hi, t_lo must be 16-byte aligned, g 4-byte aligned");
+    if (!acc_out && !gW) return fail(QBP_ERR_INVALID_ARG, "tbp_weight_gradient: acc_out and gW are both NULL");
+    if (samples < 1 || samples > 127) return fail(QBP_ERR_INVALID_ARG, "tbp_weight_gradient: needs 1 <= samples <= 127");
     const size_t head = align_up(tern_ws_bytes(), 256);
     const size_t need = qbp_tbp_weight_gradient_workspace_bytes(d, rows, N, K);
     if (!ws || ws_bytes < need) return fail(QBP_ERR_WORKSPACE, "tbp_weight_gradient: workspace of %zu bytes needed, %zu given", need, ws_bytes);

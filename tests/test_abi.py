@@ -117,3 +117,22 @@ def test_workspace_queries_are_pure(lib):
         C.c_int64(10), C.c_int64(64), 0)
     assert lib.qbp_gemm_s8_workspace_bytes(C.c_int64(4096), C.c_int64(4096), C.c_int64(4096)) >= 4096 * 12
     assert lib.qbp_rangebn_workspace_bytes(C.c_int64(1000), C.c_int64(64)) > 0
+
+
+def test_host_side_refusals_of_the_low_bit_entry_points(lib):
+    i64 = C.c_int64
+    null = C.c_void_p(0)
+    fake = C.c_void_p(4096)            # never dereferenced: validation fails first
+    big = C.c_size_t(1 << 30)
+    assert lib.qbp_binarize_s8(null, i64(8), fake, null, null) == -1
+    assert lib.qbp_stc_ternarize_s8(fake, i64(8), 0, C.c_uint64(0), 0, fake, fake, fake, big, null) == -1        # samples < 1
+    assert lib.qbp_stc_ternarize_s8(fake, i64(8), 128, C.c_uint64(0), 0, fake, fake, fake, big, null) == -1      # samples > 127
+    assert lib.qbp_stc_ternarize_s8(fake, i64(8), 1, C.c_uint64(0), 0, fake, fake, fake, C.c_size_t(16), null) == -4
+    # Algorithm 1: what the weight-gradient product would refuse is refused before the ternariser runs
+    assert lib.qbp_tbp_weight_gradient(null, i64(64), i64(24), i64(32), fake, fake, fake, 1, C.c_uint64(0), 0, fake, fake, fake,
+                                       null, fake, fake, big, null) == -2
+    assert lib.qbp_tbp_weight_gradient(null, i64(64), i64(32), i64(32), fake, fake, fake, 1, C.c_uint64(0), 0, fake, fake, fake,
+                                       null, null, fake, big, null) == -1                                      # no output wanted
+    assert lib.qbp_pack_bits(fake, i64(1), i64(0), 0, fake, null) == -1
+    assert lib.qbp_xnor_gemm_bits(i64(0), i64(1), i64(1), fake, fake, fake, null) == -1
+    assert lib.qbp_gated_xnor_gemm_bits(i64(1), i64(1), i64(1), fake, null, fake, fake, null) == -1
