@@ -20,6 +20,23 @@ def test_binarize_sign_convention_and_bit_order():
     assert O.pack_bits(tern, mask=True).tolist() == [[2, 2]] and O.pack_bits(tern).tolist() == [[0, 2]]
 
 
+def test_binarised_gaussian_vector_keeps_the_papers_angle():
+    """The paper's supplement prints the angle between a Gaussian vector and its sign binarisation: arccos sqrt(2 / pi),
+    about 37 degrees (tests/golden/paper_constants.txt)."""
+    import math
+    from pathlib import Path
+    val = tol = None
+    for line in (Path(__file__).parent / "golden" / "paper_constants.txt").read_text().splitlines():
+        f = line.split("#")[0].split()
+        if len(f) == 3 and f[0] == "binary_quantization_angle_degrees":
+            val, tol = float(f[1]), float(f[2])
+    x = np.random.Generator(np.random.PCG64(3)).normal(0, 1, 200000).astype(np.float32)
+    b = O.binarize(x).astype(np.float64)
+    cos = float(x.astype(np.float64) @ b) / (np.linalg.norm(x.astype(np.float64)) * np.linalg.norm(b))
+    angle = math.degrees(math.acos(cos))
+    assert abs(angle - val) <= tol and abs(angle - math.degrees(math.acos(math.sqrt(2 / math.pi)))) < 0.2
+
+
 def test_xnor_popcount_product_is_the_plus_minus_one_dot_product():
     for M, N, K in ((5, 7, 70), (3, 4, 32), (2, 2, 1), (6, 5, 257)):
         A = _pm1((M, K), 1 + K); B = _pm1((N, K), 2 + K)
