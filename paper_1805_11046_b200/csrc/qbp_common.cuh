@@ -201,6 +201,28 @@ __device__ __forceinline__ float bn_dx(float d, float ind, float s, float g, flo
 // Floats as integers that compare the same way (and back): for atomic minima and maxima of floats.
 __device__ __forceinline__ int float_order(float f) { const int b = __float_as_int(f); return b ^ ((b >> 31) & 0x7fffffff); }
 __device__ __forceinline__ float order_float(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+__device__ __forceinline__ float bn_scale(float lo, float hi, float Cn);
+// The rectifier's mask of a Range BN output as a threshold on the input.  y(x) = bn_y(bn_xhat(x, mu, s), g, b) is a
+// monotone function of x (every operation is rounded on its own and monotone, s >= 0): rising for g >= 0, falling for
+// g < 0, so {x : y(x) > 0} is a ray, and its end is found by bisection over the floats in their order (33 evaluations
+// of y).  Returns (t, sgn) with  y(x) > 0  <=>  sgn * x >= t  for finite x (sgn = +-1; t = +-inf: none / all).
+__device__ inline float2 relu_threshold(float mu, float s, float g, float b)
+{
+    const bool rising = !(g < 0.0f);
+    long long lo = float_order(-3.402823466e38f), hi = float_order(3.402823466e38f);
+    auto on = [&](long long k) { return bn_y(bn_xhat(order_float((int)k), mu, s), g, b) > 0.0f; };
+    const float sgn = rising ? 1.0f : -1.0f;
+    // (towards `far` the output rises: the ray is [threshold, far])
+    const bool at_far = on(rising ? hi : lo), at_near = on(rising ? lo : hi);
+    if (!at_far) return make_float2(INFINITY, sgn);
+    if (at_near) return make_float2(-INFINITY, sgn);
+    if (rising) {                       // smallest key that is on
+        while (hi - lo > 1) { const long long mid = lo + (hi - lo) / 2; if (on(mid)) hi = mid; else lo = mid; }
+        return make_float2(order_float((int)hi), 1.0f);
+    }
+    while (hi - lo > 1) { const long long mid = lo + (hi - lo) / 2; if (on(mid)) lo = mid; else hi = mid; }   // largest key that is on
+    return make_float2(-order_float((int)lo), -1.0f);
+}
 __device__ __forceinline__ float bn_scale(float lo, float hi, float Cn)
 {
     float r = __fsub_rn(hi, lo);

@@ -387,7 +387,10 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
                                                               const float *__restrict__ ext = nullptr,
                                                               const float *__restrict__ vmin = nullptr,
                                                               const float *__restrict__ vmax = nullptr, float Cn_f = 0.0f,
-                                                              float2 *__restrict__ chan_range = nullptr)
+                                                              float2 *__restrict__ chan_range = nullptr,
+                                                              const float *__restrict__ mean = nullptr,
+                                                              const float *__restrict__ beta = nullptr,
+                                                              float2 *__restrict__ relu_thr = nullptr)
 {
     const int c = blockIdx.x;
     double a = 0.0, b = 0.0;
@@ -448,6 +451,8 @@ __global__ void __launch_bounds__(128) bn_bwd_finalize_kernel(const double *__re
                 }
             }
             chan_range[c] = make_float2(rlo, rhi);
+            // (the rectifier's mask of this channel as a threshold on x, for the pass that follows)
+            if (relu_thr) relu_thr[c] = relu_threshold(mean[c], s, gf, beta ? beta[c] : 0.0f);
         }
     }
 }
@@ -475,24 +480,25 @@ __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel
     const float *__restrict__ beta, float Cn, const float2 *__restrict__ coef, float *__restrict__ g_out,
     const qbp_qparams *__restrict__ qp8, const qbp_qparams *__restrict__ qp16, uint32_t id8, uint32_t id16,
     const __grid_constant__ PhiloxKeys keys, uint32_t *__restrict__ q8, uint32_t *__restrict__ q_hi, uint32_t *__restrict__ q_lo,
-    uint32_t lo_flip, int32_t *__restrict__ rowsum8, unsigned long long *__restrict__ chansum16)
+    uint32_t lo_flip, int32_t *__restrict__ rowsum8, unsigned long long *__restrict__ chansum16,
+    const float2 *__restrict__ relu_thr)
 {
     const bool rowsum_pieces = tw > 32 || gridDim.y > 1;
     const ScanPos p = scan_pos<4>(C, tw);
     uint32_t cs16[4] = {0u, 0u, 0u, 0u};          // unsigned codes of this thread's rows (fewer than 65536 rows)
     int mine = 0;
     const int rpb = kScanThreads / tw;
-    float mu[4], s[4], g[4], b[4], lo[4], hi[4], m1[4], k2[4];
+    float s[4], g[4], lo[4], hi[4], m1[4], k2[4], thr[4], tsg[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const int c = p.active ? p.col + e : 0;
-        mu[e] = mean[c];
         lo[e] = vmin[c]; hi[e] = vmax[c];
         s[e] = bn_scale(lo[e], hi[e], Cn);
         g[e] = gamma ? gamma[c] : 1.0f;
-        b[e] = beta ? beta[c] : 0.0f;
         const float2 cf = coef[c];
         m1[e] = cf.x; k2[e] = cf.y;
+        const float2 th = RELU ? relu_thr[c] : make_float2(0.0f, 1.0f);   // (the mask y > 0 as sgn * x >= threshold)
+        thr[e] = th.x; tsg[e] = th.y;
     }
     // both codes in fixed point with 16 fraction bits (quantize_sr8_byte2 / quantize_sr16_top_half)
     const float inv8 = __fdiv_rn(1.0f, qp8->scale) * 65536.0f, zp8 = (float)(qp8->zero_point + 128) * 65536.0f;
@@ -536,7 +542,7 @@ __global__ void __launch_bounds__(kScanThreads, 3) bn_bwd_apply_bifurcate_kernel
                 for (int e = 0; e < 4; ++e) {
                     const float xv = ax[e];
                     float d = ad[e];
-                    if (RELU && !(bn_y(bn_xhat(xv, mu[e], s[e]), g[e], b[e]) > 0.0f)) d = 0.0f;
+                    if (RELU && !(__fmul_rn(tsg[e], xv) >= thr[e])) d = 0.0f;
                     const float ind = (xv == hi[e] ? 1.0f : 0.0f) - (xv == lo[e] ? 1.0f : 0.0f);
                     v[e] = bn_dx(d, ind, s[e], g[e], m1[e], k2[e]);
                 }
@@ -681,7 +687,7 @@ static size_t bn_ws_bytes(int64_t C)
     size_t per = (size_t)kScanMaxStrips * (size_t)C;
     return 2 * align_up(per * sizeof(double), 256) + 2 * align_up(per * sizeof(float), 256) +
            align_up((size_t)C * sizeof(float2), 256) + 256 + align_up(6 * per * sizeof(float), 256) +
-           align_up((size_t)C * sizeof(float2), 256);
+           2 * align_up((size_t)C * sizeof(float2), 256);
 }
 
 static int check_bn(const char *who, const void *a, const void *b, int64_t n, int64_t C, const void *ws, size_t ws_bytes)
@@ -893,7 +899,7 @@ static int bn_bwd_stats_launch(const float *dy, const float *x, int64_t n_rows, 
                                const float *beta, int relu, const float *save_mean, const float *save_min,
                                const float *save_max, float *dgamma, float *dbeta, float2 *coef, double *sum_dy,
                                double *sum_dyx, double *pa, double *pb, cudaStream_t st, float *ext = nullptr,
-                               float2 *chan_range = nullptr)
+                               float2 *chan_range = nullptr, float2 *relu_thr = nullptr)
 {
     const bool al = aligned16(x) && aligned16(dy);
     const bool v4 = al && C % 4 == 0;
@@ -915,7 +921,7 @@ static int bn_bwd_stats_launch(const float *dy, const float *x, int64_t n_rows, 
     QBP_LAUNCH_OK("bn_bwd_stats_kernel");
     QBP_TRACE_BEGIN(st);
     bn_bwd_finalize_kernel<<<(int)C, 128, 0, st>>>(pa, pb, g.nbx, (int)C, n_stat, gamma, Cnd, dgamma, dbeta, coef, sum_dy, sum_dyx,
-                                                   ext, save_min, save_max, Cn, chan_range);
+                                                   ext, save_min, save_max, Cn, chan_range, save_mean, beta, relu_thr);
     QBP_LAUNCH_OK("bn_bwd_finalize_kernel");
     return QBP_OK;
 }
@@ -977,8 +983,9 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
     w.take<char>(256);
     float *ext = w.take<float>(6 * (size_t)kScanMaxStrips * C);
     float2 *chan_range = w.take<float2>((size_t)C);
+    float2 *relu_thr = w.take<float2>((size_t)C);
     if ((rc = bn_bwd_stats_launch(dy, x, n, n, C, gamma, beta, relu, save_mean, save_min, save_max, dgamma, dbeta, coef, nullptr,
-                                  nullptr, pa, pb, st, ext, chan_range)))
+                                  nullptr, pa, pb, st, ext, chan_range, relu ? relu_thr : nullptr)))
         return rc;
     if ((rc = launch_range_finalize(chan_range, (int)C, qp8, qp16, st, after_range))) return rc;
     if (tot16) QBP_CUDA_OK(cudaMemsetAsync(tot16, 0, sizeof(int64_t) * (size_t)C, st));
@@ -993,7 +1000,7 @@ int rangebn_bwd_bifurcate_impl(const float *dy, const float *x, int64_t n, int64
     int32_t *row_sums_arg = row_sums8;
     if (row_sums8 && (ga.tw > 32 || ga.slabs > 1)) QBP_CUDA_OK(cudaMemsetAsync(row_sums8, 0, sizeof(int32_t) * (size_t)n, st));
     QBP_TRACE_BEGIN(st);
-#define QBP_BN_BAB(R, G, T) do { static PerDeviceOnce once_; QBP_SMEM_OPT_IN(once_, (bn_bwd_apply_bifurcate_kernel<R, G, T>), kBabRingBytes); bn_bwd_apply_bifurcate_kernel<R, G, T><<<grid, kScanThreads, kBabRingBytes, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg, reinterpret_cast<unsigned long long *>(tot16)); } while (0)
+#define QBP_BN_BAB(R, G, T) do { static PerDeviceOnce once_; QBP_SMEM_OPT_IN(once_, (bn_bwd_apply_bifurcate_kernel<R, G, T>), kBabRingBytes); bn_bwd_apply_bifurcate_kernel<R, G, T><<<grid, kScanThreads, kBabRingBytes, st>>>(dy, x, n, (int)C, ga.tw, save_mean, save_min, save_max, gamma, beta, Cn, coef, g_out, qp8, qp16, id8, id16, keys, reinterpret_cast<uint32_t *>(q8), reinterpret_cast<uint32_t *>(hi), reinterpret_cast<uint32_t *>(lo), flip, row_sums_arg, reinterpret_cast<unsigned long long *>(tot16), relu_thr); } while (0)
 #define QBP_BN_BAB2(R, G) do { if (tot16) QBP_BN_BAB(R, G, true); else QBP_BN_BAB(R, G, false); } while (0)
     if (g_out) { if (relu) QBP_BN_BAB2(true, true); else QBP_BN_BAB2(false, true); }
     else       { if (relu) QBP_BN_BAB2(true, false); else QBP_BN_BAB2(false, false); }
