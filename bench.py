@@ -36,11 +36,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
 # (captured at the full batch of 256).  None: not captured.
 # Keyed by (kernel, occurrence within the step), like KERNEL_WORK; dropped when a kernel changes.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {("bn_bwd_apply_bifurcate_kernel", 0): (411.1e6 + 134.3e6) / 51380224}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {("bn_bwd_apply_bifurcate_kernel", 0): (411.1e6 + 134.0e6) / 51380224}
 # Kernels bound by plain instruction issue rather than by HBM: thread instructions per element, from the same
 # captures (smsp__inst_executed.sum x 32 / elements).  Their roofline is the issue rate of the SMs:
 # SMs x 4 schedulers x 1 warp instruction per clock x 32 threads x the maximum SM clock.
-ALU_INSTR_PER_ELEMENT = {("bn_bwd_apply_bifurcate_kernel", 0): 1.006e8 * 32 / 51380224}
+ALU_INSTR_PER_ELEMENT = {("bn_bwd_apply_bifurcate_kernel", 0): 9.761e7 * 32 / 51380224}
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 
 
