@@ -432,3 +432,47 @@ def test_conv_layers_of_other_shapes_stagewise(B, batch, hw, cin, cout, R):
                dy=synth.normal((batch, hw, hw, cout), 92, std=0.1), seed=5, id8=7, id16=7,
                conv=dict(N=batch, H=hw, W=hw, C=cin, K=cout, R=R, S=R, stride=1, pad=pad))
     _check_layer(B, cfg, True, cfg["conv"], _sampler(50 + cin + cout))
+
+
+@pytest.mark.parametrize("kind", ["conv", "linear"])
+def test_backward_with_mixed_gamma_and_beta(B, kind):
+    """The layer's backward with a rectifier and per-channel gamma of both signs, zero and tiny, beta of both signs: the
+    second pass takes the rectifier's mask as a per-channel threshold on the product's output, which must agree with
+    the forward formula for rising, falling and constant channels.  Gradient against the oracle, codes of the GPU's
+    gradient bit for bit."""
+    import torch
+    from paper_1805_11046_b200 import layer
+    if kind == "conv":
+        cfg = dict(x=synth.relu_normal((3, 10, 10, 32), 60), w=synth.kaiming_normal((64, 3, 3, 32), 61),
+                   dy=synth.normal((3, 10, 10, 64), 62, std=0.1))
+        conv = B.conv_desc(3, 10, 10, 32, 64, 3, 3, 1, 1)
+        L = layer.QuantizedLayer(conv=conv, relu=True, seed=4, tensor_id8=3, tensor_id16=3)
+    else:
+        cfg = dict(x=synth.relu_normal((96, 128), 60), w=synth.kaiming_normal((128, 64), 61), dy=synth.normal((96, 64), 62, std=0.1))
+        L = layer.QuantizedLayer(batch=96, in_features=128, out_features=64, relu=True, seed=4, tensor_id8=3, tensor_id16=3)
+    K = 64
+    gamma = synth.normal((K,), 63)
+    gamma[0] = 0.0; gamma[1] = -0.0; gamma[2] = 1e-30; gamma[3] = -1e-30; gamma[4] = -2.5; gamma[5] = 3.0
+    beta = synth.normal((K,), 64) * np.float32(0.5)
+    beta[0] = 0.25; beta[1] = -0.25; beta[6] = 0.0; beta[7] = 100.0; beta[8] = -100.0
+    gd, bd = to_dev(gamma), to_dev(beta)
+    y = L.forward(to_dev(cfg["x"]), to_dev(cfg["w"]), gd, bd)
+    dx, dw, dgamma, dbeta = L.backward(to_dev(cfg["dy"]))
+    torch.cuda.synchronize()
+    assert L.status() == 0
+    z2 = to_host(L.z).reshape(-1, K); dy2 = cfg["dy"].reshape(-1, K)
+    oy, _, _, _ = O.rangebn_fwd(z2, gamma, beta, relu=True)
+    assert rel_err(to_host(y).reshape(-1, K), oy)[0] <= FP32_TOL
+    mean, vmin, vmax = to_host(L.save_mean), to_host(L.save_min), to_host(L.save_max)
+    og, odg, odb = O.rangebn_bwd(dy2, z2, mean, vmin, vmax, gamma, beta, relu=True)
+    g = to_host(L.g)
+    # per channel: a wrong mask in one channel must not hide behind the others
+    got = g.reshape(-1, K)
+    for c in range(K):
+        den = max(float(np.abs(og[:, c]).max()), 1e-30)
+        assert float(np.abs(got[:, c] - og[:, c]).max()) / den <= FP32_TOL or float(np.abs(og[:, c]).max()) < 1e-20, c
+    assert rel_err(to_host(dgamma), odg)[0] <= FP32_TOL and rel_err(to_host(dbeta), odb)[0] <= FP32_TOL
+    g8, g16 = O.bifurcate(g, 4, 3, 3)
+    ohi, olo = O.limb_split(g16.q)
+    assert np.array_equal(to_host(L.g8), g8.q) and np.array_equal(to_host(L.ghi), ohi)
+    assert np.array_equal(to_host(L.glo) ^ np.uint8(0x80), olo)
